@@ -1,0 +1,181 @@
+"""Float64 CPU oracle (test infrastructure, not the product).
+
+ctypes front end of ``laplace_oracle.c``.  Arrays go in and come out as
+C-contiguous float64 numpy arrays.  Nothing here imports or is imported by the
+CUDA package; only tests, the smoke check and the benchmark's CPU-baseline leg
+may use it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "laplace_oracle.c")
+_LIB = os.path.join(_HERE, "liblaplace_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, OpenMP over heads) if it is stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, _SRC, "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Problem(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("H", ctypes.c_int32), ("n", ctypes.c_int32),
+        ("d", ctypes.c_int32), ("m", ctypes.c_int32),
+        ("lambda_", ctypes.c_double),
+        ("ns_iters", ctypes.c_int32),
+        ("ridge_eps", ctypes.c_double),
+        ("ns_alpha", ctypes.c_double),
+        ("map_mode", ctypes.c_int32),
+        ("lm_mode", ctypes.c_int32),
+        ("prefix", ctypes.c_int32), ("gh", ctypes.c_int32), ("gw", ctypes.c_int32),
+        ("mh", ctypes.c_int32), ("mw", ctypes.c_int32),
+    ]
+
+
+@dataclass
+class Problem:
+    """Arguments of the path in the paper's notation (B, heads, n tokens, head dim d, m landmarks)."""
+    B: int
+    H: int
+    n: int
+    d: int
+    m: int
+    lam: float
+    ns_iters: int
+    ridge_eps: float = 1e-6
+    ns_alpha: float = 0.0
+    map_mode: int = 1
+    lm_mode: int = 1
+    prefix: int = 0
+    gh: int = 0
+    gw: int = 0
+    mh: int = 0
+    mw: int = 0
+
+    def c(self) -> _Problem:
+        return _Problem(self.B, self.H, self.n, self.d, self.m, float(self.lam), self.ns_iters,
+                        float(self.ridge_eps), float(self.ns_alpha), self.map_mode, self.lm_mode,
+                        self.prefix, self.gh, self.gw, self.mh, self.mw)
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def _p(a):
+    if a is None:
+        return None
+    assert a.dtype == np.float64 and a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _f64(a):
+    return None if a is None else np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def l1_kernel(A, Bm, lam, want_rowsum=False):
+    """K[b,i,j] = exp(-||A[b,i]-Bm[b,j]||_1 / lam).  A [batch,na,d], Bm [batch,nb,d]."""
+    A, Bm = _f64(A), _f64(Bm)
+    batch, na, d = A.shape
+    nb = Bm.shape[1]
+    K = np.empty((batch, na, nb))
+    rs = np.empty((batch, na)) if want_rowsum else None
+    _load().oracle_l1_kernel(batch, na, nb, d, _p(A), _p(Bm), ctypes.c_double(lam), _p(K), _p(rs))
+    return (K, rs) if want_rowsum else K
+
+
+def l1_kernel_bwd(A, Bm, lam, dK):
+    A, Bm, dK = _f64(A), _f64(Bm), _f64(dK)
+    batch, na, d = A.shape
+    nb = Bm.shape[1]
+    dA, dB = np.empty_like(A), np.empty_like(Bm)
+    _load().oracle_l1_kernel_bwd(batch, na, nb, d, _p(A), _p(Bm), ctypes.c_double(lam), _p(dK), _p(dA), _p(dB))
+    return dA, dB
+
+
+def ns_pinv(W, iters, eps=0.0, alpha=0.0, want_hist=False):
+    """Newton-Schulz T-step iterate of (W + eps I)^-1.  W [batch,m,m].  Returns X, resid, alpha(, X_hist)."""
+    W = _f64(W)
+    batch, m, _ = W.shape
+    X = np.empty_like(W)
+    hist = np.empty((batch, max(iters, 1), m, m)) if want_hist else None
+    resid = np.empty(batch)
+    aout = np.empty(batch)
+    _load().oracle_ns_pinv(batch, m, _p(W), iters, ctypes.c_double(eps), ctypes.c_double(alpha),
+                           _p(X), _p(hist), _p(resid), _p(aout))
+    if want_hist:
+        return X, resid, aout, hist[:, :iters]
+    return X, resid, aout
+
+
+def ns_pinv_bwd(W, iters, eps, alpha, dX):
+    W, dX = _f64(W), _f64(dX)
+    batch, m, _ = W.shape
+    dW = np.empty_like(W)
+    _load().oracle_ns_pinv_bwd(batch, m, _p(W), iters, ctypes.c_double(eps), ctypes.c_double(alpha), _p(dX), _p(dW))
+    return dW
+
+
+def landmarks_pool(p: Problem, K):
+    K = _f64(K)
+    L = np.empty((p.B, p.H, p.m, p.d))
+    cp = p.c()
+    _load().oracle_landmarks_pool(ctypes.byref(cp), _p(K), _p(L))
+    return L
+
+
+def landmarks_pool_bwd(p: Problem, dL):
+    dL = _f64(dL)
+    dK = np.empty((p.B, p.H, p.n, p.d))
+    cp = p.c()
+    _load().oracle_landmarks_pool_bwd(ctypes.byref(cp), _p(dL), _p(dK))
+    return dK
+
+
+def forward(p: Problem, Q, K, V, L=None, whiten=None, want=()):
+    """O [B,H,n,d]; ``want`` names intermediates to return as well (L C R W X M Y Z)."""
+    Q, K, V, L, whiten = _f64(Q), _f64(K), _f64(V), _f64(L), _f64(whiten)
+    BH = p.B * p.H
+    shapes = {"L": (BH, p.m, p.d), "C": (BH, p.n, p.m), "R": (BH, p.m, p.n), "W": (BH, p.m, p.m),
+              "X": (BH, p.m, p.m), "M": (BH, p.m, p.d), "Y": (BH, p.m, p.d), "Z": (BH, p.n, p.m)}
+    extra = {k: (np.empty(shapes[k]) if k in want else None) for k in shapes}
+    O = np.empty((p.B, p.H, p.n, p.d))
+    cp = p.c()
+    _load().oracle_fwd(ctypes.byref(cp), _p(Q), _p(K), _p(V), _p(L), _p(whiten), _p(O),
+                       *[_p(extra[k]) for k in ("L", "C", "R", "W", "X", "M", "Y", "Z")])
+    if want:
+        return O, {k: extra[k] for k in want}
+    return O
+
+
+def backward(p: Problem, Q, K, V, dO, L=None, whiten=None):
+    """Returns dQ, dK, dV, dL (dL is None when the landmarks are pooled from K)."""
+    Q, K, V, L, whiten, dO = _f64(Q), _f64(K), _f64(V), _f64(L), _f64(whiten), _f64(dO)
+    dQ, dK, dV = np.empty_like(Q), np.empty_like(Q), np.empty_like(Q)
+    dL = np.empty((p.B, p.H, p.m, p.d)) if p.lm_mode == 0 else None
+    cp = p.c()
+    _load().oracle_bwd(ctypes.byref(cp), _p(Q), _p(K), _p(V), _p(L), _p(whiten), _p(dO),
+                       _p(dQ), _p(dK), _p(dV), _p(dL))
+    return dQ, dK, dV, dL

@@ -1,0 +1,344 @@
+"""Pins for the float64 oracle: closed forms, brute force, invariants, finite differences.
+
+None of these re-type the oracle's own code path: brute force is written with
+numpy broadcasting, closed forms come from the mathematics (Kac-Murdock-Szego
+inverse, spectral form of the Newton-Schulz polynomial), and gradients are
+checked against central differences of the oracle's *forward*.
+"""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import Problem
+
+GOLD = {}
+with open(os.path.join(os.path.dirname(__file__), "golden", "hand_values.txt")) as fh:
+    for line in fh:
+        if line.startswith("#") or "|" not in line:
+            continue
+        name, val, _ = [t.strip() for t in line.split("|")]
+        GOLD[name] = float(val)
+
+
+def np_l1(A, Bm, lam):
+    """Brute force with broadcasting: exp(-sum_c |a_ic - b_jc| / lam)."""
+    return np.exp(-np.abs(A[:, None, :] - Bm[None, :, :]).sum(-1) / lam)
+
+
+# --------------------------------------------------------------------------- kernel
+def test_l1_hand_values():
+    k = oracle.l1_kernel(np.zeros((1, 1, 4)), np.ones((1, 1, 4)), 4.0)
+    assert k[0, 0, 0] == pytest.approx(GOLD["k_unit_offset"], rel=1e-15)
+    k = oracle.l1_kernel(np.array([[[0.5, -1.0]]]), np.array([[[0.25, 1.0]]]), 2.0)
+    assert k[0, 0, 0] == pytest.approx(GOLD["k_two_dim"], rel=1e-15)
+
+
+def test_l1_bruteforce_and_properties():
+    rng = np.random.default_rng(1)
+    A = rng.standard_normal((3, 17, 5))
+    Bm = rng.standard_normal((3, 9, 5))
+    K, rs = oracle.l1_kernel(A, Bm, 2.5, want_rowsum=True)
+    for b in range(3):
+        np.testing.assert_allclose(K[b], np_l1(A[b], Bm[b], 2.5), rtol=1e-14)
+    np.testing.assert_allclose(rs, K.sum(-1), rtol=1e-14)
+    # product form over coordinates
+    prod = np.prod(np.exp(-np.abs(A[0][:, None, :] - Bm[0][None, :, :]) / 2.5), axis=-1)
+    np.testing.assert_allclose(K[0], prod, rtol=1e-13)
+    # symmetry, unit diagonal, range
+    S = oracle.l1_kernel(A, A, 2.5)
+    np.testing.assert_array_equal(S, S.transpose(0, 2, 1))
+    np.testing.assert_array_equal(np.diagonal(S, axis1=1, axis2=2), 1.0)
+    assert (S > 0).all() and (S <= 1).all()
+    # triangle inequality of the l1 distance: k(x,z) >= k(x,y) k(y,z)
+    KB = oracle.l1_kernel(Bm, Bm, 2.5)
+    lhs = K[0][:, None, :]                       # k(a_i, b_j) for every middle point b_k
+    rhs = K[0][:, :, None] * KB[0][None, :, :]   # k(a_i, b_k) k(b_k, b_j)
+    assert (lhs + 1e-15 >= rhs).all()
+
+
+def test_l1_single_pair_gradient_norm():
+    # App. A: ||grad_x k||_2 = sqrt(d)/lambda * k when no coordinate ties
+    x = np.zeros((1, 1, 4)); y = np.ones((1, 1, 4))
+    dA, dB = oracle.l1_kernel_bwd(x, y, 4.0, np.ones((1, 1, 1)))
+    assert np.linalg.norm(dA) == pytest.approx(GOLD["grad_norm_unit_offset"], rel=1e-15)
+    # x < y in every coordinate: d k / d x_c = -(1/lambda) sign(x-y) k = +k/lambda
+    np.testing.assert_allclose(dA, +GOLD["k_unit_offset"] / 4.0)
+    np.testing.assert_allclose(dB, -GOLD["k_unit_offset"] / 4.0)
+
+
+def test_l1_gradient_tie_is_zero():
+    x = np.array([[[1.0, 2.0]]]); y = np.array([[[1.0, 3.0]]])
+    dA, dB = oracle.l1_kernel_bwd(x, y, 1.0, np.ones((1, 1, 1)))
+    assert dA[0, 0, 0] == 0.0 and dB[0, 0, 0] == 0.0
+    assert dA[0, 0, 1] == pytest.approx(np.exp(-1.0))
+
+
+def test_l1_bwd_finite_differences():
+    rng = np.random.default_rng(2)
+    A = rng.standard_normal((2, 6, 4)); Bm = rng.standard_normal((2, 5, 4))
+    dK = rng.standard_normal((2, 6, 5))
+    dA, dB = oracle.l1_kernel_bwd(A, Bm, 1.7, dK)
+    f = lambda a, b: float((oracle.l1_kernel(a, b, 1.7) * dK).sum())
+    h = 1e-6
+    for arr, grad, which in ((A, dA, 0), (Bm, dB, 1)):
+        for idx in [(0, 0, 0), (1, 3, 2), (0, 4, 3), (1, 2, 1)]:
+            p = arr.copy(); p[idx] += h
+            q = arr.copy(); q[idx] -= h
+            fd = (f(p, Bm) - f(q, Bm)) / (2 * h) if which == 0 else (f(A, p) - f(A, q)) / (2 * h)
+            assert grad[idx] == pytest.approx(fd, rel=1e-7, abs=1e-9)
+
+
+# --------------------------------------------------------------------------- landmark kernel + Newton-Schulz
+def kms(m, rho):
+    idx = np.arange(m)
+    return rho ** np.abs(idx[:, None] - idx[None, :])
+
+
+def test_kms_closed_form_inverse():
+    # d = 1, equally spaced points, lambda = 1/ln 2 -> W_ij = (1/2)^|i-j|
+    pts = np.arange(4, dtype=np.float64).reshape(1, 4, 1)
+    W = oracle.l1_kernel(pts, pts, 1.0 / np.log(2.0))
+    np.testing.assert_allclose(W[0], kms(4, 0.5), rtol=1e-14)
+    X, resid, alpha = oracle.ns_pinv(W, 60, eps=0.0)
+    assert resid[0] < 1e-12
+    assert X[0, 0, 0] == pytest.approx(GOLD["kms_inv_corner"], rel=1e-12)
+    assert X[0, 3, 3] == pytest.approx(GOLD["kms_inv_corner"], rel=1e-12)
+    assert X[0, 1, 1] == pytest.approx(GOLD["kms_inv_inner_diag"], rel=1e-12)
+    assert X[0, 1, 2] == pytest.approx(GOLD["kms_inv_offdiag"], rel=1e-12)
+    assert X[0, 2, 1] == pytest.approx(GOLD["kms_inv_offdiag"], rel=1e-12)
+    assert abs(X[0, 0, 2]) < 1e-12 and abs(X[0, 0, 3]) < 1e-12
+    # general m, rho: tridiagonal closed form
+    m, rho = 9, 0.8
+    Winv = np.zeros((m, m))
+    for i in range(m):
+        Winv[i, i] = (1 + rho * rho) if 0 < i < m - 1 else 1.0
+        if i + 1 < m:
+            Winv[i, i + 1] = Winv[i + 1, i] = -rho
+    Winv /= (1 - rho * rho)
+    X, resid, _ = oracle.ns_pinv(kms(m, rho)[None], 80)
+    np.testing.assert_allclose(X[0], Winv, atol=1e-10)
+
+
+def test_ns_alpha_rule_and_spectral_closed_form():
+    # For symmetric W: I - W X_T = (I - alpha W^2)^(2^T), so in the eigenbasis of W
+    # X_T = U diag((1 - (1 - alpha w_i^2)^(2^T)) / w_i) U^T  -- pins the UNCONVERGED iterate.
+    rng = np.random.default_rng(3)
+    pts = rng.standard_normal((1, 12, 6))
+    W = oracle.l1_kernel(pts, pts, 6.0)[0]
+    eps = 1e-3
+    We = W + eps * np.eye(12)
+    for T in (0, 1, 3, 6):
+        X, resid, alpha = oracle.ns_pinv(W[None], T, eps=eps)
+        a = 1.0 / (np.abs(We).sum(0).max() * np.abs(We).sum(1).max())
+        assert alpha[0] == pytest.approx(a, rel=1e-14)
+        w, U = np.linalg.eigh(We)
+        xs = (1.0 - (1.0 - a * w * w) ** (2 ** T)) / w
+        np.testing.assert_allclose(X[0], (U * xs) @ U.T, rtol=0, atol=1e-12 * np.abs(xs).max())
+        assert resid[0] == pytest.approx(np.linalg.norm(np.eye(12) - We @ X[0]), rel=1e-10)
+
+
+def test_ns_nonsymmetric_matches_definition():
+    # Alg. 2 is stated for a general W (X_0 = alpha W^T): check against a direct numpy loop
+    rng = np.random.default_rng(4)
+    W = np.eye(5) + 0.2 * rng.standard_normal((5, 5))
+    a = 1.0 / (np.abs(W).sum(0).max() * np.abs(W).sum(1).max())
+    X = a * W.T
+    hist = []
+    for _ in range(5):
+        hist.append(X)
+        X = X @ (2 * np.eye(5) - W @ X)
+    Xo, _, alpha, Xh = oracle.ns_pinv(W[None], 5, want_hist=True)
+    np.testing.assert_allclose(Xo[0], X, rtol=1e-13)
+    np.testing.assert_allclose(Xh[0], np.stack(hist), rtol=1e-13)
+    Xc, resid, _ = oracle.ns_pinv(W[None], 50)
+    np.testing.assert_allclose(Xc[0], np.linalg.inv(W), atol=1e-11)
+
+
+def test_ns_converges_to_inverse_and_residual_monotone():
+    rng = np.random.default_rng(5)
+    pts = rng.standard_normal((2, 16, 8))
+    W = oracle.l1_kernel(pts, pts, 8.0)
+    # symmetric, unit diagonal, positive definite
+    np.testing.assert_array_equal(W, W.transpose(0, 2, 1))
+    for b in range(2):
+        np.linalg.cholesky(W[b])
+    prev = None
+    for T in range(0, 45, 3):
+        X, resid, _ = oracle.ns_pinv(W, T, eps=1e-9)
+        if prev is not None:
+            assert (resid <= prev * (1 + 1e-9) + 1e-13).all()
+        prev = resid
+    X, resid, _ = oracle.ns_pinv(W, 45, eps=0.0)
+    for b in range(2):
+        assert np.abs(X[b] @ W[b] - np.eye(16)).max() < 1e-10
+
+
+def test_ns_degenerate_cases():
+    X, resid, alpha = oracle.ns_pinv(np.eye(7)[None], 0)
+    np.testing.assert_allclose(X[0], np.eye(7), rtol=1e-15)          # alpha = 1, X_0 = I
+    X, resid, alpha = oracle.ns_pinv(np.array([[[4.0]]]), 0)          # m = 1: alpha = 1/16, X_0 = 1/4
+    assert X[0, 0, 0] == pytest.approx(0.25)
+    X, _, _ = oracle.ns_pinv(np.array([[[4.0]]]), 3, eps=1.0)         # exact at X_0 already: 1/(W+eps)
+    assert X[0, 0, 0] == pytest.approx(0.2)
+
+
+def test_ns_literal_alpha_diverges():
+    # alpha = 2/||W||_2 as printed in Alg. 2 violates ||I - alpha W W^T|| < 1 for unit-diagonal W
+    rng = np.random.default_rng(6)
+    pts = rng.standard_normal((1, 16, 8))
+    W = oracle.l1_kernel(pts, pts, 8.0)
+    lit = 2.0 / np.linalg.norm(W[0], 2)
+    with np.errstate(all="ignore"):
+        X, resid, alpha = oracle.ns_pinv(W, 8, alpha=lit)
+    assert alpha[0] == lit
+    assert not np.isfinite(resid[0]) or resid[0] > 1e6
+
+
+@pytest.mark.parametrize("kappa", [2.0, 10.0, 50.0])
+def test_ns_condition_number_sweep(kappa):
+    # Fig. 6 setting: SPD matrices of prescribed condition number, error ||X_k - W^-1||_F / ||W^-1||_F
+    rng = np.random.default_rng(7)
+    Qm, _ = np.linalg.qr(rng.standard_normal((24, 24)))
+    w = np.geomspace(1.0, 1.0 / kappa, 24)
+    W = (Qm * w) @ Qm.T
+    W = 0.5 * (W + W.T)
+    Winv = np.linalg.inv(W)
+    errs = []
+    for T in range(0, 30, 2):
+        X, _, _ = oracle.ns_pinv(W[None], T)
+        errs.append(np.linalg.norm(X[0] - Winv) / np.linalg.norm(Winv))
+    assert all(e2 <= e1 * (1 + 1e-9) + 1e-14 for e1, e2 in zip(errs, errs[1:]))
+    assert errs[-1] < 1e-10
+
+
+def test_ns_bwd_finite_differences():
+    rng = np.random.default_rng(8)
+    pts = rng.standard_normal((1, 5, 3))
+    W = oracle.l1_kernel(pts, pts, 3.0) + 0.01 * rng.standard_normal((1, 5, 5))  # general (non-symmetric)
+    dX = rng.standard_normal((1, 5, 5))
+    for alpha in (0.0, 0.03):
+        dW = oracle.ns_pinv_bwd(W, 4, 1e-3, alpha, dX)
+        f = lambda w: float((oracle.ns_pinv(w, 4, eps=1e-3, alpha=alpha)[0] * dX).sum())
+        h = 1e-6
+        for i in range(5):
+            for j in range(5):
+                p = W.copy(); p[0, i, j] += h
+                q = W.copy(); q[0, i, j] -= h
+                assert dW[0, i, j] == pytest.approx((f(p) - f(q)) / (2 * h), rel=2e-6, abs=1e-8)
+
+
+# --------------------------------------------------------------------------- pooling
+def test_pool_divisible_and_adjoint():
+    p = Problem(B=1, H=2, n=1 + 6 * 4, d=3, m=6, lam=3.0, ns_iters=2, prefix=1, gh=6, gw=4, mh=3, mw=2)
+    rng = np.random.default_rng(9)
+    K = rng.standard_normal((1, 2, p.n, 3))
+    L = oracle.landmarks_pool(p, K)
+    grid = K[:, :, 1:].reshape(1, 2, 6, 4, 3)
+    hand = grid.reshape(1, 2, 3, 2, 2, 2, 3).mean(axis=(3, 5)).reshape(1, 2, 6, 3)   # 2x2 / stride-2 means
+    np.testing.assert_allclose(L, hand, rtol=1e-14)
+    U = rng.standard_normal(L.shape)
+    dK = oracle.landmarks_pool_bwd(p, U)
+    assert float((L * U).sum()) == pytest.approx(float((K * dK).sum()), rel=1e-12)
+    assert np.abs(dK[:, :, 0]).max() == 0.0          # prefix token is never pooled
+
+
+def test_pool_adaptive_bins_overlap_and_identity():
+    # 14 -> 4 bins: floor(a*14/4) .. ceil((a+1)*14/4): [0,4) [3,7) [7,11) [10,14)
+    p = Problem(B=1, H=1, n=14, d=1, m=4, lam=1.0, ns_iters=0, gh=1, gw=14, mh=1, mw=4)
+    K = np.arange(14, dtype=np.float64).reshape(1, 1, 14, 1)
+    L = oracle.landmarks_pool(p, K)[0, 0, :, 0]
+    np.testing.assert_allclose(L, [1.5, 4.5, 8.5, 11.5])
+    # each row of the pooling matrix sums to one: pooling a constant gives the constant
+    L1 = oracle.landmarks_pool(p, np.ones((1, 1, 14, 1)))
+    np.testing.assert_allclose(L1, 1.0)
+    # bins == grid: landmarks are the keys themselves
+    p2 = Problem(B=1, H=1, n=12, d=2, m=12, lam=1.0, ns_iters=0, gh=3, gw=4, mh=3, mw=4)
+    K2 = np.random.default_rng(10).standard_normal((1, 1, 12, 2))
+    np.testing.assert_array_equal(oracle.landmarks_pool(p2, K2), K2)
+
+
+# --------------------------------------------------------------------------- the whole chain
+def exact_attention(Q, K, V, lam, s=None, map_mode=1):
+    """Eq. 4 + Eq. 7 without any approximation: Z_full V with Z_full built from G = k(Q, K)."""
+    G = np_l1(Q, K, lam)
+    n = K.shape[0]
+    if map_mode == 0:
+        return G @ V
+    s = np.ones(n) if s is None else s
+    Z = (G - G.mean(1, keepdims=True)) * s[None, :] + 1.0 / n
+    return Z @ V
+
+
+@pytest.mark.parametrize("map_mode", [0, 1])
+def test_m_equals_n_reproduces_exact_attention(map_mode):
+    rng = np.random.default_rng(11)
+    n, d = 12, 4
+    p = Problem(B=1, H=2, n=n, d=d, m=n, lam=float(d), ns_iters=60, ridge_eps=0.0, map_mode=map_mode,
+                lm_mode=1, gh=3, gw=4, mh=3, mw=4)
+    Q, K, V = (rng.standard_normal((1, 2, n, d)) for _ in range(3))
+    s = rng.uniform(0.5, 2.0, (2, n))
+    O = oracle.forward(p, Q, K, V, whiten=s)
+    for h in range(2):
+        ref = exact_attention(Q[0, h], K[0, h], V[0, h], float(d), s[h], map_mode)
+        np.testing.assert_allclose(O[0, h], ref, atol=1e-9)
+
+
+def test_intermediates_and_folded_form():
+    rng = np.random.default_rng(12)
+    n, d, m = 20, 4, 5
+    p = Problem(B=2, H=2, n=n, d=d, m=m, lam=float(d), ns_iters=3, lm_mode=1, gh=4, gw=5, mh=1, mw=5)
+    Q, K, V = (rng.standard_normal((2, 2, n, d)) for _ in range(3))
+    s = rng.uniform(0.5, 2.0, (2, m))
+    O, x = oracle.forward(p, Q, K, V, whiten=s, want=("L", "C", "R", "W", "X", "M", "Y", "Z"))
+    for bh in range(4):
+        q, k, v = Q.reshape(4, n, d)[bh], K.reshape(4, n, d)[bh], V.reshape(4, n, d)[bh]
+        L = np.stack([k.reshape(4, 5, d)[:, b].mean(0) for b in range(5)])   # 4x5 grid -> 1x5 bins = column means
+        np.testing.assert_allclose(x["L"][bh], L, rtol=1e-14)
+        np.testing.assert_allclose(x["C"][bh], np_l1(q, L, d), rtol=1e-13)
+        np.testing.assert_allclose(x["R"][bh], np_l1(L, k, d), rtol=1e-13)
+        np.testing.assert_allclose(x["W"][bh], np_l1(L, L, d), rtol=1e-13)
+        sh = s[bh % 2]
+        # rows of Z sum to one when s = 1 (checked below); with s general the centred part is scaled
+        Z = (x["C"][bh] - x["C"][bh].mean(1, keepdims=True)) * sh + 1.0 / m
+        np.testing.assert_allclose(x["Z"][bh], Z, rtol=1e-13)
+        Y = x["X"][bh] @ (x["R"][bh] @ v)
+        np.testing.assert_allclose(x["Y"][bh], Y, rtol=1e-12)
+        # folded form: O = C Ytilde + 1 ybar^T
+        Yt = sh[:, None] * Y - (sh[:, None] * Y).mean(0, keepdims=True)
+        ybar = Y.mean(0)
+        np.testing.assert_allclose(O.reshape(4, n, d)[bh], x["C"][bh] @ Yt + ybar, rtol=1e-10, atol=1e-12)
+    O1, x1 = oracle.forward(p, Q, K, V, whiten=None, want=("Z",))
+    np.testing.assert_allclose(x1["Z"].sum(-1), GOLD["z_row_sum"], rtol=1e-13)
+
+
+@pytest.mark.parametrize("lm_mode,map_mode,use_s", [(1, 1, True), (1, 0, False), (0, 1, True), (0, 1, False)])
+def test_full_backward_finite_differences(lm_mode, map_mode, use_s):
+    rng = np.random.default_rng(13 + lm_mode + 2 * map_mode)
+    n, d, m, T = 24, 6, 6, 4
+    p = Problem(B=1, H=2, n=n, d=d, m=m, lam=float(d), ns_iters=T, ridge_eps=1e-6, map_mode=map_mode,
+                lm_mode=lm_mode, gh=4, gw=6, mh=2, mw=3)
+    Q, K, V, dO = (rng.standard_normal((1, 2, n, d)) for _ in range(4))
+    L = rng.standard_normal((1, 2, m, d)) if lm_mode == 0 else None
+    s = rng.uniform(0.5, 2.0, (2, m)) if use_s else None
+    dQ, dK, dV, dL = oracle.backward(p, Q, K, V, dO, L=L, whiten=s)
+    loss = lambda q, k, v, l: float((oracle.forward(p, q, k, v, L=l, whiten=s) * dO).sum())
+    h = 1e-6
+    probes = [(0, 0, 0, 0), (0, 1, 7, 3), (0, 0, 23, 5), (0, 1, 11, 2), (0, 0, 5, 1)]
+    for name, arr, grad in (("Q", Q, dQ), ("K", K, dK), ("V", V, dV)):
+        for idx in probes:
+            a = {"Q": Q, "K": K, "V": V}
+            plus = dict(a); minus = dict(a)
+            plus[name] = arr.copy(); plus[name][idx] += h
+            minus[name] = arr.copy(); minus[name][idx] -= h
+            fd = (loss(plus["Q"], plus["K"], plus["V"], L) - loss(minus["Q"], minus["K"], minus["V"], L)) / (2 * h)
+            assert grad[idx] == pytest.approx(fd, rel=5e-6, abs=1e-8), (name, idx)
+    if lm_mode == 0:
+        for idx in [(0, 0, 0, 0), (0, 1, 5, 5), (0, 0, 3, 2)]:
+            lp = L.copy(); lp[idx] += h
+            lm_ = L.copy(); lm_[idx] -= h
+            fd = (loss(Q, K, V, lp) - loss(Q, K, V, lm_)) / (2 * h)
+            assert dL[idx] == pytest.approx(fd, rel=5e-6, abs=1e-8)
+    else:
+        assert dL is None
