@@ -1,0 +1,151 @@
+/*
+ * laplace_nystrom.h -- C ABI of the B200 (sm_100a) library for Nystrom-approximated
+ * Laplacian-kernel attention, forward and backward (LaplacianFormer, arXiv 2604.20368).
+ *
+ * Per (batch, head), with Q,K,V in R^{n x d}, m landmarks L in R^{m x d}, decay lambda,
+ * T Newton-Schulz steps, ridge eps and a diagonal whitening scale s in R^m:
+ *
+ *   k(x,y) = exp(-||x - y||_1 / lambda)              Laplacian kernel (Sec. 1)
+ *   L  = average pooling of K over the token grid    landmark selection (Sec. 4.2)
+ *   C  = k(Q,L) [n x m]                               Eq. 8
+ *   W  = k(L,L) + eps I [m x m]                       Eq. 9 and the ridge of Alg. 2
+ *   R  = k(L,K) [m x n]                               the C^T factor of Alg. 1
+ *   X_0 = alpha W^T, X_{k+1} = X_k (2I - W X_k)       Alg. 2, X = X_T, alpha = 1/(||W||_1 ||W||_inf)
+ *   M  = R V,  Y = X M
+ *   Z_il = s_l (C_il - mean_l' C_il') + 1/m           Prop. 3 / Eq. 11 with the diagonal whitening of Eq. 6
+ *   O  = Z Y                                          Eq. 7 with the kernel matrix in Nystrom form
+ *
+ * Conventions common to every entry point
+ *   - Every pointer is a DEVICE pointer unless it is the ln_problem itself (host).
+ *   - The caller owns every buffer.  The library allocates nothing, keeps no state between
+ *     calls, never synchronises the device: it validates arguments on the host, enqueues
+ *     kernels on `stream` (a cudaStream_t passed as void*; NULL = the default stream) and
+ *     returns.  LN_OK means "enqueued".
+ *   - Tensors are contiguous, row-major, 16-byte aligned.  Outputs are fully overwritten.
+ *     Inputs are never modified and must not alias outputs.
+ *   - Storage type of the [.,.,.,d] tensors is `dtype` (LN_F32 or LN_BF16); all arithmetic and
+ *     every on-device intermediate is fp32.
+ *   - Errors: LN_ERR_ARG (NULL required pointer, non-positive size, m > n, lambda <= 0 or not
+ *     finite, T < 0, eps < 0, grid inconsistent with n or m, misaligned pointer),
+ *     LN_ERR_UNSUPPORTED (d not in {32, 64, 128} or m > 256 for the attention entry points),
+ *     LN_ERR_WORKSPACE (ws_bytes too small), LN_ERR_CUDA (a launch failed).  Nothing is
+ *     enqueued when an argument error is returned.
+ */
+#ifndef LAPLACE_NYSTROM_H_
+#define LAPLACE_NYSTROM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { LN_OK = 0, LN_ERR_ARG = -1, LN_ERR_UNSUPPORTED = -2, LN_ERR_WORKSPACE = -3, LN_ERR_CUDA = -4 } ln_status;
+typedef enum { LN_F32 = 0, LN_BF16 = 1 } ln_dtype;
+
+/* The problem statement of Alg. 1 / Alg. 2 in the paper's notation. */
+typedef struct ln_problem {
+  int32_t B, H, n, d, m;  /* Q,K,V,O,dO,dQ,dK,dV: [B,H,n,d];  L,dL: [B,H,m,d]                             */
+  float lambda;           /* decay of the Laplacian kernel, > 0                                           */
+  int32_t ns_iters;       /* T >= 0 Newton-Schulz steps (Alg. 2)                                          */
+  float ridge_eps;        /* eps >= 0 added to the diagonal of k(L,L) (Alg. 2)                            */
+  float ns_alpha;         /* <= 0: alpha = 1/(||W||_1 ||W||_inf);  > 0: used as given, not differentiated */
+  int32_t dtype;          /* ln_dtype of the [.,.,.,d] tensors                                            */
+  int32_t map_mode;       /* 0: O = C X R V;  1: injective map of Prop. 3 applied to the rows of C        */
+  const float* whiten;    /* device [H,m] fp32 whitening scale s (Eq. 6), or NULL = ones; a constant      */
+  int32_t lm_mode;        /* 0: landmarks L given by the caller;  1: L = adaptive average pooling of K    */
+  int32_t prefix, gh, gw, mh, mw; /* lm_mode 1: n = prefix + gh*gw, m = mh*mw.  Bin (a,b) averages grid  */
+                          /* rows floor(a*gh/mh) .. ceil((a+1)*gh/mh)-1 and columns likewise; the first   */
+                          /* `prefix` tokens (class tokens) are ordinary queries/keys but are not pooled. */
+} ln_problem;
+
+const char* ln_status_string(int status);
+
+/*
+ * Sizes of the two caller-provided buffers of the attention entry points, in bytes.
+ *   saved: context handed from laplace_nystrom_fwd to laplace_nystrom_bwd (landmarks, the kernel
+ *          blocks C and R, W, the Newton-Schulz iterates X_0..X_T, M, the folded Y).  Contents are
+ *          defined only between a fwd and the matching bwd.
+ *   ws:    scratch whose contents are undefined between calls.  `with_saved` = 1 when a saved buffer
+ *          will be passed (training), 0 for inference, where the context lives in ws as well.
+ * Both return 0 for an invalid problem.
+ */
+size_t laplace_nystrom_saved_bytes(const ln_problem* p);
+size_t laplace_nystrom_workspace_bytes(const ln_problem* p, int32_t with_saved);
+
+/*
+ * Forward of the whole path (Alg. 1 + Alg. 2 + Prop. 3).
+ *   Q,K,V  [B,H,n,d] dtype;  L [B,H,m,d] dtype, required iff lm_mode == 0 (else NULL);
+ *   O      [B,H,n,d] dtype, overwritten;
+ *   saved  NULL for inference, else laplace_nystrom_saved_bytes(p) bytes;
+ *   ws     laplace_nystrom_workspace_bytes(p, saved != NULL) bytes;
+ *   dev_status NULL or int32 [B*H]: per head, bit0 = X_T is not finite (written by the device).
+ */
+int laplace_nystrom_fwd(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L,
+                        void* O, void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * Backward of the whole path: the exact adjoint of what laplace_nystrom_fwd computes, including
+ * the T unrolled Newton-Schulz steps and alpha's dependence on W (App. A gives the kernel
+ * gradient -(1/lambda) sign(x - y) k, with sign(0) = 0).
+ *   dO [B,H,n,d] dtype;  saved: the buffer the matching fwd filled;
+ *   dQ,dK,dV [B,H,n,d] dtype, overwritten;
+ *   dL [B,H,m,d] dtype: required when lm_mode == 0; must be NULL when lm_mode == 1 (the
+ *   landmark gradient is folded into dK through the pooling adjoint).
+ *   ws: laplace_nystrom_workspace_bytes(p, 1) bytes.
+ */
+int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L,
+                        const void* dO, const void* saved, void* dQ, void* dK, void* dV, void* dL,
+                        void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * Newton-Schulz iterate of (W + eps I)^-1 (Alg. 2), batched over `batch` independent m x m
+ * fp32 matrices.  X [batch,m,m] receives X_T.  X_hist is NULL or [batch,iters+1,m,m] and
+ * receives X_0 .. X_T.  resid is NULL or [batch] and receives ||I - (W + eps I) X_T||_F.
+ * alpha <= 0 selects 1/(||W||_1 ||W||_inf).  ws: ns_pinv_workspace_bytes(batch, m, iters).
+ */
+size_t ns_pinv_workspace_bytes(int32_t batch, int32_t m, int32_t iters);
+int ns_pinv(int32_t batch, int32_t m, const float* W, int32_t iters, float ridge_eps, float alpha,
+            float* X, float* X_hist, float* resid, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Adjoint of ns_pinv: given dX = dLoss/dX_T returns dW = dLoss/dW [batch,m,m] (W before the ridge).
+ * X_hist: the [batch,iters+1,m,m] history a previous ns_pinv wrote, or NULL to recompute it.
+ * With alpha <= 0 the dependence of alpha on W is differentiated (arg-max ties -> lowest index).
+ * ws: ns_pinv_workspace_bytes(batch, m, iters).
+ */
+int ns_pinv_bwd(int32_t batch, int32_t m, const float* W, int32_t iters, float ridge_eps, float alpha,
+                const float* X_hist, const float* dX, float* dW, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Laplacian kernel block (Sec. 1, Eq. 8): Kout[b,i,j] = exp(-||A[b,i,:] - Bm[b,j,:]||_1 / lambda).
+ * A [batch,na,d], Bm [batch,nb,d] of `dtype`; Kout [batch,na,nb] fp32; rowsum NULL or [batch,na]
+ * fp32 = sum_j Kout[b,i,j].  Any d >= 1.
+ */
+int l1_kernel(int32_t batch, int32_t na, int32_t nb, int32_t d, const void* A, const void* Bm, int32_t dtype,
+              float lambda, float* Kout, float* rowsum, void* stream);
+
+/*
+ * Adjoint of l1_kernel (App. A): with g = dKmat * Kmat / lambda,
+ *   dA[b,i,:] = -sum_j g_ij sign(A_i - B_j),  dB[b,j,:] = +sum_i g_ij sign(A_i - B_j),  sign(0) = 0.
+ * Kmat: the block a previous l1_kernel wrote, or NULL to recompute it.  dA, dB have `dtype` and
+ * are overwritten.  ws: l1_kernel_bwd_workspace_bytes(batch, na, nb, d) bytes of scratch.
+ */
+size_t l1_kernel_bwd_workspace_bytes(int32_t batch, int32_t na, int32_t nb, int32_t d);
+int l1_kernel_bwd(int32_t batch, int32_t na, int32_t nb, int32_t d, const void* A, const void* Bm, int32_t dtype,
+                  float lambda, const float* Kmat, const float* dKmat, void* dA, void* dB,
+                  void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Landmark selection by average pooling of the keys over the token grid (Sec. 4.2), lm_mode 1
+ * geometry of `p`.  K [B,H,n,d] dtype -> L [B,H,m,d] fp32.  The backward overwrites dK [B,H,n,d]
+ * (dtype) with pool^T(dL), dL [B,H,m,d] fp32.
+ */
+int landmarks_pool(const ln_problem* p, const void* K, float* L, void* stream);
+int landmarks_pool_bwd(const ln_problem* p, const float* dL, void* dK, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAPLACE_NYSTROM_H_ */

@@ -1,0 +1,259 @@
+"""Thin ctypes binding of ``include/laplace_nystrom.h``.
+
+Argument marshalling only: every step of the path runs in the CUDA library.  torch is used
+for device memory and streams.  There is no CPU fallback: if the shared library cannot be
+loaded, or a tensor is not on a CUDA device, the call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass, field
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+LN_F32, LN_BF16 = 0, 1
+_STATUS = {0: "ok", -1: "invalid argument", -2: "outside the supported envelope",
+           -3: "workspace too small", -4: "CUDA launch failed"}
+
+EXPORTS = [
+    "ln_status_string", "laplace_nystrom_saved_bytes", "laplace_nystrom_workspace_bytes",
+    "laplace_nystrom_fwd", "laplace_nystrom_bwd", "ns_pinv_workspace_bytes", "ns_pinv", "ns_pinv_bwd",
+    "l1_kernel", "l1_kernel_bwd_workspace_bytes", "l1_kernel_bwd", "landmarks_pool", "landmarks_pool_bwd",
+]
+
+
+class LnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        super().__init__(f"{where}: status {status} ({_STATUS.get(status, 'unknown')})")
+        self.status = status
+
+
+class _CProblem(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("H", ctypes.c_int32), ("n", ctypes.c_int32), ("d", ctypes.c_int32),
+        ("m", ctypes.c_int32), ("lambda_", ctypes.c_float), ("ns_iters", ctypes.c_int32),
+        ("ridge_eps", ctypes.c_float), ("ns_alpha", ctypes.c_float), ("dtype", ctypes.c_int32),
+        ("map_mode", ctypes.c_int32), ("whiten", ctypes.c_void_p), ("lm_mode", ctypes.c_int32),
+        ("prefix", ctypes.c_int32), ("gh", ctypes.c_int32), ("gw", ctypes.c_int32),
+        ("mh", ctypes.c_int32), ("mw", ctypes.c_int32),
+    ]
+
+
+@dataclass
+class Problem:
+    """The problem statement in the paper's notation (B, heads, n tokens, head dim d, m landmarks,
+    decay lambda, Newton-Schulz iteration count)."""
+    B: int
+    H: int
+    n: int
+    d: int
+    m: int
+    lam: float
+    ns_iters: int
+    ridge_eps: float = 1e-6
+    ns_alpha: float = 0.0
+    dtype: int = LN_BF16
+    map_mode: int = 1
+    whiten: Optional[torch.Tensor] = field(default=None, repr=False)   # device fp32 [H, m] or None
+    lm_mode: int = 1
+    prefix: int = 0
+    gh: int = 0
+    gw: int = 0
+    mh: int = 0
+    mw: int = 0
+
+    def c(self) -> _CProblem:
+        w = None
+        if self.whiten is not None:
+            assert self.whiten.is_cuda and self.whiten.dtype == torch.float32 and self.whiten.is_contiguous()
+            assert tuple(self.whiten.shape) == (self.H, self.m)
+            w = self.whiten.data_ptr()
+        return _CProblem(self.B, self.H, self.n, self.d, self.m, float(self.lam), self.ns_iters,
+                         float(self.ridge_eps), float(self.ns_alpha), self.dtype, self.map_mode, w,
+                         self.lm_mode, self.prefix, self.gh, self.gw, self.mh, self.mw)
+
+    @property
+    def torch_dtype(self):
+        return torch.float32 if self.dtype == LN_F32 else torch.bfloat16
+
+
+_lib = None
+
+
+def lib():
+    """Load (building first if the sources are newer) the CUDA shared library; raises if impossible."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        try:
+            path = _build.build()
+        except Exception as e:   # no nvcc on this machine: use the library that travelled with the tree
+            if not os.path.exists(path):
+                raise RuntimeError(f"CUDA library {path} is missing and could not be built: {e}") from e
+        L = ctypes.CDLL(path)
+        vp, i32, f32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_float, ctypes.c_size_t
+        pp = ctypes.POINTER(_CProblem)
+        L.ln_status_string.restype = ctypes.c_char_p
+        L.ln_status_string.argtypes = [ctypes.c_int]
+        L.laplace_nystrom_saved_bytes.restype = sz
+        L.laplace_nystrom_saved_bytes.argtypes = [pp]
+        L.laplace_nystrom_workspace_bytes.restype = sz
+        L.laplace_nystrom_workspace_bytes.argtypes = [pp, i32]
+        L.laplace_nystrom_fwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.laplace_nystrom_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.ns_pinv_workspace_bytes.restype = sz
+        L.ns_pinv_workspace_bytes.argtypes = [i32, i32, i32]
+        L.ns_pinv.argtypes = [i32, i32, vp, i32, f32, f32, vp, vp, vp, vp, sz, vp]
+        L.ns_pinv_bwd.argtypes = [i32, i32, vp, i32, f32, f32, vp, vp, vp, vp, sz, vp]
+        L.l1_kernel.argtypes = [i32, i32, i32, i32, vp, vp, i32, f32, vp, vp, vp]
+        L.l1_kernel_bwd_workspace_bytes.restype = sz
+        L.l1_kernel_bwd_workspace_bytes.argtypes = [i32, i32, i32, i32]
+        L.l1_kernel_bwd.argtypes = [i32, i32, i32, i32, vp, vp, i32, f32, vp, vp, vp, vp, vp, sz, vp]
+        L.landmarks_pool.argtypes = [pp, vp, vp, vp]
+        L.landmarks_pool_bwd.argtypes = [pp, vp, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("tensor must live on a CUDA device (there is no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return t.data_ptr()
+
+
+def _stream(stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise LnError(status, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return LN_F32
+    if t.dtype == torch.bfloat16:
+        return LN_BF16
+    raise ValueError(f"unsupported storage dtype {t.dtype}")
+
+
+def _bytes(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 16), dtype=torch.uint8, device=device)
+
+
+# ------------------------------------------------------------------------------------------ sizes
+def laplace_nystrom_saved_bytes(p: Problem) -> int:
+    cp = p.c()
+    return int(lib().laplace_nystrom_saved_bytes(ctypes.byref(cp)))
+
+
+def laplace_nystrom_workspace_bytes(p: Problem, with_saved: bool) -> int:
+    cp = p.c()
+    return int(lib().laplace_nystrom_workspace_bytes(ctypes.byref(cp), int(with_saved)))
+
+
+# ------------------------------------------------------------------------------------------ attention
+def laplace_nystrom_fwd(p: Problem, Q, K, V, L=None, O=None, saved=None, ws=None, dev_status=None, stream=None):
+    """O = Z Y (Alg. 1 + Alg. 2 + Prop. 3).  ``saved``: a uint8 tensor of laplace_nystrom_saved_bytes(p)
+    for training, or None for inference.  Returns O."""
+    if O is None:
+        O = torch.empty_like(Q)
+    if ws is None:
+        ws = _bytes(laplace_nystrom_workspace_bytes(p, saved is not None), Q.device)
+    cp = p.c()
+    st = lib().laplace_nystrom_fwd(ctypes.byref(cp), _ptr(Q), _ptr(K), _ptr(V), _ptr(L), _ptr(O), _ptr(saved),
+                                   _ptr(ws), ws.numel(), _ptr(dev_status), _stream(stream))
+    _check(st, "laplace_nystrom_fwd")
+    return O
+
+
+def laplace_nystrom_bwd(p: Problem, Q, K, V, dO, saved, L=None, dQ=None, dK=None, dV=None, dL=None, ws=None,
+                        stream=None):
+    """Exact adjoint of laplace_nystrom_fwd.  Returns dQ, dK, dV, dL (dL is None when lm_mode == 1)."""
+    dQ = torch.empty_like(Q) if dQ is None else dQ
+    dK = torch.empty_like(K) if dK is None else dK
+    dV = torch.empty_like(V) if dV is None else dV
+    if p.lm_mode == 0 and dL is None:
+        dL = torch.empty_like(L)
+    if ws is None:
+        ws = _bytes(laplace_nystrom_workspace_bytes(p, True), Q.device)
+    cp = p.c()
+    st = lib().laplace_nystrom_bwd(ctypes.byref(cp), _ptr(Q), _ptr(K), _ptr(V), _ptr(L), _ptr(dO), _ptr(saved),
+                                   _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dL), _ptr(ws), ws.numel(), None,
+                                   _stream(stream))
+    _check(st, "laplace_nystrom_bwd")
+    return dQ, dK, dV, dL
+
+
+# ------------------------------------------------------------------------------------------ Newton-Schulz
+def ns_pinv(W, iters: int, ridge_eps: float = 0.0, alpha: float = 0.0, want_hist=False, want_resid=False,
+            stream=None):
+    """T-step Newton-Schulz iterate of (W + eps I)^-1 (Alg. 2).  W: device fp32 [batch, m, m]."""
+    batch, m, _ = W.shape
+    X = torch.empty_like(W)
+    hist = torch.empty((batch, iters + 1, m, m), dtype=torch.float32, device=W.device) if want_hist else None
+    resid = torch.empty((batch,), dtype=torch.float32, device=W.device) if want_resid else None
+    ws = _bytes(lib().ns_pinv_workspace_bytes(batch, m, iters), W.device)
+    st = lib().ns_pinv(batch, m, _ptr(W), iters, ridge_eps, alpha, _ptr(X), _ptr(hist), _ptr(resid), _ptr(ws),
+                       ws.numel(), _stream(stream))
+    _check(st, "ns_pinv")
+    return X, hist, resid
+
+
+def ns_pinv_bwd(W, iters: int, ridge_eps: float, alpha: float, dX, X_hist=None, stream=None):
+    batch, m, _ = W.shape
+    dW = torch.empty_like(W)
+    ws = _bytes(lib().ns_pinv_workspace_bytes(batch, m, iters), W.device)
+    st = lib().ns_pinv_bwd(batch, m, _ptr(W), iters, ridge_eps, alpha, _ptr(X_hist), _ptr(dX), _ptr(dW), _ptr(ws),
+                           ws.numel(), _stream(stream))
+    _check(st, "ns_pinv_bwd")
+    return dW
+
+
+# ------------------------------------------------------------------------------------------ kernel block
+def l1_kernel(A, Bm, lam: float, want_rowsum=False, stream=None):
+    """K[b,i,j] = exp(-||A[b,i]-Bm[b,j]||_1 / lam) (Sec. 1, Eq. 8).  A [batch,na,d], Bm [batch,nb,d]."""
+    batch, na, d = A.shape
+    nb = Bm.shape[1]
+    Kout = torch.empty((batch, na, nb), dtype=torch.float32, device=A.device)
+    rs = torch.empty((batch, na), dtype=torch.float32, device=A.device) if want_rowsum else None
+    st = lib().l1_kernel(batch, na, nb, d, _ptr(A), _ptr(Bm), _dtype_code(A), lam, _ptr(Kout), _ptr(rs),
+                         _stream(stream))
+    _check(st, "l1_kernel")
+    return (Kout, rs) if want_rowsum else Kout
+
+
+def l1_kernel_bwd(A, Bm, lam: float, dK, Kmat=None, stream=None):
+    batch, na, d = A.shape
+    nb = Bm.shape[1]
+    dA, dB = torch.empty_like(A), torch.empty_like(Bm)
+    ws = _bytes(lib().l1_kernel_bwd_workspace_bytes(batch, na, nb, d), A.device)
+    st = lib().l1_kernel_bwd(batch, na, nb, d, _ptr(A), _ptr(Bm), _dtype_code(A), lam, _ptr(Kmat), _ptr(dK),
+                             _ptr(dA), _ptr(dB), _ptr(ws), ws.numel(), _stream(stream))
+    _check(st, "l1_kernel_bwd")
+    return dA, dB
+
+
+# ------------------------------------------------------------------------------------------ landmarks
+def landmarks_pool(p: Problem, K, stream=None):
+    L = torch.empty((p.B, p.H, p.m, p.d), dtype=torch.float32, device=K.device)
+    cp = p.c()
+    _check(lib().landmarks_pool(ctypes.byref(cp), _ptr(K), _ptr(L), _stream(stream)), "landmarks_pool")
+    return L
+
+
+def landmarks_pool_bwd(p: Problem, dL, stream=None):
+    dK = torch.empty((p.B, p.H, p.n, p.d), dtype=p.torch_dtype, device=dL.device)
+    cp = p.c()
+    _check(lib().landmarks_pool_bwd(ctypes.byref(cp), _ptr(dL), _ptr(dK), _stream(stream)), "landmarks_pool_bwd")
+    return dK

@@ -1,0 +1,430 @@
+// C ABI of the Laplacian-Nystrom library: host-side validation, buffer layout and launches.
+#include <math.h>
+#include <stdint.h>
+
+#include "../../include/laplace_nystrom.h"
+#include "ln_kernels.cuh"
+
+using namespace ln;
+
+namespace {
+
+constexpr int kSMs = 148;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Bump allocator over a caller-provided buffer; with base == nullptr it only measures.
+struct Carver {
+  char* base; size_t off;
+  explicit Carver(void* b) : base(static_cast<char*>(b)), off(0) {}
+  float* take(size_t nfloats) {
+    float* p = base ? reinterpret_cast<float*>(base + off) : nullptr;
+    off += align_up(nfloats * sizeof(float), 256);
+    return p;
+  }
+};
+
+struct Plan {
+  int BH, n, d, m, T, ldm, rpc, chunks;
+};
+
+bool make_plan(const ln_problem* p, Plan* pl) {
+  if (!p) return false;
+  pl->BH = p->B * p->H; pl->n = p->n; pl->d = p->d; pl->m = p->m; pl->T = p->ns_iters;
+  pl->ldm = (p->m + 3) & ~3;
+  // token chunks per head for the reductions over tokens: enough CTAs to fill the GPU twice
+  int want = (2 * kSMs + pl->BH - 1) / pl->BH;
+  if (want < 1) want = 1;
+  int rpc = (p->n + want - 1) / want;
+  rpc = (rpc + 31) / 32 * 32;
+  pl->rpc = rpc;
+  pl->chunks = (p->n + rpc - 1) / rpc;
+  return true;
+}
+
+// Forward context (saved for the backward pass, or carved from ws for inference)
+struct Ctx { float *Lf, *C, *Rt, *mu, *W, *Xh, *M, *Yt, *ybar; NsHdr* hdr; size_t bytes; };
+Ctx carve_ctx(const Plan& pl, void* base) {
+  Carver c(base); Ctx x;
+  const size_t BH = pl.BH, n = pl.n, d = pl.d, m = pl.m;
+  x.Lf = c.take(BH * m * d);
+  x.C = c.take(BH * n * pl.ldm);
+  x.Rt = c.take(BH * n * pl.ldm);
+  x.mu = c.take(BH * n);
+  x.W = c.take(BH * m * m);
+  x.Xh = c.take(BH * (pl.T + 1) * m * m);
+  x.M = c.take(BH * m * d);
+  x.Yt = c.take(BH * m * d);
+  x.ybar = c.take(BH * d);
+  x.hdr = reinterpret_cast<NsHdr*>(c.take(BH * (sizeof(NsHdr) / sizeof(float))));
+  x.bytes = c.off;
+  return x;
+}
+
+struct FwdWs { float *Mpart, *Wr, *P, *Y; size_t bytes; };
+FwdWs carve_fwd_ws(const Plan& pl, void* base) {
+  Carver c(base); FwdWs w;
+  const size_t BH = pl.BH, d = pl.d, m = pl.m;
+  w.Mpart = c.take(BH * pl.chunks * m * d);
+  w.Wr = c.take(BH * m * m);
+  w.P = c.take(BH * m * m);
+  w.Y = c.take(BH * m * d);
+  w.bytes = c.off;
+  return w;
+}
+
+struct BwdWs {
+  float *G, *dYtpart, *dybpart, *dLCpart, *dLRpart, *dY, *dM, *Wr, *P, *Hm, *Ga, *Gb, *dW, *dX, *GW, *dLW, *dLtot, *dKpart;
+  size_t bytes;
+};
+BwdWs carve_bwd_ws(const Plan& pl, void* base) {
+  Carver c(base); BwdWs w;
+  const size_t BH = pl.BH, n = pl.n, d = pl.d, m = pl.m, ch = pl.chunks;
+  w.G = c.take(BH * n * pl.ldm);
+  w.dYtpart = c.take(BH * ch * m * d);
+  w.dybpart = c.take(BH * ch * d);
+  w.dLCpart = c.take(BH * ch * m * d);
+  w.dLRpart = c.take(BH * ch * m * d);
+  w.dY = c.take(BH * m * d);
+  w.dM = c.take(BH * m * d);
+  w.Wr = c.take(BH * m * m);
+  w.P = c.take(BH * m * m);
+  w.Hm = c.take(BH * m * m);
+  w.Ga = c.take(BH * m * m);
+  w.Gb = c.take(BH * m * m);
+  w.dW = c.take(BH * m * m);
+  w.dX = c.take(BH * m * m);
+  w.GW = c.take(BH * m * pl.ldm);
+  w.dLW = c.take(BH * m * d);
+  w.dLtot = c.take(BH * m * d);
+  w.dKpart = c.take(BH * n * d);
+  w.bytes = c.off;
+  return w;
+}
+
+int validate(const ln_problem* p) {
+  if (!p) return LN_ERR_ARG;
+  if (p->B <= 0 || p->H <= 0 || p->n <= 0 || p->d <= 0 || p->m <= 0) return LN_ERR_ARG;
+  if (p->m > p->n) return LN_ERR_ARG;
+  if (!(p->lambda > 0.f) || !isfinite(p->lambda)) return LN_ERR_ARG;
+  if (p->ns_iters < 0) return LN_ERR_ARG;
+  if (!(p->ridge_eps >= 0.f) || !isfinite(p->ridge_eps)) return LN_ERR_ARG;
+  if (!isfinite(p->ns_alpha)) return LN_ERR_ARG;
+  if (p->dtype != LN_F32 && p->dtype != LN_BF16) return LN_ERR_ARG;
+  if (p->map_mode != 0 && p->map_mode != 1) return LN_ERR_ARG;
+  if (p->lm_mode != 0 && p->lm_mode != 1) return LN_ERR_ARG;
+  if (p->whiten && !aligned16(p->whiten)) return LN_ERR_ARG;
+  if (p->lm_mode == 1) {
+    if (p->prefix < 0 || p->gh <= 0 || p->gw <= 0 || p->mh <= 0 || p->mw <= 0) return LN_ERR_ARG;
+    if ((long long)p->prefix + (long long)p->gh * p->gw != p->n) return LN_ERR_ARG;
+    if ((long long)p->mh * p->mw != p->m) return LN_ERR_ARG;
+    if (p->mh > p->gh || p->mw > p->gw) return LN_ERR_ARG;
+  }
+  if ((long long)p->B * p->H > 65535) return LN_ERR_UNSUPPORTED;
+  if (p->d != 32 && p->d != 64 && p->d != 128) return LN_ERR_UNSUPPORTED;
+  if (p->m > 256) return LN_ERR_UNSUPPORTED;
+  return LN_OK;
+}
+
+PoolGeom geom_of(const ln_problem* p) {
+  PoolGeom g; g.n = p->n; g.d = p->d; g.m = p->m; g.prefix = p->prefix; g.gh = p->gh; g.gw = p->gw; g.mh = p->mh; g.mw = p->mw;
+  return g;
+}
+
+inline int launch_ok() { return cudaGetLastError() == cudaSuccess ? LN_OK : LN_ERR_CUDA; }
+inline unsigned cdiv(long long a, long long b) { return (unsigned)((a + b - 1) / b); }
+
+template <typename TA, typename TB>
+void launch_l1(const TA* A, const TB* Bm, float* E, float* rowsum, int batch, int na, int nb, int d,
+               int lde, float lambda, cudaStream_t st) {
+  const float nscale = -1.4426950408889634f / lambda;
+  dim3 grid(cdiv(na, L1_TA), batch);
+  k_l1<TA, TB><<<grid, 256, 0, st>>>(A, Bm, E, rowsum, na, nb, d, (long long)na * d, (long long)nb * d,
+                                     (long long)na * lde, lde, nscale);
+}
+
+// ------------------------------------------------------------------------------------------
+template <typename T, int D>
+int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const T* V, const T* L, T* O,
+             const Ctx& x, const FwdWs& w, int32_t* dev_status, cudaStream_t st) {
+  const int BH = pl.BH, n = pl.n, m = pl.m;
+  // landmarks (Sec. 4.2)
+  if (p->lm_mode == 1) {
+    k_pool<T><<<dim3(m, BH), 128, 0, st>>>(K, x.Lf, geom_of(p));
+  } else {
+    const long long cnt = (long long)BH * m * D;
+    k_to_f32<T><<<cdiv(cnt, 256), 256, 0, st>>>(L, x.Lf, cnt);
+  }
+  // the three kernel blocks: C = k(Q,L) with its row sums, R^T = k(K,L), W = k(L,L)
+  launch_l1<T, float>(Q, x.Lf, x.C, p->map_mode == 1 ? x.mu : nullptr, BH, n, m, D, pl.ldm, p->lambda, st);
+  if (p->map_mode == 1) k_scale<<<cdiv((long long)BH * n, 256), 256, 0, st>>>(x.mu, (long long)BH * n, 1.f / (float)m);
+  launch_l1<T, float>(K, x.Lf, x.Rt, nullptr, BH, n, m, D, pl.ldm, p->lambda, st);
+  launch_l1<float, float>(x.Lf, x.Lf, x.W, nullptr, BH, m, m, D, m, p->lambda, st);
+  // M = R V, partial over token chunks
+  k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, w.Mpart, nullptr, n, m, pl.rpc);
+  // Newton-Schulz, Y = X M, folded map
+  k_mid_fwd<D><<<BH, 256, 0, st>>>(m, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode, p->whiten, x.W, w.Wr, w.P,
+                                   x.Xh, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt, x.ybar, dev_status);
+  // O = (C - mu) Ytilde + ybar
+  k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr, x.Yt, x.ybar, O, n, m);
+  return launch_ok();
+}
+
+template <typename T, int D>
+int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const T* V, const T* dO,
+             const Ctx& x, const BwdWs& w, T* dQ, T* dK, T* dV, T* dL, cudaStream_t st) {
+  const int BH = pl.BH, n = pl.n, m = pl.m, ch = pl.chunks;
+  const float inv_lambda = 1.f / p->lambda;
+  const float* mu = p->map_mode == 1 ? x.mu : nullptr;
+  // query side: Z'^T dO and column sums of dO; g^C = (dO Ytilde^T) o C / lambda; dQ; landmark part
+  k_tn<T, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc);
+  k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(dO, x.Yt, x.C, pl.ldm, w.G, n, m, inv_lambda);
+  k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m);
+  k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc);
+  // per head: dY, dX, dM, Newton-Schulz adjoint, symmetrised landmark-block upstream
+  k_mid_bwd<D><<<BH, 256, 0, st>>>(m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten, x.W, x.Xh, x.hdr, x.M,
+                                   w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P, w.Hm, w.Ga, w.Gb, w.dW, w.dX,
+                                   w.dY, w.dM, w.GW);
+  k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, st>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m);
+  // key side: g^R = (V dM^T) o R^T / lambda; dV = R^T dM; dK (kernel part); landmark part
+  k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(V, w.dM, x.Rt, pl.ldm, w.G, n, m, inv_lambda);
+  k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m);
+  k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dKpart, n, m);
+  k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dLRpart, n, m, pl.rpc);
+  // landmark gradient and its way back to the keys
+  const int md = m * D;
+  if (p->lm_mode == 1) {
+    k_reduce3<float><<<dim3(cdiv(md, 256), BH), 256, 0, st>>>(w.dLCpart, ch, w.dLRpart, ch, w.dLW, 1, w.dLtot, md);
+    k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256), BH), 256, 0, st>>>(w.dKpart, w.dLtot, dK, geom_of(p), 1);
+  } else {
+    k_reduce3<T><<<dim3(cdiv(md, 256), BH), 256, 0, st>>>(w.dLCpart, ch, w.dLRpart, ch, w.dLW, 1, dL, md);
+    k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256), BH), 256, 0, st>>>(w.dKpart, nullptr, dK, geom_of(p), 0);
+  }
+  return launch_ok();
+}
+
+template <typename T>
+int fwd_dispatch_d(const ln_problem* p, const Plan& pl, const void* Q, const void* K, const void* V, const void* L,
+                   void* O, const Ctx& x, const FwdWs& w, int32_t* ds, cudaStream_t st) {
+  const T *q = (const T*)Q, *k = (const T*)K, *v = (const T*)V, *l = (const T*)L; T* o = (T*)O;
+  switch (p->d) {
+    case 32: return fwd_impl<T, 32>(p, pl, q, k, v, l, o, x, w, ds, st);
+    case 64: return fwd_impl<T, 64>(p, pl, q, k, v, l, o, x, w, ds, st);
+    case 128: return fwd_impl<T, 128>(p, pl, q, k, v, l, o, x, w, ds, st);
+  }
+  return LN_ERR_UNSUPPORTED;
+}
+template <typename T>
+int bwd_dispatch_d(const ln_problem* p, const Plan& pl, const void* Q, const void* K, const void* V, const void* dO,
+                   const Ctx& x, const BwdWs& w, void* dQ, void* dK, void* dV, void* dL, cudaStream_t st) {
+  const T *q = (const T*)Q, *k = (const T*)K, *v = (const T*)V, *g = (const T*)dO;
+  switch (p->d) {
+    case 32: return bwd_impl<T, 32>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, st);
+    case 64: return bwd_impl<T, 64>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, st);
+    case 128: return bwd_impl<T, 128>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, st);
+  }
+  return LN_ERR_UNSUPPORTED;
+}
+
+// ---- stand-alone ns_pinv scratch
+struct NsWs { float *Wr, *P, *Hm, *Ga, *Gb, *Xh; NsHdr* hdr; size_t bytes; };
+NsWs carve_ns_ws(int batch, int m, int T, void* base) {
+  Carver c(base); NsWs w;
+  const size_t mm = (size_t)m * m, b = batch;
+  w.Wr = c.take(b * mm); w.P = c.take(b * mm); w.Hm = c.take(b * mm); w.Ga = c.take(b * mm); w.Gb = c.take(b * mm);
+  w.Xh = c.take(b * (T + 1) * mm);
+  w.hdr = reinterpret_cast<NsHdr*>(c.take(b * (sizeof(NsHdr) / sizeof(float))));
+  w.bytes = c.off;
+  return w;
+}
+
+}  // namespace
+
+namespace {
+struct L1BwdWs { float *Kmat, *G, *part; int rpc, chunks; size_t bytes; };
+L1BwdWs carve_l1bwd(int batch, int na, int nb, int d, void* base) {
+  Carver c(base); L1BwdWs w;
+  int want = (2 * kSMs + batch - 1) / batch; if (want < 1) want = 1;
+  int rpc = (na + want - 1) / want; rpc = (rpc + 31) / 32 * 32;
+  w.rpc = rpc; w.chunks = (na + rpc - 1) / rpc;
+  w.Kmat = c.take((size_t)batch * na * nb);
+  w.G = c.take((size_t)batch * na * nb);
+  w.part = c.take((size_t)batch * w.chunks * nb * d);
+  w.bytes = c.off;
+  return w;
+}
+template <typename T, int D>
+void l1_bwd_impl(int batch, int na, int nb, const T* A, const T* Bm, float lambda, const float* Kmat, const float* dK,
+                 T* dA, T* dB, const L1BwdWs& w, cudaStream_t st) {
+  if (!Kmat) { launch_l1<T, T>(A, Bm, w.Kmat, nullptr, batch, na, nb, D, nb, lambda, st); Kmat = w.Kmat; }
+  const long long cnt = (long long)batch * na * nb;
+  k_g_elem<<<cdiv(cnt, 256), 256, 0, st>>>(Kmat, dK, w.G, cnt, 1.f / lambda);
+  k_sign_rows<T, T, T, D><<<dim3(cdiv(na, 64), batch), 256, 0, st>>>(A, Bm, w.G, nb, dA, na, nb);
+  k_sign_cols<T, T, D><<<dim3(w.chunks, cdiv(nb, 64), batch), 256, 0, st>>>(A, Bm, w.G, nb, w.part, na, nb, w.rpc);
+  k_reduce3<T><<<dim3(cdiv(nb * D, 256), batch), 256, 0, st>>>(w.part, w.chunks, nullptr, 0, nullptr, 0, dB, nb * D);
+}
+}  // namespace
+
+// ==========================================================================================
+extern "C" {
+
+const char* ln_status_string(int s) {
+  switch (s) {
+    case LN_OK: return "ok";
+    case LN_ERR_ARG: return "invalid argument";
+    case LN_ERR_UNSUPPORTED: return "outside the supported envelope";
+    case LN_ERR_WORKSPACE: return "workspace too small";
+    case LN_ERR_CUDA: return "CUDA launch failed";
+  }
+  return "unknown status";
+}
+
+size_t laplace_nystrom_saved_bytes(const ln_problem* p) {
+  if (validate(p) != LN_OK) return 0;
+  Plan pl; make_plan(p, &pl);
+  return carve_ctx(pl, nullptr).bytes;
+}
+
+size_t laplace_nystrom_workspace_bytes(const ln_problem* p, int32_t with_saved) {
+  if (validate(p) != LN_OK) return 0;
+  Plan pl; make_plan(p, &pl);
+  const size_t f = carve_fwd_ws(pl, nullptr).bytes, b = carve_bwd_ws(pl, nullptr).bytes;
+  size_t ws = f > b ? f : b;
+  if (!with_saved) ws = f + carve_ctx(pl, nullptr).bytes;
+  return ws;
+}
+
+int laplace_nystrom_fwd(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L, void* O,
+                        void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
+  int s = validate(p);
+  if (s != LN_OK) return s;
+  if (!Q || !K || !V || !O || !ws) return LN_ERR_ARG;
+  if ((p->lm_mode == 0) != (L != nullptr)) return LN_ERR_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(ws) || !aligned16(L) ||
+      !aligned16(saved))
+    return LN_ERR_ARG;
+  if (ws_bytes < laplace_nystrom_workspace_bytes(p, saved != nullptr)) return LN_ERR_WORKSPACE;
+  Plan pl; make_plan(p, &pl);
+  const FwdWs w = carve_fwd_ws(pl, ws);
+  const Ctx x = carve_ctx(pl, saved ? saved : static_cast<char*>(ws) + w.bytes);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (p->dtype == LN_F32) return fwd_dispatch_d<float>(p, pl, Q, K, V, L, O, x, w, dev_status, st);
+  return fwd_dispatch_d<bf16>(p, pl, Q, K, V, L, O, x, w, dev_status, st);
+}
+
+int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L,
+                        const void* dO, const void* saved, void* dQ, void* dK, void* dV, void* dL, void* ws,
+                        size_t ws_bytes, int32_t* dev_status, void* stream) {
+  (void)dev_status;
+  int s = validate(p);
+  if (s != LN_OK) return s;
+  if (!Q || !K || !V || !dO || !saved || !dQ || !dK || !dV || !ws) return LN_ERR_ARG;
+  if ((p->lm_mode == 0) != (L != nullptr)) return LN_ERR_ARG;
+  if ((p->lm_mode == 0) != (dL != nullptr)) return LN_ERR_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dO) || !aligned16(saved) || !aligned16(dQ) ||
+      !aligned16(dK) || !aligned16(dV) || !aligned16(dL) || !aligned16(ws))
+    return LN_ERR_ARG;
+  if (ws_bytes < laplace_nystrom_workspace_bytes(p, 1)) return LN_ERR_WORKSPACE;
+  Plan pl; make_plan(p, &pl);
+  const BwdWs w = carve_bwd_ws(pl, ws);
+  const Ctx x = carve_ctx(pl, const_cast<void*>(saved));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (p->dtype == LN_F32) return bwd_dispatch_d<float>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, st);
+  return bwd_dispatch_d<bf16>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, st);
+}
+
+size_t ns_pinv_workspace_bytes(int32_t batch, int32_t m, int32_t iters) {
+  if (batch <= 0 || m <= 0 || iters < 0) return 0;
+  return carve_ns_ws(batch, m, iters, nullptr).bytes;
+}
+
+int ns_pinv(int32_t batch, int32_t m, const float* W, int32_t iters, float ridge_eps, float alpha, float* X,
+            float* X_hist, float* resid, void* ws, size_t ws_bytes, void* stream) {
+  if (batch <= 0 || m <= 0 || iters < 0 || !W || !X || !ws) return LN_ERR_ARG;
+  if (!(ridge_eps >= 0.f) || !isfinite(ridge_eps) || !isfinite(alpha)) return LN_ERR_ARG;
+  if (!aligned16(W) || !aligned16(X) || !aligned16(X_hist) || !aligned16(ws)) return LN_ERR_ARG;
+  if (m > 256) return LN_ERR_UNSUPPORTED;
+  if (ws_bytes < ns_pinv_workspace_bytes(batch, m, iters)) return LN_ERR_WORKSPACE;
+  const NsWs w = carve_ns_ws(batch, m, iters, ws);
+  k_ns_pinv<<<batch, 256, 0, static_cast<cudaStream_t>(stream)>>>(m, iters, ridge_eps, alpha, W, w.Wr, w.P,
+                                                                  X_hist ? X_hist : w.Xh, w.hdr, X, resid);
+  return launch_ok();
+}
+
+int ns_pinv_bwd(int32_t batch, int32_t m, const float* W, int32_t iters, float ridge_eps, float alpha,
+                const float* X_hist, const float* dX, float* dW, void* ws, size_t ws_bytes, void* stream) {
+  if (batch <= 0 || m <= 0 || iters < 0 || !W || !dX || !dW || !ws) return LN_ERR_ARG;
+  if (!(ridge_eps >= 0.f) || !isfinite(ridge_eps) || !isfinite(alpha)) return LN_ERR_ARG;
+  if (!aligned16(W) || !aligned16(dX) || !aligned16(dW) || !aligned16(X_hist) || !aligned16(ws)) return LN_ERR_ARG;
+  if (m > 256) return LN_ERR_UNSUPPORTED;
+  if (ws_bytes < ns_pinv_workspace_bytes(batch, m, iters)) return LN_ERR_WORKSPACE;
+  const NsWs w = carve_ns_ws(batch, m, iters, ws);
+  k_ns_pinv_bwd<<<batch, 256, 0, static_cast<cudaStream_t>(stream)>>>(m, iters, ridge_eps, alpha, W, w.Wr, w.P, w.Hm,
+                                                                      w.Ga, w.Gb, w.Xh, X_hist, w.hdr, dX, dW);
+  return launch_ok();
+}
+
+int l1_kernel(int32_t batch, int32_t na, int32_t nb, int32_t d, const void* A, const void* Bm, int32_t dtype,
+              float lambda, float* Kout, float* rowsum, void* stream) {
+  if (batch <= 0 || na <= 0 || nb <= 0 || d <= 0 || !A || !Bm || !Kout) return LN_ERR_ARG;
+  if (!(lambda > 0.f) || !isfinite(lambda)) return LN_ERR_ARG;
+  if (dtype != LN_F32 && dtype != LN_BF16) return LN_ERR_ARG;
+  if (!aligned16(A) || !aligned16(Bm) || !aligned16(Kout) || !aligned16(rowsum)) return LN_ERR_ARG;
+  if (batch > 65535) return LN_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (dtype == LN_F32) launch_l1<float, float>((const float*)A, (const float*)Bm, Kout, rowsum, batch, na, nb, d, nb, lambda, st);
+  else launch_l1<bf16, bf16>((const bf16*)A, (const bf16*)Bm, Kout, rowsum, batch, na, nb, d, nb, lambda, st);
+  return launch_ok();
+}
+
+
+size_t l1_kernel_bwd_workspace_bytes(int32_t batch, int32_t na, int32_t nb, int32_t d) {
+  if (batch <= 0 || na <= 0 || nb <= 0 || d <= 0) return 0;
+  return carve_l1bwd(batch, na, nb, d, nullptr).bytes;
+}
+
+int l1_kernel_bwd(int32_t batch, int32_t na, int32_t nb, int32_t d, const void* A, const void* Bm, int32_t dtype,
+                  float lambda, const float* Kmat, const float* dKmat, void* dA, void* dB, void* ws, size_t ws_bytes,
+                  void* stream) {
+  if (batch <= 0 || na <= 0 || nb <= 0 || d <= 0 || !A || !Bm || !dKmat || !dA || !dB || !ws) return LN_ERR_ARG;
+  if (!(lambda > 0.f) || !isfinite(lambda)) return LN_ERR_ARG;
+  if (dtype != LN_F32 && dtype != LN_BF16) return LN_ERR_ARG;
+  if (!aligned16(A) || !aligned16(Bm) || !aligned16(Kmat) || !aligned16(dKmat) || !aligned16(dA) || !aligned16(dB) ||
+      !aligned16(ws))
+    return LN_ERR_ARG;
+  if (d != 32 && d != 64 && d != 128) return LN_ERR_UNSUPPORTED;
+  if (batch > 65535) return LN_ERR_UNSUPPORTED;
+  if (ws_bytes < l1_kernel_bwd_workspace_bytes(batch, na, nb, d)) return LN_ERR_WORKSPACE;
+  const L1BwdWs w = carve_l1bwd(batch, na, nb, d, ws);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+#define LN_L1B(T, D) l1_bwd_impl<T, D>(batch, na, nb, (const T*)A, (const T*)Bm, lambda, Kmat, dKmat, (T*)dA, (T*)dB, w, st)
+  if (dtype == LN_F32) { if (d == 32) LN_L1B(float, 32); else if (d == 64) LN_L1B(float, 64); else LN_L1B(float, 128); }
+  else { if (d == 32) LN_L1B(bf16, 32); else if (d == 64) LN_L1B(bf16, 64); else LN_L1B(bf16, 128); }
+#undef LN_L1B
+  return launch_ok();
+}
+
+int landmarks_pool(const ln_problem* p, const void* K, float* L, void* stream) {
+  int s = validate(p);
+  if (s != LN_OK) return s;
+  if (p->lm_mode != 1 || !K || !L || !aligned16(K) || !aligned16(L)) return LN_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  dim3 grid(p->m, p->B * p->H);
+  if (p->dtype == LN_F32) k_pool<float><<<grid, 128, 0, st>>>((const float*)K, L, geom_of(p));
+  else k_pool<bf16><<<grid, 128, 0, st>>>((const bf16*)K, L, geom_of(p));
+  return launch_ok();
+}
+
+int landmarks_pool_bwd(const ln_problem* p, const float* dL, void* dK, void* stream) {
+  int s = validate(p);
+  if (s != LN_OK) return s;
+  if (p->lm_mode != 1 || !dL || !dK || !aligned16(dL) || !aligned16(dK)) return LN_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  dim3 grid(cdiv((long long)p->n * (p->d / 4), 256), p->B * p->H);
+  if (p->dtype == LN_F32) k_pool_bwd<float><<<grid, 256, 0, st>>>(nullptr, dL, (float*)dK, geom_of(p), 1);
+  else k_pool_bwd<bf16><<<grid, 256, 0, st>>>(nullptr, dL, (bf16*)dK, geom_of(p), 1);
+  return launch_ok();
+}
+
+}  // extern "C"

@@ -1,0 +1,75 @@
+// Shared device helpers of the Laplacian-Nystrom kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ln {
+
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ float to_f(float x) { return x; }
+__device__ __forceinline__ float to_f(bf16 x) { return __bfloat162float(x); }
+
+template <typename T> __device__ __forceinline__ T from_f(float x);
+template <> __device__ __forceinline__ float from_f<float>(float x) { return x; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float x) { return __float2bfloat16_rn(x); }
+
+// Four consecutive elements as fp32.  The address must be aligned to 4 elements.
+__device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 ld4(const bf16* p) {
+  uint2 r = *reinterpret_cast<const uint2*>(p);
+  float4 v;
+  v.x = __uint_as_float(r.x << 16);
+  v.y = __uint_as_float(r.x & 0xffff0000u);
+  v.z = __uint_as_float(r.y << 16);
+  v.w = __uint_as_float(r.y & 0xffff0000u);
+  return v;
+}
+__device__ __forceinline__ void st4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+__device__ __forceinline__ void st4(bf16* p, float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
+  __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 r;
+  r.x = *reinterpret_cast<uint32_t*>(&lo);
+  r.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = r;
+}
+
+// 2^x, approximate (relative error about 2^-22); the exponent of the Laplacian kernel is
+// evaluated as 2^(-dist * log2(e) / lambda).
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// g * sign(t) with sign(0) = 0: the kernel gradient of App. A (stated there for t != 0), with
+// the midpoint sub-gradient at a tie.
+__device__ __forceinline__ float signed_g(float t, float g) { return t > 0.f ? g : (t < 0.f ? -g : 0.f); }
+
+// Column set a thread owns in a [rows x D] tile worked on by 16 column-threads: DC = D/16
+// columns, laid out so that the 16 threads read one contiguous 256-byte (128 for D = 32) run.
+template <int D> struct ColMap {
+  static constexpr int DC = D / 16;
+  // index q in [0, DC) -> column
+  __device__ static __forceinline__ int col(int tc, int q) {
+    if (D == 32) return tc * 2 + q;
+    return (q >> 2) * 64 + tc * 4 + (q & 3);
+  }
+};
+
+template <int D> __device__ __forceinline__ void ld_cols(const float* row, int tc, float (&v)[D / 16]) {
+  if (D == 32) {
+    float2 a = *reinterpret_cast<const float2*>(row + tc * 2);
+    v[0] = a.x; v[1] = a.y;
+  } else {
+#pragma unroll
+    for (int h = 0; h < D / 64; ++h) {
+      float4 a = *reinterpret_cast<const float4*>(row + h * 64 + tc * 4);
+      v[h * 4 + 0] = a.x; v[h * 4 + 1] = a.y; v[h * 4 + 2] = a.z; v[h * 4 + 3] = a.w;
+    }
+  }
+}
+
+}  // namespace ln

@@ -1,0 +1,901 @@
+// FP32 CUDA-core kernels of the Laplacian-Nystrom path.  Every kernel works on one
+// (batch*head) slice per blockIdx.z / blockIdx.y and a tile of tokens or landmarks per
+// blockIdx.x.  All intermediates are fp32; only the [.,.,.,d] user tensors have a storage type.
+#pragma once
+#include "ln_common.cuh"
+
+namespace ln {
+
+// =====================================================================================
+// Laplacian kernel block (Sec. 1, Eq. 8):  E[i][j] = exp(-sum_c |a_ic - b_jc| / lambda)
+// CTA: 128 rows of A x (all of B in blocks of 64); thread: 8 x 4 pairs; d in chunks of 32
+// staged in shared memory dimension-major so one 128-bit load serves four rows.
+// =====================================================================================
+constexpr int L1_TA = 128, L1_TB = 64, L1_DC = 32;
+
+template <typename TA, typename TB>
+__global__ void __launch_bounds__(256) k_l1(const TA* __restrict__ A, const TB* __restrict__ Bm,
+                                            float* __restrict__ E, float* __restrict__ rowsum, int na, int nb, int d,
+                                            long long sA, long long sB, long long sE, int lde, float nscale) {
+  __shared__ __align__(16) float As[L1_DC][L1_TA + 4];
+  __shared__ __align__(16) float Bs[L1_DC][L1_TB + 4];
+  const int b = blockIdx.y, i0 = blockIdx.x * L1_TA;
+  A += (long long)b * sA;
+  Bm += (long long)b * sB;
+  E += (long long)b * sE;
+  const int tid = threadIdx.x, tj = tid & 15, ti = tid >> 4;
+  const bool vec = (d % 8) == 0;
+  float rs[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) rs[i] = 0.f;
+
+  for (int j0 = 0; j0 < nb; j0 += L1_TB) {
+    float acc[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int c0 = 0; c0 < d; c0 += L1_DC) {
+      __syncthreads();
+      {  // A chunk: 128 rows x 32 dims; thread = (row, 16-dim half)
+        const int r = tid & 127, cb = (tid >> 7) * 16, gi = i0 + r;
+        const TA* src = A + (long long)gi * d + c0 + cb;
+        if (vec && gi < na && c0 + cb + 16 <= d) {
+#pragma unroll
+          for (int k = 0; k < 16; k += 4) {
+            float4 v = ld4(src + k);
+            As[cb + k][r] = v.x; As[cb + k + 1][r] = v.y; As[cb + k + 2][r] = v.z; As[cb + k + 3][r] = v.w;
+          }
+        } else {
+#pragma unroll 4
+          for (int k = 0; k < 16; ++k) As[cb + k][r] = (gi < na && c0 + cb + k < d) ? to_f(src[k]) : 0.f;
+        }
+      }
+      {  // B chunk: 64 rows x 32 dims; thread = (row, 8-dim quarter)
+        const int r = tid & 63, cb = (tid >> 6) * 8, gj = j0 + r;
+        const TB* src = Bm + (long long)gj * d + c0 + cb;
+        if (vec && gj < nb && c0 + cb + 8 <= d) {
+#pragma unroll
+          for (int k = 0; k < 8; k += 4) {
+            float4 v = ld4(src + k);
+            Bs[cb + k][r] = v.x; Bs[cb + k + 1][r] = v.y; Bs[cb + k + 2][r] = v.z; Bs[cb + k + 3][r] = v.w;
+          }
+        } else {
+#pragma unroll 4
+          for (int k = 0; k < 8; ++k) Bs[cb + k][r] = (gj < nb && c0 + cb + k < d) ? to_f(src[k]) : 0.f;
+        }
+      }
+      __syncthreads();
+#pragma unroll 8
+      for (int c = 0; c < L1_DC; ++c) {
+        const float4 a0 = *reinterpret_cast<const float4*>(&As[c][ti * 8]);
+        const float4 a1 = *reinterpret_cast<const float4*>(&As[c][ti * 8 + 4]);
+        const float4 bb = *reinterpret_cast<const float4*>(&Bs[c][tj * 4]);
+        const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+        const float bv[4] = {bb.x, bb.y, bb.z, bb.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i][j] += fabsf(a[i] - bv[j]);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int gi = i0 + ti * 8 + i;
+      if (gi >= na) continue;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int gj = j0 + tj * 4 + j;
+        if (gj < nb) {
+          const float e = ex2(acc[i][j] * nscale);
+          E[(long long)gi * lde + gj] = e;
+          rs[i] += e;
+        } else if (gj < lde) {
+          E[(long long)gi * lde + gj] = 0.f;   // padding columns of a padded leading dimension
+        }
+      }
+    }
+  }
+  if (rowsum) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      float v = rs[i];
+      v += __shfl_xor_sync(0xffffffffu, v, 1);
+      v += __shfl_xor_sync(0xffffffffu, v, 2);
+      v += __shfl_xor_sync(0xffffffffu, v, 4);
+      v += __shfl_xor_sync(0xffffffffu, v, 8);
+      const int gi = i0 + ti * 8 + i;
+      if (tj == 0 && gi < na) rowsum[(long long)b * na + gi] = v;
+    }
+  }
+}
+
+// rowsum -> row mean (Prop. 3 step 2), in place
+__global__ void k_scale(float* x, long long count, float s) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) x[i] *= s;
+}
+
+// storage type -> fp32 copy
+template <typename T> __global__ void k_to_f32(const T* __restrict__ x, float* __restrict__ y, long long count) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) y[i] = to_f(x[i]);
+}
+
+// =====================================================================================
+// Landmark selection: adaptive average pooling of the keys over the token grid (Sec. 4.2)
+// =====================================================================================
+struct PoolGeom { int n, d, m, prefix, gh, gw, mh, mw; };
+__host__ __device__ inline int bin_lo(int a, int g, int mb) { return (int)(((long long)a * g) / mb); }
+__host__ __device__ inline int bin_hi(int a, int g, int mb) { return (int)((((long long)(a + 1)) * g + mb - 1) / mb); }
+
+template <typename T>
+__global__ void k_pool(const T* __restrict__ K, float* __restrict__ L, PoolGeom g) {
+  const int l = blockIdx.x, bh = blockIdx.y, c = threadIdx.x;
+  if (c >= g.d) return;
+  const int a = l / g.mw, bb = l % g.mw;
+  const int r0 = bin_lo(a, g.gh, g.mh), r1 = bin_hi(a, g.gh, g.mh);
+  const int c0 = bin_lo(bb, g.gw, g.mw), c1 = bin_hi(bb, g.gw, g.mw);
+  const T* Kh = K + (long long)bh * g.n * g.d;
+  float s = 0.f;
+  for (int r = r0; r < r1; ++r)
+    for (int q = c0; q < c1; ++q) s += to_f(Kh[(long long)(g.prefix + r * g.gw + q) * g.d + c]);
+  L[((long long)bh * g.m + l) * g.d + c] = s / (float)((r1 - r0) * (c1 - c0));
+}
+
+// dK[j] = dKpart[j] (may be NULL) + sum over the bins containing token j of dL[bin] / |bin|
+// (pooling adjoint); with pool == 0 it only converts dKpart to the storage type.
+template <typename T>
+__global__ void k_pool_bwd(const float* __restrict__ dKpart, const float* __restrict__ dL, T* __restrict__ dK,
+                           PoolGeom g, int pool) {
+  const int bh = blockIdx.y;
+  const int per_row = g.d / 4;
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long long)g.n * per_row) return;
+  const int j = (int)(idx / per_row), c = (int)(idx % per_row) * 4;
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (dKpart) v = ld4(dKpart + ((long long)bh * g.n + j) * g.d + c);
+  if (pool && j >= g.prefix) {
+    const int r = (j - g.prefix) / g.gw, q = (j - g.prefix) % g.gw;
+    int a_lo = (int)(((long long)r * g.mh) / g.gh) - 1; if (a_lo < 0) a_lo = 0;
+    int b_lo = (int)(((long long)q * g.mw) / g.gw) - 1; if (b_lo < 0) b_lo = 0;
+    for (int a = a_lo; a < g.mh && a <= a_lo + 2; ++a) {
+      const int r0 = bin_lo(a, g.gh, g.mh), r1 = bin_hi(a, g.gh, g.mh);
+      if (r < r0 || r >= r1) continue;
+      for (int bb = b_lo; bb < g.mw && bb <= b_lo + 2; ++bb) {
+        const int c0 = bin_lo(bb, g.gw, g.mw), c1 = bin_hi(bb, g.gw, g.mw);
+        if (q < c0 || q >= c1) continue;
+        const float inv = 1.f / (float)((r1 - r0) * (c1 - c0));
+        const float4 t = ld4(dL + ((long long)bh * g.m + a * g.mw + bb) * g.d + c);
+        v.x += t.x * inv; v.y += t.y * inv; v.z += t.z * inv; v.w += t.w * inv;
+      }
+    }
+  }
+  st4(dK + ((long long)bh * g.n + j) * g.d + c, v);
+}
+
+// out[e] = sum_p parts[p][e] for up to three part arrays laid out [BH][np][count]
+template <typename TO>
+__global__ void k_reduce3(const float* __restrict__ p0, int n0, const float* __restrict__ p1, int n1,
+                          const float* __restrict__ p2, int n2, TO* __restrict__ out, int count) {
+  const int bh = blockIdx.y;
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= count) return;
+  float s = 0.f;
+  for (int p = 0; p < n0; ++p) s += p0[((long long)bh * n0 + p) * count + e];
+  for (int p = 0; p < n1; ++p) s += p1[((long long)bh * n1 + p) * count + e];
+  for (int p = 0; p < n2; ++p) s += p2[((long long)bh * n2 + p) * count + e];
+  out[(long long)bh * count + e] = from_f<TO>(s);
+}
+
+// =====================================================================================
+// part[chunk][l][c] = sum_{j in chunk} (E[j][l] - mu[j]) * U[j][c]     (reduction over tokens)
+// Used for M = R V (mu = NULL) and for the centred Z'^T dO of the backward pass.
+// Optionally also colsum_part[chunk][c] = sum_j U[j][c].
+// grid (chunks, ceil(m/64), BH); thread: 4 landmarks x D/16 columns
+// =====================================================================================
+template <typename TU, int D>
+__global__ void __launch_bounds__(256) k_tn(const float* __restrict__ E, int lde, const float* __restrict__ mu,
+                                            const TU* __restrict__ U, float* __restrict__ part,
+                                            float* __restrict__ colsum_part, int n, int m, int rpc) {
+  constexpr int DC = D / 16;
+  __shared__ __align__(16) float Es[32][64 + 4];
+  __shared__ __align__(16) float Us[32][D + 4];
+  const int chunk = blockIdx.x, l0 = blockIdx.y * 64, bh = blockIdx.z, nchunks = gridDim.x;
+  const int tid = threadIdx.x, tl = tid >> 4, tc = tid & 15;
+  E += (long long)bh * n * lde;
+  U += (long long)bh * n * D;
+  if (mu) mu += (long long)bh * n;
+  const int jbeg = chunk * rpc, jend = min(n, jbeg + rpc);
+  float acc[4][DC], cs[DC];
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+#pragma unroll
+    for (int q = 0; q < DC; ++q) acc[k][q] = 0.f;
+#pragma unroll
+  for (int q = 0; q < DC; ++q) cs[q] = 0.f;
+
+  for (int j0 = jbeg; j0 < jend; j0 += 32) {
+    __syncthreads();
+    {  // E tile: 32 tokens x 64 landmarks, 8 per thread
+      const int r = tid >> 3, cb = (tid & 7) * 8, j = j0 + r;
+      const float mj = (mu && j < jend) ? mu[j] : 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; k += 4) {
+        const int l = l0 + cb + k;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (j < jend && l < m) {
+          if (l + 3 < lde && (lde & 3) == 0) v = ld4(E + (long long)j * lde + l);
+          else {
+            v.x = E[(long long)j * lde + l];
+            if (l + 1 < m) v.y = E[(long long)j * lde + l + 1];
+            if (l + 2 < m) v.z = E[(long long)j * lde + l + 2];
+            if (l + 3 < m) v.w = E[(long long)j * lde + l + 3];
+          }
+          v.x = (l < m) ? v.x - mj : 0.f;
+          v.y = (l + 1 < m) ? v.y - mj : 0.f;
+          v.z = (l + 2 < m) ? v.z - mj : 0.f;
+          v.w = (l + 3 < m) ? v.w - mj : 0.f;
+        }
+        *reinterpret_cast<float4*>(&Es[r][cb + k]) = v;
+      }
+    }
+    for (int idx = tid; idx < 32 * (D / 4); idx += 256) {
+      const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4, j = j0 + r;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (j < jend) v = ld4(U + (long long)j * D + c4);
+      *reinterpret_cast<float4*>(&Us[r][c4]) = v;
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int jj = 0; jj < 32; ++jj) {
+      const float4 e4 = *reinterpret_cast<const float4*>(&Es[jj][tl * 4]);
+      float u[DC];
+      ld_cols<D>(&Us[jj][0], tc, u);
+      const float e[4] = {e4.x, e4.y, e4.z, e4.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int q = 0; q < DC; ++q) acc[k][q] = fmaf(e[k], u[q], acc[k][q]);
+      if (colsum_part && tl == 0)
+#pragma unroll
+        for (int q = 0; q < DC; ++q) cs[q] += u[q];
+    }
+  }
+  float* out = part + ((long long)bh * nchunks + chunk) * m * D;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int l = l0 + tl * 4 + k;
+    if (l < m)
+#pragma unroll
+      for (int q = 0; q < DC; ++q) out[(long long)l * D + ColMap<D>::col(tc, q)] = acc[k][q];
+  }
+  if (colsum_part && tl == 0 && blockIdx.y == 0)
+#pragma unroll
+    for (int q = 0; q < DC; ++q) colsum_part[((long long)bh * nchunks + chunk) * D + ColMap<D>::col(tc, q)] = cs[q];
+}
+
+// =====================================================================================
+// O[i][c] = sum_l (E[i][l] - mu[i]) * Y[l][c] + ybar[c]      (reduction over landmarks)
+// Used for O = Z' Ytilde + ybar (Eq. 7 in folded form) and dV = R^T dM (mu, ybar = NULL).
+// grid (ceil(n/64), BH); thread: 4 tokens x D/16 columns
+// =====================================================================================
+template <typename TO, int D>
+__global__ void __launch_bounds__(256) k_nn(const float* __restrict__ E, int lde, const float* __restrict__ mu,
+                                            const float* __restrict__ Y, const float* __restrict__ ybar,
+                                            TO* __restrict__ O, int n, int m) {
+  constexpr int DC = D / 16;
+  __shared__ __align__(16) float Es[64][32 + 4];
+  __shared__ __align__(16) float Ys[32][D + 4];
+  const int i0 = blockIdx.x * 64, bh = blockIdx.y;
+  const int tid = threadIdx.x, tt = tid >> 4, tc = tid & 15;
+  E += (long long)bh * n * lde;
+  Y += (long long)bh * m * D;
+  O += (long long)bh * n * D;
+  float acc[4][DC];
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+#pragma unroll
+    for (int q = 0; q < DC; ++q) acc[k][q] = 0.f;
+
+  for (int l0 = 0; l0 < m; l0 += 32) {
+    __syncthreads();
+    {  // E tile: 64 tokens x 32 landmarks
+      const int r = tid >> 2, cb = (tid & 3) * 8, i = i0 + r;
+      const float mi = (mu && i < n) ? mu[(long long)bh * n + i] : 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; k += 4) {
+        const int l = l0 + cb + k;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (i < n && l < m) {
+          if (l + 3 < lde && (lde & 3) == 0) v = ld4(E + (long long)i * lde + l);
+          else {
+            v.x = E[(long long)i * lde + l];
+            if (l + 1 < m) v.y = E[(long long)i * lde + l + 1];
+            if (l + 2 < m) v.z = E[(long long)i * lde + l + 2];
+            if (l + 3 < m) v.w = E[(long long)i * lde + l + 3];
+          }
+          v.x = (l < m) ? v.x - mi : 0.f;
+          v.y = (l + 1 < m) ? v.y - mi : 0.f;
+          v.z = (l + 2 < m) ? v.z - mi : 0.f;
+          v.w = (l + 3 < m) ? v.w - mi : 0.f;
+        }
+        *reinterpret_cast<float4*>(&Es[r][cb + k]) = v;
+      }
+    }
+    for (int idx = tid; idx < 32 * (D / 4); idx += 256) {
+      const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4, l = l0 + r;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (l < m) v = ld4(Y + (long long)l * D + c4);
+      *reinterpret_cast<float4*>(&Ys[r][c4]) = v;
+    }
+    __syncthreads();
+#pragma unroll 2
+    for (int ll = 0; ll < 32; ll += 4) {
+      float e[4][4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float4 t = *reinterpret_cast<const float4*>(&Es[tt * 4 + k][ll]);
+        e[k][0] = t.x; e[k][1] = t.y; e[k][2] = t.z; e[k][3] = t.w;
+      }
+#pragma unroll
+      for (int s = 0; s < 4; ++s) {
+        float y[DC];
+        ld_cols<D>(&Ys[ll + s][0], tc, y);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+#pragma unroll
+          for (int q = 0; q < DC; ++q) acc[k][q] = fmaf(e[k][s], y[q], acc[k][q]);
+      }
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int i = i0 + tt * 4 + k;
+    if (i < n)
+#pragma unroll
+      for (int q = 0; q < DC; ++q) {
+        const int c = ColMap<D>::col(tc, q);
+        const float yb = ybar ? ybar[(long long)bh * D + c] : 0.f;
+        O[(long long)i * D + c] = from_f<TO>(acc[k][q] + yb);
+      }
+  }
+}
+
+// =====================================================================================
+// G[i][l] = (sum_c U[i][c] * Y[l][c]) * E[i][l] / lambda       (reduction over d)
+// The upstream gradient of a kernel block times the kernel value (App. A): with U = dO, Y = Ytilde
+// it is dC o C / lambda, with U = V, Y = dM it is dR o R / lambda.
+// grid (ceil(n/64), ceil(m/64), BH); thread: tokens tt*4+k, landmarks tl+16q
+// =====================================================================================
+template <typename TU, int D>
+__global__ void __launch_bounds__(256) k_nt_g(const TU* __restrict__ U, const float* __restrict__ Y,
+                                              const float* __restrict__ E, int lde, float* __restrict__ G,
+                                              int n, int m, float inv_lambda) {
+  constexpr int DK = (D < 64) ? D : 64;
+  __shared__ __align__(16) float Us[64][DK + 4];
+  __shared__ __align__(16) float Ys[64][DK + 4];
+  const int i0 = blockIdx.x * 64, l0 = blockIdx.y * 64, bh = blockIdx.z;
+  const int tid = threadIdx.x, tt = tid >> 4, tl = tid & 15;
+  U += (long long)bh * n * D;
+  Y += (long long)bh * m * D;
+  E += (long long)bh * n * lde;
+  G += (long long)bh * n * lde;
+  float acc[4][4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+#pragma unroll
+    for (int q = 0; q < 4; ++q) acc[k][q] = 0.f;
+  for (int c0 = 0; c0 < D; c0 += DK) {
+    __syncthreads();
+    for (int idx = tid; idx < 64 * (DK / 4); idx += 256) {
+      const int r = idx / (DK / 4), c4 = (idx % (DK / 4)) * 4;
+      float4 u = make_float4(0.f, 0.f, 0.f, 0.f), y = u;
+      if (i0 + r < n) u = ld4(U + (long long)(i0 + r) * D + c0 + c4);
+      if (l0 + r < m) y = ld4(Y + (long long)(l0 + r) * D + c0 + c4);
+      *reinterpret_cast<float4*>(&Us[r][c4]) = u;
+      *reinterpret_cast<float4*>(&Ys[r][c4]) = y;
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int c = 0; c < DK; c += 4) {
+      float4 u[4], y[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) u[k] = *reinterpret_cast<const float4*>(&Us[tt * 4 + k][c]);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) y[q] = *reinterpret_cast<const float4*>(&Ys[tl + 16 * q][c]);
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          acc[k][q] += u[k].x * y[q].x + u[k].y * y[q].y + u[k].z * y[q].z + u[k].w * y[q].w;
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int i = i0 + tt * 4 + k;
+    if (i >= n) continue;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int l = l0 + tl + 16 * q;
+      if (l < m) G[(long long)i * lde + l] = acc[k][q] * E[(long long)i * lde + l] * inv_lambda;
+      else if (l < lde) G[(long long)i * lde + l] = 0.f;
+    }
+  }
+}
+
+// G = dK o K / lambda, elementwise (stand-alone l1_kernel_bwd)
+__global__ void k_g_elem(const float* __restrict__ Kmat, const float* __restrict__ dK, float* __restrict__ G,
+                         long long count, float inv_lambda) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) G[i] = dK[i] * Kmat[i] * inv_lambda;
+}
+
+// =====================================================================================
+// Sign pass over the landmarks (App. A):  out[i][c] = -sum_l G[i][l] * sign(tok[i][c] - L[l][c])
+// grid (ceil(n/64), BH); thread: 4 tokens x D/16 dims, token values held in registers
+// =====================================================================================
+template <typename TT, typename TL, typename TO, int D>
+__global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, const TL* __restrict__ Lm,
+                                                   const float* __restrict__ G, int ldg, TO* __restrict__ out,
+                                                   int n, int m) {
+  constexpr int DC = D / 16;
+  __shared__ __align__(16) float Ls[32][D + 4];
+  __shared__ __align__(16) float Gs[64][32 + 4];
+  const int i0 = blockIdx.x * 64, bh = blockIdx.y;
+  const int tid = threadIdx.x, tt = tid >> 4, tc = tid & 15;
+  tok += (long long)bh * n * D;
+  Lm += (long long)bh * m * D;
+  G += (long long)bh * n * ldg;
+  out += (long long)bh * n * D;
+  float q[4][DC], acc[4][DC];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int i = i0 + tt * 4 + k;
+#pragma unroll
+    for (int s = 0; s < DC; ++s) {
+      acc[k][s] = 0.f;
+      q[k][s] = (i < n) ? to_f(tok[(long long)i * D + ColMap<D>::col(tc, s)]) : 0.f;
+    }
+  }
+  for (int l0 = 0; l0 < m; l0 += 32) {
+    __syncthreads();
+    for (int idx = tid; idx < 32 * (D / 4); idx += 256) {
+      const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (l0 + r < m) v = ld4(Lm + (long long)(l0 + r) * D + c4);
+      *reinterpret_cast<float4*>(&Ls[r][c4]) = v;
+    }
+    {  // G tile: 64 tokens x 32 landmarks (zero outside)
+      const int r = tid >> 2, cb = (tid & 3) * 8, i = i0 + r;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int l = l0 + cb + k;
+        Gs[r][cb + k] = (i < n && l < m) ? G[(long long)i * ldg + l] : 0.f;
+      }
+    }
+    __syncthreads();
+#pragma unroll 2
+    for (int ll = 0; ll < 32; ll += 4) {
+      float g[4][4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float4 t = *reinterpret_cast<const float4*>(&Gs[tt * 4 + k][ll]);
+        g[k][0] = t.x; g[k][1] = t.y; g[k][2] = t.z; g[k][3] = t.w;
+      }
+#pragma unroll
+      for (int s = 0; s < 4; ++s) {
+        float lv[DC];
+        ld_cols<D>(&Ls[ll + s][0], tc, lv);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+#pragma unroll
+          for (int c = 0; c < DC; ++c) acc[k][c] += signed_g(q[k][c] - lv[c], g[k][s]);
+      }
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int i = i0 + tt * 4 + k;
+    if (i < n)
+#pragma unroll
+      for (int c = 0; c < DC; ++c) out[(long long)i * D + ColMap<D>::col(tc, c)] = from_f<TO>(-acc[k][c]);
+  }
+}
+
+// =====================================================================================
+// Sign pass over the tokens:  part[chunk][l][c] = +sum_{i in chunk} G[i][l] * sign(tok[i][c] - L[l][c])
+// grid (chunks, ceil(m/64), BH); thread: 4 landmarks x D/16 dims, landmark values in registers
+// =====================================================================================
+template <typename TT, typename TL, int D>
+__global__ void __launch_bounds__(256) k_sign_cols(const TT* __restrict__ tok, const TL* __restrict__ Lm,
+                                                   const float* __restrict__ G, int ldg, float* __restrict__ part,
+                                                   int n, int m, int rpc) {
+  constexpr int DC = D / 16;
+  __shared__ __align__(16) float Ts[32][D + 4];
+  __shared__ __align__(16) float Gs[32][64 + 4];
+  const int chunk = blockIdx.x, l0 = blockIdx.y * 64, bh = blockIdx.z, nchunks = gridDim.x;
+  const int tid = threadIdx.x, tl = tid >> 4, tc = tid & 15;
+  tok += (long long)bh * n * D;
+  Lm += (long long)bh * m * D;
+  G += (long long)bh * n * ldg;
+  const int ibeg = chunk * rpc, iend = min(n, ibeg + rpc);
+  float lv[4][DC], acc[4][DC];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int l = l0 + tl * 4 + k;
+#pragma unroll
+    for (int s = 0; s < DC; ++s) {
+      acc[k][s] = 0.f;
+      lv[k][s] = (l < m) ? to_f(Lm[(long long)l * D + ColMap<D>::col(tc, s)]) : 0.f;
+    }
+  }
+  for (int j0 = ibeg; j0 < iend; j0 += 32) {
+    __syncthreads();
+    for (int idx = tid; idx < 32 * (D / 4); idx += 256) {
+      const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (j0 + r < iend) v = ld4(tok + (long long)(j0 + r) * D + c4);
+      *reinterpret_cast<float4*>(&Ts[r][c4]) = v;
+    }
+    {  // G tile: 32 tokens x 64 landmarks (zero outside)
+      const int r = tid >> 3, cb = (tid & 7) * 8, i = j0 + r;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int l = l0 + cb + k;
+        Gs[r][cb + k] = (i < iend && l < m) ? G[(long long)i * ldg + l] : 0.f;
+      }
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int jj = 0; jj < 32; ++jj) {
+      const float4 g4 = *reinterpret_cast<const float4*>(&Gs[jj][tl * 4]);
+      const float g[4] = {g4.x, g4.y, g4.z, g4.w};
+      float tv[DC];
+      ld_cols<D>(&Ts[jj][0], tc, tv);
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int c = 0; c < DC; ++c) acc[k][c] += signed_g(tv[c] - lv[k][c], g[k]);
+    }
+  }
+  float* out = part + ((long long)bh * nchunks + chunk) * m * D;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int l = l0 + tl * 4 + k;
+    if (l < m)
+#pragma unroll
+      for (int c = 0; c < DC; ++c) out[(long long)l * D + ColMap<D>::col(tc, c)] = acc[k][c];
+  }
+}
+
+// =====================================================================================
+// Whole-CTA fp32 GEMM on global (L2-resident) row-major matrices:
+//   C = beta * Cin + alpha * op(A) op(B),  op(A) is M x K, op(B) is K x N.
+// Executed by all 256 threads of a CTA; ends with __syncthreads(), so a following call may
+// read C.  Cin may equal C (each element is read and written by the same thread).
+// =====================================================================================
+struct GemmSmem { float As[16][64 + 4]; float Bs[16][64 + 4]; };
+
+template <bool TRA, bool TRB>
+__device__ void cta_gemm(int M, int N, int K, const float* A, int lda, const float* Bm, int ldb,
+                         float* C, int ldc, float alpha, float beta, const float* Cin, GemmSmem& sm) {
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  for (int i0 = 0; i0 < M; i0 += 64)
+    for (int j0 = 0; j0 < N; j0 += 64) {
+      float acc[4][4];
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int s = 0; s < 4; ++s) acc[r][s] = 0.f;
+      for (int k0 = 0; k0 < K; k0 += 16) {
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int idx = tid + e * 256;   // 1024 elements per operand tile
+          if (TRA) {                       // op(A)(i,k) = A[k][i]: i fastest
+            const int kk = idx >> 6, i = idx & 63;
+            sm.As[kk][i] = (k0 + kk < K && i0 + i < M) ? A[(long long)(k0 + kk) * lda + i0 + i] : 0.f;
+          } else {                         // op(A)(i,k) = A[i][k]: k fastest
+            const int i = idx >> 4, kk = idx & 15;
+            sm.As[kk][i] = (k0 + kk < K && i0 + i < M) ? A[(long long)(i0 + i) * lda + k0 + kk] : 0.f;
+          }
+          if (TRB) {                       // op(B)(k,j) = B[j][k]: k fastest
+            const int j = idx >> 4, kk = idx & 15;
+            sm.Bs[kk][j] = (k0 + kk < K && j0 + j < N) ? Bm[(long long)(j0 + j) * ldb + k0 + kk] : 0.f;
+          } else {                         // op(B)(k,j) = B[k][j]: j fastest
+            const int kk = idx >> 6, j = idx & 63;
+            sm.Bs[kk][j] = (k0 + kk < K && j0 + j < N) ? Bm[(long long)(k0 + kk) * ldb + j0 + j] : 0.f;
+          }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) {
+          const float4 a = *reinterpret_cast<const float4*>(&sm.As[kk][ty * 4]);
+          const float4 b = *reinterpret_cast<const float4*>(&sm.Bs[kk][tx * 4]);
+          const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+          for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int s = 0; s < 4; ++s) acc[r][s] = fmaf(av[r], bv[s], acc[r][s]);
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int i = i0 + ty * 4 + r;
+        if (i >= M) continue;
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+          const int j = j0 + tx * 4 + s;
+          if (j >= N) continue;
+          float v = alpha * acc[r][s];
+          if (beta != 0.f) v += beta * Cin[(long long)i * ldc + j];
+          C[(long long)i * ldc + j] = v;
+        }
+      }
+    }
+  __syncthreads();
+}
+
+// Block-wide sum of one float per thread (256 threads); result valid in every thread.
+__device__ inline float block_sum(float v, float* red /* >= 8 floats of shared memory */) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float s = 0.f;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w];
+  __syncthreads();
+  return s;
+}
+
+// Header kept per matrix beside the Newton-Schulz iterates.
+struct NsHdr { float alpha, n1, ninf; int jstar, istar, auto_alpha, pad0, pad1; };
+
+// =====================================================================================
+// Newton-Schulz forward for one m x m matrix (Alg. 2), whole CTA.
+//   Wr <- W + eps I;  alpha = 1/(||Wr||_1 ||Wr||_inf) unless given;  X_0 = alpha Wr^T;
+//   X_{k+1} = X_k (2I - Wr X_k);  Xh[k] = X_k for k = 0..T.
+// W, Wr, P: [m][m] in global memory; Xh: [T+1][m][m].
+// =====================================================================================
+__device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const float* W, float* Wr, float* P,
+                               float* Xh, NsHdr* hdr, GemmSmem& sm, float* red /* 2*256 + 8 floats */) {
+  const int tid = threadIdx.x;
+  const long long mm = (long long)m * m;
+  for (long long e = tid; e < mm; e += 256) {
+    const int i = (int)(e / m), j = (int)(e % m);
+    Wr[e] = W[e] + (i == j ? eps : 0.f);
+  }
+  __syncthreads();
+  float* colsum = red;          // [256]
+  float* rowsum = red + 256;    // [256]
+  if (tid < m) {
+    float cs = 0.f, rs = 0.f;
+    for (int i = 0; i < m; ++i) { cs += fabsf(Wr[(long long)i * m + tid]); rs += fabsf(Wr[(long long)tid * m + i]); }
+    colsum[tid] = cs; rowsum[tid] = rs;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    float n1 = -1.f, ninf = -1.f; int js = 0, is = 0;
+    for (int t = 0; t < m; ++t) {                 // strict > keeps the lowest index on ties
+      if (colsum[t] > n1) { n1 = colsum[t]; js = t; }
+      if (rowsum[t] > ninf) { ninf = rowsum[t]; is = t; }
+    }
+    hdr->n1 = n1; hdr->ninf = ninf; hdr->jstar = js; hdr->istar = is;
+    hdr->auto_alpha = !(alpha_in > 0.f);
+    hdr->alpha = (alpha_in > 0.f) ? alpha_in : 1.f / (n1 * ninf);
+    hdr->pad0 = hdr->pad1 = 0;
+  }
+  __syncthreads();
+  const float alpha = hdr->alpha;
+  for (long long e = tid; e < mm; e += 256) {
+    const int i = (int)(e / m), j = (int)(e % m);
+    Xh[e] = alpha * Wr[(long long)j * m + i];
+  }
+  __syncthreads();
+  for (int k = 0; k < T; ++k) {
+    const float* X = Xh + (long long)k * mm;
+    float* Xn = Xh + (long long)(k + 1) * mm;
+    cta_gemm<false, false>(m, m, m, Wr, m, X, m, P, m, -1.f, 0.f, nullptr, sm);   // P = -Wr X_k
+    for (int i = tid; i < m; i += 256) P[(long long)i * m + i] += 2.f;             // 2I - Wr X_k
+    __syncthreads();
+    cta_gemm<false, false>(m, m, m, X, m, P, m, Xn, m, 1.f, 0.f, nullptr, sm);     // X_{k+1}
+  }
+}
+
+// =====================================================================================
+// Exact adjoint of ns_forward_dev: given G0 = dLoss/dX_T returns dW = dLoss/dW.
+// Scratch matrices [m][m]: P, Hm, Ga, Gb.  Xh holds X_0..X_T, Wr = W + eps I, hdr from the forward.
+// =====================================================================================
+__device__ void ns_backward_dev(int m, int T, const float* Wr, const float* Xh, const NsHdr* hdr,
+                                const float* G0, float* dW, float* P, float* Hm, float* Ga, float* Gb,
+                                GemmSmem& sm, float* red) {
+  const int tid = threadIdx.x;
+  const long long mm = (long long)m * m;
+  for (long long e = tid; e < mm; e += 256) { Ga[e] = G0[e]; dW[e] = 0.f; }
+  __syncthreads();
+  float* G = Ga; float* Gn = Gb;
+  for (int k = T - 1; k >= 0; --k) {
+    const float* A = Xh + (long long)k * mm;                                        // X_{k+1} = 2A - A P, P = Wr A
+    cta_gemm<false, false>(m, m, m, Wr, m, A, m, P, m, 1.f, 0.f, nullptr, sm);      // P = Wr A
+    cta_gemm<true, false>(m, m, m, A, m, G, m, Hm, m, 1.f, 0.f, nullptr, sm);       // H = A^T G
+    cta_gemm<false, true>(m, m, m, Hm, m, A, m, dW, m, -1.f, 1.f, dW, sm);          // dW -= H A^T
+    cta_gemm<false, true>(m, m, m, G, m, P, m, Gn, m, -1.f, 2.f, G, sm);            // Gn = 2G - G P^T
+    cta_gemm<true, false>(m, m, m, Wr, m, Hm, m, Gn, m, -1.f, 1.f, Gn, sm);         // Gn -= Wr^T H
+    float* t = G; G = Gn; Gn = t;
+  }
+  // X_0 = alpha Wr^T
+  const float alpha = hdr->alpha;
+  float part = 0.f;
+  for (long long e = tid; e < mm; e += 256) {
+    const int i = (int)(e / m), j = (int)(e % m);
+    part += G[e] * Wr[(long long)j * m + i];
+  }
+  const float dalpha = block_sum(part, red);
+  for (long long e = tid; e < mm; e += 256) {
+    const int j = (int)(e / m), i = (int)(e % m);      // dW[j][i] += alpha G[i][j]
+    dW[e] += alpha * G[(long long)i * m + j];
+  }
+  __syncthreads();
+  if (hdr->auto_alpha) {
+    const int js = hdr->jstar, is = hdr->istar;
+    const float c1 = dalpha * (-alpha / hdr->n1), c2 = dalpha * (-alpha / hdr->ninf);
+    for (int i = tid; i < m; i += 256) {
+      const float w = Wr[(long long)i * m + js];
+      dW[(long long)i * m + js] += c1 * (w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f));
+    }
+    __syncthreads();
+    for (int j = tid; j < m; j += 256) {
+      const float w = Wr[(long long)is * m + j];
+      dW[(long long)is * m + j] += c2 * (w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f));
+    }
+    __syncthreads();
+  }
+}
+
+// ------------------------------------------------------------------ stand-alone ns_pinv / ns_pinv_bwd
+__global__ void __launch_bounds__(256) k_ns_pinv(int m, int T, float eps, float alpha_in, const float* W,
+                                                 float* Wr, float* P, float* Xh, NsHdr* hdr, float* X,
+                                                 float* resid) {
+  __shared__ GemmSmem sm;
+  __shared__ float red[2 * 256 + 8];
+  const int b = blockIdx.x;
+  const long long mm = (long long)m * m;
+  W += b * mm; Wr += b * mm; P += b * mm; Xh += (long long)b * (T + 1) * mm; hdr += b;
+  ns_forward_dev(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red);
+  const float* XT = Xh + (long long)T * mm;
+  if (X) for (long long e = threadIdx.x; e < mm; e += 256) X[b * mm + e] = XT[e];
+  if (resid) {
+    cta_gemm<false, false>(m, m, m, Wr, m, XT, m, P, m, 1.f, 0.f, nullptr, sm);
+    float part = 0.f;
+    for (long long e = threadIdx.x; e < mm; e += 256) {
+      const int i = (int)(e / m), j = (int)(e % m);
+      const float r = (i == j ? 1.f : 0.f) - P[e];
+      part += r * r;
+    }
+    const float s = block_sum(part, red);
+    if (threadIdx.x == 0) resid[b] = sqrtf(s);
+  }
+}
+
+// recompute != 0: run the forward first (Xh, hdr, Wr are scratch); else Xh is the caller's history
+// and only Wr / hdr are rebuilt from W.
+__global__ void __launch_bounds__(256) k_ns_pinv_bwd(int m, int T, float eps, float alpha_in, const float* W,
+                                                     float* Wr, float* P, float* Hm, float* Ga, float* Gb,
+                                                     float* Xh_scratch, const float* Xh_given, NsHdr* hdr,
+                                                     const float* dX, float* dW) {
+  __shared__ GemmSmem sm;
+  __shared__ float red[2 * 256 + 8];
+  const int b = blockIdx.x;
+  const long long mm = (long long)m * m;
+  W += b * mm; Wr += b * mm; P += b * mm; Hm += b * mm; Ga += b * mm; Gb += b * mm; hdr += b;
+  float* Xs = Xh_scratch + (long long)b * (T + 1) * mm;
+  // T = 0 when the history is given: only Wr, the norms and alpha are rebuilt
+  ns_forward_dev(m, Xh_given ? 0 : T, eps, alpha_in, W, Wr, P, Xs, hdr, sm, red);
+  const float* Xh = Xh_given ? Xh_given + (long long)b * (T + 1) * mm : Xs;
+  ns_backward_dev(m, T, Wr, Xh, hdr, dX + b * mm, dW + b * mm, P, Hm, Ga, Gb, sm, red);
+}
+
+// =====================================================================================
+// Per-head middle of the forward pass: reduce M over the token chunks, Newton-Schulz, Y = X M,
+// then fold the injective map (Prop. 3) into Ytilde_l = s_l Y_l - mean_l'(s_l' Y_l'), ybar = mean_l Y_l
+// so that O = (C - mu) Ytilde + ybar.  One CTA per head.
+// =====================================================================================
+template <int D>
+__global__ void __launch_bounds__(256) k_mid_fwd(int m, int T, float eps, float alpha_in, int H, int map_mode,
+                                                 const float* __restrict__ whiten, const float* W, float* Wr,
+                                                 float* P, float* Xh, NsHdr* hdr, const float* Mpart, int nchunks,
+                                                 float* Mout, float* Y, float* Yt, float* ybar, int* dev_status) {
+  __shared__ GemmSmem sm;
+  __shared__ float red[2 * 256 + 8];
+  const int bh = blockIdx.x, tid = threadIdx.x;
+  const long long mm = (long long)m * m, md = (long long)m * D;
+  W += bh * mm; Wr += bh * mm; P += bh * mm; Xh += (long long)bh * (T + 1) * mm; hdr += bh;
+  Mout += bh * md; Y += bh * md; Yt += bh * md; ybar += (long long)bh * D;
+  Mpart += (long long)bh * nchunks * md;
+  for (long long e = tid; e < md; e += 256) {
+    float s = 0.f;
+    for (int p = 0; p < nchunks; ++p) s += Mpart[p * md + e];
+    Mout[e] = s;
+  }
+  ns_forward_dev(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red);
+  const float* XT = Xh + (long long)T * mm;
+  if (dev_status) {
+    float bad = 0.f;
+    for (long long e = tid; e < mm; e += 256) bad += isfinite(XT[e]) ? 0.f : 1.f;
+    bad = block_sum(bad, red);
+    if (tid == 0) dev_status[bh] = bad > 0.f ? 1 : 0;
+  }
+  cta_gemm<false, false>(m, D, m, XT, m, Mout, D, Y, D, 1.f, 0.f, nullptr, sm);      // Y = X M
+  const float* s = whiten ? whiten + (long long)(bh % H) * m : nullptr;
+  if (tid < D) {
+    const int c = tid;
+    if (map_mode == 1) {
+      float sy = 0.f, y1 = 0.f;
+      for (int l = 0; l < m; ++l) { const float y = Y[(long long)l * D + c]; sy += (s ? s[l] : 1.f) * y; y1 += y; }
+      sy /= (float)m;
+      for (int l = 0; l < m; ++l) Yt[(long long)l * D + c] = (s ? s[l] : 1.f) * Y[(long long)l * D + c] - sy;
+      ybar[c] = y1 / (float)m;
+    } else {
+      for (int l = 0; l < m; ++l) Yt[(long long)l * D + c] = Y[(long long)l * D + c];
+      ybar[c] = 0.f;
+    }
+  }
+}
+
+// =====================================================================================
+// Per-head middle of the backward pass.  Inputs: partial sums of Z'^T dO and of the column sums
+// of dO over the token chunks; the forward context.  Outputs: dM (for dR = dM V^T, dV = R^T dM)
+// and GW = (dW o K_LL + (dW o K_LL)^T) / lambda, the symmetrised upstream of the landmark block,
+// so that dL_l -= sum_l' GW[l][l'] sign(L_l - L_l').
+// =====================================================================================
+template <int D>
+__global__ void __launch_bounds__(256) k_mid_bwd(int m, int T, int H, int map_mode, float inv_lambda, int ldm,
+                                                 const float* __restrict__ whiten, const float* W,
+                                                 const float* Xh, const NsHdr* hdr, const float* Msaved,
+                                                 const float* dYtpart, const float* dybpart, int nchunks,
+                                                 float eps, float* Wr, float* P, float* Hm, float* Ga, float* Gb,
+                                                 float* dWm, float* dXm, float* dY, float* dM, float* GW) {
+  __shared__ GemmSmem sm;
+  __shared__ float red[2 * 256 + 8];
+  const int bh = blockIdx.x, tid = threadIdx.x;
+  const long long mm = (long long)m * m, md = (long long)m * D;
+  W += bh * mm; Xh += (long long)bh * (T + 1) * mm; hdr += bh; Msaved += bh * md;
+  Wr += bh * mm; P += bh * mm; Hm += bh * mm; Ga += bh * mm; Gb += bh * mm; dWm += bh * mm; dXm += bh * mm;
+  dY += bh * md; dM += bh * md; GW += (long long)bh * m * ldm;
+  dYtpart += (long long)bh * nchunks * md; dybpart += (long long)bh * nchunks * D;
+  const float* s = whiten ? whiten + (long long)(bh % H) * m : nullptr;
+  float* dyb = red;   // [D] column sums of dO
+  if (tid < D) {
+    float t = 0.f;
+    for (int p = 0; p < nchunks; ++p) t += dybpart[(long long)p * D + tid];
+    dyb[tid] = t;
+  }
+  __syncthreads();
+  for (long long e = tid; e < md; e += 256) {
+    float t = 0.f;
+    for (int p = 0; p < nchunks; ++p) t += dYtpart[p * md + e];
+    const int l = (int)(e / D), c = (int)(e % D);
+    // Ytilde = P_c diag(s) Y, ybar = Y^T 1/m  ->  dY = diag(s) (centred Z'^T dO) + (1/m) 1 dyb^T
+    dY[e] = (map_mode == 1) ? (s ? s[l] : 1.f) * t + dyb[c] / (float)m : t;
+  }
+  for (long long e = tid; e < mm; e += 256) {
+    const int i = (int)(e / m), j = (int)(e % m);
+    Wr[e] = W[e] + (i == j ? eps : 0.f);
+  }
+  __syncthreads();
+  const float* XT = Xh + (long long)T * mm;
+  cta_gemm<false, true>(m, m, D, dY, D, Msaved, D, dXm, m, 1.f, 0.f, nullptr, sm);   // dX = dY M^T
+  cta_gemm<true, false>(m, D, m, XT, m, dY, D, dM, D, 1.f, 0.f, nullptr, sm);        // dM = X^T dY
+  ns_backward_dev(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red);
+  for (long long e = tid; e < (long long)m * ldm; e += 256) {
+    const int i = (int)(e / ldm), j = (int)(e % ldm);
+    float v = 0.f;
+    if (j < m) v = (dWm[(long long)i * m + j] * W[(long long)i * m + j] + dWm[(long long)j * m + i] * W[(long long)j * m + i]) * inv_lambda;
+    GW[e] = v;
+  }
+}
+
+}  // namespace ln

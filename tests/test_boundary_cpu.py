@@ -1,0 +1,112 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, sizes are sane, and argument errors are reported before anything is launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2604_20368_b200 as ln
+from paper_2604_20368_b200 import binding, synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "laplace_nystrom.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"\b(?:int|size_t|const char\*)\s+(\w+)\s*\(", text)
+    return sorted(set(names))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = binding.lib()
+    syms = declared_symbols()
+    assert set(syms) == set(binding.EXPORTS)
+    for s in syms:
+        assert hasattr(lib, s), s
+    assert lib.ln_status_string(0) == b"ok"
+    assert lib.ln_status_string(-3) == b"workspace too small"
+
+
+def _problem(**kw):
+    cfg = synth.CONFIGS["cfg2"]
+    p = ln.problem_from_config(cfg)
+    for k, v in kw.items():
+        setattr(p, k, v)
+    return p
+
+
+def test_sizes_positive_and_monotone():
+    p = _problem()
+    sb = ln.laplace_nystrom_saved_bytes(p)
+    assert sb > 0
+    assert ln.laplace_nystrom_workspace_bytes(p, True) > 0
+    assert ln.laplace_nystrom_workspace_bytes(p, False) >= sb
+    assert ln.laplace_nystrom_saved_bytes(_problem(B=128)) > sb
+    assert binding.lib().ns_pinv_workspace_bytes(4, 64, 6) > 0
+    assert binding.lib().ns_pinv_workspace_bytes(0, 64, 6) == 0
+    assert binding.lib().l1_kernel_bwd_workspace_bytes(2, 100, 30, 64) > 0
+
+
+@pytest.mark.parametrize("kw", [
+    dict(lam=0.0), dict(lam=float("nan")), dict(ns_iters=-1), dict(ridge_eps=-1.0), dict(m=500),
+    dict(n=196), dict(mh=6), dict(dtype=7), dict(map_mode=2), dict(B=0), dict(gh=0),
+])
+def test_invalid_problem_is_rejected_on_the_host(kw):
+    p = _problem(**kw)
+    assert ln.laplace_nystrom_saved_bytes(p) == 0
+    cp = p.c()
+    fake = ctypes.c_void_p(4096)   # never dereferenced: validation fails first
+    st = binding.lib().laplace_nystrom_fwd(ctypes.byref(cp), fake, fake, fake, None, fake, None, fake, 1 << 40,
+                                          None, None)
+    assert st in (-1, -2)
+
+
+def test_unsupported_envelope_and_null_and_workspace():
+    lib = binding.lib()
+    fake = ctypes.c_void_p(4096)
+    cp = _problem(d=48).c()
+    assert lib.laplace_nystrom_fwd(ctypes.byref(cp), fake, fake, fake, None, fake, None, fake, 1 << 40, None, None) == -2
+    cp = _problem().c()
+    assert lib.laplace_nystrom_fwd(ctypes.byref(cp), None, fake, fake, None, fake, None, fake, 1 << 40, None, None) == -1
+    assert lib.laplace_nystrom_fwd(ctypes.byref(cp), fake, fake, fake, None, fake, None, fake, 16, None, None) == -3
+    # lm_mode 1 forbids a landmark tensor, misaligned pointers are refused
+    assert lib.laplace_nystrom_fwd(ctypes.byref(cp), fake, fake, fake, fake, fake, None, fake, 1 << 40, None, None) == -1
+    odd = ctypes.c_void_p(4100)
+    assert lib.laplace_nystrom_fwd(ctypes.byref(cp), odd, fake, fake, None, fake, None, fake, 1 << 40, None, None) == -1
+    assert lib.ns_pinv(1, 300, fake, 2, 0.0, 0.0, fake, None, None, fake, 1 << 40, None) == -2
+    assert lib.ns_pinv(1, 8, fake, 2, 0.0, 0.0, fake, None, None, fake, 8, None) == -3
+    assert lib.l1_kernel(1, 4, 4, 0, fake, fake, 0, 1.0, fake, None, None) == -1
+    assert lib.l1_kernel_bwd(1, 4, 4, 48, fake, fake, 0, 1.0, None, fake, fake, fake, fake, 1 << 40, None) == -2
+
+
+def test_binding_refuses_cpu_tensors():
+    import torch
+    with pytest.raises(ValueError):
+        ln.l1_kernel(torch.zeros(1, 4, 8), torch.zeros(1, 4, 8), 1.0)
+
+
+def test_config_table_matches_the_workloads():
+    c = synth.CONFIGS
+    assert (c["cfg1"].n, c["cfg1"].m, c["cfg1"].dtype, c["cfg1"].backward) == (196, 32, "f32", False)
+    assert (c["cfg2"].n, c["cfg2"].m, c["cfg2"].B * c["cfg2"].H) == (197, 49, 384)
+    assert (c["cfg3"].n, c["cfg3"].m) == (3136, 64)
+    assert [c[k].n for k in ("cfg4a", "cfg4b", "cfg4c")] == [3136, 12544, 50176]
+    assert c["cfg5_m256_T12"].n == 4096 and c["cfg5_m256_T12"].d == 128
+    for cfg in c.values():
+        assert cfg.mh * cfg.mw == cfg.m and cfg.lam == cfg.d
+
+
+def test_generator_is_seeded_and_duplicates_bins():
+    import torch
+    cfg = synth.shrink(synth.CONFIGS["cfg5_m64_T4"], B=1, H=2)
+    a, b = synth.make_inputs(cfg), synth.make_inputs(cfg)
+    for k in a:
+        assert torch.equal(a[k], b[k])
+    assert a["Q"].dtype == torch.bfloat16 and a["whiten"].shape == (2, 64)
+    # about 10 % of the keys are copies: count rows that occur more than once
+    K = a["K"][0, 0].to(torch.float32)
+    uniq = torch.unique(K, dim=0).shape[0]
+    ndup_tokens = K.shape[0] - uniq
+    assert ndup_tokens == 7 * 64          # ceil(0.1*64) = 7 bins of 8x8 tokens

@@ -1,0 +1,240 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the float64 oracle on the same
+seeded inputs, element by element.  Tolerances are norm-wise relative errors: 1e-4 for fp32
+storage, 2e-2 for bf16 storage (outputs and gradients alike)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2604_20368_b200 as ln
+from paper_2604_20368_b200 import synth
+from parity import TOL, compare, f64, rel_err, run_gpu, run_oracle_heads
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _rand(shape, seed, dtype):
+    x = torch.from_numpy(np.random.default_rng(seed).standard_normal(shape, dtype=np.float32))
+    return x.to(dtype)
+
+
+# ------------------------------------------------------------------------------------------ l1_kernel
+@pytest.mark.parametrize("batch,na,nb,d", [(3, 197, 49, 64), (1, 1, 1, 1), (2, 130, 131, 7), (1, 300, 70, 128),
+                                           (2, 64, 256, 32), (1, 129, 65, 40)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_l1_kernel(batch, na, nb, d, dtype):
+    A, Bm = _rand((batch, na, d), 1, dtype), _rand((batch, nb, d), 2, dtype)
+    lam = float(max(d, 2))
+    K, rs = ln.l1_kernel(A.to(DEV), Bm.to(DEV), lam, want_rowsum=True)
+    Ko, rso = oracle.l1_kernel(f64(A), f64(Bm), lam, want_rowsum=True)
+    assert rel_err(f64(K), Ko) < 2e-6
+    assert np.abs(f64(K) - Ko).max() < 4e-6
+    assert rel_err(f64(rs), rso) < 2e-6
+
+
+def test_l1_kernel_exact_properties():
+    A = _rand((2, 90, 64), 3, torch.float32).to(DEV)
+    K = ln.l1_kernel(A, A, 64.0)
+    assert torch.equal(K, K.transpose(1, 2))                      # |a-b| = |b-a| in the same order
+    assert torch.equal(torch.diagonal(K, dim1=1, dim2=2), torch.ones(2, 90, device=DEV))
+
+
+@pytest.mark.parametrize("batch,na,nb,d", [(2, 197, 49, 64), (1, 70, 130, 32), (1, 33, 5, 128), (3, 1, 1, 32)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("recompute", [False, True])
+def test_l1_kernel_bwd(batch, na, nb, d, dtype, recompute):
+    A, Bm = _rand((batch, na, d), 4, dtype), _rand((batch, nb, d), 5, dtype)
+    if na > 4 and nb > 2:                 # exact ties: sign(0) = 0 on both sides
+        A[0, 3] = Bm[0, 1]
+        A[0, 4, : d // 2] = Bm[0, 2, : d // 2]
+    dK = _rand((batch, na, nb), 6, torch.float32)
+    lam = float(d)
+    Kmat = None if recompute else ln.l1_kernel(A.to(DEV), Bm.to(DEV), lam)
+    dA, dB = ln.l1_kernel_bwd(A.to(DEV), Bm.to(DEV), lam, dK.to(DEV), Kmat=Kmat)
+    dAo, dBo = oracle.l1_kernel_bwd(f64(A), f64(Bm), lam, f64(dK))
+    tol = 1e-5 if dtype == torch.float32 else 5e-3    # bf16: only the output rounding
+    assert rel_err(f64(dA), dAo) < tol
+    assert rel_err(f64(dB), dBo) < tol
+
+
+# ------------------------------------------------------------------------------------------ ns_pinv
+def _kernel_matrices(batch, m, d, seed):
+    pts = np.random.default_rng(seed).standard_normal((batch, m, d))
+    return oracle.l1_kernel(pts, pts, float(d)).astype(np.float32)
+
+
+@pytest.mark.parametrize("m,T", [(1, 0), (1, 3), (5, 4), (49, 6), (64, 8), (130, 8), (256, 12), (32, 0)])
+def test_ns_pinv(m, T):
+    W = _kernel_matrices(3, m, 16, 7)
+    X, hist, resid = ln.ns_pinv(torch.from_numpy(W).to(DEV), T, ridge_eps=1e-6, want_hist=True, want_resid=True)
+    Xo, resido, alphao, histo = oracle.ns_pinv(W, T, eps=float(np.float32(1e-6)), want_hist=True)
+    assert rel_err(f64(X), Xo) < 2e-5
+    if T > 0:
+        assert rel_err(f64(hist)[:, :T], histo) < 2e-5
+    assert rel_err(f64(hist)[:, T], Xo) < 2e-5
+    assert np.allclose(f64(resid), resido, rtol=1e-3, atol=1e-4)
+
+
+def test_ns_pinv_converges_and_given_alpha():
+    W = _kernel_matrices(2, 24, 8, 8)
+    X, _, resid = ln.ns_pinv(torch.from_numpy(W).to(DEV), 40, ridge_eps=0.0, want_resid=True)
+    eye = np.eye(24)
+    for b in range(2):
+        assert np.abs(f64(X)[b] @ W[b].astype(np.float64) - eye).max() < 5e-3   # fp32 limit at cond ~ 1e2
+    Xa, _, _ = ln.ns_pinv(torch.from_numpy(W).to(DEV), 3, alpha=0.01)
+    Xo, _, _ = oracle.ns_pinv(W, 3, alpha=float(np.float32(0.01)))
+    assert rel_err(f64(Xa), Xo) < 2e-5
+
+
+@pytest.mark.parametrize("m,T", [(1, 2), (5, 4), (49, 6), (64, 8), (130, 4), (256, 4), (16, 0)])
+@pytest.mark.parametrize("given_hist", [False, True])
+def test_ns_pinv_bwd(m, T, given_hist):
+    W = _kernel_matrices(2, m, 16, 9)
+    dX = np.random.default_rng(10).standard_normal((2, m, m)).astype(np.float32)
+    Wd = torch.from_numpy(W).to(DEV)
+    hist = ln.ns_pinv(Wd, T, ridge_eps=1e-6, want_hist=True)[1] if given_hist else None
+    dW = ln.ns_pinv_bwd(Wd, T, 1e-6, 0.0, torch.from_numpy(dX).to(DEV), X_hist=hist)
+    dWo = oracle.ns_pinv_bwd(W, T, float(np.float32(1e-6)), 0.0, dX)
+    assert rel_err(f64(dW), dWo) < 1e-4
+    dWa = ln.ns_pinv_bwd(Wd, T, 1e-6, 0.02, torch.from_numpy(dX).to(DEV))
+    dWao = oracle.ns_pinv_bwd(W, T, float(np.float32(1e-6)), float(np.float32(0.02)), dX)
+    assert rel_err(f64(dWa), dWao) < 1e-4
+
+
+# ------------------------------------------------------------------------------------------ pooling
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg4a"])
+def test_landmarks_pool_fwd_bwd(name):
+    cfg = synth.shrink(synth.CONFIGS[name], B=1, H=2)
+    inp = synth.make_inputs(cfg)
+    p = ln.problem_from_config(cfg)
+    op = oracle.Problem(B=1, H=2, n=cfg.n, d=cfg.d, m=cfg.m, lam=cfg.lam, ns_iters=0, prefix=cfg.prefix,
+                        gh=cfg.gh, gw=cfg.gw, mh=cfg.mh, mw=cfg.mw)
+    L = ln.landmarks_pool(p, inp["K"].to(DEV))
+    Lo = oracle.landmarks_pool(op, f64(inp["K"]))
+    assert rel_err(f64(L), Lo) < 1e-6
+    dL = torch.from_numpy(np.random.default_rng(11).standard_normal((1, 2, cfg.m, cfg.d), dtype=np.float32))
+    dK = ln.landmarks_pool_bwd(p, dL.to(DEV))
+    dKo = oracle.landmarks_pool_bwd(op, f64(dL))
+    assert rel_err(f64(dK), dKo) < (1e-6 if cfg.dtype == "f32" else 4e-3)
+
+
+# ------------------------------------------------------------------------------------------ whole path
+def _run_case(cfg, use_whiten=True, map_mode=1, backward=True, heads=None, tol=None):
+    inp = synth.make_inputs(cfg)
+    heads = list(range(cfg.B * cfg.H)) if heads is None else heads
+    g = run_gpu(cfg, inp, use_whiten=use_whiten, map_mode=map_mode, backward=backward)
+    assert int(g["status"].abs().max()) == 0
+    o = run_oracle_heads(cfg, inp, heads, use_whiten=use_whiten, map_mode=map_mode, backward=backward)
+    errs = compare(cfg, g, o, heads)
+    tol = TOL[cfg.dtype] if tol is None else tol
+    for k, e in errs.items():
+        assert e < tol, (cfg.name, k, e, errs)
+    return errs
+
+
+def test_cfg1_tiny_fp32_forward():
+    _run_case(synth.CONFIGS["cfg1"], backward=False)
+
+
+def test_cfg1_fp32_forward_and_backward():
+    from dataclasses import replace
+    _run_case(replace(synth.CONFIGS["cfg1"], backward=True))
+
+
+@pytest.mark.parametrize("use_whiten,map_mode", [(True, 1), (False, 1), (False, 0)])
+def test_cfg2_shape_small_batch(use_whiten, map_mode):
+    _run_case(synth.shrink(synth.CONFIGS["cfg2"], B=2), use_whiten=use_whiten, map_mode=map_mode)
+
+
+def test_cfg2_shape_fp32_storage():
+    from dataclasses import replace
+    _run_case(replace(synth.shrink(synth.CONFIGS["cfg2"], B=1), dtype="f32"))
+
+
+def test_cfg3_shape_small_batch():
+    _run_case(synth.shrink(synth.CONFIGS["cfg3"], B=2))
+
+
+def test_cfg4a_shape_small_batch():
+    _run_case(synth.shrink(synth.CONFIGS["cfg4a"], B=1))
+
+
+@pytest.mark.parametrize("name", ["cfg5_m64_T4", "cfg5_m128_T8", "cfg5_m256_T12"])
+def test_cfg5_shape_small_batch(name):
+    _run_case(synth.shrink(synth.CONFIGS[name], B=1, H=2))
+
+
+def test_cfg2_full_size_sampled_heads():
+    cfg = synth.CONFIGS["cfg2"]
+    heads = [0, 1, 5, 6, 100, 191, 192, 300, 382, 383]
+    _run_case(cfg, heads=heads)
+
+
+def test_cfg3_full_size_sampled_heads():
+    cfg = synth.CONFIGS["cfg3"]
+    _run_case(cfg, heads=[0, 13, 31])
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_given_landmarks_and_their_gradient(dtype):
+    # lm_mode 0: caller-provided landmarks, dL returned
+    rng = np.random.default_rng(21)
+    B, H, n, d, m, T = 1, 2, 150, 32, 20, 5
+    td = torch.float32 if dtype == "f32" else torch.bfloat16
+    Q, K, V, dO = (torch.from_numpy(rng.standard_normal((B, H, n, d), dtype=np.float32)).to(td) for _ in range(4))
+    L = torch.from_numpy(rng.standard_normal((B, H, m, d), dtype=np.float32)).to(td)
+    wh = torch.from_numpy(rng.uniform(0.5, 2.0, (H, m)).astype(np.float32))
+    p = ln.Problem(B=B, H=H, n=n, d=d, m=m, lam=float(d), ns_iters=T, dtype=ln.LN_F32 if dtype == "f32" else ln.LN_BF16,
+                   whiten=wh.to(DEV), lm_mode=0)
+    saved = torch.empty(ln.laplace_nystrom_saved_bytes(p), dtype=torch.uint8, device=DEV)
+    args = [t.to(DEV) for t in (Q, K, V)]
+    O = ln.laplace_nystrom_fwd(p, *args, L=L.to(DEV), saved=saved)
+    dQ, dK, dV, dL = ln.laplace_nystrom_bwd(p, *args, dO.to(DEV), saved, L=L.to(DEV))
+    op = oracle.Problem(B=B, H=H, n=n, d=d, m=m, lam=float(d), ns_iters=T, ridge_eps=float(np.float32(1e-6)), lm_mode=0)
+    Oo = oracle.forward(op, f64(Q), f64(K), f64(V), L=f64(L), whiten=f64(wh))
+    dQo, dKo, dVo, dLo = oracle.backward(op, f64(Q), f64(K), f64(V), f64(dO), L=f64(L), whiten=f64(wh))
+    for name, got, ref in (("O", O, Oo), ("dQ", dQ, dQo), ("dK", dK, dKo), ("dV", dV, dVo), ("dL", dL, dLo)):
+        assert rel_err(f64(got), ref) < TOL[dtype], name
+
+
+def test_inference_without_saved_matches_training_forward():
+    cfg = synth.shrink(synth.CONFIGS["cfg2"], B=1)
+    inp = synth.make_inputs(cfg)
+    a = run_gpu(cfg, inp, backward=False)["O"]
+    b = run_gpu(cfg, inp, backward=True)["O"]
+    assert torch.equal(a, b)
+
+
+def test_m_equals_n_reproduces_exact_attention_on_gpu():
+    # landmarks = keys (bins == grid), many Newton-Schulz steps: Nystrom is exact (oracle pin, here on GPU)
+    cfg = synth.Config("mn", B=1, H=2, d=32, m=48, T=40, gh=6, gw=8, mh=6, mw=8, dtype="f32", seed=5,
+                       ridge_eps=0.0)
+    inp = synth.make_inputs(cfg)
+    g = run_gpu(cfg, inp, backward=False)
+    Q, K, V = (f64(inp[k])[0] for k in ("Q", "K", "V"))
+    s = f64(inp["whiten"])
+    for h in range(2):
+        G = np.exp(-np.abs(Q[h][:, None, :] - K[h][None, :, :]).sum(-1) / cfg.lam)
+        Z = (G - G.mean(1, keepdims=True)) * s[h][None, :] + 1.0 / cfg.n
+        assert rel_err(f64(g["O"])[0, h], Z @ V[h]) < 2e-3      # fp32 inverse of a cond ~ 1e2 matrix
+
+
+def test_runs_twice_bit_identical():
+    cfg = synth.shrink(synth.CONFIGS["cfg3"], B=1)
+    inp = synth.make_inputs(cfg)
+    a, b = run_gpu(cfg, inp), run_gpu(cfg, inp)
+    for k in ("O", "dQ", "dK", "dV"):
+        assert torch.equal(a[k], b[k]), k
+
+
+def test_singular_landmarks_are_flagged_finite():
+    # all keys identical -> K_LL is all ones; the ridge keeps Newton-Schulz finite
+    cfg = synth.shrink(synth.CONFIGS["cfg1"], H=1)
+    inp = synth.make_inputs(cfg)
+    inp["K"][:] = inp["K"][0, 0, 0]
+    g = run_gpu(cfg, inp, backward=False)
+    assert int(g["status"].abs().max()) == 0
+    assert torch.isfinite(g["O"]).all()
+    o = run_oracle_heads(cfg, inp, [0], backward=False)
+    assert rel_err(f64(g["O"])[0, 0], o["O"][0]) < 1e-4
