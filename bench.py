@@ -1,0 +1,308 @@
+#!/usr/bin/env python
+"""Benchmark of the hot path: forward+backward Nystrom Laplacian attention, tokens/s.
+
+One step = one pass of the whole path (laplace_nystrom_fwd + laplace_nystrom_bwd through the
+C ABI) over one batch of synthetic input of the chosen workload (default: the DeiT-Small-shaped
+configuration the metric is quoted on).  Every rank of a multi-GPU launch runs the same workload
+on its own GPU (heads are independent, no collective), so scaling is weak.
+
+    python bench.py --gpus 1 --steps 20 --warmup 5
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+    python bench.py --impl reference      # the float64 CPU oracle on the host cores
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2604_20368_b200 import synth
+
+METRIC = "nystrom_laplacian_attention_fwd_bwd_tokens_per_s"
+UNIT = "tokens/s"
+# FP32 CUDA-core peak for plain ALU work (one add or subtract per lane per clock):
+# 148 SMs x 128 lanes x 1.965 GHz
+ALU_PEAK_TLANEOPS = 148 * 128 * 1.965e9 / 1e12
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="cfg2", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--B", type=int, default=0, help="override the batch size (profiling of a smaller case)")
+    return ap.parse_args()
+
+
+def workload_dict(cfg, extra=None):
+    d = {"workload": f"{cfg.name}: B={cfg.B} heads={cfg.H} n={cfg.n} d={cfg.d} m={cfg.m} lambda=d T={cfg.T} "
+                     f"{cfg.dtype} storage / fp32 accumulate, {'fwd+bwd' if cfg.backward else 'fwd only'}",
+         "B": cfg.B, "heads": cfg.H, "n": cfg.n, "d": cfg.d, "m": cfg.m, "ns_iters": cfg.T,
+         "tokens_per_step_per_gpu": cfg.B * cfg.n}
+    if extra:
+        d.update(extra)
+    return d
+
+
+# ------------------------------------------------------------------------------------------ oracle arm
+def oracle_pass(cfg, inp, heads):
+    """Time the float64 oracle (as it stands) on the listed heads; returns seconds."""
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import oracle
+    from parity import run_oracle_heads
+    oracle.build()
+    t0 = time.perf_counter()
+    run_oracle_heads(cfg, inp, heads, backward=cfg.backward)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(cfg, inp, budget_s=20.0):
+    import oracle
+    BH = cfg.B * cfg.H
+    probe = list(range(min(BH, max(1, oracle.num_threads()))))
+    t = oracle_pass(cfg, inp, probe)
+    per_head = t / len(probe)
+    k = int(min(BH, max(len(probe), budget_s / max(per_head, 1e-9))))
+    heads = list(range(k))
+    t = oracle_pass(cfg, inp, heads)
+    return {"value": k * cfg.n / t, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"heads 0..{k - 1} of {BH} (all n={cfg.n} tokens each), one pass, {t:.2f} s wall"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = synth.CONFIGS[args.config]
+    import oracle
+    inp = synth.make_inputs(cfg)
+    BH = cfg.B * cfg.H
+    # each step is a bounded sample: as many heads as fit about 1.5 s
+    per_head = oracle_pass(cfg, inp, list(range(min(BH, oracle.num_threads())))) / min(BH, oracle.num_threads())
+    k = int(min(BH, max(oracle.num_threads(), 1.5 / max(per_head, 1e-9))))
+    heads = list(range(k))
+    for _ in range(args.warmup):
+        oracle_pass(cfg, inp, heads)
+    t = sum(oracle_pass(cfg, inp, heads) for _ in range(args.steps))
+    value = args.steps * k * cfg.n / t
+    sample = f"heads 0..{k - 1} of {BH} per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_dict(cfg, {"sample": sample}),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            t = [x.strip() for x in line.split(",")]
+            if len(t) < 9:
+                continue
+            try:
+                sm.append(float(t[1])); mx.append(float(t[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), t[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------ our arm
+def l1_lane_ops(cfg, kernel):
+    """Algorithmic FP32 lane-operations of one launch of an l1 kernel: 2 per (pair, dim) in the forward
+    (subtract, accumulate |.|), all heads."""
+    BH = cfg.B * cfg.H
+    pairs = {"l1_C": cfg.n * cfg.m, "l1_R": cfg.n * cfg.m, "l1_W": cfg.m * cfg.m}[kernel]
+    return 2.0 * cfg.d * pairs * BH
+
+
+def run_ours(args):
+    import paper_2604_20368_b200 as ln
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+    cfg = synth.CONFIGS[args.config]
+    if args.B > 0:
+        cfg = synth.shrink(cfg, B=args.B)
+    inp = synth.make_inputs(cfg)
+    names = ("Q", "K", "V", "dO")
+    es = 4 if cfg.dtype == "f32" else 2
+    in_bytes = 4 * cfg.B * cfg.H * cfg.n * cfg.d * es
+    # rotate through enough input sets that a step's inputs are not L2-resident (126 MB L2)
+    nsets = max(2, int(np.ceil(3 * 126e6 / in_bytes)))
+    nsets = min(nsets, 16)
+    sets = []
+    for s in range(nsets):
+        sets.append({k: inp[k].to(dev).clone() for k in names})
+    wh = inp["whiten"].to(dev)
+    p = ln.problem_from_config(cfg, whiten=wh)
+    saved = torch.empty(ln.laplace_nystrom_saved_bytes(p), dtype=torch.uint8, device=dev)
+    ws = torch.empty(ln.laplace_nystrom_workspace_bytes(p, True), dtype=torch.uint8, device=dev)
+    O = torch.empty_like(sets[0]["Q"]); dQ = torch.empty_like(O); dK = torch.empty_like(O); dV = torch.empty_like(O)
+
+    def step(i):
+        s = sets[i % nsets]
+        ln.laplace_nystrom_fwd(p, s["Q"], s["K"], s["V"], O=O, saved=saved, ws=ws)
+        if cfg.backward:
+            ln.laplace_nystrom_bwd(p, s["Q"], s["K"], s["V"], s["dO"], saved, dQ=dQ, dK=dK, dV=dV, ws=ws)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for i in range(steps):
+            fn(i)
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            import torch.distributed as dist
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms = timed(step, args.steps)
+    clocks = sampler.stop() if sampler else None
+    tokens = cfg.B * cfg.n * world
+    value = tokens * args.steps / (ms * 1e-3)
+
+    # ---- end to end: pinned host inputs -> device, path, results -> pinned host, every step
+    host_in = {k: inp[k].pin_memory() for k in names}
+    host_out = {k: torch.empty_like(inp["Q"]).pin_memory() for k in ("O", "dQ", "dK", "dV")}
+    dev_in = {k: torch.empty_like(sets[0][k]) for k in names}
+
+    def step_e2e(i):
+        for k in names:
+            dev_in[k].copy_(host_in[k], non_blocking=True)
+        ln.laplace_nystrom_fwd(p, dev_in["Q"], dev_in["K"], dev_in["V"], O=O, saved=saved, ws=ws)
+        host_out["O"].copy_(O, non_blocking=True)
+        if cfg.backward:
+            ln.laplace_nystrom_bwd(p, dev_in["Q"], dev_in["K"], dev_in["V"], dev_in["dO"], saved, dQ=dQ, dK=dK, dV=dV, ws=ws)
+            for k, t in (("dQ", dQ), ("dK", dK), ("dV", dV)):
+                host_out[k].copy_(t, non_blocking=True)
+
+    for i in range(3):
+        step_e2e(i)
+    ms_e2e = timed(step_e2e, args.steps)
+    e2e_value = tokens * args.steps / (ms_e2e * 1e-3)
+    one = cfg.B * cfg.H * cfg.n * cfg.d * es
+    e2e = {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / args.steps,
+           "h2d_bytes_per_step": (4 if cfg.backward else 3) * one, "d2h_bytes_per_step": (4 if cfg.backward else 1) * one}
+
+    # ---- per-kernel durations (events around every launch, separate pass so the bracketing
+    # does not perturb the number above)
+    torch.cuda.synchronize()
+    ln.trace_begin()
+    for i in range(args.steps):
+        step(i)
+    trace = ln.trace_end()
+    launches_per_step = len(trace) // args.steps
+    per = {}
+    for name, t in trace:
+        a = per.setdefault(name, [0, 0.0]); a[0] += 1; a[1] += t
+    total_traced = sum(v[1] for v in per.values())
+    kernels = {k: {"launches_per_step": v[0] // args.steps, "avg_us": 1e3 * v[1] / v[0], "share": v[1] / total_traced}
+               for k, v in sorted(per.items(), key=lambda kv: -kv[1][1])}
+    dom = max((k for k in per if k in ("l1_C", "l1_R")), key=lambda k: per[k][1])
+    dom_avg_s = per[dom][1] / per[dom][0] * 1e-3
+    achieved = l1_lane_ops(cfg, dom) / dom_avg_s / 1e12
+    roofline = {"bound": "alu", "kernel": dom, "achieved": achieved, "peak": ALU_PEAK_TLANEOPS, "unit": "Tlane-op/s",
+                "frac": achieved / ALU_PEAK_TLANEOPS, "traffic": None,
+                "peak_source": "derived: 148 SMs x 128 FP32 lanes x 1.965 GHz, one add/sub per lane per clock",
+                "kernel_share_of_step": per[dom][1] / total_traced}
+    # whole-path roofline: algorithmic l1 lane-ops (2 fwd + 3 bwd per pair-dim) at the ALU peak
+    P = 2 * cfg.n * cfg.m + cfg.m * cfg.m
+    path_ops = (2.0 + (3.0 if cfg.backward else 0.0)) * cfg.d * P * cfg.B * cfg.H
+    path_roof_s = path_ops / (ALU_PEAK_TLANEOPS * 1e12)
+    roofline["path_frac"] = path_roof_s / (ms * 1e-3 / args.steps)
+
+    if rank != 0:
+        return
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_dict(cfg, {"l2": f"rotating {nsets} input sets ({nsets * in_bytes / 1e6:.0f} MB > 126 MB L2)",
+                                      "parallelism": f"replicas x{world} (heads independent, no collective)"}),
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "roofline": roofline, "kernels": kernels,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        out["cpu_baseline"] = cpu_baseline(cfg, inp)
+    print(json.dumps(out))
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -145,6 +145,17 @@ int l1_kernel_bwd(int32_t batch, int32_t na, int32_t nb, int32_t d, const void* 
 int landmarks_pool(const ln_problem* p, const void* K, float* L, void* stream);
 int landmarks_pool_bwd(const ln_problem* p, const float* dL, void* dK, void* stream);
 
+/*
+ * Profiling aid, off by default and not thread-safe (the paper has no counterpart; Sec. 4.3 only
+ * reports kernel times).  Between ln_trace_begin and ln_trace_end every kernel the library
+ * launches is bracketed by two CUDA events on its stream.  ln_trace_end synchronises the device,
+ * writes the number of traced launches to *count and, for the first `capacity` of them, the
+ * duration in milliseconds to ms[i] and a static name to names[i] (either array may be NULL).
+ * These two calls create and destroy CUDA events; no other entry point allocates anything.
+ */
+int ln_trace_begin(void);
+int ln_trace_end(int32_t capacity, int32_t* count, float* ms, const char** names);
+
 #ifdef __cplusplus
 }
 #endif

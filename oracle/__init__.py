@@ -43,6 +43,7 @@ class _Problem(ctypes.Structure):
         ("lm_mode", ctypes.c_int32),
         ("prefix", ctypes.c_int32), ("gh", ctypes.c_int32), ("gw", ctypes.c_int32),
         ("mh", ctypes.c_int32), ("mw", ctypes.c_int32),
+        ("lm_f32", ctypes.c_int32),
     ]
 
 
@@ -65,11 +66,12 @@ class Problem:
     gw: int = 0
     mh: int = 0
     mw: int = 0
+    lm_f32: int = 0   # 1: pooled landmarks rounded to single precision (what the device stores)
 
     def c(self) -> _Problem:
         return _Problem(self.B, self.H, self.n, self.d, self.m, float(self.lam), self.ns_iters,
                         float(self.ridge_eps), float(self.ns_alpha), self.map_mode, self.lm_mode,
-                        self.prefix, self.gh, self.gw, self.mh, self.mw)
+                        self.prefix, self.gh, self.gw, self.mh, self.mw, self.lm_f32)
 
 
 def _load():

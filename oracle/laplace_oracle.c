@@ -36,7 +36,9 @@
  *   - sign(0) = 0 in the kernel gradient (App. A states it only for t != 0),
  *     and its sign is the appendix's minus, not the introduction's plus;
  *   - pooling is adaptive (bin a covers rows floor(a*gh/mh) .. ceil((a+1)*gh/mh)-1),
- *     which equals r x r / stride r pooling whenever r divides the grid.
+ *     which equals r x r / stride r pooling whenever r divides the grid;
+ *   - optionally (lm_f32) a pooled landmark is the single-precision value nearest to the
+ *     exact mean, so that sign(token - landmark) is decided on the numbers the device holds.
  *
  * Pins (tests/test_oracle_*.py): hand values, brute force in numpy, the
  * Kac-Murdock-Szego closed-form inverse, the spectral closed form of the
@@ -62,6 +64,7 @@ typedef struct oracle_problem {
   int32_t map_mode; /* 0: O = C X R V;  1: injective map of Prop. 3 applied to the rows of C */
   int32_t lm_mode;  /* 0: landmarks given;  1: landmarks = adaptive average pooling of K */
   int32_t prefix, gh, gw, mh, mw; /* lm_mode 1: n = prefix + gh*gw, m = mh*mw */
+  int32_t lm_f32;   /* 1: pooled landmarks are rounded to single precision before use (see fwd_single) */
 } oracle_problem;
 
 int oracle_num_threads(void) {
@@ -382,8 +385,16 @@ static void ctx_free(head_ctx* x) {
 static void fwd_single(const oracle_problem* p, const double* Q, const double* K, const double* V,
                        const double* Lin, const double* s, head_ctx* x, double* O) {
   int n = p->n, d = p->d, m = p->m;
-  if (p->lm_mode == 1) pool_single(p, K, x->L);                    /* landmarks */
-  else memcpy(x->L, Lin, sizeof(double) * (size_t)m * d);
+  if (p->lm_mode == 1) {                                            /* landmarks */
+    pool_single(p, K, x->L);
+    /* The gradient of the kernel holds sign(token - landmark), which is discontinuous: a pooled
+       landmark that lies within rounding distance of a token decides that sign differently in
+       different precisions.  With lm_f32 the landmark is DEFINED as the single-precision value
+       nearest to the exact mean, the precision the device keeps landmarks in, so that both sides
+       take the decision on the same numbers. */
+    if (p->lm_f32)
+      for (size_t e = 0; e < (size_t)m * d; ++e) x->L[e] = (double)(float)x->L[e];
+  } else memcpy(x->L, Lin, sizeof(double) * (size_t)m * d);
   l1_block(n, m, d, Q, x->L, p->lambda, x->C);                      /* Eq. 8 */
   l1_block(m, m, d, x->L, x->L, p->lambda, x->W);                   /* Eq. 9 (ridge added inside Newton-Schulz) */
   l1_block(m, n, d, x->L, K, p->lambda, x->R);

@@ -23,6 +23,7 @@ EXPORTS = [
     "ln_status_string", "laplace_nystrom_saved_bytes", "laplace_nystrom_workspace_bytes",
     "laplace_nystrom_fwd", "laplace_nystrom_bwd", "ns_pinv_workspace_bytes", "ns_pinv", "ns_pinv_bwd",
     "l1_kernel", "l1_kernel_bwd_workspace_bytes", "l1_kernel_bwd", "landmarks_pool", "landmarks_pool_bwd",
+    "ln_trace_begin", "ln_trace_end",
 ]
 
 
@@ -115,6 +116,7 @@ def lib():
         L.l1_kernel_bwd.argtypes = [i32, i32, i32, i32, vp, vp, i32, f32, vp, vp, vp, vp, vp, sz, vp]
         L.landmarks_pool.argtypes = [pp, vp, vp, vp]
         L.landmarks_pool_bwd.argtypes = [pp, vp, vp, vp]
+        L.ln_trace_end.argtypes = [i32, ctypes.POINTER(i32), ctypes.POINTER(f32), ctypes.POINTER(ctypes.c_char_p)]
         _lib = L
     return _lib
 
@@ -257,3 +259,19 @@ def landmarks_pool_bwd(p: Problem, dL, stream=None):
     cp = p.c()
     _check(lib().landmarks_pool_bwd(ctypes.byref(cp), _ptr(dL), _ptr(dK), _stream(stream)), "landmarks_pool_bwd")
     return dK
+
+
+# ------------------------------------------------------------------------------------------ profiling aid
+def trace_begin():
+    """Start bracketing every library launch with CUDA events (profiling only)."""
+    _check(lib().ln_trace_begin(), "ln_trace_begin")
+
+
+def trace_end(capacity: int = 2048):
+    """Stop tracing; returns [(kernel name, milliseconds), ...] in launch order (synchronises)."""
+    cnt = ctypes.c_int32(0)
+    ms = (ctypes.c_float * capacity)()
+    names = (ctypes.c_char_p * capacity)()
+    _check(lib().ln_trace_end(capacity, ctypes.byref(cnt), ms, names), "ln_trace_end")
+    k = min(cnt.value, capacity)
+    return [(names[i].decode(), float(ms[i])) for i in range(k)]

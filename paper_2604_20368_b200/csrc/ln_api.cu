@@ -135,13 +135,35 @@ PoolGeom geom_of(const ln_problem* p) {
 inline int launch_ok() { return cudaGetLastError() == cudaSuccess ? LN_OK : LN_ERR_CUDA; }
 inline unsigned cdiv(long long a, long long b) { return (unsigned)((a + b - 1) / b); }
 
+// Profiling aid: when switched on by ln_trace_begin every launch is bracketed by two CUDA events
+// on its stream.  Off by default; the product path never touches it.
+constexpr int kTraceCap = 2048;
+struct Trace {
+  bool on = false;
+  int count = 0;
+  cudaEvent_t ev[2 * kTraceCap];
+  const char* name[kTraceCap];
+} g_trace;
+struct TraceScope {
+  cudaStream_t st; int slot;
+  TraceScope(const char* name, cudaStream_t s) : st(s), slot(-1) {
+    if (g_trace.on && g_trace.count < kTraceCap) {
+      slot = g_trace.count++;
+      g_trace.name[slot] = name;
+      cudaEventRecord(g_trace.ev[2 * slot], st);
+    }
+  }
+  ~TraceScope() { if (slot >= 0) cudaEventRecord(g_trace.ev[2 * slot + 1], st); }
+};
+#define LN_LAUNCH(name, st, ...) do { TraceScope ts_(name, st); __VA_ARGS__; } while (0)
+
 template <typename TA, typename TB>
-void launch_l1(const TA* A, const TB* Bm, float* E, float* rowsum, int batch, int na, int nb, int d,
+void launch_l1(const char* name, const TA* A, const TB* Bm, float* E, float* rowsum, int batch, int na, int nb, int d,
                int lde, float lambda, cudaStream_t st) {
   const float nscale = -1.4426950408889634f / lambda;
   dim3 grid(cdiv(na, L1_TA), batch);
-  k_l1<TA, TB><<<grid, 256, 0, st>>>(A, Bm, E, rowsum, na, nb, d, (long long)na * d, (long long)nb * d,
-                                     (long long)na * lde, lde, nscale);
+  LN_LAUNCH(name, st, k_l1<TA, TB><<<grid, 256, 0, st>>>(A, Bm, E, rowsum, na, nb, d, (long long)na * d, (long long)nb * d,
+                                     (long long)na * lde, lde, nscale));
 }
 
 // ------------------------------------------------------------------------------------------
@@ -151,23 +173,23 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const int BH = pl.BH, n = pl.n, m = pl.m;
   // landmarks (Sec. 4.2)
   if (p->lm_mode == 1) {
-    k_pool<T><<<dim3(m, BH), 128, 0, st>>>(K, x.Lf, geom_of(p));
+    LN_LAUNCH("k_pool", st, k_pool<T><<<dim3(m, BH), 128, 0, st>>>(K, x.Lf, geom_of(p)));
   } else {
     const long long cnt = (long long)BH * m * D;
-    k_to_f32<T><<<cdiv(cnt, 256), 256, 0, st>>>(L, x.Lf, cnt);
+    LN_LAUNCH("k_to_f32", st, k_to_f32<T><<<cdiv(cnt, 256), 256, 0, st>>>(L, x.Lf, cnt));
   }
   // the three kernel blocks: C = k(Q,L) with its row sums, R^T = k(K,L), W = k(L,L)
-  launch_l1<T, float>(Q, x.Lf, x.C, p->map_mode == 1 ? x.mu : nullptr, BH, n, m, D, pl.ldm, p->lambda, st);
-  if (p->map_mode == 1) k_scale<<<cdiv((long long)BH * n, 256), 256, 0, st>>>(x.mu, (long long)BH * n, 1.f / (float)m);
-  launch_l1<T, float>(K, x.Lf, x.Rt, nullptr, BH, n, m, D, pl.ldm, p->lambda, st);
-  launch_l1<float, float>(x.Lf, x.Lf, x.W, nullptr, BH, m, m, D, m, p->lambda, st);
+  launch_l1<T, float>("l1_C", Q, x.Lf, x.C, p->map_mode == 1 ? x.mu : nullptr, BH, n, m, D, pl.ldm, p->lambda, st);
+  if (p->map_mode == 1) LN_LAUNCH("k_scale", st, k_scale<<<cdiv((long long)BH * n, 256), 256, 0, st>>>(x.mu, (long long)BH * n, 1.f / (float)m));
+  launch_l1<T, float>("l1_R", K, x.Lf, x.Rt, nullptr, BH, n, m, D, pl.ldm, p->lambda, st);
+  launch_l1<float, float>("l1_W", x.Lf, x.Lf, x.W, nullptr, BH, m, m, D, m, p->lambda, st);
   // M = R V, partial over token chunks
-  k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, w.Mpart, nullptr, n, m, pl.rpc);
+  LN_LAUNCH("tn_M", st, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, w.Mpart, nullptr, n, m, pl.rpc));
   // Newton-Schulz, Y = X M, folded map
-  k_mid_fwd<D><<<BH, 256, 0, st>>>(m, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode, p->whiten, x.W, w.Wr, w.P,
-                                   x.Xh, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt, x.ybar, dev_status);
+  LN_LAUNCH("k_mid_fwd", st, k_mid_fwd<D><<<BH, 256, 0, st>>>(m, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode, p->whiten, x.W, w.Wr, w.P,
+                                   x.Xh, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt, x.ybar, dev_status));
   // O = (C - mu) Ytilde + ybar
-  k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr, x.Yt, x.ybar, O, n, m);
+  LN_LAUNCH("nn_O", st, k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr, x.Yt, x.ybar, O, n, m));
   return launch_ok();
 }
 
@@ -178,28 +200,28 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const float inv_lambda = 1.f / p->lambda;
   const float* mu = p->map_mode == 1 ? x.mu : nullptr;
   // query side: Z'^T dO and column sums of dO; g^C = (dO Ytilde^T) o C / lambda; dQ; landmark part
-  k_tn<T, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc);
-  k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(dO, x.Yt, x.C, pl.ldm, w.G, n, m, inv_lambda);
-  k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m);
-  k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc);
+  LN_LAUNCH("tn_dY", st, k_tn<T, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
+  LN_LAUNCH("ntg_C", st, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(dO, x.Yt, x.C, pl.ldm, w.G, n, m, inv_lambda));
+  LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m));
+  LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
   // per head: dY, dX, dM, Newton-Schulz adjoint, symmetrised landmark-block upstream
-  k_mid_bwd<D><<<BH, 256, 0, st>>>(m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten, x.W, x.Xh, x.hdr, x.M,
+  LN_LAUNCH("k_mid_bwd", st, k_mid_bwd<D><<<BH, 256, 0, st>>>(m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten, x.W, x.Xh, x.hdr, x.M,
                                    w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P, w.Hm, w.Ga, w.Gb, w.dW, w.dX,
-                                   w.dY, w.dM, w.GW);
-  k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, st>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m);
+                                   w.dY, w.dM, w.GW));
+  LN_LAUNCH("sign_rows_dLW", st, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, st>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));
   // key side: g^R = (V dM^T) o R^T / lambda; dV = R^T dM; dK (kernel part); landmark part
-  k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(V, w.dM, x.Rt, pl.ldm, w.G, n, m, inv_lambda);
-  k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m);
-  k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dKpart, n, m);
-  k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dLRpart, n, m, pl.rpc);
+  LN_LAUNCH("ntg_R", st, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(V, w.dM, x.Rt, pl.ldm, w.G, n, m, inv_lambda));
+  LN_LAUNCH("nn_dV", st, k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
+  LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dKpart, n, m));
+  LN_LAUNCH("sign_cols_dLR", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dLRpart, n, m, pl.rpc));
   // landmark gradient and its way back to the keys
   const int md = m * D;
   if (p->lm_mode == 1) {
-    k_reduce3<float><<<dim3(cdiv(md, 256), BH), 256, 0, st>>>(w.dLCpart, ch, w.dLRpart, ch, w.dLW, 1, w.dLtot, md);
-    k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256), BH), 256, 0, st>>>(w.dKpart, w.dLtot, dK, geom_of(p), 1);
+    LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 256), BH), 256, 0, st>>>(w.dLCpart, ch, w.dLRpart, ch, w.dLW, 1, w.dLtot, md));
+    LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256), BH), 256, 0, st>>>(w.dKpart, w.dLtot, dK, geom_of(p), 1));
   } else {
-    k_reduce3<T><<<dim3(cdiv(md, 256), BH), 256, 0, st>>>(w.dLCpart, ch, w.dLRpart, ch, w.dLW, 1, dL, md);
-    k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256), BH), 256, 0, st>>>(w.dKpart, nullptr, dK, geom_of(p), 0);
+    LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(md, 256), BH), 256, 0, st>>>(w.dLCpart, ch, w.dLRpart, ch, w.dLW, 1, dL, md));
+    LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256), BH), 256, 0, st>>>(w.dKpart, nullptr, dK, geom_of(p), 0));
   }
   return launch_ok();
 }
@@ -257,17 +279,40 @@ L1BwdWs carve_l1bwd(int batch, int na, int nb, int d, void* base) {
 template <typename T, int D>
 void l1_bwd_impl(int batch, int na, int nb, const T* A, const T* Bm, float lambda, const float* Kmat, const float* dK,
                  T* dA, T* dB, const L1BwdWs& w, cudaStream_t st) {
-  if (!Kmat) { launch_l1<T, T>(A, Bm, w.Kmat, nullptr, batch, na, nb, D, nb, lambda, st); Kmat = w.Kmat; }
+  if (!Kmat) { launch_l1<T, T>("l1_kernel", A, Bm, w.Kmat, nullptr, batch, na, nb, D, nb, lambda, st); Kmat = w.Kmat; }
   const long long cnt = (long long)batch * na * nb;
-  k_g_elem<<<cdiv(cnt, 256), 256, 0, st>>>(Kmat, dK, w.G, cnt, 1.f / lambda);
-  k_sign_rows<T, T, T, D><<<dim3(cdiv(na, 64), batch), 256, 0, st>>>(A, Bm, w.G, nb, dA, na, nb);
-  k_sign_cols<T, T, D><<<dim3(w.chunks, cdiv(nb, 64), batch), 256, 0, st>>>(A, Bm, w.G, nb, w.part, na, nb, w.rpc);
-  k_reduce3<T><<<dim3(cdiv(nb * D, 256), batch), 256, 0, st>>>(w.part, w.chunks, nullptr, 0, nullptr, 0, dB, nb * D);
+  LN_LAUNCH("k_g_elem", st, k_g_elem<<<cdiv(cnt, 256), 256, 0, st>>>(Kmat, dK, w.G, cnt, 1.f / lambda));
+  LN_LAUNCH("k_sign_rows", st, k_sign_rows<T, T, T, D><<<dim3(cdiv(na, 64), batch), 256, 0, st>>>(A, Bm, w.G, nb, dA, na, nb));
+  LN_LAUNCH("k_sign_cols", st, k_sign_cols<T, T, D><<<dim3(w.chunks, cdiv(nb, 64), batch), 256, 0, st>>>(A, Bm, w.G, nb, w.part, na, nb, w.rpc));
+  LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(nb * D, 256), batch), 256, 0, st>>>(w.part, w.chunks, nullptr, 0, nullptr, 0, dB, nb * D));
 }
 }  // namespace
 
 // ==========================================================================================
 extern "C" {
+
+int ln_trace_begin(void) {
+  if (g_trace.on) return LN_ERR_ARG;
+  for (int i = 0; i < 2 * kTraceCap; ++i)
+    if (cudaEventCreate(&g_trace.ev[i]) != cudaSuccess) return LN_ERR_CUDA;
+  g_trace.count = 0;
+  g_trace.on = true;
+  return LN_OK;
+}
+
+int ln_trace_end(int32_t capacity, int32_t* count, float* ms, const char** names) {
+  if (!g_trace.on || !count || capacity < 0) return LN_ERR_ARG;
+  g_trace.on = false;
+  int status = LN_OK;
+  if (cudaDeviceSynchronize() != cudaSuccess) status = LN_ERR_CUDA;
+  *count = g_trace.count;
+  for (int i = 0; i < g_trace.count && i < capacity && status == LN_OK; ++i) {
+    if (ms && cudaEventElapsedTime(&ms[i], g_trace.ev[2 * i], g_trace.ev[2 * i + 1]) != cudaSuccess) status = LN_ERR_CUDA;
+    if (names) names[i] = g_trace.name[i];
+  }
+  for (int i = 0; i < 2 * kTraceCap; ++i) cudaEventDestroy(g_trace.ev[i]);
+  return status;
+}
 
 const char* ln_status_string(int s) {
   switch (s) {
@@ -347,8 +392,8 @@ int ns_pinv(int32_t batch, int32_t m, const float* W, int32_t iters, float ridge
   if (m > 256) return LN_ERR_UNSUPPORTED;
   if (ws_bytes < ns_pinv_workspace_bytes(batch, m, iters)) return LN_ERR_WORKSPACE;
   const NsWs w = carve_ns_ws(batch, m, iters, ws);
-  k_ns_pinv<<<batch, 256, 0, static_cast<cudaStream_t>(stream)>>>(m, iters, ridge_eps, alpha, W, w.Wr, w.P,
-                                                                  X_hist ? X_hist : w.Xh, w.hdr, X, resid);
+  LN_LAUNCH("k_ns_pinv", static_cast<cudaStream_t>(stream), k_ns_pinv<<<batch, 256, 0, static_cast<cudaStream_t>(stream)>>>(m, iters, ridge_eps, alpha, W, w.Wr, w.P,
+                                                                  X_hist ? X_hist : w.Xh, w.hdr, X, resid));
   return launch_ok();
 }
 
@@ -360,8 +405,8 @@ int ns_pinv_bwd(int32_t batch, int32_t m, const float* W, int32_t iters, float r
   if (m > 256) return LN_ERR_UNSUPPORTED;
   if (ws_bytes < ns_pinv_workspace_bytes(batch, m, iters)) return LN_ERR_WORKSPACE;
   const NsWs w = carve_ns_ws(batch, m, iters, ws);
-  k_ns_pinv_bwd<<<batch, 256, 0, static_cast<cudaStream_t>(stream)>>>(m, iters, ridge_eps, alpha, W, w.Wr, w.P, w.Hm,
-                                                                      w.Ga, w.Gb, w.Xh, X_hist, w.hdr, dX, dW);
+  LN_LAUNCH("k_ns_pinv_bwd", static_cast<cudaStream_t>(stream), k_ns_pinv_bwd<<<batch, 256, 0, static_cast<cudaStream_t>(stream)>>>(m, iters, ridge_eps, alpha, W, w.Wr, w.P, w.Hm,
+                                                                      w.Ga, w.Gb, w.Xh, X_hist, w.hdr, dX, dW));
   return launch_ok();
 }
 
@@ -373,8 +418,8 @@ int l1_kernel(int32_t batch, int32_t na, int32_t nb, int32_t d, const void* A, c
   if (!aligned16(A) || !aligned16(Bm) || !aligned16(Kout) || !aligned16(rowsum)) return LN_ERR_ARG;
   if (batch > 65535) return LN_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (dtype == LN_F32) launch_l1<float, float>((const float*)A, (const float*)Bm, Kout, rowsum, batch, na, nb, d, nb, lambda, st);
-  else launch_l1<bf16, bf16>((const bf16*)A, (const bf16*)Bm, Kout, rowsum, batch, na, nb, d, nb, lambda, st);
+  if (dtype == LN_F32) launch_l1<float, float>("l1_kernel", (const float*)A, (const float*)Bm, Kout, rowsum, batch, na, nb, d, nb, lambda, st);
+  else launch_l1<bf16, bf16>("l1_kernel", (const bf16*)A, (const bf16*)Bm, Kout, rowsum, batch, na, nb, d, nb, lambda, st);
   return launch_ok();
 }
 
@@ -411,8 +456,8 @@ int landmarks_pool(const ln_problem* p, const void* K, float* L, void* stream) {
   if (p->lm_mode != 1 || !K || !L || !aligned16(K) || !aligned16(L)) return LN_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   dim3 grid(p->m, p->B * p->H);
-  if (p->dtype == LN_F32) k_pool<float><<<grid, 128, 0, st>>>((const float*)K, L, geom_of(p));
-  else k_pool<bf16><<<grid, 128, 0, st>>>((const bf16*)K, L, geom_of(p));
+  if (p->dtype == LN_F32) LN_LAUNCH("k_pool", st, k_pool<float><<<grid, 128, 0, st>>>((const float*)K, L, geom_of(p)));
+  else LN_LAUNCH("k_pool", st, k_pool<bf16><<<grid, 128, 0, st>>>((const bf16*)K, L, geom_of(p)));
   return launch_ok();
 }
 
@@ -422,8 +467,8 @@ int landmarks_pool_bwd(const ln_problem* p, const float* dL, void* dK, void* str
   if (p->lm_mode != 1 || !dL || !dK || !aligned16(dL) || !aligned16(dK)) return LN_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   dim3 grid(cdiv((long long)p->n * (p->d / 4), 256), p->B * p->H);
-  if (p->dtype == LN_F32) k_pool_bwd<float><<<grid, 256, 0, st>>>(nullptr, dL, (float*)dK, geom_of(p), 1);
-  else k_pool_bwd<bf16><<<grid, 256, 0, st>>>(nullptr, dL, (bf16*)dK, geom_of(p), 1);
+  if (p->dtype == LN_F32) LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<float><<<grid, 256, 0, st>>>(nullptr, dL, (float*)dK, geom_of(p), 1));
+  else LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<bf16><<<grid, 256, 0, st>>>(nullptr, dL, (bf16*)dK, geom_of(p), 1));
   return launch_ok();
 }
 

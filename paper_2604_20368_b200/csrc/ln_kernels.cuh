@@ -138,10 +138,13 @@ __global__ void k_pool(const T* __restrict__ K, float* __restrict__ L, PoolGeom 
   const int r0 = bin_lo(a, g.gh, g.mh), r1 = bin_hi(a, g.gh, g.mh);
   const int c0 = bin_lo(bb, g.gw, g.mw), c1 = bin_hi(bb, g.gw, g.mw);
   const T* Kh = K + (long long)bh * g.n * g.d;
-  float s = 0.f;
+  // The mean is accumulated in double and rounded once, so that the stored landmark is the fp32
+  // value nearest to the exact mean: sign(token - landmark) in the backward pass then does not
+  // depend on the order of a single-precision summation.
+  double s = 0.0;
   for (int r = r0; r < r1; ++r)
-    for (int q = c0; q < c1; ++q) s += to_f(Kh[(long long)(g.prefix + r * g.gw + q) * g.d + c]);
-  L[((long long)bh * g.m + l) * g.d + c] = s / (float)((r1 - r0) * (c1 - c0));
+    for (int q = c0; q < c1; ++q) s += (double)to_f(Kh[(long long)(g.prefix + r * g.gw + q) * g.d + c]);
+  L[((long long)bh * g.m + l) * g.d + c] = (float)(s / (double)((r1 - r0) * (c1 - c0)));
 }
 
 // dK[j] = dKpart[j] (may be NULL) + sum over the bins containing token j of dL[bin] / |bin|

@@ -27,7 +27,7 @@ def f64(t: torch.Tensor) -> np.ndarray:
 def oracle_problem(cfg: synth.Config, H=None, map_mode=1, lm_mode=1) -> oracle.Problem:
     return oracle.Problem(B=cfg.B if H is None else 1, H=cfg.H if H is None else H, n=cfg.n, d=cfg.d, m=cfg.m,
                           lam=cfg.lam, ns_iters=cfg.T, ridge_eps=cfg.ridge_eps, map_mode=map_mode, lm_mode=lm_mode,
-                          prefix=cfg.prefix, gh=cfg.gh, gw=cfg.gw, mh=cfg.mh, mw=cfg.mw)
+                          prefix=cfg.prefix, gh=cfg.gh, gw=cfg.gw, mh=cfg.mh, mw=cfg.mw, lm_f32=1)
 
 
 def run_gpu(cfg: synth.Config, inp, use_whiten=True, map_mode=1, backward=True):

@@ -97,8 +97,9 @@ def test_ns_pinv_bwd(m, T, given_hist):
     dW = ln.ns_pinv_bwd(Wd, T, 1e-6, 0.0, torch.from_numpy(dX).to(DEV), X_hist=hist)
     dWo = oracle.ns_pinv_bwd(W, T, float(np.float32(1e-6)), 0.0, dX)
     assert rel_err(f64(dW), dWo) < 1e-4
-    dWa = ln.ns_pinv_bwd(Wd, T, 1e-6, 0.02, torch.from_numpy(dX).to(DEV))
-    dWao = oracle.ns_pinv_bwd(W, T, float(np.float32(1e-6)), float(np.float32(0.02)), dX)
+    a = float(np.float32(0.9 / (m * m)))          # a given alpha inside the convergence region
+    dWa = ln.ns_pinv_bwd(Wd, T, 1e-6, a, torch.from_numpy(dX).to(DEV))
+    dWao = oracle.ns_pinv_bwd(W, T, float(np.float32(1e-6)), a, dX)
     assert rel_err(f64(dWa), dWao) < 1e-4
 
 
