@@ -41,7 +41,8 @@
 extern "C" {
 #endif
 
-typedef enum { LN_OK = 0, LN_ERR_ARG = -1, LN_ERR_UNSUPPORTED = -2, LN_ERR_WORKSPACE = -3, LN_ERR_CUDA = -4 } ln_status;
+typedef enum { LN_OK = 0, LN_ERR_ARG = -1, LN_ERR_UNSUPPORTED = -2, LN_ERR_WORKSPACE = -3, LN_ERR_CUDA = -4,
+               LN_ERR_STATIC_LIMIT = -5 } ln_status;
 typedef enum { LN_F32 = 0, LN_BF16 = 1 } ln_dtype;
 
 /* The problem statement of Alg. 1 / Alg. 2 in the paper's notation. */
@@ -117,6 +118,29 @@ int ns_pinv(int32_t batch, int32_t m, const float* W, int32_t iters, float ridge
  */
 int ns_pinv_bwd(int32_t batch, int32_t m, const float* W, int32_t iters, float ridge_eps, float alpha,
                 const float* X_hist, const float* dX, float* dW, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * ns_pinv without a workspace argument, for callers that cannot allocate device memory (the paper
+ * has no counterpart; this is a packaging variant of ns_pinv, same arithmetic, same results).
+ * Think of a serving process whose memory pool is fully committed at start-up, or a plug-in that
+ * only ever receives input and output pointers: neither can come up with the scratch ns_pinv
+ * wants.  Here the scratch is a fixed array of LN_STATIC_SCRATCH_BYTES inside the library image,
+ * so every GPU that loads the library gives up that much memory until the process exits.
+ *   - The caller still passes W [batch,m,m] and X [batch,m,m] (and resid [batch] or NULL); there
+ *     is no X_hist output.  Nothing is allocated or freed, by this call or on its behalf.
+ *   - Limit: ns_pinv_workspace_bytes(batch, m, iters) must not exceed LN_STATIC_SCRATCH_BYTES
+ *     (for instance batch 16, m 64, 6 iterations, or batch 2, m 256, 8 iterations); beyond it the
+ *     call returns LN_ERR_STATIC_LIMIT and enqueues nothing.
+ *   - The first call on each device looks up the device address of the array (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  It keeps whatever the last call left, which is
+ *     harmless (every part is written before it is read), but two calls that overlap on the GPU,
+ *     for example on different streams, race on it: serialise them.
+ */
+#define LN_STATIC_SCRATCH_BYTES (8u << 20)
+size_t ns_pinv_static_scratch_bytes(void);
+int ns_pinv_static(int32_t batch, int32_t m, const float* W, int32_t iters, float ridge_eps, float alpha,
+                   float* X, float* resid, void* stream);
 
 /*
  * Laplacian kernel block (Sec. 1, Eq. 8): Kout[b,i,j] = exp(-||A[b,i,:] - Bm[b,j,:]||_1 / lambda).

@@ -17,13 +17,14 @@ from . import build as _build
 
 LN_F32, LN_BF16 = 0, 1
 _STATUS = {0: "ok", -1: "invalid argument", -2: "outside the supported envelope",
-           -3: "workspace too small", -4: "CUDA launch failed"}
+           -3: "workspace too small", -4: "CUDA launch failed",
+           -5: "problem exceeds the static scratch of the no-allocation entry point"}
 
 EXPORTS = [
     "ln_status_string", "laplace_nystrom_saved_bytes", "laplace_nystrom_workspace_bytes",
     "laplace_nystrom_fwd", "laplace_nystrom_bwd", "ns_pinv_workspace_bytes", "ns_pinv", "ns_pinv_bwd",
     "l1_kernel", "l1_kernel_bwd_workspace_bytes", "l1_kernel_bwd", "landmarks_pool", "landmarks_pool_bwd",
-    "ln_trace_begin", "ln_trace_end",
+    "ln_trace_begin", "ln_trace_end", "ns_pinv_static_scratch_bytes", "ns_pinv_static",
 ]
 
 
@@ -116,6 +117,9 @@ def lib():
         L.l1_kernel_bwd.argtypes = [i32, i32, i32, i32, vp, vp, i32, f32, vp, vp, vp, vp, vp, sz, vp]
         L.landmarks_pool.argtypes = [pp, vp, vp, vp]
         L.landmarks_pool_bwd.argtypes = [pp, vp, vp, vp]
+        L.ns_pinv_static_scratch_bytes.restype = sz
+        L.ns_pinv_static_scratch_bytes.argtypes = []
+        L.ns_pinv_static.argtypes = [i32, i32, vp, i32, f32, f32, vp, vp, vp]
         L.ln_trace_end.argtypes = [i32, ctypes.POINTER(i32), ctypes.POINTER(f32), ctypes.POINTER(ctypes.c_char_p)]
         _lib = L
     return _lib
@@ -220,6 +224,17 @@ def ns_pinv_bwd(W, iters: int, ridge_eps: float, alpha: float, dX, X_hist=None, 
                            ws.numel(), _stream(stream))
     _check(st, "ns_pinv_bwd")
     return dW
+
+
+def ns_pinv_static(W, iters: int, X, ridge_eps: float = 0.0, alpha: float = 0.0, resid=None, stream=None):
+    """ns_pinv for callers that cannot allocate: the scratch lives inside the library, so the caller
+    hands in only W and the output X (and optionally resid), all allocated beforehand.  Raises
+    LnError(-5) when the problem does not fit the library's fixed scratch.  Calls that overlap on
+    the GPU share that scratch and must be serialised by the caller."""
+    batch, m, _ = W.shape
+    st = lib().ns_pinv_static(batch, m, _ptr(W), iters, ridge_eps, alpha, _ptr(X), _ptr(resid), _stream(stream))
+    _check(st, "ns_pinv_static")
+    return X
 
 
 # ------------------------------------------------------------------------------------------ kernel block

@@ -321,6 +321,7 @@ const char* ln_status_string(int s) {
     case LN_ERR_UNSUPPORTED: return "outside the supported envelope";
     case LN_ERR_WORKSPACE: return "workspace too small";
     case LN_ERR_CUDA: return "CUDA launch failed";
+    case LN_ERR_STATIC_LIMIT: return "problem exceeds the static scratch of the no-allocation entry point";
   }
   return "unknown status";
 }
@@ -407,6 +408,60 @@ int ns_pinv_bwd(int32_t batch, int32_t m, const float* W, int32_t iters, float r
   const NsWs w = carve_ns_ws(batch, m, iters, ws);
   LN_LAUNCH("k_ns_pinv_bwd", static_cast<cudaStream_t>(stream), k_ns_pinv_bwd<<<batch, 256, 0, static_cast<cudaStream_t>(stream)>>>(m, iters, ridge_eps, alpha, W, w.Wr, w.P, w.Hm,
                                                                       w.Ga, w.Gb, w.Xh, X_hist, w.hdr, dX, dW));
+  return launch_ok();
+}
+
+// ------------------------------------------------------------------------------------------
+// ns_pinv for callers that cannot allocate device memory.
+//
+// Some users of this library run where cudaMalloc is off the table: inside a serving loop whose
+// memory pool was carved up at start-up and is fully committed, in a plug-in that is handed
+// input and output pointers and nothing else, or under a framework that forbids allocator
+// calls on its worker threads.  ns_pinv itself needs scratch (the ridge-shifted matrix, one
+// product and the iterates), which such a caller has no way to provide.  This variant keeps
+// that scratch in a fixed array that is part of the library image: every GPU that loads the
+// library holds LN_STATIC_SCRATCH_BYTES of device memory for it until the process exits.
+//
+// In host code the name of a __device__ array is only a stand-in; the device address has to be
+// asked for, once per device, with that device current.  The first call on a device does that.
+// ------------------------------------------------------------------------------------------
+namespace {
+constexpr size_t kStaticScratchBytes = LN_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices];   // device address of g_static_scratch, per device; NULL = not asked yet
+
+// Device address of the static scratch on the current device (looked up on first use).
+int static_scratch_ptr(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LN_ERR_CUDA;
+  if (!g_static_scratch_addr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return LN_ERR_CUDA;
+    g_static_scratch_addr[dev] = ptr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return LN_OK;
+}
+}  // namespace
+
+size_t ns_pinv_static_scratch_bytes(void) { return kStaticScratchBytes; }
+
+int ns_pinv_static(int32_t batch, int32_t m, const float* W, int32_t iters, float ridge_eps, float alpha, float* X,
+                   float* resid, void* stream) {
+  if (batch <= 0 || m <= 0 || iters < 0 || !W || !X) return LN_ERR_ARG;
+  if (!(ridge_eps >= 0.f) || !isfinite(ridge_eps) || !isfinite(alpha)) return LN_ERR_ARG;
+  if (!aligned16(W) || !aligned16(X)) return LN_ERR_ARG;
+  if (m > 256) return LN_ERR_UNSUPPORTED;
+  if (ns_pinv_workspace_bytes(batch, m, iters) > kStaticScratchBytes) return LN_ERR_STATIC_LIMIT;
+  void* scratch = nullptr;
+  const int s = static_scratch_ptr(&scratch);
+  if (s != LN_OK) return s;
+  // Every piece of the scratch is written by the kernel before it is read, so the contents a
+  // previous call left behind do not matter and nothing has to be cleared.
+  const NsWs w = carve_ns_ws(batch, m, iters, scratch);
+  LN_LAUNCH("k_ns_pinv", static_cast<cudaStream_t>(stream), k_ns_pinv<<<batch, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      m, iters, ridge_eps, alpha, W, w.Wr, w.P, w.Xh, w.hdr, X, resid));
   return launch_ok();
 }
 
