@@ -4,6 +4,8 @@
 
 #include "../../include/laplace_nystrom.h"
 #include "ln_kernels.cuh"
+#include "ln_mma.cuh"
+#include <type_traits>
 
 using namespace ln;
 
@@ -159,11 +161,11 @@ struct TraceScope {
 
 template <typename TA, typename TB>
 void launch_l1(const char* name, const TA* A, const TB* Bm, float* E, float* rowsum, int batch, int na, int nb, int d,
-               int lde, float lambda, cudaStream_t st) {
+               int lde, float lambda, cudaStream_t st, float rs_scale = 1.f) {
   const float nscale = -1.4426950408889634f / lambda;
   dim3 grid(cdiv(na, L1_TA), batch);
   LN_LAUNCH(name, st, k_l1<TA, TB><<<grid, 256, 0, st>>>(A, Bm, E, rowsum, na, nb, d, (long long)na * d, (long long)nb * d,
-                                     (long long)na * lde, lde, nscale));
+                                     (long long)na * lde, lde, nscale, rs_scale));
 }
 
 // ------------------------------------------------------------------------------------------
@@ -179,17 +181,23 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     LN_LAUNCH("k_to_f32", st, k_to_f32<T><<<cdiv(cnt, 256), 256, 0, st>>>(L, x.Lf, cnt));
   }
   // the three kernel blocks: C = k(Q,L) with its row sums, R^T = k(K,L), W = k(L,L)
-  launch_l1<T, float>("l1_C", Q, x.Lf, x.C, p->map_mode == 1 ? x.mu : nullptr, BH, n, m, D, pl.ldm, p->lambda, st);
-  if (p->map_mode == 1) LN_LAUNCH("k_scale", st, k_scale<<<cdiv((long long)BH * n, 256), 256, 0, st>>>(x.mu, (long long)BH * n, 1.f / (float)m));
+  launch_l1<T, float>("l1_C", Q, x.Lf, x.C, p->map_mode == 1 ? x.mu : nullptr, BH, n, m, D, pl.ldm, p->lambda, st,
+                      1.f / (float)m);   // row means (Prop. 3 step 2)
   launch_l1<T, float>("l1_R", K, x.Lf, x.Rt, nullptr, BH, n, m, D, pl.ldm, p->lambda, st);
   launch_l1<float, float>("l1_W", x.Lf, x.Lf, x.W, nullptr, BH, m, m, D, m, p->lambda, st);
   // M = R V, partial over token chunks
-  LN_LAUNCH("tn_M", st, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, w.Mpart, nullptr, n, m, pl.rpc));
+  if constexpr (std::is_same<T, bf16>::value)
+    LN_LAUNCH("tn_M", st, k_tn_mma<D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, w.Mpart, nullptr, n, m, pl.rpc));
+  else
+    LN_LAUNCH("tn_M", st, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, w.Mpart, nullptr, n, m, pl.rpc));
   // Newton-Schulz, Y = X M, folded map
   LN_LAUNCH("k_mid_fwd", st, k_mid_fwd<D><<<BH, 256, 0, st>>>(m, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode, p->whiten, x.W, w.Wr, w.P,
                                    x.Xh, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt, x.ybar, dev_status));
   // O = (C - mu) Ytilde + ybar
-  LN_LAUNCH("nn_O", st, k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr, x.Yt, x.ybar, O, n, m));
+  if constexpr (std::is_same<T, bf16>::value)
+    LN_LAUNCH("nn_O", st, k_nn_mma<D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr, x.Yt, x.ybar, O, n, m));
+  else
+    LN_LAUNCH("nn_O", st, k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr, x.Yt, x.ybar, O, n, m));
   return launch_ok();
 }
 
@@ -200,8 +208,13 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const float inv_lambda = 1.f / p->lambda;
   const float* mu = p->map_mode == 1 ? x.mu : nullptr;
   // query side: Z'^T dO and column sums of dO; g^C = (dO Ytilde^T) o C / lambda; dQ; landmark part
-  LN_LAUNCH("tn_dY", st, k_tn<T, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
-  LN_LAUNCH("ntg_C", st, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(dO, x.Yt, x.C, pl.ldm, w.G, n, m, inv_lambda));
+  if constexpr (std::is_same<T, bf16>::value) {
+    LN_LAUNCH("tn_dY", st, k_tn_mma<D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
+    LN_LAUNCH("ntg_C", st, k_nt_g_mma<D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(dO, x.Yt, x.C, pl.ldm, w.G, n, m, inv_lambda));
+  } else {
+    LN_LAUNCH("tn_dY", st, k_tn<T, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
+    LN_LAUNCH("ntg_C", st, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(dO, x.Yt, x.C, pl.ldm, w.G, n, m, inv_lambda));
+  }
   LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m));
   LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
   // per head: dY, dX, dM, Newton-Schulz adjoint, symmetrised landmark-block upstream
@@ -210,8 +223,13 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
                                    w.dY, w.dM, w.GW));
   LN_LAUNCH("sign_rows_dLW", st, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, st>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));
   // key side: g^R = (V dM^T) o R^T / lambda; dV = R^T dM; dK (kernel part); landmark part
-  LN_LAUNCH("ntg_R", st, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(V, w.dM, x.Rt, pl.ldm, w.G, n, m, inv_lambda));
-  LN_LAUNCH("nn_dV", st, k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
+  if constexpr (std::is_same<T, bf16>::value) {
+    LN_LAUNCH("ntg_R", st, k_nt_g_mma<D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(V, w.dM, x.Rt, pl.ldm, w.G, n, m, inv_lambda));
+    LN_LAUNCH("nn_dV", st, k_nn_mma<D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
+  } else {
+    LN_LAUNCH("ntg_R", st, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(V, w.dM, x.Rt, pl.ldm, w.G, n, m, inv_lambda));
+    LN_LAUNCH("nn_dV", st, k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
+  }
   LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dKpart, n, m));
   LN_LAUNCH("sign_cols_dLR", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dLRpart, n, m, pl.rpc));
   // landmark gradient and its way back to the keys

@@ -44,9 +44,16 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// g * sign(t) with sign(0) = 0: the kernel gradient of App. A (stated there for t != 0), with
-// the midpoint sub-gradient at a tie.
-__device__ __forceinline__ float signed_g(float t, float g) { return t > 0.f ? g : (t < 0.f ? -g : 0.f); }
+// (sign(t) + 1) / 2 = 0, 1/2, 1 for t < 0, t == 0, t > 0, as one saturating multiply-add on the FMA
+// pipe (compare/select instructions would run on the half-rate ALU pipe).  The kernel gradient of
+// App. A needs sum_j g_j sign(t_j) = 2 sum_j g_j half_step(t_j) - sum_j g_j, with sign(0) = 0 (the
+// appendix states the gradient for t != 0; a tie takes the midpoint sub-gradient).  Exact for every
+// |t| >= 2^-101; a smaller non-zero difference is treated as a tie.
+__device__ __forceinline__ float half_step(float t) {
+  float r;
+  asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(t), "f"(1.2676506e30f /* 2^100 */), "f"(0.5f));
+  return r;
+}
 
 // Column set a thread owns in a [rows x D] tile worked on by 16 column-threads: DC = D/16
 // columns, laid out so that the 16 threads read one contiguous 256-byte (128 for D = 32) run.

@@ -16,7 +16,8 @@ constexpr int L1_TA = 128, L1_TB = 64, L1_DC = 32;
 template <typename TA, typename TB>
 __global__ void __launch_bounds__(256) k_l1(const TA* __restrict__ A, const TB* __restrict__ Bm,
                                             float* __restrict__ E, float* __restrict__ rowsum, int na, int nb, int d,
-                                            long long sA, long long sB, long long sE, int lde, float nscale) {
+                                            long long sA, long long sB, long long sE, int lde, float nscale,
+                                            float rs_scale) {
   __shared__ __align__(16) float As[L1_DC][L1_TA + 4];
   __shared__ __align__(16) float Bs[L1_DC][L1_TB + 4];
   const int b = blockIdx.y, i0 = blockIdx.x * L1_TA;
@@ -106,15 +107,9 @@ __global__ void __launch_bounds__(256) k_l1(const TA* __restrict__ A, const TB* 
       v += __shfl_xor_sync(0xffffffffu, v, 4);
       v += __shfl_xor_sync(0xffffffffu, v, 8);
       const int gi = i0 + ti * 8 + i;
-      if (tj == 0 && gi < na) rowsum[(long long)b * na + gi] = v;
+      if (tj == 0 && gi < na) rowsum[(long long)b * na + gi] = v * rs_scale;
     }
   }
-}
-
-// rowsum -> row mean (Prop. 3 step 2), in place
-__global__ void k_scale(float* x, long long count, float s) {
-  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < count) x[i] *= s;
 }
 
 // storage type -> fp32 copy
@@ -452,10 +447,11 @@ __global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, c
   Lm += (long long)bh * m * D;
   G += (long long)bh * n * ldg;
   out += (long long)bh * n * D;
-  float q[4][DC], acc[4][DC];
+  float q[4][DC], acc[4][DC], gsum[4];
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const int i = i0 + tt * 4 + k;
+    gsum[k] = 0.f;
 #pragma unroll
     for (int s = 0; s < DC; ++s) {
       acc[k][s] = 0.f;
@@ -492,9 +488,11 @@ __global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, c
         float lv[DC];
         ld_cols<D>(&Ls[ll + s][0], tc, lv);
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
+        for (int k = 0; k < 4; ++k) {
+          gsum[k] += g[k][s];
 #pragma unroll
-          for (int c = 0; c < DC; ++c) acc[k][c] += signed_g(q[k][c] - lv[c], g[k][s]);
+          for (int c = 0; c < DC; ++c) acc[k][c] = fmaf(g[k][s], half_step(q[k][c] - lv[c]), acc[k][c]);
+        }
       }
     }
   }
@@ -503,7 +501,8 @@ __global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, c
     const int i = i0 + tt * 4 + k;
     if (i < n)
 #pragma unroll
-      for (int c = 0; c < DC; ++c) out[(long long)i * D + ColMap<D>::col(tc, c)] = from_f<TO>(-acc[k][c]);
+      for (int c = 0; c < DC; ++c)
+        out[(long long)i * D + ColMap<D>::col(tc, c)] = from_f<TO>(gsum[k] - 2.f * acc[k][c]);
   }
 }
 
@@ -524,10 +523,11 @@ __global__ void __launch_bounds__(256) k_sign_cols(const TT* __restrict__ tok, c
   Lm += (long long)bh * m * D;
   G += (long long)bh * n * ldg;
   const int ibeg = chunk * rpc, iend = min(n, ibeg + rpc);
-  float lv[4][DC], acc[4][DC];
+  float lv[4][DC], acc[4][DC], gsum[4];
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const int l = l0 + tl * 4 + k;
+    gsum[k] = 0.f;
 #pragma unroll
     for (int s = 0; s < DC; ++s) {
       acc[k][s] = 0.f;
@@ -558,9 +558,11 @@ __global__ void __launch_bounds__(256) k_sign_cols(const TT* __restrict__ tok, c
       float tv[DC];
       ld_cols<D>(&Ts[jj][0], tc, tv);
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
+      for (int k = 0; k < 4; ++k) {
+        gsum[k] += g[k];
 #pragma unroll
-        for (int c = 0; c < DC; ++c) acc[k][c] += signed_g(tv[c] - lv[k][c], g[k]);
+        for (int c = 0; c < DC; ++c) acc[k][c] = fmaf(g[k], half_step(tv[c] - lv[k][c]), acc[k][c]);
+      }
     }
   }
   float* out = part + ((long long)bh * nchunks + chunk) * m * D;
@@ -569,7 +571,7 @@ __global__ void __launch_bounds__(256) k_sign_cols(const TT* __restrict__ tok, c
     const int l = l0 + tl * 4 + k;
     if (l < m)
 #pragma unroll
-      for (int c = 0; c < DC; ++c) out[(long long)l * D + ColMap<D>::col(tc, c)] = acc[k][c];
+      for (int c = 0; c < DC; ++c) out[(long long)l * D + ColMap<D>::col(tc, c)] = 2.f * acc[k][c] - gsum[k];
   }
 }
 
