@@ -4,7 +4,6 @@
 
 #include "../../include/laplace_nystrom.h"
 #include "ln_kernels.cuh"
-#include "ln_mma.cuh"
 #include <type_traits>
 
 using namespace ln;
@@ -191,8 +190,18 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   else
     LN_LAUNCH("tn_M", st, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, w.Mpart, nullptr, n, m, pl.rpc));
   // Newton-Schulz, Y = X M, folded map
-  LN_LAUNCH("k_mid_fwd", st, k_mid_fwd<D><<<BH, 256, 0, st>>>(m, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode, p->whiten, x.W, w.Wr, w.P,
-                                   x.Xh, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt, x.ybar, dev_status));
+  {
+    constexpr bool TC = std::is_same<T, bf16>::value;
+    auto launch = [&](auto kern, size_t smem) {
+      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      LN_LAUNCH("k_mid_fwd", st, kern<<<BH, 256, smem, st>>>(m, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode, p->whiten,
+                                                          x.W, w.Wr, w.P, x.Xh, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt,
+                                                          x.ybar, dev_status));
+    };
+    if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * NsTile<64>::mat_bytes);
+    else if (TC && m <= 128) launch(k_mid_fwd<D, TC, TC ? 128 : 0>, 3 * NsTile<128>::mat_bytes);
+    else launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));
+  }
   // O = (C - mu) Ytilde + ybar
   if constexpr (std::is_same<T, bf16>::value)
     LN_LAUNCH("nn_O", st, k_nn_mma<D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr, x.Yt, x.ybar, O, n, m));
@@ -218,9 +227,17 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m));
   LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
   // per head: dY, dX, dM, Newton-Schulz adjoint, symmetrised landmark-block upstream
-  LN_LAUNCH("k_mid_bwd", st, k_mid_bwd<D><<<BH, 256, 0, st>>>(m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten, x.W, x.Xh, x.hdr, x.M,
-                                   w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P, w.Hm, w.Ga, w.Gb, w.dW, w.dX,
-                                   w.dY, w.dM, w.GW));
+  {
+    constexpr bool TC = std::is_same<T, bf16>::value;
+    auto launch = [&](auto kern, size_t smem) {
+      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      LN_LAUNCH("k_mid_bwd", st, kern<<<BH, 256, smem, st>>>(m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten, x.W, x.Xh,
+                                                          x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P, w.Hm,
+                                                          w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW));
+    };
+    if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 5 * NsTile<64>::mat_bytes);
+    else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
+  }
   LN_LAUNCH("sign_rows_dLW", st, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, st>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));
   // key side: g^R = (V dM^T) o R^T / lambda; dV = R^T dM; dK (kernel part); landmark part
   if constexpr (std::is_same<T, bf16>::value) {

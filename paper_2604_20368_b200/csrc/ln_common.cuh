@@ -79,4 +79,20 @@ template <int D> __device__ __forceinline__ void ld_cols(const float* row, int t
   }
 }
 
+// Block-wide sum of one float per thread (256 threads); result valid in every thread.
+__device__ inline float block_sum(float v, float* red /* >= 8 floats of shared memory */) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float s = 0.f;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w];
+  __syncthreads();
+  return s;
+}
+
+// Header kept per matrix beside the Newton-Schulz iterates.
+struct NsHdr { float alpha, n1, ninf; int jstar, istar, auto_alpha, pad0, pad1; };
+
 }  // namespace ln

@@ -3,6 +3,8 @@
 // blockIdx.x.  All intermediates are fp32; only the [.,.,.,d] user tensors have a storage type.
 #pragma once
 #include "ln_common.cuh"
+#include "ln_mma.cuh"
+#include "ln_ns_smem.cuh"
 
 namespace ln {
 
@@ -643,21 +645,26 @@ __device__ void cta_gemm(int M, int N, int K, const float* A, int lda, const flo
   __syncthreads();
 }
 
-// Block-wide sum of one float per thread (256 threads); result valid in every thread.
-__device__ inline float block_sum(float v, float* red /* >= 8 floats of shared memory */) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
-  __syncthreads();
-  float s = 0.f;
-  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w];
-  __syncthreads();
-  return s;
-}
+// Shared memory of the per-head kernels: one of the two GEMM engines is used per instantiation.
+union __align__(16) NsSmem { GemmSmem f; MmaGemmSmem t; };
 
-// Header kept per matrix beside the Newton-Schulz iterates.
-struct NsHdr { float alpha, n1, ninf; int jstar, istar, auto_alpha, pad0, pad1; };
+// C = beta*Cin + alpha*op(A)op(B) + diag*I on either engine: TC = tensor cores with split-bf16
+// operands (bf16-storage path), else exact fp32 FFMA (fp32-storage path, stand-alone ns_pinv).
+template <bool TC, bool TRA, bool TRB>
+__device__ __forceinline__ void ns_gemm(int M, int N, int K, const float* A, int lda, const float* Bm, int ldb,
+                                        float* C, int ldc, float alpha, float beta, const float* Cin, float diag,
+                                        NsSmem& sm) {
+  if (TC) {
+    cta_gemm_mma<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.t);
+  } else {
+    cta_gemm<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, sm.f);
+    if (diag != 0.f) {
+      const int lim = M < N ? M : N;
+      for (int i = threadIdx.x; i < lim; i += 256) C[(long long)i * ldc + i] += diag;
+      __syncthreads();
+    }
+  }
+}
 
 // =====================================================================================
 // Newton-Schulz forward for one m x m matrix (Alg. 2), whole CTA.
@@ -665,8 +672,9 @@ struct NsHdr { float alpha, n1, ninf; int jstar, istar, auto_alpha, pad0, pad1; 
 //   X_{k+1} = X_k (2I - Wr X_k);  Xh[k] = X_k for k = 0..T.
 // W, Wr, P: [m][m] in global memory; Xh: [T+1][m][m].
 // =====================================================================================
+template <bool TC>
 __device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const float* W, float* Wr, float* P,
-                               float* Xh, NsHdr* hdr, GemmSmem& sm, float* red /* 2*256 + 8 floats */) {
+                               float* Xh, NsHdr* hdr, NsSmem& sm, float* red /* 2*256 + 8 floats */) {
   const int tid = threadIdx.x;
   const long long mm = (long long)m * m;
   for (long long e = tid; e < mm; e += 256) {
@@ -703,10 +711,8 @@ __device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const fl
   for (int k = 0; k < T; ++k) {
     const float* X = Xh + (long long)k * mm;
     float* Xn = Xh + (long long)(k + 1) * mm;
-    cta_gemm<false, false>(m, m, m, Wr, m, X, m, P, m, -1.f, 0.f, nullptr, sm);   // P = -Wr X_k
-    for (int i = tid; i < m; i += 256) P[(long long)i * m + i] += 2.f;             // 2I - Wr X_k
-    __syncthreads();
-    cta_gemm<false, false>(m, m, m, X, m, P, m, Xn, m, 1.f, 0.f, nullptr, sm);     // X_{k+1}
+    ns_gemm<TC, false, false>(m, m, m, Wr, m, X, m, P, m, -1.f, 0.f, nullptr, 2.f, sm);   // P = 2I - Wr X_k
+    ns_gemm<TC, false, false>(m, m, m, X, m, P, m, Xn, m, 1.f, 0.f, nullptr, 0.f, sm);    // X_{k+1} = X_k P
   }
 }
 
@@ -714,9 +720,10 @@ __device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const fl
 // Exact adjoint of ns_forward_dev: given G0 = dLoss/dX_T returns dW = dLoss/dW.
 // Scratch matrices [m][m]: P, Hm, Ga, Gb.  Xh holds X_0..X_T, Wr = W + eps I, hdr from the forward.
 // =====================================================================================
+template <bool TC>
 __device__ void ns_backward_dev(int m, int T, const float* Wr, const float* Xh, const NsHdr* hdr,
                                 const float* G0, float* dW, float* P, float* Hm, float* Ga, float* Gb,
-                                GemmSmem& sm, float* red) {
+                                NsSmem& sm, float* red) {
   const int tid = threadIdx.x;
   const long long mm = (long long)m * m;
   for (long long e = tid; e < mm; e += 256) { Ga[e] = G0[e]; dW[e] = 0.f; }
@@ -724,11 +731,11 @@ __device__ void ns_backward_dev(int m, int T, const float* Wr, const float* Xh, 
   float* G = Ga; float* Gn = Gb;
   for (int k = T - 1; k >= 0; --k) {
     const float* A = Xh + (long long)k * mm;                                        // X_{k+1} = 2A - A P, P = Wr A
-    cta_gemm<false, false>(m, m, m, Wr, m, A, m, P, m, 1.f, 0.f, nullptr, sm);      // P = Wr A
-    cta_gemm<true, false>(m, m, m, A, m, G, m, Hm, m, 1.f, 0.f, nullptr, sm);       // H = A^T G
-    cta_gemm<false, true>(m, m, m, Hm, m, A, m, dW, m, -1.f, 1.f, dW, sm);          // dW -= H A^T
-    cta_gemm<false, true>(m, m, m, G, m, P, m, Gn, m, -1.f, 2.f, G, sm);            // Gn = 2G - G P^T
-    cta_gemm<true, false>(m, m, m, Wr, m, Hm, m, Gn, m, -1.f, 1.f, Gn, sm);         // Gn -= Wr^T H
+    ns_gemm<TC, false, false>(m, m, m, Wr, m, A, m, P, m, 1.f, 0.f, nullptr, 0.f, sm);      // P = Wr A
+    ns_gemm<TC, true, false>(m, m, m, A, m, G, m, Hm, m, 1.f, 0.f, nullptr, 0.f, sm);       // H = A^T G
+    ns_gemm<TC, false, true>(m, m, m, Hm, m, A, m, dW, m, -1.f, 1.f, dW, 0.f, sm);          // dW -= H A^T
+    ns_gemm<TC, false, true>(m, m, m, G, m, P, m, Gn, m, -1.f, 2.f, G, 0.f, sm);            // Gn = 2G - G P^T
+    ns_gemm<TC, true, false>(m, m, m, Wr, m, Hm, m, Gn, m, -1.f, 1.f, Gn, 0.f, sm);         // Gn -= Wr^T H
     float* t = G; G = Gn; Gn = t;
   }
   // X_0 = alpha Wr^T
@@ -764,16 +771,16 @@ __device__ void ns_backward_dev(int m, int T, const float* Wr, const float* Xh, 
 __global__ void __launch_bounds__(256) k_ns_pinv(int m, int T, float eps, float alpha_in, const float* W,
                                                  float* Wr, float* P, float* Xh, NsHdr* hdr, float* X,
                                                  float* resid) {
-  __shared__ GemmSmem sm;
+  __shared__ NsSmem sm;
   __shared__ float red[2 * 256 + 8];
   const int b = blockIdx.x;
   const long long mm = (long long)m * m;
   W += b * mm; Wr += b * mm; P += b * mm; Xh += (long long)b * (T + 1) * mm; hdr += b;
-  ns_forward_dev(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red);
+  ns_forward_dev<false>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red);
   const float* XT = Xh + (long long)T * mm;
   if (X) for (long long e = threadIdx.x; e < mm; e += 256) X[b * mm + e] = XT[e];
   if (resid) {
-    cta_gemm<false, false>(m, m, m, Wr, m, XT, m, P, m, 1.f, 0.f, nullptr, sm);
+    ns_gemm<false, false, false>(m, m, m, Wr, m, XT, m, P, m, 1.f, 0.f, nullptr, 0.f, sm);
     float part = 0.f;
     for (long long e = threadIdx.x; e < mm; e += 256) {
       const int i = (int)(e / m), j = (int)(e % m);
@@ -791,16 +798,16 @@ __global__ void __launch_bounds__(256) k_ns_pinv_bwd(int m, int T, float eps, fl
                                                      float* Wr, float* P, float* Hm, float* Ga, float* Gb,
                                                      float* Xh_scratch, const float* Xh_given, NsHdr* hdr,
                                                      const float* dX, float* dW) {
-  __shared__ GemmSmem sm;
+  __shared__ NsSmem sm;
   __shared__ float red[2 * 256 + 8];
   const int b = blockIdx.x;
   const long long mm = (long long)m * m;
   W += b * mm; Wr += b * mm; P += b * mm; Hm += b * mm; Ga += b * mm; Gb += b * mm; hdr += b;
   float* Xs = Xh_scratch + (long long)b * (T + 1) * mm;
   // T = 0 when the history is given: only Wr, the norms and alpha are rebuilt
-  ns_forward_dev(m, Xh_given ? 0 : T, eps, alpha_in, W, Wr, P, Xs, hdr, sm, red);
+  ns_forward_dev<false>(m, Xh_given ? 0 : T, eps, alpha_in, W, Wr, P, Xs, hdr, sm, red);
   const float* Xh = Xh_given ? Xh_given + (long long)b * (T + 1) * mm : Xs;
-  ns_backward_dev(m, T, Wr, Xh, hdr, dX + b * mm, dW + b * mm, P, Hm, Ga, Gb, sm, red);
+  ns_backward_dev<false>(m, T, Wr, Xh, hdr, dX + b * mm, dW + b * mm, P, Hm, Ga, Gb, sm, red);
 }
 
 // =====================================================================================
@@ -808,12 +815,14 @@ __global__ void __launch_bounds__(256) k_ns_pinv_bwd(int m, int T, float eps, fl
 // then fold the injective map (Prop. 3) into Ytilde_l = s_l Y_l - mean_l'(s_l' Y_l'), ybar = mean_l Y_l
 // so that O = (C - mu) Ytilde + ybar.  One CTA per head.
 // =====================================================================================
-template <int D>
+template <int D, bool TC, int MP>
 __global__ void __launch_bounds__(256) k_mid_fwd(int m, int T, float eps, float alpha_in, int H, int map_mode,
                                                  const float* __restrict__ whiten, const float* W, float* Wr,
                                                  float* P, float* Xh, NsHdr* hdr, const float* Mpart, int nchunks,
                                                  float* Mout, float* Y, float* Yt, float* ybar, int* dev_status) {
-  __shared__ GemmSmem sm;
+  // dynamic shared memory: the Newton-Schulz matrices (MP > 0), reused afterwards by the GEMM engine
+  extern __shared__ __align__(16) unsigned char dyn_smem[];
+  NsSmem& sm = *reinterpret_cast<NsSmem*>(dyn_smem);
   __shared__ float red[2 * 256 + 8];
   const int bh = blockIdx.x, tid = threadIdx.x;
   const long long mm = (long long)m * m, md = (long long)m * D;
@@ -825,7 +834,12 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int T, float eps, float 
     for (int p = 0; p < nchunks; ++p) s += Mpart[p * md + e];
     Mout[e] = s;
   }
-  ns_forward_dev(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red);
+  if constexpr (MP > 0) {
+    ns_forward_smem<MP>(m, T, eps, alpha_in, W, Xh, hdr, reinterpret_cast<bf16*>(dyn_smem), red);
+    __syncthreads();
+  } else {
+    ns_forward_dev<TC>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red);
+  }
   const float* XT = Xh + (long long)T * mm;
   if (dev_status) {
     float bad = 0.f;
@@ -833,7 +847,7 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int T, float eps, float 
     bad = block_sum(bad, red);
     if (tid == 0) dev_status[bh] = bad > 0.f ? 1 : 0;
   }
-  cta_gemm<false, false>(m, D, m, XT, m, Mout, D, Y, D, 1.f, 0.f, nullptr, sm);      // Y = X M
+  ns_gemm<TC, false, false>(m, D, m, XT, m, Mout, D, Y, D, 1.f, 0.f, nullptr, 0.f, sm);   // Y = X M
   const float* s = whiten ? whiten + (long long)(bh % H) * m : nullptr;
   if (tid < D) {
     const int c = tid;
@@ -856,14 +870,15 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int T, float eps, float 
 // and GW = (dW o K_LL + (dW o K_LL)^T) / lambda, the symmetrised upstream of the landmark block,
 // so that dL_l -= sum_l' GW[l][l'] sign(L_l - L_l').
 // =====================================================================================
-template <int D>
+template <int D, bool TC, int MP>
 __global__ void __launch_bounds__(256) k_mid_bwd(int m, int T, int H, int map_mode, float inv_lambda, int ldm,
                                                  const float* __restrict__ whiten, const float* W,
                                                  const float* Xh, const NsHdr* hdr, const float* Msaved,
                                                  const float* dYtpart, const float* dybpart, int nchunks,
                                                  float eps, float* Wr, float* P, float* Hm, float* Ga, float* Gb,
                                                  float* dWm, float* dXm, float* dY, float* dM, float* GW) {
-  __shared__ GemmSmem sm;
+  extern __shared__ __align__(16) unsigned char dyn_smem[];
+  NsSmem& sm = *reinterpret_cast<NsSmem*>(dyn_smem);
   __shared__ float red[2 * 256 + 8];
   const int bh = blockIdx.x, tid = threadIdx.x;
   const long long mm = (long long)m * m, md = (long long)m * D;
@@ -892,9 +907,10 @@ __global__ void __launch_bounds__(256) k_mid_bwd(int m, int T, int H, int map_mo
   }
   __syncthreads();
   const float* XT = Xh + (long long)T * mm;
-  cta_gemm<false, true>(m, m, D, dY, D, Msaved, D, dXm, m, 1.f, 0.f, nullptr, sm);   // dX = dY M^T
-  cta_gemm<true, false>(m, D, m, XT, m, dY, D, dM, D, 1.f, 0.f, nullptr, sm);        // dM = X^T dY
-  ns_backward_dev(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red);
+  ns_gemm<TC, false, true>(m, m, D, dY, D, Msaved, D, dXm, m, 1.f, 0.f, nullptr, 0.f, sm);   // dX = dY M^T
+  ns_gemm<TC, true, false>(m, D, m, XT, m, dY, D, dM, D, 1.f, 0.f, nullptr, 0.f, sm);        // dM = X^T dY
+  if constexpr (MP > 0) ns_backward_smem<MP>(m, T, eps, W, Xh, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
+  else ns_backward_dev<TC>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red);
   for (long long e = tid; e < (long long)m * ldm; e += 256) {
     const int i = (int)(e / ldm), j = (int)(e % ldm);
     float v = 0.f;

@@ -345,4 +345,109 @@ __global__ void __launch_bounds__(256) k_nt_g_mma(const bf16* __restrict__ U, co
   }
 }
 
+// =====================================================================================
+// Whole-CTA GEMM on global (L2-resident) row-major fp32 matrices with tensor cores:
+//   C = beta * Cin + alpha * op(A) op(B) (+ diag on the diagonal),  op(A) is M x K, op(B) is K x N.
+// Operands are staged in K-chunks of 32 through shared memory in their stored orientation, split
+// into bf16 hi + lo on the way in (three MMAs per product: hi*hi, hi*lo, lo*hi), accumulated in
+// fp32 registers.  The next chunk is fetched into registers while the current one is multiplied.
+// Executed by all 256 threads (8 warps = 4 row blocks of 16 x 2 column halves of 32 per 64 x 64
+// output tile); ends with __syncthreads().  Cin may equal C.
+// =====================================================================================
+struct __align__(16) MmaGemmSmem {
+  bf16 Ah[2560], Al[2560], Bh[2560], Bl[2560];   // [64][40] or [32][72] bf16
+};
+
+// Stage geometry: "row-chunk" form = 64 rows x 32 cols ([64][40]); "col-chunk" form = 32 rows x 64 cols ([32][72]).
+// 8 floats per thread: thread -> (row, 8 consecutive columns).
+template <bool WIDE>   // WIDE: 32 x 64 (col-chunk), else 64 x 32 (row-chunk)
+__device__ __forceinline__ void gemm_fetch(const float* src, int ld, int r0, int c0, int rmax, int cmax, float (&v)[8]) {
+  const int tid = threadIdx.x;
+  const int r = WIDE ? (tid >> 3) : (tid >> 2);
+  const int c = WIDE ? (tid & 7) * 8 : (tid & 3) * 8;
+  const int gr = r0 + r, gc = c0 + c;
+  const float* p = src + (long long)gr * ld + gc;
+  if (gr < rmax && gc + 7 < cmax && (ld & 3) == 0 && (gc & 3) == 0) {
+    const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  } else {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) v[q] = (gr < rmax && gc + q < cmax) ? p[q] : 0.f;
+  }
+}
+template <bool WIDE>
+__device__ __forceinline__ void gemm_stash(bf16* hi, bf16* lo, const float (&v)[8]) {
+  const int tid = threadIdx.x;
+  const int r = WIDE ? (tid >> 3) : (tid >> 2);
+  const int c = WIDE ? (tid & 7) * 8 : (tid & 3) * 8;
+  constexpr int LD = WIDE ? 72 : 40;
+  uint2 h0, l0, h1, l1;
+  split4(make_float4(v[0], v[1], v[2], v[3]), h0, l0);
+  split4(make_float4(v[4], v[5], v[6], v[7]), h1, l1);
+  *reinterpret_cast<uint4*>(hi + r * LD + c) = make_uint4(h0.x, h0.y, h1.x, h1.y);
+  *reinterpret_cast<uint4*>(lo + r * LD + c) = make_uint4(l0.x, l0.y, l1.x, l1.y);
+}
+
+template <bool TRA, bool TRB>
+__device__ void cta_gemm_mma(int M, int N, int K, const float* A, int lda, const float* Bm, int ldb, float* C,
+                             int ldc, float alpha, float beta, const float* Cin, float diag, MmaGemmSmem& sm) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int wm = (warp & 3) * 16, wn = (warp >> 2) * 32;
+  const int g = lane >> 2, t4 = lane & 3;
+  for (int i0 = 0; i0 < M; i0 += 64)
+    for (int j0 = 0; j0 < N; j0 += 64) {
+      float acc[4][4];
+#pragma unroll
+      for (int t = 0; t < 4; ++t)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[t][q] = 0.f;
+      float va[8], vb[8];
+      // op(A) = A: stored [M][K] -> row-chunk form; op(A) = A^T: stored [K][M] -> col-chunk form
+      if (TRA) gemm_fetch<true>(A, lda, 0, i0, K, M, va); else gemm_fetch<false>(A, lda, i0, 0, M, K, va);
+      // op(B) = B: stored [K][N] -> col-chunk form; op(B) = B^T: stored [N][K] -> row-chunk form
+      if (TRB) gemm_fetch<false>(Bm, ldb, j0, 0, N, K, vb); else gemm_fetch<true>(Bm, ldb, 0, j0, K, N, vb);
+      for (int k0 = 0; k0 < K; k0 += 32) {
+        __syncthreads();
+        gemm_stash<TRA>(sm.Ah, sm.Al, va);
+        gemm_stash<!TRB>(sm.Bh, sm.Bl, vb);
+        __syncthreads();
+        if (k0 + 32 < K) {
+          if (TRA) gemm_fetch<true>(A, lda, k0 + 32, i0, K, M, va); else gemm_fetch<false>(A, lda, i0, k0 + 32, M, K, va);
+          if (TRB) gemm_fetch<false>(Bm, ldb, j0, k0 + 32, N, K, vb); else gemm_fetch<true>(Bm, ldb, k0 + 32, j0, K, N, vb);
+        }
+#pragma unroll
+        for (int kk = 0; kk < 32; kk += 16) {
+          uint32_t ah[4], al[4];
+          if (TRA) { ldsm_x4_t(ah, addr_at(sm.Ah, 72, kk, wm)); ldsm_x4_t(al, addr_at(sm.Al, 72, kk, wm)); }
+          else     { ldsm_x4(ah, addr_a(sm.Ah, 40, wm, kk));    ldsm_x4(al, addr_a(sm.Al, 40, wm, kk)); }
+#pragma unroll
+          for (int t = 0; t < 4; t += 2) {
+            uint32_t bh4[4], bl4[4];
+            if (TRB) { ldsm_x4(bh4, addr_b(sm.Bh, 40, wn + t * 8, kk));    ldsm_x4(bl4, addr_b(sm.Bl, 40, wn + t * 8, kk)); }
+            else     { ldsm_x4_t(bh4, addr_bt(sm.Bh, 72, kk, wn + t * 8)); ldsm_x4_t(bl4, addr_bt(sm.Bl, 72, kk, wn + t * 8)); }
+            mma_bf16(acc[t], al, bh4[0], bh4[1]);
+            mma_bf16(acc[t], ah, bl4[0], bl4[1]);
+            mma_bf16(acc[t], ah, bh4[0], bh4[1]);
+            mma_bf16(acc[t + 1], al, bh4[2], bh4[3]);
+            mma_bf16(acc[t + 1], ah, bl4[2], bl4[3]);
+            mma_bf16(acc[t + 1], ah, bh4[2], bh4[3]);
+          }
+        }
+      }
+#pragma unroll
+      for (int t = 0; t < 4; ++t)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int i = i0 + wm + g + (q >> 1) * 8, j = j0 + wn + t * 8 + 2 * t4 + (q & 1);
+          if (i < M && j < N) {
+            float v = alpha * acc[t][q];
+            if (beta != 0.f) v += beta * Cin[(long long)i * ldc + j];
+            if (i == j) v += diag;
+            C[(long long)i * ldc + j] = v;
+          }
+        }
+    }
+  __syncthreads();
+}
+
 }  // namespace ln
