@@ -159,7 +159,7 @@ def l1_lane_ops(cfg, kernel):
     """Algorithmic FP32 lane-operations of one launch of an l1 kernel: 2 per (pair, dim) in the forward
     (subtract, accumulate |.|), all heads."""
     BH = cfg.B * cfg.H
-    pairs = {"l1_C": cfg.n * cfg.m, "l1_R": cfg.n * cfg.m, "l1_W": cfg.m * cfg.m}[kernel]
+    pairs = {"l1_CRW": 2 * cfg.n * cfg.m + cfg.m * cfg.m}[kernel]
     return 2.0 * cfg.d * pairs * BH
 
 
@@ -267,7 +267,7 @@ def run_ours(args):
     total_traced = sum(v[1] for v in per.values())
     kernels = {k: {"launches_per_step": v[0] // args.steps, "avg_us": 1e3 * v[1] / v[0], "share": v[1] / total_traced}
                for k, v in sorted(per.items(), key=lambda kv: -kv[1][1])}
-    dom = max((k for k in per if k in ("l1_C", "l1_R")), key=lambda k: per[k][1])
+    dom = "l1_CRW"
     dom_avg_s = per[dom][1] / per[dom][0] * 1e-3
     achieved = l1_lane_ops(cfg, dom) / dom_avg_s / 1e12
     roofline = {"bound": "alu", "kernel": dom, "achieved": achieved, "peak": ALU_PEAK_TLANEOPS, "unit": "Tlane-op/s",

@@ -121,6 +121,8 @@ int validate(const ln_problem* p) {
     if ((long long)p->prefix + (long long)p->gh * p->gw != p->n) return LN_ERR_ARG;
     if ((long long)p->mh * p->mw != p->m) return LN_ERR_ARG;
     if (p->mh > p->gh || p->mw > p->gw) return LN_ERR_ARG;
+    if ((long long)p->gh * (p->mh + 1) >= (1ll << 31) || (long long)p->gw * (p->mw + 1) >= (1ll << 31)) return LN_ERR_UNSUPPORTED;
+    if ((long long)p->n * p->d / 4 >= (1ll << 32)) return LN_ERR_UNSUPPORTED;
   }
   if ((long long)p->B * p->H > 65535) return LN_ERR_UNSUPPORTED;
   if (p->d != 32 && p->d != 64 && p->d != 128) return LN_ERR_UNSUPPORTED;
@@ -158,13 +160,47 @@ struct TraceScope {
 };
 #define LN_LAUNCH(name, st, ...) do { TraceScope ts_(name, st); __VA_ARGS__; } while (0)
 
+// Tile of the l1 kernel for a problem: LG landmark groups of 4 (<= 16), TG token groups of 8,
+// LG * TG <= 256 threads (two CTAs per SM), chosen so that the tiles hug the problem.
+struct L1Launch { dim3 grid, block; size_t smem; };
+L1Launch plan_l1(int na_max, int nb, int batch, int nprob) {
+  int LG = (nb + 3) / 4; if (LG > 16) LG = 16; if (LG < 1) LG = 1;
+  int tg_cap = 256 / LG; if (tg_cap > 32) tg_cap = 32;       // at most 256 tokens per tile
+  const int groups = (na_max + 7) / 8;
+  const int tiles = (groups + tg_cap - 1) / tg_cap;
+  int TG = (groups + tiles - 1) / tiles; if (TG < 1) TG = 1;
+  L1Launch l;
+  l.block = dim3(LG, TG);
+  l.grid = dim3((na_max + 8 * TG - 1) / (8 * TG), batch, nprob);
+  l.smem = sizeof(float) * ((size_t)(8 * TG + 4 * LG) * L1_PITCH + (size_t)8 * TG * LG);
+  return l;
+}
+
+template <typename T> constexpr int is_f32() { return std::is_same<T, float>::value ? 1 : 0; }
+
+L1Prob l1_prob(const void* A, int a_f32, float* E, float* rowsum, int na, int d, int lde, float rs_scale) {
+  L1Prob q; q.A = A; q.E = E; q.rowsum = rowsum; q.sA = (long long)na * d; q.sE = (long long)na * lde;
+  q.na = na; q.lde = lde; q.a_f32 = a_f32; q.rs_scale = rs_scale;
+  return q;
+}
+
+void launch_l1_args(const char* name, L1Args& a, int nprob, int batch, cudaStream_t st) {
+  int na_max = 0;
+  for (int i = 0; i < nprob; ++i) na_max = a.p[i].na > na_max ? a.p[i].na : na_max;
+  const L1Launch l = plan_l1(na_max, a.nb, batch, nprob);
+  cudaFuncSetAttribute(k_l1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.smem);
+  LN_LAUNCH(name, st, k_l1<<<l.grid, l.block, l.smem, st>>>(a));
+}
+
 template <typename TA, typename TB>
 void launch_l1(const char* name, const TA* A, const TB* Bm, float* E, float* rowsum, int batch, int na, int nb, int d,
                int lde, float lambda, cudaStream_t st, float rs_scale = 1.f) {
-  const float nscale = -1.4426950408889634f / lambda;
-  dim3 grid(cdiv(na, L1_TA), batch);
-  LN_LAUNCH(name, st, k_l1<TA, TB><<<grid, 256, 0, st>>>(A, Bm, E, rowsum, na, nb, d, (long long)na * d, (long long)nb * d,
-                                     (long long)na * lde, lde, nscale, rs_scale));
+  L1Args a;
+  a.p[0] = l1_prob(A, is_f32<TA>(), E, rowsum, na, d, lde, rs_scale);
+  a.p[1] = a.p[0]; a.p[2] = a.p[0];
+  a.Bm = Bm; a.sB = (long long)nb * d; a.nb = nb; a.d = d; a.b_f32 = is_f32<TB>();
+  a.nscale = -1.4426950408889634f / lambda;
+  launch_l1_args(name, a, 1, batch, st);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -174,16 +210,21 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const int BH = pl.BH, n = pl.n, m = pl.m;
   // landmarks (Sec. 4.2)
   if (p->lm_mode == 1) {
-    LN_LAUNCH("k_pool", st, k_pool<T><<<dim3(m, BH), 128, 0, st>>>(K, x.Lf, geom_of(p)));
+    LN_LAUNCH("k_pool", st, k_pool<T><<<dim3(cdiv(m, 256 / (D / 4)), BH), 256, 0, st>>>(K, x.Lf, geom_of(p)));
   } else {
     const long long cnt = (long long)BH * m * D;
     LN_LAUNCH("k_to_f32", st, k_to_f32<T><<<cdiv(cnt, 256), 256, 0, st>>>(L, x.Lf, cnt));
   }
   // the three kernel blocks: C = k(Q,L) with its row sums, R^T = k(K,L), W = k(L,L)
-  launch_l1<T, float>("l1_C", Q, x.Lf, x.C, p->map_mode == 1 ? x.mu : nullptr, BH, n, m, D, pl.ldm, p->lambda, st,
-                      1.f / (float)m);   // row means (Prop. 3 step 2)
-  launch_l1<T, float>("l1_R", K, x.Lf, x.Rt, nullptr, BH, n, m, D, pl.ldm, p->lambda, st);
-  launch_l1<float, float>("l1_W", x.Lf, x.Lf, x.W, nullptr, BH, m, m, D, m, p->lambda, st);
+  {
+    L1Args a;
+    a.p[0] = l1_prob(Q, is_f32<T>(), x.C, p->map_mode == 1 ? x.mu : nullptr, n, D, pl.ldm, 1.f / (float)m);  // row means (Prop. 3 step 2)
+    a.p[1] = l1_prob(K, is_f32<T>(), x.Rt, nullptr, n, D, pl.ldm, 1.f);
+    a.p[2] = l1_prob(x.Lf, 1, x.W, nullptr, m, D, m, 1.f);
+    a.Bm = x.Lf; a.sB = (long long)m * D; a.nb = m; a.d = D; a.b_f32 = 1;
+    a.nscale = -1.4426950408889634f / p->lambda;
+    launch_l1_args("l1_CRW", a, 3, BH, st);
+  }
   // M = R V, partial over token chunks
   if constexpr (std::is_same<T, bf16>::value)
     LN_LAUNCH("tn_M", st, k_tn_mma<D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, w.Mpart, nullptr, n, m, pl.rpc));
@@ -236,6 +277,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
                                                           w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW));
     };
     if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 5 * NsTile<64>::mat_bytes);
+    else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * NsTile<128>::mat_bytes + kStage128Bytes);
     else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
   }
   LN_LAUNCH("sign_rows_dLW", st, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, st>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));
@@ -252,10 +294,10 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // landmark gradient and its way back to the keys
   const int md = m * D;
   if (p->lm_mode == 1) {
-    LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 256), BH), 256, 0, st>>>(w.dLCpart, ch, w.dLRpart, ch, w.dLW, 1, w.dLtot, md));
+    LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, ch, w.dLRpart, ch, w.dLW, 1, w.dLtot, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256), BH), 256, 0, st>>>(w.dKpart, w.dLtot, dK, geom_of(p), 1));
   } else {
-    LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(md, 256), BH), 256, 0, st>>>(w.dLCpart, ch, w.dLRpart, ch, w.dLW, 1, dL, md));
+    LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, ch, w.dLRpart, ch, w.dLW, 1, dL, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256), BH), 256, 0, st>>>(w.dKpart, nullptr, dK, geom_of(p), 0));
   }
   return launch_ok();
@@ -319,7 +361,7 @@ void l1_bwd_impl(int batch, int na, int nb, const T* A, const T* Bm, float lambd
   LN_LAUNCH("k_g_elem", st, k_g_elem<<<cdiv(cnt, 256), 256, 0, st>>>(Kmat, dK, w.G, cnt, 1.f / lambda));
   LN_LAUNCH("k_sign_rows", st, k_sign_rows<T, T, T, D><<<dim3(cdiv(na, 64), batch), 256, 0, st>>>(A, Bm, w.G, nb, dA, na, nb));
   LN_LAUNCH("k_sign_cols", st, k_sign_cols<T, T, D><<<dim3(w.chunks, cdiv(nb, 64), batch), 256, 0, st>>>(A, Bm, w.G, nb, w.part, na, nb, w.rpc));
-  LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(nb * D, 256), batch), 256, 0, st>>>(w.part, w.chunks, nullptr, 0, nullptr, 0, dB, nb * D));
+  LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(nb * D, 1024), batch), 256, 0, st>>>(w.part, w.chunks, nullptr, 0, nullptr, 0, dB, nb * D));
 }
 }  // namespace
 
@@ -545,9 +587,9 @@ int landmarks_pool(const ln_problem* p, const void* K, float* L, void* stream) {
   if (s != LN_OK) return s;
   if (p->lm_mode != 1 || !K || !L || !aligned16(K) || !aligned16(L)) return LN_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  dim3 grid(p->m, p->B * p->H);
-  if (p->dtype == LN_F32) LN_LAUNCH("k_pool", st, k_pool<float><<<grid, 128, 0, st>>>((const float*)K, L, geom_of(p)));
-  else LN_LAUNCH("k_pool", st, k_pool<bf16><<<grid, 128, 0, st>>>((const bf16*)K, L, geom_of(p)));
+  dim3 grid(cdiv(p->m, 256 / (p->d / 4)), p->B * p->H);
+  if (p->dtype == LN_F32) LN_LAUNCH("k_pool", st, k_pool<float><<<grid, 256, 0, st>>>((const float*)K, L, geom_of(p)));
+  else LN_LAUNCH("k_pool", st, k_pool<bf16><<<grid, 256, 0, st>>>((const bf16*)K, L, geom_of(p)));
   return launch_ok();
 }
 

@@ -55,6 +55,25 @@ __device__ __forceinline__ float half_step(float t) {
   return r;
 }
 
+// Sum of nparts partial arrays (fixed order p = 0, 1, ...), four consecutive elements at `off`.
+// Eight independent loads are issued per batch so that their latencies overlap.
+__device__ __forceinline__ float4 sum_parts4(const float* __restrict__ parts, int nparts, long long stride, long long off) {
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  int p = 0;
+  for (; p + 8 <= nparts; p += 8) {
+    float4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = *reinterpret_cast<const float4*>(parts + (long long)(p + u) * stride + off);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
+  }
+  for (; p < nparts; ++p) {
+    const float4 v = *reinterpret_cast<const float4*>(parts + (long long)p * stride + off);
+    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+  }
+  return s;
+}
+
 // Column set a thread owns in a [rows x D] tile worked on by 16 column-threads: DC = D/16
 // columns, laid out so that the 16 threads read one contiguous 256-byte (128 for D = 32) run.
 template <int D> struct ColMap {

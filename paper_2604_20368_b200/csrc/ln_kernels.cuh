@@ -10,106 +10,151 @@ namespace ln {
 
 // =====================================================================================
 // Laplacian kernel block (Sec. 1, Eq. 8):  E[i][j] = exp(-sum_c |a_ic - b_jc| / lambda)
-// CTA: 128 rows of A x (all of B in blocks of 64); thread: 8 x 4 pairs; d in chunks of 32
-// staged in shared memory dimension-major so one 128-bit load serves four rows.
+//
+// Block = (LG, TG) threads: thread (tj, ti) owns the 8 x 4 pairs of tokens ti + TG*k (k < 8) and
+// landmarks tj + LG*q (q < 4) of a (8 TG) x (4 LG) tile, so the tile follows the problem size
+// (n = 197, m = 49 run as one 200 x 52 tile per head instead of two 128 x 64 tiles).  Operands
+// are staged in shared memory token-major as fp32 in chunks of 32 dims straight from coalesced
+// 16-byte global loads (no transpose); a thread reads four dims of a row with one 128-bit load.
+// Per (pair, dim) the work is two FP32 instructions: subtract, add |.|.
+// Up to three problems that share the landmark operand (C = k(Q,L), R^T = k(K,L), W = k(L,L)) go
+// in one launch (blockIdx.z).
 // =====================================================================================
-constexpr int L1_TA = 128, L1_TB = 64, L1_DC = 32;
+constexpr int L1_DC = 32;            // dims per staged chunk
+constexpr int L1_PITCH = L1_DC + 4;  // floats per staged row
 
-template <typename TA, typename TB>
-__global__ void __launch_bounds__(256) k_l1(const TA* __restrict__ A, const TB* __restrict__ Bm,
-                                            float* __restrict__ E, float* __restrict__ rowsum, int na, int nb, int d,
-                                            long long sA, long long sB, long long sE, int lde, float nscale,
-                                            float rs_scale) {
-  __shared__ __align__(16) float As[L1_DC][L1_TA + 4];
-  __shared__ __align__(16) float Bs[L1_DC][L1_TB + 4];
-  const int b = blockIdx.y, i0 = blockIdx.x * L1_TA;
-  A += (long long)b * sA;
-  Bm += (long long)b * sB;
-  E += (long long)b * sE;
-  const int tid = threadIdx.x, tj = tid & 15, ti = tid >> 4;
+struct L1Prob {
+  const void* A; float* E; float* rowsum;
+  long long sA, sE;      // per-batch strides of A (elements) and E
+  int na, lde, a_f32;
+  float rs_scale;
+};
+struct L1Args {
+  L1Prob p[3];
+  const void* Bm; long long sB;
+  int nb, d, b_f32;
+  float nscale;          // -log2(e) / lambda
+};
+
+// 8 consecutive elements of a row -> fp32 (zero outside [0, d)); vec: the row start is 16-byte aligned
+__device__ __forceinline__ void l1_fetch8(const void* base, bool f32, long long row_off, int c, int d, bool vec, float (&v)[8]) {
+  if (f32) {
+    const float* p = reinterpret_cast<const float*>(base) + row_off + c;
+    if (vec && c + 8 <= d) {
+      const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+      v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    } else {
+#pragma unroll
+      for (int q = 0; q < 8; ++q) v[q] = (c + q < d) ? p[q] : 0.f;
+    }
+  } else {
+    const bf16* p = reinterpret_cast<const bf16*>(base) + row_off + c;
+    if (vec && c + 8 <= d) {
+      const uint4 r = *reinterpret_cast<const uint4*>(p);
+      const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) { v[2 * q] = __uint_as_float(w[q] << 16); v[2 * q + 1] = __uint_as_float(w[q] & 0xffff0000u); }
+    } else {
+#pragma unroll
+      for (int q = 0; q < 8; ++q) v[q] = (c + q < d) ? __bfloat162float(p[q]) : 0.f;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256, 2) k_l1(const L1Args args) {
+  extern __shared__ __align__(16) float l1_smem[];
+  const L1Prob pr = args.p[blockIdx.z];
+  const int LG = blockDim.x, TG = blockDim.y, tj = threadIdx.x, ti = threadIdx.y;
+  const int tid = ti * LG + tj, nthr = LG * TG;
+  const int TA = 8 * TG, TB = 4 * LG;
+  const int i0 = blockIdx.x * TA, b = blockIdx.y;
+  if (i0 >= pr.na) return;
+  float* As = l1_smem;                    // [TA][L1_PITCH]
+  float* Bs = l1_smem + TA * L1_PITCH;    // [TB][L1_PITCH]
+  float* Rs = Bs + TB * L1_PITCH;         // [TA][LG] row-sum partials
+  const int na = pr.na, nb = args.nb, d = args.d, lde = pr.lde;
   const bool vec = (d % 8) == 0;
+  float* E = pr.E + (long long)b * pr.sE;
   float rs[8];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) rs[i] = 0.f;
+  for (int k = 0; k < 8; ++k) rs[k] = 0.f;
 
-  for (int j0 = 0; j0 < nb; j0 += L1_TB) {
+  for (int j0 = 0; j0 < nb; j0 += TB) {
     float acc[8][4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int k = 0; k < 8; ++k)
 #pragma unroll
-      for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+      for (int q = 0; q < 4; ++q) acc[k][q] = 0.f;
 
     for (int c0 = 0; c0 < d; c0 += L1_DC) {
       __syncthreads();
-      {  // A chunk: 128 rows x 32 dims; thread = (row, 16-dim half)
-        const int r = tid & 127, cb = (tid >> 7) * 16, gi = i0 + r;
-        const TA* src = A + (long long)gi * d + c0 + cb;
-        if (vec && gi < na && c0 + cb + 16 <= d) {
+      for (int idx = tid; idx < TA * 4; idx += nthr) {     // A chunk: TA rows x 4 pieces of 8 dims
+        const int r = idx >> 2, c8 = (idx & 3) * 8, gi = i0 + r;
+        float v[8];
+        if (gi < na) l1_fetch8(pr.A, pr.a_f32, (long long)b * pr.sA + (long long)gi * d, c0 + c8, d, vec, v);
+        else {
 #pragma unroll
-          for (int k = 0; k < 16; k += 4) {
-            float4 v = ld4(src + k);
-            As[cb + k][r] = v.x; As[cb + k + 1][r] = v.y; As[cb + k + 2][r] = v.z; As[cb + k + 3][r] = v.w;
-          }
-        } else {
-#pragma unroll 4
-          for (int k = 0; k < 16; ++k) As[cb + k][r] = (gi < na && c0 + cb + k < d) ? to_f(src[k]) : 0.f;
+          for (int q = 0; q < 8; ++q) v[q] = 0.f;
         }
+        *reinterpret_cast<float4*>(As + r * L1_PITCH + c8) = make_float4(v[0], v[1], v[2], v[3]);
+        *reinterpret_cast<float4*>(As + r * L1_PITCH + c8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
       }
-      {  // B chunk: 64 rows x 32 dims; thread = (row, 8-dim quarter)
-        const int r = tid & 63, cb = (tid >> 6) * 8, gj = j0 + r;
-        const TB* src = Bm + (long long)gj * d + c0 + cb;
-        if (vec && gj < nb && c0 + cb + 8 <= d) {
+      for (int idx = tid; idx < TB * 4; idx += nthr) {     // B chunk
+        const int r = idx >> 2, c8 = (idx & 3) * 8, gj = j0 + r;
+        float v[8];
+        if (gj < nb) l1_fetch8(args.Bm, args.b_f32, (long long)b * args.sB + (long long)gj * d, c0 + c8, d, vec, v);
+        else {
 #pragma unroll
-          for (int k = 0; k < 8; k += 4) {
-            float4 v = ld4(src + k);
-            Bs[cb + k][r] = v.x; Bs[cb + k + 1][r] = v.y; Bs[cb + k + 2][r] = v.z; Bs[cb + k + 3][r] = v.w;
-          }
-        } else {
-#pragma unroll 4
-          for (int k = 0; k < 8; ++k) Bs[cb + k][r] = (gj < nb && c0 + cb + k < d) ? to_f(src[k]) : 0.f;
+          for (int q = 0; q < 8; ++q) v[q] = 0.f;
         }
+        *reinterpret_cast<float4*>(Bs + r * L1_PITCH + c8) = make_float4(v[0], v[1], v[2], v[3]);
+        *reinterpret_cast<float4*>(Bs + r * L1_PITCH + c8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
       }
       __syncthreads();
-#pragma unroll 8
-      for (int c = 0; c < L1_DC; ++c) {
-        const float4 a0 = *reinterpret_cast<const float4*>(&As[c][ti * 8]);
-        const float4 a1 = *reinterpret_cast<const float4*>(&As[c][ti * 8 + 4]);
-        const float4 bb = *reinterpret_cast<const float4*>(&Bs[c][tj * 4]);
-        const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-        const float bv[4] = {bb.x, bb.y, bb.z, bb.w};
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
+      for (int c4 = 0; c4 < L1_DC; c4 += 4) {
+        float4 a[8], bv[4];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) acc[i][j] += fabsf(a[i] - bv[j]);
+        for (int k = 0; k < 8; ++k) a[k] = *reinterpret_cast<const float4*>(As + (ti + TG * k) * L1_PITCH + c4);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) bv[q] = *reinterpret_cast<const float4*>(Bs + (tj + LG * q) * L1_PITCH + c4);
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            acc[k][q] += fabsf(a[k].x - bv[q].x);
+            acc[k][q] += fabsf(a[k].y - bv[q].y);
+            acc[k][q] += fabsf(a[k].z - bv[q].z);
+            acc[k][q] += fabsf(a[k].w - bv[q].w);
+          }
       }
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int gi = i0 + ti * 8 + i;
+    for (int k = 0; k < 8; ++k) {
+      const int gi = i0 + ti + TG * k;
       if (gi >= na) continue;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int gj = j0 + tj * 4 + j;
+      for (int q = 0; q < 4; ++q) {
+        const int gj = j0 + tj + LG * q;
         if (gj < nb) {
-          const float e = ex2(acc[i][j] * nscale);
+          const float e = ex2(acc[k][q] * args.nscale);
           E[(long long)gi * lde + gj] = e;
-          rs[i] += e;
+          rs[k] += e;
         } else if (gj < lde) {
           E[(long long)gi * lde + gj] = 0.f;   // padding columns of a padded leading dimension
         }
       }
     }
   }
-  if (rowsum) {
+  if (pr.rowsum) {      // fixed-order reduction over the LG threads of a row
+    __syncthreads();
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      float v = rs[i];
-      v += __shfl_xor_sync(0xffffffffu, v, 1);
-      v += __shfl_xor_sync(0xffffffffu, v, 2);
-      v += __shfl_xor_sync(0xffffffffu, v, 4);
-      v += __shfl_xor_sync(0xffffffffu, v, 8);
-      const int gi = i0 + ti * 8 + i;
-      if (tj == 0 && gi < na) rowsum[(long long)b * na + gi] = v * rs_scale;
+    for (int k = 0; k < 8; ++k) Rs[(ti + TG * k) * LG + tj] = rs[k];
+    __syncthreads();
+    for (int r = tid; r < TA; r += nthr) {
+      float v = 0.f;
+      for (int t = 0; t < LG; ++t) v += Rs[r * LG + t];
+      if (i0 + r < na) pr.rowsum[(long long)b * na + i0 + r] = v * pr.rs_scale;
     }
   }
 }
@@ -124,13 +169,17 @@ template <typename T> __global__ void k_to_f32(const T* __restrict__ x, float* _
 // Landmark selection: adaptive average pooling of the keys over the token grid (Sec. 4.2)
 // =====================================================================================
 struct PoolGeom { int n, d, m, prefix, gh, gw, mh, mw; };
-__host__ __device__ inline int bin_lo(int a, int g, int mb) { return (int)(((long long)a * g) / mb); }
-__host__ __device__ inline int bin_hi(int a, int g, int mb) { return (int)((((long long)(a + 1)) * g + mb - 1) / mb); }
+// 32-bit on purpose (64-bit division costs two orders of magnitude more on the device); the host
+// checks that gh * mh and gw * mw stay below 2^31.
+__host__ __device__ inline int bin_lo(int a, int g, int mb) { return (int)(((unsigned)a * (unsigned)g) / (unsigned)mb); }
+__host__ __device__ inline int bin_hi(int a, int g, int mb) { return (int)(((unsigned)(a + 1) * (unsigned)g + (unsigned)mb - 1u) / (unsigned)mb); }
 
+// grid (ceil(m / (256 / (d/4))), BH); thread = (landmark, 4 dims)
 template <typename T>
-__global__ void k_pool(const T* __restrict__ K, float* __restrict__ L, PoolGeom g) {
-  const int l = blockIdx.x, bh = blockIdx.y, c = threadIdx.x;
-  if (c >= g.d) return;
+__global__ void __launch_bounds__(256) k_pool(const T* __restrict__ K, float* __restrict__ L, PoolGeom g) {
+  const int quads = g.d / 4, lpb = 256 / quads;
+  const int l = blockIdx.x * lpb + (int)threadIdx.x / quads, bh = blockIdx.y, c = ((int)threadIdx.x % quads) * 4;
+  if (l >= g.m || (int)threadIdx.x >= lpb * quads) return;
   const int a = l / g.mw, bb = l % g.mw;
   const int r0 = bin_lo(a, g.gh, g.mh), r1 = bin_hi(a, g.gh, g.mh);
   const int c0 = bin_lo(bb, g.gw, g.mw), c1 = bin_hi(bb, g.gw, g.mw);
@@ -138,10 +187,15 @@ __global__ void k_pool(const T* __restrict__ K, float* __restrict__ L, PoolGeom 
   // The mean is accumulated in double and rounded once, so that the stored landmark is the fp32
   // value nearest to the exact mean: sign(token - landmark) in the backward pass then does not
   // depend on the order of a single-precision summation.
-  double s = 0.0;
+  double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
   for (int r = r0; r < r1; ++r)
-    for (int q = c0; q < c1; ++q) s += (double)to_f(Kh[(long long)(g.prefix + r * g.gw + q) * g.d + c]);
-  L[((long long)bh * g.m + l) * g.d + c] = (float)(s / (double)((r1 - r0) * (c1 - c0)));
+    for (int q = c0; q < c1; ++q) {
+      const float4 v = ld4(Kh + (long long)(g.prefix + r * g.gw + q) * g.d + c);
+      s0 += (double)v.x; s1 += (double)v.y; s2 += (double)v.z; s3 += (double)v.w;
+    }
+  const double cnt = (double)((r1 - r0) * (c1 - c0));
+  st4(L + ((long long)bh * g.m + l) * g.d + c,
+      make_float4((float)(s0 / cnt), (float)(s1 / cnt), (float)(s2 / cnt), (float)(s3 / cnt)));
 }
 
 // dK[j] = dKpart[j] (may be NULL) + sum over the bins containing token j of dL[bin] / |bin|
@@ -150,16 +204,16 @@ template <typename T>
 __global__ void k_pool_bwd(const float* __restrict__ dKpart, const float* __restrict__ dL, T* __restrict__ dK,
                            PoolGeom g, int pool) {
   const int bh = blockIdx.y;
-  const int per_row = g.d / 4;
-  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (long long)g.n * per_row) return;
+  const unsigned per_row = g.d / 4;
+  const unsigned idx = blockIdx.x * blockDim.x + threadIdx.x;     // n * d / 4 < 2^32
+  if (idx >= (unsigned)g.n * per_row) return;
   const int j = (int)(idx / per_row), c = (int)(idx % per_row) * 4;
   float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
   if (dKpart) v = ld4(dKpart + ((long long)bh * g.n + j) * g.d + c);
   if (pool && j >= g.prefix) {
     const int r = (j - g.prefix) / g.gw, q = (j - g.prefix) % g.gw;
-    int a_lo = (int)(((long long)r * g.mh) / g.gh) - 1; if (a_lo < 0) a_lo = 0;
-    int b_lo = (int)(((long long)q * g.mw) / g.gw) - 1; if (b_lo < 0) b_lo = 0;
+    int a_lo = (int)(((unsigned)r * (unsigned)g.mh) / (unsigned)g.gh) - 1; if (a_lo < 0) a_lo = 0;
+    int b_lo = (int)(((unsigned)q * (unsigned)g.mw) / (unsigned)g.gw) - 1; if (b_lo < 0) b_lo = 0;
     for (int a = a_lo; a < g.mh && a <= a_lo + 2; ++a) {
       const int r0 = bin_lo(a, g.gh, g.mh), r1 = bin_hi(a, g.gh, g.mh);
       if (r < r0 || r >= r1) continue;
@@ -175,18 +229,17 @@ __global__ void k_pool_bwd(const float* __restrict__ dKpart, const float* __rest
   st4(dK + ((long long)bh * g.n + j) * g.d + c, v);
 }
 
-// out[e] = sum_p parts[p][e] for up to three part arrays laid out [BH][np][count]
+// out[e] = sum_p parts[p][e] for up to three part arrays laid out [BH][np][count]; count % 4 == 0
 template <typename TO>
 __global__ void k_reduce3(const float* __restrict__ p0, int n0, const float* __restrict__ p1, int n1,
                           const float* __restrict__ p2, int n2, TO* __restrict__ out, int count) {
   const int bh = blockIdx.y;
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  const int e = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (e >= count) return;
-  float s = 0.f;
-  for (int p = 0; p < n0; ++p) s += p0[((long long)bh * n0 + p) * count + e];
-  for (int p = 0; p < n1; ++p) s += p1[((long long)bh * n1 + p) * count + e];
-  for (int p = 0; p < n2; ++p) s += p2[((long long)bh * n2 + p) * count + e];
-  out[(long long)bh * count + e] = from_f<TO>(s);
+  float4 s = sum_parts4(p0 + (long long)bh * n0 * count, n0, count, e);
+  if (n1 > 0) { const float4 t = sum_parts4(p1 + (long long)bh * n1 * count, n1, count, e); s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w; }
+  if (n2 > 0) { const float4 t = sum_parts4(p2 + (long long)bh * n2 * count, n2, count, e); s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w; }
+  st4(out + (long long)bh * count + e, s);
 }
 
 // =====================================================================================
@@ -477,8 +530,9 @@ __global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, c
       }
     }
     __syncthreads();
+    const int lcount = min(32, (m - l0 + 3) & ~3);     // landmarks of this chunk, rounded up to 4 (the rest is zero)
 #pragma unroll 2
-    for (int ll = 0; ll < 32; ll += 4) {
+    for (int ll = 0; ll < lcount; ll += 4) {
       float g[4][4];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
@@ -553,8 +607,9 @@ __global__ void __launch_bounds__(256) k_sign_cols(const TT* __restrict__ tok, c
       }
     }
     __syncthreads();
+    const int jcount = min(32, iend - j0);
 #pragma unroll 4
-    for (int jj = 0; jj < 32; ++jj) {
+    for (int jj = 0; jj < jcount; ++jj) {
       const float4 g4 = *reinterpret_cast<const float4*>(&Gs[jj][tl * 4]);
       const float g[4] = {g4.x, g4.y, g4.z, g4.w};
       float tv[DC];
@@ -829,11 +884,8 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int T, float eps, float 
   W += bh * mm; Wr += bh * mm; P += bh * mm; Xh += (long long)bh * (T + 1) * mm; hdr += bh;
   Mout += bh * md; Y += bh * md; Yt += bh * md; ybar += (long long)bh * D;
   Mpart += (long long)bh * nchunks * md;
-  for (long long e = tid; e < md; e += 256) {
-    float s = 0.f;
-    for (int p = 0; p < nchunks; ++p) s += Mpart[p * md + e];
-    Mout[e] = s;
-  }
+  for (long long e = (long long)tid * 4; e < md; e += 1024)
+    *reinterpret_cast<float4*>(Mout + e) = sum_parts4(Mpart, nchunks, md, e);
   if constexpr (MP > 0) {
     ns_forward_smem<MP>(m, T, eps, alpha_in, W, Xh, hdr, reinterpret_cast<bf16*>(dyn_smem), red);
     __syncthreads();
@@ -894,12 +946,17 @@ __global__ void __launch_bounds__(256) k_mid_bwd(int m, int T, int H, int map_mo
     dyb[tid] = t;
   }
   __syncthreads();
-  for (long long e = tid; e < md; e += 256) {
-    float t = 0.f;
-    for (int p = 0; p < nchunks; ++p) t += dYtpart[p * md + e];
+  for (long long e = (long long)tid * 4; e < md; e += 1024) {
+    const float4 t = sum_parts4(dYtpart, nchunks, md, e);
     const int l = (int)(e / D), c = (int)(e % D);
     // Ytilde = P_c diag(s) Y, ybar = Y^T 1/m  ->  dY = diag(s) (centred Z'^T dO) + (1/m) 1 dyb^T
-    dY[e] = (map_mode == 1) ? (s ? s[l] : 1.f) * t + dyb[c] / (float)m : t;
+    float4 o = t;
+    if (map_mode == 1) {
+      const float sl = s ? s[l] : 1.f, im = 1.f / (float)m;
+      o.x = sl * t.x + dyb[c] * im; o.y = sl * t.y + dyb[c + 1] * im;
+      o.z = sl * t.z + dyb[c + 2] * im; o.w = sl * t.w + dyb[c + 3] * im;
+    }
+    *reinterpret_cast<float4*>(dY + e) = o;
   }
   for (long long e = tid; e < mm; e += 256) {
     const int i = (int)(e / m), j = (int)(e % m);
@@ -909,7 +966,8 @@ __global__ void __launch_bounds__(256) k_mid_bwd(int m, int T, int H, int map_mo
   const float* XT = Xh + (long long)T * mm;
   ns_gemm<TC, false, true>(m, m, D, dY, D, Msaved, D, dXm, m, 1.f, 0.f, nullptr, 0.f, sm);   // dX = dY M^T
   ns_gemm<TC, true, false>(m, D, m, XT, m, dY, D, dM, D, 1.f, 0.f, nullptr, 0.f, sm);        // dM = X^T dY
-  if constexpr (MP > 0) ns_backward_smem<MP>(m, T, eps, W, Xh, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
+  if constexpr (MP == 64) ns_backward_smem<64>(m, T, eps, W, Xh, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
+  else if constexpr (MP == 128) ns_backward_smem128(m, T, eps, W, Xh, hdr, dXm, dWm, Ga, Gb, reinterpret_cast<bf16*>(dyn_smem), red);
   else ns_backward_dev<TC>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red);
   for (long long e = tid; e < (long long)m * ldm; e += 256) {
     const int i = (int)(e / ldm), j = (int)(e % ldm);

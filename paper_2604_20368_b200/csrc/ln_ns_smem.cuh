@@ -36,29 +36,43 @@ __device__ __forceinline__ void smem_gemm(float (&acc)[NsTile<MP>::MT][NsTile<MP
 #pragma unroll
         for (int q = 0; q < 4; ++q) acc[a][t][q] = 0.f;
   }
+  // all fragments of a k-step are fetched before its MMAs are issued, so the loads of the next
+  // step overlap the tensor-core work of this one
 #pragma unroll 2
   for (int k0 = 0; k0 < MP; k0 += 16) {
-    uint32_t ah[MT][4], al[MT][4];
+    uint32_t ah[MT][4], al[MT][4], bh4[NT / 2][4], bl4[NT / 2][4];
 #pragma unroll
     for (int a = 0; a < MT; ++a) {
       if (TRA) { ldsm_x4_t(ah[a], addr_at(A, LD, k0, wm + a * 16)); ldsm_x4_t(al[a], addr_at(A + MAT, LD, k0, wm + a * 16)); }
       else     { ldsm_x4(ah[a], addr_a(A, LD, wm + a * 16, k0));    ldsm_x4(al[a], addr_a(A + MAT, LD, wm + a * 16, k0)); }
     }
 #pragma unroll
-    for (int t = 0; t < NT; t += 2) {
-      uint32_t bh4[4], bl4[4];
-      if (TRB) { ldsm_x4(bh4, addr_b(Bm, LD, wn + t * 8, k0));    ldsm_x4(bl4, addr_b(Bm + MAT, LD, wn + t * 8, k0)); }
-      else     { ldsm_x4_t(bh4, addr_bt(Bm, LD, k0, wn + t * 8)); ldsm_x4_t(bl4, addr_bt(Bm + MAT, LD, k0, wn + t * 8)); }
-#pragma unroll
-      for (int a = 0; a < MT; ++a) {
-        mma_bf16(acc[a][t], al[a], bh4[0], bh4[1]);
-        mma_bf16(acc[a][t], ah[a], bl4[0], bl4[1]);
-        mma_bf16(acc[a][t], ah[a], bh4[0], bh4[1]);
-        mma_bf16(acc[a][t + 1], al[a], bh4[2], bh4[3]);
-        mma_bf16(acc[a][t + 1], ah[a], bl4[2], bl4[3]);
-        mma_bf16(acc[a][t + 1], ah[a], bh4[2], bh4[3]);
-      }
+    for (int t = 0; t < NT / 2; ++t) {
+      if (TRB) { ldsm_x4(bh4[t], addr_b(Bm, LD, wn + t * 16, k0));    ldsm_x4(bl4[t], addr_b(Bm + MAT, LD, wn + t * 16, k0)); }
+      else     { ldsm_x4_t(bh4[t], addr_bt(Bm, LD, k0, wn + t * 16)); ldsm_x4_t(bl4[t], addr_bt(Bm + MAT, LD, k0, wn + t * 16)); }
     }
+    // three passes (lo*hi, hi*lo, hi*hi) so that consecutive MMAs hit different accumulators
+#pragma unroll
+    for (int a = 0; a < MT; ++a)
+#pragma unroll
+      for (int t = 0; t < NT / 2; ++t) {
+        mma_bf16(acc[a][2 * t], al[a], bh4[t][0], bh4[t][1]);
+        mma_bf16(acc[a][2 * t + 1], al[a], bh4[t][2], bh4[t][3]);
+      }
+#pragma unroll
+    for (int a = 0; a < MT; ++a)
+#pragma unroll
+      for (int t = 0; t < NT / 2; ++t) {
+        mma_bf16(acc[a][2 * t], ah[a], bl4[t][0], bl4[t][1]);
+        mma_bf16(acc[a][2 * t + 1], ah[a], bl4[t][2], bl4[t][3]);
+      }
+#pragma unroll
+    for (int a = 0; a < MT; ++a)
+#pragma unroll
+      for (int t = 0; t < NT / 2; ++t) {
+        mma_bf16(acc[a][2 * t], ah[a], bh4[t][0], bh4[t][1]);
+        mma_bf16(acc[a][2 * t + 1], ah[a], bh4[t][2], bh4[t][3]);
+      }
   }
 }
 
@@ -107,22 +121,35 @@ __device__ __forceinline__ void frag_to_global(const float (&acc)[NsTile<MP>::MT
       }
 }
 
-// global fp32 [m][m] (+ diag on the diagonal, times scale, optionally transposed) -> shared hi/lo, zero padded
+// global fp32 [m][m] (+ diag on the diagonal, times scale, optionally transposed) -> shared hi/lo, zero padded.
+// Eight independent loads are issued before anything is stored, so their latencies overlap.
 template <int MP>
-__device__ __forceinline__ void global_to_smem(const float* src, int m, float diag, float scale, bool transpose, bf16* dst) {
+__device__ __forceinline__ void global_to_smem(const float* __restrict__ src, int m, float diag, float scale, bool transpose,
+                                               bf16* dst) {
   using TL = NsTile<MP>;
-  for (int e = threadIdx.x; e < MP * MP; e += 256) {
-    const int i = e / MP, j = e % MP;
-    float v = 0.f;
-    if (i < m && j < m) {
-      v = transpose ? src[(long long)j * m + i] : src[(long long)i * m + j];
-      if (i == j) v += diag;
-      v *= scale;
+  constexpr int PER = MP * MP / 256;       // elements per thread
+#pragma unroll 1
+  for (int b0 = 0; b0 < PER; b0 += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int e = (b0 + u) * 256 + threadIdx.x, i = e / MP, j = e % MP;
+      float x = 0.f;
+      if (i < m && j < m) {
+        x = transpose ? src[(long long)j * m + i] : src[(long long)i * m + j];
+        if (i == j) x += diag;
+        x *= scale;
+      }
+      v[u] = x;
     }
-    bf16 h, l;
-    split2(v, h, l);
-    dst[i * TL::LD + j] = h;
-    dst[TL::MAT + i * TL::LD + j] = l;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int e = (b0 + u) * 256 + threadIdx.x, i = e / MP, j = e % MP;
+      bf16 h, l;
+      split2(v[u], h, l);
+      dst[i * TL::LD + j] = h;
+      dst[TL::MAT + i * TL::LD + j] = l;
+    }
   }
 }
 
@@ -281,6 +308,196 @@ __device__ void ns_backward_smem(int m, int T, float eps, const float* W, const 
           dW[(long long)i * m + j] = v;
         }
       }
+  __syncthreads();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Adjoint for 64 < m <= 128.  Five hi/lo matrices of 128 x 128 do not fit in one SM's shared
+// memory, so three stay resident (A = X_k, G, and H which is later reused for P) while W, which
+// only ever appears as the left operand (W A and W^T H), is streamed from global memory (L2) in
+// K-chunks of 32 through a small staging buffer.  G and dW are kept in fp32 in global memory and
+// touched fragment-wise (each thread reads and writes only its own elements).
+// smem: 3 * NsTile<128>::mat_bytes + kStage128Bytes.
+// ---------------------------------------------------------------------------------------------
+constexpr int kStageEl = 128 * 40;                                    // bf16 elements of one staged part (hi or lo)
+constexpr size_t kStage128Bytes = (size_t)2 * kStageEl * sizeof(bf16);
+
+// acc (+)= op(W + eps I) B, W [m][m] in global memory, B resident ([K][N], hi/lo); TRA: op = transpose
+template <bool TRA>
+__device__ void smem_gemm_stream_w(float (&acc)[2][8][4], const float* W, int m, float eps, bf16* stage, const bf16* Bm,
+                                   bool accumulate) {
+  using TL = NsTile<128>;
+  const int tid = threadIdx.x, wm = TL::wm(), wn = TL::wn();
+  if (!accumulate) {
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+      for (int t = 0; t < 8; ++t)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[a][t][q] = 0.f;
+  }
+  // row-chunk form (TRA = false): stage[128][40], thread -> (row tid/2, 16 cols); chunk = W[:, k0..k0+31]
+  // col-chunk form (TRA = true) : stage[32][136], thread -> (row tid/8, 16 cols); chunk = W[k0..k0+31, :]
+  const int r = TRA ? (tid >> 3) : (tid >> 1), cb = TRA ? (tid & 7) * 16 : (tid & 1) * 16;
+  constexpr int LDS_ = TRA ? 136 : 40;
+  float v[16];
+  auto fetch = [&](int k0) {
+    const int gr = TRA ? k0 + r : r, gc = TRA ? cb : k0 + cb;
+#pragma unroll
+    for (int q = 0; q < 16; ++q) {
+      const int cc = gc + q;
+      float x = (gr < m && cc < m) ? W[(long long)gr * m + cc] : 0.f;
+      if (gr == cc && gr < m) x += eps;
+      v[q] = x;
+    }
+  };
+  fetch(0);
+  for (int k0 = 0; k0 < 128; k0 += 32) {
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 16; q += 4) {
+      uint2 h, l;
+      split4(make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]), h, l);
+      *reinterpret_cast<uint2*>(stage + r * LDS_ + cb + q) = h;
+      *reinterpret_cast<uint2*>(stage + kStageEl + r * LDS_ + cb + q) = l;
+    }
+    __syncthreads();
+    if (k0 + 32 < 128) fetch(k0 + 32);
+#pragma unroll
+    for (int kk = 0; kk < 32; kk += 16) {
+      uint32_t ah[2][4], al[2][4];
+#pragma unroll
+      for (int a = 0; a < 2; ++a) {
+        if (TRA) { ldsm_x4_t(ah[a], addr_at(stage, 136, kk, wm + a * 16)); ldsm_x4_t(al[a], addr_at(stage + kStageEl, 136, kk, wm + a * 16)); }
+        else     { ldsm_x4(ah[a], addr_a(stage, 40, wm + a * 16, kk));     ldsm_x4(al[a], addr_a(stage + kStageEl, 40, wm + a * 16, kk)); }
+      }
+      uint32_t bh4[4][4], bl4[4][4];
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        ldsm_x4_t(bh4[t], addr_bt(Bm, TL::LD, k0 + kk, wn + t * 16));
+        ldsm_x4_t(bl4[t], addr_bt(Bm + TL::MAT, TL::LD, k0 + kk, wn + t * 16));
+      }
+#pragma unroll
+      for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          mma_bf16(acc[a][2 * t], al[a], bh4[t][0], bh4[t][1]);
+          mma_bf16(acc[a][2 * t + 1], al[a], bh4[t][2], bh4[t][3]);
+        }
+#pragma unroll
+      for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          mma_bf16(acc[a][2 * t], ah[a], bl4[t][0], bl4[t][1]);
+          mma_bf16(acc[a][2 * t + 1], ah[a], bl4[t][2], bl4[t][3]);
+        }
+#pragma unroll
+      for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          mma_bf16(acc[a][2 * t], ah[a], bh4[t][0], bh4[t][1]);
+          mma_bf16(acc[a][2 * t + 1], ah[a], bh4[t][2], bh4[t][3]);
+        }
+    }
+  }
+  __syncthreads();
+}
+
+// Gf, T1: global fp32 [m][m] scratch.  dW: output (global fp32 [m][m]).
+__device__ void ns_backward_smem128(int m, int T, float eps, const float* W, const float* Xh, const NsHdr* hdr,
+                                    const float* G0, float* dW, float* Gf, float* T1, bf16* smem, float* red) {
+  using TL = NsTile<128>;
+  constexpr int MP = 128;
+  bf16* sA = smem; bf16* sG = smem + 2 * TL::MAT; bf16* sH = smem + 4 * TL::MAT; bf16* stage = smem + 6 * TL::MAT;
+  const long long mm = (long long)m * m;
+  float acc[2][8][4];
+  for (long long e = threadIdx.x; e < mm; e += 256) { Gf[e] = G0[e]; dW[e] = 0.f; }
+  global_to_smem<MP>(G0, m, 0.f, 1.f, false, sG);
+  for (int k = T - 1; k >= 0; --k) {
+    __syncthreads();
+    global_to_smem<MP>(Xh + (long long)k * mm, m, 0.f, 1.f, false, sA);     // A = X_k
+    __syncthreads();
+    smem_gemm<MP, true, false>(acc, sA, sG, false);                        // H = A^T G
+    frag_to_smem<MP>(acc, sH);
+    __syncthreads();
+    smem_gemm<MP, false, true>(acc, sH, sA, false);                        // H A^T
+    // dW -= H A^T on this thread's own elements; all loads of a tile row are issued before the stores
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+      float old[8][4];
+#pragma unroll
+      for (int t = 0; t < 8; ++t)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          int i, j;
+          frag_ij<MP>(a, t, q, i, j);
+          old[t][q] = (i < m && j < m) ? dW[(long long)i * m + j] : 0.f;
+        }
+#pragma unroll
+      for (int t = 0; t < 8; ++t)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          int i, j;
+          frag_ij<MP>(a, t, q, i, j);
+          if (i < m && j < m) dW[(long long)i * m + j] = old[t][q] - acc[a][t][q];
+        }
+    }
+    smem_gemm_stream_w<true>(acc, W, m, eps, stage, sH, false);             // W^T H
+    frag_to_global<MP>(acc, T1, m);
+    smem_gemm_stream_w<false>(acc, W, m, eps, stage, sA, false);            // P = W A
+    frag_to_smem<MP>(acc, sH);                                             // H is dead: its buffer takes P
+    __syncthreads();
+    smem_gemm<MP, false, true>(acc, sG, sH, false);                        // G P^T
+    __syncthreads();                                                       // every warp is done reading sG
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+      float g0[8][4], t1[8][4];
+#pragma unroll
+      for (int t = 0; t < 8; ++t)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          int i, j;
+          frag_ij<MP>(a, t, q, i, j);
+          const bool in = i < m && j < m;
+          g0[t][q] = in ? Gf[(long long)i * m + j] : 0.f;
+          t1[t][q] = in ? T1[(long long)i * m + j] : 0.f;
+        }
+#pragma unroll
+      for (int t = 0; t < 8; ++t)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          int i, j;
+          frag_ij<MP>(a, t, q, i, j);
+          const float gn = 2.f * g0[t][q] - acc[a][t][q] - t1[t][q];   // 2G - G P^T - W^T H
+          if (i < m && j < m) Gf[(long long)i * m + j] = gn;
+          acc[a][t][q] = (i < m && j < m) ? gn : 0.f;
+        }
+    }
+    frag_to_smem<MP>(acc, sG);
+  }
+  __syncthreads();
+  // acc holds G in fragment layout when T > 0; reload it so that T = 0 works too
+  const float alpha = hdr->alpha;
+  float part = 0.f;
+  for (long long e = threadIdx.x; e < mm; e += 256) {
+    const int i = (int)(e / m), j = (int)(e % m);
+    part += Gf[e] * (W[(long long)j * m + i] + (i == j ? eps : 0.f));
+  }
+  const float dalpha = block_sum(part, red);
+  const bool aa = hdr->auto_alpha != 0;
+  const int js = hdr->jstar, is = hdr->istar;
+  const float c1 = dalpha * (-alpha / hdr->n1), c2 = dalpha * (-alpha / hdr->ninf);
+  for (long long e = threadIdx.x; e < mm; e += 256) {
+    const int i = (int)(e / m), j = (int)(e % m);
+    float v = dW[e] + alpha * Gf[(long long)j * m + i];
+    if (aa) {
+      const float w = W[e] + (i == j ? eps : 0.f);
+      const float sg = w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f);
+      if (j == js) v += c1 * sg;
+      if (i == is) v += c2 * sg;
+    }
+    dW[e] = v;
+  }
   __syncthreads();
 }
 
