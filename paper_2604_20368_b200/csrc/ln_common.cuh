@@ -55,6 +55,15 @@ __device__ __forceinline__ float half_step(float t) {
   return r;
 }
 
+// Packed pair arithmetic (two fp32 lanes per instruction): the FP32 pipe does not get faster, but a
+// pair costs one issue slot instead of two, which leaves slots for the shared-memory loads.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 add2(f32x2 x, f32x2 y) { f32x2 z; asm("add.f32x2 %0, %1, %2;" : "=l"(z) : "l"(x), "l"(y)); return z; }
+__device__ __forceinline__ f32x2 fma2(f32x2 x, f32x2 y, f32x2 c) { f32x2 z; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(z) : "l"(x), "l"(y), "l"(c)); return z; }
+__device__ __forceinline__ float lo32(f32x2 x) { return __uint_as_float((unsigned)x); }
+__device__ __forceinline__ float hi32(f32x2 x) { return __uint_as_float((unsigned)(x >> 32)); }
+__device__ __forceinline__ f32x2 pack2(float a, float b) { return (f32x2)__float_as_uint(a) | ((f32x2)__float_as_uint(b) << 32); }
+
 // Sum of nparts partial arrays (fixed order p = 0, 1, ...), four consecutive elements at `off`.
 // Eight independent loads are issued per batch so that their latencies overlap.
 __device__ __forceinline__ float4 sum_parts4(const float* __restrict__ parts, int nparts, long long stride, long long off) {
@@ -113,5 +122,25 @@ __device__ inline float block_sum(float v, float* red /* >= 8 floats of shared m
 
 // Header kept per matrix beside the Newton-Schulz iterates.
 struct NsHdr { float alpha, n1, ninf; int jstar, istar, auto_alpha, pad0, pad1; };
+
+// The same columns as ld_cols, as D/32 packed pairs of adjacent dims.
+template <int D> __device__ __forceinline__ void ld_col_pairs(const float* row, int tc, f32x2 (&v)[D / 32]) {
+  if (D == 32) {
+    v[0] = *reinterpret_cast<const f32x2*>(row + tc * 2);
+  } else {
+#pragma unroll
+    for (int h = 0; h < D / 64; ++h) {
+      const ulonglong2 a = *reinterpret_cast<const ulonglong2*>(row + h * 64 + tc * 4);
+      v[2 * h] = a.x; v[2 * h + 1] = a.y;
+    }
+  }
+}
+
+// acc += g * half_step(t) on a pair of dims: one packed add, two saturating multiply-adds, one packed
+// multiply-add (the saturating form has no packed variant).
+__device__ __forceinline__ f32x2 sign_step2(f32x2 x, f32x2 neg_y, f32x2 gg, f32x2 acc) {
+  const f32x2 t = add2(x, neg_y);
+  return fma2(gg, pack2(half_step(lo32(t)), half_step(hi32(t))), acc);
+}
 
 }  // namespace ln

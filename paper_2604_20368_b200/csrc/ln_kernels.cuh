@@ -107,25 +107,27 @@ __global__ void __launch_bounds__(256, 2) k_l1(const L1Args args) {
 #pragma unroll
           for (int q = 0; q < 8; ++q) v[q] = 0.f;
         }
-        *reinterpret_cast<float4*>(Bs + r * L1_PITCH + c8) = make_float4(v[0], v[1], v[2], v[3]);
-        *reinterpret_cast<float4*>(Bs + r * L1_PITCH + c8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
+        // the landmark operand is stored negated: a - b becomes one packed add per two dims
+        *reinterpret_cast<float4*>(Bs + r * L1_PITCH + c8) = make_float4(-v[0], -v[1], -v[2], -v[3]);
+        *reinterpret_cast<float4*>(Bs + r * L1_PITCH + c8 + 4) = make_float4(-v[4], -v[5], -v[6], -v[7]);
       }
       __syncthreads();
 #pragma unroll
       for (int c4 = 0; c4 < L1_DC; c4 += 4) {
-        float4 a[8], bv[4];
+        ulonglong2 a[8], nb[4];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) a[k] = *reinterpret_cast<const float4*>(As + (ti + TG * k) * L1_PITCH + c4);
+        for (int k = 0; k < 8; ++k) a[k] = *reinterpret_cast<const ulonglong2*>(As + (ti + TG * k) * L1_PITCH + c4);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) bv[q] = *reinterpret_cast<const float4*>(Bs + (tj + LG * q) * L1_PITCH + c4);
+        for (int q = 0; q < 4; ++q) nb[q] = *reinterpret_cast<const ulonglong2*>(Bs + (tj + LG * q) * L1_PITCH + c4);
 #pragma unroll
         for (int k = 0; k < 8; ++k)
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
-            acc[k][q] += fabsf(a[k].x - bv[q].x);
-            acc[k][q] += fabsf(a[k].y - bv[q].y);
-            acc[k][q] += fabsf(a[k].z - bv[q].z);
-            acc[k][q] += fabsf(a[k].w - bv[q].w);
+            const f32x2 t0 = add2(a[k].x, nb[q].x), t1 = add2(a[k].y, nb[q].y);   // dims c4, c4+1 and c4+2, c4+3
+            acc[k][q] += fabsf(lo32(t0));
+            acc[k][q] += fabsf(hi32(t0));
+            acc[k][q] += fabsf(lo32(t1));
+            acc[k][q] += fabsf(hi32(t1));
           }
       }
     }
@@ -502,15 +504,19 @@ __global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, c
   Lm += (long long)bh * m * D;
   G += (long long)bh * n * ldg;
   out += (long long)bh * n * D;
-  float q[4][DC], acc[4][DC], gsum[4];
+  constexpr int DP = DC / 2;                 // packed pairs of adjacent dims
+  f32x2 qp[4][DP], acc[4][DP];
+  float gsum[4];
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const int i = i0 + tt * 4 + k;
     gsum[k] = 0.f;
 #pragma unroll
-    for (int s = 0; s < DC; ++s) {
-      acc[k][s] = 0.f;
-      q[k][s] = (i < n) ? to_f(tok[(long long)i * D + ColMap<D>::col(tc, s)]) : 0.f;
+    for (int s = 0; s < DP; ++s) {
+      acc[k][s] = 0ull;
+      const float q0 = (i < n) ? to_f(tok[(long long)i * D + ColMap<D>::col(tc, 2 * s)]) : 0.f;
+      const float q1 = (i < n) ? to_f(tok[(long long)i * D + ColMap<D>::col(tc, 2 * s + 1)]) : 0.f;
+      qp[k][s] = pack2(q0, q1);
     }
   }
   for (int l0 = 0; l0 < m; l0 += 32) {
@@ -519,7 +525,7 @@ __global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, c
       const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
       float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
       if (l0 + r < m) v = ld4(Lm + (long long)(l0 + r) * D + c4);
-      *reinterpret_cast<float4*>(&Ls[r][c4]) = v;
+      *reinterpret_cast<float4*>(&Ls[r][c4]) = make_float4(-v.x, -v.y, -v.z, -v.w);   // negated: q - L is a packed add
     }
     {  // G tile: 64 tokens x 32 landmarks (zero outside)
       const int r = tid >> 2, cb = (tid & 3) * 8, i = i0 + r;
@@ -541,13 +547,14 @@ __global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, c
       }
 #pragma unroll
       for (int s = 0; s < 4; ++s) {
-        float lv[DC];
-        ld_cols<D>(&Ls[ll + s][0], tc, lv);
+        f32x2 nl[DP];
+        ld_col_pairs<D>(&Ls[ll + s][0], tc, nl);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           gsum[k] += g[k][s];
+          const f32x2 gg = pack2(g[k][s], g[k][s]);
 #pragma unroll
-          for (int c = 0; c < DC; ++c) acc[k][c] = fmaf(g[k][s], half_step(q[k][c] - lv[c]), acc[k][c]);
+          for (int c = 0; c < DP; ++c) acc[k][c] = sign_step2(qp[k][c], nl[c], gg, acc[k][c]);
         }
       }
     }
@@ -557,8 +564,10 @@ __global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, c
     const int i = i0 + tt * 4 + k;
     if (i < n)
 #pragma unroll
-      for (int c = 0; c < DC; ++c)
-        out[(long long)i * D + ColMap<D>::col(tc, c)] = from_f<TO>(gsum[k] - 2.f * acc[k][c]);
+      for (int c = 0; c < DP; ++c) {
+        out[(long long)i * D + ColMap<D>::col(tc, 2 * c)] = from_f<TO>(gsum[k] - 2.f * lo32(acc[k][c]));
+        out[(long long)i * D + ColMap<D>::col(tc, 2 * c + 1)] = from_f<TO>(gsum[k] - 2.f * hi32(acc[k][c]));
+      }
   }
 }
 
@@ -579,15 +588,19 @@ __global__ void __launch_bounds__(256) k_sign_cols(const TT* __restrict__ tok, c
   Lm += (long long)bh * m * D;
   G += (long long)bh * n * ldg;
   const int ibeg = chunk * rpc, iend = min(n, ibeg + rpc);
-  float lv[4][DC], acc[4][DC], gsum[4];
+  constexpr int DP = DC / 2;
+  f32x2 nl[4][DP], acc[4][DP];                // negated landmark values, accumulators, as pairs of adjacent dims
+  float gsum[4];
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const int l = l0 + tl * 4 + k;
     gsum[k] = 0.f;
 #pragma unroll
-    for (int s = 0; s < DC; ++s) {
-      acc[k][s] = 0.f;
-      lv[k][s] = (l < m) ? to_f(Lm[(long long)l * D + ColMap<D>::col(tc, s)]) : 0.f;
+    for (int s = 0; s < DP; ++s) {
+      acc[k][s] = 0ull;
+      const float v0 = (l < m) ? to_f(Lm[(long long)l * D + ColMap<D>::col(tc, 2 * s)]) : 0.f;
+      const float v1 = (l < m) ? to_f(Lm[(long long)l * D + ColMap<D>::col(tc, 2 * s + 1)]) : 0.f;
+      nl[k][s] = pack2(-v0, -v1);
     }
   }
   for (int j0 = ibeg; j0 < iend; j0 += 32) {
@@ -612,13 +625,14 @@ __global__ void __launch_bounds__(256) k_sign_cols(const TT* __restrict__ tok, c
     for (int jj = 0; jj < jcount; ++jj) {
       const float4 g4 = *reinterpret_cast<const float4*>(&Gs[jj][tl * 4]);
       const float g[4] = {g4.x, g4.y, g4.z, g4.w};
-      float tv[DC];
-      ld_cols<D>(&Ts[jj][0], tc, tv);
+      f32x2 tv[DP];
+      ld_col_pairs<D>(&Ts[jj][0], tc, tv);
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         gsum[k] += g[k];
+        const f32x2 gg = pack2(g[k], g[k]);
 #pragma unroll
-        for (int c = 0; c < DC; ++c) acc[k][c] = fmaf(g[k], half_step(tv[c] - lv[k][c]), acc[k][c]);
+        for (int c = 0; c < DP; ++c) acc[k][c] = sign_step2(tv[c], nl[k][c], gg, acc[k][c]);
       }
     }
   }
@@ -628,7 +642,10 @@ __global__ void __launch_bounds__(256) k_sign_cols(const TT* __restrict__ tok, c
     const int l = l0 + tl * 4 + k;
     if (l < m)
 #pragma unroll
-      for (int c = 0; c < DC; ++c) out[(long long)l * D + ColMap<D>::col(tc, c)] = 2.f * acc[k][c] - gsum[k];
+      for (int c = 0; c < DP; ++c) {
+        out[(long long)l * D + ColMap<D>::col(tc, 2 * c)] = 2.f * lo32(acc[k][c]) - gsum[k];
+        out[(long long)l * D + ColMap<D>::col(tc, 2 * c + 1)] = 2.f * hi32(acc[k][c]) - gsum[k];
+      }
   }
 }
 
