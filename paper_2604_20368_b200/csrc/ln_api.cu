@@ -45,7 +45,7 @@ bool make_plan(const ln_problem* p, Plan* pl) {
 }
 
 // Forward context (saved for the backward pass, or carved from ws for inference)
-struct Ctx { float *Lf, *C, *Rt, *mu, *W, *Xh, *M, *Yt, *ybar; NsHdr* hdr; size_t bytes; };
+struct Ctx { float *Lf, *C, *Rt, *mu, *W, *Xh, *Ph, *M, *Yt, *ybar; NsHdr* hdr; size_t bytes; };
 Ctx carve_ctx(const Plan& pl, void* base) {
   Carver c(base); Ctx x;
   const size_t BH = pl.BH, n = pl.n, d = pl.d, m = pl.m;
@@ -54,7 +54,8 @@ Ctx carve_ctx(const Plan& pl, void* base) {
   x.Rt = c.take(BH * n * pl.ldm);
   x.mu = c.take(BH * n);
   x.W = c.take(BH * m * m);
-  x.Xh = c.take(BH * (pl.T + 1) * m * m);
+  x.Xh = c.take(BH * (pl.T + 1) * m * pl.ldm);   // leading dimension ldm on the shared-memory path, m otherwise
+  x.Ph = c.take(BH * (pl.T > 0 ? pl.T : 1) * m * pl.ldm);   // W X_k of the forward pass (tensor-core path)
   x.M = c.take(BH * m * d);
   x.Yt = c.take(BH * m * d);
   x.ybar = c.take(BH * d);
@@ -68,8 +69,8 @@ FwdWs carve_fwd_ws(const Plan& pl, void* base) {
   Carver c(base); FwdWs w;
   const size_t BH = pl.BH, d = pl.d, m = pl.m;
   w.Mpart = c.take(BH * pl.chunks * m * d);
-  w.Wr = c.take(BH * m * m);
-  w.P = c.take(BH * m * m);
+  w.Wr = c.take(BH * m * pl.ldm);
+  w.P = c.take(BH * m * pl.ldm);
   w.Y = c.take(BH * m * d);
   w.bytes = c.off;
   return w;
@@ -89,13 +90,13 @@ BwdWs carve_bwd_ws(const Plan& pl, void* base) {
   w.dLRpart = c.take(BH * ch * m * d);
   w.dY = c.take(BH * m * d);
   w.dM = c.take(BH * m * d);
-  w.Wr = c.take(BH * m * m);
-  w.P = c.take(BH * m * m);
-  w.Hm = c.take(BH * m * m);
-  w.Ga = c.take(BH * m * m);
-  w.Gb = c.take(BH * m * m);
-  w.dW = c.take(BH * m * m);
-  w.dX = c.take(BH * m * m);
+  w.Wr = c.take(BH * m * pl.ldm);
+  w.P = c.take(BH * m * pl.ldm);
+  w.Hm = c.take(BH * m * pl.ldm);
+  w.Ga = c.take(BH * m * pl.ldm);
+  w.Gb = c.take(BH * m * pl.ldm);
+  w.dW = c.take(BH * m * pl.ldm);
+  w.dX = c.take(BH * m * pl.ldm);
   w.GW = c.take(BH * m * pl.ldm);
   w.dLW = c.take(BH * m * d);
   w.dLtot = c.take(BH * m * d);
@@ -235,8 +236,8 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     constexpr bool TC = std::is_same<T, bf16>::value;
     auto launch = [&](auto kern, size_t smem) {
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      LN_LAUNCH("k_mid_fwd", st, kern<<<BH, 256, smem, st>>>(m, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode, p->whiten,
-                                                          x.W, w.Wr, w.P, x.Xh, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt,
+      LN_LAUNCH("k_mid_fwd", st, kern<<<BH, 256, smem, st>>>(m, pl.ldm, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode, p->whiten,
+                                                          x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt,
                                                           x.ybar, dev_status));
     };
     if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * NsTile<64>::mat_bytes);
@@ -273,11 +274,11 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     auto launch = [&](auto kern, size_t smem) {
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       LN_LAUNCH("k_mid_bwd", st, kern<<<BH, 256, smem, st>>>(m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten, x.W, x.Xh,
-                                                          x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P, w.Hm,
+                                                          x.Ph, x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P, w.Hm,
                                                           w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW));
     };
-    if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 5 * NsTile<64>::mat_bytes);
-    else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * NsTile<128>::mat_bytes + kStage128Bytes);
+    if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 3 * NsTile<64>::mat_bytes);
+    else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * NsTile<128>::mat_bytes);
     else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
   }
   LN_LAUNCH("sign_rows_dLW", st, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, st>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));

@@ -888,9 +888,9 @@ __global__ void __launch_bounds__(256) k_ns_pinv_bwd(int m, int T, float eps, fl
 // so that O = (C - mu) Ytilde + ybar.  One CTA per head.
 // =====================================================================================
 template <int D, bool TC, int MP>
-__global__ void __launch_bounds__(256) k_mid_fwd(int m, int T, float eps, float alpha_in, int H, int map_mode,
+__global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float eps, float alpha_in, int H, int map_mode,
                                                  const float* __restrict__ whiten, const float* W, float* Wr,
-                                                 float* P, float* Xh, NsHdr* hdr, const float* Mpart, int nchunks,
+                                                 float* P, float* Xh, float* Ph, NsHdr* hdr, const float* Mpart, int nchunks,
                                                  float* Mout, float* Y, float* Yt, float* ybar, int* dev_status) {
   // dynamic shared memory: the Newton-Schulz matrices (MP > 0), reused afterwards by the GEMM engine
   extern __shared__ __align__(16) unsigned char dyn_smem[];
@@ -898,51 +898,66 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int T, float eps, float 
   __shared__ float red[2 * 256 + 8];
   const int bh = blockIdx.x, tid = threadIdx.x;
   const long long mm = (long long)m * m, md = (long long)m * D;
-  W += bh * mm; Wr += bh * mm; P += bh * mm; Xh += (long long)bh * (T + 1) * mm; hdr += bh;
+  // the iterate histories of the shared-memory path use the padded leading dimension (128-bit accesses)
+  const int ldx = (MP > 0) ? ldm : m;
+  const long long mx = (long long)m * ldx;
+  W += bh * mm; Wr += bh * mm; P += bh * mm; Xh += (long long)bh * (T + 1) * mx; hdr += bh;
+  if (Ph) Ph += (long long)bh * T * mx;
   Mout += bh * md; Y += bh * md; Yt += bh * md; ybar += (long long)bh * D;
   Mpart += (long long)bh * nchunks * md;
   for (long long e = (long long)tid * 4; e < md; e += 1024)
     *reinterpret_cast<float4*>(Mout + e) = sum_parts4(Mpart, nchunks, md, e);
   if constexpr (MP > 0) {
-    ns_forward_smem<MP>(m, T, eps, alpha_in, W, Xh, hdr, reinterpret_cast<bf16*>(dyn_smem), red);
+    ns_forward_smem<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, hdr, reinterpret_cast<bf16*>(dyn_smem), red);
     __syncthreads();
   } else {
     ns_forward_dev<TC>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red);
   }
-  const float* XT = Xh + (long long)T * mm;
+  const float* XT = Xh + (long long)T * mx;
   if (dev_status) {
     float bad = 0.f;
-    for (long long e = tid; e < mm; e += 256) bad += isfinite(XT[e]) ? 0.f : 1.f;
+    for (int e = tid; e < m * m; e += 256) bad += isfinite(XT[(long long)(e / m) * ldx + e % m]) ? 0.f : 1.f;
     bad = block_sum(bad, red);
     if (tid == 0) dev_status[bh] = bad > 0.f ? 1 : 0;
   }
-  ns_gemm<TC, false, false>(m, D, m, XT, m, Mout, D, Y, D, 1.f, 0.f, nullptr, 0.f, sm);   // Y = X M
+  ns_gemm<TC, false, false>(m, D, m, XT, ldx, Mout, D, Y, D, 1.f, 0.f, nullptr, 0.f, sm);   // Y = X M
   const float* s = whiten ? whiten + (long long)(bh % H) * m : nullptr;
+  // fold the injective map (Prop. 3): column means over the landmarks first (eight independent loads per
+  // batch), then every element in parallel
+  float* colstat = red;            // [2][D]: mean_l s_l Y_lc and mean_l Y_lc
   if (tid < D) {
-    const int c = tid;
-    if (map_mode == 1) {
-      float sy = 0.f, y1 = 0.f;
-      for (int l = 0; l < m; ++l) { const float y = Y[(long long)l * D + c]; sy += (s ? s[l] : 1.f) * y; y1 += y; }
-      sy /= (float)m;
-      for (int l = 0; l < m; ++l) Yt[(long long)l * D + c] = (s ? s[l] : 1.f) * Y[(long long)l * D + c] - sy;
-      ybar[c] = y1 / (float)m;
-    } else {
-      for (int l = 0; l < m; ++l) Yt[(long long)l * D + c] = Y[(long long)l * D + c];
-      ybar[c] = 0.f;
+    float sy = 0.f, y1 = 0.f;
+    for (int l0 = 0; l0 < m; l0 += 8) {
+      float y[8], w[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int l = l0 + u;
+        y[u] = (l < m) ? Y[(long long)l * D + tid] : 0.f;
+        w[u] = (l < m && s) ? s[l] : 1.f;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { sy += w[u] * y[u]; y1 += y[u]; }
     }
+    colstat[tid] = sy / (float)m;
+    colstat[D + tid] = y1 / (float)m;
+    ybar[tid] = (map_mode == 1) ? y1 / (float)m : 0.f;
+  }
+  __syncthreads();
+  for (long long e = (long long)tid * 4; e < md; e += 1024) {
+    const int l = (int)(e / D), c = (int)(e % D);
+    float4 y = *reinterpret_cast<const float4*>(Y + e);
+    if (map_mode == 1) {
+      const float sl = s ? s[l] : 1.f;
+      y.x = sl * y.x - colstat[c]; y.y = sl * y.y - colstat[c + 1];
+      y.z = sl * y.z - colstat[c + 2]; y.w = sl * y.w - colstat[c + 3];
+    }
+    *reinterpret_cast<float4*>(Yt + e) = y;
   }
 }
-
-// =====================================================================================
-// Per-head middle of the backward pass.  Inputs: partial sums of Z'^T dO and of the column sums
-// of dO over the token chunks; the forward context.  Outputs: dM (for dR = dM V^T, dV = R^T dM)
-// and GW = (dW o K_LL + (dW o K_LL)^T) / lambda, the symmetrised upstream of the landmark block,
-// so that dL_l -= sum_l' GW[l][l'] sign(L_l - L_l').
-// =====================================================================================
 template <int D, bool TC, int MP>
 __global__ void __launch_bounds__(256) k_mid_bwd(int m, int T, int H, int map_mode, float inv_lambda, int ldm,
                                                  const float* __restrict__ whiten, const float* W,
-                                                 const float* Xh, const NsHdr* hdr, const float* Msaved,
+                                                 const float* Xh, const float* Ph, const NsHdr* hdr, const float* Msaved,
                                                  const float* dYtpart, const float* dybpart, int nchunks,
                                                  float eps, float* Wr, float* P, float* Hm, float* Ga, float* Gb,
                                                  float* dWm, float* dXm, float* dY, float* dM, float* GW) {
@@ -951,8 +966,10 @@ __global__ void __launch_bounds__(256) k_mid_bwd(int m, int T, int H, int map_mo
   __shared__ float red[2 * 256 + 8];
   const int bh = blockIdx.x, tid = threadIdx.x;
   const long long mm = (long long)m * m, md = (long long)m * D;
-  W += bh * mm; Xh += (long long)bh * (T + 1) * mm; hdr += bh; Msaved += bh * md;
-  Wr += bh * mm; P += bh * mm; Hm += bh * mm; Ga += bh * mm; Gb += bh * mm; dWm += bh * mm; dXm += bh * mm;
+  const int ldx = (MP > 0) ? ldm : m;
+  const long long mx = (long long)m * ldx, ms = (long long)m * ldm;    // ms: size of one scratch matrix slot
+  W += bh * mm; Xh += (long long)bh * (T + 1) * mx; Ph += (long long)bh * T * mx; hdr += bh; Msaved += bh * md;
+  Wr += bh * ms; P += bh * ms; Hm += bh * ms; Ga += bh * ms; Gb += bh * ms; dWm += bh * ms; dXm += bh * ms;
   dY += bh * md; dM += bh * md; GW += (long long)bh * m * ldm;
   dYtpart += (long long)bh * nchunks * md; dybpart += (long long)bh * nchunks * D;
   const float* s = whiten ? whiten + (long long)(bh % H) * m : nullptr;
@@ -975,22 +992,31 @@ __global__ void __launch_bounds__(256) k_mid_bwd(int m, int T, int H, int map_mo
     }
     *reinterpret_cast<float4*>(dY + e) = o;
   }
-  for (long long e = tid; e < mm; e += 256) {
-    const int i = (int)(e / m), j = (int)(e % m);
-    Wr[e] = W[e] + (i == j ? eps : 0.f);
+  if constexpr (MP == 0) {
+    for (long long e = tid; e < mm; e += 256) {
+      const int i = (int)(e / m), j = (int)(e % m);
+      Wr[e] = W[e] + (i == j ? eps : 0.f);
+    }
   }
   __syncthreads();
-  const float* XT = Xh + (long long)T * mm;
-  ns_gemm<TC, false, true>(m, m, D, dY, D, Msaved, D, dXm, m, 1.f, 0.f, nullptr, 0.f, sm);   // dX = dY M^T
-  ns_gemm<TC, true, false>(m, D, m, XT, m, dY, D, dM, D, 1.f, 0.f, nullptr, 0.f, sm);        // dM = X^T dY
-  if constexpr (MP == 64) ns_backward_smem<64>(m, T, eps, W, Xh, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
-  else if constexpr (MP == 128) ns_backward_smem128(m, T, eps, W, Xh, hdr, dXm, dWm, Ga, Gb, reinterpret_cast<bf16*>(dyn_smem), red);
+  const float* XT = Xh + (long long)T * mx;
+  ns_gemm<TC, false, true>(m, m, D, dY, D, Msaved, D, dXm, ldx, 1.f, 0.f, nullptr, 0.f, sm);   // dX = dY M^T
+  ns_gemm<TC, true, false>(m, D, m, XT, ldx, dY, D, dM, D, 1.f, 0.f, nullptr, 0.f, sm);        // dM = X^T dY
+  if constexpr (MP > 0) ns_backward_smem<MP>(m, T, eps, W, Xh, Ph, ldx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
   else ns_backward_dev<TC>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red);
-  for (long long e = tid; e < (long long)m * ldm; e += 256) {
-    const int i = (int)(e / ldm), j = (int)(e % ldm);
-    float v = 0.f;
-    if (j < m) v = (dWm[(long long)i * m + j] * W[(long long)i * m + j] + dWm[(long long)j * m + i] * W[(long long)j * m + i]) * inv_lambda;
-    GW[e] = v;
+  // GW = (dW o K_LL + (dW o K_LL)^T) / lambda; four elements per batch so that the loads overlap
+  for (long long e0 = (long long)tid * 4; e0 < (long long)m * ldm; e0 += 1024) {
+    float a[4], b[4], c[4], d4[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const long long e = e0 + u;
+      const int i = (int)(e / ldm), j = (int)(e % ldm);
+      const bool in = j < m;
+      a[u] = in ? dWm[(long long)i * ldx + j] : 0.f;  b[u] = in ? W[(long long)i * m + j] : 0.f;
+      c[u] = in ? dWm[(long long)j * ldx + i] : 0.f;  d4[u] = in ? W[(long long)j * m + i] : 0.f;
+    }
+    *reinterpret_cast<float4*>(GW + e0) = make_float4((a[0] * b[0] + c[0] * d4[0]) * inv_lambda, (a[1] * b[1] + c[1] * d4[1]) * inv_lambda,
+                                                      (a[2] * b[2] + c[2] * d4[2]) * inv_lambda, (a[3] * b[3] + c[3] * d4[3]) * inv_lambda);
   }
 }
 

@@ -6,6 +6,9 @@
 // of X gives a zero row or column of X (2I - W X)).
 #pragma once
 #include "ln_mma.cuh"
+#ifdef LN_TIMING
+#include <cstdio>
+#endif
 
 namespace ln {
 
@@ -107,7 +110,7 @@ __device__ __forceinline__ void frag_to_smem(const float (&acc)[NsTile<MP>::MT][
 
 // registers (fragment layout) -> global fp32 [m][m]
 template <int MP>
-__device__ __forceinline__ void frag_to_global(const float (&acc)[NsTile<MP>::MT][NsTile<MP>::NT][4], float* dst, int m) {
+__device__ __forceinline__ void frag_to_global(const float (&acc)[NsTile<MP>::MT][NsTile<MP>::NT][4], float* dst, int m, int ld) {
   using TL = NsTile<MP>;
 #pragma unroll
   for (int a = 0; a < TL::MT; ++a)
@@ -117,7 +120,7 @@ __device__ __forceinline__ void frag_to_global(const float (&acc)[NsTile<MP>::MT
       for (int q = 0; q < 4; ++q) {
         int i, j;
         frag_ij<MP>(a, t, q, i, j);
-        if (i < m && j < m) dst[(long long)i * m + j] = acc[a][t][q];
+        if (i < m && j < m) dst[(long long)i * ld + j] = acc[a][t][q];
       }
 }
 
@@ -182,25 +185,73 @@ __device__ inline void ns_norms(int m, float eps, float alpha_in, const float* W
 }
 
 // Forward iteration.  smem: three matrices (W, X, P), 3 * NsTile<MP>::mat_bytes.  Xh (global, [T+1][m][m])
-// receives X_0 .. X_T in fp32.
+// receives X_0 .. X_T in fp32; Ph (global, [T][m][m], may be NULL) receives W X_0 .. W X_{T-1}; both with
+// leading dimension ld >= m.
 template <int MP>
-__device__ void ns_forward_smem(int m, int T, float eps, float alpha_in, const float* W, float* Xh, NsHdr* hdr,
-                                bf16* smem, float* red) {
+__device__ void ns_forward_smem(int m, int T, float eps, float alpha_in, const float* W, float* Xh, float* Ph, int ld,
+                                NsHdr* hdr, bf16* smem, float* red) {
   using TL = NsTile<MP>;
   bf16* sW = smem; bf16* sX = smem + 2 * TL::MAT; bf16* sP = smem + 4 * TL::MAT;
-  const long long mm = (long long)m * m;
-  ns_norms(m, eps, alpha_in, W, hdr, red);
+  const long long mm = (long long)m * ld;      // stride of one matrix of the histories (leading dimension ld)
+  // W + eps I is first staged in fp32 (in the space of P, which is not needed yet): norms, the split
+  // copy of W, X_0 = alpha W^T and its fp32 copy for the backward pass are all built from there, so
+  // global memory is read exactly once, coalesced.
+  float* Wf = reinterpret_cast<float*>(sP);
+  constexpr int PF = MP + 4;
+  constexpr int PER = MP * MP / 256;
+#pragma unroll 1
+  for (int b0 = 0; b0 < PER; b0 += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int e = (b0 + u) * 256 + threadIdx.x, i = e / MP, j = e % MP;
+      v[u] = (i < m && j < m) ? W[(long long)i * m + j] + (i == j ? eps : 0.f) : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int e = (b0 + u) * 256 + threadIdx.x, i = e / MP, j = e % MP;
+      Wf[i * PF + j] = v[u];
+    }
+  }
+  __syncthreads();
+  {
+    float* colsum = red; float* rowsum = red + 256;
+    const int t = threadIdx.x;
+    if (t < m) {
+      float cs = 0.f, rs = 0.f;
+      for (int i = 0; i < m; ++i) { cs += fabsf(Wf[i * PF + t]); rs += fabsf(Wf[t * PF + i]); }
+      colsum[t] = cs; rowsum[t] = rs;
+    }
+    __syncthreads();
+    if (t == 0) {
+      float n1 = -1.f, ninf = -1.f; int js = 0, is = 0;
+      for (int q = 0; q < m; ++q) {                 // strict > keeps the lowest index on ties
+        if (colsum[q] > n1) { n1 = colsum[q]; js = q; }
+        if (rowsum[q] > ninf) { ninf = rowsum[q]; is = q; }
+      }
+      hdr->n1 = n1; hdr->ninf = ninf; hdr->jstar = js; hdr->istar = is;
+      hdr->auto_alpha = !(alpha_in > 0.f);
+      hdr->alpha = (alpha_in > 0.f) ? alpha_in : 1.f / (n1 * ninf);
+      hdr->pad0 = hdr->pad1 = 0;
+    }
+    __syncthreads();
+  }
   const float alpha = hdr->alpha;
-  global_to_smem<MP>(W, m, eps, 1.f, false, sW);
-  global_to_smem<MP>(W, m, eps, alpha, true, sX);                       // X_0 = alpha (W + eps I)^T
-  for (long long e = threadIdx.x; e < mm; e += 256) {
-    const int i = (int)(e / m), j = (int)(e % m);
-    Xh[e] = alpha * (W[(long long)j * m + i] + (i == j ? eps : 0.f));
+  for (int e = threadIdx.x; e < MP * MP; e += 256) {
+    const int i = e / MP, j = e % MP;
+    bf16 h, l;
+    split2(Wf[i * PF + j], h, l);
+    sW[i * TL::LD + j] = h; sW[TL::MAT + i * TL::LD + j] = l;
+    const float x0 = alpha * Wf[j * PF + i];                          // X_0 = alpha (W + eps I)^T
+    split2(x0, h, l);
+    sX[i * TL::LD + j] = h; sX[TL::MAT + i * TL::LD + j] = l;
+    if (i < m && j < m) Xh[(long long)i * ld + j] = x0;
   }
   __syncthreads();
   float acc[TL::MT][TL::NT][4];
   for (int k = 0; k < T; ++k) {
     smem_gemm<MP, false, false>(acc, sW, sX, false);                    // W X_k
+    if (Ph) frag_to_global<MP>(acc, Ph + (long long)k * mm, m, ld);     // kept for the backward pass
 #pragma unroll
     for (int a = 0; a < TL::MT; ++a)
 #pragma unroll
@@ -214,289 +265,168 @@ __device__ void ns_forward_smem(int m, int T, float eps, float alpha_in, const f
     frag_to_smem<MP>(acc, sP);
     __syncthreads();
     smem_gemm<MP, false, false>(acc, sX, sP, false);                    // X_{k+1} = X_k (2I - W X_k)
-    frag_to_global<MP>(acc, Xh + (long long)(k + 1) * mm, m);
+    frag_to_global<MP>(acc, Xh + (long long)(k + 1) * mm, m, ld);
     __syncthreads();                                                    // every warp is done reading X_k
     frag_to_smem<MP>(acc, sX);
     __syncthreads();
   }
 }
 
-// Adjoint.  smem: five matrices (W, A, G, P, H).  Xh: fp32 history from the forward pass; G0 = dLoss/dX_T
-// (global fp32).  Writes dW (global fp32 [m][m]); Gt is a global fp32 [m][m] scratch.
+// global fp32 [m][m] with leading dimension ld -> shared hi/lo, with 128-bit loads when ld allows it
+// (columns >= m of a padded row hold nothing defined and are masked to zero)
 template <int MP>
-__device__ void ns_backward_smem(int m, int T, float eps, const float* W, const float* Xh, const NsHdr* hdr,
-                                 const float* G0, float* dW, float* Gt, bf16* smem, float* red) {
+__device__ __forceinline__ void global_to_smem_fast(const float* __restrict__ src, int m, int ld, bf16* dst) {
   using TL = NsTile<MP>;
-  bf16* sW = smem; bf16* sA = smem + 2 * TL::MAT; bf16* sG = smem + 4 * TL::MAT;
-  bf16* sP = smem + 6 * TL::MAT; bf16* sH = smem + 8 * TL::MAT;
-  const long long mm = (long long)m * m;
-  float G[TL::MT][TL::NT][4], dWr[TL::MT][TL::NT][4], acc[TL::MT][TL::NT][4];
-  global_to_smem<MP>(W, m, eps, 1.f, false, sW);
+  if ((ld & 3) == 0) {
+    constexpr int PER4 = MP * MP / 4 / 256;       // float4 pieces per thread
+#pragma unroll 1
+    for (int b0 = 0; b0 < PER4; b0 += 8) {
+      float4 v[8];
 #pragma unroll
-  for (int a = 0; a < TL::MT; ++a)
-#pragma unroll
-    for (int t = 0; t < TL::NT; ++t)
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        int i, j;
-        frag_ij<MP>(a, t, q, i, j);
-        G[a][t][q] = (i < m && j < m) ? G0[(long long)i * m + j] : 0.f;
-        dWr[a][t][q] = 0.f;
+      for (int u = 0; u < 8; ++u) {
+        const int e = ((b0 + u) * 256 + threadIdx.x) * 4, i = e / MP, j = e % MP;
+        v[u] = (b0 + u < PER4 && i < m && j < m) ? *reinterpret_cast<const float4*>(src + (long long)i * ld + j)
+                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
       }
-  frag_to_smem<MP>(G, sG);
-  for (int k = T - 1; k >= 0; --k) {
-    __syncthreads();                                                    // previous readers of sA, sG writers done
-    global_to_smem<MP>(Xh + (long long)k * mm, m, 0.f, 1.f, false, sA);  // A = X_k
-    __syncthreads();
-    smem_gemm<MP, true, false>(acc, sA, sG, false);                     // H = A^T G
-    frag_to_smem<MP>(acc, sH);
-    smem_gemm<MP, false, false>(acc, sW, sA, false);                    // P = W A
-    frag_to_smem<MP>(acc, sP);
-    __syncthreads();
-    smem_gemm<MP, false, true>(acc, sH, sA, false);                     // H A^T
 #pragma unroll
-    for (int a = 0; a < TL::MT; ++a)
-#pragma unroll
-      for (int t = 0; t < TL::NT; ++t)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) dWr[a][t][q] -= acc[a][t][q];       // dW -= H A^T
-    smem_gemm<MP, false, true>(acc, sG, sP, false);                     // G P^T
-    smem_gemm<MP, true, false>(acc, sW, sH, true);                      // + W^T H
-#pragma unroll
-    for (int a = 0; a < TL::MT; ++a)
-#pragma unroll
-      for (int t = 0; t < TL::NT; ++t)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) G[a][t][q] = 2.f * G[a][t][q] - acc[a][t][q];
-    __syncthreads();                                                    // every warp is done reading sG
-    frag_to_smem<MP>(G, sG);
+      for (int u = 0; u < 8; ++u) {
+        if (b0 + u >= PER4) break;
+        const int e = ((b0 + u) * 256 + threadIdx.x) * 4, i = e / MP, j = e % MP;
+        float4 x = v[u];
+        if (j + 1 >= m) x.y = 0.f;
+        if (j + 2 >= m) x.z = 0.f;
+        if (j + 3 >= m) x.w = 0.f;
+        uint2 h, l;
+        split4(x, h, l);
+        *reinterpret_cast<uint2*>(dst + i * TL::LD + j) = h;
+        *reinterpret_cast<uint2*>(dst + TL::MAT + i * TL::LD + j) = l;
+      }
+    }
+  } else {
+    for (int e = threadIdx.x; e < MP * MP; e += 256) {
+      const int i = e / MP, j = e % MP;
+      bf16 h, l;
+      split2((i < m && j < m) ? src[(long long)i * ld + j] : 0.f, h, l);
+      dst[i * TL::LD + j] = h;
+      dst[TL::MAT + i * TL::LD + j] = l;
+    }
   }
-  // X_0 = alpha (W + eps I)^T:  d alpha = <G, W^T>,  dW += alpha G^T, then the alpha(W) terms
-  const float alpha = hdr->alpha;
-  float part = 0.f;
-#pragma unroll
-  for (int a = 0; a < TL::MT; ++a)
-#pragma unroll
-    for (int t = 0; t < TL::NT; ++t)
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        int i, j;
-        frag_ij<MP>(a, t, q, i, j);
-        if (i < m && j < m) part += G[a][t][q] * (W[(long long)j * m + i] + (i == j ? eps : 0.f));
-      }
-  frag_to_global<MP>(G, Gt, m);
-  const float dalpha = block_sum(part, red);                            // contains __syncthreads: Gt is visible
-  const bool aa = hdr->auto_alpha != 0;
-  const int js = hdr->jstar, is = hdr->istar;
-  const float c1 = dalpha * (-alpha / hdr->n1), c2 = dalpha * (-alpha / hdr->ninf);
-#pragma unroll
-  for (int a = 0; a < TL::MT; ++a)
-#pragma unroll
-    for (int t = 0; t < TL::NT; ++t)
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        int i, j;
-        frag_ij<MP>(a, t, q, i, j);
-        if (i < m && j < m) {
-          float v = dWr[a][t][q] + alpha * Gt[(long long)j * m + i];
-          if (aa) {
-            const float w = W[(long long)i * m + j] + (i == j ? eps : 0.f);
-            const float sg = w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f);
-            if (j == js) v += c1 * sg;
-            if (i == is) v += c2 * sg;
-          }
-          dW[(long long)i * m + j] = v;
-        }
-      }
-  __syncthreads();
 }
 
-// ---------------------------------------------------------------------------------------------
-// Adjoint for 64 < m <= 128.  Five hi/lo matrices of 128 x 128 do not fit in one SM's shared
-// memory, so three stay resident (A = X_k, G, and H which is later reused for P) while W, which
-// only ever appears as the left operand (W A and W^T H), is streamed from global memory (L2) in
-// K-chunks of 32 through a small staging buffer.  G and dW are kept in fp32 in global memory and
-// touched fragment-wise (each thread reads and writes only its own elements).
-// smem: 3 * NsTile<128>::mat_bytes + kStage128Bytes.
-// ---------------------------------------------------------------------------------------------
-constexpr int kStageEl = 128 * 40;                                    // bf16 elements of one staged part (hi or lo)
-constexpr size_t kStage128Bytes = (size_t)2 * kStageEl * sizeof(bf16);
-
-// acc (+)= op(W + eps I) B, W [m][m] in global memory, B resident ([K][N], hi/lo); TRA: op = transpose
-template <bool TRA>
-__device__ void smem_gemm_stream_w(float (&acc)[2][8][4], const float* W, int m, float eps, bf16* stage, const bf16* Bm,
-                                   bool accumulate) {
-  using TL = NsTile<128>;
-  const int tid = threadIdx.x, wm = TL::wm(), wn = TL::wn();
-  if (!accumulate) {
+// Adjoint of the iteration for a symmetric W (the landmark kernel matrix is symmetric bit for bit).
+// Per step k (A = X_k, P = W A saved by the forward pass):
+//     H = A^T G,   dW -= H A^T,   G <- 2G - G P^T - P^T G.
+// The last term is W^T H = (A W)^T G in general; for symmetric W every iterate is a polynomial in W,
+// so A W = W A = P up to rounding, and W itself is not needed inside the loop.  Three matrices are
+// resident (A and P share a buffer, G, H): 3 * NsTile<MP>::mat_bytes of shared memory.
+// Xh, Ph: fp32 histories [T+1][m][m] and [T][m][m]; G0 = dLoss/dX_T; Gf: global fp32 [m][m] scratch
+// that holds G in full precision (each thread touches only its own fragment elements).
+template <int MP>
+__device__ void ns_backward_smem(int m, int T, float eps, const float* W, const float* Xh, const float* Ph, int ld,
+                                 const NsHdr* hdr, const float* G0, float* dW, float* Gf, bf16* smem, float* red) {
+  using TL = NsTile<MP>;
+  bf16* sA = smem; bf16* sG = smem + 2 * TL::MAT; bf16* sH = smem + 4 * TL::MAT;
+  const long long mm = (long long)m * ld;      // every [m][m] matrix here except W has leading dimension ld
+  float acc[TL::MT][TL::NT][4], dWr[TL::MT][TL::NT][4];
 #pragma unroll
-    for (int a = 0; a < 2; ++a)
+  for (int a = 0; a < TL::MT; ++a)
 #pragma unroll
-      for (int t = 0; t < 8; ++t)
+    for (int t = 0; t < TL::NT; ++t)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) acc[a][t][q] = 0.f;
-  }
-  // row-chunk form (TRA = false): stage[128][40], thread -> (row tid/2, 16 cols); chunk = W[:, k0..k0+31]
-  // col-chunk form (TRA = true) : stage[32][136], thread -> (row tid/8, 16 cols); chunk = W[k0..k0+31, :]
-  const int r = TRA ? (tid >> 3) : (tid >> 1), cb = TRA ? (tid & 7) * 16 : (tid & 1) * 16;
-  constexpr int LDS_ = TRA ? 136 : 40;
-  float v[16];
-  auto fetch = [&](int k0) {
-    const int gr = TRA ? k0 + r : r, gc = TRA ? cb : k0 + cb;
-#pragma unroll
-    for (int q = 0; q < 16; ++q) {
-      const int cc = gc + q;
-      float x = (gr < m && cc < m) ? W[(long long)gr * m + cc] : 0.f;
-      if (gr == cc && gr < m) x += eps;
-      v[q] = x;
-    }
-  };
-  fetch(0);
-  for (int k0 = 0; k0 < 128; k0 += 32) {
-    __syncthreads();
-#pragma unroll
-    for (int q = 0; q < 16; q += 4) {
-      uint2 h, l;
-      split4(make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]), h, l);
-      *reinterpret_cast<uint2*>(stage + r * LDS_ + cb + q) = h;
-      *reinterpret_cast<uint2*>(stage + kStageEl + r * LDS_ + cb + q) = l;
-    }
-    __syncthreads();
-    if (k0 + 32 < 128) fetch(k0 + 32);
-#pragma unroll
-    for (int kk = 0; kk < 32; kk += 16) {
-      uint32_t ah[2][4], al[2][4];
-#pragma unroll
-      for (int a = 0; a < 2; ++a) {
-        if (TRA) { ldsm_x4_t(ah[a], addr_at(stage, 136, kk, wm + a * 16)); ldsm_x4_t(al[a], addr_at(stage + kStageEl, 136, kk, wm + a * 16)); }
-        else     { ldsm_x4(ah[a], addr_a(stage, 40, wm + a * 16, kk));     ldsm_x4(al[a], addr_a(stage + kStageEl, 40, wm + a * 16, kk)); }
-      }
-      uint32_t bh4[4][4], bl4[4][4];
-#pragma unroll
-      for (int t = 0; t < 4; ++t) {
-        ldsm_x4_t(bh4[t], addr_bt(Bm, TL::LD, k0 + kk, wn + t * 16));
-        ldsm_x4_t(bl4[t], addr_bt(Bm + TL::MAT, TL::LD, k0 + kk, wn + t * 16));
-      }
-#pragma unroll
-      for (int a = 0; a < 2; ++a)
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          mma_bf16(acc[a][2 * t], al[a], bh4[t][0], bh4[t][1]);
-          mma_bf16(acc[a][2 * t + 1], al[a], bh4[t][2], bh4[t][3]);
-        }
-#pragma unroll
-      for (int a = 0; a < 2; ++a)
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          mma_bf16(acc[a][2 * t], ah[a], bl4[t][0], bl4[t][1]);
-          mma_bf16(acc[a][2 * t + 1], ah[a], bl4[t][2], bl4[t][3]);
-        }
-#pragma unroll
-      for (int a = 0; a < 2; ++a)
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          mma_bf16(acc[a][2 * t], ah[a], bh4[t][0], bh4[t][1]);
-          mma_bf16(acc[a][2 * t + 1], ah[a], bh4[t][2], bh4[t][3]);
-        }
-    }
-  }
-  __syncthreads();
-}
-
-// Gf, T1: global fp32 [m][m] scratch.  dW: output (global fp32 [m][m]).
-__device__ void ns_backward_smem128(int m, int T, float eps, const float* W, const float* Xh, const NsHdr* hdr,
-                                    const float* G0, float* dW, float* Gf, float* T1, bf16* smem, float* red) {
-  using TL = NsTile<128>;
-  constexpr int MP = 128;
-  bf16* sA = smem; bf16* sG = smem + 2 * TL::MAT; bf16* sH = smem + 4 * TL::MAT; bf16* stage = smem + 6 * TL::MAT;
-  const long long mm = (long long)m * m;
-  float acc[2][8][4];
-  for (long long e = threadIdx.x; e < mm; e += 256) { Gf[e] = G0[e]; dW[e] = 0.f; }
-  global_to_smem<MP>(G0, m, 0.f, 1.f, false, sG);
+      for (int q = 0; q < 4; ++q) dWr[a][t][q] = 0.f;
+  for (long long e = threadIdx.x; e < mm; e += 256) Gf[e] = G0[e];
+  global_to_smem_fast<MP>(G0, m, ld, sG);
   for (int k = T - 1; k >= 0; --k) {
     __syncthreads();
-    global_to_smem<MP>(Xh + (long long)k * mm, m, 0.f, 1.f, false, sA);     // A = X_k
+    global_to_smem_fast<MP>(Xh + (long long)k * mm, m, ld, sA);                // A = X_k
     __syncthreads();
     smem_gemm<MP, true, false>(acc, sA, sG, false);                        // H = A^T G
     frag_to_smem<MP>(acc, sH);
     __syncthreads();
-    smem_gemm<MP, false, true>(acc, sH, sA, false);                        // H A^T
-    // dW -= H A^T on this thread's own elements; all loads of a tile row are issued before the stores
-#pragma unroll
-    for (int a = 0; a < 2; ++a) {
-      float old[8][4];
-#pragma unroll
-      for (int t = 0; t < 8; ++t)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          int i, j;
-          frag_ij<MP>(a, t, q, i, j);
-          old[t][q] = (i < m && j < m) ? dW[(long long)i * m + j] : 0.f;
-        }
-#pragma unroll
-      for (int t = 0; t < 8; ++t)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          int i, j;
-          frag_ij<MP>(a, t, q, i, j);
-          if (i < m && j < m) dW[(long long)i * m + j] = old[t][q] - acc[a][t][q];
-        }
-    }
-    smem_gemm_stream_w<true>(acc, W, m, eps, stage, sH, false);             // W^T H
-    frag_to_global<MP>(acc, T1, m);
-    smem_gemm_stream_w<false>(acc, W, m, eps, stage, sA, false);            // P = W A
-    frag_to_smem<MP>(acc, sH);                                             // H is dead: its buffer takes P
+    smem_gemm<MP, false, true>(dWr, sH, sA, true);                         // accumulates H A^T (dW = -sum)
+    __syncthreads();                                                       // every warp is done reading A
+    global_to_smem_fast<MP>(Ph + (long long)k * mm, m, ld, sA);                // P = W X_k from the forward pass
     __syncthreads();
-    smem_gemm<MP, false, true>(acc, sG, sH, false);                        // G P^T
-    __syncthreads();                                                       // every warp is done reading sG
+    smem_gemm<MP, false, true>(acc, sG, sA, false);                        // G P^T
+    smem_gemm<MP, true, false>(acc, sA, sG, true);                         // + P^T G
+    __syncthreads();                                                       // every warp is done reading G
 #pragma unroll
-    for (int a = 0; a < 2; ++a) {
-      float g0[8][4], t1[8][4];
+    for (int a = 0; a < TL::MT; ++a) {
+      float2 g0[TL::NT][2];
 #pragma unroll
-      for (int t = 0; t < 8; ++t)
+      for (int t = 0; t < TL::NT; ++t)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int h = 0; h < 2; ++h) {
           int i, j;
-          frag_ij<MP>(a, t, q, i, j);
-          const bool in = i < m && j < m;
-          g0[t][q] = in ? Gf[(long long)i * m + j] : 0.f;
-          t1[t][q] = in ? T1[(long long)i * m + j] : 0.f;
+          frag_ij<MP>(a, t, 2 * h, i, j);                                  // j is even: (j, j+1) are this thread's
+          if (i < m && j + 1 < m && (ld & 1) == 0) g0[t][h] = *reinterpret_cast<const float2*>(Gf + (long long)i * ld + j);
+          else {
+            g0[t][h].x = (i < m && j < m) ? Gf[(long long)i * ld + j] : 0.f;
+            g0[t][h].y = (i < m && j + 1 < m) ? Gf[(long long)i * ld + j + 1] : 0.f;
+          }
         }
 #pragma unroll
-      for (int t = 0; t < 8; ++t)
+      for (int t = 0; t < TL::NT; ++t)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int h = 0; h < 2; ++h) {
           int i, j;
-          frag_ij<MP>(a, t, q, i, j);
-          const float gn = 2.f * g0[t][q] - acc[a][t][q] - t1[t][q];   // 2G - G P^T - W^T H
-          if (i < m && j < m) Gf[(long long)i * m + j] = gn;
-          acc[a][t][q] = (i < m && j < m) ? gn : 0.f;
+          frag_ij<MP>(a, t, 2 * h, i, j);
+          float2 gn;
+          gn.x = (i < m && j < m) ? 2.f * g0[t][h].x - acc[a][t][2 * h] : 0.f;
+          gn.y = (i < m && j + 1 < m) ? 2.f * g0[t][h].y - acc[a][t][2 * h + 1] : 0.f;
+          if (i < m && j + 1 < m && (ld & 1) == 0) *reinterpret_cast<float2*>(Gf + (long long)i * ld + j) = gn;
+          else {
+            if (i < m && j < m) Gf[(long long)i * ld + j] = gn.x;
+            if (i < m && j + 1 < m) Gf[(long long)i * ld + j + 1] = gn.y;
+          }
+          acc[a][t][2 * h] = gn.x; acc[a][t][2 * h + 1] = gn.y;
         }
     }
     frag_to_smem<MP>(acc, sG);
   }
+  // dW so far (minus the accumulated sum) goes to global memory in fragment layout
+#pragma unroll
+  for (int a = 0; a < TL::MT; ++a)
+#pragma unroll
+    for (int t = 0; t < TL::NT; ++t)
+#pragma unroll
+      for (int q = 0; q < 4; ++q) dWr[a][t][q] = -dWr[a][t][q];
+  frag_to_global<MP>(dWr, dW, m, ld);
   __syncthreads();
-  // acc holds G in fragment layout when T > 0; reload it so that T = 0 works too
+  // X_0 = alpha (W + eps I)^T:  d alpha = <G, W^T>,  dW += alpha G^T, then the alpha(W) terms
   const float alpha = hdr->alpha;
   float part = 0.f;
-  for (long long e = threadIdx.x; e < mm; e += 256) {
-    const int i = (int)(e / m), j = (int)(e % m);
-    part += Gf[e] * (W[(long long)j * m + i] + (i == j ? eps : 0.f));
+  const int mlog = m * m;
+  for (int e = threadIdx.x; e < mlog; e += 256) {
+    const int i = e / m, j = e % m;
+    part += Gf[(long long)i * ld + j] * (W[(long long)j * m + i] + (i == j ? eps : 0.f));
   }
   const float dalpha = block_sum(part, red);
   const bool aa = hdr->auto_alpha != 0;
   const int js = hdr->jstar, is = hdr->istar;
   const float c1 = dalpha * (-alpha / hdr->n1), c2 = dalpha * (-alpha / hdr->ninf);
-  for (long long e = threadIdx.x; e < mm; e += 256) {
-    const int i = (int)(e / m), j = (int)(e % m);
-    float v = dW[e] + alpha * Gf[(long long)j * m + i];
-    if (aa) {
-      const float w = W[e] + (i == j ? eps : 0.f);
-      const float sg = w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f);
-      if (j == js) v += c1 * sg;
-      if (i == is) v += c2 * sg;
+  for (int e0 = threadIdx.x; e0 < mlog; e0 += 1024) {
+    float d0[4], gt[4], w0[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + u * 256, i = e / m, j = e % m;
+      const bool in = e < mlog;
+      d0[u] = in ? dW[(long long)i * ld + j] : 0.f; gt[u] = in ? Gf[(long long)j * ld + i] : 0.f; w0[u] = in ? W[e] : 0.f;
     }
-    dW[e] = v;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + u * 256;
+      if (e >= mlog) break;
+      const int i = e / m, j = e % m;
+      float v = d0[u] + alpha * gt[u];
+      if (aa) {
+        const float w = w0[u] + (i == j ? eps : 0.f);
+        const float sg = w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f);
+        if (j == js) v += c1 * sg;
+        if (i == is) v += c2 * sg;
+      }
+      dW[(long long)i * ld + j] = v;
+    }
   }
   __syncthreads();
 }
