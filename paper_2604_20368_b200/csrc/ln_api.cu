@@ -241,7 +241,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
                                                           x.ybar, dev_status));
     };
     if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * NsTile<64>::mat_bytes);
-    else if (TC && m <= 128) launch(k_mid_fwd<D, TC, TC ? 128 : 0>, 3 * NsTile<128>::mat_bytes);
+    else if (TC && m <= 128) launch(k_mid_fwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
     else launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));
   }
   // O = (C - mu) Ytilde + ybar
@@ -254,7 +254,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
 
 template <typename T, int D>
 int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const T* V, const T* dO,
-             const Ctx& x, const BwdWs& w, T* dQ, T* dK, T* dV, T* dL, cudaStream_t st) {
+             const Ctx& x, const BwdWs& w, T* dQ, T* dK, T* dV, T* dL, int32_t* dev_status, cudaStream_t st) {
   const int BH = pl.BH, n = pl.n, m = pl.m, ch = pl.chunks;
   const float inv_lambda = 1.f / p->lambda;
   const float* mu = p->map_mode == 1 ? x.mu : nullptr;
@@ -275,10 +275,10 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       LN_LAUNCH("k_mid_bwd", st, kern<<<BH, 256, smem, st>>>(m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten, x.W, x.Xh,
                                                           x.Ph, x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P, w.Hm,
-                                                          w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW));
+                                                          w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status));
     };
     if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 3 * NsTile<64>::mat_bytes);
-    else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * NsTile<128>::mat_bytes);
+    else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
     else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
   }
   LN_LAUNCH("sign_rows_dLW", st, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, st>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));
@@ -317,12 +317,12 @@ int fwd_dispatch_d(const ln_problem* p, const Plan& pl, const void* Q, const voi
 }
 template <typename T>
 int bwd_dispatch_d(const ln_problem* p, const Plan& pl, const void* Q, const void* K, const void* V, const void* dO,
-                   const Ctx& x, const BwdWs& w, void* dQ, void* dK, void* dV, void* dL, cudaStream_t st) {
+                   const Ctx& x, const BwdWs& w, void* dQ, void* dK, void* dV, void* dL, int32_t* ds, cudaStream_t st) {
   const T *q = (const T*)Q, *k = (const T*)K, *v = (const T*)V, *g = (const T*)dO;
   switch (p->d) {
-    case 32: return bwd_impl<T, 32>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, st);
-    case 64: return bwd_impl<T, 64>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, st);
-    case 128: return bwd_impl<T, 128>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, st);
+    case 32: return bwd_impl<T, 32>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st);
+    case 64: return bwd_impl<T, 64>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st);
+    case 128: return bwd_impl<T, 128>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st);
   }
   return LN_ERR_UNSUPPORTED;
 }
@@ -440,7 +440,6 @@ int laplace_nystrom_fwd(const ln_problem* p, const void* Q, const void* K, const
 int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L,
                         const void* dO, const void* saved, void* dQ, void* dK, void* dV, void* dL, void* ws,
                         size_t ws_bytes, int32_t* dev_status, void* stream) {
-  (void)dev_status;
   int s = validate(p);
   if (s != LN_OK) return s;
   if (!Q || !K || !V || !dO || !saved || !dQ || !dK || !dV || !ws) return LN_ERR_ARG;
@@ -454,8 +453,8 @@ int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const
   const BwdWs w = carve_bwd_ws(pl, ws);
   const Ctx x = carve_ctx(pl, const_cast<void*>(saved));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (p->dtype == LN_F32) return bwd_dispatch_d<float>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, st);
-  return bwd_dispatch_d<bf16>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, st);
+  if (p->dtype == LN_F32) return bwd_dispatch_d<float>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, dev_status, st);
+  return bwd_dispatch_d<bf16>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, dev_status, st);
 }
 
 size_t ns_pinv_workspace_bytes(int32_t batch, int32_t m, int32_t iters) {

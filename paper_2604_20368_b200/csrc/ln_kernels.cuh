@@ -5,6 +5,7 @@
 #include "ln_common.cuh"
 #include "ln_mma.cuh"
 #include "ln_ns_smem.cuh"
+#include "ln_ns_umma.cuh"
 
 namespace ln {
 
@@ -907,7 +908,12 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float ep
   Mpart += (long long)bh * nchunks * md;
   for (long long e = (long long)tid * 4; e < md; e += 1024)
     *reinterpret_cast<float4*>(Mout + e) = sum_parts4(Mpart, nchunks, md, e);
-  if constexpr (MP > 0) {
+  bool tc_ok = true;
+  if constexpr (MP == 128) {        // tcgen05 + TMEM
+    __shared__ UmmaCtl ctl;
+    tc_ok = ns_forward_umma(m, T, eps, alpha_in, W, Xh, Ph, ldx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
+    __syncthreads();
+  } else if constexpr (MP == 64) {  // mma.sync from shared memory
     ns_forward_smem<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, hdr, reinterpret_cast<bf16*>(dyn_smem), red);
     __syncthreads();
   } else {
@@ -918,7 +924,7 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float ep
     float bad = 0.f;
     for (int e = tid; e < m * m; e += 256) bad += isfinite(XT[(long long)(e / m) * ldx + e % m]) ? 0.f : 1.f;
     bad = block_sum(bad, red);
-    if (tid == 0) dev_status[bh] = bad > 0.f ? 1 : 0;
+    if (tid == 0) dev_status[bh] = (bad > 0.f ? 1 : 0) | (tc_ok ? 0 : 2);   // bit1: a bounded tensor-core wait ran out
   }
   ns_gemm<TC, false, false>(m, D, m, XT, ldx, Mout, D, Y, D, 1.f, 0.f, nullptr, 0.f, sm);   // Y = X M
   const float* s = whiten ? whiten + (long long)(bh % H) * m : nullptr;
@@ -960,7 +966,7 @@ __global__ void __launch_bounds__(256) k_mid_bwd(int m, int T, int H, int map_mo
                                                  const float* Xh, const float* Ph, const NsHdr* hdr, const float* Msaved,
                                                  const float* dYtpart, const float* dybpart, int nchunks,
                                                  float eps, float* Wr, float* P, float* Hm, float* Ga, float* Gb,
-                                                 float* dWm, float* dXm, float* dY, float* dM, float* GW) {
+                                                 float* dWm, float* dXm, float* dY, float* dM, float* GW, int* dev_status) {
   extern __shared__ __align__(16) unsigned char dyn_smem[];
   NsSmem& sm = *reinterpret_cast<NsSmem*>(dyn_smem);
   __shared__ float red[2 * 256 + 8];
@@ -1002,7 +1008,11 @@ __global__ void __launch_bounds__(256) k_mid_bwd(int m, int T, int H, int map_mo
   const float* XT = Xh + (long long)T * mx;
   ns_gemm<TC, false, true>(m, m, D, dY, D, Msaved, D, dXm, ldx, 1.f, 0.f, nullptr, 0.f, sm);   // dX = dY M^T
   ns_gemm<TC, true, false>(m, D, m, XT, ldx, dY, D, dM, D, 1.f, 0.f, nullptr, 0.f, sm);        // dM = X^T dY
-  if constexpr (MP > 0) ns_backward_smem<MP>(m, T, eps, W, Xh, Ph, ldx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
+  if constexpr (MP == 128) {
+    __shared__ UmmaCtl ctl;
+    const bool tc_ok = ns_backward_umma(m, T, eps, W, Xh, Ph, ldx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
+    if (dev_status && !tc_ok && tid == 0) atomicOr(dev_status + bh, 2);
+  } else if constexpr (MP == 64) ns_backward_smem<MP>(m, T, eps, W, Xh, Ph, ldx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
   else ns_backward_dev<TC>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red);
   // GW = (dW o K_LL + (dW o K_LL)^T) / lambda; four elements per batch so that the loads overlap
   for (long long e0 = (long long)tid * 4; e0 < (long long)m * ldm; e0 += 1024) {

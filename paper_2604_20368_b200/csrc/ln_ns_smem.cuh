@@ -313,6 +313,48 @@ __device__ __forceinline__ void global_to_smem_fast(const float* __restrict__ sr
   }
 }
 
+// End of the adjoint, shared by the shared-memory and tcgen05 paths.  On entry dW holds minus the
+// accumulated sum of H A^T and Gf the final G (both global fp32, leading dimension ld).
+__device__ inline void ns_backward_tail(int m, float eps, const float* W, int ld, const NsHdr* hdr, float* dW, const float* Gf,
+                                        float* red) {
+  // X_0 = alpha (W + eps I)^T:  d alpha = <G, W^T>,  dW += alpha G^T, then the alpha(W) terms
+  const float alpha = hdr->alpha;
+  float part = 0.f;
+  const int mlog = m * m;
+  for (int e = threadIdx.x; e < mlog; e += 256) {
+    const int i = e / m, j = e % m;
+    part += Gf[(long long)i * ld + j] * (W[(long long)j * m + i] + (i == j ? eps : 0.f));
+  }
+  const float dalpha = block_sum(part, red);
+  const bool aa = hdr->auto_alpha != 0;
+  const int js = hdr->jstar, is = hdr->istar;
+  const float c1 = dalpha * (-alpha / hdr->n1), c2 = dalpha * (-alpha / hdr->ninf);
+  for (int e0 = threadIdx.x; e0 < mlog; e0 += 1024) {
+    float d0[4], gt[4], w0[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + u * 256, i = e / m, j = e % m;
+      const bool in = e < mlog;
+      d0[u] = in ? dW[(long long)i * ld + j] : 0.f; gt[u] = in ? Gf[(long long)j * ld + i] : 0.f; w0[u] = in ? W[e] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + u * 256;
+      if (e >= mlog) break;
+      const int i = e / m, j = e % m;
+      float v = d0[u] + alpha * gt[u];
+      if (aa) {
+        const float w = w0[u] + (i == j ? eps : 0.f);
+        const float sg = w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f);
+        if (j == js) v += c1 * sg;
+        if (i == is) v += c2 * sg;
+      }
+      dW[(long long)i * ld + j] = v;
+    }
+  }
+  __syncthreads();
+}
+
 // Adjoint of the iteration for a symmetric W (the landmark kernel matrix is symmetric bit for bit).
 // Per step k (A = X_k, P = W A saved by the forward pass):
 //     H = A^T G,   dW -= H A^T,   G <- 2G - G P^T - P^T G.
@@ -393,41 +435,7 @@ __device__ void ns_backward_smem(int m, int T, float eps, const float* W, const 
       for (int q = 0; q < 4; ++q) dWr[a][t][q] = -dWr[a][t][q];
   frag_to_global<MP>(dWr, dW, m, ld);
   __syncthreads();
-  // X_0 = alpha (W + eps I)^T:  d alpha = <G, W^T>,  dW += alpha G^T, then the alpha(W) terms
-  const float alpha = hdr->alpha;
-  float part = 0.f;
-  const int mlog = m * m;
-  for (int e = threadIdx.x; e < mlog; e += 256) {
-    const int i = e / m, j = e % m;
-    part += Gf[(long long)i * ld + j] * (W[(long long)j * m + i] + (i == j ? eps : 0.f));
-  }
-  const float dalpha = block_sum(part, red);
-  const bool aa = hdr->auto_alpha != 0;
-  const int js = hdr->jstar, is = hdr->istar;
-  const float c1 = dalpha * (-alpha / hdr->n1), c2 = dalpha * (-alpha / hdr->ninf);
-  for (int e0 = threadIdx.x; e0 < mlog; e0 += 1024) {
-    float d0[4], gt[4], w0[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int e = e0 + u * 256, i = e / m, j = e % m;
-      const bool in = e < mlog;
-      d0[u] = in ? dW[(long long)i * ld + j] : 0.f; gt[u] = in ? Gf[(long long)j * ld + i] : 0.f; w0[u] = in ? W[e] : 0.f;
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int e = e0 + u * 256;
-      if (e >= mlog) break;
-      const int i = e / m, j = e % m;
-      float v = d0[u] + alpha * gt[u];
-      if (aa) {
-        const float w = w0[u] + (i == j ? eps : 0.f);
-        const float sg = w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f);
-        if (j == js) v += c1 * sg;
-        if (i == is) v += c2 * sg;
-      }
-      dW[(long long)i * ld + j] = v;
-    }
-  }
+  ns_backward_tail(m, eps, W, ld, hdr, dW, Gf, red);
   __syncthreads();
 }
 

@@ -1,0 +1,303 @@
+// Newton-Schulz (Alg. 2) and its adjoint for 64 < m <= 128 on the 5th-generation tensor cores:
+// tcgen05.mma issued by one thread, operands as bf16 hi + lo images in shared memory (three MMAs
+// per product: lo*hi, hi*lo, hi*hi), fp32 accumulators in tensor memory (TMEM), read back with
+// tcgen05.ld for the epilogue that produces the next operand image.  One CTA of 256 threads per head;
+// the iterate never leaves the SM except for the fp32 history the backward pass needs.
+//
+// Thread t owns row 32*(warp%4) + lane of a 128 x 128 accumulator and the column half warp/4.
+#pragma once
+#include "ln_ns_smem.cuh"
+#include "ln_umma.cuh"
+#ifdef LN_TIMING
+#include <cstdio>
+#endif
+
+namespace ln {
+
+constexpr int UM = 128;                       // padded matrix size of this path
+constexpr int UIMG = UM * UM;                 // bf16 elements of one image part (hi or lo)
+constexpr size_t kUmmaMatBytes = (size_t)2 * UIMG * sizeof(bf16);   // hi + lo = 64 KiB
+
+struct UmmaCtl {                              // small static shared state of the tcgen05 kernels
+  unsigned long long mbar;
+  uint32_t tmem_base;
+  int timeout;
+};
+
+// D[tmem_col .. +128) (+)= op(A) op(B) with split operands (hi at image, lo at image + UIMG); one thread.
+//   a_k: A image rows are M (A = X) else rows are K (A = X^T);  b_k: B image rows are N (B = X^T) else rows are K (B = X)
+__device__ __forceinline__ void umma_gemm(uint32_t tmem_d, const bf16* A, bool a_k, const bf16* Bm, bool b_k, bool accumulate) {
+  const uint32_t idesc = umma::instr_desc(UM, !a_k, !b_k);
+  bool acc = accumulate;
+#pragma unroll 1
+  for (int part = 0; part < 3; ++part) {      // lo*hi, hi*lo, hi*hi
+    const bf16* a = A + (part == 0 ? UIMG : 0);
+    const bf16* b = Bm + (part == 1 ? UIMG : 0);
+#pragma unroll
+    for (int ks = 0; ks < UM / 16; ++ks) {
+      umma::mma(tmem_d, umma::operand_desc(a, UM, a_k, ks), umma::operand_desc(b, UM, b_k, ks), idesc, acc);
+      acc = true;
+    }
+  }
+}
+
+// issue (thread 0) + wait (everyone); returns false on a timed-out wait
+// `phase` is each thread's own copy of the mbarrier phase (identical in all threads)
+__device__ __forceinline__ bool umma_run(UmmaCtl& ctl, uint32_t& phase, uint32_t tmem_d, const bf16* A, bool a_k, const bf16* Bm,
+                                         bool b_k, bool accumulate, const bf16* A2 = nullptr, bool a2_k = true,
+                                         const bf16* B2 = nullptr, bool b2_k = true) {
+  if (threadIdx.x == 0) {
+    umma::fence_after_sync();
+    umma_gemm(tmem_d, A, a_k, Bm, b_k, accumulate);
+    if (A2) umma_gemm(tmem_d, A2, a2_k, B2, b2_k, true);
+    umma::commit(&ctl.mbar);
+  }
+  const bool ok = umma::mbar_wait(&ctl.mbar, phase & 1);
+  phase ^= 1u;
+  umma::fence_after_sync();
+  return ok;
+}
+
+// 64 consecutive columns (this thread's half) of its accumulator row
+__device__ __forceinline__ void umma_row(uint32_t tmem_base, int col0, float (&v)[64]) {
+  float a[32], b[32];
+  umma::tmem_ld32(umma::tmem_addr(tmem_base, col0), a);
+  umma::tmem_ld32(umma::tmem_addr(tmem_base, col0 + 32), b);
+#pragma unroll
+  for (int q = 0; q < 32; ++q) { v[q] = a[q]; v[32 + q] = b[q]; }
+}
+
+// this thread's 64 values of row i -> global fp32 row (leading dimension ld, a multiple of 4): 128-bit stores.
+// Columns in [m, ld) receive whatever the accumulator holds there (zero); readers mask them anyway.
+__device__ __forceinline__ void umma_row_to_global(const float (&v)[64], float* dst_row, int j0, int ld) {
+#pragma unroll
+  for (int p = 0; p < 16; ++p) {
+    const int c = j0 + 4 * p;
+    if (c < ld) *reinterpret_cast<float4*>(dst_row + c) = make_float4(v[4 * p], v[4 * p + 1], v[4 * p + 2], v[4 * p + 3]);
+  }
+}
+
+// this thread's 64 values of row i -> the hi/lo image (eight 16-byte pieces each)
+__device__ __forceinline__ void umma_row_to_image(const float (&v)[64], int i, int j0, bf16* image) {
+#pragma unroll
+  for (int p = 0; p < 8; ++p) {
+    uint2 h0, l0, h1, l1;
+    split4(make_float4(v[8 * p], v[8 * p + 1], v[8 * p + 2], v[8 * p + 3]), h0, l0);
+    split4(make_float4(v[8 * p + 4], v[8 * p + 5], v[8 * p + 6], v[8 * p + 7]), h1, l1);
+    const int off = umma::img(i, j0 + 8 * p, UM);
+    *reinterpret_cast<uint4*>(image + off) = make_uint4(h0.x, h0.y, h1.x, h1.y);
+    *reinterpret_cast<uint4*>(image + UIMG + off) = make_uint4(l0.x, l0.y, l1.x, l1.y);
+  }
+}
+
+// global fp32 [m][m] (leading dimension ld) -> image, zero outside m x m.  256 threads, 8 pieces in flight.
+__device__ __forceinline__ void umma_load_image(const float* __restrict__ src, int m, int ld, bf16* image) {
+  const bool vec = (ld & 3) == 0;
+#pragma unroll 1
+  for (int b0 = 0; b0 < UM * UM / 8 / 256; b0 += 4) {       // 2048 pieces of 8 floats, 8 per thread
+    float v[4][8];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int pc = (b0 + u) * 256 + threadIdx.x, i = pc >> 4, j = (pc & 15) * 8;
+      if (i < m && j < m && vec) {
+        const float4 x = *reinterpret_cast<const float4*>(src + (long long)i * ld + j);
+        const float4 y = (j + 4 < ld) ? *reinterpret_cast<const float4*>(src + (long long)i * ld + j + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w; v[u][4] = y.x; v[u][5] = y.y; v[u][6] = y.z; v[u][7] = y.w;
+      } else {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[u][q] = (i < m && j + q < m) ? src[(long long)i * ld + j + q] : 0.f;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int pc = (b0 + u) * 256 + threadIdx.x, i = pc >> 4, j = (pc & 15) * 8;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) if (j + q >= m) v[u][q] = 0.f;       // padded columns of a row hold nothing defined
+      uint2 h0, l0, h1, l1;
+      split4(make_float4(v[u][0], v[u][1], v[u][2], v[u][3]), h0, l0);
+      split4(make_float4(v[u][4], v[u][5], v[u][6], v[u][7]), h1, l1);
+      const int off = umma::img(i, j, UM);
+      *reinterpret_cast<uint4*>(image + off) = make_uint4(h0.x, h0.y, h1.x, h1.y);
+      *reinterpret_cast<uint4*>(image + UIMG + off) = make_uint4(l0.x, l0.y, l1.x, l1.y);
+    }
+  }
+}
+
+__device__ __forceinline__ void umma_begin(UmmaCtl& ctl, int ncols) {
+  if (threadIdx.x == 0) { umma::mbar_init(&ctl.mbar, 1); ctl.timeout = 0; }
+  if ((threadIdx.x >> 5) == 0) umma::tmem_alloc(&ctl.tmem_base, ncols);
+  umma::fence_before_sync();
+  __syncthreads();
+  umma::fence_after_sync();
+}
+__device__ __forceinline__ void umma_end(UmmaCtl& ctl, int ncols) {
+  umma::fence_before_sync();
+  __syncthreads();
+  if ((threadIdx.x >> 5) == 0) umma::tmem_dealloc(ctl.tmem_base, ncols);
+}
+// end of a step: what the threads wrote to shared memory becomes visible to the tensor core, and
+// their TMEM reads are ordered before the next MMA that overwrites the accumulator
+__device__ __forceinline__ void umma_step_done(UmmaCtl& ctl, bool ok) {
+  if (!ok) ctl.timeout = 1;
+  umma::fence_smem_to_mma();
+  umma::fence_before_sync();
+  __syncthreads();
+}
+
+// Forward iteration.  smem: images W, X, P (3 * kUmmaMatBytes).  Xh [T+1][m][ld], Ph [T][m][ld] fp32 in global.
+// Returns false if a tensor-core wait timed out.
+__device__ bool ns_forward_umma(int m, int T, float eps, float alpha_in, const float* W, float* Xh, float* Ph, int ld,
+                                NsHdr* hdr, bf16* smem, float* red, UmmaCtl& ctl) {
+  bf16* sW = smem; bf16* sX = smem + 2 * UIMG; bf16* sP = smem + 4 * UIMG;
+  const long long mm = (long long)m * ld;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64;
+  umma_begin(ctl, 128);
+  uint32_t phase = 0;
+  // W + eps I staged in fp32 in the space of P: norms, images of W and X_0, fp32 X_0 all come from there
+  float* Wf = reinterpret_cast<float*>(sP);      // [128][128], pitch 128
+#pragma unroll 1
+  for (int b0 = 0; b0 < UM * UM / 256; b0 += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int e = (b0 + u) * 256 + tid, i = e >> 7, j = e & 127;
+      v[u] = (i < m && j < m) ? W[(long long)i * m + j] + (i == j ? eps : 0.f) : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) Wf[(b0 + u) * 256 + tid] = v[u];
+  }
+  __syncthreads();
+  {
+    float* colsum = red; float* rowsum = red + 256;
+    if (tid < m) {
+      float cs = 0.f, rs = 0.f;
+      for (int i = 0; i < m; ++i) cs += fabsf(Wf[i * UM + tid]);
+      for (int i = 0; i < UM; ++i) rs += fabsf(Wf[tid * UM + ((i + tid) & 127)]);   // rotated start: no bank conflicts; padding is zero
+      colsum[tid] = cs; rowsum[tid] = rs;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      float n1 = -1.f, ninf = -1.f; int js = 0, is = 0;
+      for (int q = 0; q < m; ++q) {
+        if (colsum[q] > n1) { n1 = colsum[q]; js = q; }
+        if (rowsum[q] > ninf) { ninf = rowsum[q]; is = q; }
+      }
+      hdr->n1 = n1; hdr->ninf = ninf; hdr->jstar = js; hdr->istar = is;
+      hdr->auto_alpha = !(alpha_in > 0.f);
+      hdr->alpha = (alpha_in > 0.f) ? alpha_in : 1.f / (n1 * ninf);
+      hdr->pad0 = hdr->pad1 = 0;
+    }
+    __syncthreads();
+  }
+  const float alpha = hdr->alpha;
+  {  // this thread's row: 64 columns of W and of X_0 = alpha W^T
+    float w[64], x0[64];
+#pragma unroll
+    for (int q = 0; q < 64; ++q) { w[q] = Wf[row * UM + col0 + q]; x0[q] = alpha * Wf[(col0 + q) * UM + row]; }
+    umma_row_to_image(w, row, col0, sW);
+    umma_row_to_image(x0, row, col0, sX);
+    if (row < m) umma_row_to_global(x0, Xh + (long long)row * ld, col0, ld);
+  }
+  bool ok = true;
+  umma_step_done(ctl, true);
+#ifdef LN_TIMING
+  long long tf[6] = {0, 0, 0, 0, 0, 0}, tf0 = clock64(), tf1;
+#define LN_FT(i) do { tf1 = clock64(); tf[i] += tf1 - tf0; tf0 = tf1; } while (0)
+#else
+#define LN_FT(i) do { } while (0)
+#endif
+  for (int k = 0; k < T; ++k) {
+    ok &= umma_run(ctl, phase, ctl.tmem_base, sW, true, sX, false, false);                   // D = W X_k
+    LN_FT(0);
+    {
+      float v[64];
+      umma_row(ctl.tmem_base, col0, v);
+      if (Ph && row < m) umma_row_to_global(v, Ph + (long long)k * mm + (long long)row * ld, col0, ld);
+#pragma unroll
+      for (int q = 0; q < 64; ++q) v[q] = ((row == col0 + q && row < m) ? 2.f : 0.f) - v[q];   // 2I - W X_k
+      umma_row_to_image(v, row, col0, sP);
+    }
+    LN_FT(1);
+    umma_step_done(ctl, ok);
+    LN_FT(2);
+    ok &= umma_run(ctl, phase, ctl.tmem_base, sX, true, sP, false, false);                   // D = X_k (2I - W X_k)
+    LN_FT(3);
+    {
+      float v[64];
+      umma_row(ctl.tmem_base, col0, v);
+      if (row < m) umma_row_to_global(v, Xh + (long long)(k + 1) * mm + (long long)row * ld, col0, ld);
+      umma_row_to_image(v, row, col0, sX);     // the MMAs that read X_k have completed
+    }
+    LN_FT(4);
+    umma_step_done(ctl, ok);
+    LN_FT(5);
+  }
+#ifdef LN_TIMING
+  if (blockIdx.x == 0 && (threadIdx.x == 0 || threadIdx.x == 100))
+    printf("ns_fwd_umma t%d cycles per iter: mma1 %lld epi1 %lld sync %lld mma2 %lld epi2 %lld sync %lld\n", (int)threadIdx.x,
+           tf[0] / T, tf[1] / T, tf[2] / T, tf[3] / T, tf[4] / T, tf[5] / T);
+#endif
+  ok &= (ctl.timeout == 0);
+  umma_end(ctl, 128);
+  return ok;
+}
+
+// Adjoint for a symmetric W (see ns_backward_smem for the algebra).  smem: images A (also used for P), G, H.
+// TMEM: 128 columns for the running product, 128 for dW accumulated over all steps.
+__device__ bool ns_backward_umma(int m, int T, float eps, const float* W, const float* Xh, const float* Ph, int ld,
+                                 const NsHdr* hdr, const float* G0, float* dW, float* Gf, bf16* smem, float* red,
+                                 UmmaCtl& ctl) {
+  bf16* sA = smem; bf16* sG = smem + 2 * UIMG; bf16* sH = smem + 4 * UIMG;
+  const long long mm = (long long)m * ld;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64;
+  umma_begin(ctl, 256);
+  uint32_t phase = 0;
+  const uint32_t t_acc = ctl.tmem_base, t_dw = ctl.tmem_base + 128;
+  float G[64];                                 // this thread's part of G in full precision
+#pragma unroll
+  for (int q = 0; q < 64; ++q) G[q] = (row < m && col0 + q < m) ? G0[(long long)row * ld + col0 + q] : 0.f;
+  umma_row_to_image(G, row, col0, sG);
+  bool ok = true;
+  for (int k = T - 1; k >= 0; --k) {
+    umma_load_image(Xh + (long long)k * mm, m, ld, sA);                               // A = X_k
+    umma_step_done(ctl, ok);
+    ok &= umma_run(ctl, phase, t_acc, sA, false, sG, false, false);                          // H = A^T G
+    {
+      float v[64];
+      umma_row(t_acc, col0, v);
+      umma_row_to_image(v, row, col0, sH);
+    }
+    umma_step_done(ctl, ok);
+    ok &= umma_run(ctl, phase, t_dw, sH, true, sA, true, k != T - 1);                        // dW accumulator += H A^T
+    umma_load_image(Ph + (long long)k * mm, m, ld, sA);                               // P = W X_k (A is no longer read)
+    umma_step_done(ctl, ok);
+    ok &= umma_run(ctl, phase, t_acc, sG, true, sA, true, false, sA, false, sG, false);      // G P^T + P^T G
+    {
+      float v[64];
+      umma_row(t_acc, col0, v);
+#pragma unroll
+      for (int q = 0; q < 64; ++q) G[q] = (row < m && col0 + q < m) ? 2.f * G[q] - v[q] : 0.f;
+      umma_row_to_image(G, row, col0, sG);
+    }
+  }
+  umma_step_done(ctl, ok);
+  {  // dW = -(accumulated sum), G -> global for the transposed accesses of the tail
+    float v[64];
+    if (T > 0) umma_row(t_dw, col0, v);
+#pragma unroll
+    for (int q = 0; q < 64; ++q) v[q] = (T > 0) ? -v[q] : 0.f;
+    if (row < m) {
+      umma_row_to_global(v, dW + (long long)row * ld, col0, ld);
+      umma_row_to_global(G, Gf + (long long)row * ld, col0, ld);
+    }
+  }
+  ok &= (ctl.timeout == 0);
+  umma_end(ctl, 256);
+  __syncthreads();
+  ns_backward_tail(m, eps, W, ld, hdr, dW, Gf, red);
+  return ok;
+}
+
+}  // namespace ln
