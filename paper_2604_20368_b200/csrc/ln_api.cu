@@ -209,6 +209,7 @@ template <typename T, int D>
 int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const T* V, const T* L, T* O,
              const Ctx& x, const FwdWs& w, int32_t* dev_status, cudaStream_t st) {
   const int BH = pl.BH, n = pl.n, m = pl.m;
+  if (dev_status) cudaMemsetAsync(dev_status, 0, sizeof(int32_t) * BH, st);   // the kernels OR their flags into it
   // landmarks (Sec. 4.2)
   if (p->lm_mode == 1) {
     LN_LAUNCH("k_pool", st, k_pool<T><<<dim3(cdiv(m, 256 / (D / 4)), BH), 256, 0, st>>>(K, x.Lf, geom_of(p)));
@@ -258,6 +259,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const int BH = pl.BH, n = pl.n, m = pl.m, ch = pl.chunks;
   const float inv_lambda = 1.f / p->lambda;
   const float* mu = p->map_mode == 1 ? x.mu : nullptr;
+  if (dev_status) cudaMemsetAsync(dev_status, 0, sizeof(int32_t) * BH, st);
   // query side: Z'^T dO and column sums of dO; g^C = (dO Ytilde^T) o C / lambda; dQ; landmark part
   if constexpr (std::is_same<T, bf16>::value) {
     LN_LAUNCH("tn_dY", st, k_tn_mma<D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));

@@ -719,7 +719,7 @@ __device__ void cta_gemm(int M, int N, int K, const float* A, int lda, const flo
 }
 
 // Shared memory of the per-head kernels: one of the two GEMM engines is used per instantiation.
-union __align__(16) NsSmem { GemmSmem f; MmaGemmSmem t; };
+union __align__(16) NsSmem { GemmSmem f; MmaGemmSmem t; MmaGemmSmemBig b; };
 
 // C = beta*Cin + alpha*op(A)op(B) + diag*I on either engine: TC = tensor cores with split-bf16
 // operands (bf16-storage path), else exact fp32 FFMA (fp32-storage path, stand-alone ns_pinv).
@@ -728,7 +728,8 @@ __device__ __forceinline__ void ns_gemm(int M, int N, int K, const float* A, int
                                         float* C, int ldc, float alpha, float beta, const float* Cin, float diag,
                                         NsSmem& sm) {
   if (TC) {
-    cta_gemm_mma<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.t);
+    if (M > 128 && N > 64) cta_gemm_mma_big<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.b);
+    else cta_gemm_mma<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.t);
   } else {
     cta_gemm<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, sm.f);
     if (diag != 0.f) {
@@ -924,7 +925,7 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float ep
     float bad = 0.f;
     for (int e = tid; e < m * m; e += 256) bad += isfinite(XT[(long long)(e / m) * ldx + e % m]) ? 0.f : 1.f;
     bad = block_sum(bad, red);
-    if (tid == 0) dev_status[bh] = (bad > 0.f ? 1 : 0) | (tc_ok ? 0 : 2);   // bit1: a bounded tensor-core wait ran out
+    if (tid == 0) atomicOr(dev_status + bh, (bad > 0.f ? 1 : 0) | (tc_ok ? 0 : 2));   // bit1: a bounded tensor-core wait ran out
   }
   ns_gemm<TC, false, false>(m, D, m, XT, ldx, Mout, D, Y, D, 1.f, 0.f, nullptr, 0.f, sm);   // Y = X M
   const float* s = whiten ? whiten + (long long)(bh % H) * m : nullptr;
