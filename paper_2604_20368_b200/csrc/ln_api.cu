@@ -34,10 +34,14 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   if (!p) return false;
   pl->BH = p->B * p->H; pl->n = p->n; pl->d = p->d; pl->m = p->m; pl->T = p->ns_iters;
   pl->ldm = (p->m + 3) & ~3;
-  // token chunks per head for the reductions over tokens: enough CTAs to fill the GPU twice
-  int want = (2 * kSMs + pl->BH - 1) / pl->BH;
+  // token chunks per head for the reductions over tokens: about eight waves of CTAs (two per SM) so that
+  // the last wave costs little, but at least 64 tokens per chunk
+  const int mblk = (p->m + 63) / 64;
+  int want = (16 * kSMs + pl->BH * mblk - 1) / (pl->BH * mblk);
+  if (want > 16) want = 16;        // the per-head kernels sum the partial results serially
   if (want < 1) want = 1;
   int rpc = (p->n + want - 1) / want;
+  if (rpc < 256) rpc = 256;
   rpc = (rpc + 31) / 32 * 32;
   pl->rpc = rpc;
   pl->chunks = (p->n + rpc - 1) / rpc;

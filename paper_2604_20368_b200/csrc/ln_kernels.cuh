@@ -204,8 +204,15 @@ __global__ void __launch_bounds__(256) k_pool(const T* __restrict__ K, float* __
 // dK[j] = dKpart[j] (may be NULL) + sum over the bins containing token j of dL[bin] / |bin|
 // (pooling adjoint); with pool == 0 it only converts dKpart to the storage type.
 template <typename T>
-__global__ void k_pool_bwd(const float* __restrict__ dKpart, const float* __restrict__ dL, T* __restrict__ dK,
-                           PoolGeom g, int pool) {
+__global__ void __launch_bounds__(256) k_pool_bwd(const float* __restrict__ dKpart, const float* __restrict__ dL, T* __restrict__ dK,
+                                                  PoolGeom g, int pool) {
+  // bin boundaries once per CTA (a division each) instead of several per thread
+  __shared__ int rlo[256], rhi[256], clo[256], chi[256];
+  if (pool) {
+    for (int a = threadIdx.x; a < g.mh; a += 256) { rlo[a] = bin_lo(a, g.gh, g.mh); rhi[a] = bin_hi(a, g.gh, g.mh); }
+    for (int b = threadIdx.x; b < g.mw; b += 256) { clo[b] = bin_lo(b, g.gw, g.mw); chi[b] = bin_hi(b, g.gw, g.mw); }
+    __syncthreads();
+  }
   const int bh = blockIdx.y;
   const unsigned per_row = g.d / 4;
   const unsigned idx = blockIdx.x * blockDim.x + threadIdx.x;     // n * d / 4 < 2^32
@@ -215,15 +222,13 @@ __global__ void k_pool_bwd(const float* __restrict__ dKpart, const float* __rest
   if (dKpart) v = ld4(dKpart + ((long long)bh * g.n + j) * g.d + c);
   if (pool && j >= g.prefix) {
     const int r = (j - g.prefix) / g.gw, q = (j - g.prefix) % g.gw;
-    int a_lo = (int)(((unsigned)r * (unsigned)g.mh) / (unsigned)g.gh) - 1; if (a_lo < 0) a_lo = 0;
-    int b_lo = (int)(((unsigned)q * (unsigned)g.mw) / (unsigned)g.gw) - 1; if (b_lo < 0) b_lo = 0;
-    for (int a = a_lo; a < g.mh && a <= a_lo + 2; ++a) {
-      const int r0 = bin_lo(a, g.gh, g.mh), r1 = bin_hi(a, g.gh, g.mh);
-      if (r < r0 || r >= r1) continue;
-      for (int bb = b_lo; bb < g.mw && bb <= b_lo + 2; ++bb) {
-        const int c0 = bin_lo(bb, g.gw, g.mw), c1 = bin_hi(bb, g.gw, g.mw);
-        if (q < c0 || q >= c1) continue;
-        const float inv = 1.f / (float)((r1 - r0) * (c1 - c0));
+    // a token row lies in bin floor(r mh / gh) and, where neighbouring bins overlap, in the next one too
+    const int a0 = (int)(((unsigned)r * (unsigned)g.mh) / (unsigned)g.gh), b0 = (int)(((unsigned)q * (unsigned)g.mw) / (unsigned)g.gw);
+    for (int a = (a0 > 0 ? a0 - 1 : 0); a <= a0 + 1 && a < g.mh; ++a) {
+      if (r < rlo[a] || r >= rhi[a]) continue;
+      for (int bb = (b0 > 0 ? b0 - 1 : 0); bb <= b0 + 1 && bb < g.mw; ++bb) {
+        if (q < clo[bb] || q >= chi[bb]) continue;
+        const float inv = 1.f / (float)((rhi[a] - rlo[a]) * (chi[bb] - clo[bb]));
         const float4 t = ld4(dL + ((long long)bh * g.m + a * g.mw + bb) * g.d + c);
         v.x += t.x * inv; v.y += t.y * inv; v.z += t.z * inv; v.w += t.w * inv;
       }
@@ -723,12 +728,13 @@ union __align__(16) NsSmem { GemmSmem f; MmaGemmSmem t; MmaGemmSmemBig b; };
 
 // C = beta*Cin + alpha*op(A)op(B) + diag*I on either engine: TC = tensor cores with split-bf16
 // operands (bf16-storage path), else exact fp32 FFMA (fp32-storage path, stand-alone ns_pinv).
-template <bool TC, bool TRA, bool TRB>
+template <bool TC, bool TRA, bool TRB, bool BIG = false>
 __device__ __forceinline__ void ns_gemm(int M, int N, int K, const float* A, int lda, const float* Bm, int ldb,
                                         float* C, int ldc, float alpha, float beta, const float* Cin, float diag,
                                         NsSmem& sm) {
   if (TC) {
-    if (M > 128 && N > 64) cta_gemm_mma_big<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.b);
+    // the 128 x 128-tile engine is compiled only where m can exceed 128 (it costs registers)
+    if (BIG && M > 128 && N > 64) cta_gemm_mma_big<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.b);
     else cta_gemm_mma<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.t);
   } else {
     cta_gemm<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, sm.f);
@@ -785,8 +791,8 @@ __device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const fl
   for (int k = 0; k < T; ++k) {
     const float* X = Xh + (long long)k * mm;
     float* Xn = Xh + (long long)(k + 1) * mm;
-    ns_gemm<TC, false, false>(m, m, m, Wr, m, X, m, P, m, -1.f, 0.f, nullptr, 2.f, sm);   // P = 2I - Wr X_k
-    ns_gemm<TC, false, false>(m, m, m, X, m, P, m, Xn, m, 1.f, 0.f, nullptr, 0.f, sm);    // X_{k+1} = X_k P
+    ns_gemm<TC, false, false, true>(m, m, m, Wr, m, X, m, P, m, -1.f, 0.f, nullptr, 2.f, sm);   // P = 2I - Wr X_k
+    ns_gemm<TC, false, false, true>(m, m, m, X, m, P, m, Xn, m, 1.f, 0.f, nullptr, 0.f, sm);    // X_{k+1} = X_k P
   }
 }
 
@@ -805,11 +811,11 @@ __device__ void ns_backward_dev(int m, int T, const float* Wr, const float* Xh, 
   float* G = Ga; float* Gn = Gb;
   for (int k = T - 1; k >= 0; --k) {
     const float* A = Xh + (long long)k * mm;                                        // X_{k+1} = 2A - A P, P = Wr A
-    ns_gemm<TC, false, false>(m, m, m, Wr, m, A, m, P, m, 1.f, 0.f, nullptr, 0.f, sm);      // P = Wr A
-    ns_gemm<TC, true, false>(m, m, m, A, m, G, m, Hm, m, 1.f, 0.f, nullptr, 0.f, sm);       // H = A^T G
-    ns_gemm<TC, false, true>(m, m, m, Hm, m, A, m, dW, m, -1.f, 1.f, dW, 0.f, sm);          // dW -= H A^T
-    ns_gemm<TC, false, true>(m, m, m, G, m, P, m, Gn, m, -1.f, 2.f, G, 0.f, sm);            // Gn = 2G - G P^T
-    ns_gemm<TC, true, false>(m, m, m, Wr, m, Hm, m, Gn, m, -1.f, 1.f, Gn, 0.f, sm);         // Gn -= Wr^T H
+    ns_gemm<TC, false, false, true>(m, m, m, Wr, m, A, m, P, m, 1.f, 0.f, nullptr, 0.f, sm);      // P = Wr A
+    ns_gemm<TC, true, false, true>(m, m, m, A, m, G, m, Hm, m, 1.f, 0.f, nullptr, 0.f, sm);       // H = A^T G
+    ns_gemm<TC, false, true, true>(m, m, m, Hm, m, A, m, dW, m, -1.f, 1.f, dW, 0.f, sm);          // dW -= H A^T
+    ns_gemm<TC, false, true, true>(m, m, m, G, m, P, m, Gn, m, -1.f, 2.f, G, 0.f, sm);            // Gn = 2G - G P^T
+    ns_gemm<TC, true, false, true>(m, m, m, Wr, m, Hm, m, Gn, m, -1.f, 1.f, Gn, 0.f, sm);         // Gn -= Wr^T H
     float* t = G; G = Gn; Gn = t;
   }
   // X_0 = alpha Wr^T
