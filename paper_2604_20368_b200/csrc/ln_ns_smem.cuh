@@ -6,9 +6,6 @@
 // of X gives a zero row or column of X (2I - W X)).
 #pragma once
 #include "ln_mma.cuh"
-#ifdef LN_TIMING
-#include <cstdio>
-#endif
 
 namespace ln {
 

@@ -8,9 +8,6 @@
 #pragma once
 #include "ln_ns_smem.cuh"
 #include "ln_umma.cuh"
-#ifdef LN_TIMING
-#include <cstdio>
-#endif
 
 namespace ln {
 
@@ -201,15 +198,8 @@ __device__ bool ns_forward_umma(int m, int T, float eps, float alpha_in, const f
   }
   bool ok = true;
   umma_step_done(ctl, true);
-#ifdef LN_TIMING
-  long long tf[6] = {0, 0, 0, 0, 0, 0}, tf0 = clock64(), tf1;
-#define LN_FT(i) do { tf1 = clock64(); tf[i] += tf1 - tf0; tf0 = tf1; } while (0)
-#else
-#define LN_FT(i) do { } while (0)
-#endif
   for (int k = 0; k < T; ++k) {
     ok &= umma_run(ctl, phase, ctl.tmem_base, sW, true, sX, false, false);                   // D = W X_k
-    LN_FT(0);
     {
       float v[64];
       umma_row(ctl.tmem_base, col0, v);
@@ -218,26 +208,16 @@ __device__ bool ns_forward_umma(int m, int T, float eps, float alpha_in, const f
       for (int q = 0; q < 64; ++q) v[q] = ((row == col0 + q && row < m) ? 2.f : 0.f) - v[q];   // 2I - W X_k
       umma_row_to_image(v, row, col0, sP);
     }
-    LN_FT(1);
     umma_step_done(ctl, ok);
-    LN_FT(2);
     ok &= umma_run(ctl, phase, ctl.tmem_base, sX, true, sP, false, false);                   // D = X_k (2I - W X_k)
-    LN_FT(3);
     {
       float v[64];
       umma_row(ctl.tmem_base, col0, v);
       if (row < m) umma_row_to_global(v, Xh + (long long)(k + 1) * mm + (long long)row * ld, col0, ld);
       umma_row_to_image(v, row, col0, sX);     // the MMAs that read X_k have completed
     }
-    LN_FT(4);
     umma_step_done(ctl, ok);
-    LN_FT(5);
   }
-#ifdef LN_TIMING
-  if (blockIdx.x == 0 && (threadIdx.x == 0 || threadIdx.x == 100))
-    printf("ns_fwd_umma t%d cycles per iter: mma1 %lld epi1 %lld sync %lld mma2 %lld epi2 %lld sync %lld\n", (int)threadIdx.x,
-           tf[0] / T, tf[1] / T, tf[2] / T, tf[3] / T, tf[4] / T, tf[5] / T);
-#endif
   ok &= (ctl.timeout == 0);
   umma_end(ctl, 128);
   return ok;
