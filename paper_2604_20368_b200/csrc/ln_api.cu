@@ -4,6 +4,7 @@
 
 #include "../../include/laplace_nystrom.h"
 #include "ln_kernels.cuh"
+#include "ln_sign2.cuh"
 #include <type_traits>
 
 using namespace ln;
@@ -28,6 +29,8 @@ struct Carver {
 
 struct Plan {
   int BH, n, d, m, T, ldm, rpc, chunks;
+  int s2_tg, s2_rpc, s2_chunks;      // fused sign pass: token groups per tile, tokens per chunk, chunks (0 = not used)
+  size_t s2_smem;
 };
 
 bool make_plan(const ln_problem* p, Plan* pl) {
@@ -45,6 +48,22 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   rpc = (rpc + 31) / 32 * 32;
   pl->rpc = rpc;
   pl->chunks = (p->n + rpc - 1) / rpc;
+  // fused sign pass (64-dim slabs): token tiles of 8 * TG tokens that hug n, chunks for about three waves
+  pl->s2_tg = pl->s2_rpc = pl->s2_chunks = 0; pl->s2_smem = 0;
+  if (p->d % 64 == 0) {
+    const int groups = (p->n + 7) / 8;
+    int tiles = (groups + 15) / 16;
+    int TG = (groups + tiles - 1) / tiles; TG += TG & 1; if (TG > 16) TG = 16;
+    tiles = (p->n + 8 * TG - 1) / (8 * TG);
+    const int slabs = p->d / 64;
+    int wantc = (6 * kSMs + pl->BH * slabs - 1) / (pl->BH * slabs);
+    if (wantc > 16) wantc = 16;
+    if (wantc > tiles) wantc = tiles;
+    if (wantc < 1) wantc = 1;
+    const int tpc = (tiles + wantc - 1) / wantc;
+    pl->s2_tg = TG; pl->s2_rpc = tpc * 8 * TG; pl->s2_chunks = (p->n + pl->s2_rpc - 1) / pl->s2_rpc;
+    pl->s2_smem = sizeof(float) * (size_t)sign2_smem(p->m, TG).total;
+  }
   return true;
 }
 
@@ -87,11 +106,12 @@ struct BwdWs {
 BwdWs carve_bwd_ws(const Plan& pl, void* base) {
   Carver c(base); BwdWs w;
   const size_t BH = pl.BH, n = pl.n, d = pl.d, m = pl.m, ch = pl.chunks;
+  const size_t chs = pl.s2_chunks > 0 ? (size_t)pl.s2_chunks : ch;     // chunks of the landmark-gradient partials
   w.G = c.take(BH * n * pl.ldm);
   w.dYtpart = c.take(BH * ch * m * d);
   w.dybpart = c.take(BH * ch * d);
-  w.dLCpart = c.take(BH * ch * m * d);
-  w.dLRpart = c.take(BH * ch * m * d);
+  w.dLCpart = c.take(BH * chs * m * d);
+  w.dLRpart = c.take(BH * chs * m * d);
   w.dY = c.take(BH * m * d);
   w.dM = c.take(BH * m * d);
   w.Wr = c.take(BH * m * pl.ldm);
@@ -272,8 +292,17 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     LN_LAUNCH("tn_dY", st, k_tn<T, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
     LN_LAUNCH("ntg_C", st, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(dO, x.Yt, x.C, pl.ldm, w.G, n, m, inv_lambda));
   }
-  LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m));
-  LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
+  const bool fused_sign = pl.s2_chunks > 0;
+  const int chs = fused_sign ? pl.s2_chunks : ch;
+  if (fused_sign) {
+    cudaFuncSetAttribute(k_sign2<T, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.s2_smem);
+    cudaFuncSetAttribute(k_sign2<T, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.s2_smem);
+    LN_LAUNCH("sign2_dQ_dLC", st, k_sign2<T, T><<<dim3(chs, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(
+        Q, x.Lf, w.G, pl.ldm, dQ, w.dLCpart, n, m, D, pl.s2_rpc));
+  } else {
+    LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m));
+    LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
+  }
   // per head: dY, dX, dM, Newton-Schulz adjoint, symmetrised landmark-block upstream
   {
     constexpr bool TC = std::is_same<T, bf16>::value;
@@ -296,15 +325,20 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     LN_LAUNCH("ntg_R", st, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(V, w.dM, x.Rt, pl.ldm, w.G, n, m, inv_lambda));
     LN_LAUNCH("nn_dV", st, k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
   }
-  LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dKpart, n, m));
-  LN_LAUNCH("sign_cols_dLR", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dLRpart, n, m, pl.rpc));
+  if (fused_sign) {
+    LN_LAUNCH("sign2_dK_dLR", st, k_sign2<T, float><<<dim3(chs, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(
+        K, x.Lf, w.G, pl.ldm, w.dKpart, w.dLRpart, n, m, D, pl.s2_rpc));
+  } else {
+    LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dKpart, n, m));
+    LN_LAUNCH("sign_cols_dLR", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dLRpart, n, m, pl.rpc));
+  }
   // landmark gradient and its way back to the keys
   const int md = m * D;
   if (p->lm_mode == 1) {
-    LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, ch, w.dLRpart, ch, w.dLW, 1, w.dLtot, md));
+    LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chs, w.dLRpart, chs, w.dLW, 1, w.dLtot, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256), BH), 256, 0, st>>>(w.dKpart, w.dLtot, dK, geom_of(p), 1));
   } else {
-    LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, ch, w.dLRpart, ch, w.dLW, 1, dL, md));
+    LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chs, w.dLRpart, chs, w.dLW, 1, dL, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256), BH), 256, 0, st>>>(w.dKpart, nullptr, dK, geom_of(p), 0));
   }
   return launch_ok();
