@@ -29,6 +29,7 @@ struct Carver {
 
 struct Plan {
   int BH, n, d, m, T, ldm, rpc, chunks;
+  long long hslot;                   // floats per slot of the Newton-Schulz histories
   int s2_tg, s2_rpc, s2_chunks;      // fused sign pass: token groups per tile, tokens per chunk, chunks (0 = not used)
   size_t s2_smem;
 };
@@ -37,6 +38,9 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   if (!p) return false;
   pl->BH = p->B * p->H; pl->n = p->n; pl->d = p->d; pl->m = p->m; pl->T = p->ns_iters;
   pl->ldm = (p->m + 3) & ~3;
+  // history slots: fp32 [m][ldm], except on the m <= 64 tensor-core path, whose slots hold operand images
+  pl->hslot = (long long)p->m * pl->ldm;
+  if (p->dtype == LN_BF16 && p->m <= 64 && pl->hslot < (long long)(NsTile<64>::mat_bytes / 4)) pl->hslot = NsTile<64>::mat_bytes / 4;
   // token chunks per head for the reductions over tokens: about eight waves of CTAs (two per SM) so that
   // the last wave costs little, but at least 64 tokens per chunk
   const int mblk = (p->m + 63) / 64;
@@ -77,8 +81,8 @@ Ctx carve_ctx(const Plan& pl, void* base) {
   x.Rt = c.take(BH * n * pl.ldm);
   x.mu = c.take(BH * n);
   x.W = c.take(BH * m * m);
-  x.Xh = c.take(BH * (pl.T + 1) * m * pl.ldm);   // leading dimension ldm on the shared-memory path, m otherwise
-  x.Ph = c.take(BH * (pl.T > 0 ? pl.T : 1) * m * pl.ldm);   // W X_k of the forward pass (tensor-core path)
+  x.Xh = c.take(BH * (pl.T + 1) * (size_t)pl.hslot);
+  x.Ph = c.take(BH * (pl.T > 0 ? pl.T : 1) * (size_t)pl.hslot);   // W X_k (or 2I - W X_k) of the forward pass (tensor-core paths)
   x.M = c.take(BH * m * d);
   x.Yt = c.take(BH * m * d);
   x.ybar = c.take(BH * d);
@@ -185,19 +189,23 @@ struct TraceScope {
 };
 #define LN_LAUNCH(name, st, ...) do { TraceScope ts_(name, st); __VA_ARGS__; } while (0)
 
-// Tile of the l1 kernel for a problem: LG landmark groups of 4 (<= 16), TG token groups of 8,
-// LG * TG <= 256 threads (two CTAs per SM), chosen so that the tiles hug the problem.
-struct L1Launch { dim3 grid, block; size_t smem; };
-L1Launch plan_l1(int na_max, int nb, int batch, int nprob) {
-  int LG = (nb + 3) / 4; if (LG > 16) LG = 16; if (LG < 1) LG = 1;
+// Tile of the l1 kernel for a problem: LG landmark groups of QN (4 or 2) landmarks, TG token groups of 8,
+// LG * TG <= 256 threads, chosen so that the tiles hug the problem.  Small heads (few pairs per CTA) take
+// the two-landmark thread tile, which fits three CTAs per SM.
+struct L1Launch { dim3 grid, block; size_t smem; int qn; };
+L1Launch plan_l1(int na_max, int nb, int d, int batch, int nprob) {
+  const int qn = ((long long)na_max * nb * d <= (1ll << 20)) ? 2 : 4;
+  const int lg_cap = (qn == 4) ? 16 : 32;
+  int LG = (nb + qn - 1) / qn; if (LG > lg_cap) LG = lg_cap; if (LG < 1) LG = 1;
   int tg_cap = 256 / LG; if (tg_cap > 32) tg_cap = 32;       // at most 256 tokens per tile
   const int groups = (na_max + 7) / 8;
   const int tiles = (groups + tg_cap - 1) / tg_cap;
   int TG = (groups + tiles - 1) / tiles; if (TG < 1) TG = 1;
   L1Launch l;
+  l.qn = qn;
   l.block = dim3(LG, TG);
   l.grid = dim3((na_max + 8 * TG - 1) / (8 * TG), batch, nprob);
-  l.smem = sizeof(float) * ((size_t)(8 * TG + 4 * LG) * L1_PITCH + (size_t)8 * TG * LG);
+  l.smem = sizeof(float) * ((size_t)(8 * TG + qn * LG) * L1_PITCH + (size_t)8 * TG * LG);
   return l;
 }
 
@@ -212,9 +220,14 @@ L1Prob l1_prob(const void* A, int a_f32, float* E, float* rowsum, int na, int d,
 void launch_l1_args(const char* name, L1Args& a, int nprob, int batch, cudaStream_t st) {
   int na_max = 0;
   for (int i = 0; i < nprob; ++i) na_max = a.p[i].na > na_max ? a.p[i].na : na_max;
-  const L1Launch l = plan_l1(na_max, a.nb, batch, nprob);
-  cudaFuncSetAttribute(k_l1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.smem);
-  LN_LAUNCH(name, st, k_l1<<<l.grid, l.block, l.smem, st>>>(a));
+  const L1Launch l = plan_l1(na_max, a.nb, a.d, batch, nprob);
+  if (l.qn == 4) {
+    cudaFuncSetAttribute(k_l1<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.smem);
+    LN_LAUNCH(name, st, k_l1<4><<<l.grid, l.block, l.smem, st>>>(a));
+  } else {
+    cudaFuncSetAttribute(k_l1<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.smem);
+    LN_LAUNCH(name, st, k_l1<2><<<l.grid, l.block, l.smem, st>>>(a));
+  }
 }
 
 template <typename TA, typename TB>
@@ -263,7 +276,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       LN_LAUNCH("k_mid_fwd", st, kern<<<BH, 256, smem, st>>>(m, pl.ldm, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode, p->whiten,
                                                           x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt,
-                                                          x.ybar, dev_status));
+                                                          x.ybar, dev_status, pl.hslot));
     };
     if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * NsTile<64>::mat_bytes);
     else if (TC && m <= 128) launch(k_mid_fwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
@@ -310,9 +323,9 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       LN_LAUNCH("k_mid_bwd", st, kern<<<BH, 256, smem, st>>>(m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten, x.W, x.Xh,
                                                           x.Ph, x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P, w.Hm,
-                                                          w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status));
+                                                          w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot));
     };
-    if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 3 * NsTile<64>::mat_bytes);
+    if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 4 * NsTile<64>::mat_bytes);
     else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
     else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
   }

@@ -62,12 +62,15 @@ __device__ __forceinline__ void l1_fetch8(const void* base, bool f32, long long 
   }
 }
 
-__global__ void __launch_bounds__(256, 2) k_l1(const L1Args args) {
+// QN = landmarks per thread: 4 (128 registers, two CTAs per SM) for large problems; 2 (three CTAs per
+// SM) where a CTA lives too briefly for two of them to hide each other's loads and epilogues.
+template <int QN>
+__global__ void __launch_bounds__(256, QN == 4 ? 2 : 3) k_l1(const L1Args args) {
   extern __shared__ __align__(16) float l1_smem[];
   const L1Prob pr = args.p[blockIdx.z];
   const int LG = blockDim.x, TG = blockDim.y, tj = threadIdx.x, ti = threadIdx.y;
   const int tid = ti * LG + tj, nthr = LG * TG;
-  const int TA = 8 * TG, TB = 4 * LG;
+  const int TA = 8 * TG, TB = QN * LG;
   const int i0 = blockIdx.x * TA, b = blockIdx.y;
   if (i0 >= pr.na) return;
   float* As = l1_smem;                    // [TA][L1_PITCH]
@@ -81,11 +84,11 @@ __global__ void __launch_bounds__(256, 2) k_l1(const L1Args args) {
   for (int k = 0; k < 8; ++k) rs[k] = 0.f;
 
   for (int j0 = 0; j0 < nb; j0 += TB) {
-    float acc[8][4];
+    float acc[8][QN];
 #pragma unroll
     for (int k = 0; k < 8; ++k)
 #pragma unroll
-      for (int q = 0; q < 4; ++q) acc[k][q] = 0.f;
+      for (int q = 0; q < QN; ++q) acc[k][q] = 0.f;
 
     for (int c0 = 0; c0 < d; c0 += L1_DC) {
       __syncthreads();
@@ -115,15 +118,15 @@ __global__ void __launch_bounds__(256, 2) k_l1(const L1Args args) {
       __syncthreads();
 #pragma unroll
       for (int c4 = 0; c4 < L1_DC; c4 += 4) {
-        ulonglong2 a[8], nb[4];
+        ulonglong2 a[8], nb[QN];
 #pragma unroll
         for (int k = 0; k < 8; ++k) a[k] = *reinterpret_cast<const ulonglong2*>(As + (ti + TG * k) * L1_PITCH + c4);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) nb[q] = *reinterpret_cast<const ulonglong2*>(Bs + (tj + LG * q) * L1_PITCH + c4);
+        for (int q = 0; q < QN; ++q) nb[q] = *reinterpret_cast<const ulonglong2*>(Bs + (tj + LG * q) * L1_PITCH + c4);
 #pragma unroll
         for (int k = 0; k < 8; ++k)
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
+          for (int q = 0; q < QN; ++q) {
             const f32x2 t0 = add2(a[k].x, nb[q].x), t1 = add2(a[k].y, nb[q].y);   // dims c4, c4+1 and c4+2, c4+3
             acc[k][q] += fabsf(lo32(t0));
             acc[k][q] += fabsf(hi32(t0));
@@ -137,7 +140,7 @@ __global__ void __launch_bounds__(256, 2) k_l1(const L1Args args) {
       const int gi = i0 + ti + TG * k;
       if (gi >= na) continue;
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
+      for (int q = 0; q < QN; ++q) {
         const int gj = j0 + tj + LG * q;
         if (gj < nb) {
           const float e = ex2(acc[k][q] * args.nscale);
@@ -899,7 +902,9 @@ template <int D, bool TC, int MP>
 __global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float eps, float alpha_in, int H, int map_mode,
                                                  const float* __restrict__ whiten, const float* W, float* Wr,
                                                  float* P, float* Xh, float* Ph, NsHdr* hdr, const float* Mpart, int nchunks,
-                                                 float* Mout, float* Y, float* Yt, float* ybar, int* dev_status) {
+                                                 float* Mout, float* Y, float* Yt, float* ybar, int* dev_status,
+                                                 long long hslot) {
+  // hslot: floats per slot of the iterate histories (used by the MP = 64 path, whose slots hold operand images)
   // dynamic shared memory: the Newton-Schulz matrices (MP > 0), reused afterwards by the GEMM engine
   extern __shared__ __align__(16) unsigned char dyn_smem[];
   NsSmem& sm = *reinterpret_cast<NsSmem*>(dyn_smem);
@@ -908,7 +913,7 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float ep
   const long long mm = (long long)m * m, md = (long long)m * D;
   // the iterate histories of the shared-memory path use the padded leading dimension (128-bit accesses)
   const int ldx = (MP > 0) ? ldm : m;
-  const long long mx = (long long)m * ldx;
+  const long long mx = (MP == 64) ? hslot : (long long)m * ldx;
   W += bh * mm; Wr += bh * mm; P += bh * mm; Xh += (long long)bh * (T + 1) * mx; hdr += bh;
   if (Ph) Ph += (long long)bh * T * mx;
   Mout += bh * md; Y += bh * md; Yt += bh * md; ybar += (long long)bh * D;
@@ -921,7 +926,7 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float ep
     tc_ok = ns_forward_umma(m, T, eps, alpha_in, W, Xh, Ph, ldx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
     __syncthreads();
   } else if constexpr (MP == 64) {  // mma.sync from shared memory
-    ns_forward_smem<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, hdr, reinterpret_cast<bf16*>(dyn_smem), red);
+    ns_forward_smem<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red);
     __syncthreads();
   } else {
     ns_forward_dev<TC>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red);
@@ -973,14 +978,16 @@ __global__ void __launch_bounds__(256) k_mid_bwd(int m, int T, int H, int map_mo
                                                  const float* Xh, const float* Ph, const NsHdr* hdr, const float* Msaved,
                                                  const float* dYtpart, const float* dybpart, int nchunks,
                                                  float eps, float* Wr, float* P, float* Hm, float* Ga, float* Gb,
-                                                 float* dWm, float* dXm, float* dY, float* dM, float* GW, int* dev_status) {
+                                                 float* dWm, float* dXm, float* dY, float* dM, float* GW, int* dev_status,
+                                                 long long hslot) {
   extern __shared__ __align__(16) unsigned char dyn_smem[];
   NsSmem& sm = *reinterpret_cast<NsSmem*>(dyn_smem);
   __shared__ float red[2 * 256 + 8];
   const int bh = blockIdx.x, tid = threadIdx.x;
   const long long mm = (long long)m * m, md = (long long)m * D;
   const int ldx = (MP > 0) ? ldm : m;
-  const long long mx = (long long)m * ldx, ms = (long long)m * ldm;    // ms: size of one scratch matrix slot
+  const long long mx = (MP == 64) ? hslot : (long long)m * ldx;       // one slot of the iterate histories
+  const long long ms = (long long)m * ldm;                             // one scratch matrix
   W += bh * mm; Xh += (long long)bh * (T + 1) * mx; Ph += (long long)bh * T * mx; hdr += bh; Msaved += bh * md;
   Wr += bh * ms; P += bh * ms; Hm += bh * ms; Ga += bh * ms; Gb += bh * ms; dWm += bh * ms; dXm += bh * ms;
   dY += bh * md; dM += bh * md; GW += (long long)bh * m * ldm;
@@ -1019,7 +1026,7 @@ __global__ void __launch_bounds__(256) k_mid_bwd(int m, int T, int H, int map_mo
     __shared__ UmmaCtl ctl;
     const bool tc_ok = ns_backward_umma(m, T, eps, W, Xh, Ph, ldx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
     if (dev_status && !tc_ok && tid == 0) atomicOr(dev_status + bh, 2);
-  } else if constexpr (MP == 64) ns_backward_smem<MP>(m, T, eps, W, Xh, Ph, ldx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
+  } else if constexpr (MP == 64) ns_backward_smem<MP>(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
   else ns_backward_dev<TC>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red);
   // GW = (dW o K_LL + (dW o K_LL)^T) / lambda; four elements per batch so that the loads overlap
   for (long long e0 = (long long)tid * 4; e0 < (long long)m * ldm; e0 += 1024) {

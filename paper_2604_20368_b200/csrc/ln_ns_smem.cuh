@@ -181,15 +181,38 @@ __device__ inline void ns_norms(int m, float eps, float alpha_in, const float* W
   __syncthreads();
 }
 
-// Forward iteration.  smem: three matrices (W, X, P), 3 * NsTile<MP>::mat_bytes.  Xh (global, [T+1][m][m])
-// receives X_0 .. X_T in fp32; Ph (global, [T][m][m], may be NULL) receives W X_0 .. W X_{T-1}; both with
-// leading dimension ld >= m.
+
+// One matrix of this path as it lies in shared memory (hi part, lo part, rows of NsTile<MP>::LD bf16) is also
+// the format of the iterate history in global memory: the forward pass copies its operand images out, the
+// backward pass copies them back in with cp.async, and nothing is split or converted twice.
+template <int MP> __device__ __forceinline__ void image_to_global(const bf16* src, float* dst) {
+  constexpr int CH = (int)(NsTile<MP>::mat_bytes / 16);
+  const uint4* s4 = reinterpret_cast<const uint4*>(src);
+  uint4* d4 = reinterpret_cast<uint4*>(dst);
+  for (int c = threadIdx.x; c < CH; c += 256) d4[c] = s4[c];
+}
+// asynchronous global -> shared copy of one image; every thread commits exactly one group per call
+template <int MP> __device__ __forceinline__ void image_prefetch(const float* src, bf16* dst, bool issue) {
+  constexpr int CH = (int)(NsTile<MP>::mat_bytes / 16);
+  if (issue) {
+    const char* g = reinterpret_cast<const char*>(src);
+    const uint32_t s0 = smem_u32(dst);
+    for (int c = threadIdx.x; c < CH; c += 256)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s0 + 16u * c), "l"(g + 16ll * c) : "memory");
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+}
+// all but the most recent group of this thread have landed
+__device__ __forceinline__ void image_wait_all_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+
+// Forward iteration.  smem: three matrices (W, X, P), 3 * NsTile<MP>::mat_bytes.  Histories in global memory,
+// slots of hs floats: Xh slot k < T receives the operand image of X_k, slot T receives X_T in fp32 (leading
+// dimension ld >= m); Ph slot k (may be NULL) receives the image of Q_k = 2I - W X_k.
 template <int MP>
 __device__ void ns_forward_smem(int m, int T, float eps, float alpha_in, const float* W, float* Xh, float* Ph, int ld,
-                                NsHdr* hdr, bf16* smem, float* red) {
+                                long long hs, NsHdr* hdr, bf16* smem, float* red) {
   using TL = NsTile<MP>;
   bf16* sW = smem; bf16* sX = smem + 2 * TL::MAT; bf16* sP = smem + 4 * TL::MAT;
-  const long long mm = (long long)m * ld;      // stride of one matrix of the histories (leading dimension ld)
   // W + eps I is first staged in fp32 (in the space of P, which is not needed yet): norms, the split
   // copy of W, X_0 = alpha W^T and its fp32 copy for the backward pass are all built from there, so
   // global memory is read exactly once, coalesced.
@@ -242,13 +265,13 @@ __device__ void ns_forward_smem(int m, int T, float eps, float alpha_in, const f
     const float x0 = alpha * Wf[j * PF + i];                          // X_0 = alpha (W + eps I)^T
     split2(x0, h, l);
     sX[i * TL::LD + j] = h; sX[TL::MAT + i * TL::LD + j] = l;
-    if (i < m && j < m) Xh[(long long)i * ld + j] = x0;
+    if (T == 0 && i < m && j < m) Xh[(long long)i * ld + j] = x0;
   }
   __syncthreads();
+  if (T > 0) image_to_global<MP>(sX, Xh);
   float acc[TL::MT][TL::NT][4];
   for (int k = 0; k < T; ++k) {
     smem_gemm<MP, false, false>(acc, sW, sX, false);                    // W X_k
-    if (Ph) frag_to_global<MP>(acc, Ph + (long long)k * mm, m, ld);     // kept for the backward pass
 #pragma unroll
     for (int a = 0; a < TL::MT; ++a)
 #pragma unroll
@@ -261,11 +284,13 @@ __device__ void ns_forward_smem(int m, int T, float eps, float alpha_in, const f
         }
     frag_to_smem<MP>(acc, sP);
     __syncthreads();
+    if (Ph) image_to_global<MP>(sP, Ph + k * hs);                       // kept for the backward pass
     smem_gemm<MP, false, false>(acc, sX, sP, false);                    // X_{k+1} = X_k (2I - W X_k)
-    frag_to_global<MP>(acc, Xh + (long long)(k + 1) * mm, m, ld);
+    if (k + 1 == T) frag_to_global<MP>(acc, Xh + T * hs, m, ld);
     __syncthreads();                                                    // every warp is done reading X_k
     frag_to_smem<MP>(acc, sX);
     __syncthreads();
+    if (k + 1 < T) image_to_global<MP>(sX, Xh + (k + 1) * hs);
   }
 }
 
@@ -353,77 +378,70 @@ __device__ inline void ns_backward_tail(int m, float eps, const float* W, int ld
 }
 
 // Adjoint of the iteration for a symmetric W (the landmark kernel matrix is symmetric bit for bit).
-// Per step k (A = X_k, P = W A saved by the forward pass):
-//     H = A^T G,   dW -= H A^T,   G <- 2G - G P^T - P^T G.
-// The last term is W^T H = (A W)^T G in general; for symmetric W every iterate is a polynomial in W,
-// so A W = W A = P up to rounding, and W itself is not needed inside the loop.  Three matrices are
-// resident (A and P share a buffer, G, H): 3 * NsTile<MP>::mat_bytes of shared memory.
-// Xh, Ph: fp32 histories [T+1][m][m] and [T][m][m]; G0 = dLoss/dX_T; Gf: global fp32 [m][m] scratch
-// that holds G in full precision (each thread touches only its own fragment elements).
+// Per step k (A = X_k, Q = 2I - W A, both saved as operand images by the forward pass):
+//     H = A^T G,   dW -= H A^T,   G <- G Q^T + Q^T G - 2G.
+// In general the last term of the step adjoint is W^T H = (A W)^T G; for symmetric W every iterate is a
+// polynomial in W, so A W = W A up to rounding, (A W)^T G = (2I - Q)^T G, and W itself is not needed inside
+// the loop.  Four matrices are resident in shared memory (A, Q, G, H: 4 * NsTile<MP>::mat_bytes); A and Q of
+// the next step arrive by cp.async while this step computes.  G is kept in fp32 in registers (accumulator
+// layout) and re-split into shared memory after each update.
+// Xh, Ph: history slots of hs floats; G0 = dLoss/dX_T (fp32, leading dimension ld); Gf: global fp32 [m][ld]
+// scratch that receives the final G for the tail.
 template <int MP>
 __device__ void ns_backward_smem(int m, int T, float eps, const float* W, const float* Xh, const float* Ph, int ld,
-                                 const NsHdr* hdr, const float* G0, float* dW, float* Gf, bf16* smem, float* red) {
+                                 long long hs, const NsHdr* hdr, const float* G0, float* dW, float* Gf, bf16* smem,
+                                 float* red) {
   using TL = NsTile<MP>;
-  bf16* sA = smem; bf16* sG = smem + 2 * TL::MAT; bf16* sH = smem + 4 * TL::MAT;
-  const long long mm = (long long)m * ld;      // every [m][m] matrix here except W has leading dimension ld
-  float acc[TL::MT][TL::NT][4], dWr[TL::MT][TL::NT][4];
+  bf16* sA = smem; bf16* sQ = smem + 2 * TL::MAT; bf16* sG = smem + 4 * TL::MAT; bf16* sH = smem + 6 * TL::MAT;
+  image_prefetch<MP>(Xh + (long long)(T - 1) * hs, sA, T > 0);
+  image_prefetch<MP>(Ph + (long long)(T - 1) * hs, sQ, T > 0);
+  float acc[TL::MT][TL::NT][4], dWr[TL::MT][TL::NT][4], Gr[TL::MT][TL::NT][4];
 #pragma unroll
   for (int a = 0; a < TL::MT; ++a)
 #pragma unroll
     for (int t = 0; t < TL::NT; ++t)
 #pragma unroll
-      for (int q = 0; q < 4; ++q) dWr[a][t][q] = 0.f;
-  for (long long e = threadIdx.x; e < mm; e += 256) Gf[e] = G0[e];
-  global_to_smem_fast<MP>(G0, m, ld, sG);
+      for (int h = 0; h < 2; ++h) {
+        int i, j;
+        frag_ij<MP>(a, t, 2 * h, i, j);                                    // j is even: (j, j+1) are this thread's
+        float2 g = make_float2(0.f, 0.f);
+        if (i < m && j + 1 < m && (ld & 1) == 0) g = *reinterpret_cast<const float2*>(G0 + (long long)i * ld + j);
+        else {
+          if (i < m && j < m) g.x = G0[(long long)i * ld + j];
+          if (i < m && j + 1 < m) g.y = G0[(long long)i * ld + j + 1];
+        }
+        Gr[a][t][2 * h] = g.x; Gr[a][t][2 * h + 1] = g.y;
+        dWr[a][t][2 * h] = 0.f; dWr[a][t][2 * h + 1] = 0.f;
+      }
+  frag_to_smem<MP>(Gr, sG);
   for (int k = T - 1; k >= 0; --k) {
-    __syncthreads();
-    global_to_smem_fast<MP>(Xh + (long long)k * mm, m, ld, sA);                // A = X_k
+    image_wait_all_but_one();                                              // A = X_k has landed (Q_k may be in flight)
     __syncthreads();
     smem_gemm<MP, true, false>(acc, sA, sG, false);                        // H = A^T G
     frag_to_smem<MP>(acc, sH);
     __syncthreads();
     smem_gemm<MP, false, true>(dWr, sH, sA, true);                         // accumulates H A^T (dW = -sum)
     __syncthreads();                                                       // every warp is done reading A
-    global_to_smem_fast<MP>(Ph + (long long)k * mm, m, ld, sA);                // P = W X_k from the forward pass
+    image_prefetch<MP>(Xh + (long long)(k - 1) * hs, sA, k > 0);
+    image_wait_all_but_one();                                              // Q_k has landed
     __syncthreads();
-    smem_gemm<MP, false, true>(acc, sG, sA, false);                        // G P^T
-    smem_gemm<MP, true, false>(acc, sA, sG, true);                         // + P^T G
-    __syncthreads();                                                       // every warp is done reading G
+    smem_gemm<MP, false, true>(acc, sG, sQ, false);                        // G Q^T
+    smem_gemm<MP, true, false>(acc, sQ, sG, true);                         // + Q^T G
+    __syncthreads();                                                       // every warp is done reading G and Q
+    image_prefetch<MP>(Ph + (long long)(k - 1) * hs, sQ, k > 0);
 #pragma unroll
-    for (int a = 0; a < TL::MT; ++a) {
-      float2 g0[TL::NT][2];
-#pragma unroll
-      for (int t = 0; t < TL::NT; ++t)
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          int i, j;
-          frag_ij<MP>(a, t, 2 * h, i, j);                                  // j is even: (j, j+1) are this thread's
-          if (i < m && j + 1 < m && (ld & 1) == 0) g0[t][h] = *reinterpret_cast<const float2*>(Gf + (long long)i * ld + j);
-          else {
-            g0[t][h].x = (i < m && j < m) ? Gf[(long long)i * ld + j] : 0.f;
-            g0[t][h].y = (i < m && j + 1 < m) ? Gf[(long long)i * ld + j + 1] : 0.f;
-          }
-        }
+    for (int a = 0; a < TL::MT; ++a)
 #pragma unroll
       for (int t = 0; t < TL::NT; ++t)
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int q = 0; q < 4; ++q) {
           int i, j;
-          frag_ij<MP>(a, t, 2 * h, i, j);
-          float2 gn;
-          gn.x = (i < m && j < m) ? 2.f * g0[t][h].x - acc[a][t][2 * h] : 0.f;
-          gn.y = (i < m && j + 1 < m) ? 2.f * g0[t][h].y - acc[a][t][2 * h + 1] : 0.f;
-          if (i < m && j + 1 < m && (ld & 1) == 0) *reinterpret_cast<float2*>(Gf + (long long)i * ld + j) = gn;
-          else {
-            if (i < m && j < m) Gf[(long long)i * ld + j] = gn.x;
-            if (i < m && j + 1 < m) Gf[(long long)i * ld + j + 1] = gn.y;
-          }
-          acc[a][t][2 * h] = gn.x; acc[a][t][2 * h + 1] = gn.y;
+          frag_ij<MP>(a, t, q, i, j);
+          Gr[a][t][q] = (i < m && j < m) ? acc[a][t][q] - 2.f * Gr[a][t][q] : 0.f;
         }
-    }
-    frag_to_smem<MP>(acc, sG);
+    frag_to_smem<MP>(Gr, sG);
   }
-  // dW so far (minus the accumulated sum) goes to global memory in fragment layout
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
 #pragma unroll
   for (int a = 0; a < TL::MT; ++a)
 #pragma unroll
@@ -431,6 +449,7 @@ __device__ void ns_backward_smem(int m, int T, float eps, const float* W, const 
 #pragma unroll
       for (int q = 0; q < 4; ++q) dWr[a][t][q] = -dWr[a][t][q];
   frag_to_global<MP>(dWr, dW, m, ld);
+  frag_to_global<MP>(Gr, Gf, m, ld);
   __syncthreads();
   ns_backward_tail(m, eps, W, ld, hdr, dW, Gf, red);
   __syncthreads();
