@@ -56,8 +56,8 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   pl->s2_tg = pl->s2_rpc = pl->s2_chunks = 0; pl->s2_smem = 0;
   if (p->d % 64 == 0) {
     const int groups = (p->n + 7) / 8;
-    int tiles = (groups + 15) / 16;
-    int TG = (groups + tiles - 1) / tiles; TG += TG & 1; if (TG > 16) TG = 16;
+    int tiles = (groups + S2_TGMAX - 1) / S2_TGMAX;
+    int TG = (groups + tiles - 1) / tiles; TG += TG & 1; if (TG > S2_TGMAX) TG = S2_TGMAX; if (TG < 8) TG = 8;
     tiles = (p->n + 8 * TG - 1) / (8 * TG);
     const int slabs = p->d / 64;
     int wantc = (6 * kSMs + pl->BH * slabs - 1) / (pl->BH * slabs);
@@ -66,7 +66,7 @@ bool make_plan(const ln_problem* p, Plan* pl) {
     if (wantc < 1) wantc = 1;
     const int tpc = (tiles + wantc - 1) / wantc;
     pl->s2_tg = TG; pl->s2_rpc = tpc * 8 * TG; pl->s2_chunks = (p->n + pl->s2_rpc - 1) / pl->s2_rpc;
-    pl->s2_smem = sizeof(float) * (size_t)sign2_smem(p->m, TG).total;
+    pl->s2_smem = sign2_smem_bytes(p->m);
   }
   return true;
 }
