@@ -1,5 +1,6 @@
 // C ABI of the Laplacian-Nystrom library: host-side validation, buffer layout and launches.
 #include <math.h>
+#include <stdlib.h>
 #include <stdint.h>
 
 #include "../../include/laplace_nystrom.h"
@@ -308,10 +309,12 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const bool fused_sign = pl.s2_chunks > 0;
   const int chs = fused_sign ? pl.s2_chunks : ch;
   if (fused_sign) {
-    cudaFuncSetAttribute(k_sign2<T, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.s2_smem);
-    cudaFuncSetAttribute(k_sign2<T, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.s2_smem);
-    LN_LAUNCH("sign2_dQ_dLC", st, k_sign2<T, T><<<dim3(chs, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(
-        Q, x.Lf, w.G, pl.ldm, dQ, w.dLCpart, n, m, D, pl.s2_rpc));
+    auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
+      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.s2_smem);
+      LN_LAUNCH(name, st, kern<<<dim3(chs, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(tokp, x.Lf, w.G, pl.ldm, rowsp, partp, n, m, D, pl.s2_rpc));
+    };
+    if (pl.s2_tg == S2_TGMAX) launch2("sign2_dQ_dLC", k_sign2<T, T, 1>, Q, dQ, w.dLCpart);
+    else launch2("sign2_dQ_dLC", k_sign2<T, T, 2>, Q, dQ, w.dLCpart);
   } else {
     LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m));
     LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
@@ -339,8 +342,12 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     LN_LAUNCH("nn_dV", st, k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
   }
   if (fused_sign) {
-    LN_LAUNCH("sign2_dK_dLR", st, k_sign2<T, float><<<dim3(chs, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(
-        K, x.Lf, w.G, pl.ldm, w.dKpart, w.dLRpart, n, m, D, pl.s2_rpc));
+    auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
+      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.s2_smem);
+      LN_LAUNCH(name, st, kern<<<dim3(chs, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(tokp, x.Lf, w.G, pl.ldm, rowsp, partp, n, m, D, pl.s2_rpc));
+    };
+    if (pl.s2_tg == S2_TGMAX) launch2("sign2_dK_dLR", k_sign2<T, float, 1>, K, w.dKpart, w.dLRpart);
+    else launch2("sign2_dK_dLR", k_sign2<T, float, 2>, K, w.dKpart, w.dLRpart);
   } else {
     LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dKpart, n, m));
     LN_LAUNCH("sign_cols_dLR", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dLRpart, n, m, pl.rpc));

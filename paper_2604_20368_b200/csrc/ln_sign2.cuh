@@ -34,7 +34,8 @@ constexpr int S2_RS = S2_LS + 2 * S2_RL * S2_DS;                   // [2][TOK] r
 constexpr int S2_CS = S2_RS + 2 * S2_TOK;                          // [mr] column sums of g over the chunk
 __host__ __device__ inline size_t sign2_smem_bytes(int m) { return sizeof(float) * (size_t)(S2_CS + (m + S2_RL - 1) / S2_RL * S2_RL); }
 
-template <typename TT, typename TO>
+// NR = float2 column outputs per thread and round: 1 with 256 threads, 2 with 128 .. 254.
+template <typename TT, typename TO, int NR>
 __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, const float* __restrict__ Lm,
                                                   const float* __restrict__ G, int ldg, TO* __restrict__ rows,
                                                   float* __restrict__ part, int n, int m, int D, int rpc) {
@@ -71,19 +72,23 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
   const int ldst = (lpiece >> 4) * S2_DS + (lpiece & 15) * 4;      // float index inside one buffer of Ls
   float rs = 0.f;                                                  // sum over the rounds of a tile of this thread's g values
 
+  // fetch of the round the pointers stand at; tok_ok: this thread's token of that tile is inside the chunk
+  const float* gp = gsrc;
+  const float* lp = lsrc;
   auto fetch = [&](int tile, int r, float4& gq, float4& lq) {
     gq = make_float4(0.f, 0.f, 0.f, 0.f); lq = gq;
     const int lg = r * S2_RL + 4 * lhalf;
     if (ibeg + tile * TT8 + ltok < iend && lg < m) {
-      const float* gp = gsrc + (long long)tile * TT8 * ldg + r * S2_RL;
       if (gvec) gq = *reinterpret_cast<const float4*>(gp);
       else { gq.x = gp[0]; if (lg + 1 < m) gq.y = gp[1]; if (lg + 2 < m) gq.z = gp[2]; if (lg + 3 < m) gq.w = gp[3]; }
       if (lg + 1 >= m) gq.y = 0.f;
       if (lg + 2 >= m) gq.z = 0.f;
       if (lg + 3 >= m) gq.w = 0.f;
     }
-    if (lpiece >= 0 && r * S2_RL + (lpiece >> 4) < m) lq = *reinterpret_cast<const float4*>(lsrc + (long long)r * S2_RL * D);
+    if (lpiece >= 0 && r * S2_RL + (lpiece >> 4) < m) lq = *reinterpret_cast<const float4*>(lp);
   };
+  const long long g_tile_step = (long long)TT8 * ldg - (long long)(nrounds - 1) * S2_RL;   // last round of a tile -> round 0 of the next
+  const long long l_wrap = (long long)(nrounds - 1) * S2_RL * D;
   auto stash = [&](int buf, int tile, int r, const float4& gq, const float4& lq) {
     f32x2* g2 = Gs + buf * (S2_RL * S2_TOK) + gdst;
     g2[0] = pack2(gq.x, gq.x); g2[S2_TOK] = pack2(gq.y, gq.y); g2[2 * S2_TOK] = pack2(gq.z, gq.z); g2[3 * S2_TOK] = pack2(gq.w, gq.w);
@@ -115,22 +120,30 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
   __syncthreads();
   fold_colsum(0, 0);
 
-  constexpr int NOUT = 4;        // column outputs per thread and round (512 per round, at least 128 threads)
+  // column outputs of a round: 8 landmarks x 64 dims = 256 float2; thread o takes landmark o / 32, dims 2 (o % 32)
+  int cjj[NR], coff[NR];
+#pragma unroll
+  for (int u = 0; u < NR; ++u) {
+    const int o = tid + u * nthr;
+    cjj[u] = (o < S2_RL * 32) ? (o >> 5) : (1 << 20);          // out of range -> never below the landmarks left
+    coff[u] = (o >> 5) * D + 2 * (o & 31);
+  }
+  float* outr = outp;                         // outputs of the current round: outp + r * RL * D
   f32x2 qp[8][2], accR[8][2];
   int tile = 0, r = 0;
   for (int it = 0; it < total; ++it) {
     const int buf = it & 1;
     int tile_n = tile, r_n = r + 1;             // the round after this one
-    if (r_n == nrounds) { r_n = 0; ++tile_n; }
+    if (r_n == nrounds) { r_n = 0; ++tile_n; gp += g_tile_step; lp -= l_wrap; }
+    else { gp += S2_RL; lp += S2_RL * D; }
     float4 gq, lq;
     const bool more = it + 1 < total;
     if (more) fetch(tile_n, r_n, gq, lq);
-    float prev[NOUT];                           // running column sums of this round's landmarks (earlier tiles)
+    const int mleft = m - r * S2_RL;            // landmarks of this round that exist
+    float2 prev[NR];                            // running column sums of this round's landmarks (earlier tiles)
 #pragma unroll
-    for (int u = 0; u < NOUT; ++u) {
-      const int o = tid + u * nthr, l = r * S2_RL + (o >> 6);
-      prev[u] = (tile > 0 && o < S2_RL * S2_DS && l < m) ? outp[(long long)l * D + (o & 63)] : 0.f;
-    }
+    for (int u = 0; u < NR; ++u)
+      prev[u] = (tile > 0 && cjj[u] < mleft) ? *reinterpret_cast<const float2*>(outr + coff[u]) : make_float2(0.f, 0.f);
     if (r == 0) {
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
@@ -184,20 +197,23 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
     // column partials of this round -> running sums (fixed order over the token groups)
     const bool last_tile = tile == ntiles - 1;
 #pragma unroll
-    for (int u = 0; u < NOUT; ++u) {
-      const int o = tid + u * nthr, l = r * S2_RL + (o >> 6);
-      if (o < S2_RL * S2_DS && l < m) {
-        const float* src = Cp + buf * (S2_RL * S2_TGMAX * S2_DS) + (o >> 6) * (S2_TGMAX * S2_DS) + (o & 63);
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    for (int u = 0; u < NR; ++u) {
+      if (cjj[u] < mleft) {
+        const int o = tid + u * nthr;
+        const float* src = Cp + buf * (S2_RL * S2_TGMAX * S2_DS) + (o >> 5) * (S2_TGMAX * S2_DS) + 2 * (o & 31);
+        float2 s0 = make_float2(0.f, 0.f), s1 = s0;
 #pragma unroll
-        for (int g = 0; g < S2_TGMAX; g += 4) {
-          s0 += src[g * S2_DS]; s1 += src[(g + 1) * S2_DS]; s2 += src[(g + 2) * S2_DS]; s3 += src[(g + 3) * S2_DS];
+        for (int g = 0; g < S2_TGMAX; g += 2) {
+          const float2 a = *reinterpret_cast<const float2*>(src + g * S2_DS), b2 = *reinterpret_cast<const float2*>(src + (g + 1) * S2_DS);
+          s0.x += a.x; s0.y += a.y; s1.x += b2.x; s1.y += b2.y;
         }
-        const float v = prev[u] + ((s0 + s1) + (s2 + s3));
-        outp[(long long)l * D + (o & 63)] = last_tile ? 2.f * v - colsum[l] : v;
+        float2 v = make_float2(prev[u].x + (s0.x + s1.x), prev[u].y + (s0.y + s1.y));
+        if (last_tile) { const float cs = colsum[r * S2_RL + cjj[u]]; v.x = 2.f * v.x - cs; v.y = 2.f * v.y - cs; }
+        *reinterpret_cast<float2*>(outr + coff[u]) = v;
       }
     }
     if (more) fold_colsum(buf ^ 1, r_n);
+    if (r_n == 0) outr = outp; else outr += S2_RL * D;
     tile = tile_n; r = r_n;
   }
 }
