@@ -118,17 +118,22 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
     fetch(0, 0, gq, lq); stash(0, 0, 0, gq, lq);
   }
   __syncthreads();
-  fold_colsum(0, 0);
 
   // column outputs of a round: 8 landmarks x 64 dims = 256 float2; thread o takes landmark o / 32, dims 2 (o % 32)
-  int cjj[NR], coff[NR];
+  int cjj[NR], coff[NR], csrc[NR];
 #pragma unroll
   for (int u = 0; u < NR; ++u) {
     const int o = tid + u * nthr;
     cjj[u] = (o < S2_RL * 32) ? (o >> 5) : (1 << 20);          // out of range -> never below the landmarks left
     coff[u] = (o >> 5) * D + 2 * (o & 31);
+    csrc[u] = (o >> 5) * (S2_TGMAX * S2_DS) + 2 * (o & 31);
   }
-  float* outr = outp;                         // outputs of the current round: outp + r * RL * D
+  // The column partials of a round are added up while the NEXT round computes (their loads and adds are spread
+  // over its instruction stream), so that no phase of a round leaves the FMA pipe without work.
+  int red_buf = 0, red_mleft = 0, red_r = 0;    // the round whose partials are pending (red_mleft = 0: none)
+  bool red_last = false, red_first = true;
+  float* red_out = outp;
+  float* outr = outp;                           // outputs of the current round: outp + r * RL * D
   f32x2 qp[8][2], accR[8][2];
   int tile = 0, r = 0;
   for (int it = 0; it < total; ++it) {
@@ -139,11 +144,12 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
     float4 gq, lq;
     const bool more = it + 1 < total;
     if (more) fetch(tile_n, r_n, gq, lq);
-    const int mleft = m - r * S2_RL;            // landmarks of this round that exist
-    float2 prev[NR];                            // running column sums of this round's landmarks (earlier tiles)
+    float2 pend[NR], pend2[NR];                 // pending round: running sums of earlier tiles, then + partials
 #pragma unroll
-    for (int u = 0; u < NR; ++u)
-      prev[u] = (tile > 0 && cjj[u] < mleft) ? *reinterpret_cast<const float2*>(outr + coff[u]) : make_float2(0.f, 0.f);
+    for (int u = 0; u < NR; ++u) {
+      pend[u] = (!red_first && cjj[u] < red_mleft) ? *reinterpret_cast<const float2*>(red_out + coff[u]) : make_float2(0.f, 0.f);
+      pend2[u] = make_float2(0.f, 0.f);
+    }
     if (r == 0) {
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
@@ -157,8 +163,21 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
     const f32x2* g2 = Gs + buf * (S2_RL * S2_TOK) + tt * 8;
     const float* ls = Ls + buf * (S2_RL * S2_DS) + tc * 4;
     float* cp = Cp + buf * (S2_RL * S2_TGMAX * S2_DS) + tt * S2_DS + tc * 4;
+    const float* rsrc = Cp + red_buf * (S2_RL * S2_TGMAX * S2_DS);
 #pragma unroll
     for (int jj = 0; jj < S2_RL; ++jj) {
+      if ((jj & 1) == 0) {                      // a quarter of the pending round's partial sums
+#pragma unroll
+        for (int u = 0; u < NR; ++u)
+          if (cjj[u] < red_mleft) {
+            const float* src = rsrc + csrc[u] + (jj * 2) * S2_DS;
+            const float2 a0 = *reinterpret_cast<const float2*>(src), a1 = *reinterpret_cast<const float2*>(src + S2_DS);
+            const float2 a2 = *reinterpret_cast<const float2*>(src + 2 * S2_DS), a3 = *reinterpret_cast<const float2*>(src + 3 * S2_DS);
+            pend[u].x += a0.x; pend[u].y += a0.y; pend2[u].x += a1.x; pend2[u].y += a1.y;
+            pend[u].x += a2.x; pend[u].y += a2.y; pend2[u].x += a3.x; pend2[u].y += a3.y;
+          }
+      }
+      if (jj == 1) fold_colsum(buf, r);         // column sums of this round's g tile
       const ulonglong2 nl = *reinterpret_cast<const ulonglong2*>(ls + jj * S2_DS);
       f32x2 gg[8];
 #pragma unroll
@@ -180,6 +199,13 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
       ulonglong2 cs; cs.x = c0; cs.y = c1;
       *reinterpret_cast<ulonglong2*>(cp + jj * (S2_TGMAX * S2_DS)) = cs;
     }
+#pragma unroll
+    for (int u = 0; u < NR; ++u)
+      if (cjj[u] < red_mleft) {
+        float2 v = make_float2(pend[u].x + pend2[u].x, pend[u].y + pend2[u].y);
+        if (red_last) { const float cs = colsum[red_r * S2_RL + cjj[u]]; v.x = 2.f * v.x - cs; v.y = 2.f * v.y - cs; }
+        *reinterpret_cast<float2*>(red_out + coff[u]) = v;
+      }
     if (r == nrounds - 1) {                     // all landmarks seen: rows of this token tile
       const float* rsum = rowsum + (tile & 1) * S2_TOK + tt * 8;
 #pragma unroll
@@ -194,28 +220,24 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
     }
     if (more) stash(buf ^ 1, tile_n, r_n, gq, lq);
     __syncthreads();
-    // column partials of this round -> running sums (fixed order over the token groups)
-    const bool last_tile = tile == ntiles - 1;
-#pragma unroll
-    for (int u = 0; u < NR; ++u) {
-      if (cjj[u] < mleft) {
-        const int o = tid + u * nthr;
-        const float* src = Cp + buf * (S2_RL * S2_TGMAX * S2_DS) + (o >> 5) * (S2_TGMAX * S2_DS) + 2 * (o & 31);
-        float2 s0 = make_float2(0.f, 0.f), s1 = s0;
-#pragma unroll
-        for (int g = 0; g < S2_TGMAX; g += 2) {
-          const float2 a = *reinterpret_cast<const float2*>(src + g * S2_DS), b2 = *reinterpret_cast<const float2*>(src + (g + 1) * S2_DS);
-          s0.x += a.x; s0.y += a.y; s1.x += b2.x; s1.y += b2.y;
-        }
-        float2 v = make_float2(prev[u].x + (s0.x + s1.x), prev[u].y + (s0.y + s1.y));
-        if (last_tile) { const float cs = colsum[r * S2_RL + cjj[u]]; v.x = 2.f * v.x - cs; v.y = 2.f * v.y - cs; }
-        *reinterpret_cast<float2*>(outr + coff[u]) = v;
-      }
-    }
-    if (more) fold_colsum(buf ^ 1, r_n);
+    red_buf = buf; red_mleft = m - r * S2_RL; red_r = r; red_last = tile == ntiles - 1; red_first = tile == 0; red_out = outr;
     if (r_n == 0) outr = outp; else outr += S2_RL * D;
     tile = tile_n; r = r_n;
   }
+  // the last round's partials
+#pragma unroll
+  for (int u = 0; u < NR; ++u)
+    if (cjj[u] < red_mleft) {
+      const float* src = Cp + red_buf * (S2_RL * S2_TGMAX * S2_DS) + csrc[u];
+      float2 s0 = red_first ? make_float2(0.f, 0.f) : *reinterpret_cast<const float2*>(red_out + coff[u]), s1 = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int g = 0; g < S2_TGMAX; g += 2) {
+        const float2 a = *reinterpret_cast<const float2*>(src + g * S2_DS), b2 = *reinterpret_cast<const float2*>(src + (g + 1) * S2_DS);
+        s0.x += a.x; s0.y += a.y; s1.x += b2.x; s1.y += b2.y;
+      }
+      const float cs = colsum[red_r * S2_RL + cjj[u]];
+      *reinterpret_cast<float2*>(red_out + coff[u]) = make_float2(2.f * (s0.x + s1.x) - cs, 2.f * (s0.y + s1.y) - cs);
+    }
 }
 
 }  // namespace ln
