@@ -973,7 +973,7 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float ep
   }
 }
 template <int D, bool TC, int MP>
-__global__ void __launch_bounds__(256) k_mid_bwd(int m, int T, int H, int map_mode, float inv_lambda, int ldm,
+__global__ void __launch_bounds__(256, MP == 64 ? 3 : 1) k_mid_bwd(int m, int T, int H, int map_mode, float inv_lambda, int ldm,
                                                  const float* __restrict__ whiten, const float* W,
                                                  const float* Xh, const float* Ph, const NsHdr* hdr, const float* Msaved,
                                                  const float* dYtpart, const float* dybpart, int nchunks,

@@ -205,52 +205,38 @@ __global__ void __launch_bounds__(256) k_nn_mma(const float* __restrict__ E, int
 #pragma unroll
     for (int q = 0; q < 4; ++q) acc[t][q] = 0.f;
 
-  // The operand tiles of step l0 + KL are fetched into registers while step l0 is multiplied.
-  const int zr = tid >> 2, zcb = (tid & 3) * 8, zi = i0 + zr;      // Z tile: thread = (token, 8 landmarks)
-  const float mi = (mu && zi < n) ? mu[(long long)bh * n + zi] : 0.f;
-  constexpr int YP = KL * (D / 4) / 256;                            // float4 pieces of the Y tile per thread
-  float4 zq[2], yq[YP];
-  auto fetch = [&](int l0) {
+  for (int l0 = 0; l0 < m; l0 += KL) {
+    __syncthreads();
+    {  // Z tile: 64 tokens x 32 landmarks; thread = (token, 8 landmarks)
+      const int r = tid >> 2, cb = (tid & 3) * 8, i = i0 + r;
+      const float mi = (mu && i < n) ? mu[(long long)bh * n + i] : 0.f;
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      const int l = l0 + zcb + 4 * k;
-      zq[k] = (zi < n && l < m) ? ld4(E + (long long)zi * lde + l) : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int k = 0; k < 8; k += 4) {
+        const int l = l0 + cb + k;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (i < n && l < m) {
+          v = ld4(E + (long long)i * lde + l);
+          v.x = (l < m) ? v.x - mi : 0.f;
+          v.y = (l + 1 < m) ? v.y - mi : 0.f;
+          v.z = (l + 2 < m) ? v.z - mi : 0.f;
+          v.w = (l + 3 < m) ? v.w - mi : 0.f;
+        }
+        uint2 h, lo;
+        split4(v, h, lo);
+        *reinterpret_cast<uint2*>(&Zhi[r][cb + k]) = h;
+        *reinterpret_cast<uint2*>(&Zlo[r][cb + k]) = lo;
+      }
     }
-#pragma unroll
-    for (int u = 0; u < YP; ++u) {
-      const int idx = tid + u * 256, r = idx / (D / 4), c4 = (idx % (D / 4)) * 4, l = l0 + r;
-      yq[u] = (l < m) ? ld4(Y + (long long)l * D + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-  };
-  auto stash = [&](int l0) {
-#pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      const int l = l0 + zcb + 4 * k;
-      float4 v = zq[k];
-      v.x = (zi < n && l < m) ? v.x - mi : 0.f;
-      v.y = (zi < n && l + 1 < m) ? v.y - mi : 0.f;
-      v.z = (zi < n && l + 2 < m) ? v.z - mi : 0.f;
-      v.w = (zi < n && l + 3 < m) ? v.w - mi : 0.f;
+    for (int idx = tid; idx < KL * (D / 4); idx += 256) {
+      const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4, l = l0 + r;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (l < m) v = ld4(Y + (long long)l * D + c4);
       uint2 h, lo;
       split4(v, h, lo);
-      *reinterpret_cast<uint2*>(&Zhi[zr][zcb + 4 * k]) = h;
-      *reinterpret_cast<uint2*>(&Zlo[zr][zcb + 4 * k]) = lo;
-    }
-#pragma unroll
-    for (int u = 0; u < YP; ++u) {
-      const int idx = tid + u * 256, r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
-      uint2 h, lo;
-      split4(yq[u], h, lo);
       *reinterpret_cast<uint2*>(&Yhi[r][c4]) = h;
       *reinterpret_cast<uint2*>(&Ylo[r][c4]) = lo;
     }
-  };
-  fetch(0);
-  for (int l0 = 0; l0 < m; l0 += KL) {
     __syncthreads();
-    stash(l0);
-    __syncthreads();
-    if (l0 + KL < m) fetch(l0 + KL);
 #pragma unroll
     for (int k0 = 0; k0 < KL; k0 += 16) {
       uint32_t ah[4], al[4];
