@@ -210,6 +210,19 @@ L1Launch plan_l1(int na_max, int nb, int d, int batch, int nprob) {
   return l;
 }
 
+// Launch with `cl` CTAs per thread-block cluster (cl = 1: an ordinary launch).
+constexpr int kMidCluster = 4;     // CTAs that share one head on the m > 128 Newton-Schulz path
+template <typename... KArgs, typename... Args>
+void launch_clustered(void (*kern)(KArgs...), int grid, int cl, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = cl; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 template <typename T> constexpr int is_f32() { return std::is_same<T, float>::value ? 1 : 0; }
 
 L1Prob l1_prob(const void* A, int a_f32, float* E, float* rowsum, int na, int d, int lde, float rs_scale) {
@@ -273,14 +286,15 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // Newton-Schulz, Y = X M, folded map
   {
     constexpr bool TC = std::is_same<T, bf16>::value;
-    auto launch = [&](auto kern, size_t smem) {
+    auto launch = [&](auto kern, size_t smem, int cl = 1) {
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      LN_LAUNCH("k_mid_fwd", st, kern<<<BH, 256, smem, st>>>(m, pl.ldm, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode, p->whiten,
-                                                          x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt,
-                                                          x.ybar, dev_status, pl.hslot));
+      LN_LAUNCH("k_mid_fwd", st, launch_clustered(kern, BH * cl, cl, smem, st, m, pl.ldm, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode,
+                                                  p->whiten, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt,
+                                                  x.ybar, dev_status, pl.hslot));
     };
     if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * NsTile<64>::mat_bytes);
     else if (TC && m <= 128) launch(k_mid_fwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
+    else if (TC) launch(k_mid_fwd<D, TC, 0, TC ? kMidCluster : 1>, sizeof(NsSmem), kMidCluster);   // m > 128: a cluster per head
     else launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));
   }
   // O = (C - mu) Ytilde + ybar
@@ -322,14 +336,15 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // per head: dY, dX, dM, Newton-Schulz adjoint, symmetrised landmark-block upstream
   {
     constexpr bool TC = std::is_same<T, bf16>::value;
-    auto launch = [&](auto kern, size_t smem) {
+    auto launch = [&](auto kern, size_t smem, int cl = 1) {
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      LN_LAUNCH("k_mid_bwd", st, kern<<<BH, 256, smem, st>>>(m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten, x.W, x.Xh,
-                                                          x.Ph, x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P, w.Hm,
-                                                          w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot));
+      LN_LAUNCH("k_mid_bwd", st, launch_clustered(kern, BH * cl, cl, smem, st, m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten,
+                                                  x.W, x.Xh, x.Ph, x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P,
+                                                  w.Hm, w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot));
     };
     if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 4 * NsTile<64>::mat_bytes);
     else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
+    else if (TC) launch(k_mid_bwd<D, TC, 0, TC ? kMidCluster : 1>, sizeof(NsSmem), kMidCluster);
     else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
   }
   LN_LAUNCH("sign_rows_dLW", st, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, st>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));

@@ -120,6 +120,18 @@ __device__ inline float block_sum(float v, float* red /* >= 8 floats of shared m
   return s;
 }
 
+// End of a phase of a per-head kernel that CL CTAs of a thread-block cluster share (CL = 1: one CTA per head).
+// What the CTAs wrote to global memory before the barrier is visible to all of them after it.  The cluster
+// barrier is a hardware barrier (no spinning); every thread of every CTA of the cluster must reach it.
+template <int CL> __device__ __forceinline__ void phase_sync() {
+  if (CL > 1) {
+    __threadfence();
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+  } else {
+    __syncthreads();
+  }
+}
+
 // Header kept per matrix beside the Newton-Schulz iterates.
 struct NsHdr { float alpha, n1, ninf; int jstar, istar, auto_alpha, pad0, pad1; };
 

@@ -734,11 +734,11 @@ union __align__(16) NsSmem { GemmSmem f; MmaGemmSmem t; MmaGemmSmemBig b; };
 template <bool TC, bool TRA, bool TRB, bool BIG = false>
 __device__ __forceinline__ void ns_gemm(int M, int N, int K, const float* A, int lda, const float* Bm, int ldb,
                                         float* C, int ldc, float alpha, float beta, const float* Cin, float diag,
-                                        NsSmem& sm) {
+                                        NsSmem& sm, int part = 0, int nparts = 1) {
   if (TC) {
     // the 128 x 128-tile engine is compiled only where m can exceed 128 (it costs registers)
-    if (BIG && M > 128 && N > 64) cta_gemm_mma_big<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.b);
-    else cta_gemm_mma<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.t);
+    if (BIG && M > 128 && N > 64) cta_gemm_mma_big<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.b, part, nparts);
+    else cta_gemm_mma<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.t, part, nparts);
   } else {
     cta_gemm<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, sm.f);
     if (diag != 0.f) {
@@ -755,16 +755,18 @@ __device__ __forceinline__ void ns_gemm(int M, int N, int K, const float* A, int
 //   X_{k+1} = X_k (2I - Wr X_k);  Xh[k] = X_k for k = 0..T.
 // W, Wr, P: [m][m] in global memory; Xh: [T+1][m][m].
 // =====================================================================================
-template <bool TC>
+template <bool TC, int CL = 1>
 __device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const float* W, float* Wr, float* P,
-                               float* Xh, NsHdr* hdr, NsSmem& sm, float* red /* 2*256 + 8 floats */) {
-  const int tid = threadIdx.x;
+                               float* Xh, NsHdr* hdr, NsSmem& sm, float* red /* 2*256 + 8 floats */, int crank = 0) {
+  // CL CTAs of a cluster share the work (crank = this CTA's rank): element-wise phases are strided over all their
+  // threads, every product is split by output tiles, small reductions are done by each CTA for itself.
+  const int tid = threadIdx.x, gt = crank * 256 + tid, gn = 256 * CL;
   const long long mm = (long long)m * m;
-  for (long long e = tid; e < mm; e += 256) {
+  for (long long e = gt; e < mm; e += gn) {
     const int i = (int)(e / m), j = (int)(e % m);
     Wr[e] = W[e] + (i == j ? eps : 0.f);
   }
-  __syncthreads();
+  phase_sync<CL>();
   float* colsum = red;          // [256]
   float* rowsum = red + 256;    // [256]
   if (tid < m) {
@@ -773,29 +775,35 @@ __device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const fl
     colsum[tid] = cs; rowsum[tid] = rs;
   }
   __syncthreads();
-  if (tid == 0) {
+  if (tid == 0) {               // every CTA of a cluster arrives at the same values
     float n1 = -1.f, ninf = -1.f; int js = 0, is = 0;
     for (int t = 0; t < m; ++t) {                 // strict > keeps the lowest index on ties
       if (colsum[t] > n1) { n1 = colsum[t]; js = t; }
       if (rowsum[t] > ninf) { ninf = rowsum[t]; is = t; }
     }
-    hdr->n1 = n1; hdr->ninf = ninf; hdr->jstar = js; hdr->istar = is;
-    hdr->auto_alpha = !(alpha_in > 0.f);
-    hdr->alpha = (alpha_in > 0.f) ? alpha_in : 1.f / (n1 * ninf);
-    hdr->pad0 = hdr->pad1 = 0;
+    float* al = red + 512;
+    al[0] = (alpha_in > 0.f) ? alpha_in : 1.f / (n1 * ninf);
+    if (crank == 0) {
+      hdr->n1 = n1; hdr->ninf = ninf; hdr->jstar = js; hdr->istar = is;
+      hdr->auto_alpha = !(alpha_in > 0.f);
+      hdr->alpha = al[0];
+      hdr->pad0 = hdr->pad1 = 0;
+    }
   }
   __syncthreads();
-  const float alpha = hdr->alpha;
-  for (long long e = tid; e < mm; e += 256) {
+  const float alpha = red[512];
+  for (long long e = gt; e < mm; e += gn) {
     const int i = (int)(e / m), j = (int)(e % m);
     Xh[e] = alpha * Wr[(long long)j * m + i];
   }
-  __syncthreads();
+  phase_sync<CL>();
   for (int k = 0; k < T; ++k) {
     const float* X = Xh + (long long)k * mm;
     float* Xn = Xh + (long long)(k + 1) * mm;
-    ns_gemm<TC, false, false, true>(m, m, m, Wr, m, X, m, P, m, -1.f, 0.f, nullptr, 2.f, sm);   // P = 2I - Wr X_k
-    ns_gemm<TC, false, false, true>(m, m, m, X, m, P, m, Xn, m, 1.f, 0.f, nullptr, 0.f, sm);    // X_{k+1} = X_k P
+    ns_gemm<TC, false, false, true>(m, m, m, Wr, m, X, m, P, m, -1.f, 0.f, nullptr, 2.f, sm, crank, CL);   // P = 2I - Wr X_k
+    if (CL > 1) phase_sync<CL>();
+    ns_gemm<TC, false, false, true>(m, m, m, X, m, P, m, Xn, m, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);    // X_{k+1} = X_k P
+    if (CL > 1) phase_sync<CL>();
   }
 }
 
@@ -803,50 +811,54 @@ __device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const fl
 // Exact adjoint of ns_forward_dev: given G0 = dLoss/dX_T returns dW = dLoss/dW.
 // Scratch matrices [m][m]: P, Hm, Ga, Gb.  Xh holds X_0..X_T, Wr = W + eps I, hdr from the forward.
 // =====================================================================================
-template <bool TC>
+template <bool TC, int CL = 1>
 __device__ void ns_backward_dev(int m, int T, const float* Wr, const float* Xh, const NsHdr* hdr,
                                 const float* G0, float* dW, float* P, float* Hm, float* Ga, float* Gb,
-                                NsSmem& sm, float* red) {
-  const int tid = threadIdx.x;
+                                NsSmem& sm, float* red, int crank = 0) {
+  const int tid = threadIdx.x, gt = crank * 256 + tid, gn = 256 * CL;
   const long long mm = (long long)m * m;
-  for (long long e = tid; e < mm; e += 256) { Ga[e] = G0[e]; dW[e] = 0.f; }
-  __syncthreads();
+  for (long long e = gt; e < mm; e += gn) { Ga[e] = G0[e]; dW[e] = 0.f; }
+  phase_sync<CL>();
   float* G = Ga; float* Gn = Gb;
   for (int k = T - 1; k >= 0; --k) {
     const float* A = Xh + (long long)k * mm;                                        // X_{k+1} = 2A - A P, P = Wr A
-    ns_gemm<TC, false, false, true>(m, m, m, Wr, m, A, m, P, m, 1.f, 0.f, nullptr, 0.f, sm);      // P = Wr A
-    ns_gemm<TC, true, false, true>(m, m, m, A, m, G, m, Hm, m, 1.f, 0.f, nullptr, 0.f, sm);       // H = A^T G
-    ns_gemm<TC, false, true, true>(m, m, m, Hm, m, A, m, dW, m, -1.f, 1.f, dW, 0.f, sm);          // dW -= H A^T
-    ns_gemm<TC, false, true, true>(m, m, m, G, m, P, m, Gn, m, -1.f, 2.f, G, 0.f, sm);            // Gn = 2G - G P^T
-    ns_gemm<TC, true, false, true>(m, m, m, Wr, m, Hm, m, Gn, m, -1.f, 1.f, Gn, 0.f, sm);         // Gn -= Wr^T H
+    ns_gemm<TC, false, false, true>(m, m, m, Wr, m, A, m, P, m, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);      // P = Wr A
+    ns_gemm<TC, true, false, true>(m, m, m, A, m, G, m, Hm, m, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);       // H = A^T G
+    if (CL > 1) phase_sync<CL>();
+    ns_gemm<TC, false, true, true>(m, m, m, Hm, m, A, m, dW, m, -1.f, 1.f, dW, 0.f, sm, crank, CL);          // dW -= H A^T
+    ns_gemm<TC, false, true, true>(m, m, m, G, m, P, m, Gn, m, -1.f, 2.f, G, 0.f, sm, crank, CL);            // Gn = 2G - G P^T
+    ns_gemm<TC, true, false, true>(m, m, m, Wr, m, Hm, m, Gn, m, -1.f, 1.f, Gn, 0.f, sm, crank, CL);         // Gn -= Wr^T H
+    if (CL > 1) phase_sync<CL>();
     float* t = G; G = Gn; Gn = t;
   }
   // X_0 = alpha Wr^T
   const float alpha = hdr->alpha;
   float part = 0.f;
-  for (long long e = tid; e < mm; e += 256) {
+  for (long long e = tid; e < mm; e += 256) {        // every CTA of a cluster sums everything (same order, same value)
     const int i = (int)(e / m), j = (int)(e % m);
     part += G[e] * Wr[(long long)j * m + i];
   }
   const float dalpha = block_sum(part, red);
-  for (long long e = tid; e < mm; e += 256) {
+  for (long long e = gt; e < mm; e += gn) {
     const int j = (int)(e / m), i = (int)(e % m);      // dW[j][i] += alpha G[i][j]
     dW[e] += alpha * G[(long long)i * m + j];
   }
-  __syncthreads();
+  phase_sync<CL>();
   if (hdr->auto_alpha) {
     const int js = hdr->jstar, is = hdr->istar;
     const float c1 = dalpha * (-alpha / hdr->n1), c2 = dalpha * (-alpha / hdr->ninf);
-    for (int i = tid; i < m; i += 256) {
-      const float w = Wr[(long long)i * m + js];
-      dW[(long long)i * m + js] += c1 * (w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f));
-    }
+    if (crank == 0)
+      for (int i = tid; i < m; i += 256) {
+        const float w = Wr[(long long)i * m + js];
+        dW[(long long)i * m + js] += c1 * (w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f));
+      }
     __syncthreads();
-    for (int j = tid; j < m; j += 256) {
-      const float w = Wr[(long long)is * m + j];
-      dW[(long long)is * m + j] += c2 * (w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f));
-    }
-    __syncthreads();
+    if (crank == 0)
+      for (int j = tid; j < m; j += 256) {
+        const float w = Wr[(long long)is * m + j];
+        dW[(long long)is * m + j] += c2 * (w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f));
+      }
+    phase_sync<CL>();
   }
 }
 
@@ -898,8 +910,9 @@ __global__ void __launch_bounds__(256) k_ns_pinv_bwd(int m, int T, float eps, fl
 // then fold the injective map (Prop. 3) into Ytilde_l = s_l Y_l - mean_l'(s_l' Y_l'), ybar = mean_l Y_l
 // so that O = (C - mu) Ytilde + ybar.  One CTA per head.
 // =====================================================================================
-template <int D, bool TC, int MP>
-__global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float eps, float alpha_in, int H, int map_mode,
+// CL > 1 (generic path only): CL CTAs of a thread-block cluster share one head; grid = heads * CL.
+template <int D, bool TC, int MP, int CL = 1>
+__global__ void __launch_bounds__(256, CL > 1 ? 2 : 1) k_mid_fwd(int m, int ldm, int T, float eps, float alpha_in, int H, int map_mode,
                                                  const float* __restrict__ whiten, const float* W, float* Wr,
                                                  float* P, float* Xh, float* Ph, NsHdr* hdr, const float* Mpart, int nchunks,
                                                  float* Mout, float* Y, float* Yt, float* ybar, int* dev_status,
@@ -909,7 +922,8 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float ep
   extern __shared__ __align__(16) unsigned char dyn_smem[];
   NsSmem& sm = *reinterpret_cast<NsSmem*>(dyn_smem);
   __shared__ float red[2 * 256 + 8];
-  const int bh = blockIdx.x, tid = threadIdx.x;
+  const int bh = blockIdx.x / CL, crank = blockIdx.x % CL, tid = threadIdx.x;
+  const int gt = crank * 256 + tid, gn = 256 * CL;      // this thread among all threads that share the head
   const long long mm = (long long)m * m, md = (long long)m * D;
   // the iterate histories of the shared-memory path use the padded leading dimension (128-bit accesses)
   const int ldx = (MP > 0) ? ldm : m;
@@ -918,7 +932,7 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float ep
   if (Ph) Ph += (long long)bh * T * mx;
   Mout += bh * md; Y += bh * md; Yt += bh * md; ybar += (long long)bh * D;
   Mpart += (long long)bh * nchunks * md;
-  for (long long e = (long long)tid * 4; e < md; e += 1024)
+  for (long long e = (long long)gt * 4; e < md; e += 4 * gn)
     *reinterpret_cast<float4*>(Mout + e) = sum_parts4(Mpart, nchunks, md, e);
   bool tc_ok = true;
   if constexpr (MP == 128) {        // tcgen05 + TMEM
@@ -929,16 +943,17 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float ep
     ns_forward_smem<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red);
     __syncthreads();
   } else {
-    ns_forward_dev<TC>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red);
+    ns_forward_dev<TC, CL>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red, crank);
   }
   const float* XT = Xh + (long long)T * mx;
   if (dev_status) {
     float bad = 0.f;
     for (int e = tid; e < m * m; e += 256) bad += isfinite(XT[(long long)(e / m) * ldx + e % m]) ? 0.f : 1.f;
     bad = block_sum(bad, red);
-    if (tid == 0) atomicOr(dev_status + bh, (bad > 0.f ? 1 : 0) | (tc_ok ? 0 : 2));   // bit1: a bounded tensor-core wait ran out
+    if (tid == 0 && crank == 0) atomicOr(dev_status + bh, (bad > 0.f ? 1 : 0) | (tc_ok ? 0 : 2));   // bit1: a bounded tensor-core wait ran out
   }
-  ns_gemm<TC, false, false>(m, D, m, XT, ldx, Mout, D, Y, D, 1.f, 0.f, nullptr, 0.f, sm);   // Y = X M
+  ns_gemm<TC, false, false>(m, D, m, XT, ldx, Mout, D, Y, D, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // Y = X M
+  if (CL > 1) phase_sync<CL>();
   const float* s = whiten ? whiten + (long long)(bh % H) * m : nullptr;
   // fold the injective map (Prop. 3): column means over the landmarks first (eight independent loads per
   // batch), then every element in parallel
@@ -958,10 +973,10 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float ep
     }
     colstat[tid] = sy / (float)m;
     colstat[D + tid] = y1 / (float)m;
-    ybar[tid] = (map_mode == 1) ? y1 / (float)m : 0.f;
+    if (crank == 0) ybar[tid] = (map_mode == 1) ? y1 / (float)m : 0.f;
   }
   __syncthreads();
-  for (long long e = (long long)tid * 4; e < md; e += 1024) {
+  for (long long e = (long long)gt * 4; e < md; e += 4 * gn) {
     const int l = (int)(e / D), c = (int)(e % D);
     float4 y = *reinterpret_cast<const float4*>(Y + e);
     if (map_mode == 1) {
@@ -972,8 +987,8 @@ __global__ void __launch_bounds__(256) k_mid_fwd(int m, int ldm, int T, float ep
     *reinterpret_cast<float4*>(Yt + e) = y;
   }
 }
-template <int D, bool TC, int MP>
-__global__ void __launch_bounds__(256, MP == 64 ? 3 : 1) k_mid_bwd(int m, int T, int H, int map_mode, float inv_lambda, int ldm,
+template <int D, bool TC, int MP, int CL = 1>
+__global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_bwd(int m, int T, int H, int map_mode, float inv_lambda, int ldm,
                                                  const float* __restrict__ whiten, const float* W,
                                                  const float* Xh, const float* Ph, const NsHdr* hdr, const float* Msaved,
                                                  const float* dYtpart, const float* dybpart, int nchunks,
@@ -983,7 +998,8 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : 1) k_mid_bwd(int m, int T,
   extern __shared__ __align__(16) unsigned char dyn_smem[];
   NsSmem& sm = *reinterpret_cast<NsSmem*>(dyn_smem);
   __shared__ float red[2 * 256 + 8];
-  const int bh = blockIdx.x, tid = threadIdx.x;
+  const int bh = blockIdx.x / CL, crank = blockIdx.x % CL, tid = threadIdx.x;
+  const int gt = crank * 256 + tid, gn = 256 * CL;
   const long long mm = (long long)m * m, md = (long long)m * D;
   const int ldx = (MP > 0) ? ldm : m;
   const long long mx = (MP == 64) ? hslot : (long long)m * ldx;       // one slot of the iterate histories
@@ -1000,7 +1016,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : 1) k_mid_bwd(int m, int T,
     dyb[tid] = t;
   }
   __syncthreads();
-  for (long long e = (long long)tid * 4; e < md; e += 1024) {
+  for (long long e = (long long)gt * 4; e < md; e += 4 * gn) {
     const float4 t = sum_parts4(dYtpart, nchunks, md, e);
     const int l = (int)(e / D), c = (int)(e % D);
     // Ytilde = P_c diag(s) Y, ybar = Y^T 1/m  ->  dY = diag(s) (centred Z'^T dO) + (1/m) 1 dyb^T
@@ -1013,23 +1029,24 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : 1) k_mid_bwd(int m, int T,
     *reinterpret_cast<float4*>(dY + e) = o;
   }
   if constexpr (MP == 0) {
-    for (long long e = tid; e < mm; e += 256) {
+    for (long long e = gt; e < mm; e += gn) {
       const int i = (int)(e / m), j = (int)(e % m);
       Wr[e] = W[e] + (i == j ? eps : 0.f);
     }
   }
-  __syncthreads();
+  phase_sync<CL>();
   const float* XT = Xh + (long long)T * mx;
-  ns_gemm<TC, false, true>(m, m, D, dY, D, Msaved, D, dXm, ldx, 1.f, 0.f, nullptr, 0.f, sm);   // dX = dY M^T
-  ns_gemm<TC, true, false>(m, D, m, XT, ldx, dY, D, dM, D, 1.f, 0.f, nullptr, 0.f, sm);        // dM = X^T dY
+  ns_gemm<TC, false, true>(m, m, D, dY, D, Msaved, D, dXm, ldx, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // dX = dY M^T
+  ns_gemm<TC, true, false>(m, D, m, XT, ldx, dY, D, dM, D, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);        // dM = X^T dY
+  if (CL > 1) phase_sync<CL>();
   if constexpr (MP == 128) {
     __shared__ UmmaCtl ctl;
     const bool tc_ok = ns_backward_umma(m, T, eps, W, Xh, Ph, ldx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
     if (dev_status && !tc_ok && tid == 0) atomicOr(dev_status + bh, 2);
   } else if constexpr (MP == 64) ns_backward_smem<MP>(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
-  else ns_backward_dev<TC>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red);
+  else { ns_backward_dev<TC, CL>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red, crank); if (CL > 1) phase_sync<CL>(); }
   // GW = (dW o K_LL + (dW o K_LL)^T) / lambda; four elements per batch so that the loads overlap
-  for (long long e0 = (long long)tid * 4; e0 < (long long)m * ldm; e0 += 1024) {
+  for (long long e0 = (long long)gt * 4; e0 < (long long)m * ldm; e0 += 4 * gn) {
     float a[4], b[4], c[4], d4[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {

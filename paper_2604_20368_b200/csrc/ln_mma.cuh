@@ -390,12 +390,17 @@ __device__ __forceinline__ void gemm_stash(bf16* hi, bf16* lo, const float (&v)[
 
 template <bool TRA, bool TRB>
 __device__ void cta_gemm_mma(int M, int N, int K, const float* A, int lda, const float* Bm, int ldb, float* C,
-                             int ldc, float alpha, float beta, const float* Cin, float diag, MmaGemmSmem& sm) {
+                             int ldc, float alpha, float beta, const float* Cin, float diag, MmaGemmSmem& sm,
+                             int part = 0, int nparts = 1) {
+  // part / nparts: this CTA computes the output tiles whose running number is part modulo nparts (the CTAs of a
+  // cluster share one product)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int wm = (warp & 3) * 16, wn = (warp >> 2) * 32;
   const int g = lane >> 2, t4 = lane & 3;
+  int tile_no = 0;
   for (int i0 = 0; i0 < M; i0 += 64)
     for (int j0 = 0; j0 < N; j0 += 64) {
+      if ((tile_no++) % nparts != part) continue;
       float acc[4][4];
 #pragma unroll
       for (int t = 0; t < 4; ++t)
@@ -491,12 +496,15 @@ __device__ __forceinline__ void gemm_stash_big(bf16* hi, bf16* lo, const float (
 
 template <bool TRA, bool TRB>
 __device__ void cta_gemm_mma_big(int M, int N, int K, const float* A, int lda, const float* Bm, int ldb, float* C,
-                                 int ldc, float alpha, float beta, const float* Cin, float diag, MmaGemmSmemBig& sm) {
+                                 int ldc, float alpha, float beta, const float* Cin, float diag, MmaGemmSmemBig& sm,
+                                 int part = 0, int nparts = 1) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int wm = (warp & 3) * 32, wn = (warp >> 2) * 64;
   const int g = lane >> 2, t4 = lane & 3;
+  int tile_no = 0;
   for (int i0 = 0; i0 < M; i0 += 128)
     for (int j0 = 0; j0 < N; j0 += 128) {
+      if ((tile_no++) % nparts != part) continue;
       float acc[2][8][4];
 #pragma unroll
       for (int a = 0; a < 2; ++a)

@@ -56,7 +56,11 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
   const int ntiles = (iend - ibeg + TT8 - 1) / TT8, total = ntiles * nrounds;
   const bool gvec = (ldg & 3) == 0;
 
-  for (int e = tid; e < 2 * S2_RL * S2_TGMAX * S2_DS; e += nthr) Cp[e] = 0.f;     // slots >= TG stay zero
+  // group slots >= TG of the column partials are never written: they are zeroed once, the sum over slots is unrolled
+  for (int e = tid; e < 2 * S2_RL * (S2_TGMAX - TG) * S2_DS; e += nthr) {
+    const int row = e / ((S2_TGMAX - TG) * S2_DS), rest = e % ((S2_TGMAX - TG) * S2_DS);
+    Cp[row * (S2_TGMAX * S2_DS) + TG * S2_DS + rest] = 0.f;
+  }
   for (int e = tid; e < mr; e += nthr) colsum[e] = 0.f;
   if (total == 0) {
     for (int e = tid; e < m * S2_DS; e += nthr) outp[(long long)(e >> 6) * D + (e & 63)] = 0.f;
