@@ -177,6 +177,27 @@ def test_cfg3_full_size_sampled_heads():
     _run_case(cfg, heads=[0, 13, 31])
 
 
+
+# Ragged shapes for the fused sign pass (token tiles of 8 * TG tokens, rounds of 8 landmarks, several token
+# chunks per head, two 64-dim slabs) and for the per-head kernels (m <= 64, 64 < m <= 128, clustered m > 128).
+@pytest.mark.parametrize("gh,gw,mh,mw,prefix,d,dtype", [
+    (5, 7, 3, 3, 2, 64, "bf16"),        # n = 37 (one short tile), m = 9 (second round nearly empty)
+    (23, 31, 5, 10, 1, 128, "bf16"),    # n = 714, m = 50: ragged last tile and last round, two slabs
+    (40, 40, 9, 9, 0, 64, "bf16"),      # n = 1600, m = 81: tensor-core path for 64 < m <= 128, overlapping bins
+    (36, 36, 12, 12, 3, 128, "bf16"),   # n = 1299, m = 144: clustered per-head kernels, m not a multiple of 8 * 128
+    (9, 9, 3, 3, 0, 64, "f32"),         # fp32 storage through the fused pass
+])
+def test_ragged_shapes(gh, gw, mh, mw, prefix, d, dtype):
+    cfg = synth.Config("ragged", B=2, H=2, d=d, m=mh * mw, T=5, gh=gh, gw=gw, mh=mh, mw=mw, prefix=prefix,
+                       dtype=dtype, seed=77)
+    _run_case(cfg)
+
+
+def test_many_heads_several_chunks():
+    """Few heads and many tokens: the landmark gradient is summed over several token chunks per head."""
+    cfg = synth.Config("chunks", B=1, H=1, d=64, m=32, T=4, gh=96, gw=96, mh=4, mw=8, dtype="bf16", seed=5)
+    _run_case(cfg)
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_given_landmarks_and_their_gradient(dtype):
     # lm_mode 0: caller-provided landmarks, dL returned
