@@ -61,11 +61,17 @@ bool make_plan(const ln_problem* p, Plan* pl) {
     int TG = (groups + tiles - 1) / tiles; TG += TG & 1; if (TG > S2_TGMAX) TG = S2_TGMAX; if (TG < 8) TG = 8;
     tiles = (p->n + 8 * TG - 1) / (8 * TG);
     const int slabs = p->d / 64;
-    int wantc = (6 * kSMs + pl->BH * slabs - 1) / (pl->BH * slabs);
-    if (wantc > 16) wantc = 16;
-    if (wantc > tiles) wantc = tiles;
-    if (wantc < 1) wantc = 1;
-    const int tpc = (tiles + wantc - 1) / wantc;
+    // tiles per chunk: the choice that minimises waves x (time of a CTA), with a CTA's time counted in rounds of 8
+    // landmarks plus about three rounds of fixed cost, two CTAs per SM, at most 64 chunks
+    const int nrounds = (p->m + S2_RL - 1) / S2_RL, slots = 2 * kSMs;
+    int tpc = tiles; long long best = -1;
+    for (int t = 1; t <= tiles; ++t) {
+      const int chunks = (tiles + t - 1) / t;
+      if (chunks > 64) continue;
+      const long long ctas = (long long)pl->BH * slabs * chunks;
+      const long long cost = ((ctas + slots - 1) / slots) * ((long long)t * nrounds + 3);
+      if (best < 0 || cost < best) { best = cost; tpc = t; }
+    }
     pl->s2_tg = TG; pl->s2_rpc = tpc * 8 * TG; pl->s2_chunks = (p->n + pl->s2_rpc - 1) / pl->s2_rpc;
     pl->s2_smem = sign2_smem_bytes(p->m);
   }
