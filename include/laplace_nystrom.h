@@ -101,6 +101,22 @@ int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const
                         void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
 
 /*
+ * One training step of the whole path for tensors that live in HOST memory (the paper has no counterpart: a
+ * packaging of laplace_nystrom_fwd + laplace_nystrom_bwd, same arithmetic, same results).  Enqueues on `stream`:
+ * copies of hQ, hK, hV, hdO (host, [B,H,n,d] dtype; pinned memory makes the copies asynchronous) into
+ * `staging`, the forward pass, the copy of O back to hO, the backward pass, the copies of dQ, dK, dV back to
+ * hdQ, hdK, hdV.  Returns once everything is enqueued; the host outputs are valid after the stream has been
+ * synchronised.  lm_mode must be 1 (landmarks pooled from K), else LN_ERR_UNSUPPORTED.
+ *   staging: DEVICE memory, laplace_nystrom_host_staging_bytes(p) bytes, 16-byte aligned, owned by the caller;
+ *   saved, ws, dev_status: as for laplace_nystrom_fwd / _bwd (training sizes).
+ * Two calls on two streams with two sets of device buffers overlap one step's copies with the other's kernels.
+ */
+size_t laplace_nystrom_host_staging_bytes(const ln_problem* p);
+int laplace_nystrom_fwd_bwd_host(const ln_problem* p, const void* hQ, const void* hK, const void* hV, const void* hdO,
+                                 void* hO, void* hdQ, void* hdK, void* hdV, void* staging, size_t staging_bytes,
+                                 void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/*
  * Newton-Schulz iterate of (W + eps I)^-1 (Alg. 2), batched over `batch` independent m x m
  * fp32 matrices.  X [batch,m,m] receives X_T.  X_hist is NULL or [batch,iters+1,m,m] and
  * receives X_0 .. X_T.  resid is NULL or [batch] and receives ||I - (W + eps I) X_T||_F.

@@ -25,6 +25,7 @@ EXPORTS = [
     "laplace_nystrom_fwd", "laplace_nystrom_bwd", "ns_pinv_workspace_bytes", "ns_pinv", "ns_pinv_bwd",
     "l1_kernel", "l1_kernel_bwd_workspace_bytes", "l1_kernel_bwd", "landmarks_pool", "landmarks_pool_bwd",
     "ln_trace_begin", "ln_trace_end", "ns_pinv_static_scratch_bytes", "ns_pinv_static",
+    "laplace_nystrom_host_staging_bytes", "laplace_nystrom_fwd_bwd_host",
 ]
 
 
@@ -107,6 +108,9 @@ def lib():
         L.laplace_nystrom_workspace_bytes.argtypes = [pp, i32]
         L.laplace_nystrom_fwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         L.laplace_nystrom_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.laplace_nystrom_host_staging_bytes.restype = sz
+        L.laplace_nystrom_host_staging_bytes.argtypes = [pp]
+        L.laplace_nystrom_fwd_bwd_host.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp, sz, vp, vp]
         L.ns_pinv_workspace_bytes.restype = sz
         L.ns_pinv_workspace_bytes.argtypes = [i32, i32, i32]
         L.ns_pinv.argtypes = [i32, i32, vp, i32, f32, f32, vp, vp, vp, vp, sz, vp]
@@ -199,6 +203,34 @@ def laplace_nystrom_bwd(p: Problem, Q, K, V, dO, saved, L=None, dQ=None, dK=None
                                    _stream(stream))
     _check(st, "laplace_nystrom_bwd")
     return dQ, dK, dV, dL
+
+
+class HostStep:
+    """Device buffers of laplace_nystrom_fwd_bwd_host for one problem: staging, saved context, workspace."""
+
+    def __init__(self, p: Problem, device):
+        cp = p.c()
+        self.p = p
+        self.staging = _bytes(lib().laplace_nystrom_host_staging_bytes(ctypes.byref(cp)), device)
+        self.saved = _bytes(laplace_nystrom_saved_bytes(p), device)
+        self.ws = _bytes(laplace_nystrom_workspace_bytes(p, True), device)
+
+
+def _host_ptr(t: torch.Tensor):
+    if t.is_cuda or not t.is_contiguous():
+        raise ValueError("laplace_nystrom_fwd_bwd_host takes contiguous host tensors")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def laplace_nystrom_fwd_bwd_host(p: Problem, bufs: HostStep, hQ, hK, hV, hdO, hO, hdQ, hdK, hdV, stream=None):
+    """One training step on host tensors (pinned for asynchronous copies): copies in, forward, backward, copies
+    out, all enqueued on `stream`; the host outputs are valid after the stream has been synchronised."""
+    cp = p.c()
+    st = lib().laplace_nystrom_fwd_bwd_host(ctypes.byref(cp), _host_ptr(hQ), _host_ptr(hK), _host_ptr(hV),
+                                            _host_ptr(hdO), _host_ptr(hO), _host_ptr(hdQ), _host_ptr(hdK),
+                                            _host_ptr(hdV), _ptr(bufs.staging), bufs.staging.numel(),
+                                            _ptr(bufs.saved), _ptr(bufs.ws), bufs.ws.numel(), None, _stream(stream))
+    _check(st, "laplace_nystrom_fwd_bwd_host")
 
 
 # ------------------------------------------------------------------------------------------ Newton-Schulz

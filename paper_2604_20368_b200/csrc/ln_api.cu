@@ -538,6 +538,40 @@ int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const
   return bwd_dispatch_d<bf16>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, dev_status, st);
 }
 
+size_t laplace_nystrom_host_staging_bytes(const ln_problem* p) {
+  if (validate(p) != LN_OK) return 0;
+  const size_t one = ((size_t)p->B * p->H * p->n * p->d * (p->dtype == LN_F32 ? 4 : 2) + 255) / 256 * 256;
+  return 8 * one;                                  // Q, K, V, dO in; O, dQ, dK, dV out
+}
+
+int laplace_nystrom_fwd_bwd_host(const ln_problem* p, const void* hQ, const void* hK, const void* hV, const void* hdO,
+                                 void* hO, void* hdQ, void* hdK, void* hdV, void* staging, size_t staging_bytes,
+                                 void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
+  int s = validate(p);
+  if (s != LN_OK) return s;
+  if (p->lm_mode != 1) return LN_ERR_UNSUPPORTED;
+  if (!hQ || !hK || !hV || !hdO || !hO || !hdQ || !hdK || !hdV || !staging || !saved || !ws) return LN_ERR_ARG;
+  if (!aligned16(staging)) return LN_ERR_ARG;
+  if (staging_bytes < laplace_nystrom_host_staging_bytes(p)) return LN_ERR_WORKSPACE;
+  const size_t bytes = (size_t)p->B * p->H * p->n * p->d * (p->dtype == LN_F32 ? 4 : 2);
+  const size_t one = (bytes + 255) / 256 * 256;
+  char* d = static_cast<char*>(staging);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const void* hin[4] = {hQ, hK, hV, hdO};
+  for (int i = 0; i < 4; ++i)
+    if (cudaMemcpyAsync(d + i * one, hin[i], bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return LN_ERR_CUDA;
+  s = laplace_nystrom_fwd(p, d, d + one, d + 2 * one, nullptr, d + 4 * one, saved, ws, ws_bytes, dev_status, stream);
+  if (s != LN_OK) return s;
+  if (cudaMemcpyAsync(hO, d + 4 * one, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LN_ERR_CUDA;
+  s = laplace_nystrom_bwd(p, d, d + one, d + 2 * one, nullptr, d + 3 * one, saved, d + 5 * one, d + 6 * one, d + 7 * one,
+                          nullptr, ws, ws_bytes, nullptr, stream);
+  if (s != LN_OK) return s;
+  void* hout[3] = {hdQ, hdK, hdV};
+  for (int i = 0; i < 3; ++i)
+    if (cudaMemcpyAsync(hout[i], d + (5 + i) * one, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LN_ERR_CUDA;
+  return LN_OK;
+}
+
 size_t ns_pinv_workspace_bytes(int32_t batch, int32_t m, int32_t iters) {
   if (batch <= 0 || m <= 0 || iters < 0) return 0;
   return carve_ns_ws(batch, m, iters, nullptr).bytes;

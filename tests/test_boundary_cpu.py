@@ -110,3 +110,22 @@ def test_generator_is_seeded_and_duplicates_bins():
     uniq = torch.unique(K, dim=0).shape[0]
     ndup_tokens = K.shape[0] - uniq
     assert ndup_tokens == 7 * 64          # ceil(0.1*64) = 7 bins of 8x8 tokens
+
+
+def test_host_step_argument_errors_without_gpu():
+    """The host-buffer entry point validates before it touches CUDA: sizes, NULL pointers, lm_mode."""
+    lib = binding.lib()
+    p = _problem()
+    cp = p.c()
+    one = 64 * 6 * 197 * 64 * 2
+    need = lib.laplace_nystrom_host_staging_bytes(ctypes.byref(cp))
+    assert need >= 8 * one and need % 256 == 0
+    bad = _problem(lm_mode=0).c()
+    buf = ctypes.create_string_buffer(96)
+    a = ctypes.c_void_p((ctypes.addressof(buf) + 15) // 16 * 16)      # 16-byte aligned, never dereferenced
+    call = lambda prob, staging, nbytes: lib.laplace_nystrom_fwd_bwd_host(
+        ctypes.byref(prob), a, a, a, a, a, a, a, a, staging, nbytes, a, a, 1 << 40, None, None)
+    assert call(bad, a, need) == -2                     # landmarks must come from pooling
+    assert call(cp, None, need) == -1                   # NULL staging
+    assert call(cp, a, need - 1) == -3                  # staging too small
+    assert lib.laplace_nystrom_host_staging_bytes(ctypes.byref(_problem(n=0).c())) == 0

@@ -260,3 +260,22 @@ def test_singular_landmarks_are_flagged_finite():
     assert torch.isfinite(g["O"]).all()
     o = run_oracle_heads(cfg, inp, [0], backward=False)
     assert rel_err(f64(g["O"])[0, 0], o["O"][0]) < 1e-4
+
+
+def test_host_buffer_step_matches_device_path():
+    """laplace_nystrom_fwd_bwd_host (copies + forward + backward on one stream) returns the same bits as the device
+    entry points called on device copies of the same tensors."""
+    cfg = synth.shrink(synth.CONFIGS["cfg2"], B=2)
+    inp = synth.make_inputs(cfg)
+    g = run_gpu(cfg, inp)
+    wh = inp["whiten"].to(DEV)
+    p = ln.problem_from_config(cfg, whiten=wh)
+    bufs = ln.HostStep(p, DEV)
+    hin = {k: inp[k].pin_memory() for k in ("Q", "K", "V", "dO")}
+    hout = {k: torch.empty_like(inp["Q"]).pin_memory() for k in ("O", "dQ", "dK", "dV")}
+    for _ in range(2):
+        ln.laplace_nystrom_fwd_bwd_host(p, bufs, hin["Q"], hin["K"], hin["V"], hin["dO"], hout["O"], hout["dQ"],
+                                        hout["dK"], hout["dV"])
+        torch.cuda.synchronize()
+        for k in ("O", "dQ", "dK", "dV"):
+            assert torch.equal(hout[k], g[k].cpu()), k
