@@ -98,7 +98,9 @@ Ctx carve_ctx(const Plan& pl, void* base) {
   return x;
 }
 
-struct FwdWs { float *Mpart, *Wr, *P, *Y; size_t bytes; };
+struct FwdWs { float *Mpart, *Wr, *P, *Y, *Yimg; size_t bytes; };
+// floats of the split operand images of one [m][d] matrix per head (the tcgen05 product kernels read them)
+size_t image_floats(const Plan& pl) { return (size_t)((pl.m + GU_KB - 1) / GU_KB) * gu_block_floats(pl.d); }
 FwdWs carve_fwd_ws(const Plan& pl, void* base) {
   Carver c(base); FwdWs w;
   const size_t BH = pl.BH, d = pl.d, m = pl.m;
@@ -106,12 +108,13 @@ FwdWs carve_fwd_ws(const Plan& pl, void* base) {
   w.Wr = c.take(BH * m * pl.ldm);
   w.P = c.take(BH * m * pl.ldm);
   w.Y = c.take(BH * m * d);
+  w.Yimg = c.take(BH * image_floats(pl));
   w.bytes = c.off;
   return w;
 }
 
 struct BwdWs {
-  float *G, *dYtpart, *dybpart, *dLCpart, *dLRpart, *dY, *dM, *Wr, *P, *Hm, *Ga, *Gb, *dW, *dX, *GW, *dLW, *dLtot, *dKpart;
+  float *G, *dYtpart, *dybpart, *dLCpart, *dLRpart, *dY, *dM, *Wr, *P, *Hm, *Ga, *Gb, *dW, *dX, *GW, *dLW, *dLtot, *dKpart, *dMimg;
   size_t bytes;
 };
 BwdWs carve_bwd_ws(const Plan& pl, void* base) {
@@ -136,6 +139,7 @@ BwdWs carve_bwd_ws(const Plan& pl, void* base) {
   w.dLW = c.take(BH * m * d);
   w.dLtot = c.take(BH * m * d);
   w.dKpart = c.take(BH * n * d);
+  w.dMimg = c.take(BH * image_floats(pl));
   w.bytes = c.off;
   return w;
 }
@@ -290,13 +294,14 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   else
     LN_LAUNCH("tn_M", st, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, w.Mpart, nullptr, n, m, pl.rpc));
   // Newton-Schulz, Y = X M, folded map
+  const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);   // tcgen05 products over the landmarks
   {
     constexpr bool TC = std::is_same<T, bf16>::value;
     auto launch = [&](auto kern, size_t smem, int cl = 1) {
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       LN_LAUNCH("k_mid_fwd", st, launch_clustered(kern, BH * cl, cl, smem, st, m, pl.ldm, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode,
                                                   p->whiten, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt,
-                                                  x.ybar, dev_status, pl.hslot));
+                                                  x.ybar, dev_status, pl.hslot, umma_prod ? reinterpret_cast<bf16*>(w.Yimg) : nullptr));
     };
     if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * NsTile<64>::mat_bytes);
     else if (TC && m <= 128) launch(k_mid_fwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
@@ -304,7 +309,12 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     else launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));
   }
   // O = (C - mu) Ytilde + ybar
-  if constexpr (std::is_same<T, bf16>::value)
+  if constexpr (std::is_same<T, bf16>::value && (D == 64 || D == 128)) {
+    const size_t smem = nn_umma_smem<D>();
+    cudaFuncSetAttribute(k_nn_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    LN_LAUNCH("nn_O", st, k_nn_umma<D><<<dim3(cdiv(n, 128), BH), 256, smem, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr,
+                                                                              reinterpret_cast<const bf16*>(w.Yimg), x.ybar, O, n, m, dev_status));
+  } else if constexpr (std::is_same<T, bf16>::value)
     LN_LAUNCH("nn_O", st, k_nn_mma<D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr, x.Yt, x.ybar, O, n, m));
   else
     LN_LAUNCH("nn_O", st, k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr, x.Yt, x.ybar, O, n, m));
@@ -340,13 +350,15 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
   }
   // per head: dY, dX, dM, Newton-Schulz adjoint, symmetrised landmark-block upstream
+  const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);
   {
     constexpr bool TC = std::is_same<T, bf16>::value;
     auto launch = [&](auto kern, size_t smem, int cl = 1) {
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       LN_LAUNCH("k_mid_bwd", st, launch_clustered(kern, BH * cl, cl, smem, st, m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten,
                                                   x.W, x.Xh, x.Ph, x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P,
-                                                  w.Hm, w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot));
+                                                  w.Hm, w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot,
+                                                  umma_prod ? reinterpret_cast<bf16*>(w.dMimg) : nullptr));
     };
     if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 4 * NsTile<64>::mat_bytes);
     else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
@@ -357,6 +369,12 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // key side: g^R = (V dM^T) o R^T / lambda; dV = R^T dM; dK (kernel part); landmark part
   if constexpr (std::is_same<T, bf16>::value) {
     LN_LAUNCH("ntg_R", st, k_nt_g_mma<D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(V, w.dM, x.Rt, pl.ldm, w.G, n, m, inv_lambda));
+    if constexpr (D == 64 || D == 128) {
+      const size_t smem = nn_umma_smem<D>();
+      cudaFuncSetAttribute(k_nn_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      LN_LAUNCH("nn_dV", st, k_nn_umma<D><<<dim3(cdiv(n, 128), BH), 256, smem, st>>>(x.Rt, pl.ldm, nullptr, reinterpret_cast<const bf16*>(w.dMimg),
+                                                                                 nullptr, dV, n, m, dev_status));
+    } else
     LN_LAUNCH("nn_dV", st, k_nn_mma<D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
   } else {
     LN_LAUNCH("ntg_R", st, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(V, w.dM, x.Rt, pl.ldm, w.G, n, m, inv_lambda));

@@ -1,0 +1,156 @@
+// O[i][c] = sum_l (E[i][l] - mu[i]) Y[l][c] + ybar[c]  on the 5th-generation tensor cores (tcgen05 + TMEM),
+// for the two products of the path that reduce over the landmarks: O = (C - mu) Ytilde + ybar (Alg. 1, Prop. 3)
+// and dV = R^T dM.
+//
+// M = 128 tokens per CTA, N = D dims, K = landmarks in blocks of 64.  A = the E tile, converted in the kernel from
+// fp32 to a bf16 hi + lo image (K-major); B = Y, which its producer leaves in global memory already split and
+// laid out as operand images per 64-landmark block, so that a block arrives with one bulk copy while the E
+// block is being converted.  Three MMAs per product (lo*hi, hi*lo, hi*hi), fp32 accumulation in D columns of
+// TMEM, issued by one thread; the epilogue goes TMEM -> registers -> bf16 rows in shared memory -> 16-byte
+// coalesced stores.  Two CTAs per SM overlap one tile's conversion and epilogue with the other's MMAs.
+#pragma once
+#include "ln_mma.cuh"
+#include "ln_umma.cuh"
+
+namespace ln {
+
+constexpr int GU_KB = 64;                       // landmarks per block
+// floats per 64-landmark block of a split operand image of a [m][D] matrix (hi part, lo part)
+__host__ __device__ constexpr int gu_block_floats(int D) { return GU_KB * D; }
+
+// [m][D] fp32 (row-major) -> split images per 64-row block: block kb holds rows 64 kb .. 64 kb + 63 as a
+// [64][D] image (hi) followed by the same for lo; rows >= m are zero.  Strided over `nthr` threads.
+__device__ __forceinline__ void gu_write_images(const float* __restrict__ src, bf16* __restrict__ img, int m, int D,
+                                                int t0, int nthr) {
+  const int nkb = (m + GU_KB - 1) / GU_KB, per_row = D / 8;
+  for (int p = t0; p < nkb * GU_KB * per_row; p += nthr) {
+    const int l = p / per_row, c8 = (p % per_row) * 8;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+    if (l < m) { a = *reinterpret_cast<const float4*>(src + (long long)l * D + c8); b = *reinterpret_cast<const float4*>(src + (long long)l * D + c8 + 4); }
+    uint2 h0, l0, h1, l1;
+    split4(a, h0, l0); split4(b, h1, l1);
+    bf16* blk = img + (long long)(l / GU_KB) * (2 * GU_KB * D);
+    const int off = umma::img(l % GU_KB, c8, D);
+    *reinterpret_cast<uint4*>(blk + off) = make_uint4(h0.x, h0.y, h1.x, h1.y);
+    *reinterpret_cast<uint4*>(blk + GU_KB * D + off) = make_uint4(l0.x, l0.y, l1.x, l1.y);
+  }
+}
+
+// shared memory of k_nn_umma: E block images and Y block images; the bf16 staging of the output tile reuses them
+template <int D> constexpr size_t nn_umma_smem() { return (size_t)(2 * 128 * GU_KB + 2 * GU_KB * D) * sizeof(bf16); }
+
+// One 128-token tile per CTA; three CTAs per SM hide each other's load latencies.
+template <int D>
+__global__ void __launch_bounds__(256, 3) k_nn_umma(const float* __restrict__ E, int lde, const float* __restrict__ mu,
+                                                    const bf16* __restrict__ Yimg, const float* __restrict__ ybar,
+                                                    bf16* __restrict__ O, int n, int m, int* dev_status) {
+  extern __shared__ __align__(128) unsigned char gu_smem[];
+  bf16* sZ = reinterpret_cast<bf16*>(gu_smem);                 // [2][128 * 64]: hi, lo of the E block (K-major image)
+  bf16* sY = sZ + 2 * 128 * GU_KB;                             // [2][64 * D]: hi, lo of the Y block (image, rows = K)
+  __shared__ unsigned long long mbar_mma, mbar_y;
+  __shared__ uint32_t tmem_base;
+  const int i0 = blockIdx.x * 128, bh = blockIdx.y;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int nkb = (m + GU_KB - 1) / GU_KB;
+  E += (long long)bh * n * lde;
+  O += (long long)bh * n * D;
+  if (ybar) ybar += (long long)bh * D;
+  Yimg += (long long)bh * nkb * (2 * GU_KB * D);
+  if (tid == 0) { umma::mbar_init(&mbar_mma, 1); umma::mbar_init(&mbar_y, 1); }
+  if (warp == 0) umma::tmem_alloc(&tmem_base, D);
+  umma::fence_before_sync();
+  __syncthreads();
+  umma::fence_after_sync();
+  const uint32_t tacc = tmem_base;
+  // E block: thread = (token r of the tile, 32 landmarks of the block)
+  const int zr = tid >> 1, zc = (tid & 1) * 32, zi = i0 + zr;
+  const bool in = zi < n;
+  const float mi = (mu && in) ? mu[(long long)bh * n + zi] : 0.f;
+  const uint32_t idesc = umma::instr_desc(D, false, true);
+  uint32_t ph_mma = 0, ph_y = 0;
+  bool ok = true;
+  float4 v[8];                                   // this thread's piece of an E block, fetched one block ahead
+  auto fetch = [&](int kb) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int l = kb * GU_KB + zc + 4 * q;
+      v[q] = (in && l < m) ? *reinterpret_cast<const float4*>(E + (long long)zi * lde + l) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  fetch(0);
+  for (int kb = 0; kb < nkb; ++kb) {
+    if (tid == 0) {                              // the Y block arrives while the E block is converted
+      umma::mbar_expect_tx(&mbar_y, 2 * GU_KB * D * 2);
+      umma::bulk_load(sY, Yimg + (long long)kb * (2 * GU_KB * D), 2 * GU_KB * D * 2, &mbar_y);
+    }
+#pragma unroll
+    for (int q = 0; q < 8; q += 2) {
+      float4 a = v[q], b = v[q + 1];
+      const int l = kb * GU_KB + zc + 4 * q;
+      a.x = (in && l < m) ? a.x - mi : 0.f;     a.y = (in && l + 1 < m) ? a.y - mi : 0.f;
+      a.z = (in && l + 2 < m) ? a.z - mi : 0.f; a.w = (in && l + 3 < m) ? a.w - mi : 0.f;
+      b.x = (in && l + 4 < m) ? b.x - mi : 0.f; b.y = (in && l + 5 < m) ? b.y - mi : 0.f;
+      b.z = (in && l + 6 < m) ? b.z - mi : 0.f; b.w = (in && l + 7 < m) ? b.w - mi : 0.f;
+      uint2 h0, l0, h1, l1;
+      split4(a, h0, l0); split4(b, h1, l1);
+      const int off = umma::img(zr, zc + 4 * q, GU_KB);
+      *reinterpret_cast<uint4*>(sZ + off) = make_uint4(h0.x, h0.y, h1.x, h1.y);
+      *reinterpret_cast<uint4*>(sZ + 128 * GU_KB + off) = make_uint4(l0.x, l0.y, l1.x, l1.y);
+    }
+    umma::fence_smem_to_mma();
+    __syncthreads();
+    if (kb + 1 < nkb) fetch(kb + 1);             // in flight while the MMAs of this block run
+    if (tid == 0) {
+      ok &= umma::mbar_wait(&mbar_y, ph_y & 1);
+      umma::fence_after_sync();
+#pragma unroll 1
+      for (int part = 0; part < 3; ++part) {     // lo*hi, hi*lo, hi*hi
+        const bf16* a = sZ + (part == 0 ? 128 * GU_KB : 0);
+        const bf16* b = sY + (part == 1 ? GU_KB * D : 0);
+#pragma unroll
+        for (int ks = 0; ks < GU_KB / 16; ++ks)
+          umma::mma(tacc, umma::operand_desc(a, GU_KB, true, ks), umma::operand_desc(b, D, false, ks), idesc,
+                    !(kb == 0 && part == 0 && ks == 0));
+      }
+      umma::commit(&mbar_mma);
+    }
+    ph_y ^= 1u;
+    ok &= umma::mbar_wait(&mbar_mma, ph_mma & 1);   // the MMAs have read both blocks: the buffers are free again
+    ph_mma ^= 1u;
+    umma::fence_after_sync();
+  }
+  // epilogue: thread = (row 32 (warp % 4) + lane, D / 2 columns); rows as bf16 through shared memory (the operand
+  // buffers, which no MMA reads any more)
+  constexpr int HC = D / 2, LDS_ = D + 8;
+  bf16* stage = reinterpret_cast<bf16*>(gu_smem);              // [128][D + 8]
+  {
+    const int row = (warp & 3) * 32 + (tid & 31), c0 = (warp >> 2) * HC;
+#pragma unroll
+    for (int cb = 0; cb < HC; cb += 32) {
+      float a[32];
+      umma::tmem_ld32(umma::tmem_addr(tacc, c0 + cb), a);
+#pragma unroll
+      for (int q = 0; q < 32; q += 8) {
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int c = c0 + cb + q + 2 * e;
+          const float y0 = ybar ? ybar[c] : 0.f, y1 = ybar ? ybar[c + 1] : 0.f;
+          const __nv_bfloat162 pr = __floats2bfloat162_rn(a[q + 2 * e] + y0, a[q + 2 * e + 1] + y1);
+          w[e] = *reinterpret_cast<const uint32_t*>(&pr);
+        }
+        *reinterpret_cast<uint4*>(stage + row * LDS_ + c0 + cb + q) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+  }
+  umma::fence_before_sync();
+  __syncthreads();
+  for (int p = tid; p < 128 * (D / 8); p += 256) {
+    const int r = p / (D / 8), c8 = (p % (D / 8)) * 8;
+    if (i0 + r < n) *reinterpret_cast<uint4*>(O + (long long)(i0 + r) * D + c8) = *reinterpret_cast<const uint4*>(stage + r * LDS_ + c8);
+  }
+  if (warp == 0) umma::tmem_dealloc(tmem_base, D);
+  if (!ok && dev_status && tid == 0) atomicOr(dev_status + bh, 2);
+}
+
+}  // namespace ln

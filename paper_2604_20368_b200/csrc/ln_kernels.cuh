@@ -6,6 +6,7 @@
 #include "ln_mma.cuh"
 #include "ln_ns_smem.cuh"
 #include "ln_ns_umma.cuh"
+#include "ln_gemm_umma.cuh"
 
 namespace ln {
 
@@ -912,11 +913,12 @@ __global__ void __launch_bounds__(256) k_ns_pinv_bwd(int m, int T, float eps, fl
 // =====================================================================================
 // CL > 1 (generic path only): CL CTAs of a thread-block cluster share one head; grid = heads * CL.
 template <int D, bool TC, int MP, int CL = 1>
-__global__ void __launch_bounds__(256, CL > 1 ? 2 : 1) k_mid_fwd(int m, int ldm, int T, float eps, float alpha_in, int H, int map_mode,
+__global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_fwd(int m, int ldm, int T, float eps, float alpha_in, int H, int map_mode,
                                                  const float* __restrict__ whiten, const float* W, float* Wr,
                                                  float* P, float* Xh, float* Ph, NsHdr* hdr, const float* Mpart, int nchunks,
                                                  float* Mout, float* Y, float* Yt, float* ybar, int* dev_status,
-                                                 long long hslot) {
+                                                 long long hslot, bf16* Yimg) {
+  // Yimg: NULL, or where Ytilde is also left as split operand images per 64-landmark block (for the tcgen05 product)
   // hslot: floats per slot of the iterate histories (used by the MP = 64 path, whose slots hold operand images)
   // dynamic shared memory: the Newton-Schulz matrices (MP > 0), reused afterwards by the GEMM engine
   extern __shared__ __align__(16) unsigned char dyn_smem[];
@@ -986,6 +988,11 @@ __global__ void __launch_bounds__(256, CL > 1 ? 2 : 1) k_mid_fwd(int m, int ldm,
     }
     *reinterpret_cast<float4*>(Yt + e) = y;
   }
+  if (Yimg != nullptr) {
+    phase_sync<CL>();                             // Ytilde of this head is complete
+    const int nkb = (m + GU_KB - 1) / GU_KB;
+    gu_write_images(Yt, Yimg + (long long)bh * nkb * (2 * GU_KB * D), m, D, gt, gn);
+  }
 }
 template <int D, bool TC, int MP, int CL = 1>
 __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_bwd(int m, int T, int H, int map_mode, float inv_lambda, int ldm,
@@ -994,7 +1001,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_bw
                                                  const float* dYtpart, const float* dybpart, int nchunks,
                                                  float eps, float* Wr, float* P, float* Hm, float* Ga, float* Gb,
                                                  float* dWm, float* dXm, float* dY, float* dM, float* GW, int* dev_status,
-                                                 long long hslot) {
+                                                 long long hslot, bf16* dMimg) {
   extern __shared__ __align__(16) unsigned char dyn_smem[];
   NsSmem& sm = *reinterpret_cast<NsSmem*>(dyn_smem);
   __shared__ float red[2 * 256 + 8];
@@ -1039,6 +1046,10 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_bw
   ns_gemm<TC, false, true>(m, m, D, dY, D, Msaved, D, dXm, ldx, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // dX = dY M^T
   ns_gemm<TC, true, false>(m, D, m, XT, ldx, dY, D, dM, D, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);        // dM = X^T dY
   if (CL > 1) phase_sync<CL>();
+  if (dMimg != nullptr) {                         // dM also as split operand images (for the tcgen05 product dV = R^T dM)
+    const int nkb = (m + GU_KB - 1) / GU_KB;
+    gu_write_images(dM, dMimg + (long long)bh * nkb * (2 * GU_KB * D), m, D, gt, gn);
+  }
   if constexpr (MP == 128) {
     __shared__ UmmaCtl ctl;
     const bool tc_ok = ns_backward_umma(m, T, eps, W, Xh, Ph, ldx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red, ctl);

@@ -71,6 +71,16 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* mbar, uint32_t par
   return done != 0;
 }
 
+// Bulk copy global -> shared of `bytes` (a multiple of 16, both addresses 16-byte aligned) by ONE thread; the
+// bytes are counted on `mbar`, which must have been told to expect them (expect_tx) beforehand.
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* mbar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(mbar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes, unsigned long long* mbar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(s32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(s32(mbar)) : "memory");
+}
+
 // TMEM allocation (whole warp; ncols a power of two in [32, 512]); the base address lands in *slot.
 __device__ __forceinline__ void tmem_alloc(uint32_t* slot, int ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(slot)), "r"(ncols));
