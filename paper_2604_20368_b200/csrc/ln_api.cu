@@ -78,8 +78,11 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   return true;
 }
 
+// floats of the split operand images of one [m][d] matrix per head (the tcgen05 product kernels read them)
+size_t image_floats(const Plan& pl) { return (size_t)((pl.m + GU_KB - 1) / GU_KB) * gu_block_floats(pl.d); }
+
 // Forward context (saved for the backward pass, or carved from ws for inference)
-struct Ctx { float *Lf, *C, *Rt, *mu, *W, *Xh, *Ph, *M, *Yt, *ybar; NsHdr* hdr; size_t bytes; };
+struct Ctx { float *Lf, *C, *Rt, *mu, *W, *Xh, *Ph, *M, *Yt, *ybar, *Yimg; NsHdr* hdr; size_t bytes; };
 Ctx carve_ctx(const Plan& pl, void* base) {
   Carver c(base); Ctx x;
   const size_t BH = pl.BH, n = pl.n, d = pl.d, m = pl.m;
@@ -93,14 +96,13 @@ Ctx carve_ctx(const Plan& pl, void* base) {
   x.M = c.take(BH * m * d);
   x.Yt = c.take(BH * m * d);
   x.ybar = c.take(BH * d);
+  x.Yimg = c.take(BH * image_floats(pl));        // Ytilde once more, as split operand images
   x.hdr = reinterpret_cast<NsHdr*>(c.take(BH * (sizeof(NsHdr) / sizeof(float))));
   x.bytes = c.off;
   return x;
 }
 
-struct FwdWs { float *Mpart, *Wr, *P, *Y, *Yimg; size_t bytes; };
-// floats of the split operand images of one [m][d] matrix per head (the tcgen05 product kernels read them)
-size_t image_floats(const Plan& pl) { return (size_t)((pl.m + GU_KB - 1) / GU_KB) * gu_block_floats(pl.d); }
+struct FwdWs { float *Mpart, *Wr, *P, *Y; size_t bytes; };
 FwdWs carve_fwd_ws(const Plan& pl, void* base) {
   Carver c(base); FwdWs w;
   const size_t BH = pl.BH, d = pl.d, m = pl.m;
@@ -108,7 +110,6 @@ FwdWs carve_fwd_ws(const Plan& pl, void* base) {
   w.Wr = c.take(BH * m * pl.ldm);
   w.P = c.take(BH * m * pl.ldm);
   w.Y = c.take(BH * m * d);
-  w.Yimg = c.take(BH * image_floats(pl));
   w.bytes = c.off;
   return w;
 }
@@ -301,7 +302,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       LN_LAUNCH("k_mid_fwd", st, launch_clustered(kern, BH * cl, cl, smem, st, m, pl.ldm, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode,
                                                   p->whiten, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt,
-                                                  x.ybar, dev_status, pl.hslot, umma_prod ? reinterpret_cast<bf16*>(w.Yimg) : nullptr));
+                                                  x.ybar, dev_status, pl.hslot, umma_prod ? reinterpret_cast<bf16*>(x.Yimg) : nullptr));
     };
     if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * NsTile<64>::mat_bytes);
     else if (TC && m <= 128) launch(k_mid_fwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
@@ -313,7 +314,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     const size_t smem = nn_umma_smem<D>();
     cudaFuncSetAttribute(k_nn_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     LN_LAUNCH("nn_O", st, k_nn_umma<D><<<dim3(cdiv(n, 128), BH), 256, smem, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr,
-                                                                              reinterpret_cast<const bf16*>(w.Yimg), x.ybar, O, n, m, dev_status));
+                                                                              reinterpret_cast<const bf16*>(x.Yimg), x.ybar, O, n, m, dev_status));
   } else if constexpr (std::is_same<T, bf16>::value)
     LN_LAUNCH("nn_O", st, k_nn_mma<D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr, x.Yt, x.ybar, O, n, m));
   else
@@ -331,6 +332,11 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // query side: Z'^T dO and column sums of dO; g^C = (dO Ytilde^T) o C / lambda; dQ; landmark part
   if constexpr (std::is_same<T, bf16>::value) {
     LN_LAUNCH("tn_dY", st, k_tn_mma<D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
+    if constexpr (D == 64 || D == 128) {
+      cudaFuncSetAttribute(k_ntg_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ntg_umma_smem<D>());
+      LN_LAUNCH("ntg_C", st, k_ntg_umma<D><<<dim3(cdiv(n, 128), BH), 256, ntg_umma_smem<D>(), st>>>(dO, reinterpret_cast<const bf16*>(x.Yimg), x.C, pl.ldm,
+                                                                                                w.G, n, m, inv_lambda, dev_status));
+    } else
     LN_LAUNCH("ntg_C", st, k_nt_g_mma<D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(dO, x.Yt, x.C, pl.ldm, w.G, n, m, inv_lambda));
   } else {
     LN_LAUNCH("tn_dY", st, k_tn<T, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
@@ -368,6 +374,10 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   LN_LAUNCH("sign_rows_dLW", st, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, st>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));
   // key side: g^R = (V dM^T) o R^T / lambda; dV = R^T dM; dK (kernel part); landmark part
   if constexpr (std::is_same<T, bf16>::value) {
+    if constexpr (D == 64 || D == 128)
+      LN_LAUNCH("ntg_R", st, k_ntg_umma<D><<<dim3(cdiv(n, 128), BH), 256, ntg_umma_smem<D>(), st>>>(V, reinterpret_cast<const bf16*>(w.dMimg), x.Rt, pl.ldm,
+                                                                                                w.G, n, m, inv_lambda, dev_status));
+    else
     LN_LAUNCH("ntg_R", st, k_nt_g_mma<D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(V, w.dM, x.Rt, pl.ldm, w.G, n, m, inv_lambda));
     if constexpr (D == 64 || D == 128) {
       const size_t smem = nn_umma_smem<D>();

@@ -37,7 +37,7 @@ __device__ __forceinline__ void gu_write_images(const float* __restrict__ src, b
 }
 
 // shared memory of k_nn_umma: E block images and Y block images; the bf16 staging of the output tile reuses them
-template <int D> constexpr size_t nn_umma_smem() { return (size_t)(2 * 128 * GU_KB + 2 * GU_KB * D) * sizeof(bf16); }
+template <int D> __host__ __device__ constexpr size_t nn_umma_smem() { return (size_t)(2 * 128 * GU_KB + 2 * GU_KB * D) * sizeof(bf16); }
 
 // One 128-token tile per CTA; three CTAs per SM hide each other's load latencies.
 template <int D>
@@ -150,6 +150,126 @@ __global__ void __launch_bounds__(256, 3) k_nn_umma(const float* __restrict__ E,
     if (i0 + r < n) *reinterpret_cast<uint4*>(O + (long long)(i0 + r) * D + c8) = *reinterpret_cast<const uint4*>(stage + r * LDS_ + c8);
   }
   if (warp == 0) umma::tmem_dealloc(tmem_base, D);
+  if (!ok && dev_status && tid == 0) atomicOr(dev_status + bh, 2);
+}
+
+// =====================================================================================
+// G[i][l] = (sum_c U[i][c] Y[l][c]) * E[i][l] / lambda   (the upstream g = dA o A / lambda of a kernel block, App. A)
+// M = 128 tokens per CTA, N = 64 landmarks per MMA (one accumulator range of 64 TMEM columns per landmark block),
+// K = D.  A = the U tile, bf16 in HBM and therefore exact: copied as it is into a K-major image.  B = Y from the
+// same pre-split block images the landmark-reducing product reads (rows = landmarks, so K-major here); two MMAs
+// per product (U * Y_hi, U * Y_lo).  Two block buffers: the bulk copy of a block overlaps the MMAs of the other.
+// Epilogue per block: TMEM -> registers, times the kernel values (read by row), fp32 rows staged in shared memory,
+// coalesced 16-byte stores.
+// =====================================================================================
+template <int D> __host__ __device__ constexpr size_t ntg_umma_smem() { return (size_t)(128 * D + 2 * 2 * GU_KB * D) * sizeof(bf16); }
+
+template <int D>
+__global__ void __launch_bounds__(256, 2) k_ntg_umma(const bf16* __restrict__ U, const bf16* __restrict__ Yimg,
+                                                     const float* __restrict__ E, int lde, float* __restrict__ G,
+                                                     int n, int m, float inv_lambda, int* dev_status) {
+  extern __shared__ __align__(128) unsigned char gu_smem[];
+  bf16* sU = reinterpret_cast<bf16*>(gu_smem);                 // [128 x D] K-major image of the U tile
+  bf16* sY = sU + 128 * D;                                     // [2 buffers][2 parts][64 * D]
+  __shared__ unsigned long long mbar_y[2], mbar_free[2], mbar_done;
+  __shared__ uint32_t tmem_base;
+  const int i0 = blockIdx.x * 128, bh = blockIdx.y;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int nkb = (m + GU_KB - 1) / GU_KB;
+  const int ncols = nkb <= 1 ? 64 : (nkb == 2 ? 128 : 256);
+  U += (long long)bh * n * D;
+  E += (long long)bh * n * lde;
+  G += (long long)bh * n * lde;
+  Yimg += (long long)bh * nkb * (2 * GU_KB * D);
+  if (tid == 0) {
+    umma::mbar_init(&mbar_y[0], 1); umma::mbar_init(&mbar_y[1], 1);
+    umma::mbar_init(&mbar_free[0], 1); umma::mbar_init(&mbar_free[1], 1);
+    umma::mbar_init(&mbar_done, 1);
+  }
+  if (warp == 0) umma::tmem_alloc(&tmem_base, ncols);
+  umma::fence_before_sync();
+  __syncthreads();
+  umma::fence_after_sync();
+  const uint32_t tacc = tmem_base;
+  constexpr uint32_t YB = 2 * GU_KB * D * 2;     // bytes of one block (hi + lo)
+  if (tid == 0)                                  // the first two blocks are on their way while the U tile is copied
+    for (int nb = 0; nb < 2 && nb < nkb; ++nb) {
+      umma::mbar_expect_tx(&mbar_y[nb], YB);
+      umma::bulk_load(sY + nb * (2 * GU_KB * D), Yimg + (long long)nb * (2 * GU_KB * D), YB, &mbar_y[nb]);
+    }
+  for (int p = tid; p < 128 * (D / 8); p += 256) {
+    const int r = p / (D / 8), c8 = (p % (D / 8)) * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (i0 + r < n) v = *reinterpret_cast<const uint4*>(U + (long long)(i0 + r) * D + c8);
+    *reinterpret_cast<uint4*>(sU + umma::img(r, c8, D)) = v;
+  }
+  umma::fence_smem_to_mma();
+  __syncthreads();
+  // kernel values of the first block for this thread's row, fetched before the products are awaited
+  const int row = (warp & 3) * 32 + (tid & 31), ch = (warp >> 2) * 32, gi = i0 + row;
+  float4 ev[8];
+  auto fetch_e = [&](int nb) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int l = nb * GU_KB + ch + 4 * q;
+      ev[q] = (gi < n && l < lde) ? *reinterpret_cast<const float4*>(E + (long long)gi * lde + l) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  fetch_e(0);
+  bool ok = true;
+  if (tid == 0) {
+    const uint32_t idesc = umma::instr_desc(GU_KB, false, false);
+    uint32_t ph_y[2] = {0, 0}, ph_f[2] = {0, 0};
+    for (int nb = 0; nb < nkb; ++nb) {
+      const int b = nb & 1;
+      ok &= umma::mbar_wait(&mbar_y[b], ph_y[b] & 1); ph_y[b] ^= 1u;
+      umma::fence_after_sync();
+      const bf16* yb = sY + b * (2 * GU_KB * D);
+#pragma unroll 1
+      for (int part = 0; part < 2; ++part)       // U * Y_hi, U * Y_lo
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks)
+          umma::mma(tacc + nb * GU_KB, umma::operand_desc(sU, D, true, ks), umma::operand_desc(yb + part * (GU_KB * D), D, true, ks),
+                    idesc, !(part == 0 && ks == 0));
+      if (nb + 2 < nkb) {                        // refill this buffer once its MMAs have read it
+        umma::commit(&mbar_free[b]);
+        ok &= umma::mbar_wait(&mbar_free[b], ph_f[b] & 1); ph_f[b] ^= 1u;
+        umma::mbar_expect_tx(&mbar_y[b], YB);
+        umma::bulk_load(sY + b * (2 * GU_KB * D), Yimg + (long long)(nb + 2) * (2 * GU_KB * D), YB, &mbar_y[b]);
+      }
+    }
+    umma::commit(&mbar_done);
+  }
+  ok &= umma::mbar_wait(&mbar_done, 0);
+  umma::fence_after_sync();
+  // epilogue, one landmark block at a time; the fp32 rows are staged in the (now idle) operand buffers
+  constexpr int LDG_ = GU_KB + 4;
+  static_assert((size_t)128 * LDG_ * sizeof(float) <= ntg_umma_smem<D>(), "staging fits in the operand buffers");
+  float* stage = reinterpret_cast<float*>(gu_smem);             // [128][64 + 4] floats = 34 KB
+  for (int nb = 0; nb < nkb; ++nb) {
+    float a[32];
+    umma::tmem_ld32(umma::tmem_addr(tacc, nb * GU_KB + ch), a);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int l = nb * GU_KB + ch + 4 * q;
+      float4 o;
+      o.x = (l < m) ? a[4 * q] * ev[q].x * inv_lambda : 0.f;
+      o.y = (l + 1 < m) ? a[4 * q + 1] * ev[q].y * inv_lambda : 0.f;
+      o.z = (l + 2 < m) ? a[4 * q + 2] * ev[q].z * inv_lambda : 0.f;
+      o.w = (l + 3 < m) ? a[4 * q + 3] * ev[q].w * inv_lambda : 0.f;
+      *reinterpret_cast<float4*>(stage + row * LDG_ + ch + 4 * q) = o;
+    }
+    if (nb + 1 < nkb) fetch_e(nb + 1);
+    __syncthreads();
+    for (int p = tid; p < 128 * (GU_KB / 4); p += 256) {
+      const int r = p / (GU_KB / 4), c4 = (p % (GU_KB / 4)) * 4, l = nb * GU_KB + c4;
+      if (i0 + r < n && l < lde) *reinterpret_cast<float4*>(G + (long long)(i0 + r) * lde + l) = *reinterpret_cast<const float4*>(stage + r * LDG_ + c4);
+    }
+    __syncthreads();
+  }
+  umma::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) umma::tmem_dealloc(tmem_base, ncols);
   if (!ok && dev_status && tid == 0) atomicOr(dev_status + bh, 2);
 }
 
