@@ -405,10 +405,10 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const int md = m * D;
   if (p->lm_mode == 1) {
     LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chs, w.dLRpart, chs, w.dLW, 1, w.dLtot, md));
-    LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256), BH), 256, 0, st>>>(w.dKpart, w.dLtot, dK, geom_of(p), 1));
+    LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, w.dLtot, dK, geom_of(p), 1));
   } else {
     LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chs, w.dLRpart, chs, w.dLW, 1, dL, md));
-    LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256), BH), 256, 0, st>>>(w.dKpart, nullptr, dK, geom_of(p), 0));
+    LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, nullptr, dK, geom_of(p), 0));
   }
   return launch_ok();
 }
@@ -741,7 +741,7 @@ int landmarks_pool_bwd(const ln_problem* p, const float* dL, void* dK, void* str
   if (s != LN_OK) return s;
   if (p->lm_mode != 1 || !dL || !dK || !aligned16(dL) || !aligned16(dK)) return LN_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  dim3 grid(cdiv((long long)p->n * (p->d / 4), 256), p->B * p->H);
+  dim3 grid(cdiv((long long)p->n * (p->d / 4), 256 * POOL_EPT), p->B * p->H);
   if (p->dtype == LN_F32) LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<float><<<grid, 256, 0, st>>>(nullptr, dL, (float*)dK, geom_of(p), 1));
   else LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<bf16><<<grid, 256, 0, st>>>(nullptr, dL, (bf16*)dK, geom_of(p), 1));
   return launch_ok();

@@ -207,6 +207,7 @@ __global__ void __launch_bounds__(256) k_pool(const T* __restrict__ K, float* __
 
 // dK[j] = dKpart[j] (may be NULL) + sum over the bins containing token j of dL[bin] / |bin|
 // (pooling adjoint); with pool == 0 it only converts dKpart to the storage type.
+constexpr int POOL_EPT = 4;      // elements (of four dims) per thread of k_pool_bwd
 template <typename T>
 __global__ void __launch_bounds__(256) k_pool_bwd(const float* __restrict__ dKpart, const float* __restrict__ dL, T* __restrict__ dK,
                                                   PoolGeom g, int pool) {
@@ -219,26 +220,32 @@ __global__ void __launch_bounds__(256) k_pool_bwd(const float* __restrict__ dKpa
   }
   const int bh = blockIdx.y;
   const unsigned per_row = g.d / 4;
-  const unsigned idx = blockIdx.x * blockDim.x + threadIdx.x;     // n * d / 4 < 2^32
-  if (idx >= (unsigned)g.n * per_row) return;
-  const int j = (int)(idx / per_row), c = (int)(idx % per_row) * 4;
-  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (dKpart) v = ld4(dKpart + ((long long)bh * g.n + j) * g.d + c);
-  if (pool && j >= g.prefix) {
-    const int r = (j - g.prefix) / g.gw, q = (j - g.prefix) % g.gw;
-    // a token row lies in bin floor(r mh / gh) and, where neighbouring bins overlap, in the next one too
-    const int a0 = (int)(((unsigned)r * (unsigned)g.mh) / (unsigned)g.gh), b0 = (int)(((unsigned)q * (unsigned)g.mw) / (unsigned)g.gw);
-    for (int a = (a0 > 0 ? a0 - 1 : 0); a <= a0 + 1 && a < g.mh; ++a) {
-      if (r < rlo[a] || r >= rhi[a]) continue;
-      for (int bb = (b0 > 0 ? b0 - 1 : 0); bb <= b0 + 1 && bb < g.mw; ++bb) {
-        if (q < clo[bb] || q >= chi[bb]) continue;
-        const float inv = 1.f / (float)((rhi[a] - rlo[a]) * (chi[bb] - clo[bb]));
-        const float4 t = ld4(dL + ((long long)bh * g.m + a * g.mw + bb) * g.d + c);
-        v.x += t.x * inv; v.y += t.y * inv; v.z += t.z * inv; v.w += t.w * inv;
+  const unsigned total = (unsigned)g.n * per_row;                  // n * d / 4 < 2^32
+  // POOL_EPT elements of four dims per thread, a CTA's share contiguous, so that the bin tables are built once
+  // per 1024 elements
+#pragma unroll
+  for (int u = 0; u < POOL_EPT; ++u) {
+    const unsigned idx = (blockIdx.x * POOL_EPT + u) * blockDim.x + threadIdx.x;
+    if (idx >= total) break;
+    const int j = (int)(idx / per_row), c = (int)(idx % per_row) * 4;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (dKpart) v = ld4(dKpart + ((long long)bh * g.n + j) * g.d + c);
+    if (pool && j >= g.prefix) {
+      const int r = (j - g.prefix) / g.gw, q = (j - g.prefix) % g.gw;
+      // a token row lies in bin floor(r mh / gh) and, where neighbouring bins overlap, in the next one too
+      const int a0 = (int)(((unsigned)r * (unsigned)g.mh) / (unsigned)g.gh), b0 = (int)(((unsigned)q * (unsigned)g.mw) / (unsigned)g.gw);
+      for (int a = (a0 > 0 ? a0 - 1 : 0); a <= a0 + 1 && a < g.mh; ++a) {
+        if (r < rlo[a] || r >= rhi[a]) continue;
+        for (int bb = (b0 > 0 ? b0 - 1 : 0); bb <= b0 + 1 && bb < g.mw; ++bb) {
+          if (q < clo[bb] || q >= chi[bb]) continue;
+          const float inv = 1.f / (float)((rhi[a] - rlo[a]) * (chi[bb] - clo[bb]));
+          const float4 t = ld4(dL + ((long long)bh * g.m + a * g.mw + bb) * g.d + c);
+          v.x += t.x * inv; v.y += t.y * inv; v.z += t.z * inv; v.w += t.w * inv;
+        }
       }
     }
+    st4(dK + ((long long)bh * g.n + j) * g.d + c, v);
   }
-  st4(dK + ((long long)bh * g.n + j) * g.d + c, v);
 }
 
 // out[e] = sum_p parts[p][e] for up to three part arrays laid out [BH][np][count]; count % 4 == 0
