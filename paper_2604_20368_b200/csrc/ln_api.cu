@@ -42,6 +42,7 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   // history slots: fp32 [m][ldm], except on the m <= 64 tensor-core path, whose slots hold operand images
   pl->hslot = (long long)p->m * pl->ldm;
   if (p->dtype == LN_BF16 && p->m <= 64 && pl->hslot < (long long)(NsTile<64>::mat_bytes / 4)) pl->hslot = NsTile<64>::mat_bytes / 4;
+  if (p->dtype == LN_BF16 && p->m > 64 && p->m <= 128) pl->hslot = (long long)(kUmmaMatBytes / 4);     // 64 KiB images >= m * ldm * 4
   // token chunks per head for the reductions over tokens: about eight waves of CTAs (two per SM) so that
   // the last wave costs little, but at least 64 tokens per chunk
   const int mblk = (p->m + 63) / 64;

@@ -936,7 +936,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_fw
   const long long mm = (long long)m * m, md = (long long)m * D;
   // the iterate histories of the shared-memory path use the padded leading dimension (128-bit accesses)
   const int ldx = (MP > 0) ? ldm : m;
-  const long long mx = (MP == 64) ? hslot : (long long)m * ldx;
+  const long long mx = (MP == 64 || MP == 128) ? hslot : (long long)m * ldx;
   W += bh * mm; Wr += bh * mm; P += bh * mm; Xh += (long long)bh * (T + 1) * mx; hdr += bh;
   if (Ph) Ph += (long long)bh * T * mx;
   Mout += bh * md; Y += bh * md; Yt += bh * md; ybar += (long long)bh * D;
@@ -946,7 +946,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_fw
   bool tc_ok = true;
   if constexpr (MP == 128) {        // tcgen05 + TMEM
     __shared__ UmmaCtl ctl;
-    tc_ok = ns_forward_umma(m, T, eps, alpha_in, W, Xh, Ph, ldx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
+    tc_ok = ns_forward_umma(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
     __syncthreads();
   } else if constexpr (MP == 64) {  // mma.sync from shared memory
     ns_forward_smem<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red);
@@ -1016,7 +1016,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_bw
   const int gt = crank * 256 + tid, gn = 256 * CL;
   const long long mm = (long long)m * m, md = (long long)m * D;
   const int ldx = (MP > 0) ? ldm : m;
-  const long long mx = (MP == 64) ? hslot : (long long)m * ldx;       // one slot of the iterate histories
+  const long long mx = (MP == 64 || MP == 128) ? hslot : (long long)m * ldx;       // one slot of the iterate histories
   const long long ms = (long long)m * ldm;                             // one scratch matrix
   W += bh * mm; Xh += (long long)bh * (T + 1) * mx; Ph += (long long)bh * T * mx; hdr += bh; Msaved += bh * md;
   Wr += bh * ms; P += bh * ms; Hm += bh * ms; Ga += bh * ms; Gb += bh * ms; dWm += bh * ms; dXm += bh * ms;
@@ -1059,7 +1059,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_bw
   }
   if constexpr (MP == 128) {
     __shared__ UmmaCtl ctl;
-    const bool tc_ok = ns_backward_umma(m, T, eps, W, Xh, Ph, ldx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
+    const bool tc_ok = ns_backward_umma(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
     if (dev_status && !tc_ok && tid == 0) atomicOr(dev_status + bh, 2);
   } else if constexpr (MP == 64) ns_backward_smem<MP>(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
   else { ns_backward_dev<TC, CL>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red, crank); if (CL > 1) phase_sync<CL>(); }

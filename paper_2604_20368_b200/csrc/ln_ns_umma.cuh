@@ -16,7 +16,8 @@ constexpr int UIMG = UM * UM;                 // bf16 elements of one image part
 constexpr size_t kUmmaMatBytes = (size_t)2 * UIMG * sizeof(bf16);   // hi + lo = 64 KiB
 
 struct UmmaCtl {                              // small static shared state of the tcgen05 kernels
-  unsigned long long mbar;
+  unsigned long long mbar;                    // completion of MMAs
+  unsigned long long mbar_ld;                 // arrival of a bulk-copied operand image
   uint32_t tmem_base;
   int timeout;
 };
@@ -40,13 +41,16 @@ __device__ __forceinline__ void umma_gemm(uint32_t tmem_d, const bf16* A, bool a
 
 // issue (thread 0) + wait (everyone); returns false on a timed-out wait
 // `phase` is each thread's own copy of the mbarrier phase (identical in all threads)
+// drain_stores: thread 0 first lets its bulk stores finish reading shared memory, so that when the barrier
+// completes the buffers those stores read may be overwritten by everybody
 __device__ __forceinline__ bool umma_run(UmmaCtl& ctl, uint32_t& phase, uint32_t tmem_d, const bf16* A, bool a_k, const bf16* Bm,
                                          bool b_k, bool accumulate, const bf16* A2 = nullptr, bool a2_k = true,
-                                         const bf16* B2 = nullptr, bool b2_k = true) {
+                                         const bf16* B2 = nullptr, bool b2_k = true, bool drain_stores = false) {
   if (threadIdx.x == 0) {
     umma::fence_after_sync();
     umma_gemm(tmem_d, A, a_k, Bm, b_k, accumulate);
     if (A2) umma_gemm(tmem_d, A2, a2_k, B2, b2_k, true);
+    if (drain_stores) umma::bulk_store_wait_read();
     umma::commit(&ctl.mbar);
   }
   const bool ok = umma::mbar_wait(&ctl.mbar, phase & 1);
@@ -121,7 +125,7 @@ __device__ __forceinline__ void umma_load_image(const float* __restrict__ src, i
 }
 
 __device__ __forceinline__ void umma_begin(UmmaCtl& ctl, int ncols) {
-  if (threadIdx.x == 0) { umma::mbar_init(&ctl.mbar, 1); ctl.timeout = 0; }
+  if (threadIdx.x == 0) { umma::mbar_init(&ctl.mbar, 1); umma::mbar_init(&ctl.mbar_ld, 1); ctl.timeout = 0; }
   if ((threadIdx.x >> 5) == 0) umma::tmem_alloc(&ctl.tmem_base, ncols);
   umma::fence_before_sync();
   __syncthreads();
@@ -141,17 +145,18 @@ __device__ __forceinline__ void umma_step_done(UmmaCtl& ctl, bool ok) {
   __syncthreads();
 }
 
-// Forward iteration.  smem: images W, X, P (3 * kUmmaMatBytes).  Xh [T+1][m][ld], Ph [T][m][ld] fp32 in global.
-// Returns false if a tensor-core wait timed out.
+// Forward iteration.  smem: images W, X, Q (3 * kUmmaMatBytes).  Histories in global memory, slots of hs floats
+// (hs * 4 >= kUmmaMatBytes): Xh slot k < T receives the operand image of X_k, slot T receives X_T in fp32 (leading
+// dimension ld); Ph slot k (may be NULL) receives the image of Q_k = 2I - W X_k.  The images leave by bulk copies
+// that one thread issues and that run beside the next product.  Returns false if a tensor-core wait timed out.
 __device__ bool ns_forward_umma(int m, int T, float eps, float alpha_in, const float* W, float* Xh, float* Ph, int ld,
-                                NsHdr* hdr, bf16* smem, float* red, UmmaCtl& ctl) {
+                                long long hs, NsHdr* hdr, bf16* smem, float* red, UmmaCtl& ctl) {
   bf16* sW = smem; bf16* sX = smem + 2 * UIMG; bf16* sP = smem + 4 * UIMG;
-  const long long mm = (long long)m * ld;
   const int tid = threadIdx.x, warp = tid >> 5;
   const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64;
   umma_begin(ctl, 128);
   uint32_t phase = 0;
-  // W + eps I staged in fp32 in the space of P: norms, images of W and X_0, fp32 X_0 all come from there
+  // W + eps I staged in fp32 in the space of Q: norms, images of W and X_0, fp32 X_0 all come from there
   float* Wf = reinterpret_cast<float*>(sP);      // [128][128], pitch 128
 #pragma unroll 1
   for (int b0 = 0; b0 < UM * UM / 256; b0 += 8) {
@@ -194,54 +199,72 @@ __device__ bool ns_forward_umma(int m, int T, float eps, float alpha_in, const f
     for (int q = 0; q < 64; ++q) { w[q] = Wf[row * UM + col0 + q]; x0[q] = alpha * Wf[(col0 + q) * UM + row]; }
     umma_row_to_image(w, row, col0, sW);
     umma_row_to_image(x0, row, col0, sX);
-    if (row < m) umma_row_to_global(x0, Xh + (long long)row * ld, col0, ld);
+    if (T == 0 && row < m) umma_row_to_global(x0, Xh + (long long)row * ld, col0, ld);
   }
   bool ok = true;
   umma_step_done(ctl, true);
+  if (tid == 0 && T > 0) umma::bulk_store(Xh, sX, (uint32_t)kUmmaMatBytes);                 // image of X_0
   for (int k = 0; k < T; ++k) {
-    ok &= umma_run(ctl, phase, ctl.tmem_base, sW, true, sX, false, false);                   // D = W X_k
+    // the store of Q_{k-1} has read sP before the barrier of this product completes
+    ok &= umma_run(ctl, phase, ctl.tmem_base, sW, true, sX, false, false, nullptr, true, nullptr, true, true);   // D = W X_k
     {
       float v[64];
       umma_row(ctl.tmem_base, col0, v);
-      if (Ph && row < m) umma_row_to_global(v, Ph + (long long)k * mm + (long long)row * ld, col0, ld);
 #pragma unroll
-      for (int q = 0; q < 64; ++q) v[q] = ((row == col0 + q && row < m) ? 2.f : 0.f) - v[q];   // 2I - W X_k
+      for (int q = 0; q < 64; ++q) v[q] = ((row == col0 + q && row < m) ? 2.f : 0.f) - v[q];   // Q_k = 2I - W X_k
       umma_row_to_image(v, row, col0, sP);
     }
     umma_step_done(ctl, ok);
-    ok &= umma_run(ctl, phase, ctl.tmem_base, sX, true, sP, false, false);                   // D = X_k (2I - W X_k)
+    if (tid == 0 && Ph) umma::bulk_store(Ph + k * hs, sP, (uint32_t)kUmmaMatBytes);
+    // the store of X_k has read sX before the barrier of this product completes
+    ok &= umma_run(ctl, phase, ctl.tmem_base, sX, true, sP, false, false, nullptr, true, nullptr, true, true);   // D = X_k Q_k
     {
       float v[64];
       umma_row(ctl.tmem_base, col0, v);
-      if (row < m) umma_row_to_global(v, Xh + (long long)(k + 1) * mm + (long long)row * ld, col0, ld);
-      umma_row_to_image(v, row, col0, sX);     // the MMAs that read X_k have completed
+      if (k + 1 == T && row < m) umma_row_to_global(v, Xh + T * hs + (long long)row * ld, col0, ld);
+      umma_row_to_image(v, row, col0, sX);     // the MMAs and the bulk store that read X_k have completed
     }
     umma_step_done(ctl, ok);
+    if (tid == 0 && k + 1 < T) umma::bulk_store(Xh + (k + 1) * hs, sX, (uint32_t)kUmmaMatBytes);
   }
+  if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");      // every image has reached global memory
   ok &= (ctl.timeout == 0);
   umma_end(ctl, 128);
   return ok;
 }
 
-// Adjoint for a symmetric W (see ns_backward_smem for the algebra).  smem: images A (also used for P), G, H.
-// TMEM: 128 columns for the running product, 128 for dW accumulated over all steps.
+// Adjoint for a symmetric W (see ns_backward_smem for the algebra): per step, with A = X_k and Q = 2I - W X_k as
+// the forward pass left them (operand images), H = A^T G, dW -= H A^T, G <- G Q^T + Q^T G - 2G.
+// smem: images A (also used for Q), G, H.  TMEM: 128 columns for the running product, 128 for dW accumulated over
+// all steps.  The images arrive by bulk copies on an mbarrier; the copy of the next A runs beside the G update.
 __device__ bool ns_backward_umma(int m, int T, float eps, const float* W, const float* Xh, const float* Ph, int ld,
-                                 const NsHdr* hdr, const float* G0, float* dW, float* Gf, bf16* smem, float* red,
-                                 UmmaCtl& ctl) {
+                                 long long hs, const NsHdr* hdr, const float* G0, float* dW, float* Gf, bf16* smem,
+                                 float* red, UmmaCtl& ctl) {
   bf16* sA = smem; bf16* sG = smem + 2 * UIMG; bf16* sH = smem + 4 * UIMG;
-  const long long mm = (long long)m * ld;
   const int tid = threadIdx.x, warp = tid >> 5;
   const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64;
   umma_begin(ctl, 256);
-  uint32_t phase = 0;
+  uint32_t phase = 0, ph_ld = 0;
   const uint32_t t_acc = ctl.tmem_base, t_dw = ctl.tmem_base + 128;
+  auto load_image = [&](const float* src) {     // one thread starts the copy into sA
+    if (tid == 0) {
+      umma::mbar_expect_tx(&ctl.mbar_ld, (uint32_t)kUmmaMatBytes);
+      umma::bulk_load(sA, src, (uint32_t)kUmmaMatBytes, &ctl.mbar_ld);
+    }
+  };
+  auto wait_image = [&]() {                     // everybody sees the image (thread 0 issues the MMAs that read it)
+    const bool got = umma::mbar_wait(&ctl.mbar_ld, ph_ld & 1);
+    ph_ld ^= 1u;
+    return got;
+  };
+  if (T > 0) load_image(Xh + (long long)(T - 1) * hs);
   float G[64];                                 // this thread's part of G in full precision
 #pragma unroll
   for (int q = 0; q < 64; ++q) G[q] = (row < m && col0 + q < m) ? G0[(long long)row * ld + col0 + q] : 0.f;
   umma_row_to_image(G, row, col0, sG);
   bool ok = true;
   for (int k = T - 1; k >= 0; --k) {
-    umma_load_image(Xh + (long long)k * mm, m, ld, sA);                               // A = X_k
+    ok &= wait_image();                                                                       // A = X_k
     umma_step_done(ctl, ok);
     ok &= umma_run(ctl, phase, t_acc, sA, false, sG, false, false);                          // H = A^T G
     {
@@ -251,14 +274,16 @@ __device__ bool ns_backward_umma(int m, int T, float eps, const float* W, const 
     }
     umma_step_done(ctl, ok);
     ok &= umma_run(ctl, phase, t_dw, sH, true, sA, true, k != T - 1);                        // dW accumulator += H A^T
-    umma_load_image(Ph + (long long)k * mm, m, ld, sA);                               // P = W X_k (A is no longer read)
+    load_image(Ph + (long long)k * hs);                                                       // Q_k (A is no longer read)
+    ok &= wait_image();
     umma_step_done(ctl, ok);
-    ok &= umma_run(ctl, phase, t_acc, sG, true, sA, true, false, sA, false, sG, false);      // G P^T + P^T G
+    ok &= umma_run(ctl, phase, t_acc, sG, true, sA, true, false, sA, false, sG, false);      // G Q^T + Q^T G
+    if (k > 0) load_image(Xh + (long long)(k - 1) * hs);                                      // next A, beside the G update
     {
       float v[64];
       umma_row(t_acc, col0, v);
 #pragma unroll
-      for (int q = 0; q < 64; ++q) G[q] = (row < m && col0 + q < m) ? 2.f * G[q] - v[q] : 0.f;
+      for (int q = 0; q < 64; ++q) G[q] = (row < m && col0 + q < m) ? v[q] - 2.f * G[q] : 0.f;
       umma_row_to_image(G, row, col0, sG);
     }
   }

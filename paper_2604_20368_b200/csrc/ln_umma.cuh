@@ -81,6 +81,14 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, 
                ::"r"(s32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(s32(mbar)) : "memory");
 }
 
+// Bulk copy shared -> global by ONE thread, as one bulk group; bulk_store_wait_read() returns once every group this
+// thread issued has finished READING shared memory (the buffer may then be overwritten).
+__device__ __forceinline__ void bulk_store(void* dst_gmem, const void* src_smem, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst_gmem), "r"(s32(src_smem)), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+
 // TMEM allocation (whole warp; ncols a power of two in [32, 512]); the base address lands in *slot.
 __device__ __forceinline__ void tmem_alloc(uint32_t* slot, int ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(slot)), "r"(ncols));
