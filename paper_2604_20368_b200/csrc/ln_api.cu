@@ -290,11 +290,13 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     a.nscale = -1.4426950408889634f / p->lambda;
     launch_l1_args("l1_CRW", a, 3, BH, st);
   }
-  // M = R V, partial over token chunks
+  // M = R V, partial over token chunks (a single chunk writes M itself)
+  float* const Mdst = pl.chunks == 1 ? x.M : w.Mpart;
+  const int Mparts = pl.chunks == 1 ? 0 : pl.chunks;
   if constexpr (std::is_same<T, bf16>::value)
-    LN_LAUNCH("tn_M", st, k_tn_mma<D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, w.Mpart, nullptr, n, m, pl.rpc));
+    LN_LAUNCH("tn_M", st, k_tn_mma<D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
   else
-    LN_LAUNCH("tn_M", st, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, w.Mpart, nullptr, n, m, pl.rpc));
+    LN_LAUNCH("tn_M", st, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
   // Newton-Schulz, Y = X M, folded map
   const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);   // tcgen05 products over the landmarks
   {
@@ -302,7 +304,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     auto launch = [&](auto kern, size_t smem, int cl = 1) {
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       LN_LAUNCH("k_mid_fwd", st, launch_clustered(kern, BH * cl, cl, smem, st, m, pl.ldm, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode,
-                                                  p->whiten, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, w.Mpart, pl.chunks, x.M, w.Y, x.Yt,
+                                                  p->whiten, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, w.Mpart, Mparts, x.M, w.Y, x.Yt,
                                                   x.ybar, dev_status, pl.hslot, umma_prod ? reinterpret_cast<bf16*>(x.Yimg) : nullptr));
     };
     if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * NsTile<64>::mat_bytes);

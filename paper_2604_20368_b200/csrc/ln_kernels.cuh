@@ -941,23 +941,25 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_fw
   if (Ph) Ph += (long long)bh * T * mx;
   Mout += bh * md; Y += bh * md; Yt += bh * md; ybar += (long long)bh * D;
   Mpart += (long long)bh * nchunks * md;
-  for (long long e = (long long)gt * 4; e < md; e += 4 * gn)
-    *reinterpret_cast<float4*>(Mout + e) = sum_parts4(Mpart, nchunks, md, e);
+  if (nchunks > 0)                               // nchunks == 0: the single partial result was written to Mout directly
+    for (long long e = (long long)gt * 4; e < md; e += 4 * gn)
+      *reinterpret_cast<float4*>(Mout + e) = sum_parts4(Mpart, nchunks, md, e);
   bool tc_ok = true;
+  float bad = 0.f;                               // non-finite entries of X_T seen by this thread
   if constexpr (MP == 128) {        // tcgen05 + TMEM
     __shared__ UmmaCtl ctl;
-    tc_ok = ns_forward_umma(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
+    tc_ok = ns_forward_umma(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl, bad);
     __syncthreads();
   } else if constexpr (MP == 64) {  // mma.sync from shared memory
-    ns_forward_smem<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red);
+    ns_forward_smem<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, bad);
     __syncthreads();
   } else {
     ns_forward_dev<TC, CL>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red, crank);
   }
   const float* XT = Xh + (long long)T * mx;
   if (dev_status) {
-    float bad = 0.f;
-    for (int e = tid; e < m * m; e += 256) bad += isfinite(XT[(long long)(e / m) * ldx + e % m]) ? 0.f : 1.f;
+    if constexpr (MP == 0)
+      for (int e = tid; e < m * m; e += 256) bad += isfinite(XT[(long long)(e / m) * ldx + e % m]) ? 0.f : 1.f;
     bad = block_sum(bad, red);
     if (tid == 0 && crank == 0) atomicOr(dev_status + bh, (bad > 0.f ? 1 : 0) | (tc_ok ? 0 : 2));   // bit1: a bounded tensor-core wait ran out
   }

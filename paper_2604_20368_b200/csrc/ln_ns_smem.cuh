@@ -210,7 +210,8 @@ __device__ __forceinline__ void image_wait_all_but_one() { asm volatile("cp.asyn
 // dimension ld >= m); Ph slot k (may be NULL) receives the image of Q_k = 2I - W X_k.
 template <int MP>
 __device__ void ns_forward_smem(int m, int T, float eps, float alpha_in, const float* W, float* Xh, float* Ph, int ld,
-                                long long hs, NsHdr* hdr, bf16* smem, float* red) {
+                                long long hs, NsHdr* hdr, bf16* smem, float* red, float& bad) {
+  // bad: this thread's count of non-finite entries of X_T (from its registers: nothing is read back)
   using TL = NsTile<MP>;
   bf16* sW = smem; bf16* sX = smem + 2 * TL::MAT; bf16* sP = smem + 4 * TL::MAT;
   // W + eps I is first staged in fp32 (in the space of P, which is not needed yet): norms, the split
@@ -265,7 +266,7 @@ __device__ void ns_forward_smem(int m, int T, float eps, float alpha_in, const f
     const float x0 = alpha * Wf[j * PF + i];                          // X_0 = alpha (W + eps I)^T
     split2(x0, h, l);
     sX[i * TL::LD + j] = h; sX[TL::MAT + i * TL::LD + j] = l;
-    if (T == 0 && i < m && j < m) Xh[(long long)i * ld + j] = x0;
+    if (T == 0 && i < m && j < m) { Xh[(long long)i * ld + j] = x0; bad += isfinite(x0) ? 0.f : 1.f; }
   }
   __syncthreads();
   if (T > 0) image_to_global<MP>(sX, Xh);
@@ -286,7 +287,15 @@ __device__ void ns_forward_smem(int m, int T, float eps, float alpha_in, const f
     __syncthreads();
     if (Ph) image_to_global<MP>(sP, Ph + k * hs);                       // kept for the backward pass
     smem_gemm<MP, false, false>(acc, sX, sP, false);                    // X_{k+1} = X_k (2I - W X_k)
-    if (k + 1 == T) frag_to_global<MP>(acc, Xh + T * hs, m, ld);
+    if (k + 1 == T) {
+      frag_to_global<MP>(acc, Xh + T * hs, m, ld);
+#pragma unroll
+      for (int a = 0; a < TL::MT; ++a)
+#pragma unroll
+        for (int t = 0; t < TL::NT; ++t)
+#pragma unroll
+          for (int q = 0; q < 4; ++q) bad += isfinite(acc[a][t][q]) ? 0.f : 1.f;      // padding is zero, hence finite
+    }
     __syncthreads();                                                    // every warp is done reading X_k
     frag_to_smem<MP>(acc, sX);
     __syncthreads();

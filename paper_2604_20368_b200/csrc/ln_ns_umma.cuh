@@ -150,7 +150,8 @@ __device__ __forceinline__ void umma_step_done(UmmaCtl& ctl, bool ok) {
 // dimension ld); Ph slot k (may be NULL) receives the image of Q_k = 2I - W X_k.  The images leave by bulk copies
 // that one thread issues and that run beside the next product.  Returns false if a tensor-core wait timed out.
 __device__ bool ns_forward_umma(int m, int T, float eps, float alpha_in, const float* W, float* Xh, float* Ph, int ld,
-                                long long hs, NsHdr* hdr, bf16* smem, float* red, UmmaCtl& ctl) {
+                                long long hs, NsHdr* hdr, bf16* smem, float* red, UmmaCtl& ctl, float& bad) {
+  // bad: this thread's count of non-finite entries of X_T (from its registers)
   bf16* sW = smem; bf16* sX = smem + 2 * UIMG; bf16* sP = smem + 4 * UIMG;
   const int tid = threadIdx.x, warp = tid >> 5;
   const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64;
@@ -200,6 +201,10 @@ __device__ bool ns_forward_umma(int m, int T, float eps, float alpha_in, const f
     umma_row_to_image(w, row, col0, sW);
     umma_row_to_image(x0, row, col0, sX);
     if (T == 0 && row < m) umma_row_to_global(x0, Xh + (long long)row * ld, col0, ld);
+    if (T == 0) {
+#pragma unroll
+      for (int q = 0; q < 64; ++q) bad += isfinite(x0[q]) ? 0.f : 1.f;
+    }
   }
   bool ok = true;
   umma_step_done(ctl, true);
@@ -221,7 +226,11 @@ __device__ bool ns_forward_umma(int m, int T, float eps, float alpha_in, const f
     {
       float v[64];
       umma_row(ctl.tmem_base, col0, v);
-      if (k + 1 == T && row < m) umma_row_to_global(v, Xh + T * hs + (long long)row * ld, col0, ld);
+      if (k + 1 == T) {
+        if (row < m) umma_row_to_global(v, Xh + T * hs + (long long)row * ld, col0, ld);
+#pragma unroll
+        for (int q = 0; q < 64; ++q) bad += isfinite(v[q]) ? 0.f : 1.f;
+      }
       umma_row_to_image(v, row, col0, sX);     // the MMAs and the bulk store that read X_k have completed
     }
     umma_step_done(ctl, ok);
