@@ -262,6 +262,25 @@ def test_singular_landmarks_are_flagged_finite():
     assert rel_err(f64(g["O"])[0, 0], o["O"][0]) < 1e-4
 
 
+@pytest.mark.parametrize("name,B,H", [("cfg2", 1, 2), ("cfg4a", 1, 1), ("cfg5_m256_T4", 1, 1), ("cfg1", 1, 1)])
+def test_diverged_iteration_sets_status_bit(name, B, H):
+    """The step size printed in Alg. 2 (2 / ||W||_2, far above 1 / (||W||_1 ||W||_inf) for a unit-diagonal W) makes
+    the iteration blow up; every Newton-Schulz engine (m <= 64, tcgen05, clustered, fp32) must report it in bit 0
+    of dev_status instead of trapping, and a sane step size must leave the flags at zero."""
+    cfg = synth.shrink(synth.CONFIGS[name], B=B, H=H)
+    inp = synth.make_inputs(cfg)
+    Q, K, V = (inp[k].to(DEV) for k in ("Q", "K", "V"))
+    for alpha, want in ((1.9, 1), (0.0, 0)):
+        p = ln.problem_from_config(cfg, whiten=inp["whiten"].to(DEV))
+        p.ns_alpha = alpha
+        p.ns_iters = max(cfg.T, 8)
+        status = torch.full((cfg.B * cfg.H,), -1, dtype=torch.int32, device=DEV)
+        ln.laplace_nystrom_fwd(p, Q, K, V, dev_status=status)
+        torch.cuda.synchronize()
+        assert all(int(v) & 1 == want for v in status.cpu()), (name, alpha, status)
+        assert all(int(v) & 2 == 0 for v in status.cpu())
+
+
 def test_host_buffer_step_matches_device_path():
     """laplace_nystrom_fwd_bwd_host (copies + forward + backward on one stream) returns the same bits as the device
     entry points called on device copies of the same tensors."""
