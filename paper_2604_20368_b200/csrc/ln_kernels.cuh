@@ -1061,11 +1061,13 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_bw
   }
   if constexpr (MP == 128) {
     __shared__ UmmaCtl ctl;
-    const bool tc_ok = ns_backward_umma(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
+    const bool tc_ok = ns_backward_umma(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, GW, ldm, inv_lambda, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
     if (dev_status && !tc_ok && tid == 0) atomicOr(dev_status + bh, 2);
   } else if constexpr (MP == 64) ns_backward_smem<MP>(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
   else { ns_backward_dev<TC, CL>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red, crank); if (CL > 1) phase_sync<CL>(); }
   // GW = (dW o K_LL + (dW o K_LL)^T) / lambda; four elements per batch so that the loads overlap
+  // (the tcgen05 engine has written GW from shared memory already)
+  if constexpr (MP != 128)
   for (long long e0 = (long long)gt * 4; e0 < (long long)m * ldm; e0 += 4 * gn) {
     float a[4], b[4], c[4], d4[4];
 #pragma unroll

@@ -246,9 +246,11 @@ __device__ bool ns_forward_umma(int m, int T, float eps, float alpha_in, const f
 // the forward pass left them (operand images), H = A^T G, dW -= H A^T, G <- G Q^T + Q^T G - 2G.
 // smem: images A (also used for Q), G, H.  TMEM: 128 columns for the running product, 128 for dW accumulated over
 // all steps.  The images arrive by bulk copies on an mbarrier; the copy of the next A runs beside the G update.
+// Output: GW [m][ldgw] = (dW o W + (dW o W)^T) / lambda, the upstream of the landmark kernel block (dW itself
+// stays on chip).
 __device__ bool ns_backward_umma(int m, int T, float eps, const float* W, const float* Xh, const float* Ph, int ld,
-                                 long long hs, const NsHdr* hdr, const float* G0, float* dW, float* Gf, bf16* smem,
-                                 float* red, UmmaCtl& ctl) {
+                                 long long hs, const NsHdr* hdr, const float* G0, float* GW, int ldgw, float inv_lambda,
+                                 bf16* smem, float* red, UmmaCtl& ctl) {
   bf16* sA = smem; bf16* sG = smem + 2 * UIMG; bf16* sH = smem + 4 * UIMG;
   const int tid = threadIdx.x, warp = tid >> 5;
   const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64;
@@ -297,20 +299,69 @@ __device__ bool ns_backward_umma(int m, int T, float eps, const float* W, const 
     }
   }
   umma_step_done(ctl, ok);
-  {  // dW = -(accumulated sum), G -> global for the transposed accesses of the tail
+  float dw[64];                                // this thread's part of -(accumulated H A^T)
+  {
     float v[64];
     if (T > 0) umma_row(t_dw, col0, v);
 #pragma unroll
-    for (int q = 0; q < 64; ++q) v[q] = (T > 0) ? -v[q] : 0.f;
-    if (row < m) {
-      umma_row_to_global(v, dW + (long long)row * ld, col0, ld);
-      umma_row_to_global(G, Gf + (long long)row * ld, col0, ld);
-    }
+    for (int q = 0; q < 64; ++q) dw[q] = (T > 0) ? -v[q] : 0.f;
   }
   ok &= (ctl.timeout == 0);
   umma_end(ctl, 256);
   __syncthreads();
-  ns_backward_tail(m, eps, W, ld, hdr, dW, Gf, red);
+  // End of the adjoint and the upstream of the landmark block, from shared memory (the operand buffers are free):
+  //   X_0 = alpha (W + eps I)^T:  d alpha = <G, Wr^T>,  dW += alpha G^T, then the alpha(W) terms;
+  //   GW = (dW o W + (dW o W)^T) / lambda.
+  // G and Wr are staged as fp32 [128][129] (the odd pitch makes the transposed reads conflict-free).
+  constexpr int PT = UM + 1;
+  float* sGf = reinterpret_cast<float*>(smem);
+  float* sWf = sGf + UM * PT;
+#pragma unroll
+  for (int q = 0; q < 64; ++q) sGf[row * PT + col0 + q] = G[q];
+  for (int e = tid; e < UM * UM; e += 256) {
+    const int i = e >> 7, j = e & 127;
+    sWf[i * PT + j] = (i < m && j < m) ? W[(long long)i * m + j] + (i == j ? eps : 0.f) : 0.f;
+  }
+  __syncthreads();
+  const float alpha = hdr->alpha;
+  float part = 0.f;
+#pragma unroll
+  for (int q = 0; q < 64; ++q) part += G[q] * sWf[(col0 + q) * PT + row];
+  const float dalpha = block_sum(part, red);
+  const bool aa = hdr->auto_alpha != 0;
+  const int js = hdr->jstar, is = hdr->istar;
+  const float c1 = dalpha * (-alpha / hdr->n1), c2 = dalpha * (-alpha / hdr->ninf);
+#pragma unroll
+  for (int q = 0; q < 64; ++q) {
+    const int j = col0 + q;
+    float v = dw[q] + alpha * sGf[j * PT + row];
+    if (aa) {
+      const float w = sWf[row * PT + j];
+      const float sg = w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f);
+      if (j == js) v += c1 * sg;
+      if (row == is) v += c2 * sg;
+    }
+    dw[q] = (row < m && j < m) ? v : 0.f;
+  }
+  __syncthreads();                             // everybody has read G
+#pragma unroll
+  for (int q = 0; q < 64; ++q) sGf[row * PT + col0 + q] = dw[q];      // now dW
+  __syncthreads();
+  if (row < m) {
+    float* grow = GW + (long long)row * ldgw;
+#pragma unroll
+    for (int q = 0; q < 64; q += 4) {
+      const int j = col0 + q;
+      if (j >= ldgw) break;
+      float o[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int jj = j + u;
+        o[u] = (jj < m) ? (dw[q + u] * sWf[row * PT + jj] + sGf[jj * PT + row] * sWf[jj * PT + row]) * inv_lambda : 0.f;
+      }
+      *reinterpret_cast<float4*>(grow + j) = make_float4(o[0], o[1], o[2], o[3]);
+    }
+  }
   return ok;
 }
 
