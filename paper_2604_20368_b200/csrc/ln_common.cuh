@@ -55,6 +55,21 @@ __device__ __forceinline__ float half_step(float t) {
   return r;
 }
 
+// min(max(a * b + c, 0), 1) in one instruction of the FMA pipe.
+__device__ __forceinline__ float sat_fma(float a, float b, float c) {
+  float r;
+  asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+// Scale s and offset b of a threshold y such that sat_fma(x, s, b) = (sign(x - y) + 1) / 2 exactly for every
+// bf16 x: s = 2^(22 - exponent(y)), at most 2^126; b = -y s + 1/2 (exact: |y| s < 2^23).
+__device__ __forceinline__ void fold_pair(float y, float& s, float& b) {
+  const int e = (int)((__float_as_uint(y) >> 23) & 0xffu);
+  const int es = e < 23 ? 253 : 276 - e;
+  s = __uint_as_float((unsigned)es << 23);
+  b = fmaf(-y, s, 0.5f);
+}
+
 // Packed pair arithmetic (two fp32 lanes per instruction): the FP32 pipe does not get faster, but a
 // pair costs one issue slot instead of two, which leaves slots for the shared-memory loads.
 typedef unsigned long long f32x2;

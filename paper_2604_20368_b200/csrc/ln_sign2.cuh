@@ -3,9 +3,17 @@
 // For a block A_ij = k(x_i, y_j) with upstream g_ij = dA_ij * A_ij / lambda,
 //     rows[i][c]        = - sum_j              g_ij sign(x_ic - y_jc)          (gradient w.r.t. the tokens x)
 //     part[chunk][j][c] = + sum_{i in chunk}   g_ij sign(x_ic - y_jc)          (gradient w.r.t. the landmarks y)
-// with sign(0) = 0.  Both sums share the difference t = x - y and the step h = half_step(t); per
-// (pair, dim) the FMA pipe sees one packed subtract, one saturating multiply-add and two packed
-// multiply-adds (4 lane-operations; two separate passes cost 6).
+// with sign(0) = 0.  Both sums share the step h = (sign(x - y) + 1) / 2; per (pair, dim) the FMA pipe sees
+// one saturating multiply-add and two packed multiply-adds (3 lane-operations), plus one packed
+// subtract where the tokens are fp32 (two separate passes cost 6).
+//
+// bf16 tokens: the subtraction is folded into the saturating multiply-add.  For a landmark value y with
+// exponent e (y = +-1.f * 2^e) take s = 2^(22 - e) and b = -y s + 1/2: |y| s lies in [2^22, 2^23), where
+// the spacing of fp32 is 1/2, so b is exact, and  h = sat(fma(x, s, b)) = sat(round((x - y) s + 1/2)).
+// A bf16 x that differs from y differs by at least one unit in the last place of y (x - y is a multiple
+// of the smaller of the two spacings, and bf16's is the larger unless x is 2^16 times smaller than y),
+// so (x - y) s is 0 or at least 1/2 in magnitude: h is exactly 0, 1/2 or 1.  y = 0 (and |y| < 2^-104)
+// take s = 2^126.  The pairs (s, b) are formed once per landmark tile by the threads that load it.
 //
 // grid (chunks, D/64, heads); block (16, TG), TG even, 8 <= TG <= 16.  Thread (tc, tt) owns 8 tokens
 // (tt*8 .. tt*8+7 of the current token tile) and 4 dims (4 tc .. 4 tc + 3 of the CTA's 64-dim slab).
@@ -29,8 +37,9 @@ constexpr int S2_TOK = 8 * S2_TGMAX;
 // shared memory, in floats
 constexpr int S2_CP = 0;                                           // [2][RL][TGMAX][64] column partials
 constexpr int S2_GS = S2_CP + 2 * S2_RL * S2_TGMAX * S2_DS;        // [2][RL][TOK] pairs (g, g)
-constexpr int S2_LS = S2_GS + 2 * S2_RL * S2_TOK * 2;              // [2][RL][64] negated landmark values
-constexpr int S2_RS = S2_LS + 2 * S2_RL * S2_DS;                   // [2][TOK] row sums of g
+constexpr int S2_LS = S2_GS + 2 * S2_RL * S2_TOK * 2;              // [2][RL][2][64]: negated landmark values, or scales s and offsets b
+constexpr int S2_LROW = 2 * S2_DS;
+constexpr int S2_RS = S2_LS + 2 * S2_RL * S2_LROW;                 // [2][TOK] row sums of g
 constexpr int S2_CS = S2_RS + 2 * S2_TOK;                          // [mr] column sums of g over the chunk
 __host__ __device__ inline size_t sign2_smem_bytes(int m) { return sizeof(float) * (size_t)(S2_CS + (m + S2_RL - 1) / S2_RL * S2_RL); }
 
@@ -73,7 +82,8 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
   const float* gsrc = G + ((long long)bh * n + ibeg + ltok) * ldg + 4 * lhalf;        // this thread's g row, round 0
   const float* lsrc = Lm + (long long)bh * m * D + slab * S2_DS + (lpiece >> 4) * D + (lpiece & 15) * 4;
   const int gdst = lhalf * 4 * S2_TOK + ltok;                      // f32x2 index inside one buffer of Gs
-  const int ldst = (lpiece >> 4) * S2_DS + (lpiece & 15) * 4;      // float index inside one buffer of Ls
+  const int ldst = (lpiece >> 4) * S2_LROW + (lpiece & 15) * 4;    // float index inside one buffer of Ls
+  constexpr bool FOLD = sizeof(TT) == 2;                           // bf16 tokens: subtraction folded into the step
   float rs = 0.f;                                                  // sum over the rounds of a tile of this thread's g values
 
   // fetch of the round the pointers stand at; tok_ok: this thread's token of that tile is inside the chunk
@@ -96,7 +106,17 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
   auto stash = [&](int buf, int tile, int r, const float4& gq, const float4& lq) {
     f32x2* g2 = Gs + buf * (S2_RL * S2_TOK) + gdst;
     g2[0] = pack2(gq.x, gq.x); g2[S2_TOK] = pack2(gq.y, gq.y); g2[2 * S2_TOK] = pack2(gq.z, gq.z); g2[3 * S2_TOK] = pack2(gq.w, gq.w);
-    if (lpiece >= 0) *reinterpret_cast<float4*>(Ls + buf * (S2_RL * S2_DS) + ldst) = make_float4(-lq.x, -lq.y, -lq.z, -lq.w);
+    if (lpiece >= 0) {
+      float* ld = Ls + buf * (S2_RL * S2_LROW) + ldst;
+      if constexpr (FOLD) {
+        float4 sc, of;
+        fold_pair(lq.x, sc.x, of.x); fold_pair(lq.y, sc.y, of.y); fold_pair(lq.z, sc.z, of.z); fold_pair(lq.w, sc.w, of.w);
+        *reinterpret_cast<float4*>(ld) = sc;
+        *reinterpret_cast<float4*>(ld + S2_DS) = of;
+      } else {
+        *reinterpret_cast<float4*>(ld) = make_float4(-lq.x, -lq.y, -lq.z, -lq.w);
+      }
+    }
     if (r == 0) rs = 0.f;
     rs += (gq.x + gq.y) + (gq.z + gq.w);
     if (r == nrounds - 1) {
@@ -165,7 +185,7 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
       }
     }
     const f32x2* g2 = Gs + buf * (S2_RL * S2_TOK) + tt * 8;
-    const float* ls = Ls + buf * (S2_RL * S2_DS) + tc * 4;
+    const float* ls = Ls + buf * (S2_RL * S2_LROW) + tc * 4;
     float* cp = Cp + buf * (S2_RL * S2_TGMAX * S2_DS) + tt * S2_DS + tc * 4;
     const float* rsrc = Cp + red_buf * (S2_RL * S2_TGMAX * S2_DS);
 #pragma unroll
@@ -182,7 +202,9 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
           }
       }
       if (jj == 1) fold_colsum(buf, r);         // column sums of this round's g tile
-      const ulonglong2 nl = *reinterpret_cast<const ulonglong2*>(ls + jj * S2_DS);
+      const ulonglong2 nl = *reinterpret_cast<const ulonglong2*>(ls + jj * S2_LROW);
+      float4 ob = make_float4(0.f, 0.f, 0.f, 0.f);
+      if constexpr (FOLD) ob = *reinterpret_cast<const float4*>(ls + jj * S2_LROW + S2_DS);
       f32x2 gg[8];
 #pragma unroll
       for (int k2 = 0; k2 < 4; ++k2) {
@@ -192,9 +214,15 @@ __global__ void __launch_bounds__(256, 2) k_sign2(const TT* __restrict__ tok, co
       f32x2 c0 = 0ull, c1 = 0ull;
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
-        const f32x2 t0 = add2(qp[k][0], nl.x), t1 = add2(qp[k][1], nl.y);
-        const f32x2 h0 = pack2(half_step(lo32(t0)), half_step(hi32(t0)));
-        const f32x2 h1 = pack2(half_step(lo32(t1)), half_step(hi32(t1)));
+        f32x2 h0, h1;
+        if constexpr (FOLD) {
+          h0 = pack2(sat_fma(lo32(qp[k][0]), lo32(nl.x), ob.x), sat_fma(hi32(qp[k][0]), hi32(nl.x), ob.y));
+          h1 = pack2(sat_fma(lo32(qp[k][1]), lo32(nl.y), ob.z), sat_fma(hi32(qp[k][1]), hi32(nl.y), ob.w));
+        } else {
+          const f32x2 t0 = add2(qp[k][0], nl.x), t1 = add2(qp[k][1], nl.y);
+          h0 = pack2(half_step(lo32(t0)), half_step(hi32(t0)));
+          h1 = pack2(half_step(lo32(t1)), half_step(hi32(t1)));
+        }
         accR[k][0] = fma2(gg[k], h0, accR[k][0]);
         accR[k][1] = fma2(gg[k], h1, accR[k][1]);
         c0 = fma2(gg[k], h0, c0);
