@@ -17,10 +17,12 @@
  *
  * Conventions common to every entry point
  *   - Every pointer is a DEVICE pointer unless it is the ln_problem itself (host).
- *   - The caller owns every buffer.  The library allocates nothing, keeps no state between
- *     calls, never synchronises the device: it validates arguments on the host, enqueues
- *     kernels on `stream` (a cudaStream_t passed as void*; NULL = the default stream) and
- *     returns.  LN_OK means "enqueued".
+ *   - The caller owns every buffer.  The library allocates no device memory and never
+ *     synchronises the device: it validates arguments on the host, enqueues kernels on
+ *     `stream` (a cudaStream_t passed as void*; NULL = the default stream) and returns.
+ *     LN_OK means "enqueued".  The only state kept between calls is one extra stream and a
+ *     few events per device (see ln_set_overlap), created by the first bf16 attention call on
+ *     that device: that call should come before any stream capture.
  *   - Tensors are contiguous, row-major, 16-byte aligned.  Outputs are fully overwritten.
  *     Inputs are never modified and must not alias outputs.
  *   - Storage type of the [.,.,.,d] tensors is `dtype` (LN_F32 or LN_BF16); all arithmetic and
@@ -191,10 +193,23 @@ int landmarks_pool_bwd(const ln_problem* p, const float* dL, void* dK, void* str
  * launches is bracketed by two CUDA events on its stream.  ln_trace_end synchronises the device,
  * writes the number of traced launches to *count and, for the first `capacity` of them, the
  * duration in milliseconds to ms[i] and a static name to names[i] (either array may be NULL).
- * These two calls create and destroy CUDA events; no other entry point allocates anything.
+ * These two calls create and destroy CUDA events.
  */
 int ln_trace_begin(void);
 int ln_trace_end(int32_t capacity, int32_t* count, float* ms, const char** names);
+
+/*
+ * Overlap of the per-head kernels with the token-sized ones (the paper has no counterpart; Alg. 1
+ * fixes the data flow only).  Newton-Schulz needs nothing but W = k(L,L), and its adjoint and
+ * the landmark-block gradient nothing but Z'^T dO, so laplace_nystrom_fwd / _bwd (bf16 storage)
+ * enqueue them on a second stream that belongs to the library: forked from `stream` by an event
+ * after the kernels they depend on, joined back into `stream` by an event before the first
+ * kernel that needs their results.  Seen from the caller all work is ordered on `stream` as
+ * before.  enabled = 0 keeps every launch on `stream`; the default is 1.  Returns the previous
+ * setting.  While a trace is being recorded the overlap is off, so that each launch is timed
+ * running alone.
+ */
+int ln_set_overlap(int enabled);
 
 #ifdef __cplusplus
 }

@@ -25,7 +25,7 @@ EXPORTS = [
     "laplace_nystrom_fwd", "laplace_nystrom_bwd", "ns_pinv_workspace_bytes", "ns_pinv", "ns_pinv_bwd",
     "l1_kernel", "l1_kernel_bwd_workspace_bytes", "l1_kernel_bwd", "landmarks_pool", "landmarks_pool_bwd",
     "ln_trace_begin", "ln_trace_end", "ns_pinv_static_scratch_bytes", "ns_pinv_static",
-    "laplace_nystrom_host_staging_bytes", "laplace_nystrom_fwd_bwd_host",
+    "laplace_nystrom_host_staging_bytes", "laplace_nystrom_fwd_bwd_host", "ln_set_overlap",
 ]
 
 
@@ -125,6 +125,7 @@ def lib():
         L.ns_pinv_static_scratch_bytes.argtypes = []
         L.ns_pinv_static.argtypes = [i32, i32, vp, i32, f32, f32, vp, vp, vp]
         L.ln_trace_end.argtypes = [i32, ctypes.POINTER(i32), ctypes.POINTER(f32), ctypes.POINTER(ctypes.c_char_p)]
+        L.ln_set_overlap.argtypes = [i32]
         _lib = L
     return _lib
 
@@ -306,6 +307,12 @@ def landmarks_pool_bwd(p: Problem, dL, stream=None):
     cp = p.c()
     _check(lib().landmarks_pool_bwd(ctypes.byref(cp), _ptr(dL), _ptr(dK), _stream(stream)), "landmarks_pool_bwd")
     return dK
+
+
+def set_overlap(enabled: bool) -> bool:
+    """Whether the per-head kernels run on the library's second stream beside the token-sized ones
+    (default on); returns the previous setting."""
+    return bool(lib().ln_set_overlap(1 if enabled else 0))
 
 
 # ------------------------------------------------------------------------------------------ profiling aid

@@ -6,6 +6,7 @@
 #include "../../include/laplace_nystrom.h"
 #include "ln_kernels.cuh"
 #include "ln_sign2.cuh"
+#include <mutex>
 #include <type_traits>
 
 using namespace ln;
@@ -32,6 +33,8 @@ struct Plan {
   int BH, n, d, m, T, ldm, rpc, chunks;
   long long hslot;                   // floats per slot of the Newton-Schulz histories
   int s2_tg, s2_rpc, s2_chunks;      // fused sign pass: token groups per tile, tokens per chunk, chunks (0 = not used)
+  int s2q_rpc, s2q_chunks;           // the same for the query-side pass, which shares the GPU with the per-head kernel
+  int mid_sms;                       // SMs the per-head kernels occupy (Newton-Schulz and its adjoint)
   size_t s2_smem;
 };
 
@@ -55,7 +58,9 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   pl->rpc = rpc;
   pl->chunks = (p->n + rpc - 1) / rpc;
   // fused sign pass (64-dim slabs): token tiles of 8 * TG tokens that hug n, chunks for about three waves
-  pl->s2_tg = pl->s2_rpc = pl->s2_chunks = 0; pl->s2_smem = 0;
+  pl->s2_tg = pl->s2_rpc = pl->s2_chunks = pl->s2q_rpc = pl->s2q_chunks = 0; pl->s2_smem = 0;
+  // per-head kernels (bf16 storage): three CTAs per SM for m <= 64, one for m <= 128, else clusters of four CTAs, two per SM
+  pl->mid_sms = p->m <= 64 ? (pl->BH + 2) / 3 : (p->m <= 128 ? pl->BH : 2 * pl->BH);
   if (p->d % 64 == 0) {
     const int groups = (p->n + 7) / 8;
     int tiles = (groups + S2_TGMAX - 1) / S2_TGMAX;
@@ -64,16 +69,28 @@ bool make_plan(const ln_problem* p, Plan* pl) {
     const int slabs = p->d / 64;
     // tiles per chunk: the choice that minimises waves x (time of a CTA), with a CTA's time counted in rounds of 8
     // landmarks plus about three rounds of fixed cost, two CTAs per SM, at most 64 chunks
-    const int nrounds = (p->m + S2_RL - 1) / S2_RL, slots = 2 * kSMs;
-    int tpc = tiles; long long best = -1;
-    for (int t = 1; t <= tiles; ++t) {
-      const int chunks = (tiles + t - 1) / t;
-      if (chunks > 64) continue;
-      const long long ctas = (long long)pl->BH * slabs * chunks;
-      const long long cost = ((ctas + slots - 1) / slots) * ((long long)t * nrounds + 3);
-      if (best < 0 || cost < best) { best = cost; tpc = t; }
-    }
+    const int nrounds = (p->m + S2_RL - 1) / S2_RL;
+    auto tiles_per_chunk = [&](int slots) {
+      int tpc = tiles; long long best = -1;
+      for (int t = 1; t <= tiles; ++t) {
+        const int chunks = (tiles + t - 1) / t;
+        if (chunks > 64) continue;
+        const long long ctas = (long long)pl->BH * slabs * chunks;
+        const long long cost = ((ctas + slots - 1) / slots) * ((long long)t * nrounds + 3);
+        if (best < 0 || cost < best) { best = cost; tpc = t; }
+      }
+      return tpc;
+    };
+    const int tpc = tiles_per_chunk(2 * kSMs);
     pl->s2_tg = TG; pl->s2_rpc = tpc * 8 * TG; pl->s2_chunks = (p->n + pl->s2_rpc - 1) / pl->s2_rpc;
+    // The query-side pass runs beside the Newton-Schulz adjoint (one CTA per head on the library's second stream).
+    // While that kernel lives, every SM that holds one of its CTAs has one place less for a CTA of the sign pass (both
+    // places for 64 < m <= 128, whose CTA fills an SM).  With few heads the pass is planned for the places that are
+    // left; with many heads the two kernels take turns anyway and the plan is that of the pass running alone.
+    int lost = p->m <= 64 ? pl->BH : (p->m <= 128 ? 2 * pl->BH : 4 * pl->BH);
+    if (p->dtype != LN_BF16 || lost > kSMs) lost = 0;
+    const int tpq = tiles_per_chunk(2 * kSMs - lost);
+    pl->s2q_rpc = tpq * 8 * TG; pl->s2q_chunks = (p->n + pl->s2q_rpc - 1) / pl->s2q_rpc;
     pl->s2_smem = sign2_smem_bytes(p->m);
   }
   return true;
@@ -123,10 +140,11 @@ BwdWs carve_bwd_ws(const Plan& pl, void* base) {
   Carver c(base); BwdWs w;
   const size_t BH = pl.BH, n = pl.n, d = pl.d, m = pl.m, ch = pl.chunks;
   const size_t chs = pl.s2_chunks > 0 ? (size_t)pl.s2_chunks : ch;     // chunks of the landmark-gradient partials
+  const size_t chq = pl.s2_chunks > 0 ? (size_t)pl.s2q_chunks : ch;
   w.G = c.take(BH * n * pl.ldm);
   w.dYtpart = c.take(BH * ch * m * d);
   w.dybpart = c.take(BH * ch * d);
-  w.dLCpart = c.take(BH * chs * m * d);
+  w.dLCpart = c.take(BH * chq * m * d);
   w.dLRpart = c.take(BH * chs * m * d);
   w.dY = c.take(BH * m * d);
   w.dM = c.take(BH * m * d);
@@ -201,6 +219,49 @@ struct TraceScope {
   ~TraceScope() { if (slot >= 0) cudaEventRecord(g_trace.ev[2 * slot + 1], st); }
 };
 #define LN_LAUNCH(name, st, ...) do { TraceScope ts_(name, st); __VA_ARGS__; } while (0)
+
+// Side stream.  The per-head kernels (Newton-Schulz and its adjoint: one CTA or cluster per head, bound by the
+// latency of a chain of small products) do not depend on the token-sized kernels next to them, so the entry
+// points enqueue them on a second stream of the library, forked from and joined back into the caller's stream
+// with events: to the caller everything is still ordered on the stream it passed.  One stream and a ring of
+// events per device, created at the first call on that device.  Switched off while a trace is recorded (so that
+// the per-launch times are those of kernels running alone) and by ln_set_overlap(0).
+constexpr int kSideDevices = 64, kSideEvents = 16;
+struct SideState { bool tried = false, ok = false; cudaStream_t s = nullptr; cudaEvent_t ev[kSideEvents]; unsigned next = 0; };
+SideState g_side[kSideDevices];
+std::mutex g_side_mu;
+bool g_overlap = true;
+struct Side {
+  cudaStream_t s = nullptr; cudaEvent_t fork_ev = nullptr, join_ev = nullptr;
+  bool on() const { return s != nullptr; }
+  // everything enqueued on `st` so far precedes what is enqueued on the side stream from now on
+  void fork(cudaStream_t st) const { cudaEventRecord(fork_ev, st); cudaStreamWaitEvent(s, fork_ev, 0); }
+  // everything enqueued on the side stream so far precedes what is enqueued on `st` from now on
+  void join(cudaStream_t st) const { cudaEventRecord(join_ev, s); cudaStreamWaitEvent(st, join_ev, 0); }
+};
+Side side_acquire(bool want) {
+  Side r;
+  if (!want || !g_overlap || g_trace.on) return r;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kSideDevices) return r;
+  std::lock_guard<std::mutex> lk(g_side_mu);
+  SideState& d = g_side[dev];
+  if (!d.tried) {
+    d.tried = true;
+    // highest priority: its few large CTAs (up to a whole SM each) are placed before the pending small CTAs of
+    // the kernels on the caller's stream, which would otherwise keep every SM partly occupied until their grids end
+    int prio_lo = 0, prio_hi = 0;
+    bool ok = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithPriority(&d.s, cudaStreamNonBlocking, prio_hi) == cudaSuccess;
+    for (int i = 0; ok && i < kSideEvents; ++i) ok = cudaEventCreateWithFlags(&d.ev[i], cudaEventDisableTiming) == cudaSuccess;
+    d.ok = ok;
+    if (!ok) cudaGetLastError();
+  }
+  if (!d.ok) return r;
+  r.s = d.s; r.fork_ev = d.ev[d.next]; r.join_ev = d.ev[d.next + 1];
+  d.next = (d.next + 2) % kSideEvents;
+  return r;
+}
 
 // Tile of the l1 kernel for a problem: LG landmark groups of QN (4 or 2) landmarks, TG token groups of 8,
 // LG * TG <= 256 threads, chosen so that the tiles hug the problem.  Small heads (few pairs per CTA) take
@@ -281,37 +342,55 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     LN_LAUNCH("k_to_f32", st, k_to_f32<T><<<cdiv(cnt, 256), 256, 0, st>>>(L, x.Lf, cnt));
   }
   // the three kernel blocks: C = k(Q,L) with its row sums, R^T = k(K,L), W = k(L,L)
-  {
-    L1Args a;
-    a.p[0] = l1_prob(Q, is_f32<T>(), x.C, p->map_mode == 1 ? x.mu : nullptr, n, D, pl.ldm, 1.f / (float)m);  // row means (Prop. 3 step 2)
-    a.p[1] = l1_prob(K, is_f32<T>(), x.Rt, nullptr, n, D, pl.ldm, 1.f);
-    a.p[2] = l1_prob(x.Lf, 1, x.W, nullptr, m, D, m, 1.f);
-    a.Bm = x.Lf; a.sB = (long long)m * D; a.nb = m; a.d = D; a.b_f32 = 1;
-    a.nscale = -1.4426950408889634f / p->lambda;
-    launch_l1_args("l1_CRW", a, 3, BH, st);
-  }
-  // M = R V, partial over token chunks (a single chunk writes M itself)
-  float* const Mdst = pl.chunks == 1 ? x.M : w.Mpart;
-  const int Mparts = pl.chunks == 1 ? 0 : pl.chunks;
-  if constexpr (std::is_same<T, bf16>::value)
-    LN_LAUNCH("tn_M", st, k_tn_mma<D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
-  else
-    LN_LAUNCH("tn_M", st, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
-  // Newton-Schulz, Y = X M, folded map
+  // (only where the per-head kernel leaves at least half of the SMs to the others: with more heads the two halves of
+  // the split launch cost more than the overlap returns)
+  const Side side = side_acquire(std::is_same<T, bf16>::value && 2 * pl.mid_sms <= kSMs);
   const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);   // tcgen05 products over the landmarks
-  {
+  const float* const Mparts_src = w.Mpart;
+  const int Mparts = pl.chunks == 1 ? 0 : pl.chunks;
+  // Newton-Schulz (phase bit 0) and Y = X M with the folded map (phase bit 1), one CTA or cluster per head
+  auto launch_mid = [&](cudaStream_t s, int phase) {
     constexpr bool TC = std::is_same<T, bf16>::value;
     auto launch = [&](auto kern, size_t smem, int cl = 1) {
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      LN_LAUNCH("k_mid_fwd", st, launch_clustered(kern, BH * cl, cl, smem, st, m, pl.ldm, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode,
-                                                  p->whiten, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, w.Mpart, Mparts, x.M, w.Y, x.Yt,
-                                                  x.ybar, dev_status, pl.hslot, umma_prod ? reinterpret_cast<bf16*>(x.Yimg) : nullptr));
+      LN_LAUNCH(phase == 3 ? "k_mid_fwd" : (phase == 1 ? "k_mid_fwd_ns" : "k_mid_fwd_y"), s,
+                launch_clustered(kern, BH * cl, cl, smem, s, m, pl.ldm, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode,
+                                 p->whiten, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, Mparts_src, Mparts, x.M, w.Y, x.Yt,
+                                 x.ybar, dev_status, pl.hslot, umma_prod ? reinterpret_cast<bf16*>(x.Yimg) : nullptr, phase));
     };
     if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * NsTile<64>::mat_bytes);
     else if (TC && m <= 128) launch(k_mid_fwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
     else if (TC) launch(k_mid_fwd<D, TC, 0, TC ? kMidCluster : 1>, sizeof(NsSmem), kMidCluster);   // m > 128: a cluster per head
     else launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));
+  };
+  {
+    L1Args a;
+    a.Bm = x.Lf; a.sB = (long long)m * D; a.nb = m; a.d = D; a.b_f32 = 1;
+    a.nscale = -1.4426950408889634f / p->lambda;
+    const L1Prob pc = l1_prob(Q, is_f32<T>(), x.C, p->map_mode == 1 ? x.mu : nullptr, n, D, pl.ldm, 1.f / (float)m);  // row means (Prop. 3 step 2)
+    const L1Prob pr = l1_prob(K, is_f32<T>(), x.Rt, nullptr, n, D, pl.ldm, 1.f);
+    const L1Prob pw = l1_prob(x.Lf, 1, x.W, nullptr, m, D, m, 1.f);
+    if (side.on()) {       // W first; the iteration on it then runs beside the token-sized blocks and M = R V
+      a.p[0] = pw; a.p[1] = pw; a.p[2] = pw;
+      launch_l1_args("l1_W", a, 1, BH, st);
+      side.fork(st);
+      launch_mid(side.s, 1);
+      a.p[0] = pc; a.p[1] = pr; a.p[2] = pr;
+      launch_l1_args("l1_CR", a, 2, BH, st);
+    } else {
+      a.p[0] = pc; a.p[1] = pr; a.p[2] = pw;
+      launch_l1_args("l1_CRW", a, 3, BH, st);
+    }
   }
+  // M = R V, partial over token chunks (a single chunk writes M itself)
+  float* const Mdst = pl.chunks == 1 ? x.M : w.Mpart;
+  if constexpr (std::is_same<T, bf16>::value)
+    LN_LAUNCH("tn_M", st, k_tn_mma<D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
+  else
+    LN_LAUNCH("tn_M", st, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
+  // Newton-Schulz, Y = X M, folded map
+  if (side.on()) { side.join(st); launch_mid(st, 2); }
+  else launch_mid(st, 3);
   // O = (C - mu) Ytilde + ybar
   if constexpr (std::is_same<T, bf16>::value && (D == 64 || D == 128)) {
     const size_t smem = nn_umma_smem<D>();
@@ -347,10 +426,31 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   }
   const bool fused_sign = pl.s2_chunks > 0;
   const int chs = fused_sign ? pl.s2_chunks : ch;
+  const int chq = fused_sign ? pl.s2q_chunks : ch;    // chunks of the query-side landmark-gradient partials
+  // The per-head kernel and the landmark-block sign pass need Z'^T dO only: with a side stream they run beside
+  // the query-side kernels and are joined before the key side, which needs dM.
+  const Side side = side_acquire(std::is_same<T, bf16>::value);
+  const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);
+  auto launch_mid = [&](cudaStream_t s) {
+    constexpr bool TC = std::is_same<T, bf16>::value;
+    auto launch = [&](auto kern, size_t smem, int cl = 1) {
+      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      LN_LAUNCH("k_mid_bwd", s, launch_clustered(kern, BH * cl, cl, smem, s, m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten,
+                                                 x.W, x.Xh, x.Ph, x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P,
+                                                 w.Hm, w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot,
+                                                 umma_prod ? reinterpret_cast<bf16*>(w.dMimg) : nullptr));
+    };
+    if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 4 * NsTile<64>::mat_bytes);
+    else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
+    else if (TC) launch(k_mid_bwd<D, TC, 0, TC ? kMidCluster : 1>, sizeof(NsSmem), kMidCluster);
+    else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
+    LN_LAUNCH("sign_rows_dLW", s, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, s>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));
+  };
+  if (side.on()) { side.fork(st); launch_mid(side.s); }
   if (fused_sign) {
     auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.s2_smem);
-      LN_LAUNCH(name, st, kern<<<dim3(chs, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(tokp, x.Lf, w.G, pl.ldm, rowsp, partp, n, m, D, pl.s2_rpc));
+      LN_LAUNCH(name, st, kern<<<dim3(chq, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(tokp, x.Lf, w.G, pl.ldm, rowsp, partp, n, m, D, pl.s2q_rpc));
     };
     if (pl.s2_tg == S2_TGMAX) launch2("sign2_dQ_dLC", k_sign2<T, T, 1>, Q, dQ, w.dLCpart);
     else launch2("sign2_dQ_dLC", k_sign2<T, T, 2>, Q, dQ, w.dLCpart);
@@ -358,23 +458,9 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m));
     LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
   }
-  // per head: dY, dX, dM, Newton-Schulz adjoint, symmetrised landmark-block upstream
-  const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);
-  {
-    constexpr bool TC = std::is_same<T, bf16>::value;
-    auto launch = [&](auto kern, size_t smem, int cl = 1) {
-      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      LN_LAUNCH("k_mid_bwd", st, launch_clustered(kern, BH * cl, cl, smem, st, m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten,
-                                                  x.W, x.Xh, x.Ph, x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P,
-                                                  w.Hm, w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot,
-                                                  umma_prod ? reinterpret_cast<bf16*>(w.dMimg) : nullptr));
-    };
-    if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 4 * NsTile<64>::mat_bytes);
-    else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
-    else if (TC) launch(k_mid_bwd<D, TC, 0, TC ? kMidCluster : 1>, sizeof(NsSmem), kMidCluster);
-    else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
-  }
-  LN_LAUNCH("sign_rows_dLW", st, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, st>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));
+  // per head: dY, dX, dM, Newton-Schulz adjoint, symmetrised landmark-block upstream; landmark-block sign pass
+  if (side.on()) side.join(st);
+  else launch_mid(st);
   // key side: g^R = (V dM^T) o R^T / lambda; dV = R^T dM; dK (kernel part); landmark part
   if constexpr (std::is_same<T, bf16>::value) {
     if constexpr (D == 64 || D == 128)
@@ -407,10 +493,10 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // landmark gradient and its way back to the keys
   const int md = m * D;
   if (p->lm_mode == 1) {
-    LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chs, w.dLRpart, chs, w.dLW, 1, w.dLtot, md));
+    LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, w.dLtot, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, w.dLtot, dK, geom_of(p), 1));
   } else {
-    LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chs, w.dLRpart, chs, w.dLW, 1, dL, md));
+    LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, dL, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, nullptr, dK, geom_of(p), 0));
   }
   return launch_ok();
@@ -502,6 +588,13 @@ int ln_trace_end(int32_t capacity, int32_t* count, float* ms, const char** names
   }
   for (int i = 0; i < 2 * kTraceCap; ++i) cudaEventDestroy(g_trace.ev[i]);
   return status;
+}
+
+int ln_set_overlap(int enabled) {
+  std::lock_guard<std::mutex> lk(g_side_mu);
+  const int before = g_overlap ? 1 : 0;
+  g_overlap = enabled != 0;
+  return before;
 }
 
 const char* ln_status_string(int s) {

@@ -924,7 +924,10 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_fw
                                                  const float* __restrict__ whiten, const float* W, float* Wr,
                                                  float* P, float* Xh, float* Ph, NsHdr* hdr, const float* Mpart, int nchunks,
                                                  float* Mout, float* Y, float* Yt, float* ybar, int* dev_status,
-                                                 long long hslot, bf16* Yimg) {
+                                                 long long hslot, bf16* Yimg, int phase) {
+  // phase: bit 0 = Newton-Schulz (needs W only), bit 1 = everything that needs M (sum of the partials, Y, map fold).
+  // The two halves may run as two launches, the first beside the kernels that produce M; X_T passes through
+  // global memory either way.
   // Yimg: NULL, or where Ytilde is also left as split operand images per 64-landmark block (for the tcgen05 product)
   // hslot: floats per slot of the iterate histories (used by the MP = 64 path, whose slots hold operand images)
   // dynamic shared memory: the Newton-Schulz matrices (MP > 0), reused afterwards by the GEMM engine
@@ -941,9 +944,11 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_fw
   if (Ph) Ph += (long long)bh * T * mx;
   Mout += bh * md; Y += bh * md; Yt += bh * md; ybar += (long long)bh * D;
   Mpart += (long long)bh * nchunks * md;
-  if (nchunks > 0)                               // nchunks == 0: the single partial result was written to Mout directly
+  if ((phase & 2) && nchunks > 0)                // nchunks == 0: the single partial result was written to Mout directly
     for (long long e = (long long)gt * 4; e < md; e += 4 * gn)
       *reinterpret_cast<float4*>(Mout + e) = sum_parts4(Mpart, nchunks, md, e);
+  const float* XT = Xh + (long long)T * mx;
+  if (phase & 1) {
   bool tc_ok = true;
   float bad = 0.f;                               // non-finite entries of X_T seen by this thread
   if constexpr (MP == 128) {        // tcgen05 + TMEM
@@ -956,13 +961,15 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_fw
   } else {
     ns_forward_dev<TC, CL>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red, crank);
   }
-  const float* XT = Xh + (long long)T * mx;
   if (dev_status) {
     if constexpr (MP == 0)
       for (int e = tid; e < m * m; e += 256) bad += isfinite(XT[(long long)(e / m) * ldx + e % m]) ? 0.f : 1.f;
     bad = block_sum(bad, red);
     if (tid == 0 && crank == 0) atomicOr(dev_status + bh, (bad > 0.f ? 1 : 0) | (tc_ok ? 0 : 2));   // bit1: a bounded tensor-core wait ran out
   }
+  }
+  if (!(phase & 2)) return;
+  if (!(phase & 1)) phase_sync<CL>();             // the M sums of all threads that share the head
   ns_gemm<TC, false, false>(m, D, m, XT, ldx, Mout, D, Y, D, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // Y = X M
   if (CL > 1) phase_sync<CL>();
   const float* s = whiten ? whiten + (long long)(bh % H) * m : nullptr;

@@ -250,6 +250,25 @@ def test_runs_twice_bit_identical():
         assert torch.equal(a[k], b[k]), k
 
 
+@pytest.mark.parametrize("name,B", [("cfg2", 8), ("cfg3", 2), ("cfg4a", 1), ("cfg5_m128_T8", 1), ("cfg5_m256_T4", 1)])
+def test_overlap_on_the_side_stream_changes_no_bit(name, B):
+    """With the per-head kernels on the library's second stream (the default) the results are the bits of
+    the single-stream order, call after call: the fork and join events order every producer before its consumers."""
+    cfg = synth.shrink(synth.CONFIGS[name], B=B)
+    inp = synth.make_inputs(cfg)
+    before = ln.set_overlap(False)
+    try:
+        ref = run_gpu(cfg, inp)
+        ln.set_overlap(True)
+        for _ in range(3):
+            got = run_gpu(cfg, inp)
+            for k in ("O", "dQ", "dK", "dV"):
+                assert torch.equal(ref[k], got[k]), (name, k)
+            assert int(got["status"].abs().max()) == 0
+    finally:
+        ln.set_overlap(before)
+
+
 def test_singular_landmarks_are_flagged_finite():
     # all keys identical -> K_LL is all ones; the ridge keeps Newton-Schulz finite
     cfg = synth.shrink(synth.CONFIGS["cfg1"], H=1)
