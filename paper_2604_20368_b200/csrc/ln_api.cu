@@ -133,7 +133,7 @@ FwdWs carve_fwd_ws(const Plan& pl, void* base) {
 }
 
 struct BwdWs {
-  float *G, *dYtpart, *dybpart, *dLCpart, *dLRpart, *dY, *dM, *Wr, *P, *Hm, *Ga, *Gb, *dW, *dX, *GW, *dLW, *dLtot, *dKpart, *dMimg;
+  float *G, *G2, *dYtpart, *dybpart, *dLCpart, *dLRpart, *dY, *dM, *Wr, *P, *Hm, *Ga, *Gb, *dW, *dX, *GW, *dLW, *dLtot, *dKpart, *dMimg;
   size_t bytes;
 };
 BwdWs carve_bwd_ws(const Plan& pl, void* base) {
@@ -142,6 +142,7 @@ BwdWs carve_bwd_ws(const Plan& pl, void* base) {
   const size_t chs = pl.s2_chunks > 0 ? (size_t)pl.s2_chunks : ch;     // chunks of the landmark-gradient partials
   const size_t chq = pl.s2_chunks > 0 ? (size_t)pl.s2q_chunks : ch;
   w.G = c.take(BH * n * pl.ldm);
+  w.G2 = c.take(BH * n * pl.ldm);       // upstream of the key-side block (its own buffer: it is formed while the query side reads G)
   w.dYtpart = c.take(BH * ch * m * d);
   w.dybpart = c.take(BH * ch * d);
   w.dLCpart = c.take(BH * chq * m * d);
@@ -232,10 +233,10 @@ SideState g_side[kSideDevices];
 std::mutex g_side_mu;
 bool g_overlap = true;
 struct Side {
-  cudaStream_t s = nullptr; cudaEvent_t fork_ev = nullptr, join_ev = nullptr;
+  cudaStream_t s = nullptr; cudaEvent_t fork_ev[2] = {nullptr, nullptr}, join_ev = nullptr;
   bool on() const { return s != nullptr; }
-  // everything enqueued on `st` so far precedes what is enqueued on the side stream from now on
-  void fork(cudaStream_t st) const { cudaEventRecord(fork_ev, st); cudaStreamWaitEvent(s, fork_ev, 0); }
+  // everything enqueued on `st` so far precedes what is enqueued on the side stream from now on (k-th fork of a call)
+  void fork(cudaStream_t st, int k = 0) const { cudaEventRecord(fork_ev[k], st); cudaStreamWaitEvent(s, fork_ev[k], 0); }
   // everything enqueued on the side stream so far precedes what is enqueued on `st` from now on
   void join(cudaStream_t st) const { cudaEventRecord(join_ev, s); cudaStreamWaitEvent(st, join_ev, 0); }
 };
@@ -258,8 +259,8 @@ Side side_acquire(bool want) {
     if (!ok) cudaGetLastError();
   }
   if (!d.ok) return r;
-  r.s = d.s; r.fork_ev = d.ev[d.next]; r.join_ev = d.ev[d.next + 1];
-  d.next = (d.next + 2) % kSideEvents;
+  r.s = d.s; r.fork_ev[0] = d.ev[d.next]; r.fork_ev[1] = d.ev[d.next + 1]; r.join_ev = d.ev[d.next + 2];
+  d.next = (d.next + 4) % kSideEvents;
   return r;
 }
 
@@ -342,9 +343,9 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     LN_LAUNCH("k_to_f32", st, k_to_f32<T><<<cdiv(cnt, 256), 256, 0, st>>>(L, x.Lf, cnt));
   }
   // the three kernel blocks: C = k(Q,L) with its row sums, R^T = k(K,L), W = k(L,L)
-  // (only where the per-head kernel leaves at least half of the SMs to the others: with more heads the two halves of
-  // the split launch cost more than the overlap returns)
-  const Side side = side_acquire(std::is_same<T, bf16>::value && 2 * pl.mid_sms <= kSMs);
+  // (not for many small heads, where the per-head kernel fills the GPU and the split launches cost more than the
+  // overlap returns)
+  const Side side = side_acquire(std::is_same<T, bf16>::value && (2 * pl.mid_sms <= kSMs || (long long)n * m * D > (1ll << 22)));
   const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);   // tcgen05 products over the landmarks
   const float* const Mparts_src = w.Mpart;
   const int Mparts = pl.chunks == 1 ? 0 : pl.chunks;
@@ -370,13 +371,16 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     const L1Prob pc = l1_prob(Q, is_f32<T>(), x.C, p->map_mode == 1 ? x.mu : nullptr, n, D, pl.ldm, 1.f / (float)m);  // row means (Prop. 3 step 2)
     const L1Prob pr = l1_prob(K, is_f32<T>(), x.Rt, nullptr, n, D, pl.ldm, 1.f);
     const L1Prob pw = l1_prob(x.Lf, 1, x.W, nullptr, m, D, m, 1.f);
-    if (side.on()) {       // W first; the iteration on it then runs beside the token-sized blocks and M = R V
+    if (side.on()) {
+      // W first: the iteration on it runs beside the token-sized blocks.  Then R^T: M = R V (bound by memory) and the
+      // rest of the per-head work run beside the query block C (bound by arithmetic), which only the last product needs.
       a.p[0] = pw; a.p[1] = pw; a.p[2] = pw;
       launch_l1_args("l1_W", a, 1, BH, st);
-      side.fork(st);
+      side.fork(st, 0);
       launch_mid(side.s, 1);
-      a.p[0] = pc; a.p[1] = pr; a.p[2] = pr;
-      launch_l1_args("l1_CR", a, 2, BH, st);
+      a.p[0] = pr; a.p[1] = pr; a.p[2] = pr;
+      launch_l1_args("l1_R", a, 1, BH, st);
+      side.fork(st, 1);
     } else {
       a.p[0] = pc; a.p[1] = pr; a.p[2] = pw;
       launch_l1_args("l1_CRW", a, 3, BH, st);
@@ -384,13 +388,22 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   }
   // M = R V, partial over token chunks (a single chunk writes M itself)
   float* const Mdst = pl.chunks == 1 ? x.M : w.Mpart;
+  const cudaStream_t sm_ = side.on() ? side.s : st;          // stream of M = R V and of what follows from it
   if constexpr (std::is_same<T, bf16>::value)
-    LN_LAUNCH("tn_M", st, k_tn_mma<D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
+    LN_LAUNCH("tn_M", sm_, k_tn_mma<D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, sm_>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
   else
-    LN_LAUNCH("tn_M", st, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
+    LN_LAUNCH("tn_M", sm_, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, sm_>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
   // Newton-Schulz, Y = X M, folded map
-  if (side.on()) { side.join(st); launch_mid(st, 2); }
-  else launch_mid(st, 3);
+  if (side.on()) {
+    launch_mid(side.s, 2);
+    L1Args a;
+    a.Bm = x.Lf; a.sB = (long long)m * D; a.nb = m; a.d = D; a.b_f32 = 1;
+    a.nscale = -1.4426950408889634f / p->lambda;
+    a.p[0] = l1_prob(Q, is_f32<T>(), x.C, p->map_mode == 1 ? x.mu : nullptr, n, D, pl.ldm, 1.f / (float)m);
+    a.p[1] = a.p[0]; a.p[2] = a.p[0];
+    launch_l1_args("l1_C", a, 1, BH, st);
+    side.join(st);
+  } else launch_mid(st, 3);
   // O = (C - mu) Ytilde + ybar
   if constexpr (std::is_same<T, bf16>::value && (D == 64 || D == 128)) {
     const size_t smem = nn_umma_smem<D>();
@@ -446,7 +459,29 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
     LN_LAUNCH("sign_rows_dLW", s, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, s>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));
   };
-  if (side.on()) { side.fork(st); launch_mid(side.s); }
+  // key-side products: g^R = (V dM^T) o R^T / lambda and dV = R^T dM (they need dM from the per-head kernel)
+  auto launch_key_products = [&](cudaStream_t s) {
+    if constexpr (std::is_same<T, bf16>::value) {
+      if constexpr (D == 64 || D == 128)
+        LN_LAUNCH("ntg_R", s, k_ntg_umma<D><<<dim3(cdiv(n, 128), BH), 256, ntg_umma_smem<D>(), s>>>(V, reinterpret_cast<const bf16*>(w.dMimg), x.Rt, pl.ldm,
+                                                                                                w.G2, n, m, inv_lambda, dev_status));
+      else
+        LN_LAUNCH("ntg_R", s, k_nt_g_mma<D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, s>>>(V, w.dM, x.Rt, pl.ldm, w.G2, n, m, inv_lambda));
+      if constexpr (D == 64 || D == 128) {
+        const size_t smem = nn_umma_smem<D>();
+        cudaFuncSetAttribute(k_nn_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        LN_LAUNCH("nn_dV", s, k_nn_umma<D><<<dim3(cdiv(n, 128), BH), 256, smem, s>>>(x.Rt, pl.ldm, nullptr, reinterpret_cast<const bf16*>(w.dMimg),
+                                                                                 nullptr, dV, n, m, dev_status));
+      } else
+        LN_LAUNCH("nn_dV", s, k_nn_mma<D><<<dim3(cdiv(n, 64), BH), 256, 0, s>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
+    } else {
+      LN_LAUNCH("ntg_R", s, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, s>>>(V, w.dM, x.Rt, pl.ldm, w.G2, n, m, inv_lambda));
+      LN_LAUNCH("nn_dV", s, k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, s>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
+    }
+  };
+  // side stream: per-head kernel, landmark-block sign pass and the key-side products (bound by latency and by memory)
+  // run beside the query-side sign pass (bound by arithmetic)
+  if (side.on()) { side.fork(st); launch_mid(side.s); launch_key_products(side.s); }
   if (fused_sign) {
     auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.s2_smem);
@@ -458,37 +493,19 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m));
     LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
   }
-  // per head: dY, dX, dM, Newton-Schulz adjoint, symmetrised landmark-block upstream; landmark-block sign pass
   if (side.on()) side.join(st);
-  else launch_mid(st);
-  // key side: g^R = (V dM^T) o R^T / lambda; dV = R^T dM; dK (kernel part); landmark part
-  if constexpr (std::is_same<T, bf16>::value) {
-    if constexpr (D == 64 || D == 128)
-      LN_LAUNCH("ntg_R", st, k_ntg_umma<D><<<dim3(cdiv(n, 128), BH), 256, ntg_umma_smem<D>(), st>>>(V, reinterpret_cast<const bf16*>(w.dMimg), x.Rt, pl.ldm,
-                                                                                                w.G, n, m, inv_lambda, dev_status));
-    else
-    LN_LAUNCH("ntg_R", st, k_nt_g_mma<D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(V, w.dM, x.Rt, pl.ldm, w.G, n, m, inv_lambda));
-    if constexpr (D == 64 || D == 128) {
-      const size_t smem = nn_umma_smem<D>();
-      cudaFuncSetAttribute(k_nn_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      LN_LAUNCH("nn_dV", st, k_nn_umma<D><<<dim3(cdiv(n, 128), BH), 256, smem, st>>>(x.Rt, pl.ldm, nullptr, reinterpret_cast<const bf16*>(w.dMimg),
-                                                                                 nullptr, dV, n, m, dev_status));
-    } else
-    LN_LAUNCH("nn_dV", st, k_nn_mma<D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
-  } else {
-    LN_LAUNCH("ntg_R", st, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(V, w.dM, x.Rt, pl.ldm, w.G, n, m, inv_lambda));
-    LN_LAUNCH("nn_dV", st, k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
-  }
+  else { launch_mid(st); launch_key_products(st); }
+  // key side: dK (kernel part); landmark part
   if (fused_sign) {
     auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.s2_smem);
-      LN_LAUNCH(name, st, kern<<<dim3(chs, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(tokp, x.Lf, w.G, pl.ldm, rowsp, partp, n, m, D, pl.s2_rpc));
+      LN_LAUNCH(name, st, kern<<<dim3(chs, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(tokp, x.Lf, w.G2, pl.ldm, rowsp, partp, n, m, D, pl.s2_rpc));
     };
     if (pl.s2_tg == S2_TGMAX) launch2("sign2_dK_dLR", k_sign2<T, float, 1>, K, w.dKpart, w.dLRpart);
     else launch2("sign2_dK_dLR", k_sign2<T, float, 2>, K, w.dKpart, w.dLRpart);
   } else {
-    LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dKpart, n, m));
-    LN_LAUNCH("sign_cols_dLR", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(K, x.Lf, w.G, pl.ldm, w.dLRpart, n, m, pl.rpc));
+    LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G2, pl.ldm, w.dKpart, n, m));
+    LN_LAUNCH("sign_cols_dLR", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(K, x.Lf, w.G2, pl.ldm, w.dLRpart, n, m, pl.rpc));
   }
   // landmark gradient and its way back to the keys
   const int md = m * D;
