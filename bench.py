@@ -282,9 +282,10 @@ def run_ours(args):
     value = tokens * args.steps / (ms * 1e-3)
 
     # ---- end to end through the host-buffer entry point of the C ABI: every step copies Q, K, V, dO from pinned
-    # host memory, runs forward + backward, and copies O, dQ, dK, dV back to pinned host memory.  Two sets of
-    # device buffers on two streams, so that one step's copies overlap the other step's kernels.
-    nslot = 2
+    # host memory, runs forward + backward, and copies O, dQ, dK, dV back to pinned host memory.  Three sets of
+    # device buffers on three streams, so that one step's copies in, another's kernels and a third's copies out overlap
+    # (a step is copy in -> kernels -> copy out on its own stream; PCIe carries both directions at once).
+    nslot = 3
     host_in = {k: inp[k].pin_memory() for k in names}
     host_out = [{k: torch.empty_like(inp["Q"]).pin_memory() for k in ("O", "dQ", "dK", "dV")} for _ in range(nslot)]
     if cfg.backward:
@@ -323,7 +324,7 @@ def run_ours(args):
         for i in range(3):
             step_e2e(i)
         ms_e2e = timed_streams(args.steps)
-        e2e_how = "laplace_nystrom_fwd_bwd_host, pinned host tensors, 2 streams x 2 device buffer sets"
+        e2e_how = f"laplace_nystrom_fwd_bwd_host, pinned host tensors, {nslot} streams x {nslot} device buffer sets"
     else:   # forward-only workload: copies around laplace_nystrom_fwd
         dev_in = {k: torch.empty_like(sets[0][k]) for k in names}
 

@@ -221,6 +221,9 @@ __global__ void __launch_bounds__(256) k_pool_bwd(const float* __restrict__ dKpa
   const int bh = blockIdx.y;
   const unsigned per_row = g.d / 4;
   const unsigned total = (unsigned)g.n * per_row;                  // n * d / 4 < 2^32
+  const bool even = (g.gh % g.mh) == 0 && (g.gw % g.mw) == 0;      // the pooling of Sec. 4.2 proper: r x r windows, stride r
+  const int bh_rows = g.gh / g.mh, bh_cols = g.gw / g.mw;
+  const float even_inv = 1.f / (float)(bh_rows * bh_cols);
   // POOL_EPT elements of four dims per thread, a CTA's share contiguous, so that the bin tables are built once
   // per 1024 elements
 #pragma unroll
@@ -230,7 +233,12 @@ __global__ void __launch_bounds__(256) k_pool_bwd(const float* __restrict__ dKpa
     const int j = (int)(idx / per_row), c = (int)(idx % per_row) * 4;
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
     if (dKpart) v = ld4(dKpart + ((long long)bh * g.n + j) * g.d + c);
-    if (pool && j >= g.prefix) {
+    if (pool && j >= g.prefix && even) {
+      // bins of equal size that do not overlap: one bin per token
+      const int r = (j - g.prefix) / g.gw, q = (j - g.prefix) % g.gw;
+      const float4 t = ld4(dL + ((long long)bh * g.m + (r / bh_rows) * g.mw + q / bh_cols) * g.d + c);
+      v.x += t.x * even_inv; v.y += t.y * even_inv; v.z += t.z * even_inv; v.w += t.w * even_inv;
+    } else if (pool && j >= g.prefix) {
       const int r = (j - g.prefix) / g.gw, q = (j - g.prefix) % g.gw;
       // a token row lies in bin floor(r mh / gh) and, where neighbouring bins overlap, in the next one too
       const int a0 = (int)(((unsigned)r * (unsigned)g.mh) / (unsigned)g.gh), b0 = (int)(((unsigned)q * (unsigned)g.mw) / (unsigned)g.gw);
