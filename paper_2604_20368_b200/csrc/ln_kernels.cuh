@@ -773,7 +773,9 @@ __device__ __forceinline__ void ns_gemm(int M, int N, int K, const float* A, int
 // =====================================================================================
 template <bool TC, int CL = 1>
 __device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const float* W, float* Wr, float* P,
-                               float* Xh, NsHdr* hdr, NsSmem& sm, float* red /* 2*256 + 8 floats */, int crank = 0) {
+                               float* Xh, NsHdr* hdr, NsSmem& sm, float* red /* 2*256 + 8 floats */, int crank = 0,
+                               float* Qh = nullptr) {
+  // Qh: NULL, or a history [T][m][m] that keeps Q_k = 2I - Wr X_k for the adjoint (which then need not form Wr X_k again)
   // CL CTAs of a cluster share the work (crank = this CTA's rank): element-wise phases are strided over all their
   // threads, every product is split by output tiles, small reductions are done by each CTA for itself.
   const int tid = threadIdx.x, gt = crank * 256 + tid, gn = 256 * CL;
@@ -816,9 +818,10 @@ __device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const fl
   for (int k = 0; k < T; ++k) {
     const float* X = Xh + (long long)k * mm;
     float* Xn = Xh + (long long)(k + 1) * mm;
-    ns_gemm<TC, false, false, true>(m, m, m, Wr, m, X, m, P, m, -1.f, 0.f, nullptr, 2.f, sm, crank, CL);   // P = 2I - Wr X_k
+    float* Q = Qh ? Qh + (long long)k * mm : P;
+    ns_gemm<TC, false, false, true>(m, m, m, Wr, m, X, m, Q, m, -1.f, 0.f, nullptr, 2.f, sm, crank, CL);   // Q = 2I - Wr X_k
     if (CL > 1) phase_sync<CL>();
-    ns_gemm<TC, false, false, true>(m, m, m, X, m, P, m, Xn, m, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);    // X_{k+1} = X_k P
+    ns_gemm<TC, false, false, true>(m, m, m, X, m, Q, m, Xn, m, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);    // X_{k+1} = X_k Q
     if (CL > 1) phase_sync<CL>();
   }
 }
@@ -830,7 +833,9 @@ __device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const fl
 template <bool TC, int CL = 1>
 __device__ void ns_backward_dev(int m, int T, const float* Wr, const float* Xh, const NsHdr* hdr,
                                 const float* G0, float* dW, float* P, float* Hm, float* Ga, float* Gb,
-                                NsSmem& sm, float* red, int crank = 0) {
+                                NsSmem& sm, float* red, int crank = 0, const float* Qh = nullptr) {
+  // Qh: NULL, or the history of Q_k = 2I - Wr X_k the forward pass kept: 2G - G (Wr X_k)^T is then G Q_k^T, four
+  // products per step instead of five
   const int tid = threadIdx.x, gt = crank * 256 + tid, gn = 256 * CL;
   const long long mm = (long long)m * m;
   for (long long e = gt; e < mm; e += gn) { Ga[e] = G0[e]; dW[e] = 0.f; }
@@ -838,11 +843,12 @@ __device__ void ns_backward_dev(int m, int T, const float* Wr, const float* Xh, 
   float* G = Ga; float* Gn = Gb;
   for (int k = T - 1; k >= 0; --k) {
     const float* A = Xh + (long long)k * mm;                                        // X_{k+1} = 2A - A P, P = Wr A
-    ns_gemm<TC, false, false, true>(m, m, m, Wr, m, A, m, P, m, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);      // P = Wr A
+    if (!Qh) ns_gemm<TC, false, false, true>(m, m, m, Wr, m, A, m, P, m, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);      // P = Wr A
     ns_gemm<TC, true, false, true>(m, m, m, A, m, G, m, Hm, m, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);       // H = A^T G
     if (CL > 1) phase_sync<CL>();
     ns_gemm<TC, false, true, true>(m, m, m, Hm, m, A, m, dW, m, -1.f, 1.f, dW, 0.f, sm, crank, CL);          // dW -= H A^T
-    ns_gemm<TC, false, true, true>(m, m, m, G, m, P, m, Gn, m, -1.f, 2.f, G, 0.f, sm, crank, CL);            // Gn = 2G - G P^T
+    if (Qh) ns_gemm<TC, false, true, true>(m, m, m, G, m, Qh + (long long)k * mm, m, Gn, m, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // Gn = G Q^T
+    else ns_gemm<TC, false, true, true>(m, m, m, G, m, P, m, Gn, m, -1.f, 2.f, G, 0.f, sm, crank, CL);       // Gn = 2G - G P^T
     ns_gemm<TC, true, false, true>(m, m, m, Wr, m, Hm, m, Gn, m, -1.f, 1.f, Gn, 0.f, sm, crank, CL);         // Gn -= Wr^T H
     if (CL > 1) phase_sync<CL>();
     float* t = G; G = Gn; Gn = t;
@@ -967,7 +973,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_fw
     ns_forward_smem<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, bad);
     __syncthreads();
   } else {
-    ns_forward_dev<TC, CL>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red, crank);
+    ns_forward_dev<TC, CL>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red, crank, Ph);
   }
   if (dev_status) {
     if constexpr (MP == 0)
@@ -1079,7 +1085,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_bw
     const bool tc_ok = ns_backward_umma(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, GW, ldm, inv_lambda, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
     if (dev_status && !tc_ok && tid == 0) atomicOr(dev_status + bh, 2);
   } else if constexpr (MP == 64) ns_backward_smem<MP>(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
-  else { ns_backward_dev<TC, CL>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red, crank); if (CL > 1) phase_sync<CL>(); }
+  else { ns_backward_dev<TC, CL>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red, crank, Ph); if (CL > 1) phase_sync<CL>(); }
   // GW = (dW o K_LL + (dW o K_LL)^T) / lambda; four elements per batch so that the loads overlap
   // (the tcgen05 engine has written GW from shared memory already)
   if constexpr (MP != 128)
