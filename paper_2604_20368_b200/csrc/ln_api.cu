@@ -239,6 +239,10 @@ struct Side {
   void fork(cudaStream_t st, int k = 0) const { cudaEventRecord(fork_ev[k], st); cudaStreamWaitEvent(s, fork_ev[k], 0); }
   // everything enqueued on the side stream so far precedes what is enqueued on `st` from now on
   void join(cudaStream_t st) const { cudaEventRecord(join_ev, s); cudaStreamWaitEvent(st, join_ev, 0); }
+  // a join in two halves (uses the second fork event): mark() notes what the side stream holds so far, join_mark()
+  // makes `st` wait for exactly that, whatever was enqueued on the side stream in between
+  void mark() const { cudaEventRecord(fork_ev[1], s); }
+  void join_mark(cudaStream_t st) const { cudaStreamWaitEvent(st, fork_ev[1], 0); }
 };
 Side side_acquire(bool want) {
   Side r;
@@ -457,16 +461,21 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
     else if (TC) launch(k_mid_bwd<D, TC, 0, TC ? kMidCluster : 1>, sizeof(NsSmem), kMidCluster);
     else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
-    LN_LAUNCH("sign_rows_dLW", s, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, s>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));
   };
   // key-side products: g^R = (V dM^T) o R^T / lambda and dV = R^T dM (they need dM from the per-head kernel)
-  auto launch_key_products = [&](cudaStream_t s) {
+  auto launch_ntg_R = [&](cudaStream_t s) {
     if constexpr (std::is_same<T, bf16>::value) {
       if constexpr (D == 64 || D == 128)
         LN_LAUNCH("ntg_R", s, k_ntg_umma<D><<<dim3(cdiv(n, 128), BH), 256, ntg_umma_smem<D>(), s>>>(V, reinterpret_cast<const bf16*>(w.dMimg), x.Rt, pl.ldm,
                                                                                                 w.G2, n, m, inv_lambda, dev_status));
       else
         LN_LAUNCH("ntg_R", s, k_nt_g_mma<D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, s>>>(V, w.dM, x.Rt, pl.ldm, w.G2, n, m, inv_lambda));
+    } else {
+      LN_LAUNCH("ntg_R", s, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, s>>>(V, w.dM, x.Rt, pl.ldm, w.G2, n, m, inv_lambda));
+    }
+  };
+  auto launch_nn_dV = [&](cudaStream_t s) {
+    if constexpr (std::is_same<T, bf16>::value) {
       if constexpr (D == 64 || D == 128) {
         const size_t smem = nn_umma_smem<D>();
         cudaFuncSetAttribute(k_nn_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -475,13 +484,25 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
       } else
         LN_LAUNCH("nn_dV", s, k_nn_mma<D><<<dim3(cdiv(n, 64), BH), 256, 0, s>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
     } else {
-      LN_LAUNCH("ntg_R", s, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, s>>>(V, w.dM, x.Rt, pl.ldm, w.G2, n, m, inv_lambda));
       LN_LAUNCH("nn_dV", s, k_nn<T, D><<<dim3(cdiv(n, 64), BH), 256, 0, s>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
     }
   };
-  // side stream: per-head kernel, landmark-block sign pass and the key-side products (bound by latency and by memory)
-  // run beside the query-side sign pass (bound by arithmetic)
-  if (side.on()) { side.fork(st); launch_mid(side.s); launch_key_products(side.s); }
+  auto launch_sign_W = [&](cudaStream_t s) {
+    LN_LAUNCH("sign_rows_dLW", s, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, s>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));
+  };
+  // Side stream: the per-head kernel, the landmark-block sign pass and dV (bound by latency and by memory) run beside
+  // the sign passes (bound by arithmetic).  The upstream of the key-side block, which the second sign pass waits for,
+  // joins them where the query-side sign pass is long enough to hide it (large heads); for small heads it follows the
+  // first sign pass on the caller's stream, so that only the per-head kernel stands between the two sign passes.
+  const bool ntg_on_side = side.on() && (long long)n * m * D > (1ll << 22);
+  if (side.on()) {
+    side.fork(st);
+    launch_mid(side.s);
+    if (ntg_on_side) launch_ntg_R(side.s);
+    side.mark();                     // what the second sign pass needs from this stream ends here
+    launch_nn_dV(side.s);
+    launch_sign_W(side.s);
+  }
   if (fused_sign) {
     auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.s2_smem);
@@ -493,8 +514,8 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m));
     LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
   }
-  if (side.on()) side.join(st);
-  else { launch_mid(st); launch_key_products(st); }
+  if (side.on()) { side.join_mark(st); if (!ntg_on_side) launch_ntg_R(st); }
+  else { launch_mid(st); launch_sign_W(st); launch_ntg_R(st); launch_nn_dV(st); }
   // key side: dK (kernel part); landmark part
   if (fused_sign) {
     auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
@@ -508,6 +529,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     LN_LAUNCH("sign_cols_dLR", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(K, x.Lf, w.G2, pl.ldm, w.dLRpart, n, m, pl.rpc));
   }
   // landmark gradient and its way back to the keys
+  if (side.on()) side.join(st);      // dV and the landmark-block part are complete
   const int md = m * D;
   if (p->lm_mode == 1) {
     LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, w.dLtot, md));
