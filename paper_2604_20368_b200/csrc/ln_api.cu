@@ -44,7 +44,7 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   pl->ldm = (p->m + 3) & ~3;
   // history slots: fp32 [m][ldm], except on the m <= 64 tensor-core path, whose slots hold operand images
   pl->hslot = (long long)p->m * pl->ldm;
-  if (p->dtype == LN_BF16 && p->m <= 64 && pl->hslot < (long long)(NsTile<64>::mat_bytes / 4)) pl->hslot = NsTile<64>::mat_bytes / 4;
+  if (p->dtype == LN_BF16 && p->m <= 64) pl->hslot = (long long)(kUmmaMatBytes64 / 4);                 // 16 KiB images >= m * ldm * 4
   if (p->dtype == LN_BF16 && p->m > 64 && p->m <= 128) pl->hslot = (long long)(kUmmaMatBytes / 4);     // 64 KiB images >= m * ldm * 4
   // token chunks per head for the reductions over tokens: about eight waves of CTAs (two per SM) so that
   // the last wave costs little, but at least 64 tokens per chunk
@@ -351,6 +351,12 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // overlap returns)
   const Side side = side_acquire(std::is_same<T, bf16>::value && (2 * pl.mid_sms <= kSMs || (long long)n * m * D > (1ll << 22)));
   const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);   // tcgen05 products over the landmarks
+  // Where the iteration is expected to outlast the two token-sized blocks (few heads of few tokens), only the iteration
+  // goes to the side stream; estimates in microseconds: 5 / 12 / 100 per step for m <= 64 / <= 128 / larger, and the l1
+  // blocks at about half of the FP32 peak
+  const double ns_us = pl.T * (m <= 64 ? 5.0 : (m <= 128 ? 12.0 : 100.0));
+  const double l1_us = 2.0 * 2.0 * n * m * D * BH / 20e6;
+  const bool deep = side.on() && l1_us >= ns_us;
   const float* const Mparts_src = w.Mpart;
   const int Mparts = pl.chunks == 1 ? 0 : pl.chunks;
   // Newton-Schulz (phase bit 0) and Y = X M with the folded map (phase bit 1), one CTA or cluster per head
@@ -363,7 +369,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
                                  p->whiten, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, Mparts_src, Mparts, x.M, w.Y, x.Yt,
                                  x.ybar, dev_status, pl.hslot, umma_prod ? reinterpret_cast<bf16*>(x.Yimg) : nullptr, phase));
     };
-    if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * NsTile<64>::mat_bytes);
+    if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * kUmmaMatBytes64);
     else if (TC && m <= 128) launch(k_mid_fwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
     else if (TC) launch(k_mid_fwd<D, TC, 0, TC ? kMidCluster : 1>, sizeof(NsSmem), kMidCluster);   // m > 128: a cluster per head
     else launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));
@@ -382,9 +388,14 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
       launch_l1_args("l1_W", a, 1, BH, st);
       side.fork(st, 0);
       launch_mid(side.s, 1);
-      a.p[0] = pr; a.p[1] = pr; a.p[2] = pr;
-      launch_l1_args("l1_R", a, 1, BH, st);
-      side.fork(st, 1);
+      if (deep) {
+        a.p[0] = pr; a.p[1] = pr; a.p[2] = pr;
+        launch_l1_args("l1_R", a, 1, BH, st);
+        side.fork(st, 1);
+      } else {
+        a.p[0] = pc; a.p[1] = pr; a.p[2] = pr;
+        launch_l1_args("l1_CR", a, 2, BH, st);
+      }
     } else {
       a.p[0] = pc; a.p[1] = pr; a.p[2] = pw;
       launch_l1_args("l1_CRW", a, 3, BH, st);
@@ -392,13 +403,14 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   }
   // M = R V, partial over token chunks (a single chunk writes M itself)
   float* const Mdst = pl.chunks == 1 ? x.M : w.Mpart;
-  const cudaStream_t sm_ = side.on() ? side.s : st;          // stream of M = R V and of what follows from it
+  const cudaStream_t sm_ = deep ? side.s : st;               // stream of M = R V and of what follows from it
   if constexpr (std::is_same<T, bf16>::value)
     LN_LAUNCH("tn_M", sm_, k_tn_mma<D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, sm_>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
   else
     LN_LAUNCH("tn_M", sm_, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, sm_>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
   // Newton-Schulz, Y = X M, folded map
-  if (side.on()) {
+  if (side.on() && !deep) { side.join(st); launch_mid(st, 2); }
+  else if (side.on()) {
     launch_mid(side.s, 2);
     L1Args a;
     a.Bm = x.Lf; a.sB = (long long)m * D; a.nb = m; a.d = D; a.b_f32 = 1;
@@ -457,7 +469,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
                                                  w.Hm, w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot,
                                                  umma_prod ? reinterpret_cast<bf16*>(w.dMimg) : nullptr));
     };
-    if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 4 * NsTile<64>::mat_bytes);
+    if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 4 * kUmmaMatBytes64);
     else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
     else if (TC) launch(k_mid_bwd<D, TC, 0, TC ? kMidCluster : 1>, sizeof(NsSmem), kMidCluster);
     else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));

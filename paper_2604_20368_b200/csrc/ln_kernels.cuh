@@ -4,7 +4,6 @@
 #pragma once
 #include "ln_common.cuh"
 #include "ln_mma.cuh"
-#include "ln_ns_smem.cuh"
 #include "ln_ns_umma.cuh"
 #include "ln_gemm_umma.cuh"
 
@@ -965,12 +964,9 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_fw
   if (phase & 1) {
   bool tc_ok = true;
   float bad = 0.f;                               // non-finite entries of X_T seen by this thread
-  if constexpr (MP == 128) {        // tcgen05 + TMEM
+  if constexpr (MP == 128 || MP == 64) {        // tcgen05 + TMEM, the matrix padded to MP x MP
     __shared__ UmmaCtl ctl;
-    tc_ok = ns_forward_umma(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl, bad);
-    __syncthreads();
-  } else if constexpr (MP == 64) {  // mma.sync from shared memory
-    ns_forward_smem<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, bad);
+    tc_ok = ns_forward_umma<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl, bad);
     __syncthreads();
   } else {
     ns_forward_dev<TC, CL>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red, crank, Ph);
@@ -1080,15 +1076,14 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_bw
     const int nkb = (m + GU_KB - 1) / GU_KB;
     gu_write_images(dM, dMimg + (long long)bh * nkb * (2 * GU_KB * D), m, D, gt, gn);
   }
-  if constexpr (MP == 128) {
+  if constexpr (MP == 128 || MP == 64) {
     __shared__ UmmaCtl ctl;
-    const bool tc_ok = ns_backward_umma(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, GW, ldm, inv_lambda, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
+    const bool tc_ok = ns_backward_umma<MP>(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, GW, ldm, inv_lambda, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
     if (dev_status && !tc_ok && tid == 0) atomicOr(dev_status + bh, 2);
-  } else if constexpr (MP == 64) ns_backward_smem<MP>(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, dWm, Ga, reinterpret_cast<bf16*>(dyn_smem), red);
-  else { ns_backward_dev<TC, CL>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red, crank, Ph); if (CL > 1) phase_sync<CL>(); }
+  } else { ns_backward_dev<TC, CL>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red, crank, Ph); if (CL > 1) phase_sync<CL>(); }
   // GW = (dW o K_LL + (dW o K_LL)^T) / lambda; four elements per batch so that the loads overlap
   // (the tcgen05 engine has written GW from shared memory already)
-  if constexpr (MP != 128)
+  if constexpr (MP == 0)
   for (long long e0 = (long long)gt * 4; e0 < (long long)m * ldm; e0 += 4 * gn) {
     float a[4], b[4], c[4], d4[4];
 #pragma unroll

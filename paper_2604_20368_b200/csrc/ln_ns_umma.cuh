@@ -1,19 +1,35 @@
-// Newton-Schulz (Alg. 2) and its adjoint for 64 < m <= 128 on the 5th-generation tensor cores:
+// Newton-Schulz (Alg. 2) and its adjoint for m <= 128 on the 5th-generation tensor cores:
 // tcgen05.mma issued by one thread, operands as bf16 hi + lo images in shared memory (three MMAs
 // per product: lo*hi, hi*lo, hi*hi), fp32 accumulators in tensor memory (TMEM), read back with
 // tcgen05.ld for the epilogue that produces the next operand image.  One CTA of 256 threads per head;
-// the iterate never leaves the SM except for the fp32 history the backward pass needs.
+// the iterate never leaves the SM except for the history the backward pass needs.
 //
-// Thread t owns row 32*(warp%4) + lane of a 128 x 128 accumulator and the column half warp/4.
+// Two sizes, UM = 128 (64 < m <= 128) and UM = 64 (m <= 64), the matrix padded with zeros to UM x UM.
+// UM = 128: thread t owns row 32 (warp % 4) + lane of the accumulator and the column half warp / 4 (64 values).
+// UM = 64 : an M = 64 accumulator keeps row r in TMEM lane 32 (r / 16) + r % 16, so the first 16 lanes of every warp
+//           own row 16 (warp % 4) + lane and the column half warp / 4 (32 values); the other lanes only take part
+//           in the warp-wide TMEM loads and the barriers.
 #pragma once
-#include "ln_ns_smem.cuh"
+#include "ln_mma.cuh"
 #include "ln_umma.cuh"
 
 namespace ln {
 
-constexpr int UM = 128;                       // padded matrix size of this path
-constexpr int UIMG = UM * UM;                 // bf16 elements of one image part (hi or lo)
-constexpr size_t kUmmaMatBytes = (size_t)2 * UIMG * sizeof(bf16);   // hi + lo = 64 KiB
+// geometry of one size: UIMG = bf16 elements of one image part (hi or lo), NV = values a thread owns of its row
+template <int UM> struct UmmaGeo {
+  static constexpr int UIMG = UM * UM;
+  static constexpr size_t mat_bytes = (size_t)2 * UIMG * sizeof(bf16);     // hi + lo: 64 KiB (UM = 128), 16 KiB (UM = 64)
+  static constexpr int NV = UM / 2;
+  static constexpr int LOG = UM == 128 ? 7 : 6;
+  __device__ static __forceinline__ bool active() { return UM == 128 || (threadIdx.x & 31) < 16; }
+  __device__ static __forceinline__ int row() {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    return UM == 128 ? (warp & 3) * 32 + lane : (warp & 3) * 16 + (lane & 15);
+  }
+  __device__ static __forceinline__ int col0() { return (int)(threadIdx.x >> 7) * NV; }
+};
+constexpr size_t kUmmaMatBytes = UmmaGeo<128>::mat_bytes;
+constexpr size_t kUmmaMatBytes64 = UmmaGeo<64>::mat_bytes;
 
 struct UmmaCtl {                              // small static shared state of the tcgen05 kernels
   unsigned long long mbar;                    // completion of MMAs
@@ -24,8 +40,10 @@ struct UmmaCtl {                              // small static shared state of th
 
 // D[tmem_col .. +128) (+)= op(A) op(B) with split operands (hi at image, lo at image + UIMG); one thread.
 //   a_k: A image rows are M (A = X) else rows are K (A = X^T);  b_k: B image rows are N (B = X^T) else rows are K (B = X)
+template <int UM>
 __device__ __forceinline__ void umma_gemm(uint32_t tmem_d, const bf16* A, bool a_k, const bf16* Bm, bool b_k, bool accumulate) {
-  const uint32_t idesc = umma::instr_desc(UM, !a_k, !b_k);
+  constexpr int UIMG = UmmaGeo<UM>::UIMG;
+  const uint32_t idesc = umma::instr_desc(UM, !a_k, !b_k, UM);
   bool acc = accumulate;
 #pragma unroll 1
   for (int part = 0; part < 3; ++part) {      // lo*hi, hi*lo, hi*hi
@@ -43,13 +61,14 @@ __device__ __forceinline__ void umma_gemm(uint32_t tmem_d, const bf16* A, bool a
 // `phase` is each thread's own copy of the mbarrier phase (identical in all threads)
 // drain_stores: thread 0 first lets its bulk stores finish reading shared memory, so that when the barrier
 // completes the buffers those stores read may be overwritten by everybody
+template <int UM>
 __device__ __forceinline__ bool umma_run(UmmaCtl& ctl, uint32_t& phase, uint32_t tmem_d, const bf16* A, bool a_k, const bf16* Bm,
                                          bool b_k, bool accumulate, const bf16* A2 = nullptr, bool a2_k = true,
                                          const bf16* B2 = nullptr, bool b2_k = true, bool drain_stores = false) {
   if (threadIdx.x == 0) {
     umma::fence_after_sync();
-    umma_gemm(tmem_d, A, a_k, Bm, b_k, accumulate);
-    if (A2) umma_gemm(tmem_d, A2, a2_k, B2, b2_k, true);
+    umma_gemm<UM>(tmem_d, A, a_k, Bm, b_k, accumulate);
+    if (A2) umma_gemm<UM>(tmem_d, A2, a2_k, B2, b2_k, true);
     if (drain_stores) umma::bulk_store_wait_read();
     umma::commit(&ctl.mbar);
   }
@@ -59,68 +78,41 @@ __device__ __forceinline__ bool umma_run(UmmaCtl& ctl, uint32_t& phase, uint32_t
   return ok;
 }
 
-// 64 consecutive columns (this thread's half) of its accumulator row
-__device__ __forceinline__ void umma_row(uint32_t tmem_base, int col0, float (&v)[64]) {
-  float a[32], b[32];
-  umma::tmem_ld32(umma::tmem_addr(tmem_base, col0), a);
-  umma::tmem_ld32(umma::tmem_addr(tmem_base, col0 + 32), b);
+// NV consecutive columns (this thread's half) of its accumulator row (every lane of the warp takes part in the load)
+template <int NV>
+__device__ __forceinline__ void umma_row(uint32_t tmem_base, int col0, float (&v)[NV]) {
 #pragma unroll
-  for (int q = 0; q < 32; ++q) { v[q] = a[q]; v[32 + q] = b[q]; }
+  for (int c = 0; c < NV; c += 32) {
+    float a[32];
+    umma::tmem_ld32(umma::tmem_addr(tmem_base, col0 + c), a);
+#pragma unroll
+    for (int q = 0; q < 32; ++q) v[c + q] = a[q];
+  }
 }
 
 // this thread's 64 values of row i -> global fp32 row (leading dimension ld, a multiple of 4): 128-bit stores.
 // Columns in [m, ld) receive whatever the accumulator holds there (zero); readers mask them anyway.
-__device__ __forceinline__ void umma_row_to_global(const float (&v)[64], float* dst_row, int j0, int ld) {
+template <int NV>
+__device__ __forceinline__ void umma_row_to_global(const float (&v)[NV], float* dst_row, int j0, int ld) {
 #pragma unroll
-  for (int p = 0; p < 16; ++p) {
+  for (int p = 0; p < NV / 4; ++p) {
     const int c = j0 + 4 * p;
     if (c < ld) *reinterpret_cast<float4*>(dst_row + c) = make_float4(v[4 * p], v[4 * p + 1], v[4 * p + 2], v[4 * p + 3]);
   }
 }
 
-// this thread's 64 values of row i -> the hi/lo image (eight 16-byte pieces each)
-__device__ __forceinline__ void umma_row_to_image(const float (&v)[64], int i, int j0, bf16* image) {
+// this thread's NV values of row i -> the hi/lo image of a UM x UM matrix (16-byte pieces)
+template <int UM>
+__device__ __forceinline__ void umma_row_to_image(const float (&v)[UM / 2], int i, int j0, bf16* image) {
+  constexpr int UIMG = UmmaGeo<UM>::UIMG;
 #pragma unroll
-  for (int p = 0; p < 8; ++p) {
+  for (int p = 0; p < UM / 16; ++p) {
     uint2 h0, l0, h1, l1;
     split4(make_float4(v[8 * p], v[8 * p + 1], v[8 * p + 2], v[8 * p + 3]), h0, l0);
     split4(make_float4(v[8 * p + 4], v[8 * p + 5], v[8 * p + 6], v[8 * p + 7]), h1, l1);
     const int off = umma::img(i, j0 + 8 * p, UM);
     *reinterpret_cast<uint4*>(image + off) = make_uint4(h0.x, h0.y, h1.x, h1.y);
     *reinterpret_cast<uint4*>(image + UIMG + off) = make_uint4(l0.x, l0.y, l1.x, l1.y);
-  }
-}
-
-// global fp32 [m][m] (leading dimension ld) -> image, zero outside m x m.  256 threads, 8 pieces in flight.
-__device__ __forceinline__ void umma_load_image(const float* __restrict__ src, int m, int ld, bf16* image) {
-  const bool vec = (ld & 3) == 0;
-#pragma unroll 1
-  for (int b0 = 0; b0 < UM * UM / 8 / 256; b0 += 4) {       // 2048 pieces of 8 floats, 8 per thread
-    float v[4][8];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int pc = (b0 + u) * 256 + threadIdx.x, i = pc >> 4, j = (pc & 15) * 8;
-      if (i < m && j < m && vec) {
-        const float4 x = *reinterpret_cast<const float4*>(src + (long long)i * ld + j);
-        const float4 y = (j + 4 < ld) ? *reinterpret_cast<const float4*>(src + (long long)i * ld + j + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-        v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w; v[u][4] = y.x; v[u][5] = y.y; v[u][6] = y.z; v[u][7] = y.w;
-      } else {
-#pragma unroll
-        for (int q = 0; q < 8; ++q) v[u][q] = (i < m && j + q < m) ? src[(long long)i * ld + j + q] : 0.f;
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int pc = (b0 + u) * 256 + threadIdx.x, i = pc >> 4, j = (pc & 15) * 8;
-#pragma unroll
-      for (int q = 0; q < 8; ++q) if (j + q >= m) v[u][q] = 0.f;       // padded columns of a row hold nothing defined
-      uint2 h0, l0, h1, l1;
-      split4(make_float4(v[u][0], v[u][1], v[u][2], v[u][3]), h0, l0);
-      split4(make_float4(v[u][4], v[u][5], v[u][6], v[u][7]), h1, l1);
-      const int off = umma::img(i, j, UM);
-      *reinterpret_cast<uint4*>(image + off) = make_uint4(h0.x, h0.y, h1.x, h1.y);
-      *reinterpret_cast<uint4*>(image + UIMG + off) = make_uint4(l0.x, l0.y, l1.x, l1.y);
-    }
   }
 }
 
@@ -145,26 +137,32 @@ __device__ __forceinline__ void umma_step_done(UmmaCtl& ctl, bool ok) {
   __syncthreads();
 }
 
-// Forward iteration.  smem: images W, X, Q (3 * kUmmaMatBytes).  Histories in global memory, slots of hs floats
-// (hs * 4 >= kUmmaMatBytes): Xh slot k < T receives the operand image of X_k, slot T receives X_T in fp32 (leading
+
+// Forward iteration.  smem: images W, X, Q (3 * mat_bytes).  Histories in global memory, slots of hs floats
+// (hs * 4 >= mat_bytes): Xh slot k < T receives the operand image of X_k, slot T receives X_T in fp32 (leading
 // dimension ld); Ph slot k (may be NULL) receives the image of Q_k = 2I - W X_k.  The images leave by bulk copies
 // that one thread issues and that run beside the next product.  Returns false if a tensor-core wait timed out.
+template <int UM>
 __device__ bool ns_forward_umma(int m, int T, float eps, float alpha_in, const float* W, float* Xh, float* Ph, int ld,
                                 long long hs, NsHdr* hdr, bf16* smem, float* red, UmmaCtl& ctl, float& bad) {
   // bad: this thread's count of non-finite entries of X_T (from its registers)
+  typedef UmmaGeo<UM> Geo;
+  constexpr int UIMG = Geo::UIMG, NV = Geo::NV, LOG = Geo::LOG;
+  constexpr uint32_t MATB = (uint32_t)Geo::mat_bytes;
   bf16* sW = smem; bf16* sX = smem + 2 * UIMG; bf16* sP = smem + 4 * UIMG;
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64;
-  umma_begin(ctl, 128);
+  const int tid = threadIdx.x;
+  const int row = Geo::row(), col0 = Geo::col0();
+  const bool act = Geo::active();
+  umma_begin(ctl, UM);
   uint32_t phase = 0;
   // W + eps I staged in fp32 in the space of Q: norms, images of W and X_0, fp32 X_0 all come from there
-  float* Wf = reinterpret_cast<float*>(sP);      // [128][128], pitch 128
+  float* Wf = reinterpret_cast<float*>(sP);      // [UM][UM], pitch UM
 #pragma unroll 1
   for (int b0 = 0; b0 < UM * UM / 256; b0 += 8) {
     float v[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      const int e = (b0 + u) * 256 + tid, i = e >> 7, j = e & 127;
+      const int e = (b0 + u) * 256 + tid, i = e >> LOG, j = e & (UM - 1);
       v[u] = (i < m && j < m) ? W[(long long)i * m + j] + (i == j ? eps : 0.f) : 0.f;
     }
 #pragma unroll
@@ -176,7 +174,7 @@ __device__ bool ns_forward_umma(int m, int T, float eps, float alpha_in, const f
     if (tid < m) {
       float cs = 0.f, rs = 0.f;
       for (int i = 0; i < m; ++i) cs += fabsf(Wf[i * UM + tid]);
-      for (int i = 0; i < UM; ++i) rs += fabsf(Wf[tid * UM + ((i + tid) & 127)]);   // rotated start: no bank conflicts; padding is zero
+      for (int i = 0; i < UM; ++i) rs += fabsf(Wf[tid * UM + ((i + tid) & (UM - 1))]);   // rotated start: no bank conflicts; padding is zero
       colsum[tid] = cs; rowsum[tid] = rs;
     }
     __syncthreads();
@@ -194,73 +192,89 @@ __device__ bool ns_forward_umma(int m, int T, float eps, float alpha_in, const f
     __syncthreads();
   }
   const float alpha = hdr->alpha;
-  {  // this thread's row: 64 columns of W and of X_0 = alpha W^T
-    float w[64], x0[64];
+  if (act) {  // this thread's row: NV columns of W and of X_0 = alpha W^T
+    float w[NV], x0[NV];
 #pragma unroll
-    for (int q = 0; q < 64; ++q) { w[q] = Wf[row * UM + col0 + q]; x0[q] = alpha * Wf[(col0 + q) * UM + row]; }
-    umma_row_to_image(w, row, col0, sW);
-    umma_row_to_image(x0, row, col0, sX);
-    if (T == 0 && row < m) umma_row_to_global(x0, Xh + (long long)row * ld, col0, ld);
+    for (int q = 0; q < NV; ++q) { w[q] = Wf[row * UM + col0 + q]; x0[q] = alpha * Wf[(col0 + q) * UM + row]; }
+    umma_row_to_image<UM>(w, row, col0, sW);
+    umma_row_to_image<UM>(x0, row, col0, sX);
+    if (T == 0 && row < m) umma_row_to_global<NV>(x0, Xh + (long long)row * ld, col0, ld);
     if (T == 0) {
 #pragma unroll
-      for (int q = 0; q < 64; ++q) bad += isfinite(x0[q]) ? 0.f : 1.f;
+      for (int q = 0; q < NV; ++q) bad += isfinite(x0[q]) ? 0.f : 1.f;
     }
   }
   bool ok = true;
   umma_step_done(ctl, true);
-  if (tid == 0 && T > 0) umma::bulk_store(Xh, sX, (uint32_t)kUmmaMatBytes);                 // image of X_0
+  if (tid == 0 && T > 0) umma::bulk_store(Xh, sX, MATB);                                   // image of X_0
   for (int k = 0; k < T; ++k) {
     // the store of Q_{k-1} has read sP before the barrier of this product completes
-    ok &= umma_run(ctl, phase, ctl.tmem_base, sW, true, sX, false, false, nullptr, true, nullptr, true, true);   // D = W X_k
+    ok &= umma_run<UM>(ctl, phase, ctl.tmem_base, sW, true, sX, false, false, nullptr, true, nullptr, true, true);   // D = W X_k
     {
-      float v[64];
-      umma_row(ctl.tmem_base, col0, v);
+      float v[NV];
+      umma_row<NV>(ctl.tmem_base, col0, v);
+      if (act) {
 #pragma unroll
-      for (int q = 0; q < 64; ++q) v[q] = ((row == col0 + q && row < m) ? 2.f : 0.f) - v[q];   // Q_k = 2I - W X_k
-      umma_row_to_image(v, row, col0, sP);
-    }
-    umma_step_done(ctl, ok);
-    if (tid == 0 && Ph) umma::bulk_store(Ph + k * hs, sP, (uint32_t)kUmmaMatBytes);
-    // the store of X_k has read sX before the barrier of this product completes
-    ok &= umma_run(ctl, phase, ctl.tmem_base, sX, true, sP, false, false, nullptr, true, nullptr, true, true);   // D = X_k Q_k
-    {
-      float v[64];
-      umma_row(ctl.tmem_base, col0, v);
-      if (k + 1 == T) {
-        if (row < m) umma_row_to_global(v, Xh + T * hs + (long long)row * ld, col0, ld);
-#pragma unroll
-        for (int q = 0; q < 64; ++q) bad += isfinite(v[q]) ? 0.f : 1.f;
+        for (int q = 0; q < NV; ++q) v[q] = ((row == col0 + q && row < m) ? 2.f : 0.f) - v[q];   // Q_k = 2I - W X_k
+        umma_row_to_image<UM>(v, row, col0, sP);
       }
-      umma_row_to_image(v, row, col0, sX);     // the MMAs and the bulk store that read X_k have completed
     }
     umma_step_done(ctl, ok);
-    if (tid == 0 && k + 1 < T) umma::bulk_store(Xh + (k + 1) * hs, sX, (uint32_t)kUmmaMatBytes);
+    if (tid == 0 && Ph) umma::bulk_store(Ph + k * hs, sP, MATB);
+    // the store of X_k has read sX before the barrier of this product completes
+    ok &= umma_run<UM>(ctl, phase, ctl.tmem_base, sX, true, sP, false, false, nullptr, true, nullptr, true, true);   // D = X_k Q_k
+    {
+      float v[NV];
+      umma_row<NV>(ctl.tmem_base, col0, v);
+      if (act) {
+        if (k + 1 == T) {
+          if (row < m) umma_row_to_global<NV>(v, Xh + T * hs + (long long)row * ld, col0, ld);
+#pragma unroll
+          for (int q = 0; q < NV; ++q) bad += isfinite(v[q]) ? 0.f : 1.f;
+        }
+        umma_row_to_image<UM>(v, row, col0, sX);     // the MMAs and the bulk store that read X_k have completed
+      }
+    }
+    umma_step_done(ctl, ok);
+    if (tid == 0 && k + 1 < T) umma::bulk_store(Xh + (k + 1) * hs, sX, MATB);
   }
   if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");      // every image has reached global memory
   ok &= (ctl.timeout == 0);
-  umma_end(ctl, 128);
+  umma_end(ctl, UM);
   return ok;
 }
 
-// Adjoint for a symmetric W (see ns_backward_smem for the algebra): per step, with A = X_k and Q = 2I - W X_k as
-// the forward pass left them (operand images), H = A^T G, dW -= H A^T, G <- G Q^T + Q^T G - 2G.
-// smem: images A (also used for Q), G, H.  TMEM: 128 columns for the running product, 128 for dW accumulated over
+// Adjoint of the iteration for a symmetric W (the landmark kernel matrix is symmetric bit for bit).
+// Per step k (A = X_k, Q = 2I - W A, both saved as operand images by the forward pass):
+//     H = A^T G,   dW -= H A^T,   G <- G Q^T + Q^T G - 2G.
+// In general the last term of the step adjoint is W^T H = (A W)^T G; for symmetric W every iterate is a
+// polynomial in W, so A W = W A up to rounding, (A W)^T G = (2I - Q)^T G, and W itself is not needed inside
+// the loop.  G is kept in fp32 in registers and re-split into its image after each update.
+// smem: images A (also used for Q), G, H.  TMEM: UM columns for the running product, UM for dW accumulated over
 // all steps.  The images arrive by bulk copies on an mbarrier; the copy of the next A runs beside the G update.
+// UM = 64 has room for a fourth image: Q has its own buffer, A and Q of the next step are both fetched ahead, and
+// the products dW += H A^T and G Q^T + Q^T G are issued together and waited for once (two waits per step, not three).
 // Output: GW [m][ldgw] = (dW o W + (dW o W)^T) / lambda, the upstream of the landmark kernel block (dW itself
 // stays on chip).
+template <int UM>
 __device__ bool ns_backward_umma(int m, int T, float eps, const float* W, const float* Xh, const float* Ph, int ld,
                                  long long hs, const NsHdr* hdr, const float* G0, float* GW, int ldgw, float inv_lambda,
                                  bf16* smem, float* red, UmmaCtl& ctl) {
-  bf16* sA = smem; bf16* sG = smem + 2 * UIMG; bf16* sH = smem + 4 * UIMG;
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64;
-  umma_begin(ctl, 256);
+  typedef UmmaGeo<UM> Geo;
+  constexpr int UIMG = Geo::UIMG, NV = Geo::NV, LOG = Geo::LOG;
+  constexpr uint32_t MATB = (uint32_t)Geo::mat_bytes;
+  constexpr bool QBUF = (UM == 64);
+  bf16* sA = smem; bf16* sG = smem + 2 * UIMG; bf16* sH = smem + 4 * UIMG; bf16* sQ = smem + (QBUF ? 6 : 0) * UIMG;
+  const int tid = threadIdx.x;
+  const int row = Geo::row(), col0 = Geo::col0();
+  const bool act = Geo::active();
+  umma_begin(ctl, 2 * UM);
   uint32_t phase = 0, ph_ld = 0;
-  const uint32_t t_acc = ctl.tmem_base, t_dw = ctl.tmem_base + 128;
+  const uint32_t t_acc = ctl.tmem_base, t_dw = ctl.tmem_base + UM;
   auto load_image = [&](const float* src) {     // one thread starts the copy into sA
     if (tid == 0) {
-      umma::mbar_expect_tx(&ctl.mbar_ld, (uint32_t)kUmmaMatBytes);
-      umma::bulk_load(sA, src, (uint32_t)kUmmaMatBytes, &ctl.mbar_ld);
+      umma::mbar_expect_tx(&ctl.mbar_ld, MATB);
+      umma::bulk_load(sA, src, MATB, &ctl.mbar_ld);
     }
   };
   auto wait_image = [&]() {                     // everybody sees the image (thread 0 issues the MMAs that read it)
@@ -268,89 +282,120 @@ __device__ bool ns_backward_umma(int m, int T, float eps, const float* W, const 
     ph_ld ^= 1u;
     return got;
   };
-  if (T > 0) load_image(Xh + (long long)(T - 1) * hs);
-  float G[64];                                 // this thread's part of G in full precision
+  auto load_pair = [&](int k) {                 // A = X_k and Q_k, counted on one phase of the barrier
+    if (tid == 0) {
+      umma::mbar_expect_tx(&ctl.mbar_ld, 2 * MATB);
+      umma::bulk_load(sA, Xh + (long long)k * hs, MATB, &ctl.mbar_ld);
+      umma::bulk_load(sQ, Ph + (long long)k * hs, MATB, &ctl.mbar_ld);
+    }
+  };
+  if (T > 0) { if constexpr (QBUF) load_pair(T - 1); else load_image(Xh + (long long)(T - 1) * hs); }
+  float G[NV];                                 // this thread's part of G in full precision
 #pragma unroll
-  for (int q = 0; q < 64; ++q) G[q] = (row < m && col0 + q < m) ? G0[(long long)row * ld + col0 + q] : 0.f;
-  umma_row_to_image(G, row, col0, sG);
+  for (int q = 0; q < NV; ++q) G[q] = (act && row < m && col0 + q < m) ? G0[(long long)row * ld + col0 + q] : 0.f;
+  if (act) umma_row_to_image<UM>(G, row, col0, sG);
   bool ok = true;
   for (int k = T - 1; k >= 0; --k) {
     ok &= wait_image();                                                                       // A = X_k
     umma_step_done(ctl, ok);
-    ok &= umma_run(ctl, phase, t_acc, sA, false, sG, false, false);                          // H = A^T G
+    ok &= umma_run<UM>(ctl, phase, t_acc, sA, false, sG, false, false);                      // H = A^T G
     {
-      float v[64];
-      umma_row(t_acc, col0, v);
-      umma_row_to_image(v, row, col0, sH);
+      float v[NV];
+      umma_row<NV>(t_acc, col0, v);
+      if (act) umma_row_to_image<UM>(v, row, col0, sH);
     }
     umma_step_done(ctl, ok);
-    ok &= umma_run(ctl, phase, t_dw, sH, true, sA, true, k != T - 1);                        // dW accumulator += H A^T
-    load_image(Ph + (long long)k * hs);                                                       // Q_k (A is no longer read)
-    ok &= wait_image();
-    umma_step_done(ctl, ok);
-    ok &= umma_run(ctl, phase, t_acc, sG, true, sA, true, false, sA, false, sG, false);      // G Q^T + Q^T G
-    if (k > 0) load_image(Xh + (long long)(k - 1) * hs);                                      // next A, beside the G update
+    if constexpr (QBUF) {
+      if (tid == 0) {
+        umma::fence_after_sync();
+        umma_gemm<UM>(t_dw, sH, true, sA, true, k != T - 1);                                  // dW accumulator += H A^T
+        umma_gemm<UM>(t_acc, sG, true, sQ, true, false);                                      // G Q^T
+        umma_gemm<UM>(t_acc, sQ, false, sG, false, true);                                     //   + Q^T G
+        umma::commit(&ctl.mbar);
+      }
+      ok &= umma::mbar_wait(&ctl.mbar, phase & 1);
+      phase ^= 1u;
+      umma::fence_after_sync();
+      if (k > 0) load_pair(k - 1);                                                            // next A and Q, beside the G update
+    } else {
+      ok &= umma_run<UM>(ctl, phase, t_dw, sH, true, sA, true, k != T - 1);                  // dW accumulator += H A^T
+      load_image(Ph + (long long)k * hs);                                                     // Q_k (A is no longer read)
+      ok &= wait_image();
+      umma_step_done(ctl, ok);
+      ok &= umma_run<UM>(ctl, phase, t_acc, sG, true, sA, true, false, sA, false, sG, false);   // G Q^T + Q^T G
+      if (k > 0) load_image(Xh + (long long)(k - 1) * hs);                                    // next A, beside the G update
+    }
     {
-      float v[64];
-      umma_row(t_acc, col0, v);
+      float v[NV];
+      umma_row<NV>(t_acc, col0, v);
+      if (act) {
 #pragma unroll
-      for (int q = 0; q < 64; ++q) G[q] = (row < m && col0 + q < m) ? v[q] - 2.f * G[q] : 0.f;
-      umma_row_to_image(G, row, col0, sG);
+        for (int q = 0; q < NV; ++q) G[q] = (row < m && col0 + q < m) ? v[q] - 2.f * G[q] : 0.f;
+        umma_row_to_image<UM>(G, row, col0, sG);
+      }
     }
   }
   umma_step_done(ctl, ok);
-  float dw[64];                                // this thread's part of -(accumulated H A^T)
+  float dw[NV];                                // this thread's part of -(accumulated H A^T)
   {
-    float v[64];
-    if (T > 0) umma_row(t_dw, col0, v);
+    float v[NV];
+    if (T > 0) umma_row<NV>(t_dw, col0, v);
 #pragma unroll
-    for (int q = 0; q < 64; ++q) dw[q] = (T > 0) ? -v[q] : 0.f;
+    for (int q = 0; q < NV; ++q) dw[q] = (T > 0) ? -v[q] : 0.f;
   }
   ok &= (ctl.timeout == 0);
-  umma_end(ctl, 256);
+  umma_end(ctl, 2 * UM);
   __syncthreads();
   // End of the adjoint and the upstream of the landmark block, from shared memory (the operand buffers are free):
   //   X_0 = alpha (W + eps I)^T:  d alpha = <G, Wr^T>,  dW += alpha G^T, then the alpha(W) terms;
   //   GW = (dW o W + (dW o W)^T) / lambda.
-  // G and Wr are staged as fp32 [128][129] (the odd pitch makes the transposed reads conflict-free).
+  // G and Wr are staged as fp32 [UM][UM + 1] (the odd pitch makes the transposed reads conflict-free).
   constexpr int PT = UM + 1;
   float* sGf = reinterpret_cast<float*>(smem);
   float* sWf = sGf + UM * PT;
+  if (act) {
 #pragma unroll
-  for (int q = 0; q < 64; ++q) sGf[row * PT + col0 + q] = G[q];
+    for (int q = 0; q < NV; ++q) sGf[row * PT + col0 + q] = G[q];
+  }
   for (int e = tid; e < UM * UM; e += 256) {
-    const int i = e >> 7, j = e & 127;
+    const int i = e >> LOG, j = e & (UM - 1);
     sWf[i * PT + j] = (i < m && j < m) ? W[(long long)i * m + j] + (i == j ? eps : 0.f) : 0.f;
   }
   __syncthreads();
   const float alpha = hdr->alpha;
   float part = 0.f;
+  if (act) {
 #pragma unroll
-  for (int q = 0; q < 64; ++q) part += G[q] * sWf[(col0 + q) * PT + row];
+    for (int q = 0; q < NV; ++q) part += G[q] * sWf[(col0 + q) * PT + row];
+  }
   const float dalpha = block_sum(part, red);
   const bool aa = hdr->auto_alpha != 0;
   const int js = hdr->jstar, is = hdr->istar;
   const float c1 = dalpha * (-alpha / hdr->n1), c2 = dalpha * (-alpha / hdr->ninf);
+  if (act) {
 #pragma unroll
-  for (int q = 0; q < 64; ++q) {
-    const int j = col0 + q;
-    float v = dw[q] + alpha * sGf[j * PT + row];
-    if (aa) {
-      const float w = sWf[row * PT + j];
-      const float sg = w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f);
-      if (j == js) v += c1 * sg;
-      if (row == is) v += c2 * sg;
+    for (int q = 0; q < NV; ++q) {
+      const int j = col0 + q;
+      float v = dw[q] + alpha * sGf[j * PT + row];
+      if (aa) {
+        const float w = sWf[row * PT + j];
+        const float sg = w > 0.f ? 1.f : (w < 0.f ? -1.f : 0.f);
+        if (j == js) v += c1 * sg;
+        if (row == is) v += c2 * sg;
+      }
+      dw[q] = (row < m && j < m) ? v : 0.f;
     }
-    dw[q] = (row < m && j < m) ? v : 0.f;
   }
   __syncthreads();                             // everybody has read G
+  if (act) {
 #pragma unroll
-  for (int q = 0; q < 64; ++q) sGf[row * PT + col0 + q] = dw[q];      // now dW
+    for (int q = 0; q < NV; ++q) sGf[row * PT + col0 + q] = dw[q];      // now dW
+  }
   __syncthreads();
-  if (row < m) {
+  if (act && row < m) {
     float* grow = GW + (long long)row * ldgw;
 #pragma unroll
-    for (int q = 0; q < 64; q += 4) {
+    for (int q = 0; q < NV; q += 4) {
       const int j = col0 + q;
       if (j >= ldgw) break;
       float o[4];

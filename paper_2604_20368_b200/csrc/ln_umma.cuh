@@ -37,10 +37,11 @@ __device__ __forceinline__ uint64_t operand_desc(const bf16* image, int cols, bo
   return smem_desc(s32(image) + (uint32_t)ks * 2 * row_group, row_group, 128);
 }
 
-// Instruction descriptor, kind::f16: fp32 accumulate, bf16 operands, M = 128.
-__device__ __forceinline__ uint32_t instr_desc(int N, bool a_mn_major, bool b_mn_major) {
+// Instruction descriptor, kind::f16: fp32 accumulate, bf16 operands, M = 128 (accumulator row r in TMEM lane r) or
+// M = 64 (row r in lane 32 (r / 16) + r % 16: each warp quarter holds 16 rows in its first 16 lanes).
+__device__ __forceinline__ uint32_t instr_desc(int N, bool a_mn_major, bool b_mn_major, int M = 128) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
-         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
 // D[tmem] (+)= A * B for one K-step; issued by ONE thread.
