@@ -31,6 +31,7 @@ struct Carver {
 
 struct Plan {
   int BH, n, d, m, T, ldm, rpc, chunks;
+  size_t scr;                        // floats per scratch matrix of the per-head kernels
   long long hslot;                   // floats per slot of the Newton-Schulz histories
   int s2_tg, s2_rpc, s2_chunks;      // fused sign pass: token groups per tile, tokens per chunk, chunks (0 = not used)
   int s2q_rpc, s2q_chunks;           // the same for the query-side pass, which shares the GPU with the per-head kernel
@@ -42,10 +43,13 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   if (!p) return false;
   pl->BH = p->B * p->H; pl->n = p->n; pl->d = p->d; pl->m = p->m; pl->T = p->ns_iters;
   pl->ldm = (p->m + 3) & ~3;
+  pl->scr = (size_t)p->m * pl->ldm;
+  if (p->dtype == LN_BF16 && p->m > 128) pl->scr = (size_t)kU2Slot;
   // history slots: fp32 [m][ldm], except on the m <= 64 tensor-core path, whose slots hold operand images
   pl->hslot = (long long)p->m * pl->ldm;
   if (p->dtype == LN_BF16 && p->m <= 64) pl->hslot = (long long)(kUmmaMatBytes64 / 4);                 // 16 KiB images >= m * ldm * 4
   if (p->dtype == LN_BF16 && p->m > 64 && p->m <= 128) pl->hslot = (long long)(kUmmaMatBytes / 4);     // 64 KiB images >= m * ldm * 4
+  if (p->dtype == LN_BF16 && p->m > 128) pl->hslot = kU2Slot;                                          // four 64 KiB block images
   // token chunks per head for the reductions over tokens: about eight waves of CTAs (two per SM) so that
   // the last wave costs little, but at least 64 tokens per chunk
   const int mblk = (p->m + 63) / 64;
@@ -60,7 +64,7 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   // fused sign pass (64-dim slabs): token tiles of 8 * TG tokens that hug n, chunks for about three waves
   pl->s2_tg = pl->s2_rpc = pl->s2_chunks = pl->s2q_rpc = pl->s2q_chunks = 0; pl->s2_smem = 0;
   // per-head kernels (bf16 storage): three CTAs per SM for m <= 64, one for m <= 128, else clusters of four CTAs, two per SM
-  pl->mid_sms = p->m <= 64 ? (pl->BH + 2) / 3 : (p->m <= 128 ? pl->BH : 2 * pl->BH);
+  pl->mid_sms = p->m <= 64 ? (pl->BH + 2) / 3 : (p->m <= 128 ? pl->BH : 4 * pl->BH);
   if (p->d % 64 == 0) {
     const int groups = (p->n + 7) / 8;
     int tiles = (groups + S2_TGMAX - 1) / S2_TGMAX;
@@ -125,8 +129,8 @@ FwdWs carve_fwd_ws(const Plan& pl, void* base) {
   Carver c(base); FwdWs w;
   const size_t BH = pl.BH, d = pl.d, m = pl.m;
   w.Mpart = c.take(BH * pl.chunks * m * d);
-  w.Wr = c.take(BH * m * pl.ldm);
-  w.P = c.take(BH * m * pl.ldm);
+  w.Wr = c.take(BH * pl.scr);
+  w.P = c.take(BH * pl.scr);
   w.Y = c.take(BH * m * d);
   w.bytes = c.off;
   return w;
@@ -149,13 +153,13 @@ BwdWs carve_bwd_ws(const Plan& pl, void* base) {
   w.dLRpart = c.take(BH * chs * m * d);
   w.dY = c.take(BH * m * d);
   w.dM = c.take(BH * m * d);
-  w.Wr = c.take(BH * m * pl.ldm);
-  w.P = c.take(BH * m * pl.ldm);
-  w.Hm = c.take(BH * m * pl.ldm);
-  w.Ga = c.take(BH * m * pl.ldm);
-  w.Gb = c.take(BH * m * pl.ldm);
-  w.dW = c.take(BH * m * pl.ldm);
-  w.dX = c.take(BH * m * pl.ldm);
+  w.Wr = c.take(BH * pl.scr);
+  w.P = c.take(BH * pl.scr);
+  w.Hm = c.take(BH * pl.scr);
+  w.Ga = c.take(BH * pl.scr);
+  w.Gb = c.take(BH * pl.scr);
+  w.dW = c.take(BH * pl.scr);
+  w.dX = c.take(BH * pl.scr);
   w.GW = c.take(BH * m * pl.ldm);
   w.dLW = c.take(BH * m * d);
   w.dLtot = c.take(BH * m * d);
@@ -371,7 +375,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     };
     if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * kUmmaMatBytes64);
     else if (TC && m <= 128) launch(k_mid_fwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
-    else if (TC) launch(k_mid_fwd<D, TC, 0, TC ? kMidCluster : 1>, sizeof(NsSmem), kMidCluster);   // m > 128: a cluster per head
+    else if (TC) launch(k_mid_fwd<D, TC, TC ? 256 : 0, TC ? kMidCluster : 1>, 3 * kUmmaMatBytes, kMidCluster);   // m > 128: a cluster per head
     else launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));
   };
   {
@@ -471,7 +475,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     };
     if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 4 * kUmmaMatBytes64);
     else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
-    else if (TC) launch(k_mid_bwd<D, TC, 0, TC ? kMidCluster : 1>, sizeof(NsSmem), kMidCluster);
+    else if (TC) launch(k_mid_bwd<D, TC, TC ? 256 : 0, TC ? kMidCluster : 1>, 3 * kUmmaMatBytes, kMidCluster);
     else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
   };
   // key-side products: g^R = (V dM^T) o R^T / lambda and dV = R^T dM (they need dM from the per-head kernel)

@@ -5,6 +5,7 @@
 #include "ln_common.cuh"
 #include "ln_mma.cuh"
 #include "ln_ns_umma.cuh"
+#include "ln_ns_umma256.cuh"
 #include "ln_gemm_umma.cuh"
 
 namespace ln {
@@ -825,6 +826,9 @@ __device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const fl
   }
 }
 
+template <int CL>
+__device__ void ns_backward_tail_dev(int m, const float* Wr, const NsHdr* hdr, const float* G, float* dW, float* red, int crank);
+
 // =====================================================================================
 // Exact adjoint of ns_forward_dev: given G0 = dLoss/dX_T returns dW = dLoss/dW.
 // Scratch matrices [m][m]: P, Hm, Ga, Gb.  Xh holds X_0..X_T, Wr = W + eps I, hdr from the forward.
@@ -852,7 +856,15 @@ __device__ void ns_backward_dev(int m, int T, const float* Wr, const float* Xh, 
     if (CL > 1) phase_sync<CL>();
     float* t = G; G = Gn; Gn = t;
   }
-  // X_0 = alpha Wr^T
+  ns_backward_tail_dev<CL>(m, Wr, hdr, G, dW, red, crank);
+}
+
+// End of the adjoint: X_0 = alpha Wr^T with alpha = 1 / (||Wr||_1 ||Wr||_inf) (unless given).  G = dLoss/dX_0 and dW
+// (the part accumulated over the steps) are fp32 [m][m] in global memory; dW receives the rest.  CL CTAs share it.
+template <int CL>
+__device__ void ns_backward_tail_dev(int m, const float* Wr, const NsHdr* hdr, const float* G, float* dW, float* red, int crank) {
+  const int tid = threadIdx.x, gt = crank * 256 + tid, gn = 256 * CL;
+  const long long mm = (long long)m * m;
   const float alpha = hdr->alpha;
   float part = 0.f;
   for (long long e = tid; e < mm; e += 256) {        // every CTA of a cluster sums everything (same order, same value)
@@ -933,7 +945,7 @@ __global__ void __launch_bounds__(256) k_ns_pinv_bwd(int m, int T, float eps, fl
 // =====================================================================================
 // CL > 1 (generic path only): CL CTAs of a thread-block cluster share one head; grid = heads * CL.
 template <int D, bool TC, int MP, int CL = 1>
-__global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_fwd(int m, int ldm, int T, float eps, float alpha_in, int H, int map_mode,
+__global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 : 1)) k_mid_fwd(int m, int ldm, int T, float eps, float alpha_in, int H, int map_mode,
                                                  const float* __restrict__ whiten, const float* W, float* Wr,
                                                  float* P, float* Xh, float* Ph, NsHdr* hdr, const float* Mpart, int nchunks,
                                                  float* Mout, float* Y, float* Yt, float* ybar, int* dev_status,
@@ -951,9 +963,10 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_fw
   const int gt = crank * 256 + tid, gn = 256 * CL;      // this thread among all threads that share the head
   const long long mm = (long long)m * m, md = (long long)m * D;
   // the iterate histories of the shared-memory path use the padded leading dimension (128-bit accesses)
-  const int ldx = (MP > 0) ? ldm : m;
-  const long long mx = (MP == 64 || MP == 128) ? hslot : (long long)m * ldx;
-  W += bh * mm; Wr += bh * mm; P += bh * mm; Xh += (long long)bh * (T + 1) * mx; hdr += bh;
+  const int ldx = (MP == 64 || MP == 128) ? ldm : m;
+  const long long mx = (MP > 0) ? hslot : (long long)m * ldx;
+  const long long wslot = (MP == 256) ? kU2Slot : mm;           // floats per scratch matrix
+  W += bh * mm; Wr += bh * wslot; P += bh * wslot; Xh += (long long)bh * (T + 1) * mx; hdr += bh;
   if (Ph) Ph += (long long)bh * T * mx;
   Mout += bh * md; Y += bh * md; Yt += bh * md; ybar += (long long)bh * D;
   Mpart += (long long)bh * nchunks * md;
@@ -967,6 +980,11 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_fw
   if constexpr (MP == 128 || MP == 64) {        // tcgen05 + TMEM, the matrix padded to MP x MP
     __shared__ UmmaCtl ctl;
     tc_ok = ns_forward_umma<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl, bad);
+    __syncthreads();
+  } else if constexpr (MP == 256) {             // tcgen05 + TMEM, 2 x 2 blocks of 128 shared by the four CTAs of a cluster
+    __shared__ UmmaCtl ctl;
+    __shared__ __align__(8) unsigned long long mbar_free;
+    tc_ok = ns_forward_umma256(m, T, eps, alpha_in, W, Wr, P, Xh, Ph, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl, &mbar_free, crank, bad);
     __syncthreads();
   } else {
     ns_forward_dev<TC, CL>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red, crank, Ph);
@@ -1021,7 +1039,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_fw
   }
 }
 template <int D, bool TC, int MP, int CL = 1>
-__global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_bwd(int m, int T, int H, int map_mode, float inv_lambda, int ldm,
+__global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 : 1)) k_mid_bwd(int m, int T, int H, int map_mode, float inv_lambda, int ldm,
                                                  const float* __restrict__ whiten, const float* W,
                                                  const float* Xh, const float* Ph, const NsHdr* hdr, const float* Msaved,
                                                  const float* dYtpart, const float* dybpart, int nchunks,
@@ -1034,9 +1052,9 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_bw
   const int bh = blockIdx.x / CL, crank = blockIdx.x % CL, tid = threadIdx.x;
   const int gt = crank * 256 + tid, gn = 256 * CL;
   const long long mm = (long long)m * m, md = (long long)m * D;
-  const int ldx = (MP > 0) ? ldm : m;
-  const long long mx = (MP == 64 || MP == 128) ? hslot : (long long)m * ldx;       // one slot of the iterate histories
-  const long long ms = (long long)m * ldm;                             // one scratch matrix
+  const int ldx = (MP == 64 || MP == 128) ? ldm : m;
+  const long long mx = (MP > 0) ? hslot : (long long)m * ldx;          // one slot of the iterate histories
+  const long long ms = (MP == 256) ? kU2Slot : (long long)m * ldm;     // one scratch matrix
   W += bh * mm; Xh += (long long)bh * (T + 1) * mx; Ph += (long long)bh * T * mx; hdr += bh; Msaved += bh * md;
   Wr += bh * ms; P += bh * ms; Hm += bh * ms; Ga += bh * ms; Gb += bh * ms; dWm += bh * ms; dXm += bh * ms;
   dY += bh * md; dM += bh * md; GW += (long long)bh * m * ldm;
@@ -1061,7 +1079,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_bw
     }
     *reinterpret_cast<float4*>(dY + e) = o;
   }
-  if constexpr (MP == 0) {
+  if constexpr (MP == 0 || MP == 256) {
     for (long long e = gt; e < mm; e += gn) {
       const int i = (int)(e / m), j = (int)(e % m);
       Wr[e] = W[e] + (i == j ? eps : 0.f);
@@ -1080,10 +1098,17 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : (CL > 1 ? 2 : 1)) k_mid_bw
     __shared__ UmmaCtl ctl;
     const bool tc_ok = ns_backward_umma<MP>(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, GW, ldm, inv_lambda, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
     if (dev_status && !tc_ok && tid == 0) atomicOr(dev_status + bh, 2);
+  } else if constexpr (MP == 256) {
+    __shared__ UmmaCtl ctl;
+    __shared__ __align__(8) unsigned long long mbar_free;
+    const bool tc_ok = ns_backward_umma256(m, T, Xh, Ph, dXm, Ga, Gb, Hm, P, dWm, reinterpret_cast<bf16*>(dyn_smem), ctl, &mbar_free, crank);
+    if (dev_status && !tc_ok && tid == 0 && crank == 0) atomicOr(dev_status + bh, 2);
+    ns_backward_tail_dev<CL>(m, Wr, hdr, P, dWm, red, crank);
+    phase_sync<CL>();
   } else { ns_backward_dev<TC, CL>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red, crank, Ph); if (CL > 1) phase_sync<CL>(); }
   // GW = (dW o K_LL + (dW o K_LL)^T) / lambda; four elements per batch so that the loads overlap
-  // (the tcgen05 engine has written GW from shared memory already)
-  if constexpr (MP == 0)
+  // (the single-CTA tcgen05 engines have written GW from shared memory already)
+  if constexpr (MP == 0 || MP == 256)
   for (long long e0 = (long long)gt * 4; e0 < (long long)m * ldm; e0 += 4 * gn) {
     float a[4], b[4], c[4], d4[4];
 #pragma unroll
