@@ -826,7 +826,7 @@ __device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const fl
   }
 }
 
-template <int CL>
+template <int CL, bool SYM = false>
 __device__ void ns_backward_tail_dev(int m, const float* Wr, const NsHdr* hdr, const float* G, float* dW, float* red, int crank);
 
 // =====================================================================================
@@ -861,15 +861,27 @@ __device__ void ns_backward_dev(int m, int T, const float* Wr, const float* Xh, 
 
 // End of the adjoint: X_0 = alpha Wr^T with alpha = 1 / (||Wr||_1 ||Wr||_inf) (unless given).  G = dLoss/dX_0 and dW
 // (the part accumulated over the steps) are fp32 [m][m] in global memory; dW receives the rest.  CL CTAs share it.
-template <int CL>
+// SYM: Wr is symmetric bit for bit (the landmark kernel matrix is), so <G, Wr^T> is read along the rows of both.
+template <int CL, bool SYM>
 __device__ void ns_backward_tail_dev(int m, const float* Wr, const NsHdr* hdr, const float* G, float* dW, float* red, int crank) {
   const int tid = threadIdx.x, gt = crank * 256 + tid, gn = 256 * CL;
   const long long mm = (long long)m * m;
   const float alpha = hdr->alpha;
   float part = 0.f;
-  for (long long e = tid; e < mm; e += 256) {        // every CTA of a cluster sums everything (same order, same value)
-    const int i = (int)(e / m), j = (int)(e % m);
-    part += G[e] * Wr[(long long)j * m + i];
+  if (SYM) {
+    float p4[4] = {0.f, 0.f, 0.f, 0.f};              // four independent chains: the loads of a batch overlap
+    long long e = tid;
+    for (; e + 3 * 256 < mm; e += 4 * 256) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) p4[u] += G[e + u * 256] * Wr[e + u * 256];
+    }
+    for (; e < mm; e += 256) p4[0] += G[e] * Wr[e];
+    part = (p4[0] + p4[1]) + (p4[2] + p4[3]);
+  } else {
+    for (long long e = tid; e < mm; e += 256) {      // every CTA of a cluster sums everything (same order, same value)
+      const int i = (int)(e / m), j = (int)(e % m);
+      part += G[e] * Wr[(long long)j * m + i];
+    }
   }
   const float dalpha = block_sum(part, red);
   for (long long e = gt; e < mm; e += gn) {
@@ -1103,7 +1115,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     __shared__ __align__(8) unsigned long long mbar_free;
     const bool tc_ok = ns_backward_umma256(m, T, Xh, Ph, dXm, Ga, Gb, Hm, P, dWm, reinterpret_cast<bf16*>(dyn_smem), ctl, &mbar_free, crank);
     if (dev_status && !tc_ok && tid == 0 && crank == 0) atomicOr(dev_status + bh, 2);
-    ns_backward_tail_dev<CL>(m, Wr, hdr, P, dWm, red, crank);
+    ns_backward_tail_dev<CL, true>(m, Wr, hdr, P, dWm, red, crank);
     phase_sync<CL>();
   } else { ns_backward_dev<TC, CL>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red, crank, Ph); if (CL > 1) phase_sync<CL>(); }
   // GW = (dW o K_LL + (dW o K_LL)^T) / lambda; four elements per batch so that the loads overlap

@@ -113,22 +113,27 @@ __device__ bool ns_forward_umma256(int m, int T, float eps, float alpha_in, cons
   }
   phase_sync<4>();
   {
-    float* colsum = red; float* rowsum = red + 256;
+    // Norms: Wr is symmetric bit for bit (|a - b| = |b - a| term by term in the kernel block), so the absolute row sums
+    // are the absolute column sums; a column is read along the rows (threads side by side), four rows in flight.
+    float* colsum = red;
     if (tid < m) {
-      float cs = 0.f, rs = 0.f;
-      for (int i = 0; i < m; ++i) { cs += fabsf(Wr[(long long)i * m + tid]); rs += fabsf(Wr[(long long)tid * m + i]); }
-      colsum[tid] = cs; rowsum[tid] = rs;
+      float c4[4] = {0.f, 0.f, 0.f, 0.f};
+      int i = 0;
+      for (; i + 3 < m; i += 4) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) c4[u] += fabsf(Wr[(long long)(i + u) * m + tid]);
+      }
+      for (; i < m; ++i) c4[0] += fabsf(Wr[(long long)i * m + tid]);
+      colsum[tid] = (c4[0] + c4[1]) + (c4[2] + c4[3]);
     }
     __syncthreads();
     if (tid == 0) {               // every CTA of the cluster arrives at the same values
-      float n1 = -1.f, ninf = -1.f; int js = 0, is = 0;
-      for (int t = 0; t < m; ++t) {
-        if (colsum[t] > n1) { n1 = colsum[t]; js = t; }
-        if (rowsum[t] > ninf) { ninf = rowsum[t]; is = t; }
-      }
-      red[512] = (alpha_in > 0.f) ? alpha_in : 1.f / (n1 * ninf);
+      float n1 = -1.f; int js = 0;
+      for (int t = 0; t < m; ++t)
+        if (colsum[t] > n1) { n1 = colsum[t]; js = t; }          // strict >: the lowest index on ties
+      red[512] = (alpha_in > 0.f) ? alpha_in : 1.f / (n1 * n1);
       if (crank == 0) {
-        hdr->n1 = n1; hdr->ninf = ninf; hdr->jstar = js; hdr->istar = is;
+        hdr->n1 = n1; hdr->ninf = n1; hdr->jstar = js; hdr->istar = js;
         hdr->auto_alpha = !(alpha_in > 0.f);
         hdr->alpha = red[512];
         hdr->pad0 = hdr->pad1 = 0;
