@@ -1091,11 +1091,8 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     }
     *reinterpret_cast<float4*>(dY + e) = o;
   }
-  if constexpr (MP == 0 || MP == 256) {
-    for (long long e = gt; e < mm; e += gn) {
-      const int i = (int)(e / m), j = (int)(e % m);
-      Wr[e] = W[e] + (i == j ? eps : 0.f);
-    }
+  if constexpr (MP == 0 || MP == 256) {             // m <= 256: 32-bit index arithmetic (a 64-bit division costs far more)
+    for (unsigned e = (unsigned)gt; e < (unsigned)mm; e += (unsigned)gn) Wr[e] = W[e] + (e % (unsigned)(m + 1) == 0u ? eps : 0.f);
   }
   phase_sync<CL>();
   const float* XT = Xh + (long long)T * mx;

@@ -107,10 +107,7 @@ __device__ bool ns_forward_umma256(int m, int T, float eps, float alpha_in, cons
   const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64;
   const int gi = ri * 128 + row, gj0 = ci * 128 + col0;          // this thread's row and first column in the matrix
   const long long mm = (long long)m * m;
-  for (long long e = gt; e < mm; e += gn) {
-    const int i = (int)(e / m), j = (int)(e % m);
-    Wr[e] = W[e] + (i == j ? eps : 0.f);
-  }
+  for (unsigned e = (unsigned)gt; e < (unsigned)mm; e += (unsigned)gn) Wr[e] = W[e] + (e % (unsigned)(m + 1) == 0u ? eps : 0.f);
   phase_sync<4>();
   {
     // Norms: Wr is symmetric bit for bit (|a - b| = |b - a| term by term in the kernel block), so the absolute row sums
