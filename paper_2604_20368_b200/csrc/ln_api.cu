@@ -200,7 +200,15 @@ PoolGeom geom_of(const ln_problem* p) {
   return g;
 }
 
-inline int launch_ok() { return cudaGetLastError() == cudaSuccess ? LN_OK : LN_ERR_CUDA; }
+// A launch that fails is noticed right after it (a later successful call may otherwise hide it) and reported by the
+// entry point when it returns.
+thread_local bool g_launch_failed = false;
+inline void note_launch() { if (cudaPeekAtLastError() != cudaSuccess) g_launch_failed = true; }
+inline int launch_ok() {
+  const bool bad = (cudaGetLastError() != cudaSuccess) || g_launch_failed;
+  g_launch_failed = false;
+  return bad ? LN_ERR_CUDA : LN_OK;
+}
 inline unsigned cdiv(long long a, long long b) { return (unsigned)((a + b - 1) / b); }
 
 // Profiling aid: when switched on by ln_trace_begin every launch is bracketed by two CUDA events
@@ -223,7 +231,7 @@ struct TraceScope {
   }
   ~TraceScope() { if (slot >= 0) cudaEventRecord(g_trace.ev[2 * slot + 1], st); }
 };
-#define LN_LAUNCH(name, st, ...) do { TraceScope ts_(name, st); __VA_ARGS__; } while (0)
+#define LN_LAUNCH(name, st, ...) do { TraceScope ts_(name, st); __VA_ARGS__; note_launch(); } while (0)
 
 // Side stream.  The per-head kernels (Newton-Schulz and its adjoint: one CTA or cluster per head, bound by the
 // latency of a chain of small products) do not depend on the token-sized kernels next to them, so the entry
@@ -445,18 +453,22 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const float* mu = p->map_mode == 1 ? x.mu : nullptr;
   if (dev_status) cudaMemsetAsync(dev_status, 0, sizeof(int32_t) * BH, st);
   // query side: Z'^T dO and column sums of dO; g^C = (dO Ytilde^T) o C / lambda; dQ; landmark part
-  if constexpr (std::is_same<T, bf16>::value) {
+  if constexpr (std::is_same<T, bf16>::value)
     LN_LAUNCH("tn_dY", st, k_tn_mma<D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
-    if constexpr (D == 64 || D == 128) {
-      cudaFuncSetAttribute(k_ntg_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ntg_umma_smem<D>());
-      LN_LAUNCH("ntg_C", st, k_ntg_umma<D><<<dim3(cdiv(n, 128), BH), 256, ntg_umma_smem<D>(), st>>>(dO, reinterpret_cast<const bf16*>(x.Yimg), x.C, pl.ldm,
-                                                                                                w.G, n, m, inv_lambda, dev_status));
-    } else
-    LN_LAUNCH("ntg_C", st, k_nt_g_mma<D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(dO, x.Yt, x.C, pl.ldm, w.G, n, m, inv_lambda));
-  } else {
+  else
     LN_LAUNCH("tn_dY", st, k_tn<T, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
-    LN_LAUNCH("ntg_C", st, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(dO, x.Yt, x.C, pl.ldm, w.G, n, m, inv_lambda));
-  }
+  auto launch_ntg_C = [&]() {
+    if constexpr (std::is_same<T, bf16>::value) {
+      if constexpr (D == 64 || D == 128) {
+        cudaFuncSetAttribute(k_ntg_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ntg_umma_smem<D>());
+        LN_LAUNCH("ntg_C", st, k_ntg_umma<D><<<dim3(cdiv(n, 128), BH), 256, ntg_umma_smem<D>(), st>>>(dO, reinterpret_cast<const bf16*>(x.Yimg), x.C, pl.ldm,
+                                                                                                  w.G, n, m, inv_lambda, dev_status));
+      } else
+        LN_LAUNCH("ntg_C", st, k_nt_g_mma<D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(dO, x.Yt, x.C, pl.ldm, w.G, n, m, inv_lambda));
+    } else {
+      LN_LAUNCH("ntg_C", st, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, st>>>(dO, x.Yt, x.C, pl.ldm, w.G, n, m, inv_lambda));
+    }
+  };
   const bool fused_sign = pl.s2_chunks > 0;
   const int chs = fused_sign ? pl.s2_chunks : ch;
   const int chq = fused_sign ? pl.s2q_chunks : ch;    // chunks of the query-side landmark-gradient partials
@@ -481,10 +493,11 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // key-side products: g^R = (V dM^T) o R^T / lambda and dV = R^T dM (they need dM from the per-head kernel)
   auto launch_ntg_R = [&](cudaStream_t s) {
     if constexpr (std::is_same<T, bf16>::value) {
-      if constexpr (D == 64 || D == 128)
+      if constexpr (D == 64 || D == 128) {
+        cudaFuncSetAttribute(k_ntg_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ntg_umma_smem<D>());
         LN_LAUNCH("ntg_R", s, k_ntg_umma<D><<<dim3(cdiv(n, 128), BH), 256, ntg_umma_smem<D>(), s>>>(V, reinterpret_cast<const bf16*>(w.dMimg), x.Rt, pl.ldm,
                                                                                                 w.G2, n, m, inv_lambda, dev_status));
-      else
+      } else
         LN_LAUNCH("ntg_R", s, k_nt_g_mma<D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, s>>>(V, w.dM, x.Rt, pl.ldm, w.G2, n, m, inv_lambda));
     } else {
       LN_LAUNCH("ntg_R", s, k_nt_g<T, D><<<dim3(cdiv(n, 64), cdiv(m, 64), BH), 256, 0, s>>>(V, w.dM, x.Rt, pl.ldm, w.G2, n, m, inv_lambda));
@@ -519,6 +532,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     launch_nn_dV(side.s);
     launch_sign_W(side.s);
   }
+  launch_ntg_C();
   if (fused_sign) {
     auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.s2_smem);
