@@ -955,7 +955,9 @@ __global__ void __launch_bounds__(256) k_ns_pinv_bwd(int m, int T, float eps, fl
 // then fold the injective map (Prop. 3) into Ytilde_l = s_l Y_l - mean_l'(s_l' Y_l'), ybar = mean_l Y_l
 // so that O = (C - mu) Ytilde + ybar.  One CTA per head.
 // =====================================================================================
-// CL > 1 (generic path only): CL CTAs of a thread-block cluster share one head; grid = heads * CL.
+// MP: 0 = matrices in global memory (fp32 FFMA or the cluster-shared mma.sync engine); 64 / 128 = one CTA per head on
+// tcgen05 with the matrix padded to MP; 256 = tcgen05 on 2 x 2 blocks of 128, CL = 4 CTAs of a thread-block cluster
+// per head (grid = heads * CL).
 template <int D, bool TC, int MP, int CL = 1>
 __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 : 1)) k_mid_fwd(int m, int ldm, int T, float eps, float alpha_in, int H, int map_mode,
                                                  const float* __restrict__ whiten, const float* W, float* Wr,
@@ -966,7 +968,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
   // The two halves may run as two launches, the first beside the kernels that produce M; X_T passes through
   // global memory either way.
   // Yimg: NULL, or where Ytilde is also left as split operand images per 64-landmark block (for the tcgen05 product)
-  // hslot: floats per slot of the iterate histories (used by the MP = 64 path, whose slots hold operand images)
+  // hslot: floats per slot of the iterate histories (the tcgen05 paths, whose slots hold operand images)
   // dynamic shared memory: the Newton-Schulz matrices (MP > 0), reused afterwards by the GEMM engine
   extern __shared__ __align__(16) unsigned char dyn_smem[];
   NsSmem& sm = *reinterpret_cast<NsSmem*>(dyn_smem);
@@ -974,7 +976,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
   const int bh = blockIdx.x / CL, crank = blockIdx.x % CL, tid = threadIdx.x;
   const int gt = crank * 256 + tid, gn = 256 * CL;      // this thread among all threads that share the head
   const long long mm = (long long)m * m, md = (long long)m * D;
-  // the iterate histories of the shared-memory path use the padded leading dimension (128-bit accesses)
+  // X_T of the single-CTA tcgen05 paths uses the padded leading dimension (128-bit accesses)
   const int ldx = (MP == 64 || MP == 128) ? ldm : m;
   const long long mx = (MP > 0) ? hslot : (long long)m * ldx;
   const long long wslot = (MP == 256) ? kU2Slot : mm;           // floats per scratch matrix
