@@ -276,7 +276,9 @@ def run_ours(args):
         step(i)
     sampler = ClockSampler(local) if rank == 0 else None
     t_begin = time.perf_counter()
+    launches_before = ln.launch_count()
     ms = timed(step, args.steps)
+    launches_timed = ln.launch_count() - launches_before      # kernels of this library inside the timed region
     t_end = time.perf_counter()
     tokens = cfg.B * cfg.n * world
     value = tokens * args.steps / (ms * 1e-3)
@@ -382,7 +384,7 @@ def run_ours(args):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": workload_dict(cfg, {"l2": f"rotating {nsets} input sets ({nsets * in_bytes / 1e6:.0f} MB > 126 MB L2)",
                                       "parallelism": f"replicas x{world} (heads independent, no collective)"}),
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_timed,
         "roofline": roofline, "kernels": kernels,
     }
     if not args.no_cpu_baseline and world == 1:

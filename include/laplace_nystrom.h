@@ -211,6 +211,12 @@ int ln_trace_end(int32_t capacity, int32_t* count, float* ms, const char** names
  */
 int ln_set_overlap(int enabled);
 
+/*
+ * Number of kernels this library has launched in the process so far (the paper has no counterpart; a bookkeeping aid
+ * for benchmarks that report how many launches a timed region held: read it before and after).
+ */
+uint64_t ln_launch_count(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,7 +25,7 @@ EXPORTS = [
     "laplace_nystrom_fwd", "laplace_nystrom_bwd", "ns_pinv_workspace_bytes", "ns_pinv", "ns_pinv_bwd",
     "l1_kernel", "l1_kernel_bwd_workspace_bytes", "l1_kernel_bwd", "landmarks_pool", "landmarks_pool_bwd",
     "ln_trace_begin", "ln_trace_end", "ns_pinv_static_scratch_bytes", "ns_pinv_static",
-    "laplace_nystrom_host_staging_bytes", "laplace_nystrom_fwd_bwd_host", "ln_set_overlap",
+    "laplace_nystrom_host_staging_bytes", "laplace_nystrom_fwd_bwd_host", "ln_set_overlap", "ln_launch_count",
 ]
 
 
@@ -126,6 +126,8 @@ def lib():
         L.ns_pinv_static.argtypes = [i32, i32, vp, i32, f32, f32, vp, vp, vp]
         L.ln_trace_end.argtypes = [i32, ctypes.POINTER(i32), ctypes.POINTER(f32), ctypes.POINTER(ctypes.c_char_p)]
         L.ln_set_overlap.argtypes = [i32]
+        L.ln_launch_count.restype = ctypes.c_uint64
+        L.ln_launch_count.argtypes = []
         _lib = L
     return _lib
 
@@ -313,6 +315,11 @@ def set_overlap(enabled: bool) -> bool:
     """Whether the per-head kernels run on the library's second stream beside the token-sized ones
     (default on); returns the previous setting."""
     return bool(lib().ln_set_overlap(1 if enabled else 0))
+
+
+def launch_count() -> int:
+    """Kernels the library has launched in this process so far."""
+    return int(lib().ln_launch_count())
 
 
 # ------------------------------------------------------------------------------------------ profiling aid

@@ -6,6 +6,7 @@
 #include "../../include/laplace_nystrom.h"
 #include "ln_kernels.cuh"
 #include "ln_sign2.cuh"
+#include <atomic>
 #include <mutex>
 #include <type_traits>
 
@@ -203,7 +204,11 @@ PoolGeom geom_of(const ln_problem* p) {
 // A launch that fails is noticed right after it (a later successful call may otherwise hide it) and reported by the
 // entry point when it returns.
 thread_local bool g_launch_failed = false;
-inline void note_launch() { if (cudaPeekAtLastError() != cudaSuccess) g_launch_failed = true; }
+std::atomic<unsigned long long> g_launch_count{0};      // kernels launched by this library since it was loaded
+inline void note_launch() {
+  g_launch_count.fetch_add(1, std::memory_order_relaxed);
+  if (cudaPeekAtLastError() != cudaSuccess) g_launch_failed = true;
+}
 inline int launch_ok() {
   const bool bad = (cudaGetLastError() != cudaSuccess) || g_launch_failed;
   g_launch_failed = false;
@@ -658,6 +663,8 @@ int ln_trace_end(int32_t capacity, int32_t* count, float* ms, const char** names
   for (int i = 0; i < 2 * kTraceCap; ++i) cudaEventDestroy(g_trace.ev[i]);
   return status;
 }
+
+uint64_t ln_launch_count(void) { return (uint64_t)g_launch_count.load(std::memory_order_relaxed); }
 
 int ln_set_overlap(int enabled) {
   std::lock_guard<std::mutex> lk(g_side_mu);

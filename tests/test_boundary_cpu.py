@@ -15,7 +15,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def declared_symbols():
     text = open(os.path.join(ROOT, "include", "laplace_nystrom.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    names = re.findall(r"\b(?:int|size_t|const char\*)\s+(\w+)\s*\(", text)
+    names = re.findall(r"\b(?:int|size_t|uint64_t|const char\*)\s+(\w+)\s*\(", text)
     return sorted(set(names))
 
 
