@@ -129,3 +129,13 @@ def test_host_step_argument_errors_without_gpu():
     assert call(cp, None, need) == -1                   # NULL staging
     assert call(cp, a, need - 1) == -3                  # staging too small
     assert lib.laplace_nystrom_host_staging_bytes(ctypes.byref(_problem(n=0).c())) == 0
+
+
+def test_overlap_switch_and_launch_counter_without_gpu():
+    """ln_set_overlap returns the previous setting (default on); the launch counter is readable and has not moved
+    without a launch."""
+    assert ln.set_overlap(False) is True
+    assert ln.set_overlap(True) is False
+    assert ln.set_overlap(True) is True
+    c0 = ln.launch_count()
+    assert c0 >= 0 and ln.launch_count() == c0

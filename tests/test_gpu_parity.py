@@ -193,6 +193,16 @@ def test_ragged_shapes(gh, gw, mh, mw, prefix, d, dtype):
     _run_case(cfg)
 
 
+# Every size class of the tcgen05 Newton-Schulz engines (M = 64 accumulators, M = 128, 2 x 2 blocks shared by a
+# cluster) at its edges: m just above a class boundary, m one short of the padded size, and zero, one and several steps.
+@pytest.mark.parametrize("mh,mw", [(1, 1), (7, 9), (8, 8), (5, 13), (8, 16), (10, 13), (15, 17), (16, 16)])
+@pytest.mark.parametrize("T", [0, 1, 3])
+def test_newton_schulz_engines_at_their_edges(mh, mw, T):
+    cfg = synth.Config("ns_edges", B=1, H=2, d=64, m=mh * mw, T=T, gh=20, gw=20, mh=mh, mw=mw, prefix=1,
+                       dtype="bf16", seed=123 + mh * mw + T)
+    _run_case(cfg)
+
+
 def test_many_heads_several_chunks():
     """Few heads and many tokens: the landmark gradient is summed over several token chunks per head."""
     cfg = synth.Config("chunks", B=1, H=1, d=64, m=32, T=4, gh=96, gw=96, mh=4, mw=8, dtype="bf16", seed=5)
