@@ -458,10 +458,12 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const float* mu = p->map_mode == 1 ? x.mu : nullptr;
   if (dev_status) cudaMemsetAsync(dev_status, 0, sizeof(int32_t) * BH, st);
   // query side: Z'^T dO and column sums of dO; g^C = (dO Ytilde^T) o C / lambda; dQ; landmark part
-  if constexpr (std::is_same<T, bf16>::value)
-    LN_LAUNCH("tn_dY", st, k_tn_mma<D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
-  else
-    LN_LAUNCH("tn_dY", st, k_tn<T, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
+  auto launch_tn_dY = [&](cudaStream_t s) {
+    if constexpr (std::is_same<T, bf16>::value)
+      LN_LAUNCH("tn_dY", s, k_tn_mma<D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, s>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
+    else
+      LN_LAUNCH("tn_dY", s, k_tn<T, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, s>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
+  };
   auto launch_ntg_C = [&]() {
     if constexpr (std::is_same<T, bf16>::value) {
       if constexpr (D == 64 || D == 128) {
@@ -529,8 +531,18 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // joins them where the query-side sign pass is long enough to hide it (large heads); for small heads it follows the
   // first sign pass on the caller's stream, so that only the per-head kernel stands between the two sign passes.
   const bool ntg_on_side = side.on() && (long long)n * m * D > (1ll << 22);
+  // Z'^T dO is needed by the per-head kernel only: it goes to the side stream too unless that stream is expected to be
+  // the longer one anyway (estimates in microseconds: 7 / 16 / 30 per step and wave of heads for m <= 64 / <= 128 /
+  // larger; the sign pass at 0.43 of the FP32 peak, 0.25 for small launches)
+  const int mid_waves = (int)(m <= 64 ? cdiv(BH, 3 * kSMs) : (m <= 128 ? cdiv(BH, kSMs) : cdiv(4ll * BH, kSMs)));
+  const double side_us = pl.T * (m <= 64 ? 7.0 : (m <= 128 ? 16.0 : 30.0)) * mid_waves;
+  const double sign_ops = 3.0 * n * m * D * BH;
+  const double main_us = sign_ops / (37.2e6 * (sign_ops > 4e9 ? 0.43 : 0.25));
+  const bool tn_on_side = side.on() && side_us < 0.8 * main_us;
+  if (!tn_on_side) launch_tn_dY(st);
   if (side.on()) {
     side.fork(st);
+    if (tn_on_side) launch_tn_dY(side.s);
     launch_mid(side.s);
     if (ntg_on_side) launch_ntg_R(side.s);
     side.mark();                     // what the second sign pass needs from this stream ends here
