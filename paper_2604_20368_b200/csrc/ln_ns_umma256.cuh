@@ -11,7 +11,7 @@
 // wrote.  The images the forward pass leaves (X_k, Q_k = 2I - W X_k) are the history the adjoint fetches.
 // Transposes cost nothing: an image is read K-major or MN-major through the descriptor.
 //
-// Shared memory: operand buffers sA, sB and the output image sC (3 x 64 KiB).  Thread t owns row
+// Shared memory: three 64 KiB buffers, operand blocks in rotation and the output image (sC).  Thread t owns row
 // 32 (warp % 4) + lane of its CTA's block and the column half warp / 4 (as on the 128 x 128 path).
 // Every wait is bounded; a wait that runs out is reported to the caller (results are then wrong, nothing hangs:
 // all threads of all four CTAs still reach every cluster barrier).
@@ -43,27 +43,34 @@ struct U2Ctx {
 // Writes of other CTAs to global memory (bulk copies, then the cluster barrier) are read here by bulk copies.
 __device__ __forceinline__ void u2_fence_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// All terms, one after the other through the two operand buffers; one thread fetches and issues, everybody waits for
-// the last MMA.
+// All terms, one after the other; one thread fetches and issues, everybody waits for the last MMA.  The three buffers
+// (all free between products: the output image is written after the last MMA) rotate so that the A block of the next
+// term is fetched while the MMAs of this one run; its B block follows as soon as they have completed.
+//   term i: A in buffer 2i mod 3, B in buffer (2i + 1) mod 3
 template <int NT>
 __device__ __forceinline__ void u2_run(U2Ctx& c, const U2Term (&t)[NT]) {
   constexpr uint32_t MATB = (uint32_t)kUmmaMatBytes;
   if (threadIdx.x == 0) {
+    bf16* const buf[3] = {c.sA, c.sB, c.sC};
     u2_fence_async();
+    umma::mbar_expect_tx(&c.ctl->mbar_ld, 2 * MATB);
+    umma::bulk_load(buf[0], t[0].A, MATB, &c.ctl->mbar_ld);
+    umma::bulk_load(buf[1], t[0].B, MATB, &c.ctl->mbar_ld);
 #pragma unroll 1
     for (int i = 0; i < NT; ++i) {
-      if (i > 0) {                               // the previous term has finished reading the buffers
-        umma::commit(c.mbar_free);
-        c.ok &= umma::mbar_wait(c.mbar_free, c.ph_free & 1);
-        c.ph_free ^= 1u;
-      }
-      umma::mbar_expect_tx(&c.ctl->mbar_ld, 2 * MATB);
-      umma::bulk_load(c.sA, t[i].A, MATB, &c.ctl->mbar_ld);
-      umma::bulk_load(c.sB, t[i].B, MATB, &c.ctl->mbar_ld);
+      const int ia = (2 * i) % 3, ib = (2 * i + 1) % 3;
       c.ok &= umma::mbar_wait(&c.ctl->mbar_ld, c.ph_ld & 1);
       c.ph_ld ^= 1u;
       umma::fence_after_sync();
-      umma_gemm<128>(t[i].tmem_d, c.sA, t[i].a_k, c.sB, t[i].b_k, t[i].accumulate);
+      umma_gemm<128>(t[i].tmem_d, buf[ia], t[i].a_k, buf[ib], t[i].b_k, t[i].accumulate);
+      if (i + 1 < NT) {
+        umma::mbar_expect_tx(&c.ctl->mbar_ld, 2 * MATB);
+        umma::bulk_load(buf[(2 * i + 2) % 3], t[i + 1].A, MATB, &c.ctl->mbar_ld);   // free since term i - 1 completed
+        umma::commit(c.mbar_free);                                                   // term i has finished reading
+        c.ok &= umma::mbar_wait(c.mbar_free, c.ph_free & 1);
+        c.ph_free ^= 1u;
+        umma::bulk_load(buf[(2 * i + 3) % 3], t[i + 1].B, MATB, &c.ctl->mbar_ld);   // the buffer of this term's A
+      }
     }
     umma::commit(&c.ctl->mbar);
     if (!c.ok) c.ctl->timeout = 1;
