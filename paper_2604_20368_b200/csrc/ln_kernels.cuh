@@ -743,7 +743,7 @@ __device__ void cta_gemm(int M, int N, int K, const float* A, int lda, const flo
 }
 
 // Shared memory of the per-head kernels: one of the two GEMM engines is used per instantiation.
-union __align__(16) NsSmem { GemmSmem f; MmaGemmSmem t; MmaGemmSmemBig b; };
+union __align__(16) NsSmem { GemmSmem f; MmaGemmSmem t; };
 
 // C = beta*Cin + alpha*op(A)op(B) + diag*I on either engine: TC = tensor cores with split-bf16
 // operands (bf16-storage path), else exact fp32 FFMA (fp32-storage path, stand-alone ns_pinv).
@@ -752,9 +752,7 @@ __device__ __forceinline__ void ns_gemm(int M, int N, int K, const float* A, int
                                         float* C, int ldc, float alpha, float beta, const float* Cin, float diag,
                                         NsSmem& sm, int part = 0, int nparts = 1) {
   if (TC) {
-    // the 128 x 128-tile engine is compiled only where m can exceed 128 (it costs registers)
-    if (BIG && M > 128 && N > 64) cta_gemm_mma_big<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.b, part, nparts);
-    else cta_gemm_mma<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.t, part, nparts);
+    cta_gemm_mma<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.t, part, nparts);
   } else {
     cta_gemm<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, sm.f);
     if (diag != 0.f) {

@@ -455,127 +455,5 @@ __device__ void cta_gemm_mma(int M, int N, int K, const float* A, int lda, const
   __syncthreads();
 }
 
-// Same contract as cta_gemm_mma with 128 x 128 output tiles (8 warps = 4 row blocks of 32 x 2 column halves
-// of 64): four times the tensor-core work per staged K-chunk, for the m = 256 matrices whose operands do
-// not fit in shared memory.
-struct __align__(16) MmaGemmSmemBig {
-  bf16 Ah[5120], Al[5120], Bh[5120], Bl[5120];   // [128][40] or [32][136] bf16
-};
-
-template <bool WIDE>   // WIDE: 32 rows x 128 cols ([32][136]), else 128 rows x 32 cols ([128][40]); 16 floats per thread
-__device__ __forceinline__ void gemm_fetch_big(const float* src, int ld, int r0, int c0, int rmax, int cmax, float (&v)[16]) {
-  const int tid = threadIdx.x;
-  const int r = WIDE ? (tid >> 3) : (tid >> 1), c = WIDE ? (tid & 7) * 16 : (tid & 1) * 16;
-  const int gr = r0 + r, gc = c0 + c;
-  const float* p = src + (long long)gr * ld + gc;
-  if (gr < rmax && gc + 15 < cmax && (ld & 3) == 0 && (gc & 3) == 0) {
-#pragma unroll
-    for (int q = 0; q < 16; q += 4) {
-      const float4 a = *reinterpret_cast<const float4*>(p + q);
-      v[q] = a.x; v[q + 1] = a.y; v[q + 2] = a.z; v[q + 3] = a.w;
-    }
-  } else {
-#pragma unroll
-    for (int q = 0; q < 16; ++q) v[q] = (gr < rmax && gc + q < cmax) ? p[q] : 0.f;
-  }
-}
-template <bool WIDE>
-__device__ __forceinline__ void gemm_stash_big(bf16* hi, bf16* lo, const float (&v)[16]) {
-  const int tid = threadIdx.x;
-  const int r = WIDE ? (tid >> 3) : (tid >> 1), c = WIDE ? (tid & 7) * 16 : (tid & 1) * 16;
-  constexpr int LD = WIDE ? 136 : 40;
-#pragma unroll
-  for (int q = 0; q < 16; q += 8) {
-    uint2 h0, l0, h1, l1;
-    split4(make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]), h0, l0);
-    split4(make_float4(v[q + 4], v[q + 5], v[q + 6], v[q + 7]), h1, l1);
-    *reinterpret_cast<uint4*>(hi + r * LD + c + q) = make_uint4(h0.x, h0.y, h1.x, h1.y);
-    *reinterpret_cast<uint4*>(lo + r * LD + c + q) = make_uint4(l0.x, l0.y, l1.x, l1.y);
-  }
-}
-
-template <bool TRA, bool TRB>
-__device__ void cta_gemm_mma_big(int M, int N, int K, const float* A, int lda, const float* Bm, int ldb, float* C,
-                                 int ldc, float alpha, float beta, const float* Cin, float diag, MmaGemmSmemBig& sm,
-                                 int part = 0, int nparts = 1) {
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int wm = (warp & 3) * 32, wn = (warp >> 2) * 64;
-  const int g = lane >> 2, t4 = lane & 3;
-  int tile_no = 0;
-  for (int i0 = 0; i0 < M; i0 += 128)
-    for (int j0 = 0; j0 < N; j0 += 128) {
-      if ((tile_no++) % nparts != part) continue;
-      float acc[2][8][4];
-#pragma unroll
-      for (int a = 0; a < 2; ++a)
-#pragma unroll
-        for (int t = 0; t < 8; ++t)
-#pragma unroll
-          for (int q = 0; q < 4; ++q) acc[a][t][q] = 0.f;
-      float va[16], vb[16];
-      if (TRA) gemm_fetch_big<true>(A, lda, 0, i0, K, M, va); else gemm_fetch_big<false>(A, lda, i0, 0, M, K, va);
-      if (TRB) gemm_fetch_big<false>(Bm, ldb, j0, 0, N, K, vb); else gemm_fetch_big<true>(Bm, ldb, 0, j0, K, N, vb);
-      for (int k0 = 0; k0 < K; k0 += 32) {
-        __syncthreads();
-        gemm_stash_big<TRA>(sm.Ah, sm.Al, va);
-        gemm_stash_big<!TRB>(sm.Bh, sm.Bl, vb);
-        __syncthreads();
-        if (k0 + 32 < K) {
-          if (TRA) gemm_fetch_big<true>(A, lda, k0 + 32, i0, K, M, va); else gemm_fetch_big<false>(A, lda, i0, k0 + 32, M, K, va);
-          if (TRB) gemm_fetch_big<false>(Bm, ldb, j0, k0 + 32, N, K, vb); else gemm_fetch_big<true>(Bm, ldb, k0 + 32, j0, K, N, vb);
-        }
-#pragma unroll
-        for (int kk = 0; kk < 32; kk += 16) {
-          uint32_t ah[2][4], al[2][4], bh4[4][4], bl4[4][4];
-#pragma unroll
-          for (int a = 0; a < 2; ++a) {
-            if (TRA) { ldsm_x4_t(ah[a], addr_at(sm.Ah, 136, kk, wm + a * 16)); ldsm_x4_t(al[a], addr_at(sm.Al, 136, kk, wm + a * 16)); }
-            else     { ldsm_x4(ah[a], addr_a(sm.Ah, 40, wm + a * 16, kk));     ldsm_x4(al[a], addr_a(sm.Al, 40, wm + a * 16, kk)); }
-          }
-#pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            if (TRB) { ldsm_x4(bh4[t], addr_b(sm.Bh, 40, wn + t * 16, kk));     ldsm_x4(bl4[t], addr_b(sm.Bl, 40, wn + t * 16, kk)); }
-            else     { ldsm_x4_t(bh4[t], addr_bt(sm.Bh, 136, kk, wn + t * 16)); ldsm_x4_t(bl4[t], addr_bt(sm.Bl, 136, kk, wn + t * 16)); }
-          }
-#pragma unroll
-          for (int a = 0; a < 2; ++a)
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-              mma_bf16(acc[a][2 * t], al[a], bh4[t][0], bh4[t][1]);
-              mma_bf16(acc[a][2 * t + 1], al[a], bh4[t][2], bh4[t][3]);
-            }
-#pragma unroll
-          for (int a = 0; a < 2; ++a)
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-              mma_bf16(acc[a][2 * t], ah[a], bl4[t][0], bl4[t][1]);
-              mma_bf16(acc[a][2 * t + 1], ah[a], bl4[t][2], bl4[t][3]);
-            }
-#pragma unroll
-          for (int a = 0; a < 2; ++a)
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-              mma_bf16(acc[a][2 * t], ah[a], bh4[t][0], bh4[t][1]);
-              mma_bf16(acc[a][2 * t + 1], ah[a], bh4[t][2], bh4[t][3]);
-            }
-        }
-      }
-#pragma unroll
-      for (int a = 0; a < 2; ++a)
-#pragma unroll
-        for (int t = 0; t < 8; ++t)
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const int i = i0 + wm + a * 16 + g + (q >> 1) * 8, j = j0 + wn + t * 8 + 2 * t4 + (q & 1);
-            if (i < M && j < N) {
-              float v = alpha * acc[a][t][q];
-              if (beta != 0.f) v += beta * Cin[(long long)i * ldc + j];
-              if (i == j) v += diag;
-              C[(long long)i * ldc + j] = v;
-            }
-          }
-    }
-  __syncthreads();
-}
 
 }  // namespace ln
