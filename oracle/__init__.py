@@ -181,3 +181,30 @@ def backward(p: Problem, Q, K, V, dO, L=None, whiten=None):
     _load().oracle_bwd(ctypes.byref(cp), _p(Q), _p(K), _p(V), _p(L), _p(whiten), _p(dO),
                        _p(dQ), _p(dK), _p(dV), _p(dL))
     return dQ, dK, dV, dL
+
+
+def whiten_stats(C, H, eps_w):
+    """Diagonal whitening scale of Eq. 5-6 from the query-landmark kernel block.
+
+    C: [B*H, n, m] (heads of one batch element contiguous, flat index b*H + h).  For head h and landmark l the
+    "batch of vectors" of Eq. 5 is every query row of every batch element: mu_l = mean over (b, i) of C_il,
+    sigma_l^2 = mean over (b, i) of (C_il - mu_l)^2 (the 1/B form of Eq. 5, no Bessel correction), and
+    s_l = 1 / sqrt(sigma_l^2 + eps_w) (the diagonal of D^{-1/2}, Eq. 6).  Returns s [H, m].  Two passes, float64."""
+    C = np.asarray(C, dtype=np.float64)
+    BH, n, m = C.shape
+    B = BH // H
+    s = np.empty((H, m))
+    for h in range(H):
+        rows = np.concatenate([C[b * H + h] for b in range(B)], axis=0)      # [B*n, m]
+        cnt = rows.shape[0]
+        mu = np.zeros(m)
+        for i in range(cnt):
+            mu += rows[i]
+        mu /= cnt
+        var = np.zeros(m)
+        for i in range(cnt):
+            t = rows[i] - mu
+            var += t * t
+        var /= cnt
+        s[h] = 1.0 / np.sqrt(var + eps_w)
+    return s

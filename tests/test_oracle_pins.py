@@ -342,3 +342,27 @@ def test_full_backward_finite_differences(lm_mode, map_mode, use_s):
             assert dL[idx] == pytest.approx(fd, rel=5e-6, abs=1e-8)
     else:
         assert dL is None
+
+
+def test_whiten_stats_hand_values_and_invariants():
+    """Eq. 5-6: population variance over the batch of query rows, scale 1/sqrt(sigma^2 + eps)."""
+    C = np.array([[[1.0, 7.0], [2.0, 7.0], [3.0, 7.0], [4.0, 7.0]]])            # one head, four rows, two landmarks
+    s = oracle.whiten_stats(C, 1, 0.35)
+    assert abs(s[0, 0] - GOLD["whiten_scale_1234"]) < 1e-15
+    assert abs(oracle.whiten_stats(C, 1, 0.25)[0, 1] - GOLD["whiten_scale_constant"]) < 1e-15
+    rng = np.random.default_rng(5)
+    B, H, n, m = 3, 2, 17, 5
+    C = rng.uniform(0.2, 0.8, (B * H, n, m))
+    s = oracle.whiten_stats(C, H, 1e-5)
+    # against the library's population variance, on the rows of a head gathered over the batch
+    for h in range(H):
+        rows = np.concatenate([C[b * H + h] for b in range(B)], axis=0)
+        assert np.allclose(s[h], 1.0 / np.sqrt(rows.var(axis=0) + 1e-5), rtol=1e-12)
+    # the order of the batch elements and a shift of a column do not matter; a scale a multiplies sigma by |a|
+    perm = np.concatenate([np.arange(H) + b * H for b in (2, 0, 1)])
+    assert np.allclose(oracle.whiten_stats(C[perm], H, 1e-5), s, rtol=1e-12)
+    assert np.allclose(oracle.whiten_stats(C + 3.0, H, 1e-5), s, rtol=1e-9)
+    assert np.allclose(oracle.whiten_stats(-2.0 * C, H, 0.0), oracle.whiten_stats(C, H, 0.0) / 2.0, rtol=1e-12)
+    # heads do not mix: changing head 1 leaves the scale of head 0 alone
+    C2 = C.copy(); C2[1::H] *= 1.7
+    assert np.array_equal(oracle.whiten_stats(C2, H, 1e-5)[0], s[0])
