@@ -180,6 +180,21 @@ int l1_kernel_bwd(int32_t batch, int32_t na, int32_t nb, int32_t d, const void* 
                   void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Whitening statistics (Eq. 5 and Eq. 6): the diagonal scale s [H, m] that `whiten` takes, estimated from the
+ * query-landmark kernel block C = k(Q, L) that laplace_nystrom_fwd left in `saved`.  For head h and landmark l the
+ * batch of Eq. 5 is every query row of every batch element:
+ *     mu_l = mean_{b,i} C_il,   sigma_l^2 = mean_{b,i} (C_il - mu_l)^2   (the 1/B form of Eq. 5),
+ *     s_l  = 1 / sqrt(sigma_l^2 + eps_w)                                  (the diagonal of D^{-1/2}, Eq. 6).
+ * saved: the context of a forward call on the same problem (device).  whiten_out: device [H, m] fp32, overwritten.
+ * ws: device scratch of laplace_nystrom_whiten_stats_workspace_bytes(p) bytes.  Sums are taken in double in a fixed
+ * order (results are reproducible).  The scale is a constant of the attention entry points (no gradient flows through
+ * it), as when the paper estimates it offline.  Errors as above; eps_w < 0 or not finite is LN_ERR_ARG.
+ */
+size_t laplace_nystrom_whiten_stats_workspace_bytes(const ln_problem* p);
+int laplace_nystrom_whiten_stats(const ln_problem* p, const void* saved, float eps_w, float* whiten_out, void* ws,
+                                 size_t ws_bytes, void* stream);
+
+/*
  * Landmark selection by average pooling of the keys over the token grid (Sec. 4.2), lm_mode 1
  * geometry of `p`.  K [B,H,n,d] dtype -> L [B,H,m,d] fp32.  The backward overwrites dK [B,H,n,d]
  * (dtype) with pool^T(dL), dL [B,H,m,d] fp32.

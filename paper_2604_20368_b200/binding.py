@@ -26,6 +26,7 @@ EXPORTS = [
     "l1_kernel", "l1_kernel_bwd_workspace_bytes", "l1_kernel_bwd", "landmarks_pool", "landmarks_pool_bwd",
     "ln_trace_begin", "ln_trace_end", "ns_pinv_static_scratch_bytes", "ns_pinv_static",
     "laplace_nystrom_host_staging_bytes", "laplace_nystrom_fwd_bwd_host", "ln_set_overlap", "ln_launch_count",
+    "laplace_nystrom_whiten_stats_workspace_bytes", "laplace_nystrom_whiten_stats",
 ]
 
 
@@ -128,6 +129,9 @@ def lib():
         L.ln_set_overlap.argtypes = [i32]
         L.ln_launch_count.restype = ctypes.c_uint64
         L.ln_launch_count.argtypes = []
+        L.laplace_nystrom_whiten_stats_workspace_bytes.restype = sz
+        L.laplace_nystrom_whiten_stats_workspace_bytes.argtypes = [ctypes.POINTER(_CProblem)]
+        L.laplace_nystrom_whiten_stats.argtypes = [ctypes.POINTER(_CProblem), vp, f32, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -315,6 +319,21 @@ def set_overlap(enabled: bool) -> bool:
     """Whether the per-head kernels run on the library's second stream beside the token-sized ones
     (default on); returns the previous setting."""
     return bool(lib().ln_set_overlap(1 if enabled else 0))
+
+
+def laplace_nystrom_whiten_stats(p: Problem, saved, eps_w: float = 1e-5, out=None, ws=None, stream=None):
+    """Whitening scale s [H, m] (Eq. 5-6) from the kernel block a forward call left in ``saved``."""
+    if saved is None or not saved.is_cuda:
+        raise ValueError("saved must be the CUDA context buffer of a forward call")
+    cp = p.c()
+    need = lib().laplace_nystrom_whiten_stats_workspace_bytes(ctypes.byref(cp))
+    if ws is None:
+        ws = torch.empty(max(need, 256), dtype=torch.uint8, device=saved.device)
+    if out is None:
+        out = torch.empty((p.H, p.m), dtype=torch.float32, device=saved.device)
+    _check(lib().laplace_nystrom_whiten_stats(ctypes.byref(cp), _ptr(saved), eps_w, _ptr(out), _ptr(ws), ws.numel(),
+                                              _stream(stream)), "laplace_nystrom_whiten_stats")
+    return out
 
 
 def launch_count() -> int:

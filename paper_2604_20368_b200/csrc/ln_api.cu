@@ -750,6 +750,46 @@ int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const
   return bwd_dispatch_d<bf16>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, dev_status, st);
 }
 
+namespace {
+// splits of the token rows per head for the whitening statistics: about four waves of CTAs, at least 64 rows each
+void wstat_plan(const ln_problem* p, int* nsplit, int* rows_per_split) {
+  const int BH = p->B * p->H;
+  int sp = (4 * kSMs + BH - 1) / BH;
+  if (sp > 64) sp = 64;
+  if (sp > (p->n + 63) / 64) sp = (p->n + 63) / 64;
+  if (sp < 1) sp = 1;
+  int rps = (p->n + sp - 1) / sp;
+  rps = (rps + 3) / 4 * 4;
+  *rows_per_split = rps;
+  *nsplit = (p->n + rps - 1) / rps;
+}
+}  // namespace
+
+size_t laplace_nystrom_whiten_stats_workspace_bytes(const ln_problem* p) {
+  if (validate(p) != LN_OK) return 0;
+  int sp, rps; wstat_plan(p, &sp, &rps);
+  return align_up((size_t)p->B * p->H * sp * p->m * 2 * sizeof(double), 256);
+}
+
+int laplace_nystrom_whiten_stats(const ln_problem* p, const void* saved, float eps_w, float* whiten_out, void* ws,
+                                 size_t ws_bytes, void* stream) {
+  int s = validate(p);
+  if (s != LN_OK) return s;
+  if (!saved || !whiten_out || !ws) return LN_ERR_ARG;
+  if (!(eps_w >= 0.f) || !isfinite(eps_w)) return LN_ERR_ARG;
+  if (!aligned16(saved) || !aligned16(whiten_out) || !aligned16(ws)) return LN_ERR_ARG;
+  if (ws_bytes < laplace_nystrom_whiten_stats_workspace_bytes(p)) return LN_ERR_WORKSPACE;
+  Plan pl; make_plan(p, &pl);
+  const Ctx x = carve_ctx(pl, const_cast<void*>(saved));
+  int sp, rps; wstat_plan(p, &sp, &rps);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  double* part = static_cast<double*>(ws);
+  LN_LAUNCH("k_wstat_part", st, k_wstat_part<<<dim3(sp, pl.BH), 256, 0, st>>>(x.C, pl.ldm, p->n, p->m, rps, part));
+  LN_LAUNCH("k_wstat_final", st, k_wstat_final<<<cdiv((long long)p->H * p->m, 128), 128, 0, st>>>(part, x.C, pl.ldm, p->B, p->H, p->n, p->m,
+                                                                                              sp, eps_w, whiten_out));
+  return launch_ok();
+}
+
 size_t laplace_nystrom_host_staging_bytes(const ln_problem* p) {
   if (validate(p) != LN_OK) return 0;
   const size_t one = ((size_t)p->B * p->H * p->n * p->d * (p->dtype == LN_F32 ? 4 : 2) + 255) / 256 * 256;

@@ -166,6 +166,70 @@ __global__ void __launch_bounds__(256, QN == 4 ? 2 : 3) k_l1(const L1Args args) 
   }
 }
 
+// =====================================================================================
+// Whitening statistics (Eq. 5-6): per head h and landmark l, over the query rows of every batch element,
+//     mu_l = mean C_il,  sigma_l^2 = mean (C_il - mu_l)^2,  s_l = 1 / sqrt(sigma_l^2 + eps).
+// k_wstat_part: grid (splits, BH), block 256 = 64 column quads x 4 row lanes; every thread sums its rows of its four
+// columns in double (sum and sum of squares of C - pivot, pivot = the head's first row: the sums stay small), the four
+// row lanes are added in a fixed order, and the split leaves [m][2] doubles.  k_wstat_final: one thread per (h, l)
+// adds the partial sums of all batch elements and splits in a fixed order (the pivots differ per batch element, so the
+// sums are brought to pivot 0 first) and writes s.
+// =====================================================================================
+__global__ void __launch_bounds__(256) k_wstat_part(const float* __restrict__ C, int ldc, int n, int m, int rows_per_split,
+                                                    double* __restrict__ part /* [BH][splits][m][2] */) {
+  __shared__ double red[4][256][2];
+  const int bh = blockIdx.y, split = blockIdx.x, nsplit = gridDim.x;
+  const int cq = threadIdx.x & 63, rl = threadIdx.x >> 6, c0 = cq * 4;
+  const float* Ch = C + (long long)bh * n * ldc;
+  double s1[4] = {0.0, 0.0, 0.0, 0.0}, s2[4] = {0.0, 0.0, 0.0, 0.0};
+  if (c0 < ldc) {
+    const float4 pv = *reinterpret_cast<const float4*>(Ch + c0);                 // pivot: row 0 of this head
+    const int i1 = min(n, (split + 1) * rows_per_split);
+    for (int i = split * rows_per_split + rl; i < i1; i += 4) {
+      const float4 v = *reinterpret_cast<const float4*>(Ch + (long long)i * ldc + c0);
+      const double t0 = (double)v.x - (double)pv.x, t1 = (double)v.y - (double)pv.y;
+      const double t2 = (double)v.z - (double)pv.z, t3 = (double)v.w - (double)pv.w;
+      s1[0] += t0; s1[1] += t1; s1[2] += t2; s1[3] += t3;
+      s2[0] += t0 * t0; s2[1] += t1 * t1; s2[2] += t2 * t2; s2[3] += t3 * t3;
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < 4; ++u) { red[rl][cq * 4 + u][0] = s1[u]; red[rl][cq * 4 + u][1] = s2[u]; }
+  __syncthreads();
+  const int l = threadIdx.x;
+  if (l < m) {
+    const double a = (red[0][l][0] + red[1][l][0]) + (red[2][l][0] + red[3][l][0]);
+    const double b = (red[0][l][1] + red[1][l][1]) + (red[2][l][1] + red[3][l][1]);
+    double* o = part + (((long long)bh * nsplit + split) * m + l) * 2;
+    o[0] = a; o[1] = b;
+  }
+}
+
+__global__ void k_wstat_final(const double* __restrict__ part, const float* __restrict__ C, int ldc, int B, int H, int n, int m,
+                              int nsplit, float eps, float* __restrict__ s_out /* [H][m] */) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= H * m) return;
+  const int h = idx / m, l = idx % m;
+  // sums about pivot p_b become sums about zero: sum x = S1 + N p, sum x^2 = S2 + 2 p S1 + N p^2
+  double sx = 0.0, sxx = 0.0;
+  for (int b = 0; b < B; ++b) {
+    const int bh = b * H + h;
+    const double pv = (double)C[(long long)bh * n * ldc + l];
+    double a = 0.0, q = 0.0;
+    for (int sp = 0; sp < nsplit; ++sp) {
+      const double* o = part + (((long long)bh * nsplit + sp) * m + l) * 2;
+      a += o[0]; q += o[1];
+    }
+    sx += a + (double)n * pv;
+    sxx += q + 2.0 * pv * a + (double)n * pv * pv;
+  }
+  const double cnt = (double)B * (double)n;
+  const double mu = sx / cnt;
+  double var = sxx / cnt - mu * mu;
+  if (var < 0.0) var = 0.0;
+  s_out[idx] = (float)(1.0 / sqrt(var + (double)eps));
+}
+
 // storage type -> fp32 copy
 template <typename T> __global__ void k_to_f32(const T* __restrict__ x, float* __restrict__ y, long long count) {
   long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;

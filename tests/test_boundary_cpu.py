@@ -5,6 +5,7 @@ import os
 import re
 
 import pytest
+import torch
 
 import paper_2604_20368_b200 as ln
 from paper_2604_20368_b200 import binding, synth
@@ -139,3 +140,14 @@ def test_overlap_switch_and_launch_counter_without_gpu():
     assert ln.set_overlap(True) is True
     c0 = ln.launch_count()
     assert c0 >= 0 and ln.launch_count() == c0
+
+
+def test_whiten_stats_argument_errors_without_gpu():
+    p = _problem()
+    cp = p.c()
+    lib = binding.lib()
+    assert lib.laplace_nystrom_whiten_stats_workspace_bytes(ctypes.byref(cp)) > 0
+    # NULL buffers are refused on the host before anything is enqueued
+    assert lib.laplace_nystrom_whiten_stats(ctypes.byref(cp), None, 1e-5, None, None, 0, None) == -1
+    with pytest.raises(ValueError):
+        ln.laplace_nystrom_whiten_stats(p, torch.empty(16, dtype=torch.uint8))

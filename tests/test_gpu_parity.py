@@ -8,7 +8,7 @@ import torch
 import oracle
 import paper_2604_20368_b200 as ln
 from paper_2604_20368_b200 import synth
-from parity import TOL, compare, f64, rel_err, run_gpu, run_oracle_heads
+from parity import TOL, compare, f64, oracle_problem, rel_err, run_gpu, run_oracle_heads
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -327,3 +327,30 @@ def test_host_buffer_step_matches_device_path():
         torch.cuda.synchronize()
         for k in ("O", "dQ", "dK", "dV"):
             assert torch.equal(hout[k], g[k].cpu()), k
+
+
+@pytest.mark.parametrize("name,B", [("cfg1", 1), ("cfg2", 5), ("cfg3", 2), ("cfg4a", 1), ("cfg5_m256_T4", 1)])
+def test_whiten_stats_match_the_oracle(name, B):
+    """Eq. 5-6 on the device (from the kernel block the forward pass saved) against the float64 oracle applied to the
+    oracle's own kernel block; fp32-path bar (the statistic is accumulated in double on both sides)."""
+    cfg = synth.shrink(synth.CONFIGS[name], B=B)
+    inp = synth.make_inputs(cfg)
+    Q, K, V = (inp[k].to(DEV) for k in ("Q", "K", "V"))
+    p = ln.problem_from_config(cfg, whiten=None)
+    saved = torch.empty(ln.laplace_nystrom_saved_bytes(p), dtype=torch.uint8, device=DEV)
+    ln.laplace_nystrom_fwd(p, Q, K, V, saved=saved)
+    eps_w = 1e-5
+    got = ln.laplace_nystrom_whiten_stats(p, saved, eps_w)
+    again = ln.laplace_nystrom_whiten_stats(p, saved, eps_w)
+    torch.cuda.synchronize()
+    assert torch.equal(got, again)                                   # fixed summation order
+    BH = cfg.B * cfg.H
+    op = oracle_problem(cfg)
+    _, extra = oracle.forward(op, f64(inp["Q"]), f64(inp["K"]), f64(inp["V"]), want=("C",))
+    ref = oracle.whiten_stats(extra["C"].reshape(BH, cfg.n, cfg.m), cfg.H, eps_w)
+    assert rel_err(f64(got), ref) < TOL["f32"], (name, rel_err(f64(got), ref))
+    # the estimated scale is accepted as the `whiten` input of the path
+    p2 = ln.problem_from_config(cfg, whiten=got)
+    O = ln.laplace_nystrom_fwd(p2, Q, K, V, saved=saved)
+    o = run_oracle_heads(cfg, {**inp, "whiten": torch.from_numpy(ref).float()}, [0], backward=False)
+    assert rel_err(f64(O).reshape(BH, cfg.n, cfg.d)[[0]], o["O"]) < TOL[cfg.dtype]
