@@ -373,6 +373,33 @@ def run_ours(args):
     path_roof_s = path_ops / (ALU_PEAK_TLANEOPS * 1e12)
     roofline["path_frac"] = path_roof_s / (ms * 1e-3 / args.steps)
 
+    # ---- next step beside the path (Eq. 5-6): the whitening scale estimated on the device from the saved kernel
+    # block C; bound by HBM (C is read once); L2 is flushed before every timed launch
+    whiten_stats = None
+    if cfg.backward:
+        ws_w = torch.empty(256, dtype=torch.uint8, device=dev)
+        flush = torch.zeros(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+        ln.laplace_nystrom_whiten_stats(p, saved, 1e-5)
+        times = []
+        for _ in range(5):               # device time of its two launches (events around each launch, as in the trace above)
+            flush.max()                  # read-only sweep of 256 MB: L2 holds none of C and no dirty lines
+            torch.cuda.synchronize()
+            ln.trace_begin()
+            ln.laplace_nystrom_whiten_stats(p, saved, 1e-5)
+            times.append(sum(t for _, t in ln.trace_end()))
+        del flush, ws_w
+        t_ms = float(np.median(times))
+        ldm = (cfg.m + 3) // 4 * 4
+        c_bytes = cfg.B * cfg.H * cfg.n * ldm * 4
+        peak, src = 6650.0, "fallback 6.65 TB/s"
+        try:
+            peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["hbm_gbs"]); src = "MEASURED_PEAKS.json hbm_gbs"
+        except Exception:
+            pass
+        gbs = c_bytes / (t_ms * 1e-3) / 1e9
+        whiten_stats = {"us": 1e3 * t_ms, "bytes": c_bytes, "bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                        "frac": gbs / peak, "peak_source": src, "launches": 2}
+
     if rank != 0:
         return
     # clocks: samples inside the timed region; a region shorter than three samples (a few ms) is
@@ -387,6 +414,8 @@ def run_ours(args):
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_timed,
         "roofline": roofline, "kernels": kernels,
     }
+    if whiten_stats is not None:
+        out["whiten_stats"] = whiten_stats
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(cfg, inp)
     print(json.dumps(out))

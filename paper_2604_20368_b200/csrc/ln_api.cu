@@ -751,10 +751,10 @@ int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const
 }
 
 namespace {
-// splits of the token rows per head for the whitening statistics: about four waves of CTAs, at least 64 rows each
+// splits of the token rows per head for the whitening statistics: about eight CTAs per SM, at least 64 rows each
 void wstat_plan(const ln_problem* p, int* nsplit, int* rows_per_split) {
   const int BH = p->B * p->H;
-  int sp = (4 * kSMs + BH - 1) / BH;
+  int sp = (8 * kSMs + BH - 1) / BH;
   if (sp > 64) sp = 64;
   if (sp > (p->n + 63) / 64) sp = (p->n + 63) / 64;
   if (sp < 1) sp = 1;
@@ -785,8 +785,7 @@ int laplace_nystrom_whiten_stats(const ln_problem* p, const void* saved, float e
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   double* part = static_cast<double*>(ws);
   LN_LAUNCH("k_wstat_part", st, k_wstat_part<<<dim3(sp, pl.BH), 256, 0, st>>>(x.C, pl.ldm, p->n, p->m, rps, part));
-  LN_LAUNCH("k_wstat_final", st, k_wstat_final<<<cdiv((long long)p->H * p->m, 128), 128, 0, st>>>(part, x.C, pl.ldm, p->B, p->H, p->n, p->m,
-                                                                                              sp, eps_w, whiten_out));
+  LN_LAUNCH("k_wstat_final", st, k_wstat_final<<<dim3(cdiv(p->m, 32), p->H), 256, 0, st>>>(part, p->B, p->H, p->n, p->m, sp, eps_w, whiten_out));
   return launch_ok();
 }
 

@@ -169,11 +169,12 @@ __global__ void __launch_bounds__(256, QN == 4 ? 2 : 3) k_l1(const L1Args args) 
 // =====================================================================================
 // Whitening statistics (Eq. 5-6): per head h and landmark l, over the query rows of every batch element,
 //     mu_l = mean C_il,  sigma_l^2 = mean (C_il - mu_l)^2,  s_l = 1 / sqrt(sigma_l^2 + eps).
-// k_wstat_part: grid (splits, BH), block 256 = 64 column quads x 4 row lanes; every thread sums its rows of its four
-// columns in double (sum and sum of squares of C - pivot, pivot = the head's first row: the sums stay small), the four
-// row lanes are added in a fixed order, and the split leaves [m][2] doubles.  k_wstat_final: one thread per (h, l)
-// adds the partial sums of all batch elements and splits in a fixed order (the pivots differ per batch element, so the
-// sums are brought to pivot 0 first) and writes s.
+// k_wstat_part: grid (splits, BH), block 256 = 64 column quads x 4 row lanes.  A thread walks its rows of its four
+// columns sixteen at a time (four loads in flight): within the sixteen it adds t = C - pivot and t^2 in fp32 (the
+// pivot, row 0 of the head, makes t small, so sixteen terms lose nothing), then adds the two short sums to double
+// accumulators.  The four row lanes are added in a fixed order, the sums are moved from the pivot to zero in double,
+// and the split leaves [m][2] doubles.  k_wstat_final adds the partial sums of all batch elements and splits in a
+// fixed order and writes s.
 // =====================================================================================
 __global__ void __launch_bounds__(256) k_wstat_part(const float* __restrict__ C, int ldc, int n, int m, int rows_per_split,
                                                     double* __restrict__ part /* [BH][splits][m][2] */) {
@@ -181,16 +182,31 @@ __global__ void __launch_bounds__(256) k_wstat_part(const float* __restrict__ C,
   const int bh = blockIdx.y, split = blockIdx.x, nsplit = gridDim.x;
   const int cq = threadIdx.x & 63, rl = threadIdx.x >> 6, c0 = cq * 4;
   const float* Ch = C + (long long)bh * n * ldc;
+  const int i0 = split * rows_per_split, i1 = min(n, i0 + rows_per_split);
   double s1[4] = {0.0, 0.0, 0.0, 0.0}, s2[4] = {0.0, 0.0, 0.0, 0.0};
+  float4 pv = make_float4(0.f, 0.f, 0.f, 0.f);
   if (c0 < ldc) {
-    const float4 pv = *reinterpret_cast<const float4*>(Ch + c0);                 // pivot: row 0 of this head
-    const int i1 = min(n, (split + 1) * rows_per_split);
-    for (int i = split * rows_per_split + rl; i < i1; i += 4) {
+    pv = *reinterpret_cast<const float4*>(Ch + c0);                 // pivot: row 0 of this head
+    int i = i0 + rl;
+    for (; i + 12 < i1; i += 16) {
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const float4*>(Ch + (long long)(i + 4 * u) * ldc + c0);
+      float a[4] = {0.f, 0.f, 0.f, 0.f}, q[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float t0 = v[u].x - pv.x, t1 = v[u].y - pv.y, t2 = v[u].z - pv.z, t3 = v[u].w - pv.w;
+        a[0] += t0; a[1] += t1; a[2] += t2; a[3] += t3;
+        q[0] += t0 * t0; q[1] += t1 * t1; q[2] += t2 * t2; q[3] += t3 * t3;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { s1[u] += (double)a[u]; s2[u] += (double)q[u]; }
+    }
+    for (; i < i1; i += 4) {
       const float4 v = *reinterpret_cast<const float4*>(Ch + (long long)i * ldc + c0);
-      const double t0 = (double)v.x - (double)pv.x, t1 = (double)v.y - (double)pv.y;
-      const double t2 = (double)v.z - (double)pv.z, t3 = (double)v.w - (double)pv.w;
-      s1[0] += t0; s1[1] += t1; s1[2] += t2; s1[3] += t3;
-      s2[0] += t0 * t0; s2[1] += t1 * t1; s2[2] += t2 * t2; s2[3] += t3 * t3;
+      const float t0 = v.x - pv.x, t1 = v.y - pv.y, t2 = v.z - pv.z, t3 = v.w - pv.w;
+      s1[0] += (double)t0; s1[1] += (double)t1; s1[2] += (double)t2; s1[3] += (double)t3;
+      s2[0] += (double)(t0 * t0); s2[1] += (double)(t1 * t1); s2[2] += (double)(t2 * t2); s2[3] += (double)(t3 * t3);
     }
   }
 #pragma unroll
@@ -200,34 +216,56 @@ __global__ void __launch_bounds__(256) k_wstat_part(const float* __restrict__ C,
   if (l < m) {
     const double a = (red[0][l][0] + red[1][l][0]) + (red[2][l][0] + red[3][l][0]);
     const double b = (red[0][l][1] + red[1][l][1]) + (red[2][l][1] + red[3][l][1]);
+    // from sums about the pivot p to sums about zero: sum x = a + N p, sum x^2 = b + 2 p a + N p^2
+    const double p = (double)Ch[l], cnt = (double)max(i1 - i0, 0);
     double* o = part + (((long long)bh * nsplit + split) * m + l) * 2;
-    o[0] = a; o[1] = b;
+    o[0] = a + cnt * p; o[1] = b + 2.0 * p * a + cnt * p * p;
   }
 }
 
-__global__ void k_wstat_final(const double* __restrict__ part, const float* __restrict__ C, int ldc, int B, int H, int n, int m,
-                              int nsplit, float eps, float* __restrict__ s_out /* [H][m] */) {
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= H * m) return;
-  const int h = idx / m, l = idx % m;
-  // sums about pivot p_b become sums about zero: sum x = S1 + N p, sum x^2 = S2 + 2 p S1 + N p^2
+// grid (ceil(m / 32), H), block 256: lane = landmark of the group of 32, warp w adds terms w, w + 8, ... (term t = batch
+// element t / nsplit, split t % nsplit; eight loads in flight), the eight warps are added in a fixed order
+__global__ void __launch_bounds__(256) k_wstat_final(const double* __restrict__ part, int B, int H, int n, int m, int nsplit,
+                                                     float eps, float* __restrict__ s_out /* [H][m] */) {
+  __shared__ double red[8][32][2];
+  const int h = blockIdx.y, lane = threadIdx.x & 31, w = threadIdx.x >> 5, l = blockIdx.x * 32 + lane;
+  const int terms = B * nsplit;
   double sx = 0.0, sxx = 0.0;
-  for (int b = 0; b < B; ++b) {
-    const int bh = b * H + h;
-    const double pv = (double)C[(long long)bh * n * ldc + l];
-    double a = 0.0, q = 0.0;
-    for (int sp = 0; sp < nsplit; ++sp) {
-      const double* o = part + (((long long)bh * nsplit + sp) * m + l) * 2;
-      a += o[0]; q += o[1];
+  if (l < m) {
+    int t = w, b = w / nsplit, sp = w % nsplit;
+    auto next = [&](const double*& ptr) {               // address of term t, then on to term t + 8
+      ptr = part + ((((long long)b * H + h) * nsplit + sp) * m + l) * 2;
+      t += 8; sp += 8;
+      while (sp >= nsplit) { sp -= nsplit; ++b; }
+    };
+    while (t + 56 < terms) {
+      const double* q[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) next(q[u]);
+      double2 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = *reinterpret_cast<const double2*>(q[u]);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { sx += v[u].x; sxx += v[u].y; }
     }
-    sx += a + (double)n * pv;
-    sxx += q + 2.0 * pv * a + (double)n * pv * pv;
+    while (t < terms) {
+      const double* q; next(q);
+      const double2 v = *reinterpret_cast<const double2*>(q);
+      sx += v.x; sxx += v.y;
+    }
   }
-  const double cnt = (double)B * (double)n;
-  const double mu = sx / cnt;
-  double var = sxx / cnt - mu * mu;
-  if (var < 0.0) var = 0.0;
-  s_out[idx] = (float)(1.0 / sqrt(var + (double)eps));
+  red[w][lane][0] = sx; red[w][lane][1] = sxx;
+  __syncthreads();
+  if (w == 0 && l < m) {
+    double a = 0.0, q = 0.0;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) { a += red[g][lane][0]; q += red[g][lane][1]; }
+    const double cnt = (double)B * (double)n;
+    const double mu = a / cnt;
+    double var = q / cnt - mu * mu;
+    if (var < 0.0) var = 0.0;
+    s_out[h * m + l] = (float)(1.0 / sqrt(var + (double)eps));
+  }
 }
 
 // storage type -> fp32 copy
