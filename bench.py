@@ -58,6 +58,23 @@ def workload_dict(cfg, extra=None):
     return d
 
 
+# ------------------------------------------------------------------------------------------ ranks
+def max_over_ranks(ms: float, device=None) -> float:
+    """The slowest rank's time (every rank runs the same replica workload; there is no collective on the data path).
+    With one process, or before a process group exists, it is the value itself."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_s(tokens_per_rank: int, world: int, steps: int, ms: float) -> float:
+    """Whole-job throughput: the tokens all ranks processed in `steps` steps over the slowest rank's time."""
+    return tokens_per_rank * world * steps / (ms * 1e-3)
+
+
 # ------------------------------------------------------------------------------------------ oracle arm
 def oracle_pass(cfg, inp, heads):
     """Time the float64 oracle (as it stands) on the listed heads; returns seconds."""
@@ -264,13 +281,7 @@ def run_ours(args):
             fn(i)
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            import torch.distributed as dist
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), dev)
 
     for i in range(max(args.warmup, 3)):
         step(i)
@@ -281,7 +292,7 @@ def run_ours(args):
     launches_timed = ln.launch_count() - launches_before      # kernels of this library inside the timed region
     t_end = time.perf_counter()
     tokens = cfg.B * cfg.n * world
-    value = tokens * args.steps / (ms * 1e-3)
+    value = job_tokens_per_s(cfg.B * cfg.n, world, args.steps, ms)
 
     # ---- end to end through the host-buffer entry point of the C ABI: every step copies Q, K, V, dO from pinned
     # host memory, runs forward + backward, and copies O, dQ, dK, dV back to pinned host memory.  Three sets of
@@ -315,13 +326,7 @@ def run_ours(args):
                 cur.wait_event(ev)
             e1.record(cur)
             barrier()
-            t_ms = e0.elapsed_time(e1)
-            if world > 1:
-                import torch.distributed as dist
-                t = torch.tensor([t_ms], device=dev)
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                t_ms = float(t.item())
-            return t_ms
+            return max_over_ranks(e0.elapsed_time(e1), dev)
 
         for i in range(3):
             step_e2e(i)
