@@ -366,3 +366,116 @@ def test_whiten_stats_hand_values_and_invariants():
     # heads do not mix: changing head 1 leaves the scale of head 0 alone
     C2 = C.copy(); C2[1::H] *= 1.7
     assert np.array_equal(oracle.whiten_stats(C2, H, 1e-5)[0], s[0])
+
+
+# --------------------------------------------------------------------------- pooling adjoint on overlapping bins
+def test_pool_bwd_overlapping_bins_hand_values():
+    # 14 -> 4 bins (Sec. 4.2 pooling, adaptive bins): [0,4) [3,7) [7,11) [10,14), four tokens each.
+    # Token 3 lies in bins 0 and 1 and token 10 in bins 2 and 3; every other token lies in one bin.
+    p = Problem(B=1, H=1, n=14, d=1, m=4, lam=1.0, ns_iters=0, gh=1, gw=14, mh=1, mw=4)
+    dL = np.array([1.0, 10.0, 100.0, 1000.0]).reshape(1, 1, 4, 1)
+    dK = oracle.landmarks_pool_bwd(p, dL)[0, 0, :, 0]
+    hand = np.array([0.25, 0.25, 0.25, 0.25 + 2.5, 2.5, 2.5, 2.5, 25.0, 25.0, 25.0, 25.0 + 250.0, 250.0, 250.0, 250.0])
+    np.testing.assert_allclose(dK, hand, rtol=1e-15)
+    # two-dimensional overlap: 3 x 3 grid into 2 x 2 bins of 2 x 2 tokens; the centre token lies in all four bins
+    p2 = Problem(B=1, H=1, n=9, d=1, m=4, lam=1.0, ns_iters=0, gh=3, gw=3, mh=2, mw=2)
+    dL2 = np.array([4.0, 40.0, 400.0, 4000.0]).reshape(1, 1, 4, 1)
+    dK2 = oracle.landmarks_pool_bwd(p2, dL2)[0, 0, :, 0].reshape(3, 3)
+    hand2 = np.array([[1.0, 11.0, 10.0], [101.0, 1111.0, 1010.0], [100.0, 1100.0, 1000.0]])
+    np.testing.assert_allclose(dK2, hand2, rtol=1e-15)
+
+
+@pytest.mark.parametrize("gh,gw,mh,mw,prefix", [(14, 14, 4, 8, 0), (56, 56, 8, 16, 0), (14, 14, 4, 8, 2), (5, 7, 3, 3, 1)])
+def test_pool_bwd_overlapping_bins_adjoint_identity(gh, gw, mh, mw, prefix):
+    # <pool(K), U> = <K, pool^T(U)> on the non-divisible geometries of the workloads (14 -> 4 x 8, 56 -> 8 x 16)
+    d = 3
+    p = Problem(B=1, H=2, n=prefix + gh * gw, d=d, m=mh * mw, lam=1.0, ns_iters=0, prefix=prefix, gh=gh, gw=gw, mh=mh, mw=mw)
+    rng = np.random.default_rng(31)
+    K = rng.standard_normal((1, 2, p.n, d))
+    U = rng.standard_normal((1, 2, p.m, d))
+    L = oracle.landmarks_pool(p, K)
+    dK = oracle.landmarks_pool_bwd(p, U)
+    assert float((L * U).sum()) == pytest.approx(float((K * dK).sum()), rel=1e-12)
+    assert np.abs(dK[:, :, :prefix]).max(initial=0.0) == 0.0
+    # the pooling matrix applied to unit vectors: column sums of pool^T(e_l) are one (a bin's weights sum to one)
+    for l in (0, p.m // 2, p.m - 1):
+        e = np.zeros((1, 2, p.m, d)); e[:, :, l] = 1.0
+        np.testing.assert_allclose(oracle.landmarks_pool_bwd(p, e).sum(axis=2), 1.0, rtol=1e-13)
+
+
+def test_full_backward_finite_differences_overlapping_bins():
+    # the whole backward with landmarks pooled over a grid the bins do not divide (5 x 7 -> 2 x 3, class token in front)
+    rng = np.random.default_rng(41)
+    d, T = 5, 3
+    p = Problem(B=1, H=1, n=1 + 35, d=d, m=6, lam=float(d), ns_iters=T, ridge_eps=1e-6, map_mode=1, lm_mode=1,
+                prefix=1, gh=5, gw=7, mh=2, mw=3)
+    Q, K, V, dO = (rng.standard_normal((1, 1, p.n, d)) for _ in range(4))
+    s = rng.uniform(0.5, 2.0, (1, p.m))
+    dQ, dK, dV, _ = oracle.backward(p, Q, K, V, dO, whiten=s)
+    loss = lambda k: float((oracle.forward(p, Q, k, V, whiten=s) * dO).sum())
+    h = 1e-6
+    # tokens 18 (row 2, col 3: shared by both bin rows) and 11 (row 1, col 3) lie in overlapping bins; 0 is the class token
+    for idx in [(0, 0, 0, 0), (0, 0, 18, 2), (0, 0, 11, 4), (0, 0, 35, 1), (0, 0, 4, 0)]:
+        kp = K.copy(); kp[idx] += h
+        km = K.copy(); km[idx] -= h
+        assert dK[idx] == pytest.approx((loss(kp) - loss(km)) / (2 * h), rel=5e-6, abs=1e-8), idx
+
+
+# --------------------------------------------------------------------------- landmarks rounded to single precision
+def _lm_case(seed):
+    rng = np.random.default_rng(seed)
+    p0 = Problem(B=1, H=2, n=1 + 8 * 6, d=8, m=12, lam=8.0, ns_iters=4, ridge_eps=1e-6, map_mode=1, lm_mode=1,
+                 prefix=1, gh=8, gw=6, mh=4, mw=3)
+    Q, K, V, dO = (rng.standard_normal((1, 2, p0.n, p0.d)) for _ in range(4))
+    s = rng.uniform(0.5, 2.0, (2, p0.m))
+    return p0, Q, K, V, dO, s
+
+
+def test_lm_f32_is_the_given_landmark_path_on_rounded_means():
+    # lm_f32 = 1 must be exactly: pool in float64, round each landmark coordinate to float32 (numpy's cast), and carry on
+    # as if those landmarks had been given (lm_mode 0); the landmark gradient then returns to the keys through the
+    # pooling adjoint
+    from dataclasses import replace
+    p0, Q, K, V, dO, s = _lm_case(51)
+    p1 = replace(p0, lm_f32=1)
+    L32 = oracle.landmarks_pool(p0, K).astype(np.float32).astype(np.float64)
+    pg = replace(p0, lm_mode=0)
+    O1 = oracle.forward(p1, Q, K, V, whiten=s)
+    Og = oracle.forward(pg, Q, K, V, L=L32, whiten=s)
+    np.testing.assert_array_equal(O1, Og)
+    dQ1, dK1, dV1, _ = oracle.backward(p1, Q, K, V, dO, whiten=s)
+    dQg, dKg, dVg, dLg = oracle.backward(pg, Q, K, V, dO, L=L32, whiten=s)
+    np.testing.assert_array_equal(dQ1, dQg)
+    np.testing.assert_array_equal(dV1, dVg)
+    np.testing.assert_allclose(dK1, dKg + oracle.landmarks_pool_bwd(p0, dLg), rtol=1e-13, atol=1e-15)
+    # and the flag does change the landmarks (otherwise the comparison above would be vacuous)
+    assert np.abs(L32 - oracle.landmarks_pool(p0, K)).max() > 0.0
+
+
+def test_lm_f32_moves_results_only_at_rounding_level_away_from_ties():
+    from dataclasses import replace
+    p0, Q, K, V, dO, s = _lm_case(52)
+    p1 = replace(p0, lm_f32=1)
+    L64 = oracle.landmarks_pool(p0, K)
+    L32 = L64.astype(np.float32).astype(np.float64)
+    # places where sign(token - landmark) differs between the two landmark precisions: only there can the flag move
+    # a gradient by more than rounding (an exact tie with a mean that float32 holds exactly is a tie on both sides)
+    near = 0
+    for T_ in (Q, K):
+        near += int((np.sign(T_[:, :, :, None, :] - L64[:, :, None, :, :]) != np.sign(T_[:, :, :, None, :] - L32[:, :, None, :, :])).sum())
+    assert near == 0                                    # none on this seeded case
+    O0, O1 = oracle.forward(p0, Q, K, V, whiten=s), oracle.forward(p1, Q, K, V, whiten=s)
+    assert np.linalg.norm(O0 - O1) <= 1e-7 * np.linalg.norm(O0)
+    g0 = oracle.backward(p0, Q, K, V, dO, whiten=s)[:3]
+    g1 = oracle.backward(p1, Q, K, V, dO, whiten=s)[:3]
+    for a, b in zip(g0, g1):
+        assert np.linalg.norm(a - b) <= 1e-6 * np.linalg.norm(a)
+    # a planted near-tie: one query coordinate placed between a landmark's exact mean and its float32 rounding
+    l, c = 3, 2
+    lo, hi = sorted((L64[0, 0, l, c], L32[0, 0, l, c]))
+    assert hi > lo
+    Qt = Q.copy(); Qt[0, 0, 5, c] = 0.5 * (lo + hi)
+    d0 = oracle.backward(p0, Qt, K, V, dO, whiten=s)[0]
+    d1 = oracle.backward(p1, Qt, K, V, dO, whiten=s)[0]
+    diff = np.abs(d0 - d1)
+    assert diff[0, 0, 5, c] > 1e3 * np.delete(diff[0, 0, 5], c).max()   # the sign of that one term flipped, nothing else moved
