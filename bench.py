@@ -2,9 +2,10 @@
 """Benchmark of the hot path: forward+backward Nystrom Laplacian attention, tokens/s.
 
 One step = one pass of the whole path (laplace_nystrom_fwd + laplace_nystrom_bwd through the
-C ABI) over one batch of synthetic input of the chosen workload (default: the DeiT-Small-shaped
-configuration the metric is quoted on).  Every rank of a multi-GPU launch runs the same workload
-on its own GPU (heads are independent, no collective), so scaling is weak.
+C ABI) over one batch of synthetic input of the chosen workload.  The metric names no configuration, so the default
+is the largest single-GPU one of the benchmark list (landmark / solver stress, m = 256, 12 Newton-Schulz steps); the
+same JSON line carries a `sweep` over every other configuration.  Every rank of a multi-GPU launch runs the same
+workload on its own GPU (heads are independent, no collective), so scaling is weak.
 
     python bench.py --gpus 1 --steps 20 --warmup 5
     python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
@@ -42,8 +43,9 @@ def parse():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="cfg2", choices=sorted(synth.CONFIGS))
-    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--config", default="cfg5_m256_T12", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle legs (CPU baseline, sampled-head parity)")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the sweep over all configurations")
     ap.add_argument("--B", type=int, default=0, help="override the batch size (profiling of a smaller case)")
     return ap.parse_args()
 
@@ -222,12 +224,144 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------ our arm
-def l1_lane_ops(cfg, kernel):
-    """Algorithmic FP32 lane-operations of one launch of an l1 kernel: 2 per (pair, dim) in the forward
-    (subtract, accumulate |.|), all heads."""
-    BH = cfg.B * cfg.H
-    pairs = {"l1_CRW": 2 * cfg.n * cfg.m + cfg.m * cfg.m}[kernel]
-    return 2.0 * cfg.d * pairs * BH
+def measured_peaks():
+    """HBM GB/s and sustained bf16 TFLOP/s measured on this machine (generated file), else the stated fallback."""
+    try:
+        j = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        return float(j["hbm_gbs"]), float(j["bf16_tflops_sustained"]), "of measured (MEASURED_PEAKS.json)"
+    except Exception:
+        return 6650.0, 1400.0, "of fallback (6.65 TB/s, 1.4 PFLOP/s sustained)"
+
+
+def kernel_work(cfg, name):
+    """(bound, algorithmic units of one launch) of a traced launch: FP32 lane-operations for the l1 and sign
+    kernels (2 per pair and dim forward: subtract, accumulate |.|; 3 per pair and dim backward: step, two
+    accumulations), flops for the products and the per-head kernels, bytes for the memory-bound rest."""
+    BH, n, d, m, T = cfg.B * cfg.H, cfg.n, cfg.d, cfg.m, cfg.T
+    pairs = {"l1_CRW": 2 * n * m + m * m, "l1_CR": 2 * n * m, "l1_C": n * m, "l1_R": n * m, "l1_W": m * m}
+    if name in pairs:
+        return "alu", 2.0 * d * pairs[name] * BH
+    if name.startswith("sign2_") or name in ("sign_rows_dQ", "sign_cols_dLC", "sign_rows_dK", "sign_cols_dLR"):
+        full = name.startswith("sign2_")
+        return "alu", (3.0 if full else 2.0) * d * n * m * BH
+    if name == "sign_rows_dLW":
+        return "alu", 2.0 * d * m * m * BH
+    if name.startswith(("tn_", "nn_", "ntg_")):
+        return "tensor", 2.0 * n * m * d * BH
+    if name.startswith("k_mid_fwd"):
+        return "tensor", (4.0 * T * m ** 3 + 2.0 * m * m * d) * BH
+    if name == "k_mid_bwd":
+        return "tensor", (10.0 * T * m ** 3 + 4.0 * m * m * d) * BH
+    es = 4 if cfg.dtype == "f32" else 2
+    return "hbm", float(BH * n * d * (es + 4))      # pooling, its adjoint, small reductions: one pass over a token tensor
+
+
+# DRAM bytes per head and launch of the kernels that can dominate a step, from the ncu captures summarised under
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of one launch divided by the heads of the captured case;
+# traffic grows in proportion to the heads).  Keyed by (kernel, workload family).
+NCU_DRAM_BYTES_PER_HEAD = {}
+
+
+def alu_probe(ln, dev):
+    """FP32 add rate the GPU sustains (T lane-op/s): the measured counterpart of the derived ALU peak."""
+    sink = torch.zeros(1025, dtype=torch.float32, device=dev)
+    out = {}
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    for packed in (False, True):
+        best = 0.0
+        ln.fp32_add_probe(sms * 8, 2000, packed, sink)
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ops = ln.fp32_add_probe(sms * 8, 20000, packed, sink)
+            e1.record()
+            torch.cuda.synchronize()
+            best = max(best, ops / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+        out["packed" if packed else "scalar"] = best
+    return out
+
+
+class Workload:
+    """Device buffers and the step function of one configuration."""
+
+    def __init__(self, ln, cfg, dev, inp=None):
+        self.ln, self.cfg, self.dev = ln, cfg, dev
+        self.inp = synth.make_inputs(cfg) if inp is None else inp
+        names = ("Q", "K", "V", "dO")
+        es = 4 if cfg.dtype == "f32" else 2
+        self.es = es
+        self.in_bytes = 4 * cfg.B * cfg.H * cfg.n * cfg.d * es
+        # rotate through enough input sets that a step's inputs are not L2-resident (126 MB L2)
+        self.nsets = min(max(2, int(np.ceil(3 * 126e6 / self.in_bytes))), 16)
+        self.sets = [{k: self.inp[k].to(dev).clone() for k in names} for _ in range(self.nsets)]
+        self.p = ln.problem_from_config(cfg, whiten=self.inp["whiten"].to(dev))
+        self.saved = torch.empty(ln.laplace_nystrom_saved_bytes(self.p), dtype=torch.uint8, device=dev)
+        self.ws = torch.empty(ln.laplace_nystrom_workspace_bytes(self.p, True), dtype=torch.uint8, device=dev)
+        self.O = torch.empty_like(self.sets[0]["Q"])
+        self.dQ, self.dK, self.dV = (torch.empty_like(self.O) for _ in range(3))
+        self.status = torch.zeros(cfg.B * cfg.H, dtype=torch.int32, device=dev)
+        self.status_b = torch.zeros_like(self.status)
+
+    def step(self, i):
+        ln, cfg, s = self.ln, self.cfg, self.sets[i % self.nsets]
+        ln.laplace_nystrom_fwd(self.p, s["Q"], s["K"], s["V"], O=self.O, saved=self.saved, ws=self.ws, dev_status=self.status)
+        if cfg.backward:
+            ln.laplace_nystrom_bwd(self.p, s["Q"], s["K"], s["V"], s["dO"], self.saved, dQ=self.dQ, dK=self.dK, dV=self.dV,
+                                   ws=self.ws, dev_status=self.status_b)
+
+    def path_roofline_s(self):
+        cfg = self.cfg
+        P = 2 * cfg.n * cfg.m + cfg.m * cfg.m
+        ops = (2.0 + (3.0 if cfg.backward else 0.0)) * cfg.d * P * cfg.B * cfg.H
+        return ops / (ALU_PEAK_TLANEOPS * 1e12)
+
+    def parity(self, heads):
+        """Results of step 0's inputs on the sampled heads against the float64 oracle (relative Frobenius error)."""
+        sys.path.insert(0, os.path.join(ROOT, "tests"))
+        import oracle
+        from parity import compare, run_oracle_heads
+        oracle.build()
+        self.step(0)
+        torch.cuda.synchronize()
+        g = {"O": self.O, "dQ": self.dQ, "dK": self.dK, "dV": self.dV}
+        o = run_oracle_heads(self.cfg, self.inp, heads, backward=self.cfg.backward)
+        errs = compare(self.cfg, g, o, heads)
+        flags = int(self.status.abs().max()) | int(self.status_b.abs().max())
+        return {"heads": heads, "status_flags": flags, **{k: e["fro"] for k, e in errs.items()},
+                **({"internal_max": max(e["internal"] for e in errs.values())} if cfg_is_bf16(self.cfg) else {})}
+
+
+def cfg_is_bf16(cfg):
+    return cfg.dtype == "bf16"
+
+
+def time_steps(fn, steps, barrier, dev):
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for i in range(steps):
+        fn(i)
+    e1.record()
+    barrier()
+    return max_over_ranks(e0.elapsed_time(e1), dev)
+
+
+def sweep_line(ln, name, dev, steps, warmup, with_parity):
+    """One configuration of the sweep: throughput, step time, whole-path roofline fraction and sampled-head parity."""
+    cfg = synth.CONFIGS[name]
+    w = Workload(ln, cfg, dev)
+    for i in range(warmup):
+        w.step(i)
+    sync = torch.cuda.synchronize
+    ms = [time_steps(w.step, steps, sync, dev) / steps for _ in range(3)]
+    ms_med = float(np.median(ms))
+    out = {"tokens_per_s": cfg.B * cfg.n / (ms_med * 1e-3), "ms_per_step": ms_med, "path_frac": w.path_roofline_s() / (ms_med * 1e-3)}
+    if with_parity:
+        BH = cfg.B * cfg.H
+        out["parity"] = w.parity(sorted({0, BH // 2, BH - 1}) if cfg.n <= 4096 else [BH - 1])
+    del w
+    torch.cuda.empty_cache()
+    return out
 
 
 def run_ours(args):
@@ -245,27 +379,9 @@ def run_ours(args):
     cfg = synth.CONFIGS[args.config]
     if args.B > 0:
         cfg = synth.shrink(cfg, B=args.B)
-    inp = synth.make_inputs(cfg)
-    names = ("Q", "K", "V", "dO")
-    es = 4 if cfg.dtype == "f32" else 2
-    in_bytes = 4 * cfg.B * cfg.H * cfg.n * cfg.d * es
-    # rotate through enough input sets that a step's inputs are not L2-resident (126 MB L2)
-    nsets = max(2, int(np.ceil(3 * 126e6 / in_bytes)))
-    nsets = min(nsets, 16)
-    sets = []
-    for s in range(nsets):
-        sets.append({k: inp[k].to(dev).clone() for k in names})
-    wh = inp["whiten"].to(dev)
-    p = ln.problem_from_config(cfg, whiten=wh)
-    saved = torch.empty(ln.laplace_nystrom_saved_bytes(p), dtype=torch.uint8, device=dev)
-    ws = torch.empty(ln.laplace_nystrom_workspace_bytes(p, True), dtype=torch.uint8, device=dev)
-    O = torch.empty_like(sets[0]["Q"]); dQ = torch.empty_like(O); dK = torch.empty_like(O); dV = torch.empty_like(O)
-
-    def step(i):
-        s = sets[i % nsets]
-        ln.laplace_nystrom_fwd(p, s["Q"], s["K"], s["V"], O=O, saved=saved, ws=ws)
-        if cfg.backward:
-            ln.laplace_nystrom_bwd(p, s["Q"], s["K"], s["V"], s["dO"], saved, dQ=dQ, dK=dK, dV=dV, ws=ws)
+    w = Workload(ln, cfg, dev)
+    inp, p, es, names = w.inp, w.p, w.es, ("Q", "K", "V", "dO")
+    step = w.step
 
     def barrier():
         if world > 1:
@@ -273,24 +389,20 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(fn, steps):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        e0.record()
-        for i in range(steps):
-            fn(i)
-        e1.record()
-        barrier()
-        return max_over_ranks(e0.elapsed_time(e1), dev)
-
     for i in range(max(args.warmup, 3)):
         step(i)
+    torch.cuda.synchronize()
+    # the timed region (exactly --steps steps) is repeated so that the whole measurement lasts at least ~100 ms and clock
+    # samples fall inside it; the reported time is the median region
+    probe_ms = time_steps(step, 1, barrier, dev)
+    repeats = int(min(10, max(1, np.ceil(100.0 / max(probe_ms * args.steps, 1e-3)))))
     sampler = ClockSampler(local) if rank == 0 else None
     t_begin = time.perf_counter()
     launches_before = ln.launch_count()
-    ms = timed(step, args.steps)
-    launches_timed = ln.launch_count() - launches_before      # kernels of this library inside the timed region
+    regions = [time_steps(step, args.steps, barrier, dev) for _ in range(repeats)]
+    launches_timed = (ln.launch_count() - launches_before) // repeats      # kernels of this library inside one timed region
     t_end = time.perf_counter()
+    ms = float(np.median(regions))
     tokens = cfg.B * cfg.n * world
     value = job_tokens_per_s(cfg.B * cfg.n, world, args.steps, ms)
 
@@ -332,24 +444,26 @@ def run_ours(args):
             step_e2e(i)
         ms_e2e = timed_streams(args.steps)
         e2e_how = f"laplace_nystrom_fwd_bwd_host, pinned host tensors, {nslot} streams x {nslot} device buffer sets"
+        del slots
     else:   # forward-only workload: copies around laplace_nystrom_fwd
-        dev_in = {k: torch.empty_like(sets[0][k]) for k in names}
+        dev_in = {k: torch.empty_like(w.sets[0][k]) for k in names}
 
         def step_e2e(i):
             for k in ("Q", "K", "V"):
                 dev_in[k].copy_(host_in[k], non_blocking=True)
-            ln.laplace_nystrom_fwd(p, dev_in["Q"], dev_in["K"], dev_in["V"], O=O, saved=saved, ws=ws)
-            host_out[0]["O"].copy_(O, non_blocking=True)
+            ln.laplace_nystrom_fwd(p, dev_in["Q"], dev_in["K"], dev_in["V"], O=w.O, saved=w.saved, ws=w.ws)
+            host_out[0]["O"].copy_(w.O, non_blocking=True)
 
         for i in range(3):
             step_e2e(i)
-        ms_e2e = timed(step_e2e, args.steps)
+        ms_e2e = time_steps(step_e2e, args.steps, barrier, dev)
         e2e_how = "copies from/to pinned host tensors around laplace_nystrom_fwd, one stream"
     e2e_value = tokens * args.steps / (ms_e2e * 1e-3)
     one = cfg.B * cfg.H * cfg.n * cfg.d * es
     e2e = {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / args.steps,
            "h2d_bytes_per_step": (4 if cfg.backward else 3) * one, "d2h_bytes_per_step": (4 if cfg.backward else 1) * one,
            "how": e2e_how}
+    torch.cuda.empty_cache()
 
     # ---- per-kernel durations (events around every launch, separate pass so the bracketing
     # does not perturb the number above)
@@ -358,71 +472,102 @@ def run_ours(args):
     for i in range(args.steps):
         step(i)
     trace = ln.trace_end()
-    launches_per_step = len(trace) // args.steps
     per = {}
     for name, t in trace:
         a = per.setdefault(name, [0, 0.0]); a[0] += 1; a[1] += t
     total_traced = sum(v[1] for v in per.values())
     kernels = {k: {"launches_per_step": v[0] // args.steps, "avg_us": 1e3 * v[1] / v[0], "share": v[1] / total_traced}
                for k, v in sorted(per.items(), key=lambda kv: -kv[1][1])}
-    dom = "l1_CRW"
+    hbm_peak, tc_peak, peak_src = measured_peaks()
+    alu_meas = alu_probe(ln, dev)
+    # the dominant kernel: the launch with the largest share of the traced step
+    dom = max(per, key=lambda k: per[k][1])
     dom_avg_s = per[dom][1] / per[dom][0] * 1e-3
-    achieved = l1_lane_ops(cfg, dom) / dom_avg_s / 1e12
-    roofline = {"bound": "alu", "kernel": dom, "achieved": achieved, "peak": ALU_PEAK_TLANEOPS, "unit": "Tlane-op/s",
-                "frac": achieved / ALU_PEAK_TLANEOPS, "traffic": None,
-                "peak_source": "derived: 148 SMs x 128 FP32 lanes x 1.965 GHz, one add/sub per lane per clock",
-                "kernel_share_of_step": per[dom][1] / total_traced}
+    bound, units = kernel_work(cfg, dom)
+    if bound == "alu":
+        achieved, peak, unit = units / dom_avg_s / 1e12, ALU_PEAK_TLANEOPS, "Tlane-op/s"
+        src = "derived: 148 SMs x 128 FP32 lanes x 1.965 GHz, one add/sub per lane per clock"
+    elif bound == "tensor":
+        achieved, peak, unit, src = units / dom_avg_s / 1e12, tc_peak, "TFLOP/s", "bf16_tflops_sustained " + peak_src
+    else:
+        achieved, peak, unit, src = units / dom_avg_s / 1e9, hbm_peak, "GB/s", "hbm_gbs " + peak_src
+    per_head = NCU_DRAM_BYTES_PER_HEAD.get((dom, cfg.name.split("_T")[0]))
+    roofline = {"bound": bound, "kernel": dom, "achieved": achieved, "peak": peak, "unit": unit,
+                "frac": achieved / peak, "traffic": None if per_head is None else per_head * cfg.B * cfg.H,
+                "peak_source": src, "kernel_share_of_step": per[dom][1] / total_traced}
+    if bound == "alu":
+        roofline["alu_peak_measured"] = alu_meas
+        roofline["frac_of_measured_add_rate"] = achieved / max(alu_meas["scalar"], alu_meas["packed"])
     # whole-path roofline: algorithmic l1 lane-ops (2 fwd + 3 bwd per pair-dim) at the ALU peak
-    P = 2 * cfg.n * cfg.m + cfg.m * cfg.m
-    path_ops = (2.0 + (3.0 if cfg.backward else 0.0)) * cfg.d * P * cfg.B * cfg.H
-    path_roof_s = path_ops / (ALU_PEAK_TLANEOPS * 1e12)
-    roofline["path_frac"] = path_roof_s / (ms * 1e-3 / args.steps)
+    roofline["path_frac"] = w.path_roofline_s() / (ms * 1e-3 / args.steps)
+    roofline["path_frac_of_measured_add_rate"] = roofline["path_frac"] * ALU_PEAK_TLANEOPS / max(alu_meas["scalar"], alu_meas["packed"])
+    # the ALU-bound kernels one by one
+    roofline["alu_kernels"] = {}
+    for k, v in per.items():
+        bk, uk = kernel_work(cfg, k)
+        if bk == "alu":
+            roofline["alu_kernels"][k] = uk / (v[1] / v[0] * 1e-3) / 1e12 / ALU_PEAK_TLANEOPS
 
     # ---- next step beside the path (Eq. 5-6): the whitening scale estimated on the device from the saved kernel
     # block C; bound by HBM (C is read once); L2 is flushed before every timed launch
     whiten_stats = None
     if cfg.backward:
-        ws_w = torch.empty(256, dtype=torch.uint8, device=dev)
         flush = torch.zeros(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
-        ln.laplace_nystrom_whiten_stats(p, saved, 1e-5)
+        ln.laplace_nystrom_whiten_stats(p, w.saved, 1e-5)
         times = []
         for _ in range(5):               # device time of its two launches (events around each launch, as in the trace above)
             flush.max()                  # read-only sweep of 256 MB: L2 holds none of C and no dirty lines
             torch.cuda.synchronize()
             ln.trace_begin()
-            ln.laplace_nystrom_whiten_stats(p, saved, 1e-5)
+            ln.laplace_nystrom_whiten_stats(p, w.saved, 1e-5)
             times.append(sum(t for _, t in ln.trace_end()))
-        del flush, ws_w
+        del flush
         t_ms = float(np.median(times))
         ldm = (cfg.m + 3) // 4 * 4
         c_bytes = cfg.B * cfg.H * cfg.n * ldm * 4
-        peak, src = 6650.0, "fallback 6.65 TB/s"
-        try:
-            peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["hbm_gbs"]); src = "MEASURED_PEAKS.json hbm_gbs"
-        except Exception:
-            pass
         gbs = c_bytes / (t_ms * 1e-3) / 1e9
-        whiten_stats = {"us": 1e3 * t_ms, "bytes": c_bytes, "bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
-                        "frac": gbs / peak, "peak_source": src, "launches": 2}
+        whiten_stats = {"us": 1e3 * t_ms, "bytes": c_bytes, "bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s",
+                        "frac": gbs / hbm_peak, "peak_source": peak_src, "launches": 2}
 
+    parity = None
+    if world == 1 and not args.no_cpu_baseline:
+        BH = cfg.B * cfg.H
+        parity = w.parity(sorted({0, BH // 2, BH - 1}))
     if rank != 0:
         return
-    # clocks: samples inside the timed region; a region shorter than three samples (a few ms) is
+    # clocks: samples inside the timed regions; a region shorter than three samples (a few ms) is
     # widened to everything that ran under the same load after it (end-to-end and traced passes)
-    clocks = sampler.summary([("timed region", t_begin, t_end), ("timed region + e2e and traced passes", t_begin, time.perf_counter())])
+    clocks = sampler.summary([("timed regions", t_begin, t_end), ("timed regions + e2e and traced passes", t_begin, time.perf_counter())])
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": workload_dict(cfg, {"l2": f"rotating {nsets} input sets ({nsets * in_bytes / 1e6:.0f} MB > 126 MB L2)",
-                                      "parallelism": f"replicas x{world} (heads independent, no collective)"}),
+        "vs_baseline": None,
+        "dtype": "f32 (bf16 storage; fp32 CUDA-core arithmetic and accumulation; tensor-core operands split into bf16 hi+lo)"
+                 if cfg.dtype == "bf16" else "f32",
+        "data": "synthetic",
+        "config": workload_dict(cfg, {"l2": f"rotating {w.nsets} input sets ({w.nsets * w.in_bytes / 1e6:.0f} MB > 126 MB L2)",
+                                      "parallelism": f"replicas x{world} (heads independent, no collective)",
+                                      "timed_regions": repeats, "region_ms": regions}),
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_timed,
         "roofline": roofline, "kernels": kernels,
     }
+    if parity is not None:
+        out["parity_vs_oracle"] = parity
     if whiten_stats is not None:
         out["whiten_stats"] = whiten_stats
+    inp_main = inp
+    del w
+    torch.cuda.empty_cache()
     if not args.no_cpu_baseline and world == 1:
-        out["cpu_baseline"] = cpu_baseline(cfg, inp)
+        out["cpu_baseline"] = cpu_baseline(cfg, inp_main)
+    if not args.no_sweep and world == 1 and args.B == 0:
+        # every configuration of the benchmark list in one run (a few steps each; parity on sampled heads for one
+        # variant per shape family)
+        sweep = {}
+        with_parity = {"cfg1", "cfg2", "cfg3", "cfg4a", "cfg4b", "cfg4c", "cfg5_m64_T8", "cfg5_m128_T8", "cfg5_m256_T8"}
+        for name in sorted(synth.CONFIGS):
+            sweep[name] = sweep_line(ln, name, dev, steps=5, warmup=3, with_parity=name in with_parity and not args.no_cpu_baseline)
+        out["sweep"] = sweep
     print(json.dumps(out))
 
 

@@ -21,8 +21,10 @@
  *     synchronises the device: it validates arguments on the host, enqueues kernels on
  *     `stream` (a cudaStream_t passed as void*; NULL = the default stream) and returns.
  *     LN_OK means "enqueued".  The only state kept between calls is one extra stream and a
- *     few events per device (see ln_set_overlap), created by the first bf16 attention call on
- *     that device: that call should come before any stream capture.
+ *     few events per (device, caller stream) pair (see ln_set_overlap), created by the first bf16
+ *     attention call on that pair: that call should come before any stream capture.  Calls on
+ *     different streams share none of it.  Two host threads enqueueing on the SAME stream at the
+ *     same time are not supported.
  *   - Tensors are contiguous, row-major, 16-byte aligned.  Outputs are fully overwritten.
  *     Inputs are never modified and must not alias outputs.
  *   - Storage type of the [.,.,.,d] tensors is `dtype` (LN_F32 or LN_BF16); all arithmetic and
@@ -83,7 +85,10 @@ size_t laplace_nystrom_workspace_bytes(const ln_problem* p, int32_t with_saved);
  *   O      [B,H,n,d] dtype, overwritten;
  *   saved  NULL for inference, else laplace_nystrom_saved_bytes(p) bytes;
  *   ws     laplace_nystrom_workspace_bytes(p, saved != NULL) bytes;
- *   dev_status NULL or int32 [B*H]: per head, bit0 = X_T is not finite (written by the device).
+ *   dev_status NULL or int32 [B*H], zeroed by the call and written by the device, per head:
+ *     bit 0 = X_T has a non-finite entry (a diverged iteration, e.g. a bad ns_alpha);
+ *     bit 1 = a bounded wait on the tensor cores or on a bulk copy ran out (the kernel gave up, freed its
+ *             tensor memory and returned; that head's results are then undefined).  Neither traps.
  */
 int laplace_nystrom_fwd(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L,
                         void* O, void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
@@ -97,6 +102,7 @@ int laplace_nystrom_fwd(const ln_problem* p, const void* Q, const void* K, const
  *   dL [B,H,m,d] dtype: required when lm_mode == 0; must be NULL when lm_mode == 1 (the
  *   landmark gradient is folded into dK through the pooling adjoint).
  *   ws: laplace_nystrom_workspace_bytes(p, 1) bytes.
+ *   dev_status: as for laplace_nystrom_fwd (only bit 1 can be set by the backward pass).
  */
 int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L,
                         const void* dO, const void* saved, void* dQ, void* dK, void* dV, void* dL,
@@ -110,7 +116,8 @@ int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const
  * hdQ, hdK, hdV.  Returns once everything is enqueued; the host outputs are valid after the stream has been
  * synchronised.  lm_mode must be 1 (landmarks pooled from K), else LN_ERR_UNSUPPORTED.
  *   staging: DEVICE memory, laplace_nystrom_host_staging_bytes(p) bytes, 16-byte aligned, owned by the caller;
- *   saved, ws, dev_status: as for laplace_nystrom_fwd / _bwd (training sizes).
+ *   saved, ws, dev_status: as for laplace_nystrom_fwd / _bwd (training sizes); dev_status is cleared once and
+ *   collects the flags of both passes.  Every argument check of both passes is made before the first copy.
  * Two calls on two streams with two sets of device buffers overlap one step's copies with the other's kernels.
  */
 size_t laplace_nystrom_host_staging_bytes(const ln_problem* p);
@@ -201,6 +208,34 @@ int laplace_nystrom_whiten_stats(const ln_problem* p, const void* saved, float e
  */
 int landmarks_pool(const ln_problem* p, const void* K, float* L, void* stream);
 int landmarks_pool_bwd(const ln_problem* p, const float* dL, void* dK, void* stream);
+
+/*
+ * Where an fp32 intermediate of the forward pass lies inside `saved` (the paper has no counterpart: an inspection
+ * aid, used by the parity tests to compare intermediates with the oracle's).  name: "L" landmarks [m x d],
+ * "C" = k(Q,L) [n x m], "Rt" = k(K,L) [n x m], "mu" row means of C [1 x n], "W" = k(L,L) [m x m] (before the
+ * ridge), "X" = X_T [m x m], "M" = R V [m x d], "Yt" folded Y [m x d], "ybar" [1 x d].
+ * info[0] = offset of head 0 in floats from the start of saved, info[1] = rows, info[2] = columns,
+ * info[3] = leading dimension, info[4] = floats between consecutive heads.  LN_ERR_ARG for an unknown name.
+ */
+int laplace_nystrom_saved_array(const ln_problem* p, const char* name, int64_t info[5]);
+
+/*
+ * Self-test of failure detection (the paper has no counterpart).  Launches one tiny kernel that waits, with the
+ * library's bounded wait and a limit of `probes` polls, on a barrier nothing ever arrives on; the wait gives up and
+ * the kernel ORs bit 1 into dev_status[0] (device int32, not cleared by this call) and returns normally.  Shows a
+ * caller, without hanging or faulting anything, what a timed-out wait in the attention kernels looks like.
+ */
+int ln_selftest_wait_timeout(int32_t probes, int32_t* dev_status, void* stream);
+
+/*
+ * FP32 add-rate probe (the paper has no counterpart; a measurement aid).  `blocks` CTAs of 256 threads run `iters`
+ * steps of eight independent add chains per thread, two lanes per chain and step (packed = 0: two scalar adds,
+ * packed = 1: one add.f32x2), without memory traffic.  ln_fp32_add_probe_lane_ops returns the lane-operations of
+ * such a launch; divided by its duration it is the measured counterpart of the derived FP32 peak
+ * (SMs x 128 lanes x clock).  sink: device fp32 [1025], sink[0] is read, nothing else is normally written.
+ */
+int ln_fp32_add_probe(int32_t blocks, int32_t iters, int32_t packed, float* sink, void* stream);
+int64_t ln_fp32_add_probe_lane_ops(int32_t blocks, int32_t iters);
 
 /*
  * Profiling aid, off by default and not thread-safe (the paper has no counterpart; Sec. 4.3 only

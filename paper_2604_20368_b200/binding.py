@@ -27,6 +27,7 @@ EXPORTS = [
     "ln_trace_begin", "ln_trace_end", "ns_pinv_static_scratch_bytes", "ns_pinv_static",
     "laplace_nystrom_host_staging_bytes", "laplace_nystrom_fwd_bwd_host", "ln_set_overlap", "ln_launch_count",
     "laplace_nystrom_whiten_stats_workspace_bytes", "laplace_nystrom_whiten_stats",
+    "laplace_nystrom_saved_array", "ln_selftest_wait_timeout", "ln_fp32_add_probe", "ln_fp32_add_probe_lane_ops",
 ]
 
 
@@ -132,6 +133,11 @@ def lib():
         L.laplace_nystrom_whiten_stats_workspace_bytes.restype = sz
         L.laplace_nystrom_whiten_stats_workspace_bytes.argtypes = [ctypes.POINTER(_CProblem)]
         L.laplace_nystrom_whiten_stats.argtypes = [ctypes.POINTER(_CProblem), vp, f32, vp, vp, sz, vp]
+        L.laplace_nystrom_saved_array.argtypes = [pp, ctypes.c_char_p, ctypes.POINTER(ctypes.c_int64)]
+        L.ln_selftest_wait_timeout.argtypes = [i32, vp, vp]
+        L.ln_fp32_add_probe.argtypes = [i32, i32, i32, vp, vp]
+        L.ln_fp32_add_probe_lane_ops.restype = ctypes.c_int64
+        L.ln_fp32_add_probe_lane_ops.argtypes = [i32, i32]
         _lib = L
     return _lib
 
@@ -195,8 +201,9 @@ def laplace_nystrom_fwd(p: Problem, Q, K, V, L=None, O=None, saved=None, ws=None
 
 
 def laplace_nystrom_bwd(p: Problem, Q, K, V, dO, saved, L=None, dQ=None, dK=None, dV=None, dL=None, ws=None,
-                        stream=None):
-    """Exact adjoint of laplace_nystrom_fwd.  Returns dQ, dK, dV, dL (dL is None when lm_mode == 1)."""
+                        dev_status=None, stream=None):
+    """Exact adjoint of laplace_nystrom_fwd.  Returns dQ, dK, dV, dL (dL is None when lm_mode == 1).
+    ``dev_status``: optional int32 [B*H] device tensor that receives the per-head flags."""
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(K) if dK is None else dK
     dV = torch.empty_like(V) if dV is None else dV
@@ -206,7 +213,7 @@ def laplace_nystrom_bwd(p: Problem, Q, K, V, dO, saved, L=None, dQ=None, dK=None
         ws = _bytes(laplace_nystrom_workspace_bytes(p, True), Q.device)
     cp = p.c()
     st = lib().laplace_nystrom_bwd(ctypes.byref(cp), _ptr(Q), _ptr(K), _ptr(V), _ptr(L), _ptr(dO), _ptr(saved),
-                                   _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dL), _ptr(ws), ws.numel(), None,
+                                   _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dL), _ptr(ws), ws.numel(), _ptr(dev_status),
                                    _stream(stream))
     _check(st, "laplace_nystrom_bwd")
     return dQ, dK, dV, dL
@@ -229,14 +236,16 @@ def _host_ptr(t: torch.Tensor):
     return ctypes.c_void_p(t.data_ptr())
 
 
-def laplace_nystrom_fwd_bwd_host(p: Problem, bufs: HostStep, hQ, hK, hV, hdO, hO, hdQ, hdK, hdV, stream=None):
+def laplace_nystrom_fwd_bwd_host(p: Problem, bufs: HostStep, hQ, hK, hV, hdO, hO, hdQ, hdK, hdV, stream=None,
+                                 dev_status=None):
     """One training step on host tensors (pinned for asynchronous copies): copies in, forward, backward, copies
     out, all enqueued on `stream`; the host outputs are valid after the stream has been synchronised."""
     cp = p.c()
     st = lib().laplace_nystrom_fwd_bwd_host(ctypes.byref(cp), _host_ptr(hQ), _host_ptr(hK), _host_ptr(hV),
                                             _host_ptr(hdO), _host_ptr(hO), _host_ptr(hdQ), _host_ptr(hdK),
                                             _host_ptr(hdV), _ptr(bufs.staging), bufs.staging.numel(),
-                                            _ptr(bufs.saved), _ptr(bufs.ws), bufs.ws.numel(), None, _stream(stream))
+                                            _ptr(bufs.saved), _ptr(bufs.ws), bufs.ws.numel(), _ptr(dev_status),
+                                            _stream(stream))
     _check(st, "laplace_nystrom_fwd_bwd_host")
 
 
@@ -334,6 +343,28 @@ def laplace_nystrom_whiten_stats(p: Problem, saved, eps_w: float = 1e-5, out=Non
     _check(lib().laplace_nystrom_whiten_stats(ctypes.byref(cp), _ptr(saved), eps_w, _ptr(out), _ptr(ws), ws.numel(),
                                               _stream(stream)), "laplace_nystrom_whiten_stats")
     return out
+
+
+def saved_array(p: Problem, saved: torch.Tensor, name: str) -> torch.Tensor:
+    """A strided fp32 view [B*H, rows, cols] of a named intermediate inside the forward context ``saved``
+    (laplace_nystrom_saved_array): "L", "C", "Rt", "mu", "W", "X", "M", "Yt", "ybar"."""
+    info = (ctypes.c_int64 * 5)()
+    cp = p.c()
+    _check(lib().laplace_nystrom_saved_array(ctypes.byref(cp), name.encode(), info), "laplace_nystrom_saved_array")
+    off, rows, cols, ld, stride = (int(v) for v in info)
+    flat = saved.view(torch.float32)
+    return torch.as_strided(flat, (p.B * p.H, rows, cols), (stride, ld, 1), off)
+
+
+def selftest_wait_timeout(dev_status: torch.Tensor, probes: int = 1000, stream=None):
+    """Run the bounded-wait self-test: ORs bit 1 into dev_status[0] once the wait has given up."""
+    _check(lib().ln_selftest_wait_timeout(probes, _ptr(dev_status), _stream(stream)), "ln_selftest_wait_timeout")
+
+
+def fp32_add_probe(blocks: int, iters: int, packed: bool, sink: torch.Tensor, stream=None) -> int:
+    """Launch the FP32 add-rate probe; returns the lane-operations the launch performs."""
+    _check(lib().ln_fp32_add_probe(blocks, iters, int(packed), _ptr(sink), _stream(stream)), "ln_fp32_add_probe")
+    return int(lib().ln_fp32_add_probe_lane_ops(blocks, iters))
 
 
 def launch_count() -> int:

@@ -2,19 +2,49 @@
 #include <math.h>
 #include <stdlib.h>
 #include <stdint.h>
+#include <string.h>
 
 #include "../../include/laplace_nystrom.h"
 #include "ln_kernels.cuh"
 #include "ln_sign2.cuh"
 #include <atomic>
 #include <mutex>
+#include <unordered_map>
 #include <type_traits>
 
 using namespace ln;
 
 namespace {
 
-constexpr int kSMs = 148;
+// Number of SMs of the current device (asked once per device; 148 on a B200, the fallback if the query fails).
+constexpr int kMaxDevices = 64;
+int sm_count() {
+  static std::atomic<int> cached[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+  int v = cached[dev].load(std::memory_order_relaxed);
+  if (v <= 0) {
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) { cudaGetLastError(); v = 148; }
+    cached[dev].store(v, std::memory_order_relaxed);
+  }
+  return v;
+}
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per kernel and device (again only when a larger size is
+// asked for): a table keyed by the kernel's address.
+template <typename K>
+void want_smem(K kern, size_t smem) {
+  static std::mutex mu;
+  static std::unordered_map<const void*, int> have[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = 0;
+  const void* id = reinterpret_cast<const void*>(kern);
+  std::lock_guard<std::mutex> lk(mu);
+  auto it = have[dev].find(id);
+  if (it != have[dev].end() && it->second >= (int)smem) return;
+  cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  have[dev][id] = (int)smem;
+}
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -42,6 +72,7 @@ struct Plan {
 
 bool make_plan(const ln_problem* p, Plan* pl) {
   if (!p) return false;
+  const int kSMs = sm_count();
   pl->BH = p->B * p->H; pl->n = p->n; pl->d = p->d; pl->m = p->m; pl->T = p->ns_iters;
   pl->ldm = (p->m + 3) & ~3;
   pl->scr = (size_t)p->m * pl->ldm;
@@ -220,7 +251,7 @@ inline unsigned cdiv(long long a, long long b) { return (unsigned)((a + b - 1) /
 // on its stream.  Off by default; the product path never touches it.
 constexpr int kTraceCap = 2048;
 struct Trace {
-  bool on = false;
+  std::atomic<bool> on{false};
   int count = 0;
   cudaEvent_t ev[2 * kTraceCap];
   const char* name[kTraceCap];
@@ -241,14 +272,18 @@ struct TraceScope {
 // Side stream.  The per-head kernels (Newton-Schulz and its adjoint: one CTA or cluster per head, bound by the
 // latency of a chain of small products) do not depend on the token-sized kernels next to them, so the entry
 // points enqueue them on a second stream of the library, forked from and joined back into the caller's stream
-// with events: to the caller everything is still ordered on the stream it passed.  One stream and a ring of
-// events per device, created at the first call on that device.  Switched off while a trace is recorded (so that
-// the per-launch times are those of kernels running alone) and by ln_set_overlap(0).
-constexpr int kSideDevices = 64, kSideEvents = 16;
-struct SideState { bool tried = false, ok = false; cudaStream_t s = nullptr; cudaEvent_t ev[kSideEvents]; unsigned next = 0; };
-SideState g_side[kSideDevices];
+// with events: to the caller everything is still ordered on the stream it passed.  Switched off while a trace is
+// recorded (so that the per-launch times are those of kernels running alone) and by ln_set_overlap(0).
+// One side stream and a ring of events per (device, caller stream), kept in a small table: calls on different
+// streams (or from different host threads on different streams) share nothing, so they neither serialise on a
+// common side stream nor wait on one another's events.  Two host threads that enqueue on the SAME stream at the same
+// time are not supported (the order of their work on that stream would be undefined anyway).
+constexpr int kSideSlots = 32, kSideEvents = 16;
+struct SideState { bool used = false, ok = false; int dev = -1; cudaStream_t caller = nullptr; cudaStream_t s = nullptr;
+                   cudaEvent_t ev[kSideEvents]; unsigned next = 0; };
+SideState g_side[kSideSlots];
 std::mutex g_side_mu;
-bool g_overlap = true;
+std::atomic<bool> g_overlap{true};
 struct Side {
   cudaStream_t s = nullptr; cudaEvent_t fork_ev[2] = {nullptr, nullptr}, join_ev = nullptr;
   bool on() const { return s != nullptr; }
@@ -261,27 +296,31 @@ struct Side {
   void mark() const { cudaEventRecord(fork_ev[1], s); }
   void join_mark(cudaStream_t st) const { cudaStreamWaitEvent(st, fork_ev[1], 0); }
 };
-Side side_acquire(bool want) {
+Side side_acquire(bool want, cudaStream_t caller) {
   Side r;
-  if (!want || !g_overlap || g_trace.on) return r;
+  if (!want || !g_overlap.load(std::memory_order_relaxed) || g_trace.on.load(std::memory_order_relaxed)) return r;
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kSideDevices) return r;
+  if (cudaGetDevice(&dev) != cudaSuccess) return r;
   std::lock_guard<std::mutex> lk(g_side_mu);
-  SideState& d = g_side[dev];
-  if (!d.tried) {
-    d.tried = true;
+  SideState* d = nullptr;
+  for (int i = 0; i < kSideSlots && !d; ++i)
+    if (g_side[i].used && g_side[i].dev == dev && g_side[i].caller == caller) d = &g_side[i];
+  if (!d) {
+    for (int i = 0; i < kSideSlots && !d; ++i) if (!g_side[i].used) d = &g_side[i];
+    if (!d) return r;                  // table full: this caller stream runs without overlap
+    d->used = true; d->dev = dev; d->caller = caller;
     // highest priority: its few large CTAs (up to a whole SM each) are placed before the pending small CTAs of
     // the kernels on the caller's stream, which would otherwise keep every SM partly occupied until their grids end
     int prio_lo = 0, prio_hi = 0;
     bool ok = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) == cudaSuccess;
-    ok = ok && cudaStreamCreateWithPriority(&d.s, cudaStreamNonBlocking, prio_hi) == cudaSuccess;
-    for (int i = 0; ok && i < kSideEvents; ++i) ok = cudaEventCreateWithFlags(&d.ev[i], cudaEventDisableTiming) == cudaSuccess;
-    d.ok = ok;
+    ok = ok && cudaStreamCreateWithPriority(&d->s, cudaStreamNonBlocking, prio_hi) == cudaSuccess;
+    for (int i = 0; ok && i < kSideEvents; ++i) ok = cudaEventCreateWithFlags(&d->ev[i], cudaEventDisableTiming) == cudaSuccess;
+    d->ok = ok;
     if (!ok) cudaGetLastError();
   }
-  if (!d.ok) return r;
-  r.s = d.s; r.fork_ev[0] = d.ev[d.next]; r.fork_ev[1] = d.ev[d.next + 1]; r.join_ev = d.ev[d.next + 2];
-  d.next = (d.next + 4) % kSideEvents;
+  if (!d->ok) return r;
+  r.s = d->s; r.fork_ev[0] = d->ev[d->next]; r.fork_ev[1] = d->ev[d->next + 1]; r.join_ev = d->ev[d->next + 2];
+  d->next = (d->next + 4) % kSideEvents;
   return r;
 }
 
@@ -331,10 +370,10 @@ void launch_l1_args(const char* name, L1Args& a, int nprob, int batch, cudaStrea
   for (int i = 0; i < nprob; ++i) na_max = a.p[i].na > na_max ? a.p[i].na : na_max;
   const L1Launch l = plan_l1(na_max, a.nb, a.d, batch, nprob);
   if (l.qn == 4) {
-    cudaFuncSetAttribute(k_l1<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.smem);
+    want_smem(k_l1<4>, l.smem);
     LN_LAUNCH(name, st, k_l1<4><<<l.grid, l.block, l.smem, st>>>(a));
   } else {
-    cudaFuncSetAttribute(k_l1<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.smem);
+    want_smem(k_l1<2>, l.smem);
     LN_LAUNCH(name, st, k_l1<2><<<l.grid, l.block, l.smem, st>>>(a));
   }
 }
@@ -353,9 +392,9 @@ void launch_l1(const char* name, const TA* A, const TB* Bm, float* E, float* row
 // ------------------------------------------------------------------------------------------
 template <typename T, int D>
 int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const T* V, const T* L, T* O,
-             const Ctx& x, const FwdWs& w, int32_t* dev_status, cudaStream_t st) {
-  const int BH = pl.BH, n = pl.n, m = pl.m;
-  if (dev_status) cudaMemsetAsync(dev_status, 0, sizeof(int32_t) * BH, st);   // the kernels OR their flags into it
+             const Ctx& x, const FwdWs& w, int32_t* dev_status, cudaStream_t st, bool clear_status) {
+  const int BH = pl.BH, n = pl.n, m = pl.m, kSMs = sm_count();
+  if (dev_status && clear_status) cudaMemsetAsync(dev_status, 0, sizeof(int32_t) * BH, st);   // the kernels OR their flags into it
   // landmarks (Sec. 4.2)
   if (p->lm_mode == 1) {
     LN_LAUNCH("k_pool", st, k_pool<T><<<dim3(cdiv(m, 256 / (D / 4)), BH), 256, 0, st>>>(K, x.Lf, geom_of(p)));
@@ -366,7 +405,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // the three kernel blocks: C = k(Q,L) with its row sums, R^T = k(K,L), W = k(L,L)
   // (not for many small heads, where the per-head kernel fills the GPU and the split launches cost more than the
   // overlap returns)
-  const Side side = side_acquire(std::is_same<T, bf16>::value && (2 * pl.mid_sms <= kSMs || (long long)n * m * D > (1ll << 22)));
+  const Side side = side_acquire(std::is_same<T, bf16>::value && (2 * pl.mid_sms <= kSMs || (long long)n * m * D > (1ll << 22)), st);
   const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);   // tcgen05 products over the landmarks
   // Where the iteration is expected to outlast the two token-sized blocks (few heads of few tokens), only the iteration
   // goes to the side stream; estimates in microseconds: 5 / 12 / 100 per step for m <= 64 / <= 128 / larger, and the l1
@@ -380,7 +419,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   auto launch_mid = [&](cudaStream_t s, int phase) {
     constexpr bool TC = std::is_same<T, bf16>::value;
     auto launch = [&](auto kern, size_t smem, int cl = 1) {
-      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      want_smem(kern, smem);
       LN_LAUNCH(phase == 3 ? "k_mid_fwd" : (phase == 1 ? "k_mid_fwd_ns" : "k_mid_fwd_y"), s,
                 launch_clustered(kern, BH * cl, cl, smem, s, m, pl.ldm, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode,
                                  p->whiten, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, Mparts_src, Mparts, x.M, w.Y, x.Yt,
@@ -440,7 +479,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // O = (C - mu) Ytilde + ybar
   if constexpr (std::is_same<T, bf16>::value && (D == 64 || D == 128)) {
     const size_t smem = nn_umma_smem<D>();
-    cudaFuncSetAttribute(k_nn_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    want_smem(k_nn_umma<D>, smem);
     LN_LAUNCH("nn_O", st, k_nn_umma<D><<<dim3(cdiv(n, 128), BH), 256, smem, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr,
                                                                               reinterpret_cast<const bf16*>(x.Yimg), x.ybar, O, n, m, dev_status));
   } else if constexpr (std::is_same<T, bf16>::value)
@@ -452,11 +491,11 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
 
 template <typename T, int D>
 int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const T* V, const T* dO,
-             const Ctx& x, const BwdWs& w, T* dQ, T* dK, T* dV, T* dL, int32_t* dev_status, cudaStream_t st) {
-  const int BH = pl.BH, n = pl.n, m = pl.m, ch = pl.chunks;
+             const Ctx& x, const BwdWs& w, T* dQ, T* dK, T* dV, T* dL, int32_t* dev_status, cudaStream_t st, bool clear_status) {
+  const int BH = pl.BH, n = pl.n, m = pl.m, ch = pl.chunks, kSMs = sm_count();
   const float inv_lambda = 1.f / p->lambda;
   const float* mu = p->map_mode == 1 ? x.mu : nullptr;
-  if (dev_status) cudaMemsetAsync(dev_status, 0, sizeof(int32_t) * BH, st);
+  if (dev_status && clear_status) cudaMemsetAsync(dev_status, 0, sizeof(int32_t) * BH, st);
   // query side: Z'^T dO and column sums of dO; g^C = (dO Ytilde^T) o C / lambda; dQ; landmark part
   auto launch_tn_dY = [&](cudaStream_t s) {
     if constexpr (std::is_same<T, bf16>::value)
@@ -467,7 +506,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   auto launch_ntg_C = [&]() {
     if constexpr (std::is_same<T, bf16>::value) {
       if constexpr (D == 64 || D == 128) {
-        cudaFuncSetAttribute(k_ntg_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ntg_umma_smem<D>());
+        want_smem(k_ntg_umma<D>, ntg_umma_smem<D>());
         LN_LAUNCH("ntg_C", st, k_ntg_umma<D><<<dim3(cdiv(n, 128), BH), 256, ntg_umma_smem<D>(), st>>>(dO, reinterpret_cast<const bf16*>(x.Yimg), x.C, pl.ldm,
                                                                                                   w.G, n, m, inv_lambda, dev_status));
       } else
@@ -481,12 +520,12 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const int chq = fused_sign ? pl.s2q_chunks : ch;    // chunks of the query-side landmark-gradient partials
   // The per-head kernel and the landmark-block sign pass need Z'^T dO only: with a side stream they run beside
   // the query-side kernels and are joined before the key side, which needs dM.
-  const Side side = side_acquire(std::is_same<T, bf16>::value);
+  const Side side = side_acquire(std::is_same<T, bf16>::value, st);
   const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);
   auto launch_mid = [&](cudaStream_t s) {
     constexpr bool TC = std::is_same<T, bf16>::value;
     auto launch = [&](auto kern, size_t smem, int cl = 1) {
-      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      want_smem(kern, smem);
       LN_LAUNCH("k_mid_bwd", s, launch_clustered(kern, BH * cl, cl, smem, s, m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten,
                                                  x.W, x.Xh, x.Ph, x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P,
                                                  w.Hm, w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot,
@@ -501,7 +540,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   auto launch_ntg_R = [&](cudaStream_t s) {
     if constexpr (std::is_same<T, bf16>::value) {
       if constexpr (D == 64 || D == 128) {
-        cudaFuncSetAttribute(k_ntg_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ntg_umma_smem<D>());
+        want_smem(k_ntg_umma<D>, ntg_umma_smem<D>());
         LN_LAUNCH("ntg_R", s, k_ntg_umma<D><<<dim3(cdiv(n, 128), BH), 256, ntg_umma_smem<D>(), s>>>(V, reinterpret_cast<const bf16*>(w.dMimg), x.Rt, pl.ldm,
                                                                                                 w.G2, n, m, inv_lambda, dev_status));
       } else
@@ -514,7 +553,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     if constexpr (std::is_same<T, bf16>::value) {
       if constexpr (D == 64 || D == 128) {
         const size_t smem = nn_umma_smem<D>();
-        cudaFuncSetAttribute(k_nn_umma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        want_smem(k_nn_umma<D>, smem);
         LN_LAUNCH("nn_dV", s, k_nn_umma<D><<<dim3(cdiv(n, 128), BH), 256, smem, s>>>(x.Rt, pl.ldm, nullptr, reinterpret_cast<const bf16*>(w.dMimg),
                                                                                  nullptr, dV, n, m, dev_status));
       } else
@@ -552,7 +591,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   launch_ntg_C();
   if (fused_sign) {
     auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
-      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.s2_smem);
+      want_smem(kern, pl.s2_smem);
       LN_LAUNCH(name, st, kern<<<dim3(chq, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(tokp, x.Lf, w.G, pl.ldm, rowsp, partp, n, m, D, pl.s2q_rpc));
     };
     if (pl.s2_tg == S2_TGMAX) launch2("sign2_dQ_dLC", k_sign2<T, T, 1>, Q, dQ, w.dLCpart);
@@ -566,7 +605,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // key side: dK (kernel part); landmark part
   if (fused_sign) {
     auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
-      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.s2_smem);
+      want_smem(kern, pl.s2_smem);
       LN_LAUNCH(name, st, kern<<<dim3(chs, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(tokp, x.Lf, w.G2, pl.ldm, rowsp, partp, n, m, D, pl.s2_rpc));
     };
     if (pl.s2_tg == S2_TGMAX) launch2("sign2_dK_dLR", k_sign2<T, float, 1>, K, w.dKpart, w.dLRpart);
@@ -590,23 +629,23 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
 
 template <typename T>
 int fwd_dispatch_d(const ln_problem* p, const Plan& pl, const void* Q, const void* K, const void* V, const void* L,
-                   void* O, const Ctx& x, const FwdWs& w, int32_t* ds, cudaStream_t st) {
+                   void* O, const Ctx& x, const FwdWs& w, int32_t* ds, cudaStream_t st, bool clear_status) {
   const T *q = (const T*)Q, *k = (const T*)K, *v = (const T*)V, *l = (const T*)L; T* o = (T*)O;
   switch (p->d) {
-    case 32: return fwd_impl<T, 32>(p, pl, q, k, v, l, o, x, w, ds, st);
-    case 64: return fwd_impl<T, 64>(p, pl, q, k, v, l, o, x, w, ds, st);
-    case 128: return fwd_impl<T, 128>(p, pl, q, k, v, l, o, x, w, ds, st);
+    case 32: return fwd_impl<T, 32>(p, pl, q, k, v, l, o, x, w, ds, st, clear_status);
+    case 64: return fwd_impl<T, 64>(p, pl, q, k, v, l, o, x, w, ds, st, clear_status);
+    case 128: return fwd_impl<T, 128>(p, pl, q, k, v, l, o, x, w, ds, st, clear_status);
   }
   return LN_ERR_UNSUPPORTED;
 }
 template <typename T>
 int bwd_dispatch_d(const ln_problem* p, const Plan& pl, const void* Q, const void* K, const void* V, const void* dO,
-                   const Ctx& x, const BwdWs& w, void* dQ, void* dK, void* dV, void* dL, int32_t* ds, cudaStream_t st) {
+                   const Ctx& x, const BwdWs& w, void* dQ, void* dK, void* dV, void* dL, int32_t* ds, cudaStream_t st, bool clear_status) {
   const T *q = (const T*)Q, *k = (const T*)K, *v = (const T*)V, *g = (const T*)dO;
   switch (p->d) {
-    case 32: return bwd_impl<T, 32>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st);
-    case 64: return bwd_impl<T, 64>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st);
-    case 128: return bwd_impl<T, 128>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st);
+    case 32: return bwd_impl<T, 32>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st, clear_status);
+    case 64: return bwd_impl<T, 64>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st, clear_status);
+    case 128: return bwd_impl<T, 128>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st, clear_status);
   }
   return LN_ERR_UNSUPPORTED;
 }
@@ -629,7 +668,7 @@ namespace {
 struct L1BwdWs { float *Kmat, *G, *part; int rpc, chunks; size_t bytes; };
 L1BwdWs carve_l1bwd(int batch, int na, int nb, int d, void* base) {
   Carver c(base); L1BwdWs w;
-  int want = (2 * kSMs + batch - 1) / batch; if (want < 1) want = 1;
+  int want = (2 * sm_count() + batch - 1) / batch; if (want < 1) want = 1;
   int rpc = (na + want - 1) / want; rpc = (rpc + 31) / 32 * 32;
   w.rpc = rpc; w.chunks = (na + rpc - 1) / rpc;
   w.Kmat = c.take((size_t)batch * na * nb);
@@ -679,10 +718,7 @@ int ln_trace_end(int32_t capacity, int32_t* count, float* ms, const char** names
 uint64_t ln_launch_count(void) { return (uint64_t)g_launch_count.load(std::memory_order_relaxed); }
 
 int ln_set_overlap(int enabled) {
-  std::lock_guard<std::mutex> lk(g_side_mu);
-  const int before = g_overlap ? 1 : 0;
-  g_overlap = enabled != 0;
-  return before;
+  return g_overlap.exchange(enabled != 0) ? 1 : 0;
 }
 
 const char* ln_status_string(int s) {
@@ -712,8 +748,12 @@ size_t laplace_nystrom_workspace_bytes(const ln_problem* p, int32_t with_saved) 
   return ws;
 }
 
-int laplace_nystrom_fwd(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L, void* O,
-                        void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
+}  // extern "C"
+
+namespace {
+// host-side checks of the attention entry points; nothing is enqueued when one fails
+int check_fwd_args(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L, const void* O,
+                   const void* saved, const void* ws, size_t ws_bytes) {
   int s = validate(p);
   if (s != LN_OK) return s;
   if (!Q || !K || !V || !O || !ws) return LN_ERR_ARG;
@@ -722,17 +762,11 @@ int laplace_nystrom_fwd(const ln_problem* p, const void* Q, const void* K, const
       !aligned16(saved))
     return LN_ERR_ARG;
   if (ws_bytes < laplace_nystrom_workspace_bytes(p, saved != nullptr)) return LN_ERR_WORKSPACE;
-  Plan pl; make_plan(p, &pl);
-  const FwdWs w = carve_fwd_ws(pl, ws);
-  const Ctx x = carve_ctx(pl, saved ? saved : static_cast<char*>(ws) + w.bytes);
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (p->dtype == LN_F32) return fwd_dispatch_d<float>(p, pl, Q, K, V, L, O, x, w, dev_status, st);
-  return fwd_dispatch_d<bf16>(p, pl, Q, K, V, L, O, x, w, dev_status, st);
+  return LN_OK;
 }
-
-int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L,
-                        const void* dO, const void* saved, void* dQ, void* dK, void* dV, void* dL, void* ws,
-                        size_t ws_bytes, int32_t* dev_status, void* stream) {
+int check_bwd_args(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L, const void* dO,
+                   const void* saved, const void* dQ, const void* dK, const void* dV, const void* dL, const void* ws,
+                   size_t ws_bytes) {
   int s = validate(p);
   if (s != LN_OK) return s;
   if (!Q || !K || !V || !dO || !saved || !dQ || !dK || !dV || !ws) return LN_ERR_ARG;
@@ -742,19 +776,54 @@ int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const
       !aligned16(dK) || !aligned16(dV) || !aligned16(dL) || !aligned16(ws))
     return LN_ERR_ARG;
   if (ws_bytes < laplace_nystrom_workspace_bytes(p, 1)) return LN_ERR_WORKSPACE;
+  return LN_OK;
+}
+// clear_status: zero dev_status first (the stand-alone entry points); the host-buffer step clears it once and lets
+// the backward pass OR its flags into what the forward pass left
+int fwd_entry(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L, void* O,
+              void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream, bool clear_status) {
+  const int s = check_fwd_args(p, Q, K, V, L, O, saved, ws, ws_bytes);
+  if (s != LN_OK) return s;
+  Plan pl; make_plan(p, &pl);
+  const FwdWs w = carve_fwd_ws(pl, ws);
+  const Ctx x = carve_ctx(pl, saved ? saved : static_cast<char*>(ws) + w.bytes);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (p->dtype == LN_F32) return fwd_dispatch_d<float>(p, pl, Q, K, V, L, O, x, w, dev_status, st, clear_status);
+  return fwd_dispatch_d<bf16>(p, pl, Q, K, V, L, O, x, w, dev_status, st, clear_status);
+}
+int bwd_entry(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L,
+              const void* dO, const void* saved, void* dQ, void* dK, void* dV, void* dL, void* ws,
+              size_t ws_bytes, int32_t* dev_status, void* stream, bool clear_status) {
+  const int s = check_bwd_args(p, Q, K, V, L, dO, saved, dQ, dK, dV, dL, ws, ws_bytes);
+  if (s != LN_OK) return s;
   Plan pl; make_plan(p, &pl);
   const BwdWs w = carve_bwd_ws(pl, ws);
   const Ctx x = carve_ctx(pl, const_cast<void*>(saved));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (p->dtype == LN_F32) return bwd_dispatch_d<float>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, dev_status, st);
-  return bwd_dispatch_d<bf16>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, dev_status, st);
+  if (p->dtype == LN_F32) return bwd_dispatch_d<float>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, dev_status, st, clear_status);
+  return bwd_dispatch_d<bf16>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, dev_status, st, clear_status);
 }
+}  // namespace
+
+extern "C" {
+
+int laplace_nystrom_fwd(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L, void* O,
+                        void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
+  return fwd_entry(p, Q, K, V, L, O, saved, ws, ws_bytes, dev_status, stream, true);
+}
+
+int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L,
+                        const void* dO, const void* saved, void* dQ, void* dK, void* dV, void* dL, void* ws,
+                        size_t ws_bytes, int32_t* dev_status, void* stream) {
+  return bwd_entry(p, Q, K, V, L, dO, saved, dQ, dK, dV, dL, ws, ws_bytes, dev_status, stream, true);
+}
+
 
 namespace {
 // splits of the token rows per head for the whitening statistics: about eight CTAs per SM, at least 64 rows each
 void wstat_plan(const ln_problem* p, int* nsplit, int* rows_per_split) {
   const int BH = p->B * p->H;
-  int sp = (8 * kSMs + BH - 1) / BH;
+  int sp = (8 * sm_count() + BH - 1) / BH;
   if (sp > 64) sp = 64;
   if (sp > (p->n + 63) / 64) sp = (p->n + 63) / 64;
   if (sp < 1) sp = 1;
@@ -807,15 +876,22 @@ int laplace_nystrom_fwd_bwd_host(const ln_problem* p, const void* hQ, const void
   const size_t bytes = (size_t)p->B * p->H * p->n * p->d * (p->dtype == LN_F32 ? 4 : 2);
   const size_t one = (bytes + 255) / 256 * 256;
   char* d = static_cast<char*>(staging);
+  // every check of the two passes comes before the first copy: an argument error enqueues nothing
+  s = check_fwd_args(p, d, d + one, d + 2 * one, nullptr, d + 4 * one, saved, ws, ws_bytes);
+  if (s != LN_OK) return s;
+  s = check_bwd_args(p, d, d + one, d + 2 * one, nullptr, d + 3 * one, saved, d + 5 * one, d + 6 * one, d + 7 * one,
+                     nullptr, ws, ws_bytes);
+  if (s != LN_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const void* hin[4] = {hQ, hK, hV, hdO};
   for (int i = 0; i < 4; ++i)
     if (cudaMemcpyAsync(d + i * one, hin[i], bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return LN_ERR_CUDA;
-  s = laplace_nystrom_fwd(p, d, d + one, d + 2 * one, nullptr, d + 4 * one, saved, ws, ws_bytes, dev_status, stream);
+  s = fwd_entry(p, d, d + one, d + 2 * one, nullptr, d + 4 * one, saved, ws, ws_bytes, dev_status, stream, true);
   if (s != LN_OK) return s;
   if (cudaMemcpyAsync(hO, d + 4 * one, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LN_ERR_CUDA;
-  s = laplace_nystrom_bwd(p, d, d + one, d + 2 * one, nullptr, d + 3 * one, saved, d + 5 * one, d + 6 * one, d + 7 * one,
-                          nullptr, ws, ws_bytes, nullptr, stream);
+  // the backward pass ORs its flags into the status words the forward pass cleared and wrote
+  s = bwd_entry(p, d, d + one, d + 2 * one, nullptr, d + 3 * one, saved, d + 5 * one, d + 6 * one, d + 7 * one,
+                nullptr, ws, ws_bytes, dev_status, stream, false);
   if (s != LN_OK) return s;
   void* hout[3] = {hdQ, hdK, hdV};
   for (int i = 0; i < 3; ++i)
@@ -871,19 +947,18 @@ int ns_pinv_bwd(int32_t batch, int32_t m, const float* W, int32_t iters, float r
 namespace {
 constexpr size_t kStaticScratchBytes = LN_STATIC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
-constexpr int kMaxDevices = 64;
-void* g_static_scratch_addr[kMaxDevices];   // device address of g_static_scratch, per device; NULL = not asked yet
+std::atomic<void*> g_static_scratch_addr[kMaxDevices];   // device address of g_static_scratch, per device; NULL = not asked yet
 
 // Device address of the static scratch on the current device (looked up on first use).
 int static_scratch_ptr(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LN_ERR_CUDA;
-  if (!g_static_scratch_addr[dev]) {
-    void* ptr = nullptr;
+  void* ptr = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!ptr) {      // two threads may both ask; they get the same address
     if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return LN_ERR_CUDA;
-    g_static_scratch_addr[dev] = ptr;
+    g_static_scratch_addr[dev].store(ptr, std::memory_order_release);
   }
-  *out = g_static_scratch_addr[dev];
+  *out = ptr;
   return LN_OK;
 }
 }  // namespace
@@ -969,5 +1044,42 @@ int landmarks_pool_bwd(const ln_problem* p, const float* dL, void* dK, void* str
   else LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<bf16><<<grid, 256, 0, st>>>(nullptr, dL, (bf16*)dK, geom_of(p), 1));
   return launch_ok();
 }
+
+int laplace_nystrom_saved_array(const ln_problem* p, const char* name, int64_t info[5]) {
+  if (validate(p) != LN_OK || !name || !info) return LN_ERR_ARG;
+  Plan pl; make_plan(p, &pl);
+  const Ctx x = carve_ctx(pl, reinterpret_cast<void*>(256));      // offsets relative to a fictitious base
+  auto off = [](const void* q) { return (int64_t)((reinterpret_cast<uintptr_t>(q) - 256) / sizeof(float)); };
+  const int64_t n = p->n, d = p->d, m = p->m, ldm = pl.ldm;
+  const bool img = p->dtype == LN_BF16;                            // tensor-core paths: history slots are operand images
+  const int64_t ldx = (img && m <= 128) ? ldm : m;
+  const int64_t mx = img ? pl.hslot : m * ldx;
+  struct { const char* nm; const void* ptr; int64_t rows, cols, ld, stride; } t[] = {
+    {"L", x.Lf, m, d, d, m * d}, {"C", x.C, n, m, ldm, n * ldm}, {"Rt", x.Rt, n, m, ldm, n * ldm},
+    {"mu", x.mu, 1, n, n, n}, {"W", x.W, m, m, m, m * m},
+    {"X", x.Xh + (size_t)pl.T * mx, m, m, ldx, (int64_t)(pl.T + 1) * mx},
+    {"M", x.M, m, d, d, m * d}, {"Yt", x.Yt, m, d, d, m * d}, {"ybar", x.ybar, 1, d, d, d}};
+  for (auto& e : t)
+    if (strcmp(name, e.nm) == 0) {
+      info[0] = off(e.ptr); info[1] = e.rows; info[2] = e.cols; info[3] = e.ld; info[4] = e.stride;
+      return LN_OK;
+    }
+  return LN_ERR_ARG;
+}
+
+int ln_selftest_wait_timeout(int32_t probes, int32_t* dev_status, void* stream) {
+  if (probes <= 0 || probes > (1 << 22) || !dev_status) return LN_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  LN_LAUNCH("k_selftest_wait", st, k_selftest_wait<<<1, 32, 0, st>>>(probes, dev_status));
+  return launch_ok();
+}
+
+int ln_fp32_add_probe(int32_t blocks, int32_t iters, int32_t packed, float* sink, void* stream) {
+  if (blocks <= 0 || iters <= 0 || !sink) return LN_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  LN_LAUNCH("k_fp32_add_probe", st, k_fp32_add_probe<<<blocks, 256, 0, st>>>(packed ? -iters : iters, sink));
+  return launch_ok();
+}
+int64_t ln_fp32_add_probe_lane_ops(int32_t blocks, int32_t iters) { return (int64_t)blocks * 256 * iters * kProbeChains * 2; }
 
 }  // extern "C"

@@ -1235,4 +1235,55 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
   }
 }
 
+// =====================================================================================
+// Self-test of the bounded wait every tensor-core kernel of this library uses: an mbarrier on which nothing ever
+// arrives is waited for with a probe limit; the wait must give up, and the kernel reports it the way the product
+// kernels do (bit 1 of the status word) and returns normally.
+// =====================================================================================
+__global__ void k_selftest_wait(int probes, int* dev_status) {
+  __shared__ __align__(8) unsigned long long mbar;
+  if (threadIdx.x == 0) umma::mbar_init(&mbar, 1);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const bool ok = umma::mbar_wait(&mbar, 0, probes);
+    if (!ok) atomicOr(dev_status, 2);
+  }
+}
+
+// =====================================================================================
+// FP32 add-rate probe: every thread runs kProbeChains independent chains of dependent adds, two lanes per chain and
+// step (mode 0: two scalar adds, mode 1: one packed add.f32x2), no memory traffic inside the loop.  The rate it
+// sustains is the measured counterpart of the derived lane-operation peak (SMs x 128 lanes x clock) that the
+// l1 kernels are held against.
+// =====================================================================================
+constexpr int kProbeChains = 8;
+__global__ void __launch_bounds__(256) k_fp32_add_probe(int iters, float* sink) {
+  const float x = sink[0];                       // a run-time value the compiler cannot fold
+  float a[kProbeChains], b[kProbeChains];
+#pragma unroll
+  for (int k = 0; k < kProbeChains; ++k) { a[k] = (float)k; b[k] = (float)(k + threadIdx.x); }
+  const int mode = iters < 0 ? 1 : 0, it = iters < 0 ? -iters : iters;
+  if (mode == 0) {
+#pragma unroll 4
+    for (int i = 0; i < it; ++i)
+#pragma unroll
+      for (int k = 0; k < kProbeChains; ++k) { a[k] += x; b[k] += x; }
+  } else {
+    f32x2 v[kProbeChains];
+    const f32x2 xx = pack2(x, x);
+#pragma unroll
+    for (int k = 0; k < kProbeChains; ++k) v[k] = pack2(a[k], b[k]);
+#pragma unroll 4
+    for (int i = 0; i < it; ++i)
+#pragma unroll
+      for (int k = 0; k < kProbeChains; ++k) v[k] = add2(v[k], xx);
+#pragma unroll
+    for (int k = 0; k < kProbeChains; ++k) { a[k] = lo32(v[k]); b[k] = hi32(v[k]); }
+  }
+  float t = 0.f;
+#pragma unroll
+  for (int k = 0; k < kProbeChains; ++k) t += a[k] + b[k];
+  if (t == 123456.789f) sink[1 + (blockIdx.x * 256 + threadIdx.x) % 1024] = t;    // practically never: keeps the chains alive
+}
+
 }  // namespace ln

@@ -64,9 +64,9 @@ __device__ __forceinline__ void mbar_init(unsigned long long* mbar, int count) {
 }
 // Bounded wait for phase `parity`; returns false if the limit ran out (the caller records an error
 // and carries on: results are then wrong but nothing spins for ever).
-__device__ __forceinline__ bool mbar_wait(unsigned long long* mbar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(unsigned long long* mbar, uint32_t parity, int limit = 1 << 22) {
   uint32_t done = 0;
-  for (int it = 0; it < (1 << 22) && !done; ++it)
+  for (int it = 0; it < limit && !done; ++it)
     asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                  : "=r"(done) : "r"(s32(mbar)), "r"(parity) : "memory");
   return done != 0;

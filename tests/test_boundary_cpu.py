@@ -16,7 +16,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def declared_symbols():
     text = open(os.path.join(ROOT, "include", "laplace_nystrom.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    names = re.findall(r"\b(?:int|size_t|uint64_t|const char\*)\s+(\w+)\s*\(", text)
+    names = re.findall(r"\b(?:int|size_t|uint64_t|int64_t|const char\*)\s+(\w+)\s*\(", text)
     return sorted(set(names))
 
 
@@ -151,3 +151,28 @@ def test_whiten_stats_argument_errors_without_gpu():
     assert lib.laplace_nystrom_whiten_stats(ctypes.byref(cp), None, 1e-5, None, None, 0, None) == -1
     with pytest.raises(ValueError):
         ln.laplace_nystrom_whiten_stats(p, torch.empty(16, dtype=torch.uint8))
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg4a", "cfg5_m256_T12"])
+def test_saved_array_views_lie_inside_the_context(name):
+    """The inspection entry point is pure host arithmetic: every named intermediate lies inside the saved buffer,
+    heads do not overlap, and an unknown name is an argument error."""
+    cfg = synth.CONFIGS[name]
+    p = ln.problem_from_config(cfg)
+    total = ln.laplace_nystrom_saved_bytes(p) // 4
+    cp = p.c()
+    info = (ctypes.c_int64 * 5)()
+    BH = cfg.B * cfg.H
+    spans = []
+    for nm, rows, cols in (("L", cfg.m, cfg.d), ("C", cfg.n, cfg.m), ("Rt", cfg.n, cfg.m), ("mu", 1, cfg.n),
+                           ("W", cfg.m, cfg.m), ("X", cfg.m, cfg.m), ("M", cfg.m, cfg.d), ("Yt", cfg.m, cfg.d),
+                           ("ybar", 1, cfg.d)):
+        assert binding.lib().laplace_nystrom_saved_array(ctypes.byref(cp), nm.encode(), info) == 0
+        off, r, c, ld, stride = (int(v) for v in info)
+        assert (r, c) == (rows, cols) and ld >= c and stride >= (r - 1) * ld + c
+        assert 0 <= off and off + (BH - 1) * stride + (r - 1) * ld + c <= total
+        spans.append((off, off + (BH - 1) * stride + (r - 1) * ld + c, nm))
+    spans.sort()
+    for (a0, a1, na), (b0, b1, nb) in zip(spans, spans[1:]):
+        assert a1 <= b0 or {na, nb} == {"X"}, (na, nb)
+    assert binding.lib().laplace_nystrom_saved_array(ctypes.byref(cp), b"nope", info) == -1

@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2604_20368_b200 as ln
 from paper_2604_20368_b200 import binding
 
@@ -39,12 +40,45 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row():
         torch.cuda.synchronize()
         assert torch.isfinite(X).all()
         assert _rel(X, ref) < 2e-5               # same tolerance as the ns_pinv parity test
-        assert torch.allclose(resid, ref_resid, rtol=1e-3, atol=1e-4)
+        assert torch.equal(X, ref)               # in fact the same kernel on other scratch: the same bits
+        assert torch.equal(resid, ref_resid)
+        # and against the float64 oracle's Alg. 2 iterate, at the bar the ns_pinv parity test uses
+        Xo = oracle.ns_pinv(W.cpu().double().numpy(), T, eps=float(np.float32(eps)))[0]
+        assert float(np.linalg.norm(X.cpu().double().numpy() - Xo) / np.linalg.norm(Xo)) < 2e-5
     # and once more on the first problem, now with the second call's contents lying around
     W, T, eps = calls[0]
     X = torch.empty_like(W)
     ln.ns_pinv_static(W, T, X, ridge_eps=eps)
-    assert _rel(X, ln.ns_pinv(W, T, ridge_eps=eps)[0]) < 2e-5
+    assert torch.equal(X, ln.ns_pinv(W, T, ridge_eps=eps)[0])
+
+
+def test_static_scratch_call_allocates_nothing():
+    """Free device memory as the driver reports it, and what torch's allocator holds, are the same before and
+    after a call: the entry point takes its scratch from the library image, not from an allocator."""
+    W = _matrices(4, 49, 3)
+    X = torch.empty_like(W)
+    ln.ns_pinv_static(W, 6, X)                   # first call on the device: looks up the scratch address
+    torch.cuda.synchronize()
+    free0, reserved0, alloc0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_reserved(), torch.cuda.memory_allocated()
+    for _ in range(3):
+        ln.ns_pinv_static(W, 6, X)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert torch.cuda.memory_reserved() == reserved0 and torch.cuda.memory_allocated() == alloc0
+
+
+def test_static_scratch_largest_documented_case_and_first_one_beyond():
+    lib = binding.lib()
+    limit = lib.ns_pinv_static_scratch_bytes()
+    batch, m, T = 2, 256, 8                      # the largest case the header names: just under the limit
+    assert lib.ns_pinv_workspace_bytes(batch, m, T) <= limit < lib.ns_pinv_workspace_bytes(batch, m, T + 2)
+    W = _matrices(batch, m, 4)
+    X = torch.empty_like(W)
+    ln.ns_pinv_static(W, T, X)
+    assert torch.equal(X, ln.ns_pinv(W, T)[0])
+    with pytest.raises(ln.LnError) as e:         # two more iterates no longer fit
+        ln.ns_pinv_static(W, T + 2, X)
+    assert e.value.status == -5
 
 
 def test_static_scratch_limit_is_reported_and_nothing_runs():
