@@ -262,6 +262,16 @@ int ln_trace_end(int32_t capacity, int32_t* count, float* ms, const char** names
 int ln_set_overlap(int enabled);
 
 /*
+ * Which sign pass the bf16 backward uses for the two token-sized kernel blocks (the paper has no counterpart; App. A
+ * fixes the arithmetic only).  1 (default): one kernel per block forms the upstream factor g = (U Y^T) o A / lambda
+ * on the tensor cores and consumes it in place.  0: the upstream factors are written to the workspace by separate
+ * product kernels and read back by the sign pass (the earlier arrangement, kept for comparison).  Both give the same
+ * gradients up to rounding order.  The setting is read when sizes are computed and when a call is planned: set it
+ * before laplace_nystrom_workspace_bytes and keep it for the calls that use that workspace.  Returns the previous value.
+ */
+int ln_set_fused_sign(int enabled);
+
+/*
  * Number of kernels this library has launched in the process so far (the paper has no counterpart; a bookkeeping aid
  * for benchmarks that report how many launches a timed region held: read it before and after).
  */

@@ -27,7 +27,7 @@ EXPORTS = [
     "ln_trace_begin", "ln_trace_end", "ns_pinv_static_scratch_bytes", "ns_pinv_static",
     "laplace_nystrom_host_staging_bytes", "laplace_nystrom_fwd_bwd_host", "ln_set_overlap", "ln_launch_count",
     "laplace_nystrom_whiten_stats_workspace_bytes", "laplace_nystrom_whiten_stats",
-    "laplace_nystrom_saved_array", "ln_selftest_wait_timeout", "ln_fp32_add_probe", "ln_fp32_add_probe_lane_ops",
+    "laplace_nystrom_saved_array", "ln_set_fused_sign", "ln_selftest_wait_timeout", "ln_fp32_add_probe", "ln_fp32_add_probe_lane_ops",
 ]
 
 
@@ -128,6 +128,7 @@ def lib():
         L.ns_pinv_static.argtypes = [i32, i32, vp, i32, f32, f32, vp, vp, vp]
         L.ln_trace_end.argtypes = [i32, ctypes.POINTER(i32), ctypes.POINTER(f32), ctypes.POINTER(ctypes.c_char_p)]
         L.ln_set_overlap.argtypes = [i32]
+        L.ln_set_fused_sign.argtypes = [i32]
         L.ln_launch_count.restype = ctypes.c_uint64
         L.ln_launch_count.argtypes = []
         L.laplace_nystrom_whiten_stats_workspace_bytes.restype = sz
@@ -328,6 +329,13 @@ def set_overlap(enabled: bool) -> bool:
     """Whether the per-head kernels run on the library's second stream beside the token-sized ones
     (default on); returns the previous setting."""
     return bool(lib().ln_set_overlap(1 if enabled else 0))
+
+
+def set_fused_sign(enabled: bool) -> bool:
+    """Whether the bf16 sign passes form their upstream factor on the tensor cores themselves (default) or read it
+    from the workspace, where separate product kernels left it; returns the previous setting.  Set it before the
+    workspace is sized."""
+    return bool(lib().ln_set_fused_sign(1 if enabled else 0))
 
 
 def laplace_nystrom_whiten_stats(p: Problem, saved, eps_w: float = 1e-5, out=None, ws=None, stream=None):

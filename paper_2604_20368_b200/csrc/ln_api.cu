@@ -7,6 +7,7 @@
 #include "../../include/laplace_nystrom.h"
 #include "ln_kernels.cuh"
 #include "ln_sign2.cuh"
+#include "ln_sign3.cuh"
 #include <atomic>
 #include <mutex>
 #include <unordered_map>
@@ -60,6 +61,8 @@ struct Carver {
   }
 };
 
+std::atomic<bool> g_sign3{true};      // test switch: false = the separate upstream kernels and the two-output sign pass
+
 struct Plan {
   int BH, n, d, m, T, ldm, rpc, chunks;
   size_t scr;                        // floats per scratch matrix of the per-head kernels
@@ -68,6 +71,7 @@ struct Plan {
   int s2q_rpc, s2q_chunks;           // the same for the query-side pass, which shares the GPU with the per-head kernel
   int mid_sms;                       // SMs the per-head kernels occupy (Newton-Schulz and its adjoint)
   size_t s2_smem;
+  int s3_tiles;                      // sign pass with the upstream factor formed in the kernel: token tiles per head (0 = not used)
 };
 
 bool make_plan(const ln_problem* p, Plan* pl) {
@@ -129,6 +133,9 @@ bool make_plan(const ln_problem* p, Plan* pl) {
     pl->s2q_rpc = tpq * 8 * TG; pl->s2q_chunks = (p->n + pl->s2q_rpc - 1) / pl->s2q_rpc;
     pl->s2_smem = sign2_smem_bytes(p->m);
   }
+  // bf16 storage, 64 or 128 dims: one CTA per tile of 8 * TG tokens, upstream factor on the tensor cores in the kernel
+  pl->s3_tiles = (p->dtype == LN_BF16 && (p->d == 64 || p->d == 128) && g_sign3.load(std::memory_order_relaxed))
+                     ? (p->n + 8 * pl->s2_tg - 1) / (8 * pl->s2_tg) : 0;
   return true;
 }
 
@@ -169,16 +176,18 @@ FwdWs carve_fwd_ws(const Plan& pl, void* base) {
 }
 
 struct BwdWs {
-  float *G, *G2, *dYtpart, *dybpart, *dLCpart, *dLRpart, *dY, *dM, *Wr, *P, *Hm, *Ga, *Gb, *dW, *dX, *GW, *dLW, *dLtot, *dKpart, *dMimg;
+  float *G, *G2, *dYtpart, *dybpart, *dLCpart, *dLRpart, *dY, *dM, *Wr, *P, *Hm, *Ga, *Gb, *dW, *dX, *GW, *dLW, *dLtot, *dKpart, *dMimg, *SB;
   size_t bytes;
 };
 BwdWs carve_bwd_ws(const Plan& pl, void* base) {
   Carver c(base); BwdWs w;
   const size_t BH = pl.BH, n = pl.n, d = pl.d, m = pl.m, ch = pl.chunks;
-  const size_t chs = pl.s2_chunks > 0 ? (size_t)pl.s2_chunks : ch;     // chunks of the landmark-gradient partials
-  const size_t chq = pl.s2_chunks > 0 ? (size_t)pl.s2q_chunks : ch;
-  w.G = c.take(BH * n * pl.ldm);
-  w.G2 = c.take(BH * n * pl.ldm);       // upstream of the key-side block (its own buffer: it is formed while the query side reads G)
+  size_t chs = pl.s2_chunks > 0 ? (size_t)pl.s2_chunks : ch;     // chunks of the landmark-gradient partials
+  size_t chq = pl.s2_chunks > 0 ? (size_t)pl.s2q_chunks : ch;
+  if (pl.s3_tiles > 0) chs = chq = (size_t)pl.s3_tiles;
+  // upstream factors g of the two token-sized blocks; not materialised when the sign pass forms them itself
+  w.G = c.take(pl.s3_tiles > 0 ? 0 : BH * n * pl.ldm);
+  w.G2 = c.take(pl.s3_tiles > 0 ? 0 : BH * n * pl.ldm);       // its own buffer: it is formed while the query side reads G
   w.dYtpart = c.take(BH * ch * m * d);
   w.dybpart = c.take(BH * ch * d);
   w.dLCpart = c.take(BH * chq * m * d);
@@ -197,6 +206,7 @@ BwdWs carve_bwd_ws(const Plan& pl, void* base) {
   w.dLtot = c.take(BH * m * d);
   w.dKpart = c.take(BH * n * d);
   w.dMimg = c.take(BH * image_floats(pl));
+  w.SB = c.take(pl.s3_tiles > 0 ? BH * m * 2 * d : 0);      // scale and offset of every landmark value (folded step)
   w.bytes = c.off;
   return w;
 }
@@ -516,8 +526,21 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     }
   };
   const bool fused_sign = pl.s2_chunks > 0;
-  const int chs = fused_sign ? pl.s2_chunks : ch;
-  const int chq = fused_sign ? pl.s2q_chunks : ch;    // chunks of the query-side landmark-gradient partials
+  const bool sign3 = pl.s3_tiles > 0;                 // the sign passes form their upstream factor themselves (tcgen05)
+  const int chs = sign3 ? pl.s3_tiles : (fused_sign ? pl.s2_chunks : ch);
+  const int chq = sign3 ? pl.s3_tiles : (fused_sign ? pl.s2q_chunks : ch);    // chunks of the query-side landmark-gradient partials
+  // one sign pass of a token-sized block: tokens, upstream operands (U, pre-split images of Y), kernel block A
+  auto launch_sign3 = [&](const char* name, const T* tokp, const T* Up, const float* Yimgp, const float* Ap, auto* rowsp, float* partp) {
+    if constexpr (std::is_same<T, bf16>::value && (D == 64 || D == 128)) {
+      auto go = [&](auto kern) {
+        want_smem(kern, sign3_smem_bytes());
+        LN_LAUNCH(name, st, kern<<<dim3(pl.s3_tiles, D / 64, BH), dim3(16, pl.s2_tg), sign3_smem_bytes(), st>>>(
+                      tokp, w.SB, Up, reinterpret_cast<const bf16*>(Yimgp), Ap, pl.ldm, rowsp, partp, n, m, inv_lambda, dev_status));
+      };
+      using TO = std::remove_pointer_t<decltype(rowsp)>;
+      if (pl.s2_tg == S3_TGMAX) go(k_sign3<TO, D, 1, true>); else go(k_sign3<TO, D, 2, true>);
+    }
+  };
   // The per-head kernel and the landmark-block sign pass need Z'^T dO only: with a side stream they run beside
   // the query-side kernels and are joined before the key side, which needs dM.
   const Side side = side_acquire(std::is_same<T, bf16>::value, st);
@@ -583,13 +606,18 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     side.fork(st);
     if (tn_on_side) launch_tn_dY(side.s);
     launch_mid(side.s);
-    if (ntg_on_side) launch_ntg_R(side.s);
+    if (ntg_on_side && !sign3) launch_ntg_R(side.s);
     side.mark();                     // what the second sign pass needs from this stream ends here
     launch_nn_dV(side.s);
     launch_sign_W(side.s);
   }
-  launch_ntg_C();
-  if (fused_sign) {
+  if (sign3) {
+    const long long cnt = (long long)BH * m * D;
+    LN_LAUNCH("k_fold_landmarks", st, k_fold_landmarks<<<cdiv(cnt, 256), 256, 0, st>>>(x.Lf, w.SB, D, cnt));
+    launch_sign3("sign3_dQ_dLC", Q, dO, x.Yimg, x.C, dQ, w.dLCpart);
+  } else launch_ntg_C();
+  if (sign3) {
+  } else if (fused_sign) {
     auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
       want_smem(kern, pl.s2_smem);
       LN_LAUNCH(name, st, kern<<<dim3(chq, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(tokp, x.Lf, w.G, pl.ldm, rowsp, partp, n, m, D, pl.s2q_rpc));
@@ -600,10 +628,12 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m));
     LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
   }
-  if (side.on()) { side.join_mark(st); if (!ntg_on_side) launch_ntg_R(st); }
-  else { launch_mid(st); launch_sign_W(st); launch_ntg_R(st); launch_nn_dV(st); }
+  if (side.on()) { side.join_mark(st); if (!ntg_on_side && !sign3) launch_ntg_R(st); }
+  else { launch_mid(st); launch_sign_W(st); if (!sign3) launch_ntg_R(st); launch_nn_dV(st); }
   // key side: dK (kernel part); landmark part
-  if (fused_sign) {
+  if (sign3) {
+    launch_sign3("sign3_dK_dLR", K, V, w.dMimg, x.Rt, w.dKpart, w.dLRpart);
+  } else if (fused_sign) {
     auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
       want_smem(kern, pl.s2_smem);
       LN_LAUNCH(name, st, kern<<<dim3(chs, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(tokp, x.Lf, w.G2, pl.ldm, rowsp, partp, n, m, D, pl.s2_rpc));
@@ -716,6 +746,8 @@ int ln_trace_end(int32_t capacity, int32_t* count, float* ms, const char** names
 }
 
 uint64_t ln_launch_count(void) { return (uint64_t)g_launch_count.load(std::memory_order_relaxed); }
+
+int ln_set_fused_sign(int enabled) { return g_sign3.exchange(enabled != 0) ? 1 : 0; }
 
 int ln_set_overlap(int enabled) {
   return g_overlap.exchange(enabled != 0) ? 1 : 0;

@@ -75,9 +75,21 @@ __device__ __forceinline__ void fold_pair(float y, float& s, float& b) {
 typedef unsigned long long f32x2;
 __device__ __forceinline__ f32x2 add2(f32x2 x, f32x2 y) { f32x2 z; asm("add.f32x2 %0, %1, %2;" : "=l"(z) : "l"(x), "l"(y)); return z; }
 __device__ __forceinline__ f32x2 fma2(f32x2 x, f32x2 y, f32x2 c) { f32x2 z; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(z) : "l"(x), "l"(y), "l"(c)); return z; }
-__device__ __forceinline__ float lo32(f32x2 x) { return __uint_as_float((unsigned)x); }
-__device__ __forceinline__ float hi32(f32x2 x) { return __uint_as_float((unsigned)(x >> 32)); }
-__device__ __forceinline__ f32x2 pack2(float a, float b) { return (f32x2)__float_as_uint(a) | ((f32x2)__float_as_uint(b) << 32); }
+__device__ __forceinline__ f32x2 mul2(f32x2 x, f32x2 y) { f32x2 z; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(z) : "l"(x), "l"(y)); return z; }
+// Halves of a pair and a pair from two halves, written as register-pair moves: spelled with 64-bit shifts and ORs the
+// compiler emits real integer instructions for them, which cost issue slots in the FP32-bound inner loops.
+__device__ __forceinline__ float lo32(f32x2 x) { float a, b; asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(x)); return a; }
+__device__ __forceinline__ float hi32(f32x2 x) { float a, b; asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(x)); return b; }
+__device__ __forceinline__ f32x2 pack2(float a, float b) { f32x2 z; asm("mov.b64 %0, {%1, %2};" : "=l"(z) : "f"(a), "f"(b)); return z; }
+// both halves at once
+__device__ __forceinline__ void unpack2(f32x2 x, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(x)); }
+// (min(max(x0 s + b, 0), 1), min(max(x1 s + b, 0), 1)) as a pair: two saturating multiply-adds that write the two halves
+__device__ __forceinline__ f32x2 sat_fma_pair(float x0, float x1, float s, float b) {
+  f32x2 z;
+  asm("{\n\t.reg .f32 lo, hi;\n\tfma.rn.sat.f32 lo, %1, %3, %4;\n\tfma.rn.sat.f32 hi, %2, %3, %4;\n\tmov.b64 %0, {lo, hi};\n\t}"
+      : "=l"(z) : "f"(x0), "f"(x1), "f"(s), "f"(b));
+  return z;
+}
 
 // Sum of nparts partial arrays (fixed order p = 0, 1, ...), four consecutive elements at `off`.
 // Eight independent loads are issued per batch so that their latencies overlap.

@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(256, 2) k_sign3(const bf16* __restrict__ tok, 
       float g[4] = {apre[u].x, apre[u].y, apre[u].z, apre[u].w};
       if constexpr (FUSED) {
         float da[4];
-        s3_tmem_ld4(umma::tmem_addr(tmem_base, l), da);
+        s3_tmem_ld4(tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)l, da);
 #pragma unroll
         for (int e = 0; e < 4; ++e) g[e] *= da[e];
       }
@@ -227,14 +227,15 @@ __global__ void __launch_bounds__(256, 2) k_sign3(const bf16* __restrict__ tok, 
   s3_cp_async_wait();
   __syncthreads();
 
-  // column outputs of a round: 8 landmarks x 64 dims = 256 float2; thread o takes landmark o / 32, dims 2 (o % 32)
+  // column outputs of a round: 8 landmarks x 64 dims = 256 float2; thread o takes landmark o / 32, dims 2 (o % 32).
+  // A thread's second output may not exist (o >= 256): it then adds up the partials of output 0 and stores nothing.
   int cjj[NR], coff[NR], csrc[NR];
 #pragma unroll
   for (int u = 0; u < NR; ++u) {
-    const int o = tid + u * nthr;
+    const int o = tid + u * nthr, oc = o < S3_RL * 32 ? o : 0;
     cjj[u] = (o < S3_RL * 32) ? (o >> 5) : (1 << 20);
-    coff[u] = (o >> 5) * D + 2 * (o & 31);
-    csrc[u] = (o >> 5) * (S3_TGMAX * S3_DS) + 2 * (o & 31);
+    coff[u] = (oc >> 5) * D + 2 * (oc & 31);
+    csrc[u] = (oc >> 5) * (S3_TGMAX * S3_DS) + 2 * (oc & 31);
   }
   f32x2 accR[4][4];                                                  // [token pair][dim]: lo = even token, hi = odd token
 #pragma unroll
@@ -263,10 +264,9 @@ __global__ void __launch_bounds__(256, 2) k_sign3(const bf16* __restrict__ tok, 
     }
 #pragma unroll
     for (int jj = 0; jj < S3_RL; ++jj) {
-      if (r > 0 && (jj & 1) == 0) {              // a quarter of the previous round's partial sums
-#pragma unroll
-        for (int u = 0; u < NR; ++u)
-          if (cjj[u] < mleft_prev) {
+      if ((jj & 1) == 0) {                       // a quarter of the previous round's partial sums (round 0 adds up
+#pragma unroll                                   // whatever the buffer holds and stores nothing)
+        for (int u = 0; u < NR; ++u) {
             const float* src = rsrc + csrc[u] + (jj * 2) * S3_DS;
             const float2 a0 = *reinterpret_cast<const float2*>(src), a1 = *reinterpret_cast<const float2*>(src + S3_DS);
             const float2 a2 = *reinterpret_cast<const float2*>(src + 2 * S3_DS), a3 = *reinterpret_cast<const float2*>(src + 3 * S3_DS);
@@ -280,17 +280,19 @@ __global__ void __launch_bounds__(256, 2) k_sign3(const bf16* __restrict__ tok, 
       const ulonglong2 gc = *reinterpret_cast<const ulonglong2*>(gb + jj * S3_TOK + 4);
       const f32x2 gp[4] = {ga.x, ga.y, gc.x, gc.y};                 // (g of tokens 2 kp, 2 kp + 1)
       const float sv[4] = {s4.x, s4.y, s4.z, s4.w}, bv[4] = {b4.x, b4.y, b4.z, b4.w};
-      f32x2 cacc[4] = {0ull, 0ull, 0ull, 0ull};
+      f32x2 cacc[4];
 #pragma unroll
       for (int kp = 0; kp < 4; ++kp)
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          const f32x2 h = pack2(sat_fma(x[2 * kp][c], sv[c], bv[c]), sat_fma(x[2 * kp + 1][c], sv[c], bv[c]));
+          const f32x2 h = sat_fma_pair(x[2 * kp][c], x[2 * kp + 1][c], sv[c], bv[c]);
           accR[kp][c] = fma2(gp[kp], h, accR[kp][c]);
-          cacc[c] = fma2(gp[kp], h, cacc[c]);
+          cacc[c] = kp == 0 ? mul2(gp[kp], h) : fma2(gp[kp], h, cacc[c]);
         }
-      *reinterpret_cast<float4*>(cp + jj * (S3_TGMAX * S3_DS)) =
-          make_float4(lo32(cacc[0]) + hi32(cacc[0]), lo32(cacc[1]) + hi32(cacc[1]), lo32(cacc[2]) + hi32(cacc[2]), lo32(cacc[3]) + hi32(cacc[3]));
+      float ce[4], co[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) unpack2(cacc[c], ce[c], co[c]);
+      *reinterpret_cast<float4*>(cp + jj * (S3_TGMAX * S3_DS)) = make_float4(ce[0] + co[0], ce[1] + co[1], ce[2] + co[2], ce[3] + co[3]);
     }
     if (r > 0) {
       float* dst = outp + (long long)(r - 1) * S3_RL * D;
