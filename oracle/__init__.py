@@ -208,3 +208,80 @@ def whiten_stats(C, H, eps_w):
         var /= cnt
         s[h] = 1.0 / np.sqrt(var + eps_w)
     return s
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# The steps either side of the path inside the attention block: rotary position embedding on Q and K (Sec. 5.1) and
+# Attention = Z V + DWC(V) (Eq. 7)
+def rope(X, prefix=0, base=10000.0, inverse=False):
+    """Rotary position embedding of X [B,H,n,d] (d even): channel pairs (2i, 2i+1) of the token at grid position p
+    are rotated by p * base^(-2i/d); the `prefix` leading tokens are left alone.  inverse=True applies the transpose."""
+    X = _f64(X)
+    B, H, n, d = X.shape
+    out = np.empty_like(X)
+    _load().oracle_rope(B * H, n, d, prefix, ctypes.c_double(base), int(inverse), _p(X), _p(out))
+    return out
+
+
+def dwc(V, Wd, prefix, gh, gw):
+    """Depth-wise ks x ks cross-correlation of V [B,H,n,d] over the gh x gw token grid, zero padded, one filter per
+    head and channel: Wd [H,d,ks,ks].  Prefix tokens receive 0."""
+    V, Wd = _f64(V), _f64(Wd)
+    B, H, n, d = V.shape
+    ks = Wd.shape[-1]
+    assert Wd.shape == (H, d, ks, ks) and ks % 2 == 1 and n == prefix + gh * gw
+    out = np.empty_like(V)
+    _load().oracle_dwc(B, H, n, d, prefix, gh, gw, ks, _p(V), _p(Wd), _p(out))
+    return out
+
+
+def dwc_bwd(V, Wd, dO, prefix, gh, gw):
+    """Adjoint of dwc: returns dV [B,H,n,d] and dWd [H,d,ks,ks] (summed over the batch)."""
+    V, Wd, dO = _f64(V), _f64(Wd), _f64(dO)
+    B, H, n, d = V.shape
+    ks = Wd.shape[-1]
+    dV, dWd = np.empty_like(V), np.empty_like(Wd)
+    _load().oracle_dwc_bwd(B, H, n, d, prefix, gh, gw, ks, _p(V), _p(Wd), _p(dO), _p(dV), _p(dWd))
+    return dV, dWd
+
+
+def round_bf16(x):
+    """Nearest bf16 value (ties to even) of every element, returned as float64: the storage rounding a tensor takes
+    when the device keeps it in bf16."""
+    f = np.ascontiguousarray(np.asarray(x, dtype=np.float64)).astype(np.float32)
+    bits = f.view(np.uint32)
+    bits = (bits + (np.uint32(0x7FFF) + ((bits >> np.uint32(16)) & np.uint32(1)))) & np.uint32(0xFFFF0000)
+    return bits.view(np.float32).astype(np.float64)
+
+
+def block_forward(p: Problem, Q, K, V, Wd=None, rope_base=0.0, whiten=None, store_bf16=False):
+    """The attention block around the path: rotary embedding on Q and K (rope_base > 0), the Nystrom Laplacian
+    attention, plus DWC(V) (Wd given).  store_bf16: the rotated Q and K are rounded to bf16, as a device that keeps
+    them in bf16 storage does (the kernel gradient's sign(token - landmark) must be decided on the same numbers)."""
+    Qr, Kr = _f64(Q), _f64(K)
+    if rope_base > 0:
+        Qr, Kr = rope(Qr, p.prefix, rope_base), rope(Kr, p.prefix, rope_base)
+        if store_bf16:
+            Qr, Kr = round_bf16(Qr), round_bf16(Kr)
+    O = forward(p, Qr, Kr, V, whiten=whiten)
+    if Wd is not None:
+        O = O + dwc(V, Wd, p.prefix, p.gh, p.gw)
+    return O
+
+
+def block_backward(p: Problem, Q, K, V, dO, Wd=None, rope_base=0.0, whiten=None, store_bf16=False):
+    """Adjoint of block_forward: dQ, dK, dV, dWd (None without the convolution).  The rounding of the rotated
+    tensors, where asked for, is treated as the identity (straight-through), as storage rounding is everywhere."""
+    Qr, Kr = _f64(Q), _f64(K)
+    if rope_base > 0:
+        Qr, Kr = rope(Qr, p.prefix, rope_base), rope(Kr, p.prefix, rope_base)
+        if store_bf16:
+            Qr, Kr = round_bf16(Qr), round_bf16(Kr)
+    dQr, dKr, dV, _ = backward(p, Qr, Kr, V, dO, whiten=whiten)
+    dWd = None
+    if Wd is not None:
+        dV2, dWd = dwc_bwd(V, Wd, dO, p.prefix, p.gh, p.gw)
+        dV = dV + dV2
+    if rope_base > 0:
+        dQr, dKr = rope(dQr, p.prefix, rope_base, inverse=True), rope(dKr, p.prefix, rope_base, inverse=True)
+    return dQr, dKr, dV, dWd

@@ -40,6 +40,10 @@
  *   - optionally (lm_f32) a pooled landmark is the single-precision value nearest to the
  *     exact mean, so that sign(token - landmark) is decided on the numbers the device holds.
  *
+ * Beside the path, the two steps that surround it inside the attention block (end of this file): the rotary
+ * position embedding on Q and K (Sec. 5.1; positions over the flattened token grid, class tokens not rotated) and
+ * Attention = Z V + DWC(V) (Eq. 7; one ks x ks zero-padded cross-correlation filter per head and channel).
+ *
  * Pins (tests/test_oracle_*.py): hand values, brute force in numpy, the
  * Kac-Murdock-Szego closed-form inverse, the spectral closed form of the
  * unconverged Newton-Schulz iterate, m = n reproducing exact Laplacian
@@ -505,5 +509,96 @@ void oracle_bwd(const oracle_problem* p, const double* Q, const double* K, const
     bwd_single(p, Q + h * nd, K + h * nd, V + h * nd, Lin ? Lin + h * md : NULL,
                whiten ? whiten + (size_t)(h % p->H) * m : NULL, dO + h * nd,
                dQ + h * nd, dK + h * nd, dV + h * nd, dL ? dL + h * md : NULL);
+  }
+}
+
+/* ========================================================================= */
+/* The steps either side of the path inside the attention block              */
+/*   Attention(Q, K, V) = Z V + DWC(V)              (Eq. 7)                   */
+/*   rotary position embedding on Q and K           (Sec. 5.1, implementation) */
+/* ========================================================================= */
+
+/*
+ * Rotary position embedding (Sec. 5.1 adopts RoPE; the rotation is that of the RoFormer paper it cites):
+ * token at position p, channel pair (2i, 2i+1), angle theta = p * base^(-2i/d):
+ *     x'_{2i} = x_{2i} cos(theta) - x_{2i+1} sin(theta),   x'_{2i+1} = x_{2i} sin(theta) + x_{2i+1} cos(theta).
+ * Reading: positions run over the flattened token grid (row-major), p = token index - prefix; the `prefix`
+ * leading tokens (class tokens) are not rotated.  inverse != 0 applies the transpose (the adjoint of the map).
+ * X, out: [BH, n, d], d even.
+ */
+void oracle_rope(int BH, int n, int d, int prefix, double base, int inverse, const double* X, double* out) {
+#pragma omp parallel for schedule(static)
+  for (int bh = 0; bh < BH; ++bh)
+    for (int t = 0; t < n; ++t) {
+      const double* x = X + ((size_t)bh * n + t) * d;
+      double* o = out + ((size_t)bh * n + t) * d;
+      for (int i = 0; i < d / 2; ++i) {
+        double a = x[2 * i], b = x[2 * i + 1];
+        if (t < prefix) { o[2 * i] = a; o[2 * i + 1] = b; continue; }
+        double theta = (double)(t - prefix) * pow(base, -2.0 * (double)i / (double)d);
+        double c = cos(theta), s = sin(theta);
+        if (inverse) s = -s;
+        o[2 * i] = a * c - b * s;
+        o[2 * i + 1] = a * s + b * c;
+      }
+    }
+}
+
+/*
+ * Depth-wise convolution over the value sequence (Eq. 7): every channel c of head h has its own ks x ks filter
+ * Wd[h][c][a][b] (ks odd), applied over the gh x gw token grid with zero padding (a cross-correlation, as in every
+ * deep-learning framework):
+ *     out[r, q, c] = sum_{a, b} Wd[h][c][a][b] * V[r + a - ks/2, q + b - ks/2, c].
+ * Reading: the `prefix` leading tokens are not on the grid and receive 0.
+ * V, out: [B, H, n, d] with n = prefix + gh * gw; Wd: [H, d, ks, ks].
+ */
+void oracle_dwc(int B, int H, int n, int d, int prefix, int gh, int gw, int ks, const double* V, const double* Wd, double* out) {
+  int half = ks / 2;
+#pragma omp parallel for schedule(static)
+  for (int bh = 0; bh < B * H; ++bh) {
+    int h = bh % H;
+    const double* Vh = V + (size_t)bh * n * d;
+    double* Oh = out + (size_t)bh * n * d;
+    for (int t = 0; t < prefix; ++t)
+      for (int c = 0; c < d; ++c) Oh[(size_t)t * d + c] = 0.0;
+    for (int r = 0; r < gh; ++r)
+      for (int q = 0; q < gw; ++q)
+        for (int c = 0; c < d; ++c) {
+          double acc = 0.0;
+          for (int a = 0; a < ks; ++a)
+            for (int b = 0; b < ks; ++b) {
+              int rr = r + a - half, qq = q + b - half;
+              if (rr < 0 || rr >= gh || qq < 0 || qq >= gw) continue;
+              acc += Wd[(((size_t)h * d + c) * ks + a) * ks + b] * Vh[(size_t)(prefix + rr * gw + qq) * d + c];
+            }
+          Oh[(size_t)(prefix + r * gw + q) * d + c] = acc;
+        }
+  }
+}
+
+/* Adjoint of oracle_dwc: dV [B,H,n,d] and dWd [H,d,ks,ks] (summed over the batch) from dO = dLoss/d out. */
+void oracle_dwc_bwd(int B, int H, int n, int d, int prefix, int gh, int gw, int ks, const double* V, const double* Wd,
+                    const double* dO, double* dV, double* dWd) {
+  int half = ks / 2;
+  memset(dV, 0, sizeof(double) * (size_t)B * H * n * d);
+  memset(dWd, 0, sizeof(double) * (size_t)H * d * ks * ks);
+  for (int bh = 0; bh < B * H; ++bh) {               /* serial over heads: dWd is shared by the batch elements of a head */
+    int h = bh % H;
+    const double* Vh = V + (size_t)bh * n * d;
+    const double* Gh = dO + (size_t)bh * n * d;
+    double* dVh = dV + (size_t)bh * n * d;
+    for (int r = 0; r < gh; ++r)
+      for (int q = 0; q < gw; ++q)
+        for (int c = 0; c < d; ++c) {
+          double g = Gh[(size_t)(prefix + r * gw + q) * d + c];
+          for (int a = 0; a < ks; ++a)
+            for (int b = 0; b < ks; ++b) {
+              int rr = r + a - half, qq = q + b - half;
+              if (rr < 0 || rr >= gh || qq < 0 || qq >= gw) continue;
+              size_t wi = (((size_t)h * d + c) * ks + a) * ks + b, vi = (size_t)(prefix + rr * gw + qq) * d + c;
+              dVh[vi] += Wd[wi] * g;
+              dWd[wi] += Vh[vi] * g;
+            }
+        }
   }
 }
