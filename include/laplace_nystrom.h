@@ -126,6 +126,32 @@ int laplace_nystrom_fwd_bwd_host(const ln_problem* p, const void* hQ, const void
                                  void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
 
 /*
+ * The attention block around the path (Eq. 7 and the implementation details of Sec. 5.1):
+ *     Qr = rope(Q), Kr = rope(K);   O = Z(Qr, Kr) Y(Kr, V) + DWC(V).
+ * rope: rotary position embedding, channel pairs (2i, 2i+1) of the token at grid position p (row-major over the
+ *   gh x gw grid; the `prefix` class tokens are not rotated) turn by p * rope_base^(-2i/d); rope_base = 0 switches it
+ *   off.  The rotated tensors are kept in the storage type (bf16 storage rounds them once more).
+ * DWC: depth-wise ks x ks cross-correlation over the token grid, zero padded, one filter per head and channel,
+ *   dwc_w device fp32 [H, d, ks, ks] (ks odd, <= 7), NULL = no convolution branch; prefix tokens receive nothing.
+ * lm_mode must be 1 (the grid geometry of `p` is used), else LN_ERR_UNSUPPORTED.
+ *   saved: laplace_attention_block_saved_bytes bytes; ws: laplace_attention_block_workspace_bytes bytes (both
+ *   passes); the other arguments as for laplace_nystrom_fwd / _bwd.  The backward returns dQ, dK, dV and, when the
+ *   convolution branch is on, dWd device fp32 [H, d, ks, ks] (summed over the batch in a fixed order), else dWd = NULL.
+ */
+typedef struct ln_block {
+  const float* dwc_w;
+  int32_t dwc_ks;
+  float rope_base;
+} ln_block;
+size_t laplace_attention_block_saved_bytes(const ln_problem* p, const ln_block* b);
+size_t laplace_attention_block_workspace_bytes(const ln_problem* p, const ln_block* b);
+int laplace_attention_block_fwd(const ln_problem* p, const ln_block* b, const void* Q, const void* K, const void* V, void* O,
+                                void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+int laplace_attention_block_bwd(const ln_problem* p, const ln_block* b, const void* Q, const void* K, const void* V,
+                                const void* dO, const void* saved, void* dQ, void* dK, void* dV, float* dWd, void* ws,
+                                size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/*
  * Newton-Schulz iterate of (W + eps I)^-1 (Alg. 2), batched over `batch` independent m x m
  * fp32 matrices.  X [batch,m,m] receives X_T.  X_hist is NULL or [batch,iters+1,m,m] and
  * receives X_0 .. X_T.  resid is NULL or [batch] and receives ||I - (W + eps I) X_T||_F.

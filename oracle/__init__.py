@@ -246,12 +246,11 @@ def dwc_bwd(V, Wd, dO, prefix, gh, gw):
 
 
 def round_bf16(x):
-    """Nearest bf16 value (ties to even) of every element, returned as float64: the storage rounding a tensor takes
-    when the device keeps it in bf16."""
-    f = np.ascontiguousarray(np.asarray(x, dtype=np.float64)).astype(np.float32)
-    bits = f.view(np.uint32)
-    bits = (bits + (np.uint32(0x7FFF) + ((bits >> np.uint32(16)) & np.uint32(1)))) & np.uint32(0xFFFF0000)
-    return bits.view(np.float32).astype(np.float64)
+    """Nearest bf16 value (8 significant bits, ties to even) of every element, rounded once from float64 and returned
+    as float64: the storage rounding a tensor takes when the device keeps it in bf16 (normal range only)."""
+    x = np.asarray(x, dtype=np.float64)
+    mant, expo = np.frexp(x)                       # x = mant * 2^expo, 0.5 <= |mant| < 1
+    return np.ldexp(np.rint(mant * 256.0) / 256.0, expo)      # rint rounds halves to even
 
 
 def block_forward(p: Problem, Q, K, V, Wd=None, rope_base=0.0, whiten=None, store_bf16=False):

@@ -27,7 +27,8 @@ EXPORTS = [
     "ln_trace_begin", "ln_trace_end", "ns_pinv_static_scratch_bytes", "ns_pinv_static",
     "laplace_nystrom_host_staging_bytes", "laplace_nystrom_fwd_bwd_host", "ln_set_overlap", "ln_launch_count",
     "laplace_nystrom_whiten_stats_workspace_bytes", "laplace_nystrom_whiten_stats",
-    "laplace_nystrom_saved_array", "ln_set_fused_sign", "ln_selftest_wait_timeout", "ln_fp32_add_probe", "ln_fp32_add_probe_lane_ops",
+    "laplace_nystrom_saved_array", "ln_set_fused_sign", "laplace_attention_block_saved_bytes",
+    "laplace_attention_block_workspace_bytes", "laplace_attention_block_fwd", "laplace_attention_block_bwd", "ln_selftest_wait_timeout", "ln_fp32_add_probe", "ln_fp32_add_probe_lane_ops",
 ]
 
 
@@ -46,6 +47,10 @@ class _CProblem(ctypes.Structure):
         ("prefix", ctypes.c_int32), ("gh", ctypes.c_int32), ("gw", ctypes.c_int32),
         ("mh", ctypes.c_int32), ("mw", ctypes.c_int32),
     ]
+
+
+class _CBlock(ctypes.Structure):
+    _fields_ = [("dwc_w", ctypes.c_void_p), ("dwc_ks", ctypes.c_int32), ("rope_base", ctypes.c_float)]
 
 
 @dataclass
@@ -139,6 +144,13 @@ def lib():
         L.ln_fp32_add_probe.argtypes = [i32, i32, i32, vp, vp]
         L.ln_fp32_add_probe_lane_ops.restype = ctypes.c_int64
         L.ln_fp32_add_probe_lane_ops.argtypes = [i32, i32]
+        pb = ctypes.POINTER(_CBlock)
+        L.laplace_attention_block_saved_bytes.restype = sz
+        L.laplace_attention_block_saved_bytes.argtypes = [pp, pb]
+        L.laplace_attention_block_workspace_bytes.restype = sz
+        L.laplace_attention_block_workspace_bytes.argtypes = [pp, pb]
+        L.laplace_attention_block_fwd.argtypes = [pp, pb, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.laplace_attention_block_bwd.argtypes = [pp, pb, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         _lib = L
     return _lib
 
@@ -329,6 +341,46 @@ def set_overlap(enabled: bool) -> bool:
     """Whether the per-head kernels run on the library's second stream beside the token-sized ones
     (default on); returns the previous setting."""
     return bool(lib().ln_set_overlap(1 if enabled else 0))
+
+
+class Block:
+    """The steps around the path inside the attention block: rotary embedding base (0 = off) and the depth-wise
+    convolution filters (device fp32 [H, d, ks, ks] or None)."""
+
+    def __init__(self, dwc_w: Optional[torch.Tensor] = None, rope_base: float = 0.0):
+        self.dwc_w, self.rope_base = dwc_w, float(rope_base)
+        if dwc_w is not None:
+            assert dwc_w.is_cuda and dwc_w.dtype == torch.float32 and dwc_w.is_contiguous() and dwc_w.dim() == 4
+            assert dwc_w.shape[2] == dwc_w.shape[3]
+
+    def c(self) -> _CBlock:
+        return _CBlock(None if self.dwc_w is None else self.dwc_w.data_ptr(), 0 if self.dwc_w is None else int(self.dwc_w.shape[-1]),
+                       self.rope_base)
+
+
+def laplace_attention_block_fwd(p: Problem, blk: Block, Q, K, V, saved=None, ws=None, O=None, dev_status=None, stream=None):
+    """O = Z(rope(Q), rope(K)) Y + DWC(V) (Eq. 7, Sec. 5.1).  Returns O, saved, ws (allocated when not given)."""
+    cp, cb = p.c(), blk.c()
+    if saved is None:
+        saved = _bytes(lib().laplace_attention_block_saved_bytes(ctypes.byref(cp), ctypes.byref(cb)), Q.device)
+    if ws is None:
+        ws = _bytes(lib().laplace_attention_block_workspace_bytes(ctypes.byref(cp), ctypes.byref(cb)), Q.device)
+    if O is None:
+        O = torch.empty_like(Q)
+    _check(lib().laplace_attention_block_fwd(ctypes.byref(cp), ctypes.byref(cb), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(saved),
+                                             _ptr(ws), ws.numel(), _ptr(dev_status), _stream(stream)), "laplace_attention_block_fwd")
+    return O, saved, ws
+
+
+def laplace_attention_block_bwd(p: Problem, blk: Block, Q, K, V, dO, saved, ws, dev_status=None, stream=None):
+    """Adjoint of laplace_attention_block_fwd: dQ, dK, dV, dWd (None without the convolution branch)."""
+    cp, cb = p.c(), blk.c()
+    dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+    dWd = None if blk.dwc_w is None else torch.empty_like(blk.dwc_w)
+    _check(lib().laplace_attention_block_bwd(ctypes.byref(cp), ctypes.byref(cb), _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(saved),
+                                             _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dWd), _ptr(ws), ws.numel(), _ptr(dev_status),
+                                             _stream(stream)), "laplace_attention_block_bwd")
+    return dQ, dK, dV, dWd
 
 
 def set_fused_sign(enabled: bool) -> bool:

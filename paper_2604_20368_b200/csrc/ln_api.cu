@@ -8,6 +8,7 @@
 #include "ln_kernels.cuh"
 #include "ln_sign2.cuh"
 #include "ln_sign3.cuh"
+#include "ln_block.cuh"
 #include <atomic>
 #include <mutex>
 #include <unordered_map>
@@ -1113,5 +1114,116 @@ int ln_fp32_add_probe(int32_t blocks, int32_t iters, int32_t packed, float* sink
   return launch_ok();
 }
 int64_t ln_fp32_add_probe_lane_ops(int32_t blocks, int32_t iters) { return (int64_t)blocks * 256 * iters * kProbeChains * 2; }
+
+// ------------------------------------------------------------------------------------------
+// The attention block around the path: rotary embedding on Q and K, Nystrom Laplacian attention, + DWC(V)
+// ------------------------------------------------------------------------------------------
+}  // extern "C"
+namespace {
+int validate_block(const ln_problem* p, const ln_block* b) {
+  int s = validate(p);
+  if (s != LN_OK) return s;
+  if (!b) return LN_ERR_ARG;
+  if (p->lm_mode != 1) return LN_ERR_UNSUPPORTED;            // the token grid is needed
+  if (!(b->rope_base >= 0.f) || !isfinite(b->rope_base)) return LN_ERR_ARG;
+  if (b->rope_base > 0.f && (b->rope_base <= 1.f || (p->d & 3))) return LN_ERR_ARG;
+  if (b->dwc_w && (b->dwc_ks < 1 || b->dwc_ks > 7 || (b->dwc_ks & 1) == 0 || !aligned16(b->dwc_w))) return LN_ERR_ARG;
+  return LN_OK;
+}
+size_t tensor_bytes(const ln_problem* p) { return align_up((size_t)p->B * p->H * p->n * p->d * (p->dtype == LN_F32 ? 4 : 2), 256); }
+constexpr int kDwcTokensPerChunk = 512;
+int dwc_chunks(const ln_problem* p) { return (p->gh * p->gw + kDwcTokensPerChunk - 1) / kDwcTokensPerChunk; }
+template <typename T>
+void launch_rope(const char* name, const ln_problem* p, const ln_block* b, const void* X, void* out, double sign, cudaStream_t st) {
+  const long long rows = (long long)p->B * p->H * p->n;
+  LN_LAUNCH(name, st, k_rope<T><<<cdiv(rows * (p->d / 4), 256), 256, 0, st>>>((const T*)X, (T*)out, rows, p->n, p->d, p->prefix,
+                                                                             log2((double)b->rope_base), sign));
+}
+template <typename T>
+void launch_dwc_add(const char* name, const ln_problem* p, const ln_block* b, const void* src, void* out, int flip, cudaStream_t st) {
+  LN_LAUNCH(name, st, k_dwc_add<T><<<dim3(cdiv((long long)p->gh * p->gw * (p->d / 4), 256), p->B * p->H), 256, 0, st>>>(
+                (const T*)src, b->dwc_w, (T*)out, p->H, p->n, p->d, p->prefix, p->gh, p->gw, b->dwc_ks, flip));
+}
+}  // namespace
+extern "C" {
+
+size_t laplace_attention_block_saved_bytes(const ln_problem* p, const ln_block* b) {
+  if (validate_block(p, b) != LN_OK) return 0;
+  return laplace_nystrom_saved_bytes(p) + (b->rope_base > 0.f ? 2 * tensor_bytes(p) : 0);
+}
+
+size_t laplace_attention_block_workspace_bytes(const ln_problem* p, const ln_block* b) {
+  if (validate_block(p, b) != LN_OK) return 0;
+  size_t ws = laplace_nystrom_workspace_bytes(p, 1);
+  if (b->rope_base > 0.f) ws += 2 * tensor_bytes(p);                           // gradients with respect to the rotated Q and K
+  if (b->dwc_w) ws += align_up((size_t)p->B * p->H * dwc_chunks(p) * p->d * b->dwc_ks * b->dwc_ks * sizeof(float), 256);
+  return ws;
+}
+
+int laplace_attention_block_fwd(const ln_problem* p, const ln_block* b, const void* Q, const void* K, const void* V, void* O,
+                                void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
+  int s = validate_block(p, b);
+  if (s != LN_OK) return s;
+  if (!Q || !K || !V || !O || !saved || !ws) return LN_ERR_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(saved) || !aligned16(ws)) return LN_ERR_ARG;
+  if (ws_bytes < laplace_attention_block_workspace_bytes(p, b)) return LN_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t tb = tensor_bytes(p);
+  char* sv = static_cast<char*>(saved);
+  const void *q = Q, *k = K;
+  void* inner_saved = sv;
+  if (b->rope_base > 0.f) {
+    s = check_fwd_args(p, sv, sv + tb, V, nullptr, O, sv + 2 * tb, ws, ws_bytes);
+    if (s != LN_OK) return s;
+    if (p->dtype == LN_F32) { launch_rope<float>("rope_Q", p, b, Q, sv, 1.f, st); launch_rope<float>("rope_K", p, b, K, sv + tb, 1.f, st); }
+    else { launch_rope<bf16>("rope_Q", p, b, Q, sv, 1.f, st); launch_rope<bf16>("rope_K", p, b, K, sv + tb, 1.f, st); }
+    q = sv; k = sv + tb; inner_saved = sv + 2 * tb;
+  }
+  s = fwd_entry(p, q, k, V, nullptr, O, inner_saved, ws, ws_bytes, dev_status, stream, true);
+  if (s != LN_OK) return s;
+  if (b->dwc_w) {
+    if (p->dtype == LN_F32) launch_dwc_add<float>("dwc_O", p, b, V, O, 0, st); else launch_dwc_add<bf16>("dwc_O", p, b, V, O, 0, st);
+  }
+  return launch_ok();
+}
+
+int laplace_attention_block_bwd(const ln_problem* p, const ln_block* b, const void* Q, const void* K, const void* V,
+                                const void* dO, const void* saved, void* dQ, void* dK, void* dV, float* dWd, void* ws,
+                                size_t ws_bytes, int32_t* dev_status, void* stream) {
+  int s = validate_block(p, b);
+  if (s != LN_OK) return s;
+  if (!Q || !K || !V || !dO || !saved || !dQ || !dK || !dV || !ws) return LN_ERR_ARG;
+  if ((b->dwc_w != nullptr) != (dWd != nullptr)) return LN_ERR_ARG;
+  if (!aligned16(saved) || !aligned16(ws) || !aligned16(dWd)) return LN_ERR_ARG;
+  if (ws_bytes < laplace_attention_block_workspace_bytes(p, b)) return LN_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t tb = tensor_bytes(p), base_ws = align_up(laplace_nystrom_workspace_bytes(p, 1), 256);
+  const char* sv = static_cast<const char*>(saved);
+  char* w = static_cast<char*>(ws);
+  const bool rope = b->rope_base > 0.f;
+  const void *q = rope ? (const void*)sv : Q, *k = rope ? (const void*)(sv + tb) : K;
+  void *dq = rope ? (void*)(w + base_ws) : dQ, *dk = rope ? (void*)(w + base_ws + tb) : dK;
+  float* wpart = reinterpret_cast<float*>(w + base_ws + (rope ? 2 * tb : 0));
+  s = bwd_entry(p, q, k, V, nullptr, dO, rope ? sv + 2 * tb : sv, dq, dk, dV, nullptr, ws, base_ws, dev_status, stream, true);
+  if (s != LN_OK) return s;
+  if (rope) {
+    if (p->dtype == LN_F32) { launch_rope<float>("rope_dQ", p, b, dq, dQ, -1.f, st); launch_rope<float>("rope_dK", p, b, dk, dK, -1.f, st); }
+    else { launch_rope<bf16>("rope_dQ", p, b, dq, dQ, -1.f, st); launch_rope<bf16>("rope_dK", p, b, dk, dK, -1.f, st); }
+  }
+  if (b->dwc_w) {
+    const int ch = dwc_chunks(p), BH = p->B * p->H, cnt = p->d * b->dwc_ks * b->dwc_ks;
+    if (p->dtype == LN_F32) {
+      launch_dwc_add<float>("dwc_dV", p, b, dO, dV, 1, st);
+      LN_LAUNCH("dwc_wgrad", st, k_dwc_wgrad<float><<<dim3(ch, BH), 128, 0, st>>>((const float*)V, (const float*)dO, wpart, p->n, p->d, p->prefix,
+                                                                                 p->gh, p->gw, b->dwc_ks, kDwcTokensPerChunk));
+    } else {
+      launch_dwc_add<bf16>("dwc_dV", p, b, dO, dV, 1, st);
+      LN_LAUNCH("dwc_wgrad", st, k_dwc_wgrad<bf16><<<dim3(ch, BH), 128, 0, st>>>((const bf16*)V, (const bf16*)dO, wpart, p->n, p->d, p->prefix,
+                                                                                p->gh, p->gw, b->dwc_ks, kDwcTokensPerChunk));
+    }
+    LN_LAUNCH("dwc_wreduce", st, k_dwc_wreduce<<<dim3(cdiv(cnt, 256), p->H), 256, 0, st>>>(wpart, dWd, p->B, p->H, ch, cnt));
+  }
+  return launch_ok();
+}
 
 }  // extern "C"

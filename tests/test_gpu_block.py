@@ -1,0 +1,85 @@
+"""GPU parity of the attention block around the path (rotary embedding on Q and K, Sec. 5.1; Attention = Z V + DWC(V),
+Eq. 7) against the float64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2604_20368_b200 as ln
+from paper_2604_20368_b200 import synth
+from parity import TOL, f64, metrics, oracle_problem
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _case(cfg, rope_base, ks, seed=0):
+    inp = synth.make_inputs(cfg)
+    rng = np.random.default_rng(seed)
+    Wd = None if ks == 0 else torch.from_numpy((rng.standard_normal((cfg.H, cfg.d, ks, ks)) / ks).astype(np.float32))
+    p = ln.problem_from_config(cfg, whiten=inp["whiten"].to(DEV))
+    blk = ln.Block(dwc_w=None if Wd is None else Wd.to(DEV), rope_base=rope_base)
+    Q, K, V, dO = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
+    status = torch.full((cfg.B * cfg.H,), -1, dtype=torch.int32, device=DEV)
+    O, saved, ws = ln.laplace_attention_block_fwd(p, blk, Q, K, V, dev_status=status)
+    dQ, dK, dV, dWd = ln.laplace_attention_block_bwd(p, blk, Q, K, V, dO, saved, ws)
+    torch.cuda.synchronize()
+    assert int(status.abs().max()) == 0
+    op = oracle_problem(cfg)
+    bf = cfg.dtype == "bf16"
+    args = dict(Wd=None if Wd is None else f64(Wd), rope_base=rope_base, whiten=f64(inp["whiten"]), store_bf16=bf)
+    Oo = oracle.block_forward(op, f64(inp["Q"]), f64(inp["K"]), f64(inp["V"]), **args)
+    dQo, dKo, dVo, dWo = oracle.block_backward(op, f64(inp["Q"]), f64(inp["K"]), f64(inp["V"]), f64(inp["dO"]), **args)
+    BH = cfg.B * cfg.H
+    errs = {}
+    for name, got, ref in (("O", O, Oo), ("dQ", dQ, dQo), ("dK", dK, dKo), ("dV", dV, dVo)):
+        errs[name] = metrics(f64(got).reshape(BH, cfg.n, cfg.d), ref.reshape(BH, cfg.n, cfg.d), bf)
+    print(cfg.name, rope_base, ks, {k: {a: f"{b:.1e}" for a, b in e.items()} for k, e in errs.items()})
+    for name, e in errs.items():
+        assert e["fro"] < TOL[cfg.dtype] and e["maxabs"] < TOL[cfg.dtype], (name, e)
+        assert e["row"] < 2 * TOL[cfg.dtype], (name, e)
+        if bf:      # O and dV are rounded twice on this path (once by the attention kernels, once after the convolution is added)
+            assert e["internal"] < 3e-3, (name, e)
+    if Wd is not None:
+        ew = float(np.linalg.norm(f64(dWd) - dWo) / np.linalg.norm(dWo))
+        print("dWd", ew)
+        assert ew < (1e-4 if not bf else 5e-3)
+    else:
+        assert dWd is None
+
+
+@pytest.mark.parametrize("rope_base,ks", [(10000.0, 3), (0.0, 3), (10000.0, 0), (100.0, 5)])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_block_cfg2_shape(rope_base, ks, dtype):
+    from dataclasses import replace
+    cfg = replace(synth.shrink(synth.CONFIGS["cfg2"], B=2, H=2), dtype=dtype)
+    _case(cfg, rope_base, ks)
+
+
+def test_block_large_grid_bf16():
+    # 56 x 56 tokens: positions up to 3135, where the rotation angle has to be formed in double
+    _case(synth.shrink(synth.CONFIGS["cfg4a"], B=1, H=2), 10000.0, 3)
+
+
+def test_block_without_extras_is_the_path():
+    cfg = synth.shrink(synth.CONFIGS["cfg2"], B=1)
+    inp = synth.make_inputs(cfg)
+    p = ln.problem_from_config(cfg, whiten=inp["whiten"].to(DEV))
+    Q, K, V, dO = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
+    O, saved, ws = ln.laplace_attention_block_fwd(p, ln.Block(), Q, K, V)
+    dQ, dK, dV, dWd = ln.laplace_attention_block_bwd(p, ln.Block(), Q, K, V, dO, saved, ws)
+    sv = torch.empty(ln.laplace_nystrom_saved_bytes(p), dtype=torch.uint8, device=DEV)
+    O2 = ln.laplace_nystrom_fwd(p, Q, K, V, saved=sv)
+    g2 = ln.laplace_nystrom_bwd(p, Q, K, V, dO, sv)
+    assert torch.equal(O, O2) and torch.equal(dQ, g2[0]) and torch.equal(dK, g2[1]) and torch.equal(dV, g2[2]) and dWd is None
+
+
+def test_block_argument_errors():
+    cfg = synth.shrink(synth.CONFIGS["cfg2"], B=1)
+    inp = synth.make_inputs(cfg)
+    p = ln.problem_from_config(cfg)
+    Q, K, V = (inp[k].to(DEV) for k in ("Q", "K", "V"))
+    bad = ln.Block(dwc_w=torch.zeros(cfg.H, cfg.d, 4, 4, device=DEV))      # even filter size
+    with pytest.raises(ln.LnError):
+        ln.laplace_attention_block_fwd(p, bad, Q, K, V, saved=torch.empty(1 << 20, dtype=torch.uint8, device=DEV),
+                                       ws=torch.empty(1 << 20, dtype=torch.uint8, device=DEV))
