@@ -46,6 +46,8 @@ def parse():
     ap.add_argument("--config", default="cfg5_m256_T12", choices=sorted(synth.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle legs (CPU baseline, sampled-head parity)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the sweep over all configurations")
+    ap.add_argument("--fig5", action="store_true", help="the kernel micro-benchmark of the paper's Fig. 5 setting instead of a step")
+    ap.add_argument("--fig5-T", type=int, default=8, help="Newton-Schulz steps of the micro-benchmark")
     ap.add_argument("--B", type=int, default=0, help="override the batch size (profiling of a smaller case)")
     return ap.parse_args()
 
@@ -571,8 +573,70 @@ def run_ours(args):
     print(json.dumps(out))
 
 
+# ------------------------------------------------------------------------------------------ kernel micro-benchmark
+def run_fig5(args):
+    """The paper's kernel micro-benchmark (Sec. 4.3, Fig. 5 setting: batch 1, 2 heads, 32 channels, a sweep over matrix
+    sizes): forward and backward time of the two stand-alone entry points, l1_kernel (N x N kernel matrix of N points) and
+    ns_pinv (m x m matrix, T steps), CUDA events, median of 20 launches after 3 warm-ups, with the float64 oracle timed on
+    the host cores beside each size it finishes quickly.  Prints one JSON line."""
+    import paper_2604_20368_b200 as ln
+    import oracle
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(0)
+    heads, d, T = 2, 32, args.fig5_T
+
+    def med_us(fn, reps=20):
+        for _ in range(3):
+            fn()
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return float(np.median(ts))
+
+    def cpu_ms(fn):
+        t0 = time.perf_counter(); fn(); return (time.perf_counter() - t0) * 1e3
+
+    rng = np.random.default_rng(0)
+    l1_rows, ns_rows = [], []
+    for N in (64, 128, 256, 512, 1024, 2048, 4096):
+        A = torch.from_numpy(rng.standard_normal((heads, N, d), dtype=np.float32))
+        Bm = torch.from_numpy(rng.standard_normal((heads, N, d), dtype=np.float32))
+        dK = torch.from_numpy(rng.standard_normal((heads, N, N), dtype=np.float32))
+        Ad, Bd, dKd = A.to(dev), Bm.to(dev), dK.to(dev)
+        Kmat = ln.l1_kernel(Ad, Bd, float(d))
+        row = {"size": N, "fwd_us": med_us(lambda: ln.l1_kernel(Ad, Bd, float(d))),
+               "bwd_us": med_us(lambda: ln.l1_kernel_bwd(Ad, Bd, float(d), dKd, Kmat=Kmat))}
+        if N <= 1024 and not args.no_cpu_baseline:
+            a64, b64, g64 = A.double().numpy(), Bm.double().numpy(), dK.double().numpy()
+            row["oracle_fwd_ms"] = cpu_ms(lambda: oracle.l1_kernel(a64, b64, float(d)))
+            row["oracle_bwd_ms"] = cpu_ms(lambda: oracle.l1_kernel_bwd(a64, b64, float(d), g64))
+        l1_rows.append(row)
+    for m in (32, 64, 128, 256):
+        pts = rng.standard_normal((heads, m, d))
+        W = np.exp(-np.abs(pts[:, :, None, :] - pts[:, None, :, :]).sum(-1) / d).astype(np.float32)   # inputs only: a kernel matrix to invert
+        Wd = torch.from_numpy(W).to(dev)
+        dX = torch.from_numpy(rng.standard_normal((heads, m, m), dtype=np.float32)).to(dev)
+        hist = ln.ns_pinv(Wd, T, ridge_eps=1e-6, want_hist=True)[1]
+        row = {"size": m, "iters": T, "fwd_us": med_us(lambda: ln.ns_pinv(Wd, T, ridge_eps=1e-6)),
+               "bwd_us": med_us(lambda: ln.ns_pinv_bwd(Wd, T, 1e-6, 0.0, dX, X_hist=hist))}
+        if not args.no_cpu_baseline:
+            row["oracle_fwd_ms"] = cpu_ms(lambda: oracle.ns_pinv(W, T, eps=1e-6))
+            row["oracle_bwd_ms"] = cpu_ms(lambda: oracle.ns_pinv_bwd(W, T, 1e-6, 0.0, dX.cpu().numpy()))
+        ns_rows.append(row)
+    print(json.dumps({"workload": "kernel micro-benchmark: batch 1, 2 heads, 32 channels, matrix-size sweep (Fig. 5 setting)",
+                      "unit": "us per call (device, CUDA events, median of 20); oracle: ms per call on the host cores",
+                      "oracle_cores": oracle.num_threads(), "l1_kernel": l1_rows, "ns_pinv": ns_rows,
+                      "note": "ns_pinv / ns_pinv_bwd are the stand-alone fp32 (FFMA) entry points held to 2e-5 / 1e-4 against the oracle; "
+                              "inside the attention path the same iteration runs on tcgen05 with split-bf16 operands"}))
+
+
 def main():
     args = parse()
+    if args.fig5:
+        run_fig5(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

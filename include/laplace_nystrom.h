@@ -213,6 +213,17 @@ int l1_kernel_bwd(int32_t batch, int32_t na, int32_t nb, int32_t d, const void* 
                   void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Exact Laplacian-kernel attention, forward only (Eq. 4 and Eq. 7 with the full n x n kernel matrix G = k(Q, K), which is
+ * formed tile by tile on chip and never stored): the O(n^2) reference the Nystrom path approximates; at m = n with
+ * converged Newton-Schulz the path reproduces it.  For accuracy-against-m curves, not for training.
+ *   map_mode 1: O_i = sum_j (G_ij - mu_i) V_j + (1/n) sum_j V_j, mu_i = mean_j G_ij (the injective map with unit whitening);
+ *   map_mode 0: O = G V.
+ * Q, K, V, O: [batch, n, d] of `dtype`, d in {32, 64, 128}; batch = B * heads.
+ */
+int laplace_exact_fwd(int32_t batch, int32_t n, int32_t d, int32_t dtype, float lambda, int32_t map_mode, const void* Q,
+                      const void* K, const void* V, void* O, void* stream);
+
+/*
  * Whitening statistics (Eq. 5 and Eq. 6): the diagonal scale s [H, m] that `whiten` takes, estimated from the
  * query-landmark kernel block C = k(Q, L) that laplace_nystrom_fwd left in `saved`.  For head h and landmark l the
  * batch of Eq. 5 is every query row of every batch element:

@@ -284,3 +284,17 @@ def block_backward(p: Problem, Q, K, V, dO, Wd=None, rope_base=0.0, whiten=None,
     if rope_base > 0:
         dQr, dKr = rope(dQr, p.prefix, rope_base, inverse=True), rope(dKr, p.prefix, rope_base, inverse=True)
     return dQr, dKr, dV, dWd
+
+
+def exact_attention(Q, K, V, lam, map_mode=1):
+    """Exact Laplacian-kernel attention (Eq. 4 + Eq. 7, no Nystrom approximation, unit whitening), the plain
+    definition: G = k(Q, K) [n x n], Z = G - rowmean(G) + 1/n, O = Z V (map_mode 0: O = G V).  [B,H,n,d] arrays."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    B, H, n, d = Q.shape
+    O = np.empty_like(Q)
+    for b in range(B):
+        for h in range(H):
+            G = l1_kernel(Q[b, h][None], K[b, h][None], lam)[0]
+            Z = G if map_mode == 0 else G - G.mean(axis=1, keepdims=True) + 1.0 / n
+            O[b, h] = Z @ V[b, h]
+    return O

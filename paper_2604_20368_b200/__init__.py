@@ -9,7 +9,7 @@ from .binding import (  # noqa: F401
     LN_BF16, LN_F32, LnError, Problem, l1_kernel, l1_kernel_bwd, landmarks_pool, landmarks_pool_bwd,
     laplace_nystrom_bwd, laplace_nystrom_fwd, laplace_nystrom_saved_bytes, laplace_nystrom_workspace_bytes,
     ns_pinv, ns_pinv_bwd, ns_pinv_static, trace_begin, trace_end, HostStep, laplace_nystrom_fwd_bwd_host,
-    set_overlap, set_fused_sign, Block, laplace_attention_block_fwd, laplace_attention_block_bwd, launch_count, laplace_nystrom_whiten_stats, saved_array, selftest_wait_timeout, fp32_add_probe,
+    set_overlap, set_fused_sign, laplace_exact_fwd, Block, laplace_attention_block_fwd, laplace_attention_block_bwd, launch_count, laplace_nystrom_whiten_stats, saved_array, selftest_wait_timeout, fp32_add_probe,
 )
 
 

@@ -28,7 +28,7 @@ EXPORTS = [
     "laplace_nystrom_host_staging_bytes", "laplace_nystrom_fwd_bwd_host", "ln_set_overlap", "ln_launch_count",
     "laplace_nystrom_whiten_stats_workspace_bytes", "laplace_nystrom_whiten_stats",
     "laplace_nystrom_saved_array", "ln_set_fused_sign", "laplace_attention_block_saved_bytes",
-    "laplace_attention_block_workspace_bytes", "laplace_attention_block_fwd", "laplace_attention_block_bwd", "ln_selftest_wait_timeout", "ln_fp32_add_probe", "ln_fp32_add_probe_lane_ops",
+    "laplace_attention_block_workspace_bytes", "laplace_attention_block_fwd", "laplace_attention_block_bwd", "laplace_exact_fwd", "ln_selftest_wait_timeout", "ln_fp32_add_probe", "ln_fp32_add_probe_lane_ops",
 ]
 
 
@@ -144,6 +144,7 @@ def lib():
         L.ln_fp32_add_probe.argtypes = [i32, i32, i32, vp, vp]
         L.ln_fp32_add_probe_lane_ops.restype = ctypes.c_int64
         L.ln_fp32_add_probe_lane_ops.argtypes = [i32, i32]
+        L.laplace_exact_fwd.argtypes = [i32, i32, i32, i32, f32, i32, vp, vp, vp, vp, vp]
         pb = ctypes.POINTER(_CBlock)
         L.laplace_attention_block_saved_bytes.restype = sz
         L.laplace_attention_block_saved_bytes.argtypes = [pp, pb]
@@ -381,6 +382,15 @@ def laplace_attention_block_bwd(p: Problem, blk: Block, Q, K, V, dO, saved, ws, 
                                              _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dWd), _ptr(ws), ws.numel(), _ptr(dev_status),
                                              _stream(stream)), "laplace_attention_block_bwd")
     return dQ, dK, dV, dWd
+
+
+def laplace_exact_fwd(Q, K, V, lam: float, map_mode: int = 1, stream=None):
+    """Exact (m = n) Laplacian-kernel attention of Q, K, V [B, H, n, d] (Eq. 4 + Eq. 7, full kernel matrix on chip)."""
+    B, H, n, d = Q.shape
+    O = torch.empty_like(Q)
+    _check(lib().laplace_exact_fwd(B * H, n, d, _dtype_code(Q), lam, map_mode, _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _stream(stream)),
+           "laplace_exact_fwd")
+    return O
 
 
 def set_fused_sign(enabled: bool) -> bool:

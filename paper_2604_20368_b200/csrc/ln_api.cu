@@ -9,6 +9,7 @@
 #include "ln_sign2.cuh"
 #include "ln_sign3.cuh"
 #include "ln_block.cuh"
+#include "ln_exact.cuh"
 #include <atomic>
 #include <mutex>
 #include <unordered_map>
@@ -48,6 +49,7 @@ void want_smem(K kern, size_t smem) {
   have[dev][id] = (int)smem;
 }
 
+template <typename A0, typename... R> A0 arg0(void (*)(A0, R...));   // first parameter type of a kernel (declaration only)
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -1223,6 +1225,25 @@ int laplace_attention_block_bwd(const ln_problem* p, const ln_block* b, const vo
     }
     LN_LAUNCH("dwc_wreduce", st, k_dwc_wreduce<<<dim3(cdiv(cnt, 256), p->H), 256, 0, st>>>(wpart, dWd, p->B, p->H, ch, cnt));
   }
+  return launch_ok();
+}
+
+int laplace_exact_fwd(int32_t batch, int32_t n, int32_t d, int32_t dtype, float lambda, int32_t map_mode, const void* Q,
+                      const void* K, const void* V, void* O, void* stream) {
+  if (batch <= 0 || n <= 0 || !Q || !K || !V || !O) return LN_ERR_ARG;
+  if (!(lambda > 0.f) || !isfinite(lambda) || (map_mode != 0 && map_mode != 1)) return LN_ERR_ARG;
+  if (dtype != LN_F32 && dtype != LN_BF16) return LN_ERR_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return LN_ERR_ARG;
+  if ((d != 32 && d != 64 && d != 128) || batch > 65535) return LN_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const float nscale = -1.4426950408889634f / lambda;
+  auto go = [&](auto kern, size_t smem) {
+    want_smem(kern, smem);
+    using TT = std::remove_const_t<std::remove_pointer_t<decltype(arg0(kern))>>;
+    LN_LAUNCH("k_exact_fwd", st, kern<<<dim3(cdiv(n, 64), batch), 256, smem, st>>>((const TT*)Q, (const TT*)K, (const TT*)V, (TT*)O, n, nscale, map_mode));
+  };
+  if (dtype == LN_F32) { if (d == 32) go(k_exact_fwd<float, 32>, exact_smem_bytes<32>()); else if (d == 64) go(k_exact_fwd<float, 64>, exact_smem_bytes<64>()); else go(k_exact_fwd<float, 128>, exact_smem_bytes<128>()); }
+  else { if (d == 32) go(k_exact_fwd<bf16, 32>, exact_smem_bytes<32>()); else if (d == 64) go(k_exact_fwd<bf16, 64>, exact_smem_bytes<64>()); else go(k_exact_fwd<bf16, 128>, exact_smem_bytes<128>()); }
   return launch_ok();
 }
 

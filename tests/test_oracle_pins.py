@@ -479,3 +479,18 @@ def test_lm_f32_moves_results_only_at_rounding_level_away_from_ties():
     d1 = oracle.backward(p1, Qt, K, V, dO, whiten=s)[0]
     diff = np.abs(d0 - d1)
     assert diff[0, 0, 5, c] > 1e3 * np.delete(diff[0, 0, 5], c).max()   # the sign of that one term flipped, nothing else moved
+
+
+def test_exact_attention_definition_against_brute_force_and_m_equals_n():
+    # oracle.exact_attention (the O(n^2) definition) against the broadcasting brute force of this file, and against the
+    # Nystrom chain at m = n with converged Newton-Schulz
+    rng = np.random.default_rng(61)
+    n, d = 12, 3
+    Q, K, V = (rng.standard_normal((1, 2, n, d)) for _ in range(3))
+    for map_mode in (0, 1):
+        O = oracle.exact_attention(Q, K, V, float(d), map_mode)
+        for h in range(2):
+            np.testing.assert_allclose(O[0, h], exact_attention(Q[0, h], K[0, h], V[0, h], float(d), None, map_mode), rtol=1e-13)
+        p = Problem(B=1, H=2, n=n, d=d, m=n, lam=float(d), ns_iters=40, ridge_eps=0.0, map_mode=map_mode, lm_mode=1,
+                    gh=3, gw=4, mh=3, mw=4)
+        np.testing.assert_allclose(oracle.forward(p, Q, K, V), O, rtol=1e-8, atol=1e-10)
