@@ -176,7 +176,7 @@ def backward(p: Problem, Q, K, V, dO, L=None, whiten=None):
     """Returns dQ, dK, dV, dL (dL is None when the landmarks are pooled from K)."""
     Q, K, V, L, whiten, dO = _f64(Q), _f64(K), _f64(V), _f64(L), _f64(whiten), _f64(dO)
     dQ, dK, dV = np.empty_like(Q), np.empty_like(Q), np.empty_like(Q)
-    dL = np.empty((p.B, p.H, p.m, p.d)) if p.lm_mode == 0 else None
+    dL = np.empty((p.B, p.H, p.m, p.d)) if p.lm_mode == 0 else None      # pooled landmarks (modes 1, 2): folded into dK / dQ
     cp = p.c()
     _load().oracle_bwd(ctypes.byref(cp), _p(Q), _p(K), _p(V), _p(L), _p(whiten), _p(dO),
                        _p(dQ), _p(dK), _p(dV), _p(dL))

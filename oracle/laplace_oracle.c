@@ -66,7 +66,7 @@ typedef struct oracle_problem {
   double ridge_eps;
   double ns_alpha;  /* <= 0: alpha = 1/(||W||_1 ||W||_inf); > 0: used as given, no gradient through it */
   int32_t map_mode; /* 0: O = C X R V;  1: injective map of Prop. 3 applied to the rows of C */
-  int32_t lm_mode;  /* 0: landmarks given;  1: landmarks = adaptive average pooling of K */
+  int32_t lm_mode;  /* 0: landmarks given;  1: landmarks = adaptive average pooling of K;  2: of Q (Sec. 4.2 pools the query tensor in one place) */
   int32_t prefix, gh, gw, mh, mw; /* lm_mode 1: n = prefix + gh*gw, m = mh*mw */
   int32_t lm_f32;   /* 1: pooled landmarks are rounded to single precision before use (see fwd_single) */
 } oracle_problem;
@@ -389,8 +389,8 @@ static void ctx_free(head_ctx* x) {
 static void fwd_single(const oracle_problem* p, const double* Q, const double* K, const double* V,
                        const double* Lin, const double* s, head_ctx* x, double* O) {
   int n = p->n, d = p->d, m = p->m;
-  if (p->lm_mode == 1) {                                            /* landmarks */
-    pool_single(p, K, x->L);
+  if (p->lm_mode == 1 || p->lm_mode == 2) {                         /* landmarks: pooled keys (default) or pooled queries */
+    pool_single(p, p->lm_mode == 1 ? K : Q, x->L);
     /* The gradient of the kernel holds sign(token - landmark), which is discontinuous: a pooled
        landmark that lies within rounding distance of a token decides that sign differently in
        different precisions.  With lm_f32 the landmark is DEFINED as the single-precision value
@@ -494,6 +494,7 @@ static void bwd_single(const oracle_problem* p, const double* Q, const double* K
   l1_block_bwd(m, n, d, x.L, K, p->lambda, x.R, dR, dLt, dK);     /* R = k(L, K) */
   l1_block_bwd(m, m, d, x.L, x.L, p->lambda, x.W, dW, dLt, dLt);  /* W = k(L, L) */
   if (p->lm_mode == 1) pool_single_bwd(p, dLt, dK);
+  else if (p->lm_mode == 2) pool_single_bwd(p, dLt, dQ);
   else memcpy(dL, dLt, sizeof(double) * md);
 
   free(O); free(dZ); free(dC); free(dY); free(dX); free(dM); free(dR); free(dW); free(dLt);

@@ -494,3 +494,29 @@ def test_exact_attention_definition_against_brute_force_and_m_equals_n():
         p = Problem(B=1, H=2, n=n, d=d, m=n, lam=float(d), ns_iters=40, ridge_eps=0.0, map_mode=map_mode, lm_mode=1,
                     gh=3, gw=4, mh=3, mw=4)
         np.testing.assert_allclose(oracle.forward(p, Q, K, V), O, rtol=1e-8, atol=1e-10)
+
+
+def test_landmarks_pooled_from_queries_variant():
+    # lm_mode 2 (Sec. 4.2 "Landmark Selection" pools the query tensor): the same chain with L = pool(Q); pinned against
+    # the given-landmark path fed with pool(Q), the landmark gradient returning to Q through the pooling adjoint, and
+    # against central differences
+    from dataclasses import replace
+    rng = np.random.default_rng(71)
+    p2 = Problem(B=1, H=2, n=2 + 5 * 6, d=4, m=6, lam=4.0, ns_iters=3, ridge_eps=1e-6, map_mode=1, lm_mode=2,
+                 prefix=2, gh=5, gw=6, mh=2, mw=3)
+    Q, K, V, dO = (rng.standard_normal((1, 2, p2.n, p2.d)) for _ in range(4))
+    s = rng.uniform(0.5, 2.0, (2, p2.m))
+    Lq = oracle.landmarks_pool(replace(p2, lm_mode=1), Q)
+    pg = replace(p2, lm_mode=0)
+    np.testing.assert_array_equal(oracle.forward(p2, Q, K, V, whiten=s), oracle.forward(pg, Q, K, V, L=Lq, whiten=s))
+    dQ, dK, dV, dL = oracle.backward(p2, Q, K, V, dO, whiten=s)
+    dQg, dKg, dVg, dLg = oracle.backward(pg, Q, K, V, dO, L=Lq, whiten=s)
+    assert dL is None
+    np.testing.assert_array_equal(dK, dKg)
+    np.testing.assert_array_equal(dV, dVg)
+    np.testing.assert_allclose(dQ, dQg + oracle.landmarks_pool_bwd(replace(p2, lm_mode=1), dLg), rtol=1e-13, atol=1e-15)
+    loss = lambda q: float((oracle.forward(p2, q, K, V, whiten=s) * dO).sum())
+    h = 1e-6
+    for idx in [(0, 0, 0, 0), (0, 1, 9, 2), (0, 0, 31, 3)]:
+        qp, qm = Q.copy(), Q.copy(); qp[idx] += h; qm[idx] -= h
+        assert dQ[idx] == pytest.approx((loss(qp) - loss(qm)) / (2 * h), rel=5e-6, abs=1e-8)
