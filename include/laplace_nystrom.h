@@ -59,8 +59,9 @@ typedef struct ln_problem {
   int32_t dtype;          /* ln_dtype of the [.,.,.,d] tensors                                            */
   int32_t map_mode;       /* 0: O = C X R V;  1: injective map of Prop. 3 applied to the rows of C        */
   const float* whiten;    /* device [H,m] fp32 whitening scale s (Eq. 6), or NULL = ones; a constant      */
-  int32_t lm_mode;        /* 0: landmarks L given by the caller;  1: L = adaptive average pooling of K    */
-  int32_t prefix, gh, gw, mh, mw; /* lm_mode 1: n = prefix + gh*gw, m = mh*mw.  Bin (a,b) averages grid  */
+  int32_t lm_mode;        /* 0: landmarks L given by the caller;  1: L = adaptive average pooling of K;   */
+                          /* 2: of Q (Sec. 4.2 pools the query tensor in one place): dL then returns to dQ */
+  int32_t prefix, gh, gw, mh, mw; /* lm_mode 1, 2: n = prefix + gh*gw, m = mh*mw.  Bin (a,b) averages grid  */
                           /* rows floor(a*gh/mh) .. ceil((a+1)*gh/mh)-1 and columns likewise; the first   */
                           /* `prefix` tokens (class tokens) are ordinary queries/keys but are not pooled. */
 } ln_problem;
@@ -99,8 +100,8 @@ int laplace_nystrom_fwd(const ln_problem* p, const void* Q, const void* K, const
  * gradient -(1/lambda) sign(x - y) k, with sign(0) = 0).
  *   dO [B,H,n,d] dtype;  saved: the buffer the matching fwd filled;
  *   dQ,dK,dV [B,H,n,d] dtype, overwritten;
- *   dL [B,H,m,d] dtype: required when lm_mode == 0; must be NULL when lm_mode == 1 (the
- *   landmark gradient is folded into dK through the pooling adjoint).
+ *   dL [B,H,m,d] dtype: required when lm_mode == 0; must be NULL when lm_mode is 1 or 2 (the
+ *   landmark gradient is folded into dK, or dQ, through the pooling adjoint).
  *   ws: laplace_nystrom_workspace_bytes(p, 1) bytes.
  *   dev_status: as for laplace_nystrom_fwd (only bit 1 can be set by the backward pass).
  */

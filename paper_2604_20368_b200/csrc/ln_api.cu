@@ -224,9 +224,9 @@ int validate(const ln_problem* p) {
   if (!isfinite(p->ns_alpha)) return LN_ERR_ARG;
   if (p->dtype != LN_F32 && p->dtype != LN_BF16) return LN_ERR_ARG;
   if (p->map_mode != 0 && p->map_mode != 1) return LN_ERR_ARG;
-  if (p->lm_mode != 0 && p->lm_mode != 1) return LN_ERR_ARG;
+  if (p->lm_mode < 0 || p->lm_mode > 2) return LN_ERR_ARG;
   if (p->whiten && !aligned16(p->whiten)) return LN_ERR_ARG;
-  if (p->lm_mode == 1) {
+  if (p->lm_mode >= 1) {
     if (p->prefix < 0 || p->gh <= 0 || p->gw <= 0 || p->mh <= 0 || p->mw <= 0) return LN_ERR_ARG;
     if ((long long)p->prefix + (long long)p->gh * p->gw != p->n) return LN_ERR_ARG;
     if ((long long)p->mh * p->mw != p->m) return LN_ERR_ARG;
@@ -409,8 +409,8 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const int BH = pl.BH, n = pl.n, m = pl.m, kSMs = sm_count();
   if (dev_status && clear_status) cudaMemsetAsync(dev_status, 0, sizeof(int32_t) * BH, st);   // the kernels OR their flags into it
   // landmarks (Sec. 4.2)
-  if (p->lm_mode == 1) {
-    LN_LAUNCH("k_pool", st, k_pool<T><<<dim3(cdiv(m, 256 / (D / 4)), BH), 256, 0, st>>>(K, x.Lf, geom_of(p)));
+  if (p->lm_mode >= 1) {      // pooled keys, or pooled queries (lm_mode 2)
+    LN_LAUNCH("k_pool", st, k_pool<T><<<dim3(cdiv(m, 256 / (D / 4)), BH), 256, 0, st>>>(p->lm_mode == 1 ? K : Q, x.Lf, geom_of(p)));
   } else {
     const long long cnt = (long long)BH * m * D;
     LN_LAUNCH("k_to_f32", st, k_to_f32<T><<<cdiv(cnt, 256), 256, 0, st>>>(L, x.Lf, cnt));
@@ -529,6 +529,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     }
   };
   const bool fused_sign = pl.s2_chunks > 0;
+  const bool poolQ = p->lm_mode == 2;                 // the token-side gradient that still needs the pooling adjoint is dQ, not dK
   const bool sign3 = pl.s3_tiles > 0;                 // the sign passes form their upstream factor themselves (tcgen05)
   const int chs = sign3 ? pl.s3_tiles : (fused_sign ? pl.s2_chunks : ch);
   const int chq = sign3 ? pl.s3_tiles : (fused_sign ? pl.s2q_chunks : ch);    // chunks of the query-side landmark-gradient partials
@@ -617,7 +618,8 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   if (sign3) {
     const long long cnt = (long long)BH * m * D;
     LN_LAUNCH("k_fold_landmarks", st, k_fold_landmarks<<<cdiv(cnt, 256), 256, 0, st>>>(x.Lf, w.SB, D, cnt));
-    launch_sign3("sign3_dQ_dLC", Q, dO, x.Yimg, x.C, dQ, w.dLCpart);
+    if (poolQ) launch_sign3("sign3_dQ_dLC", Q, dO, x.Yimg, x.C, w.dKpart, w.dLCpart);
+    else launch_sign3("sign3_dQ_dLC", Q, dO, x.Yimg, x.C, dQ, w.dLCpart);
   } else launch_ntg_C();
   if (sign3) {
   } else if (fused_sign) {
@@ -625,34 +627,47 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
       want_smem(kern, pl.s2_smem);
       LN_LAUNCH(name, st, kern<<<dim3(chq, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(tokp, x.Lf, w.G, pl.ldm, rowsp, partp, n, m, D, pl.s2q_rpc));
     };
-    if (pl.s2_tg == S2_TGMAX) launch2("sign2_dQ_dLC", k_sign2<T, T, 1>, Q, dQ, w.dLCpart);
-    else launch2("sign2_dQ_dLC", k_sign2<T, T, 2>, Q, dQ, w.dLCpart);
+    if (poolQ) {
+      if (pl.s2_tg == S2_TGMAX) launch2("sign2_dQ_dLC", k_sign2<T, float, 1>, Q, w.dKpart, w.dLCpart);
+      else launch2("sign2_dQ_dLC", k_sign2<T, float, 2>, Q, w.dKpart, w.dLCpart);
+    } else {
+      if (pl.s2_tg == S2_TGMAX) launch2("sign2_dQ_dLC", k_sign2<T, T, 1>, Q, dQ, w.dLCpart);
+      else launch2("sign2_dQ_dLC", k_sign2<T, T, 2>, Q, dQ, w.dLCpart);
+    }
   } else {
-    LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m));
+    if (poolQ) LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dKpart, n, m));
+    else LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m));
     LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
   }
   if (side.on()) { side.join_mark(st); if (!ntg_on_side && !sign3) launch_ntg_R(st); }
   else { launch_mid(st); launch_sign_W(st); if (!sign3) launch_ntg_R(st); launch_nn_dV(st); }
   // key side: dK (kernel part); landmark part
   if (sign3) {
-    launch_sign3("sign3_dK_dLR", K, V, w.dMimg, x.Rt, w.dKpart, w.dLRpart);
+    if (poolQ) launch_sign3("sign3_dK_dLR", K, V, w.dMimg, x.Rt, dK, w.dLRpart);
+    else launch_sign3("sign3_dK_dLR", K, V, w.dMimg, x.Rt, w.dKpart, w.dLRpart);
   } else if (fused_sign) {
     auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
       want_smem(kern, pl.s2_smem);
       LN_LAUNCH(name, st, kern<<<dim3(chs, D / 64, BH), dim3(16, pl.s2_tg), pl.s2_smem, st>>>(tokp, x.Lf, w.G2, pl.ldm, rowsp, partp, n, m, D, pl.s2_rpc));
     };
-    if (pl.s2_tg == S2_TGMAX) launch2("sign2_dK_dLR", k_sign2<T, float, 1>, K, w.dKpart, w.dLRpart);
-    else launch2("sign2_dK_dLR", k_sign2<T, float, 2>, K, w.dKpart, w.dLRpart);
+    if (poolQ) {
+      if (pl.s2_tg == S2_TGMAX) launch2("sign2_dK_dLR", k_sign2<T, T, 1>, K, dK, w.dLRpart);
+      else launch2("sign2_dK_dLR", k_sign2<T, T, 2>, K, dK, w.dLRpart);
+    } else {
+      if (pl.s2_tg == S2_TGMAX) launch2("sign2_dK_dLR", k_sign2<T, float, 1>, K, w.dKpart, w.dLRpart);
+      else launch2("sign2_dK_dLR", k_sign2<T, float, 2>, K, w.dKpart, w.dLRpart);
+    }
   } else {
-    LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G2, pl.ldm, w.dKpart, n, m));
+    if (poolQ) LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G2, pl.ldm, dK, n, m));
+    else LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G2, pl.ldm, w.dKpart, n, m));
     LN_LAUNCH("sign_cols_dLR", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(K, x.Lf, w.G2, pl.ldm, w.dLRpart, n, m, pl.rpc));
   }
   // landmark gradient and its way back to the keys
   if (side.on()) side.join(st);      // dV and the landmark-block part are complete
   const int md = m * D;
-  if (p->lm_mode == 1) {
+  if (p->lm_mode >= 1) {      // the landmark gradient returns to the pooled tensor (keys, or queries for lm_mode 2)
     LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, w.dLtot, md));
-    LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, w.dLtot, dK, geom_of(p), 1));
+    LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, w.dLtot, poolQ ? dQ : dK, geom_of(p), 1));
   } else {
     LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, dL, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, nullptr, dK, geom_of(p), 0));
@@ -904,7 +919,7 @@ int laplace_nystrom_fwd_bwd_host(const ln_problem* p, const void* hQ, const void
                                  void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
   int s = validate(p);
   if (s != LN_OK) return s;
-  if (p->lm_mode != 1) return LN_ERR_UNSUPPORTED;
+  if (p->lm_mode < 1) return LN_ERR_UNSUPPORTED;
   if (!hQ || !hK || !hV || !hdO || !hO || !hdQ || !hdK || !hdV || !staging || !saved || !ws) return LN_ERR_ARG;
   if (!aligned16(staging)) return LN_ERR_ARG;
   if (staging_bytes < laplace_nystrom_host_staging_bytes(p)) return LN_ERR_WORKSPACE;
@@ -1061,7 +1076,7 @@ int l1_kernel_bwd(int32_t batch, int32_t na, int32_t nb, int32_t d, const void* 
 int landmarks_pool(const ln_problem* p, const void* K, float* L, void* stream) {
   int s = validate(p);
   if (s != LN_OK) return s;
-  if (p->lm_mode != 1 || !K || !L || !aligned16(K) || !aligned16(L)) return LN_ERR_ARG;
+  if (p->lm_mode < 1 || !K || !L || !aligned16(K) || !aligned16(L)) return LN_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   dim3 grid(cdiv(p->m, 256 / (p->d / 4)), p->B * p->H);
   if (p->dtype == LN_F32) LN_LAUNCH("k_pool", st, k_pool<float><<<grid, 256, 0, st>>>((const float*)K, L, geom_of(p)));
@@ -1072,7 +1087,7 @@ int landmarks_pool(const ln_problem* p, const void* K, float* L, void* stream) {
 int landmarks_pool_bwd(const ln_problem* p, const float* dL, void* dK, void* stream) {
   int s = validate(p);
   if (s != LN_OK) return s;
-  if (p->lm_mode != 1 || !dL || !dK || !aligned16(dL) || !aligned16(dK)) return LN_ERR_ARG;
+  if (p->lm_mode < 1 || !dL || !dK || !aligned16(dL) || !aligned16(dK)) return LN_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   dim3 grid(cdiv((long long)p->n * (p->d / 4), 256 * POOL_EPT), p->B * p->H);
   if (p->dtype == LN_F32) LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<float><<<grid, 256, 0, st>>>(nullptr, dL, (float*)dK, geom_of(p), 1));
@@ -1126,7 +1141,7 @@ int validate_block(const ln_problem* p, const ln_block* b) {
   int s = validate(p);
   if (s != LN_OK) return s;
   if (!b) return LN_ERR_ARG;
-  if (p->lm_mode != 1) return LN_ERR_UNSUPPORTED;            // the token grid is needed
+  if (p->lm_mode < 1) return LN_ERR_UNSUPPORTED;             // the token grid is needed
   if (!(b->rope_base >= 0.f) || !isfinite(b->rope_base)) return LN_ERR_ARG;
   if (b->rope_base > 0.f && (b->rope_base <= 1.f || (p->d & 3))) return LN_ERR_ARG;
   if (b->dwc_w && (b->dwc_ks < 1 || b->dwc_ks > 7 || (b->dwc_ks & 1) == 0 || !aligned16(b->dwc_w))) return LN_ERR_ARG;
