@@ -298,3 +298,53 @@ def exact_attention(Q, K, V, lam, map_mode=1):
             Z = G if map_mode == 0 else G - G.mean(axis=1, keepdims=True) + 1.0 / n
             O[b, h] = Z @ V[b, h]
     return O
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Whitening with batch statistics (Eq. 5-6 in training mode): the diagonal scale s is estimated from the kernel block
+# C = k(Q, L) of the very batch it is applied to, and the gradient flows through the variance.
+def forward_batch_whiten(p: Problem, Q, K, V, eps_w, L=None):
+    """O and s [H, m]: s_l = 1 / sqrt(Var_{b,i}(C_il) + eps_w) over the query rows of every batch element of head h
+    (Eq. 5-6), then the path with that s (Prop. 3)."""
+    _, extra = forward(p, Q, K, V, L=L, want=("C",))
+    s = whiten_stats(extra["C"], p.H, eps_w)
+    return forward(p, Q, K, V, L=L, whiten=s), s
+
+
+def backward_batch_whiten(p: Problem, Q, K, V, dO, eps_w, L=None):
+    """Adjoint of forward_batch_whiten.  With N = B n rows per head, c_l the column mean of C over them,
+    Z_il = s_l (C_il - mu_i) + 1/m and dZ = dO Y^T:
+        ds_l = sum_{b,i} dZ_il (C_il - mu_i),   dsigma2_l = -1/2 s_l^3 ds_l,   dC_il += dsigma2_l (2/N) (C_il - c_l),
+    on top of the gradient with s held constant; the extra dC goes back through C = k(Q, L) (App. A) and, for pooled
+    landmarks, through the pooling adjoint."""
+    Q, K, V, dO = _f64(Q), _f64(K), _f64(V), _f64(dO)
+    B, H, n, d, m = p.B, p.H, p.n, p.d, p.m
+    _, x = forward(p, Q, K, V, L=L, want=("C", "L"))
+    s = whiten_stats(x["C"], H, eps_w)
+    _, x2 = forward(p, Q, K, V, L=L, whiten=s, want=("Y",))
+    dQ, dK, dV, dL = backward(p, Q, K, V, dO, L=L, whiten=s)
+    C = x["C"].reshape(B, H, n, m)
+    Y = x2["Y"].reshape(B, H, m, d)
+    Lm = x["L"].reshape(B, H, m, d)
+    N = B * n
+    for h in range(H):
+        ds = np.zeros(m)
+        for b in range(B):
+            dZ = dO[b, h] @ Y[b, h].T                                   # [n, m]
+            ds += (dZ * (C[b, h] - C[b, h].mean(axis=1, keepdims=True))).sum(axis=0)
+        cbar = C[:, h].reshape(N, m).mean(axis=0)
+        dsig2 = -0.5 * s[h] ** 3 * ds
+        for b in range(B):
+            dC = dsig2[None, :] * (2.0 / N) * (C[b, h] - cbar[None, :])
+            dq, dl = l1_kernel_bwd(Q[b, h][None], Lm[b, h][None], p.lam, dC[None])
+            dQ[b, h] += dq[0]
+            if p.lm_mode == 0:
+                dL[b, h] += dl[0]
+            else:
+                one = Problem(B=1, H=1, n=n, d=d, m=m, lam=p.lam, ns_iters=0, prefix=p.prefix, gh=p.gh, gw=p.gw, mh=p.mh, mw=p.mw)
+                back = landmarks_pool_bwd(one, dl[None])[0, 0]
+                if p.lm_mode == 1:
+                    dK[b, h] += back
+                else:
+                    dQ[b, h] += back
+    return dQ, dK, dV, dL, s

@@ -520,3 +520,37 @@ def test_landmarks_pooled_from_queries_variant():
     for idx in [(0, 0, 0, 0), (0, 1, 9, 2), (0, 0, 31, 3)]:
         qp, qm = Q.copy(), Q.copy(); qp[idx] += h; qm[idx] -= h
         assert dQ[idx] == pytest.approx((loss(qp) - loss(qm)) / (2 * h), rel=5e-6, abs=1e-8)
+
+
+# --------------------------------------------------------------------------- whitening with batch statistics
+@pytest.mark.parametrize("lm_mode", [1, 0])
+def test_batch_whitening_backward_finite_differences(lm_mode):
+    # Eq. 5-6 in training mode: s comes from the batch's own kernel block; the batch elements of a head are coupled
+    rng = np.random.default_rng(81)
+    d, T, eps_w = 4, 3, 1e-3
+    p = Problem(B=3, H=2, n=12, d=d, m=4, lam=float(d), ns_iters=T, ridge_eps=1e-6, map_mode=1, lm_mode=lm_mode,
+                gh=3, gw=4, mh=2, mw=2)
+    Q, K, V, dO = (rng.standard_normal((3, 2, p.n, d)) for _ in range(4))
+    L = rng.standard_normal((3, 2, p.m, d)) if lm_mode == 0 else None
+    O, s = oracle.forward_batch_whiten(p, Q, K, V, eps_w, L=L)
+    # the forward is the constant-scale path fed with the statistic of the already pinned whiten_stats
+    np.testing.assert_array_equal(O, oracle.forward(p, Q, K, V, L=L, whiten=s))
+    dQ, dK, dV, dL, s2 = oracle.backward_batch_whiten(p, Q, K, V, dO, eps_w, L=L)
+    np.testing.assert_array_equal(s, s2)
+    loss = lambda q, k, v, l: float((oracle.forward_batch_whiten(p, q, k, v, eps_w, L=l)[0] * dO).sum())
+    h = 1e-6
+    for name, arr, grad in (("Q", Q, dQ), ("K", K, dK), ("V", V, dV)):
+        for idx in [(0, 0, 0, 1), (2, 1, 7, 2), (1, 0, 11, 3)]:
+            a = {"Q": Q, "K": K, "V": V}
+            plus, minus = dict(a), dict(a)
+            plus[name] = arr.copy(); plus[name][idx] += h
+            minus[name] = arr.copy(); minus[name][idx] -= h
+            fd = (loss(plus["Q"], plus["K"], plus["V"], L) - loss(minus["Q"], minus["K"], minus["V"], L)) / (2 * h)
+            assert grad[idx] == pytest.approx(fd, rel=2e-5, abs=1e-8), (name, idx)
+    if lm_mode == 0:
+        for idx in [(0, 1, 1, 0), (2, 0, 3, 3)]:
+            lp, lm_ = L.copy(), L.copy(); lp[idx] += h; lm_[idx] -= h
+            assert dL[idx] == pytest.approx((loss(Q, K, V, lp) - loss(Q, K, V, lm_)) / (2 * h), rel=2e-5, abs=1e-8)
+    # the variance path matters: with s held constant the query gradient is a different one
+    dQc = oracle.backward(p, Q, K, V, dO, L=L, whiten=s)[0]
+    assert np.linalg.norm(dQc - dQ) > 1e-3 * np.linalg.norm(dQ)
