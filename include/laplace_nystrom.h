@@ -64,6 +64,14 @@ typedef struct ln_problem {
   int32_t prefix, gh, gw, mh, mw; /* lm_mode 1, 2: n = prefix + gh*gw, m = mh*mw.  Bin (a,b) averages grid  */
                           /* rows floor(a*gh/mh) .. ceil((a+1)*gh/mh)-1 and columns likewise; the first   */
                           /* `prefix` tokens (class tokens) are ordinary queries/keys but are not pooled. */
+  int32_t whiten_mode;    /* 0: `whiten` is a constant input (or NULL = ones).  1: batch statistics (Eq. 5-6 in     */
+                          /* training mode): the forward pass estimates s_l = 1/sqrt(Var_{b,i}(C_il) + whiten_eps)  */
+                          /* over the query rows of every batch element of a head inside the kernel that forms C,  */
+                          /* writes it to whiten_batch and uses it; the backward pass differentiates through the   */
+                          /* variance.  Needs map_mode 1, whiten == NULL.  The batch elements of a head are then    */
+                          /* coupled through the statistic.                                                         */
+  float whiten_eps;       /* eps of Eq. 6 (whiten_mode 1), >= 0                                                     */
+  float* whiten_batch;    /* whiten_mode 1: device [H,m] fp32 written by laplace_nystrom_fwd, read by _bwd         */
 } ln_problem;
 
 const char* ln_status_string(int status);

@@ -46,6 +46,7 @@ class _CProblem(ctypes.Structure):
         ("map_mode", ctypes.c_int32), ("whiten", ctypes.c_void_p), ("lm_mode", ctypes.c_int32),
         ("prefix", ctypes.c_int32), ("gh", ctypes.c_int32), ("gw", ctypes.c_int32),
         ("mh", ctypes.c_int32), ("mw", ctypes.c_int32),
+        ("whiten_mode", ctypes.c_int32), ("whiten_eps", ctypes.c_float), ("whiten_batch", ctypes.c_void_p),
     ]
 
 
@@ -75,6 +76,9 @@ class Problem:
     gw: int = 0
     mh: int = 0
     mw: int = 0
+    whiten_mode: int = 0          # 1: s from this batch's kernel block (Eq. 5-6), gradient through the variance
+    whiten_eps: float = 1e-5
+    whiten_batch: Optional[torch.Tensor] = field(default=None, repr=False)   # device fp32 [H, m], written by the forward pass
 
     def c(self) -> _CProblem:
         w = None
@@ -84,7 +88,8 @@ class Problem:
             w = self.whiten.data_ptr()
         return _CProblem(self.B, self.H, self.n, self.d, self.m, float(self.lam), self.ns_iters,
                          float(self.ridge_eps), float(self.ns_alpha), self.dtype, self.map_mode, w,
-                         self.lm_mode, self.prefix, self.gh, self.gw, self.mh, self.mw)
+                         self.lm_mode, self.prefix, self.gh, self.gw, self.mh, self.mw, self.whiten_mode,
+                         float(self.whiten_eps), None if self.whiten_batch is None else self.whiten_batch.data_ptr())
 
     @property
     def torch_dtype(self):

@@ -64,6 +64,26 @@ struct Carver {
   }
 };
 
+// Tile of the l1 kernel for a problem: LG landmark groups of QN (4 or 2) landmarks, TG token groups of 8,
+// LG * TG <= 256 threads, chosen so that the tiles hug the problem.  Small heads (few pairs per CTA) take
+// the two-landmark thread tile, which fits three CTAs per SM.
+struct L1Launch { dim3 grid, block; size_t smem; int qn; };
+L1Launch plan_l1(int na_max, int nb, int d, int batch, int nprob) {
+  const int qn = ((long long)na_max * nb * d <= (1ll << 20)) ? 2 : 4;
+  const int lg_cap = (qn == 4) ? 16 : 32;
+  int LG = (nb + qn - 1) / qn; if (LG > lg_cap) LG = lg_cap; if (LG < 1) LG = 1;
+  int tg_cap = 256 / LG; if (tg_cap > 32) tg_cap = 32;       // at most 256 tokens per tile
+  const int groups = (na_max + 7) / 8;
+  const int tiles = (groups + tg_cap - 1) / tg_cap;
+  int TG = (groups + tiles - 1) / tiles; if (TG < 1) TG = 1;
+  L1Launch l;
+  l.qn = qn;
+  l.block = dim3(LG, TG);
+  l.grid = dim3((na_max + 8 * TG - 1) / (8 * TG), batch, nprob);
+  l.smem = sizeof(float) * ((size_t)(8 * TG + qn * LG) * L1_PITCH + (size_t)8 * TG * LG);
+  return l;
+}
+
 std::atomic<bool> g_sign3{true};      // test switch: false = the separate upstream kernels and the two-output sign pass
 
 struct Plan {
@@ -75,6 +95,7 @@ struct Plan {
   int mid_sms;                       // SMs the per-head kernels occupy (Newton-Schulz and its adjoint)
   size_t s2_smem;
   int s3_tiles;                      // sign pass with the upstream factor formed in the kernel: token tiles per head (0 = not used)
+  int H, wmode, l1_tiles;            // heads; whitening mode; token tiles of the l1 launch that forms C (statistics partials)
 };
 
 bool make_plan(const ln_problem* p, Plan* pl) {
@@ -137,6 +158,8 @@ bool make_plan(const ln_problem* p, Plan* pl) {
     pl->s2_smem = sign2_smem_bytes(p->m);
   }
   // bf16 storage, 64 or 128 dims: one CTA per tile of 8 * TG tokens, upstream factor on the tensor cores in the kernel
+  pl->H = p->H; pl->wmode = p->whiten_mode;
+  pl->l1_tiles = (int)plan_l1(p->n, p->m, p->d, pl->BH, 1).grid.x;
   pl->s3_tiles = (p->dtype == LN_BF16 && (p->d == 64 || p->d == 128) && g_sign3.load(std::memory_order_relaxed))
                      ? (p->n + 8 * pl->s2_tg - 1) / (8 * pl->s2_tg) : 0;
   return true;
@@ -146,7 +169,7 @@ bool make_plan(const ln_problem* p, Plan* pl) {
 size_t image_floats(const Plan& pl) { return (size_t)((pl.m + GU_KB - 1) / GU_KB) * gu_block_floats(pl.d); }
 
 // Forward context (saved for the backward pass, or carved from ws for inference)
-struct Ctx { float *Lf, *C, *Rt, *mu, *W, *Xh, *Ph, *M, *Yt, *ybar, *Yimg; NsHdr* hdr; size_t bytes; };
+struct Ctx { float *Lf, *C, *Rt, *mu, *W, *Xh, *Ph, *M, *Yt, *ybar, *Yimg, *Y, *cbar; NsHdr* hdr; size_t bytes; };
 Ctx carve_ctx(const Plan& pl, void* base) {
   Carver c(base); Ctx x;
   const size_t BH = pl.BH, n = pl.n, d = pl.d, m = pl.m;
@@ -162,24 +185,26 @@ Ctx carve_ctx(const Plan& pl, void* base) {
   x.ybar = c.take(BH * d);
   x.Yimg = c.take(BH * image_floats(pl));        // Ytilde once more, as split operand images
   x.hdr = reinterpret_cast<NsHdr*>(c.take(BH * (sizeof(NsHdr) / sizeof(float))));
+  x.Y = c.take(BH * m * d);                      // Y = X M before the map is folded in (batch-statistic whitening needs it)
+  x.cbar = c.take((size_t)pl.H * m);             // column means of C over the batch (batch-statistic whitening)
   x.bytes = c.off;
   return x;
 }
 
-struct FwdWs { float *Mpart, *Wr, *P, *Y; size_t bytes; };
+struct FwdWs { float *Mpart, *Wr, *P; double* stat; size_t bytes; };
 FwdWs carve_fwd_ws(const Plan& pl, void* base) {
   Carver c(base); FwdWs w;
   const size_t BH = pl.BH, d = pl.d, m = pl.m;
   w.Mpart = c.take(BH * pl.chunks * m * d);
   w.Wr = c.take(BH * pl.scr);
   w.P = c.take(BH * pl.scr);
-  w.Y = c.take(BH * m * d);
+  w.stat = reinterpret_cast<double*>(c.take(pl.wmode == 1 ? BH * (size_t)pl.l1_tiles * m * 4 : 0));   // [BH][tiles][m][2] doubles
   w.bytes = c.off;
   return w;
 }
 
 struct BwdWs {
-  float *G, *G2, *dYtpart, *dybpart, *dLCpart, *dLRpart, *dY, *dM, *Wr, *P, *Hm, *Ga, *Gb, *dW, *dX, *GW, *dLW, *dLtot, *dKpart, *dMimg, *SB;
+  float *G, *G2, *dYtpart, *dybpart, *dLCpart, *dLRpart, *dY, *dM, *Wr, *P, *Hm, *Ga, *Gb, *dW, *dX, *GW, *dLW, *dLtot, *dKpart, *dMimg, *SB, *kap;
   size_t bytes;
 };
 BwdWs carve_bwd_ws(const Plan& pl, void* base) {
@@ -210,6 +235,7 @@ BwdWs carve_bwd_ws(const Plan& pl, void* base) {
   w.dKpart = c.take(BH * n * d);
   w.dMimg = c.take(BH * image_floats(pl));
   w.SB = c.take(pl.s3_tiles > 0 ? BH * m * 2 * d : 0);      // scale and offset of every landmark value (folded step)
+  w.kap = c.take(pl.wmode == 1 ? (size_t)pl.H * m * 2 : 0); // batch-statistic whitening: (kappa_l, cbar_l) per head and landmark
   w.bytes = c.off;
   return w;
 }
@@ -226,6 +252,11 @@ int validate(const ln_problem* p) {
   if (p->map_mode != 0 && p->map_mode != 1) return LN_ERR_ARG;
   if (p->lm_mode < 0 || p->lm_mode > 2) return LN_ERR_ARG;
   if (p->whiten && !aligned16(p->whiten)) return LN_ERR_ARG;
+  if (p->whiten_mode != 0 && p->whiten_mode != 1) return LN_ERR_ARG;
+  if (p->whiten_mode == 1) {
+    if (p->map_mode != 1 || p->whiten || !p->whiten_batch || !aligned16(p->whiten_batch)) return LN_ERR_ARG;
+    if (!(p->whiten_eps >= 0.f) || !isfinite(p->whiten_eps)) return LN_ERR_ARG;
+  }
   if (p->lm_mode >= 1) {
     if (p->prefix < 0 || p->gh <= 0 || p->gw <= 0 || p->mh <= 0 || p->mw <= 0) return LN_ERR_ARG;
     if ((long long)p->prefix + (long long)p->gh * p->gw != p->n) return LN_ERR_ARG;
@@ -337,26 +368,6 @@ Side side_acquire(bool want, cudaStream_t caller) {
   return r;
 }
 
-// Tile of the l1 kernel for a problem: LG landmark groups of QN (4 or 2) landmarks, TG token groups of 8,
-// LG * TG <= 256 threads, chosen so that the tiles hug the problem.  Small heads (few pairs per CTA) take
-// the two-landmark thread tile, which fits three CTAs per SM.
-struct L1Launch { dim3 grid, block; size_t smem; int qn; };
-L1Launch plan_l1(int na_max, int nb, int d, int batch, int nprob) {
-  const int qn = ((long long)na_max * nb * d <= (1ll << 20)) ? 2 : 4;
-  const int lg_cap = (qn == 4) ? 16 : 32;
-  int LG = (nb + qn - 1) / qn; if (LG > lg_cap) LG = lg_cap; if (LG < 1) LG = 1;
-  int tg_cap = 256 / LG; if (tg_cap > 32) tg_cap = 32;       // at most 256 tokens per tile
-  const int groups = (na_max + 7) / 8;
-  const int tiles = (groups + tg_cap - 1) / tg_cap;
-  int TG = (groups + tiles - 1) / tiles; if (TG < 1) TG = 1;
-  L1Launch l;
-  l.qn = qn;
-  l.block = dim3(LG, TG);
-  l.grid = dim3((na_max + 8 * TG - 1) / (8 * TG), batch, nprob);
-  l.smem = sizeof(float) * ((size_t)(8 * TG + qn * LG) * L1_PITCH + (size_t)8 * TG * LG);
-  return l;
-}
-
 // Launch with `cl` CTAs per thread-block cluster (cl = 1: an ordinary launch).
 constexpr int kMidCluster = 4;     // CTAs that share one head on the m > 128 Newton-Schulz path
 template <typename... KArgs, typename... Args>
@@ -372,9 +383,9 @@ void launch_clustered(void (*kern)(KArgs...), int grid, int cl, size_t smem, cud
 
 template <typename T> constexpr int is_f32() { return std::is_same<T, float>::value ? 1 : 0; }
 
-L1Prob l1_prob(const void* A, int a_f32, float* E, float* rowsum, int na, int d, int lde, float rs_scale) {
+L1Prob l1_prob(const void* A, int a_f32, float* E, float* rowsum, int na, int d, int lde, float rs_scale, double* stat = nullptr) {
   L1Prob q; q.A = A; q.E = E; q.rowsum = rowsum; q.sA = (long long)na * d; q.sE = (long long)na * lde;
-  q.na = na; q.lde = lde; q.a_f32 = a_f32; q.rs_scale = rs_scale;
+  q.na = na; q.lde = lde; q.a_f32 = a_f32; q.rs_scale = rs_scale; q.stat = stat;
   return q;
 }
 
@@ -425,7 +436,9 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // blocks at about half of the FP32 peak
   const double ns_us = pl.T * (m <= 64 ? 5.0 : (m <= 128 ? 12.0 : 100.0));
   const double l1_us = 2.0 * 2.0 * n * m * D * BH / 20e6;
-  const bool deep = side.on() && l1_us >= ns_us;
+  const bool bw = p->whiten_mode == 1;              // batch-statistic whitening: s comes out of the kernel block C of this call
+  const float* const whiten_eff = bw ? p->whiten_batch : p->whiten;
+  const bool deep = side.on() && l1_us >= ns_us && !bw;   // (the map fold then has to wait for C: no work is left to run beside it)
   const float* const Mparts_src = w.Mpart;
   const int Mparts = pl.chunks == 1 ? 0 : pl.chunks;
   // Newton-Schulz (phase bit 0) and Y = X M with the folded map (phase bit 1), one CTA or cluster per head
@@ -435,7 +448,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
       want_smem(kern, smem);
       LN_LAUNCH(phase == 3 ? "k_mid_fwd" : (phase == 1 ? "k_mid_fwd_ns" : "k_mid_fwd_y"), s,
                 launch_clustered(kern, BH * cl, cl, smem, s, m, pl.ldm, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode,
-                                 p->whiten, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, Mparts_src, Mparts, x.M, w.Y, x.Yt,
+                                 whiten_eff, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, Mparts_src, Mparts, x.M, x.Y, x.Yt,
                                  x.ybar, dev_status, pl.hslot, umma_prod ? reinterpret_cast<bf16*>(x.Yimg) : nullptr, phase));
     };
     if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * kUmmaMatBytes64);
@@ -447,7 +460,8 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     L1Args a;
     a.Bm = x.Lf; a.sB = (long long)m * D; a.nb = m; a.d = D; a.b_f32 = 1;
     a.nscale = -1.4426950408889634f / p->lambda;
-    const L1Prob pc = l1_prob(Q, is_f32<T>(), x.C, p->map_mode == 1 ? x.mu : nullptr, n, D, pl.ldm, 1.f / (float)m);  // row means (Prop. 3 step 2)
+    const L1Prob pc = l1_prob(Q, is_f32<T>(), x.C, p->map_mode == 1 ? x.mu : nullptr, n, D, pl.ldm, 1.f / (float)m,  // row means (Prop. 3 step 2)
+                              bw ? w.stat : nullptr);                                                                    // column statistics (Eq. 5)
     const L1Prob pr = l1_prob(K, is_f32<T>(), x.Rt, nullptr, n, D, pl.ldm, 1.f);
     const L1Prob pw = l1_prob(x.Lf, 1, x.W, nullptr, m, D, m, 1.f);
     if (side.on()) {
@@ -477,6 +491,9 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     LN_LAUNCH("tn_M", sm_, k_tn_mma<D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, sm_>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
   else
     LN_LAUNCH("tn_M", sm_, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, sm_>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
+  // whitening scale from the statistics the C block left (Eq. 6), before the map is folded
+  if (bw) LN_LAUNCH("k_wstat_final", st, k_wstat_final<<<dim3(cdiv(m, 32), p->H), 256, 0, st>>>(w.stat, p->B, p->H, n, m, pl.l1_tiles, p->whiten_eps,
+                                                                                               p->whiten_batch, x.cbar));
   // Newton-Schulz, Y = X M, folded map
   if (side.on() && !deep) { side.join(st); launch_mid(st, 2); }
   else if (side.on()) {
@@ -534,12 +551,15 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const int chs = sign3 ? pl.s3_tiles : (fused_sign ? pl.s2_chunks : ch);
   const int chq = sign3 ? pl.s3_tiles : (fused_sign ? pl.s2q_chunks : ch);    // chunks of the query-side landmark-gradient partials
   // one sign pass of a token-sized block: tokens, upstream operands (U, pre-split images of Y), kernel block A
-  auto launch_sign3 = [&](const char* name, const T* tokp, const T* Up, const float* Yimgp, const float* Ap, auto* rowsp, float* partp) {
+  const bool bw = p->whiten_mode == 1;                // batch-statistic whitening: the scale is the forward pass's own estimate
+  const float* const whiten_eff = bw ? p->whiten_batch : p->whiten;
+  auto launch_sign3 = [&](const char* name, const T* tokp, const T* Up, const float* Yimgp, const float* Ap, auto* rowsp, float* partp,
+                          const float* kap = nullptr) {
     if constexpr (std::is_same<T, bf16>::value && (D == 64 || D == 128)) {
       auto go = [&](auto kern) {
         want_smem(kern, sign3_smem_bytes());
         LN_LAUNCH(name, st, kern<<<dim3(pl.s3_tiles, D / 64, BH), dim3(16, pl.s2_tg), sign3_smem_bytes(), st>>>(
-                      tokp, w.SB, Up, reinterpret_cast<const bf16*>(Yimgp), Ap, pl.ldm, rowsp, partp, n, m, inv_lambda, dev_status));
+                      tokp, w.SB, Up, reinterpret_cast<const bf16*>(Yimgp), Ap, pl.ldm, rowsp, partp, n, m, inv_lambda, dev_status, kap, p->H));
       };
       using TO = std::remove_pointer_t<decltype(rowsp)>;
       if (pl.s2_tg == S3_TGMAX) go(k_sign3<TO, D, 1, true>); else go(k_sign3<TO, D, 2, true>);
@@ -553,7 +573,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     constexpr bool TC = std::is_same<T, bf16>::value;
     auto launch = [&](auto kern, size_t smem, int cl = 1) {
       want_smem(kern, smem);
-      LN_LAUNCH("k_mid_bwd", s, launch_clustered(kern, BH * cl, cl, smem, s, m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, p->whiten,
+      LN_LAUNCH("k_mid_bwd", s, launch_clustered(kern, BH * cl, cl, smem, s, m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, whiten_eff,
                                                  x.W, x.Xh, x.Ph, x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P,
                                                  w.Hm, w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot,
                                                  umma_prod ? reinterpret_cast<bf16*>(w.dMimg) : nullptr));
@@ -604,8 +624,13 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const double side_us = pl.T * (m <= 64 ? 7.0 : (m <= 128 ? 16.0 : 30.0)) * mid_waves;
   const double sign_ops = 3.0 * n * m * D * BH;
   const double main_us = sign_ops / (37.2e6 * (sign_ops > 4e9 ? 0.43 : 0.25));
-  const bool tn_on_side = side.on() && side_us < 0.8 * main_us;
+  const bool tn_on_side = side.on() && side_us < 0.8 * main_us && !bw;
   if (!tn_on_side) launch_tn_dY(st);
+  // Batch-statistic whitening: ds needs Z'^T dO of every batch element of a head, and the query-side sign pass needs
+  // the coefficient it gives, so Z'^T dO stays on the caller's stream in front of both.
+  const float* const kap = bw ? w.kap : nullptr;
+  if (bw) LN_LAUNCH("k_whiten_bwd", st, k_whiten_bwd<<<dim3(cdiv(m, 8), p->H), 256, 0, st>>>(x.Y, w.dYtpart, ch, p->whiten_batch, x.cbar, p->B, p->H,
+                                                                                            n, m, D, w.kap));
   if (side.on()) {
     side.fork(st);
     if (tn_on_side) launch_tn_dY(side.s);
@@ -618,9 +643,12 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   if (sign3) {
     const long long cnt = (long long)BH * m * D;
     LN_LAUNCH("k_fold_landmarks", st, k_fold_landmarks<<<cdiv(cnt, 256), 256, 0, st>>>(x.Lf, w.SB, D, cnt));
-    if (poolQ) launch_sign3("sign3_dQ_dLC", Q, dO, x.Yimg, x.C, w.dKpart, w.dLCpart);
-    else launch_sign3("sign3_dQ_dLC", Q, dO, x.Yimg, x.C, dQ, w.dLCpart);
-  } else launch_ntg_C();
+    if (poolQ) launch_sign3("sign3_dQ_dLC", Q, dO, x.Yimg, x.C, w.dKpart, w.dLCpart, kap);
+    else launch_sign3("sign3_dQ_dLC", Q, dO, x.Yimg, x.C, dQ, w.dLCpart, kap);
+  } else {
+    launch_ntg_C();
+    if (bw) LN_LAUNCH("k_g_whiten_add", st, k_g_whiten_add<<<dim3(cdiv((long long)n * pl.ldm, 256), BH), 256, 0, st>>>(w.G, x.C, w.kap, p->H, n, m, pl.ldm, inv_lambda));
+  }
   if (sign3) {
   } else if (fused_sign) {
     auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
@@ -904,7 +932,7 @@ int laplace_nystrom_whiten_stats(const ln_problem* p, const void* saved, float e
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   double* part = static_cast<double*>(ws);
   LN_LAUNCH("k_wstat_part", st, k_wstat_part<<<dim3(sp, pl.BH), 256, 0, st>>>(x.C, pl.ldm, p->n, p->m, rps, part));
-  LN_LAUNCH("k_wstat_final", st, k_wstat_final<<<dim3(cdiv(p->m, 32), p->H), 256, 0, st>>>(part, p->B, p->H, p->n, p->m, sp, eps_w, whiten_out));
+  LN_LAUNCH("k_wstat_final", st, k_wstat_final<<<dim3(cdiv(p->m, 32), p->H), 256, 0, st>>>(part, p->B, p->H, p->n, p->m, sp, eps_w, whiten_out, nullptr));
   return launch_ok();
 }
 

@@ -30,6 +30,7 @@ struct L1Prob {
   long long sA, sE;      // per-batch strides of A (elements) and E
   int na, lde, a_f32;
   float rs_scale;
+  double* stat;          // NULL, or column statistics of E per token tile: [batch][tiles][nb][2] = (sum_i E_ij, sum_i E_ij^2)
 };
 struct L1Args {
   L1Prob p[3];
@@ -152,6 +153,41 @@ __global__ void __launch_bounds__(256, QN == 4 ? 2 : 3) k_l1(const L1Args args) 
         }
       }
     }
+    if (pr.stat) {
+      // Column statistics of this tile for the whitening scale (Eq. 5): per landmark the sums of t = E - pivot and of
+      // t^2 over the tile's tokens, the pivot being the tile's first row (it makes t small, so that fp32 loses
+      // nothing), moved to sums about zero in double by the thread that adds up the TG token groups in a fixed order.
+      __syncthreads();                                   // every thread has finished reading the staged operands
+      float* Ps = l1_smem;                               // [TB] pivots
+      float* Sr = l1_smem + TB;                          // [TG][TB][2]
+      if (ti == 0)
+#pragma unroll
+        for (int q = 0; q < QN; ++q) Ps[tj + LG * q] = ex2(acc[0][q] * args.nscale);
+      __syncthreads();
+#pragma unroll
+      for (int q = 0; q < QN; ++q) {
+        const float pv = Ps[tj + LG * q];
+        float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          if (i0 + ti + TG * k < na) { const float t = ex2(acc[k][q] * args.nscale) - pv; s1 += t; s2 = fmaf(t, t, s2); }
+        Sr[(ti * TB + tj + LG * q) * 2] = s1;
+        Sr[(ti * TB + tj + LG * q) * 2 + 1] = s2;
+      }
+      __syncthreads();
+      for (int c = tid; c < TB; c += nthr) {
+        const int gj = j0 + c;
+        if (gj < nb) {
+          float a = 0.f, q2 = 0.f;
+          for (int t = 0; t < TG; ++t) { a += Sr[(t * TB + c) * 2]; q2 += Sr[(t * TB + c) * 2 + 1]; }
+          const double pv = (double)Ps[c], cnt = (double)min(TA, na - i0);
+          double* o = pr.stat + (((long long)b * gridDim.x + blockIdx.x) * nb + gj) * 2;
+          o[0] = (double)a + cnt * pv;
+          o[1] = (double)q2 + 2.0 * pv * (double)a + cnt * pv * pv;
+        }
+      }
+      __syncthreads();                                   // the staging buffers are free again for the next landmark tile
+    }
   }
   if (pr.rowsum) {      // fixed-order reduction over the LG threads of a row
     __syncthreads();
@@ -226,7 +262,8 @@ __global__ void __launch_bounds__(256) k_wstat_part(const float* __restrict__ C,
 // grid (ceil(m / 32), H), block 256: lane = landmark of the group of 32, warp w adds terms w, w + 8, ... (term t = batch
 // element t / nsplit, split t % nsplit; eight loads in flight), the eight warps are added in a fixed order
 __global__ void __launch_bounds__(256) k_wstat_final(const double* __restrict__ part, int B, int H, int n, int m, int nsplit,
-                                                     float eps, float* __restrict__ s_out /* [H][m] */) {
+                                                     float eps, float* __restrict__ s_out /* [H][m] */,
+                                                     float* __restrict__ mean_out /* NULL or [H][m] */) {
   __shared__ double red[8][32][2];
   const int h = blockIdx.y, lane = threadIdx.x & 31, w = threadIdx.x >> 5, l = blockIdx.x * 32 + lane;
   const int terms = B * nsplit;
@@ -265,7 +302,52 @@ __global__ void __launch_bounds__(256) k_wstat_final(const double* __restrict__ 
     double var = q / cnt - mu * mu;
     if (var < 0.0) var = 0.0;
     s_out[h * m + l] = (float)(1.0 / sqrt(var + (double)eps));
+    if (mean_out) mean_out[h * m + l] = (float)mu;
   }
+}
+
+// Gradient of the loss with respect to the batch-statistic whitening scale, turned into the coefficient of the extra
+// upstream term of the query-landmark block (Eq. 5-6 in training mode).  With Z_il = s_l (C_il - mu_i) + 1/m,
+//     ds_l = sum_{b,i} (dO_i . Y_l)(C_il - mu_i) = sum_b <Y_l, ((C - mu)^T dO)_l>,
+//     dsigma2_l = -1/2 s_l^3 ds_l,     dC_il += dsigma2_l (2/N)(C_il - cbar_l),   N = B n,
+// so kap[h][l] = (kappa_l, cbar_l) with kappa_l = -s_l^3 ds_l / N.  One warp per (head, landmark): lanes run over the
+// dims, batch elements and token chunks are added in a fixed order.  grid (ceil(m/8), H), block 256.
+__global__ void __launch_bounds__(256) k_whiten_bwd(const float* __restrict__ Y, const float* __restrict__ dYtpart, int nchunks,
+                                                    const float* __restrict__ s, const float* __restrict__ cbar, int B, int H,
+                                                    int n, int m, int d, float* __restrict__ kap /* [H][m][2] */) {
+  const int h = blockIdx.y, l = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (l >= m) return;
+  float acc = 0.f;
+  for (int b = 0; b < B; ++b) {
+    const long long bh = (long long)b * H + h;
+    for (int c = lane; c < d; c += 32) {
+      float t = 0.f;
+      for (int k = 0; k < nchunks; ++k) t += dYtpart[((bh * nchunks + k) * m + l) * d + c];
+      acc = fmaf(Y[(bh * m + l) * d + c], t, acc);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) {
+    const float sl = s[h * m + l];
+    kap[(h * m + l) * 2] = -sl * sl * sl * acc / ((float)B * (float)n);
+    kap[(h * m + l) * 2 + 1] = cbar[h * m + l];
+  }
+}
+
+// G[i][l] += kappa_l (C[i][l] - cbar_l) C[i][l] / lambda: the extra upstream term of batch-statistic whitening for the
+// paths that materialise G (fp32 storage, 32-dim heads).
+__global__ void __launch_bounds__(256) k_g_whiten_add(float* __restrict__ G, const float* __restrict__ C, const float* __restrict__ kap,
+                                                      int H, int n, int m, int ldm, float inv_lambda) {
+  const int bh = blockIdx.y;
+  const long long e = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (e >= (long long)n * ldm) return;
+  const int l = (int)(e % ldm);
+  if (l >= m) return;
+  const float* kp = kap + ((long long)(bh % H) * m + l) * 2;
+  const long long idx = (long long)bh * n * ldm + e;
+  const float c = C[idx];
+  G[idx] += kp[0] * (c - kp[1]) * c * inv_lambda;
 }
 
 // storage type -> fp32 copy

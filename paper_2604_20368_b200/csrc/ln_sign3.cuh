@@ -39,7 +39,8 @@ constexpr int S3_GS = S3_CP + 2 * S3_RL * S3_TGMAX * S3_DS;         // [2][RL][T
 constexpr int S3_SB = S3_GS + 2 * S3_RL * S3_TOK;                   // [2][RL][2][64] scales and offsets of the landmark values
 constexpr int S3_RS = S3_SB + 2 * S3_RL * 2 * S3_DS;                // [TOK] row sums of g
 constexpr int S3_CS = S3_RS + S3_TOK;                               // [<= 256] column sums of g
-constexpr int S3_END = S3_CS + 256;
+constexpr int S3_KC = S3_CS + 256;                                  // [<= 256][2] batch-whitening coefficients (kappa, cbar) per landmark
+constexpr int S3_END = S3_KC + 512;
 __host__ __device__ constexpr size_t sign3_smem_bytes() { return sizeof(float) * (size_t)S3_END; }
 static_assert((size_t)(128 * 128 + 2 * GU_KB * 128) * sizeof(bf16) <= sizeof(float) * (size_t)(S3_GS - S3_CP),
               "the operand images of the MMA phase fit in the column-partial buffers they alias");
@@ -74,7 +75,8 @@ template <typename TO, int D, int NR, bool FUSED>
 __global__ void __launch_bounds__(256, 2) k_sign3(const bf16* __restrict__ tok, const float* __restrict__ SB,
                                                   const bf16* __restrict__ U, const bf16* __restrict__ Yimg,
                                                   const float* __restrict__ A, int lda, TO* __restrict__ rows,
-                                                  float* __restrict__ part, int n, int m, float inv_lambda, int* dev_status) {
+                                                  float* __restrict__ part, int n, int m, float inv_lambda, int* dev_status,
+                                                  const float* __restrict__ kap /* NULL or [H][m][2] */, int H) {
   extern __shared__ __align__(128) float s3_smem[];
   __shared__ __align__(8) unsigned long long mbar_y, mbar_mma;
   __shared__ uint32_t tmem_base;
@@ -100,6 +102,10 @@ __global__ void __launch_bounds__(256, 2) k_sign3(const bf16* __restrict__ tok, 
   // ---- set-up that does not touch the aliased buffers: zero the never-written slots >= TG of the column partials
   // later (they alias the operands); column sums of g
   for (int e = tid; e < nrounds * S3_RL; e += nthr) colsum[e] = 0.f;
+  // batch-statistic whitening (Eq. 5-6 in training mode): the kernel block's upstream gains kappa_l (A_il - cbar_l)
+  float* const kc = s3_smem + S3_KC;
+  if (kap) for (int e = tid; e < 2 * m; e += nthr) kc[e] = kap[(long long)(bh % H) * m * 2 + e];
+  if constexpr (!FUSED) __syncthreads();
 
   // scale / offset tile of round r into buffer r & 1: 8 landmarks x (64 scales, 64 offsets) = 128 pieces of 16 bytes
   auto fetch_sb = [&](int r) {
@@ -210,6 +216,11 @@ __global__ void __launch_bounds__(256, 2) k_sign3(const bf16* __restrict__ tok, 
       if constexpr (FUSED) {
         float da[4];
         s3_tmem_ld4(tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)l, da);
+        if (kap) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            if (l + e < m) da[e] = fmaf(kc[2 * (l + e)], g[e] - kc[2 * (l + e) + 1], da[e]);
+        }
 #pragma unroll
         for (int e = 0; e < 4; ++e) g[e] *= da[e];
       }

@@ -291,6 +291,38 @@ def test_landmarks_pooled_from_queries(name, B, H):
     assert_parity(cfg, errs)
 
 
+@pytest.mark.parametrize("name,B,H,dtype", [("cfg2", 3, 2, "bf16"), ("cfg2", 2, 1, "f32"), ("cfg4a", 2, 1, "bf16"),
+                                            ("cfg5_m64_T4", 2, 1, "bf16"), ("cfg1", 2, 2, "f32")])
+def test_batch_statistic_whitening_training_mode(name, B, H, dtype):
+    """whiten_mode 1 (Eq. 5-6 in training mode): the scale is estimated inside the kernel that forms C = k(Q, L), over
+    the query rows of every batch element of a head, and the backward pass differentiates through the variance."""
+    from dataclasses import replace
+    from parity import metrics
+    cfg = replace(synth.shrink(synth.CONFIGS[name], B=B, H=H), backward=True, dtype=dtype)
+    inp = synth.make_inputs(cfg)
+    Q, K, V, dO = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
+    eps_w = 1e-5
+    p = ln.problem_from_config(cfg, whiten=None)
+    p.whiten_mode, p.whiten_eps = 1, eps_w
+    p.whiten_batch = torch.full((cfg.H, cfg.m), float("nan"), device=DEV)
+    saved = torch.empty(ln.laplace_nystrom_saved_bytes(p), dtype=torch.uint8, device=DEV)
+    O = ln.laplace_nystrom_fwd(p, Q, K, V, saved=saved)
+    dQ, dK, dV, _ = ln.laplace_nystrom_bwd(p, Q, K, V, dO, saved)
+    op = oracle_problem(cfg)
+    q, k, v, g = (f64(inp[x]) for x in ("Q", "K", "V", "dO"))
+    Oo, so = oracle.forward_batch_whiten(op, q, k, v, eps_w)
+    dQo, dKo, dVo, _, _ = oracle.backward_batch_whiten(op, q, k, v, g, eps_w)
+    assert rel_err(f64(p.whiten_batch), so) < 1e-4
+    BH = cfg.B * cfg.H
+    errs = {kk: metrics(f64(a).reshape(BH, cfg.n, cfg.d), r.reshape(BH, cfg.n, cfg.d), dtype == "bf16")
+            for kk, a, r in (("O", O, Oo), ("dQ", dQ, dQo), ("dK", dK, dKo), ("dV", dV, dVo))}
+    print(cfg.name, "batch whitening", {kk: {a: f"{b:.1e}" for a, b in e.items()} for kk, e in errs.items()})
+    assert_parity(cfg, errs)
+    # the variance path is really there: against the constant-scale gradient the query gradient differs visibly
+    dQc = oracle.backward(op, q, k, v, g, whiten=so)[0]
+    assert rel_err(f64(dQ), dQc) > 5 * rel_err(f64(dQ), dQo)
+
+
 def test_inference_without_saved_matches_training_forward():
     cfg = synth.shrink(synth.CONFIGS["cfg2"], B=1)
     inp = synth.make_inputs(cfg)
