@@ -269,17 +269,17 @@ def alu_probe(ln, dev):
     sink = torch.zeros(1025, dtype=torch.float32, device=dev)
     out = {}
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
-    for packed in (False, True):
+    for mode, name in ((0, "scalar"), (1, "packed"), (2, "sign_mix"), (3, "l1_mix")):
         best = 0.0
-        ln.fp32_add_probe(sms * 8, 2000, packed, sink)
+        ln.fp32_add_probe(sms * 8, 2000, mode, sink)
         for _ in range(3):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            ops = ln.fp32_add_probe(sms * 8, 20000, packed, sink)
+            ops = ln.fp32_add_probe(sms * 8, 20000, mode, sink)
             e1.record()
             torch.cuda.synchronize()
             best = max(best, ops / (e0.elapsed_time(e1) * 1e-3) / 1e12)
-        out["packed" if packed else "scalar"] = best
+        out[name] = best
     return out
 
 

@@ -274,14 +274,17 @@ int laplace_nystrom_saved_array(const ln_problem* p, const char* name, int64_t i
 int ln_selftest_wait_timeout(int32_t probes, int32_t* dev_status, void* stream);
 
 /*
- * FP32 add-rate probe (the paper has no counterpart; a measurement aid).  `blocks` CTAs of 256 threads run `iters`
- * steps of eight independent add chains per thread, two lanes per chain and step (packed = 0: two scalar adds,
- * packed = 1: one add.f32x2), without memory traffic.  ln_fp32_add_probe_lane_ops returns the lane-operations of
- * such a launch; divided by its duration it is the measured counterpart of the derived FP32 peak
- * (SMs x 128 lanes x clock).  sink: device fp32 [1025], sink[0] is read, nothing else is normally written.
+ * FP32 rate probe (the paper has no counterpart; a measurement aid).  `blocks` CTAs of 256 threads run `iters` steps of
+ * eight independent dependent-chains per thread, in registers only.  mode 0: two scalar adds per chain and step;
+ * 1: one packed add.f32x2; 2: the instruction mix of the sign pass of App. A as this library runs it (two saturating
+ * multiply-adds, two packed multiply-adds: 6 lane-operations); 3: the mix of the l1 forward (one packed subtract, two
+ * |.| accumulations: 4 lane-operations); 4: mix 2 with its scalar and packed instructions in separate runs; 5: mix 2
+ * with scalar instructions only.  ln_fp32_add_probe_lane_ops returns the lane-operations of such a launch;
+ * divided by its duration it is the measured counterpart of the derived FP32 peak (SMs x 128 lanes x clock), for plain
+ * adds and for the two mixes the ALU-bound kernels are made of.  sink: device fp32 [1025], sink[0] is read.
  */
-int ln_fp32_add_probe(int32_t blocks, int32_t iters, int32_t packed, float* sink, void* stream);
-int64_t ln_fp32_add_probe_lane_ops(int32_t blocks, int32_t iters);
+int ln_fp32_add_probe(int32_t blocks, int32_t iters, int32_t mode, float* sink, void* stream);
+int64_t ln_fp32_add_probe_lane_ops(int32_t blocks, int32_t iters, int32_t mode);
 
 /*
  * Profiling aid, off by default and not thread-safe (the paper has no counterpart; Sec. 4.3 only

@@ -148,7 +148,7 @@ def lib():
         L.ln_selftest_wait_timeout.argtypes = [i32, vp, vp]
         L.ln_fp32_add_probe.argtypes = [i32, i32, i32, vp, vp]
         L.ln_fp32_add_probe_lane_ops.restype = ctypes.c_int64
-        L.ln_fp32_add_probe_lane_ops.argtypes = [i32, i32]
+        L.ln_fp32_add_probe_lane_ops.argtypes = [i32, i32, i32]
         L.laplace_exact_fwd.argtypes = [i32, i32, i32, i32, f32, i32, vp, vp, vp, vp, vp]
         pb = ctypes.POINTER(_CBlock)
         L.laplace_attention_block_saved_bytes.restype = sz
@@ -436,10 +436,11 @@ def selftest_wait_timeout(dev_status: torch.Tensor, probes: int = 1000, stream=N
     _check(lib().ln_selftest_wait_timeout(probes, _ptr(dev_status), _stream(stream)), "ln_selftest_wait_timeout")
 
 
-def fp32_add_probe(blocks: int, iters: int, packed: bool, sink: torch.Tensor, stream=None) -> int:
-    """Launch the FP32 add-rate probe; returns the lane-operations the launch performs."""
-    _check(lib().ln_fp32_add_probe(blocks, iters, int(packed), _ptr(sink), _stream(stream)), "ln_fp32_add_probe")
-    return int(lib().ln_fp32_add_probe_lane_ops(blocks, iters))
+def fp32_add_probe(blocks: int, iters: int, mode: int, sink: torch.Tensor, stream=None) -> int:
+    """Launch the FP32 rate probe (mode 0 scalar adds, 1 packed adds, 2 sign-pass mix, 3 l1-forward mix); returns the
+    lane-operations the launch performs."""
+    _check(lib().ln_fp32_add_probe(blocks, iters, int(mode), _ptr(sink), _stream(stream)), "ln_fp32_add_probe")
+    return int(lib().ln_fp32_add_probe_lane_ops(blocks, iters, int(mode)))
 
 
 def launch_count() -> int:

@@ -488,7 +488,10 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   float* const Mdst = pl.chunks == 1 ? x.M : w.Mpart;
   const cudaStream_t sm_ = deep ? side.s : st;               // stream of M = R V and of what follows from it
   if constexpr (std::is_same<T, bf16>::value)
-    LN_LAUNCH("tn_M", sm_, k_tn_mma<D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, sm_>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
+  {
+    want_smem(k_tn_mma<D>, tn_mma_smem<D>());
+    LN_LAUNCH("tn_M", sm_, k_tn_mma<D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, tn_mma_smem<D>(), sm_>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
+  }
   else
     LN_LAUNCH("tn_M", sm_, k_tn<T, D><<<dim3(pl.chunks, cdiv(m, 64), BH), 256, 0, sm_>>>(x.Rt, pl.ldm, nullptr, V, Mdst, nullptr, n, m, pl.rpc));
   // whitening scale from the statistics the C block left (Eq. 6), before the map is folded
@@ -529,7 +532,10 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // query side: Z'^T dO and column sums of dO; g^C = (dO Ytilde^T) o C / lambda; dQ; landmark part
   auto launch_tn_dY = [&](cudaStream_t s) {
     if constexpr (std::is_same<T, bf16>::value)
-      LN_LAUNCH("tn_dY", s, k_tn_mma<D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, s>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
+    {
+      want_smem(k_tn_mma<D>, tn_mma_smem<D>());
+      LN_LAUNCH("tn_dY", s, k_tn_mma<D><<<dim3(ch, cdiv(m, 64), BH), 256, tn_mma_smem<D>(), s>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
+    }
     else
       LN_LAUNCH("tn_dY", s, k_tn<T, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, s>>>(x.C, pl.ldm, mu, dO, w.dYtpart, w.dybpart, n, m, pl.rpc));
   };
@@ -1152,13 +1158,16 @@ int ln_selftest_wait_timeout(int32_t probes, int32_t* dev_status, void* stream) 
   return launch_ok();
 }
 
-int ln_fp32_add_probe(int32_t blocks, int32_t iters, int32_t packed, float* sink, void* stream) {
-  if (blocks <= 0 || iters <= 0 || !sink) return LN_ERR_ARG;
+int ln_fp32_add_probe(int32_t blocks, int32_t iters, int32_t mode, float* sink, void* stream) {
+  if (blocks <= 0 || iters <= 0 || !sink || mode < 0 || mode > 5) return LN_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  LN_LAUNCH("k_fp32_add_probe", st, k_fp32_add_probe<<<blocks, 256, 0, st>>>(packed ? -iters : iters, sink));
+  LN_LAUNCH("k_fp32_add_probe", st, k_fp32_add_probe<<<blocks, 256, 0, st>>>(iters, mode, sink));
   return launch_ok();
 }
-int64_t ln_fp32_add_probe_lane_ops(int32_t blocks, int32_t iters) { return (int64_t)blocks * 256 * iters * kProbeChains * 2; }
+int64_t ln_fp32_add_probe_lane_ops(int32_t blocks, int32_t iters, int32_t mode) {
+  const int per_step[6] = {2, 2, 6, 4, 6, 6};
+  return (mode < 0 || mode > 5) ? 0 : (int64_t)blocks * 256 * iters * kProbeChains * per_step[mode];
+}
 
 // ------------------------------------------------------------------------------------------
 // The attention block around the path: rotary embedding on Q and K, Nystrom Laplacian attention, + DWC(V)

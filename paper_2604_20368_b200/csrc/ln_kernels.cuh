@@ -1339,28 +1339,98 @@ __global__ void k_selftest_wait(int probes, int* dev_status) {
 // l1 kernels are held against.
 // =====================================================================================
 constexpr int kProbeChains = 8;
-__global__ void __launch_bounds__(256) k_fp32_add_probe(int iters, float* sink) {
+// mode 0: two scalar adds per chain and step; 1: one packed add; 2: the instruction mix of the sign pass (two saturating
+// multiply-adds that form a pair h, then two packed multiply-adds g h + acc into two accumulators: 6 lane-operations
+// in 4 instructions); 3: the mix of the l1 forward (one packed subtract, two scalar |.| accumulations: 4 lane-operations
+// in 3 instructions); 4: mix 2 with scalar and packed instructions in separate runs; 5: mix 2 with scalar instructions
+// only.  Lane-operations per chain and step: 2, 2, 6, 4, 6, 6.
+__global__ void __launch_bounds__(256) k_fp32_add_probe(int iters, int mode, float* sink) {
   const float x = sink[0];                       // a run-time value the compiler cannot fold
   float a[kProbeChains], b[kProbeChains];
 #pragma unroll
   for (int k = 0; k < kProbeChains; ++k) { a[k] = (float)k; b[k] = (float)(k + threadIdx.x); }
-  const int mode = iters < 0 ? 1 : 0, it = iters < 0 ? -iters : iters;
   if (mode == 0) {
 #pragma unroll 4
-    for (int i = 0; i < it; ++i)
+    for (int i = 0; i < iters; ++i)
 #pragma unroll
       for (int k = 0; k < kProbeChains; ++k) { a[k] += x; b[k] += x; }
-  } else {
+  } else if (mode == 1) {
     f32x2 v[kProbeChains];
     const f32x2 xx = pack2(x, x);
 #pragma unroll
     for (int k = 0; k < kProbeChains; ++k) v[k] = pack2(a[k], b[k]);
 #pragma unroll 4
-    for (int i = 0; i < it; ++i)
+    for (int i = 0; i < iters; ++i)
 #pragma unroll
       for (int k = 0; k < kProbeChains; ++k) v[k] = add2(v[k], xx);
 #pragma unroll
     for (int k = 0; k < kProbeChains; ++k) { a[k] = lo32(v[k]); b[k] = hi32(v[k]); }
+  } else if (mode == 2) {
+    f32x2 r[kProbeChains], c[kProbeChains];
+    const f32x2 gg = pack2(x, x + 1.f);
+#pragma unroll
+    for (int k = 0; k < kProbeChains; ++k) { r[k] = pack2(a[k], b[k]); c[k] = pack2(b[k], a[k]); }
+#pragma unroll 4
+    for (int i = 0; i < iters; ++i)
+#pragma unroll
+      for (int k = 0; k < kProbeChains; ++k) {
+        const f32x2 h = sat_fma_pair(lo32(r[k]), hi32(c[k]), x, 0.25f);     // inputs change every step: nothing can be hoisted
+        r[k] = fma2(gg, h, r[k]);
+        c[k] = fma2(gg, h, c[k]);
+      }
+#pragma unroll
+    for (int k = 0; k < kProbeChains; ++k) { a[k] = lo32(r[k]) + hi32(c[k]); b[k] = hi32(r[k]) + lo32(c[k]); }
+  } else if (mode == 4) {      // the sign-pass mix with the scalar and the packed instructions in separate runs of 16
+    f32x2 r[kProbeChains], c[kProbeChains];
+    const f32x2 gg = pack2(x, x + 1.f);
+#pragma unroll
+    for (int k = 0; k < kProbeChains; ++k) { r[k] = pack2(a[k], b[k]); c[k] = pack2(b[k], a[k]); }
+#pragma unroll 2
+    for (int i = 0; i < iters; ++i) {
+      f32x2 h[kProbeChains];
+#pragma unroll
+      for (int k = 0; k < kProbeChains; ++k) h[k] = sat_fma_pair(lo32(r[k]), hi32(c[k]), x, 0.25f);
+#pragma unroll
+      for (int k = 0; k < kProbeChains; ++k) r[k] = fma2(gg, h[k], r[k]);
+#pragma unroll
+      for (int k = 0; k < kProbeChains; ++k) c[k] = fma2(gg, h[k], c[k]);
+    }
+#pragma unroll
+    for (int k = 0; k < kProbeChains; ++k) { a[k] = lo32(r[k]) + hi32(c[k]); b[k] = hi32(r[k]) + lo32(c[k]); }
+  } else if (mode == 5) {      // the same arithmetic with scalar instructions only (two saturating and four plain multiply-adds)
+    float r0[kProbeChains], r1[kProbeChains], c0[kProbeChains], c1[kProbeChains];
+#pragma unroll
+    for (int k = 0; k < kProbeChains; ++k) { r0[k] = a[k]; r1[k] = b[k]; c0[k] = b[k]; c1[k] = a[k]; }
+    const float g0 = x, g1 = x + 1.f;
+#pragma unroll 4
+    for (int i = 0; i < iters; ++i)
+#pragma unroll
+      for (int k = 0; k < kProbeChains; ++k) {
+        const float h0 = sat_fma(r0[k], x, 0.25f), h1 = sat_fma(c1[k], x, 0.25f);
+        r0[k] = fmaf(g0, h0, r0[k]); r1[k] = fmaf(g1, h1, r1[k]);
+        c0[k] = fmaf(g0, h0, c0[k]); c1[k] = fmaf(g1, h1, c1[k]);
+      }
+#pragma unroll
+    for (int k = 0; k < kProbeChains; ++k) { a[k] = r0[k] + c1[k]; b[k] = r1[k] + c0[k]; }
+  } else {
+    const f32x2 nb = pack2(-x, -x - 1.f);
+    f32x2 q[kProbeChains];
+#pragma unroll
+    for (int k = 0; k < kProbeChains; ++k) q[k] = pack2(a[k], b[k]);
+    float acc[kProbeChains];
+#pragma unroll
+    for (int k = 0; k < kProbeChains; ++k) acc[k] = 0.f;
+#pragma unroll 4
+    for (int i = 0; i < iters; ++i)
+#pragma unroll
+      for (int k = 0; k < kProbeChains; ++k) {
+        const f32x2 t = add2(q[k], nb);
+        q[k] = t;                                                            // the operand changes every step
+        acc[k] += fabsf(lo32(t));
+        acc[k] += fabsf(hi32(t));
+      }
+#pragma unroll
+    for (int k = 0; k < kProbeChains; ++k) { a[k] = acc[k]; b[k] = lo32(q[k]); }
   }
   float t = 0.f;
 #pragma unroll

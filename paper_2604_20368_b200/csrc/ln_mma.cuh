@@ -71,17 +71,37 @@ __device__ __forceinline__ const bf16* addr_bt(const bf16* t, int ld, int k0, in
 // ldmatrix), split hi/lo; B = U from a [token][dim] bf16 tile (transposing ldmatrix), exact.
 // grid (chunks, ceil(m/64), BH); 8 warps = 4 landmark blocks of 16 x 2 halves of the dims.
 // =====================================================================================
+// The fp32 kernel tile, the bf16 token tile and the row means of a step arrive through a ring of TN_STAGES stages
+// filled by 16-byte cp.async copies issued TN_STAGES - 1 steps ahead, so that the loop never waits for global memory;
+// the fp32 tile is then centred, split into bf16 hi + lo in a second buffer and multiplied (two MMAs per product).
+constexpr int TN_KT = 32;             // tokens per step
+constexpr int TN_STAGES = 3;
+template <int D> __host__ __device__ constexpr size_t tn_mma_smem() {
+  return (size_t)TN_STAGES * (TN_KT * 64 * 4 + TN_KT * (D + 8) * 2 + TN_KT * 4) + 2 * (size_t)TN_KT * (64 + 8) * 2 + (256 / (D / 8)) * D * 4;
+}
+__device__ __forceinline__ void tn_cp16(void* dst, const void* src, bool valid) {
+  const int sz = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void tn_cp4(void* dst, const void* src, bool valid) {
+  const int sz = valid ? 4 : 0;
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(sz) : "memory");
+}
+
 template <int D>
-__global__ void __launch_bounds__(256) k_tn_mma(const float* __restrict__ E, int lde, const float* __restrict__ mu,
-                                                const bf16* __restrict__ U, float* __restrict__ part,
-                                                float* __restrict__ colsum_part, int n, int m, int rpc) {
-  constexpr int KT = 32;            // tokens per step
-  constexpr int LDE = 64 + 8, LDU = D + 8;
+__global__ void __launch_bounds__(256, 3) k_tn_mma(const float* __restrict__ E, int lde, const float* __restrict__ mu,
+                                                   const bf16* __restrict__ U, float* __restrict__ part,
+                                                   float* __restrict__ colsum_part, int n, int m, int rpc) {
+  constexpr int KT = TN_KT, LDE = 64 + 8, LDU = D + 8;
   constexpr int NT = D / 16;        // n8-tiles per warp (half of the dims)
-  __shared__ __align__(16) bf16 Ehi[KT][LDE];
-  __shared__ __align__(16) bf16 Elo[KT][LDE];
-  __shared__ __align__(16) bf16 Us[KT][LDU];
-  __shared__ float cs_part[256 / (D / 8)][D];
+  constexpr int STAGE_BYTES = KT * 64 * 4 + KT * LDU * 2 + KT * 4;
+  extern __shared__ __align__(16) unsigned char tn_smem[];
+  auto Eraw = [&](int st) { return reinterpret_cast<float*>(tn_smem + (size_t)st * STAGE_BYTES); };                       // [KT][64]
+  auto Us = [&](int st) { return reinterpret_cast<bf16*>(tn_smem + (size_t)st * STAGE_BYTES + KT * 64 * 4); };            // [KT][LDU]
+  auto Mus = [&](int st) { return reinterpret_cast<float*>(tn_smem + (size_t)st * STAGE_BYTES + KT * 64 * 4 + KT * LDU * 2); };
+  bf16* Ehi = reinterpret_cast<bf16*>(tn_smem + (size_t)TN_STAGES * STAGE_BYTES);                                         // [KT][LDE]
+  bf16* Elo = Ehi + KT * LDE;
+  float* cs_part = reinterpret_cast<float*>(Elo + KT * LDE);                                                              // [256 / (D/8)][D]
   const int chunk = blockIdx.x, l0 = blockIdx.y * 64, bh = blockIdx.z, nchunks = gridDim.x;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int wl = (warp & 3) * 16, wc = (warp >> 2) * (D / 2);
@@ -89,6 +109,7 @@ __global__ void __launch_bounds__(256) k_tn_mma(const float* __restrict__ E, int
   U += (long long)bh * n * D;
   if (mu) mu += (long long)bh * n;
   const int jbeg = chunk * rpc, jend = min(n, jbeg + rpc);
+  const int nsteps = (jend - jbeg + KT - 1) / KT;
   float acc[NT][4];
 #pragma unroll
   for (int t = 0; t < NT; ++t)
@@ -99,34 +120,52 @@ __global__ void __launch_bounds__(256) k_tn_mma(const float* __restrict__ E, int
   for (int q = 0; q < 8; ++q) cs[q] = 0.f;
   const bool want_cs = colsum_part != nullptr && blockIdx.y == 0;
 
-  for (int j0 = jbeg; j0 < jend; j0 += KT) {
-    __syncthreads();
-    {  // E tile: 32 tokens x 64 landmarks; thread = (token, 8 landmarks)
+  auto issue = [&](int step) {          // copies of step `step` into stage step % TN_STAGES (nothing if past the end)
+    if (step < nsteps) {
+      const int st = step % TN_STAGES, j0 = jbeg + step * KT;
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {     // kernel tile: 32 rows x 16 pieces of 4 floats
+        const int idx = tid + u * 256, r = idx >> 4, c4 = (idx & 15) * 4, j = j0 + r;
+        tn_cp16(Eraw(st) + r * 64 + c4, E + (long long)j * lde + l0 + c4, j < jend && l0 + c4 < lde);
+      }
+      for (int idx = tid; idx < KT * (D / 8); idx += 256) {   // token tile: 8 bf16 per piece
+        const int r = idx / (D / 8), c8 = (idx % (D / 8)) * 8, j = j0 + r;
+        tn_cp16(Us(st) + r * LDU + c8, U + (long long)j * D + c8, j < jend);
+      }
+      if (mu && tid < KT) tn_cp4(Mus(st) + tid, mu + j0 + tid, j0 + tid < jend);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+#pragma unroll
+  for (int s0 = 0; s0 < TN_STAGES - 1; ++s0) issue(s0);
+
+  for (int step = 0; step < nsteps; ++step) {
+    const int st = step % TN_STAGES, j0 = jbeg + step * KT;
+    asm volatile("cp.async.wait_group %0;" ::"n"(TN_STAGES - 2) : "memory");
+    __syncthreads();                    // stage `st` has landed for everybody; the MMAs of the previous step have read their buffers
+    issue(step + TN_STAGES - 1);        // into the stage the previous step used, which is free now
+    {  // centre and split the kernel tile: thread = (token, 8 landmarks)
       const int r = tid >> 3, cb = (tid & 7) * 8, j = j0 + r;
-      const float mj = (mu && j < jend) ? mu[j] : 0.f;
+      const float mj = (mu && j < jend) ? Mus(st)[r] : 0.f;
 #pragma unroll
       for (int k = 0; k < 8; k += 4) {
         const int l = l0 + cb + k;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (j < jend && l < m) {
-          v = ld4(E + (long long)j * lde + l);        // lde is a multiple of 4 and >= m: in bounds
-          v.x = (l < m) ? v.x - mj : 0.f;
-          v.y = (l + 1 < m) ? v.y - mj : 0.f;
-          v.z = (l + 2 < m) ? v.z - mj : 0.f;
-          v.w = (l + 3 < m) ? v.w - mj : 0.f;
-        }
+        float4 v = *reinterpret_cast<const float4*>(Eraw(st) + r * 64 + cb + k);
+        const bool in = j < jend;
+        v.x = (in && l < m) ? v.x - mj : 0.f;
+        v.y = (in && l + 1 < m) ? v.y - mj : 0.f;
+        v.z = (in && l + 2 < m) ? v.z - mj : 0.f;
+        v.w = (in && l + 3 < m) ? v.w - mj : 0.f;
         uint2 h, lo;
         split4(v, h, lo);
-        *reinterpret_cast<uint2*>(&Ehi[r][cb + k]) = h;
-        *reinterpret_cast<uint2*>(&Elo[r][cb + k]) = lo;
+        *reinterpret_cast<uint2*>(Ehi + r * LDE + cb + k) = h;
+        *reinterpret_cast<uint2*>(Elo + r * LDE + cb + k) = lo;
       }
     }
-    for (int idx = tid; idx < KT * (D / 8); idx += 256) {   // U tile, 8 bf16 (16 bytes) per thread
-      const int r = idx / (D / 8), c8 = (idx % (D / 8)) * 8, j = j0 + r;
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (j < jend) v = *reinterpret_cast<const uint4*>(U + (long long)j * D + c8);
-      *reinterpret_cast<uint4*>(&Us[r][c8]) = v;
-      if (want_cs) {
+    if (want_cs) {
+      for (int idx = tid; idx < KT * (D / 8); idx += 256) {
+        const int r = idx / (D / 8), c8 = (idx % (D / 8)) * 8;
+        const uint4 v = *reinterpret_cast<const uint4*>(Us(st) + r * LDU + c8);
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -139,12 +178,12 @@ __global__ void __launch_bounds__(256) k_tn_mma(const float* __restrict__ E, int
 #pragma unroll
     for (int k0 = 0; k0 < KT; k0 += 16) {
       uint32_t ah[4], al[4];
-      ldsm_x4_t(ah, addr_at(&Ehi[0][0], LDE, k0, wl));
-      ldsm_x4_t(al, addr_at(&Elo[0][0], LDE, k0, wl));
+      ldsm_x4_t(ah, addr_at(Ehi, LDE, k0, wl));
+      ldsm_x4_t(al, addr_at(Elo, LDE, k0, wl));
 #pragma unroll
       for (int t = 0; t < NT; t += 2) {
         uint32_t b[4];
-        ldsm_x4_t(b, addr_bt(&Us[0][0], LDU, k0, wc + t * 8));
+        ldsm_x4_t(b, addr_bt(Us(st), LDU, k0, wc + t * 8));
         mma_bf16(acc[t], ah, b[0], b[1]);
         mma_bf16(acc[t], al, b[0], b[1]);
         mma_bf16(acc[t + 1], ah, b[2], b[3]);
@@ -152,6 +191,7 @@ __global__ void __launch_bounds__(256) k_tn_mma(const float* __restrict__ E, int
       }
     }
   }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
   float* out = part + ((long long)bh * nchunks + chunk) * m * D;
   const int g = lane >> 2, t4 = lane & 3;
 #pragma unroll
@@ -166,11 +206,11 @@ __global__ void __launch_bounds__(256) k_tn_mma(const float* __restrict__ E, int
     const int grp = tid / (D / 8), c8 = (tid % (D / 8)) * 8;
     __syncthreads();
 #pragma unroll
-    for (int q = 0; q < 8; ++q) cs_part[grp][c8 + q] = cs[q];
+    for (int q = 0; q < 8; ++q) cs_part[grp * D + c8 + q] = cs[q];
     __syncthreads();
     if (tid < D) {
       float s = 0.f;
-      for (int r = 0; r < 256 / (D / 8); ++r) s += cs_part[r][tid];
+      for (int r = 0; r < 256 / (D / 8); ++r) s += cs_part[r * D + tid];
       colsum_part[((long long)bh * nchunks + chunk) * D + tid] = s;
     }
   }

@@ -62,12 +62,14 @@ __device__ __forceinline__ void s3_cp_async16(void* dst_smem, const void* src, b
 }
 __device__ __forceinline__ void s3_cp_async_wait() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
-// 4 consecutive fp32 columns of this thread's TMEM lane
-__device__ __forceinline__ void s3_tmem_ld4(uint32_t taddr, float (&v)[4]) {
-  uint32_t r0, r1, r2, r3;
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];\n\ttcgen05.wait::ld.sync.aligned;"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(taddr) : "memory");
-  v[0] = __uint_as_float(r0); v[1] = __uint_as_float(r1); v[2] = __uint_as_float(r2); v[3] = __uint_as_float(r3);
+// 4 consecutive fp32 columns of this thread's TMEM lane, in two halves: the load is issued early and its registers
+// may be used only after s3_tmem_wait4, which names them as read-write operands so that no use can be moved ahead of it.
+__device__ __forceinline__ void s3_tmem_issue4(uint32_t taddr, uint32_t (&r)[4]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void s3_tmem_wait4(uint32_t (&r)[4]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]) : : "memory");
 }
 
 // NR = column outputs (float2) per thread and round: 1 with 256 threads, 2 with 128 .. 254.
@@ -197,6 +199,17 @@ __global__ void __launch_bounds__(256, 2) k_sign3(const bf16* __restrict__ tok, 
 
   // g of round r into buffer r & 1 (this thread's token row, its 4 or 8 landmarks of the round)
   float4 apre[2];                                                    // kernel values of the round to be produced next
+  uint32_t dpre[2][4];                                               // its dA columns, on their way out of tensor memory
+  auto fetch_d = [&](int r) {
+    if constexpr (FUSED) {
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        if (u == 1 && !two_halves) continue;
+        const int l = r * S3_RL + 4 * (u == 0 ? phalf0 : 1);
+        s3_tmem_issue4(tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)l, dpre[u]);
+      }
+    }
+  };
   auto fetch_a = [&](int r) {
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
@@ -214,8 +227,8 @@ __global__ void __launch_bounds__(256, 2) k_sign3(const bf16* __restrict__ tok, 
       const int half = (u == 0 ? phalf0 : 1), l = r * S3_RL + 4 * half;
       float g[4] = {apre[u].x, apre[u].y, apre[u].z, apre[u].w};
       if constexpr (FUSED) {
-        float da[4];
-        s3_tmem_ld4(tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)l, da);
+        s3_tmem_wait4(dpre[u]);
+        float da[4] = {__uint_as_float(dpre[u][0]), __uint_as_float(dpre[u][1]), __uint_as_float(dpre[u][2]), __uint_as_float(dpre[u][3])};
         if (kap) {
 #pragma unroll
           for (int e = 0; e < 4; ++e)
@@ -233,6 +246,7 @@ __global__ void __launch_bounds__(256, 2) k_sign3(const bf16* __restrict__ tok, 
     }
   };
   fetch_a(0);
+  fetch_d(0);
   produce(0);
   if (nrounds > 1) fetch_a(1);
   s3_cp_async_wait();
@@ -256,7 +270,7 @@ __global__ void __launch_bounds__(256, 2) k_sign3(const bf16* __restrict__ tok, 
 
   for (int r = 0; r < nrounds; ++r) {
     const int buf = r & 1;
-    if (r + 1 < nrounds) fetch_sb(r + 1);
+    if (r + 1 < nrounds) { fetch_sb(r + 1); fetch_d(r + 1); }
     const float* gb = Gs + buf * (S3_RL * S3_TOK) + tt * 8;
     const float* sb = SBs + buf * (S3_RL * 2 * S3_DS) + tc * 4;
     float* cp = Cp + buf * (S3_RL * S3_TGMAX * S3_DS) + tt * S3_DS + tc * 4;
