@@ -114,7 +114,7 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   // the last wave costs little, but at least 64 tokens per chunk
   const int mblk = (p->m + 63) / 64;
   int want = (16 * kSMs + pl->BH * mblk - 1) / (pl->BH * mblk);
-  if (want > 16) want = 16;        // the per-head kernels sum the partial results serially
+  if (want > 32) want = 32;        // the per-head kernels add up the partial results (eight loads in flight per thread)
   if (want < 1) want = 1;
   int rpc = (p->n + want - 1) / want;
   if (rpc < 256) rpc = 256;
@@ -381,6 +381,14 @@ void launch_clustered(void (*kern)(KArgs...), int grid, int cl, size_t smem, cud
   cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
+// landmark pooling: one thread per (landmark, 4 channels) for small bins, a CTA per landmark for large ones
+template <typename T>
+void launch_pool(const ln_problem* p, const T* src, float* L, cudaStream_t st) {
+  const int bin_tokens = ((p->gh + p->mh - 1) / p->mh) * ((p->gw + p->mw - 1) / p->mw);
+  if (bin_tokens >= 64) LN_LAUNCH("k_pool", st, k_pool_wide<T><<<dim3(p->m, p->B * p->H), 256, 0, st>>>(src, L, geom_of(p)));
+  else LN_LAUNCH("k_pool", st, k_pool<T><<<dim3(cdiv(p->m, 256 / (p->d / 4)), p->B * p->H), 256, 0, st>>>(src, L, geom_of(p)));
+}
+
 template <typename T> constexpr int is_f32() { return std::is_same<T, float>::value ? 1 : 0; }
 
 L1Prob l1_prob(const void* A, int a_f32, float* E, float* rowsum, int na, int d, int lde, float rs_scale, double* stat = nullptr) {
@@ -421,7 +429,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   if (dev_status && clear_status) cudaMemsetAsync(dev_status, 0, sizeof(int32_t) * BH, st);   // the kernels OR their flags into it
   // landmarks (Sec. 4.2)
   if (p->lm_mode >= 1) {      // pooled keys, or pooled queries (lm_mode 2)
-    LN_LAUNCH("k_pool", st, k_pool<T><<<dim3(cdiv(m, 256 / (D / 4)), BH), 256, 0, st>>>(p->lm_mode == 1 ? K : Q, x.Lf, geom_of(p)));
+    launch_pool<T>(p, p->lm_mode == 1 ? K : Q, x.Lf, st);
   } else {
     const long long cnt = (long long)BH * m * D;
     LN_LAUNCH("k_to_f32", st, k_to_f32<T><<<cdiv(cnt, 256), 256, 0, st>>>(L, x.Lf, cnt));
@@ -1112,9 +1120,8 @@ int landmarks_pool(const ln_problem* p, const void* K, float* L, void* stream) {
   if (s != LN_OK) return s;
   if (p->lm_mode < 1 || !K || !L || !aligned16(K) || !aligned16(L)) return LN_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  dim3 grid(cdiv(p->m, 256 / (p->d / 4)), p->B * p->H);
-  if (p->dtype == LN_F32) LN_LAUNCH("k_pool", st, k_pool<float><<<grid, 256, 0, st>>>((const float*)K, L, geom_of(p)));
-  else LN_LAUNCH("k_pool", st, k_pool<bf16><<<grid, 256, 0, st>>>((const bf16*)K, L, geom_of(p)));
+  if (p->dtype == LN_F32) launch_pool<float>(p, (const float*)K, L, st);
+  else launch_pool<bf16>(p, (const bf16*)K, L, st);
   return launch_ok();
 }
 

@@ -389,6 +389,36 @@ __global__ void __launch_bounds__(256) k_pool(const T* __restrict__ K, float* __
       make_float4((float)(s0 / cnt), (float)(s1 / cnt), (float)(s2 / cnt), (float)(s3 / cnt)));
 }
 
+// The same for large bins (high-resolution grids): one CTA per (landmark, head), 256 threads = d/4 channel quads x
+// 1024/d token lanes; lane t adds the bin's tokens t, t + lanes, ... in double (exact for any order at these sizes), the
+// lanes are added in a fixed order.  With one thread per (landmark, quad) a 28 x 14 bin is a chain of 392 dependent loads.
+template <typename T>
+__global__ void __launch_bounds__(256) k_pool_wide(const T* __restrict__ K, float* __restrict__ L, PoolGeom g) {
+  __shared__ double red[256][4];
+  const int quads = g.d / 4, lanes = 256 / quads;
+  const int l = blockIdx.x, bh = blockIdx.y, qd = (int)threadIdx.x % quads, tl = (int)threadIdx.x / quads, c = qd * 4;
+  const int a = l / g.mw, bb = l % g.mw;
+  const int r0 = bin_lo(a, g.gh, g.mh), r1 = bin_hi(a, g.gh, g.mh);
+  const int c0 = bin_lo(bb, g.gw, g.mw), c1 = bin_hi(bb, g.gw, g.mw);
+  const int bw = c1 - c0, cnt = (r1 - r0) * bw;
+  const T* Kh = K + (long long)bh * g.n * g.d;
+  double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+  if (tl < lanes)
+    for (int t = tl; t < cnt; t += lanes) {
+      const int r = r0 + t / bw, q = c0 + t % bw;
+      const float4 v = ld4(Kh + (long long)(g.prefix + r * g.gw + q) * g.d + c);
+      s0 += (double)v.x; s1 += (double)v.y; s2 += (double)v.z; s3 += (double)v.w;
+    }
+  red[threadIdx.x][0] = s0; red[threadIdx.x][1] = s1; red[threadIdx.x][2] = s2; red[threadIdx.x][3] = s3;
+  __syncthreads();
+  if (tl == 0) {
+    double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
+    for (int u = 0; u < lanes; ++u) { const double* p = red[u * quads + qd]; t0 += p[0]; t1 += p[1]; t2 += p[2]; t3 += p[3]; }
+    const double n = (double)cnt;
+    st4(L + ((long long)bh * g.m + l) * g.d + c, make_float4((float)(t0 / n), (float)(t1 / n), (float)(t2 / n), (float)(t3 / n)));
+  }
+}
+
 // dK[j] = dKpart[j] (may be NULL) + sum over the bins containing token j of dL[bin] / |bin|
 // (pooling adjoint); with pool == 0 it only converts dKpart to the storage type.
 constexpr int POOL_EPT = 4;      // elements (of four dims) per thread of k_pool_bwd
