@@ -752,6 +752,17 @@ NsWs carve_ns_ws(int batch, int m, int T, void* base) {
   return w;
 }
 
+// CTAs of a thread-block cluster that share one matrix of the stand-alone Newton-Schulz entry points (64 x 64 output
+// tiles of every product are dealt out to them)
+int ns_cluster(int m) { return m > 128 ? 8 : (m > 64 ? 4 : 1); }
+void launch_ns_pinv(int batch, int m, int iters, float eps, float alpha, const float* W, const NsWs& w, float* Xh, float* X,
+                    float* resid, cudaStream_t st) {
+  const int cl = ns_cluster(m);
+  auto go = [&](auto kern) {
+    LN_LAUNCH("k_ns_pinv", st, launch_clustered(kern, batch * cl, cl, 0, st, m, iters, eps, alpha, W, w.Wr, w.P, Xh, w.hdr, X, resid));
+  };
+  if (cl == 8) go(k_ns_pinv<8>); else if (cl == 4) go(k_ns_pinv<4>); else go(k_ns_pinv<1>);
+}
 }  // namespace
 
 namespace {
@@ -1004,8 +1015,7 @@ int ns_pinv(int32_t batch, int32_t m, const float* W, int32_t iters, float ridge
   if (m > 256) return LN_ERR_UNSUPPORTED;
   if (ws_bytes < ns_pinv_workspace_bytes(batch, m, iters)) return LN_ERR_WORKSPACE;
   const NsWs w = carve_ns_ws(batch, m, iters, ws);
-  LN_LAUNCH("k_ns_pinv", static_cast<cudaStream_t>(stream), k_ns_pinv<<<batch, 256, 0, static_cast<cudaStream_t>(stream)>>>(m, iters, ridge_eps, alpha, W, w.Wr, w.P,
-                                                                  X_hist ? X_hist : w.Xh, w.hdr, X, resid));
+  launch_ns_pinv(batch, m, iters, ridge_eps, alpha, W, w, X_hist ? X_hist : w.Xh, X, resid, static_cast<cudaStream_t>(stream));
   return launch_ok();
 }
 
@@ -1017,8 +1027,15 @@ int ns_pinv_bwd(int32_t batch, int32_t m, const float* W, int32_t iters, float r
   if (m > 256) return LN_ERR_UNSUPPORTED;
   if (ws_bytes < ns_pinv_workspace_bytes(batch, m, iters)) return LN_ERR_WORKSPACE;
   const NsWs w = carve_ns_ws(batch, m, iters, ws);
-  LN_LAUNCH("k_ns_pinv_bwd", static_cast<cudaStream_t>(stream), k_ns_pinv_bwd<<<batch, 256, 0, static_cast<cudaStream_t>(stream)>>>(m, iters, ridge_eps, alpha, W, w.Wr, w.P, w.Hm,
-                                                                      w.Ga, w.Gb, w.Xh, X_hist, w.hdr, dX, dW));
+  {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int cl = ns_cluster(m);
+    auto go = [&](auto kern) {
+      LN_LAUNCH("k_ns_pinv_bwd", st, launch_clustered(kern, batch * cl, cl, 0, st, m, iters, ridge_eps, alpha, W, w.Wr, w.P, w.Hm, w.Ga, w.Gb, w.Xh,
+                                                      X_hist, w.hdr, dX, dW));
+    };
+    if (cl == 8) go(k_ns_pinv_bwd<8>); else if (cl == 4) go(k_ns_pinv_bwd<4>); else go(k_ns_pinv_bwd<1>);
+  }
   return launch_ok();
 }
 
@@ -1070,8 +1087,7 @@ int ns_pinv_static(int32_t batch, int32_t m, const float* W, int32_t iters, floa
   // Every piece of the scratch is written by the kernel before it is read, so the contents a
   // previous call left behind do not matter and nothing has to be cleared.
   const NsWs w = carve_ns_ws(batch, m, iters, scratch);
-  LN_LAUNCH("k_ns_pinv", static_cast<cudaStream_t>(stream), k_ns_pinv<<<batch, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      m, iters, ridge_eps, alpha, W, w.Wr, w.P, w.Xh, w.hdr, X, resid));
+  launch_ns_pinv(batch, m, iters, ridge_eps, alpha, W, w, w.Xh, X, resid, static_cast<cudaStream_t>(stream));
   return launch_ok();
 }
 

@@ -898,10 +898,13 @@ struct GemmSmem { float As[16][64 + 4]; float Bs[16][64 + 4]; };
 
 template <bool TRA, bool TRB>
 __device__ void cta_gemm(int M, int N, int K, const float* A, int lda, const float* Bm, int ldb,
-                         float* C, int ldc, float alpha, float beta, const float* Cin, GemmSmem& sm) {
+                         float* C, int ldc, float alpha, float beta, const float* Cin, GemmSmem& sm, int part = 0, int nparts = 1) {
+  // nparts CTAs of a cluster share the product: output tile t goes to CTA t % nparts
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  int tile = 0;
   for (int i0 = 0; i0 < M; i0 += 64)
     for (int j0 = 0; j0 < N; j0 += 64) {
+      if ((tile++) % nparts != part) continue;
       float acc[4][4];
 #pragma unroll
       for (int r = 0; r < 4; ++r)
@@ -968,10 +971,12 @@ __device__ __forceinline__ void ns_gemm(int M, int N, int K, const float* A, int
   if (TC) {
     cta_gemm_mma<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, diag, sm.t, part, nparts);
   } else {
-    cta_gemm<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, sm.f);
+    // the diagonal term is folded into the product by the CTA that owns the tile: added after its own tiles are stored
+    cta_gemm<TRA, TRB>(M, N, K, A, lda, Bm, ldb, C, ldc, alpha, beta, Cin, sm.f, part, nparts);
     if (diag != 0.f) {
-      const int lim = M < N ? M : N;
-      for (int i = threadIdx.x; i < lim; i += 256) C[(long long)i * ldc + i] += diag;
+      const int lim = M < N ? M : N, tiles_n = (N + 63) / 64;
+      for (int i = threadIdx.x; i < lim; i += 256)
+        if (((i / 64) * tiles_n + i / 64) % nparts == part) C[(long long)i * ldc + i] += diag;
       __syncthreads();
     }
   }
@@ -1120,46 +1125,55 @@ __device__ void ns_backward_tail_dev(int m, const float* Wr, const NsHdr* hdr, c
 }
 
 // ------------------------------------------------------------------ stand-alone ns_pinv / ns_pinv_bwd
+// CL CTAs of a thread-block cluster share a matrix (grid = batch * CL): every product is split by output tiles, the
+// hardware cluster barrier ends a phase.  fp32 FFMA throughout (held to 2e-5 against the oracle).
+template <int CL>
 __global__ void __launch_bounds__(256) k_ns_pinv(int m, int T, float eps, float alpha_in, const float* W,
                                                  float* Wr, float* P, float* Xh, NsHdr* hdr, float* X,
                                                  float* resid) {
   __shared__ NsSmem sm;
   __shared__ float red[2 * 256 + 8];
-  const int b = blockIdx.x;
+  const int b = blockIdx.x / CL, crank = blockIdx.x % CL;
   const long long mm = (long long)m * m;
   W += b * mm; Wr += b * mm; P += b * mm; Xh += (long long)b * (T + 1) * mm; hdr += b;
-  ns_forward_dev<false>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red);
+  ns_forward_dev<false, CL>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red, crank);
   const float* XT = Xh + (long long)T * mm;
-  if (X) for (long long e = threadIdx.x; e < mm; e += 256) X[b * mm + e] = XT[e];
+  if (X) for (long long e = crank * 256 + threadIdx.x; e < mm; e += 256 * CL) X[b * mm + e] = XT[e];
   if (resid) {
-    ns_gemm<false, false, false>(m, m, m, Wr, m, XT, m, P, m, 1.f, 0.f, nullptr, 0.f, sm);
-    float part = 0.f;
-    for (long long e = threadIdx.x; e < mm; e += 256) {
-      const int i = (int)(e / m), j = (int)(e % m);
-      const float r = (i == j ? 1.f : 0.f) - P[e];
-      part += r * r;
+    ns_gemm<false, false, false>(m, m, m, Wr, m, XT, m, P, m, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);
+    phase_sync<CL>();
+    if (crank == 0) {
+      float part = 0.f;
+      for (long long e = threadIdx.x; e < mm; e += 256) {
+        const int i = (int)(e / m), j = (int)(e % m);
+        const float r = (i == j ? 1.f : 0.f) - P[e];
+        part += r * r;
+      }
+      const float s = block_sum(part, red);
+      if (threadIdx.x == 0) resid[b] = sqrtf(s);
     }
-    const float s = block_sum(part, red);
-    if (threadIdx.x == 0) resid[b] = sqrtf(s);
   }
+  if (CL > 1) phase_sync<CL>();      // no CTA of the cluster leaves while another may still read what it wrote
 }
 
 // recompute != 0: run the forward first (Xh, hdr, Wr are scratch); else Xh is the caller's history
 // and only Wr / hdr are rebuilt from W.
+template <int CL>
 __global__ void __launch_bounds__(256) k_ns_pinv_bwd(int m, int T, float eps, float alpha_in, const float* W,
                                                      float* Wr, float* P, float* Hm, float* Ga, float* Gb,
                                                      float* Xh_scratch, const float* Xh_given, NsHdr* hdr,
                                                      const float* dX, float* dW) {
   __shared__ NsSmem sm;
   __shared__ float red[2 * 256 + 8];
-  const int b = blockIdx.x;
+  const int b = blockIdx.x / CL, crank = blockIdx.x % CL;
   const long long mm = (long long)m * m;
   W += b * mm; Wr += b * mm; P += b * mm; Hm += b * mm; Ga += b * mm; Gb += b * mm; hdr += b;
   float* Xs = Xh_scratch + (long long)b * (T + 1) * mm;
   // T = 0 when the history is given: only Wr, the norms and alpha are rebuilt
-  ns_forward_dev<false>(m, Xh_given ? 0 : T, eps, alpha_in, W, Wr, P, Xs, hdr, sm, red);
+  ns_forward_dev<false, CL>(m, Xh_given ? 0 : T, eps, alpha_in, W, Wr, P, Xs, hdr, sm, red, crank);
   const float* Xh = Xh_given ? Xh_given + (long long)b * (T + 1) * mm : Xs;
-  ns_backward_dev<false>(m, T, Wr, Xh, hdr, dX + b * mm, dW + b * mm, P, Hm, Ga, Gb, sm, red);
+  ns_backward_dev<false, CL>(m, T, Wr, Xh, hdr, dX + b * mm, dW + b * mm, P, Hm, Ga, Gb, sm, red, crank);
+  if (CL > 1) phase_sync<CL>();
 }
 
 // =====================================================================================
