@@ -243,8 +243,8 @@ def kernel_work(cfg, name):
     pairs = {"l1_CRW": 2 * n * m + m * m, "l1_CR": 2 * n * m, "l1_C": n * m, "l1_R": n * m, "l1_W": m * m}
     if name in pairs:
         return "alu", 2.0 * d * pairs[name] * BH
-    if name.startswith("sign2_") or name in ("sign_rows_dQ", "sign_cols_dLC", "sign_rows_dK", "sign_cols_dLR"):
-        full = name.startswith("sign2_")
+    if name.startswith(("sign2_", "sign3_")) or name in ("sign_rows_dQ", "sign_cols_dLC", "sign_rows_dK", "sign_cols_dLR"):
+        full = name.startswith(("sign2_", "sign3_"))
         return "alu", (3.0 if full else 2.0) * d * n * m * BH
     if name == "sign_rows_dLW":
         return "alu", 2.0 * d * m * m * BH
@@ -261,7 +261,12 @@ def kernel_work(cfg, name):
 # DRAM bytes per head and launch of the kernels that can dominate a step, from the ncu captures summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of one launch divided by the heads of the captured case;
 # traffic grows in proportion to the heads).  Keyed by (kernel, workload family).
-NCU_DRAM_BYTES_PER_HEAD = {}
+NCU_DRAM_BYTES_PER_HEAD = {
+    # profiles/sign3_l1_products_cfg5_m256_B2.md (16 heads captured)
+    ("sign3_dQ_dLC", "cfg5_m256"): (107.05e6 + 48.69e6) / 16,
+    ("sign3_dK_dLR", "cfg5_m256"): (107.16e6 + 59.26e6) / 16,
+    ("l1_CRW", "cfg5_m256"): (36.85e6 + 81.25e6 + 2.15e6) / 16,
+}
 
 
 def alu_probe(ln, dev):
