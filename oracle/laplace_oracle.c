@@ -66,7 +66,8 @@ typedef struct oracle_problem {
   double ridge_eps;
   double ns_alpha;  /* <= 0: alpha = 1/(||W||_1 ||W||_inf); > 0: used as given, no gradient through it */
   int32_t map_mode; /* 0: O = C X R V;  1: injective map of Prop. 3 applied to the rows of C */
-  int32_t lm_mode;  /* 0: landmarks given;  1: landmarks = adaptive average pooling of K;  2: of Q (Sec. 4.2 pools the query tensor in one place) */
+  int32_t lm_mode;  /* 0: landmarks given;  1: landmarks = adaptive average pooling of K;  2: of Q (Sec. 4.2 pools the query tensor in one place);
+                       3: two landmark sets as Alg. 1 prints them, Lq = pool(Q) and Lk = pool(K): C = k(Q, Lk), W = k(Lq, Lk) (not symmetric), R = k(Lq, K) */
   int32_t prefix, gh, gw, mh, mw; /* lm_mode 1: n = prefix + gh*gw, m = mh*mw */
   int32_t lm_f32;   /* 1: pooled landmarks are rounded to single precision before use (see fwd_single) */
 } oracle_problem;
@@ -369,10 +370,14 @@ void oracle_landmarks_pool_bwd(const oracle_problem* p, const double* dL, double
 /* ------------------------------------------------------------------------- */
 typedef struct head_ctx {
   double *L, *C, *R, *W, *X, *M, *Y, *Z;
+  double *Lq;   /* query-side landmarks of the two-set variant (lm_mode 3); otherwise the same array as L */
+  double *Lq_own;
 } head_ctx;
 
 static void ctx_alloc(head_ctx* x, int n, int d, int m) {
   x->L = (double*)malloc(sizeof(double) * (size_t)m * d);
+  x->Lq_own = (double*)malloc(sizeof(double) * (size_t)m * d);
+  x->Lq = x->L;
   x->C = (double*)malloc(sizeof(double) * (size_t)n * m);
   x->R = (double*)malloc(sizeof(double) * (size_t)m * n);
   x->W = (double*)malloc(sizeof(double) * (size_t)m * m);
@@ -382,14 +387,14 @@ static void ctx_alloc(head_ctx* x, int n, int d, int m) {
   x->Z = (double*)malloc(sizeof(double) * (size_t)n * m);
 }
 static void ctx_free(head_ctx* x) {
-  free(x->L); free(x->C); free(x->R); free(x->W); free(x->X); free(x->M); free(x->Y); free(x->Z);
+  free(x->L); free(x->Lq_own); free(x->C); free(x->R); free(x->W); free(x->X); free(x->M); free(x->Y); free(x->Z);
 }
 
 /* s: whitening scale of this head ([m]) or NULL for ones */
 static void fwd_single(const oracle_problem* p, const double* Q, const double* K, const double* V,
                        const double* Lin, const double* s, head_ctx* x, double* O) {
   int n = p->n, d = p->d, m = p->m;
-  if (p->lm_mode == 1 || p->lm_mode == 2) {                         /* landmarks: pooled keys (default) or pooled queries */
+  if (p->lm_mode == 1 || p->lm_mode == 2) {                         /* one landmark set: pooled keys (default) or pooled queries */
     pool_single(p, p->lm_mode == 1 ? K : Q, x->L);
     /* The gradient of the kernel holds sign(token - landmark), which is discontinuous: a pooled
        landmark that lies within rounding distance of a token decides that sign differently in
@@ -398,10 +403,17 @@ static void fwd_single(const oracle_problem* p, const double* Q, const double* K
        take the decision on the same numbers. */
     if (p->lm_f32)
       for (size_t e = 0; e < (size_t)m * d; ++e) x->L[e] = (double)(float)x->L[e];
+  } else if (p->lm_mode == 3) {                                     /* Alg. 1 as printed: sample query and key landmarks */
+    pool_single(p, K, x->L);
+    pool_single(p, Q, x->Lq_own);
+    x->Lq = x->Lq_own;
+    if (p->lm_f32)
+      for (size_t e = 0; e < (size_t)m * d; ++e) { x->L[e] = (double)(float)x->L[e]; x->Lq[e] = (double)(float)x->Lq[e]; }
   } else memcpy(x->L, Lin, sizeof(double) * (size_t)m * d);
-  l1_block(n, m, d, Q, x->L, p->lambda, x->C);                      /* Eq. 8 */
-  l1_block(m, m, d, x->L, x->L, p->lambda, x->W);                   /* Eq. 9 (ridge added inside Newton-Schulz) */
-  l1_block(m, n, d, x->L, K, p->lambda, x->R);
+  /* x->L are the key-side landmarks (the only set unless lm_mode 3), x->Lq the query-side ones (the same array otherwise) */
+  l1_block(n, m, d, Q, x->L, p->lambda, x->C);                      /* Eq. 8: C = k(Q, K~) */
+  l1_block(m, m, d, x->Lq, x->L, p->lambda, x->W);                  /* Eq. 9: W = k(Q~, K~) (ridge added inside Newton-Schulz) */
+  l1_block(m, n, d, x->Lq, K, p->lambda, x->R);                     /* k(Q~, K) */
   ns_single(m, x->W, p->ns_iters, p->ridge_eps, p->ns_alpha, x->X, NULL);   /* Alg. 2 */
   matmul(m, n, d, x->R, V, x->M);                                   /* M = R V */
   matmul(m, m, d, x->X, x->M, x->Y);                                /* Y = X M */
@@ -490,12 +502,17 @@ static void bwd_single(const oracle_problem* p, const double* Q, const double* K
 
   memset(dQ, 0, sizeof(double) * nd);
   memset(dK, 0, sizeof(double) * nd);
-  l1_block_bwd(n, m, d, Q, x.L, p->lambda, x.C, dC, dQ, dLt);     /* C = k(Q, L) */
-  l1_block_bwd(m, n, d, x.L, K, p->lambda, x.R, dR, dLt, dK);     /* R = k(L, K) */
-  l1_block_bwd(m, m, d, x.L, x.L, p->lambda, x.W, dW, dLt, dLt);  /* W = k(L, L) */
+  /* dLt: gradient of the key-side landmarks; dLqt: of the query-side ones (the same accumulator unless lm_mode 3) */
+  double* dLq_own = (double*)calloc(md, sizeof(double));
+  double* dLqt = (p->lm_mode == 3) ? dLq_own : dLt;
+  l1_block_bwd(n, m, d, Q, x.L, p->lambda, x.C, dC, dQ, dLt);      /* C = k(Q, K~) */
+  l1_block_bwd(m, n, d, x.Lq, K, p->lambda, x.R, dR, dLqt, dK);    /* R = k(Q~, K) */
+  l1_block_bwd(m, m, d, x.Lq, x.L, p->lambda, x.W, dW, dLqt, dLt); /* W = k(Q~, K~) */
   if (p->lm_mode == 1) pool_single_bwd(p, dLt, dK);
   else if (p->lm_mode == 2) pool_single_bwd(p, dLt, dQ);
+  else if (p->lm_mode == 3) { pool_single_bwd(p, dLt, dK); pool_single_bwd(p, dLqt, dQ); }
   else memcpy(dL, dLt, sizeof(double) * md);
+  free(dLq_own);
 
   free(O); free(dZ); free(dC); free(dY); free(dX); free(dM); free(dR); free(dW); free(dLt);
   ctx_free(&x);

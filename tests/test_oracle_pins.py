@@ -554,3 +554,43 @@ def test_batch_whitening_backward_finite_differences(lm_mode):
     # the variance path matters: with s held constant the query gradient is a different one
     dQc = oracle.backward(p, Q, K, V, dO, L=L, whiten=s)[0]
     assert np.linalg.norm(dQc - dQ) > 1e-3 * np.linalg.norm(dQ)
+
+
+def test_two_landmark_sets_variant_of_alg1():
+    # lm_mode 3 (Alg. 1 as printed): Lq = pool(Q), Lk = pool(K), C = k(Q, Lk), W = k(Lq, Lk), R = k(Lq, K)
+    from dataclasses import replace
+    rng = np.random.default_rng(91)
+    p3 = Problem(B=1, H=2, n=1 + 4 * 6, d=4, m=6, lam=4.0, ns_iters=3, ridge_eps=1e-6, map_mode=1, lm_mode=3,
+                 prefix=1, gh=4, gw=6, mh=2, mw=3)
+    Q, K, V, dO = (rng.standard_normal((1, 2, p3.n, p3.d)) for _ in range(4))
+    s = rng.uniform(0.5, 2.0, (2, p3.m))
+    # the blocks are what the algorithm says: checked against the stand-alone kernel and the direct Newton-Schulz loop
+    O, x = oracle.forward(p3, Q, K, V, whiten=s, want=("C", "R", "W", "X", "M", "Y", "Z"))
+    p1 = replace(p3, lm_mode=1)
+    Lk, Lq = oracle.landmarks_pool(p1, K), oracle.landmarks_pool(p1, Q)
+    for h in range(2):
+        np.testing.assert_allclose(x["C"][h], np_l1(Q[0, h], Lk[0, h], 4.0), rtol=1e-13)
+        np.testing.assert_allclose(x["W"][h], np_l1(Lq[0, h], Lk[0, h], 4.0), rtol=1e-13)
+        np.testing.assert_allclose(x["R"][h], np_l1(Lq[0, h], K[0, h], 4.0), rtol=1e-13)
+        W = x["W"][h] + 1e-6 * np.eye(6)
+        assert np.abs(W - W.T).max() > 1e-3                         # a genuinely non-symmetric W
+        X = W.T / (np.abs(W).sum(0).max() * np.abs(W).sum(1).max())
+        for _ in range(3):
+            X = X @ (2 * np.eye(6) - W @ X)
+        np.testing.assert_allclose(x["X"][h], X, rtol=1e-11)
+        np.testing.assert_allclose(O[0, h], x["Z"][h] @ (X @ (x["R"][h] @ V[0, h])), rtol=1e-10)
+    # with Q == K the two sets coincide and the variant is the one-set path
+    np.testing.assert_allclose(oracle.forward(p3, K, K, V, whiten=s), oracle.forward(p1, K, K, V, whiten=s), rtol=1e-13)
+    # backward by central differences
+    dQ, dK, dV, dL = oracle.backward(p3, Q, K, V, dO, whiten=s)
+    assert dL is None
+    loss = lambda q, k, v: float((oracle.forward(p3, q, k, v, whiten=s) * dO).sum())
+    h_ = 1e-6
+    for name, arr, grad in (("Q", Q, dQ), ("K", K, dK), ("V", V, dV)):
+        for idx in [(0, 0, 0, 1), (0, 1, 7, 2), (0, 0, 24, 3)]:
+            a = {"Q": Q, "K": K, "V": V}
+            plus, minus = dict(a), dict(a)
+            plus[name] = arr.copy(); plus[name][idx] += h_
+            minus[name] = arr.copy(); minus[name][idx] -= h_
+            fd = (loss(plus["Q"], plus["K"], plus["V"]) - loss(minus["Q"], minus["K"], minus["V"])) / (2 * h_)
+            assert grad[idx] == pytest.approx(fd, rel=5e-6, abs=1e-8), (name, idx)
