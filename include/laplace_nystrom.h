@@ -61,7 +61,11 @@ typedef struct ln_problem {
   const float* whiten;    /* device [H,m] fp32 whitening scale s (Eq. 6), or NULL = ones; a constant      */
   int32_t lm_mode;        /* 0: landmarks L given by the caller;  1: L = adaptive average pooling of K;   */
                           /* 2: of Q (Sec. 4.2 pools the query tensor in one place): dL then returns to dQ */
-  int32_t prefix, gh, gw, mh, mw; /* lm_mode 1, 2: n = prefix + gh*gw, m = mh*mw.  Bin (a,b) averages grid  */
+                          /* 3: two landmark sets, as Alg. 1 prints them: Lq = pool(Q), Lk = pool(K),      */
+                          /*    C = k(Q,Lk), W = k(Lq,Lk) + eps I (not symmetric), R = k(Lq,K); dLq, dLk   */
+                          /*    return to dQ, dK.  The per-head iteration then runs on the general engine */
+                          /*    (mma.sync / FFMA, not tcgen05); whiten_mode 1 is LN_ERR_UNSUPPORTED.       */
+  int32_t prefix, gh, gw, mh, mw; /* lm_mode >= 1: n = prefix + gh*gw, m = mh*mw.  Bin (a,b) averages grid  */
                           /* rows floor(a*gh/mh) .. ceil((a+1)*gh/mh)-1 and columns likewise; the first   */
                           /* `prefix` tokens (class tokens) are ordinary queries/keys but are not pooled. */
   int32_t whiten_mode;    /* 0: `whiten` is a constant input (or NULL = ones).  1: batch statistics (Eq. 5-6 in     */
@@ -108,8 +112,8 @@ int laplace_nystrom_fwd(const ln_problem* p, const void* Q, const void* K, const
  * gradient -(1/lambda) sign(x - y) k, with sign(0) = 0).
  *   dO [B,H,n,d] dtype;  saved: the buffer the matching fwd filled;
  *   dQ,dK,dV [B,H,n,d] dtype, overwritten;
- *   dL [B,H,m,d] dtype: required when lm_mode == 0; must be NULL when lm_mode is 1 or 2 (the
- *   landmark gradient is folded into dK, or dQ, through the pooling adjoint).
+ *   dL [B,H,m,d] dtype: required when lm_mode == 0; must be NULL when lm_mode is 1, 2 or 3 (the
+ *   landmark gradient is folded into dK, dQ, or both, through the pooling adjoint).
  *   ws: laplace_nystrom_workspace_bytes(p, 1) bytes.
  *   dev_status: as for laplace_nystrom_fwd (only bit 1 can be set by the backward pass).
  */
@@ -259,7 +263,8 @@ int landmarks_pool_bwd(const ln_problem* p, const float* dL, void* dK, void* str
  * Where an fp32 intermediate of the forward pass lies inside `saved` (the paper has no counterpart: an inspection
  * aid, used by the parity tests to compare intermediates with the oracle's).  name: "L" landmarks [m x d],
  * "C" = k(Q,L) [n x m], "Rt" = k(K,L) [n x m], "mu" row means of C [1 x n], "W" = k(L,L) [m x m] (before the
- * ridge), "X" = X_T [m x m], "M" = R V [m x d], "Yt" folded Y [m x d], "ybar" [1 x d].
+ * ridge), "X" = X_T [m x m], "M" = R V [m x d], "Yt" folded Y [m x d], "ybar" [1 x d];
+ * lm_mode 3 only: "Lq" pooled queries [m x d] ("L" is then the pooled keys, "Rt" = k(K,Lq), "W" = k(Lq,L)).
  * info[0] = offset of head 0 in floats from the start of saved, info[1] = rows, info[2] = columns,
  * info[3] = leading dimension, info[4] = floats between consecutive heads.  LN_ERR_ARG for an unknown name.
  */

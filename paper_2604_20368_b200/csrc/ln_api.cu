@@ -96,6 +96,7 @@ struct Plan {
   size_t s2_smem;
   int s3_tiles;                      // sign pass with the upstream factor formed in the kernel: token tiles per head (0 = not used)
   int H, wmode, l1_tiles;            // heads; whitening mode; token tiles of the l1 launch that forms C (statistics partials)
+  bool two;                          // two landmark sets (Alg. 1 as printed): W = k(pool(Q), pool(K)) is not symmetric
 };
 
 bool make_plan(const ln_problem* p, Plan* pl) {
@@ -104,12 +105,15 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   pl->BH = p->B * p->H; pl->n = p->n; pl->d = p->d; pl->m = p->m; pl->T = p->ns_iters;
   pl->ldm = (p->m + 3) & ~3;
   pl->scr = (size_t)p->m * pl->ldm;
-  if (p->dtype == LN_BF16 && p->m > 128) pl->scr = (size_t)kU2Slot;
+  pl->two = p->lm_mode == 3;
+  // the tcgen05 per-head kernels use the symmetry of the landmark kernel matrix; two landmark sets take the general engine
+  const bool tcmid = p->dtype == LN_BF16 && !pl->two;
+  if (tcmid && p->m > 128) pl->scr = (size_t)kU2Slot;
   // history slots: fp32 [m][ldm], except on the m <= 64 tensor-core path, whose slots hold operand images
   pl->hslot = (long long)p->m * pl->ldm;
-  if (p->dtype == LN_BF16 && p->m <= 64) pl->hslot = (long long)(kUmmaMatBytes64 / 4);                 // 16 KiB images >= m * ldm * 4
-  if (p->dtype == LN_BF16 && p->m > 64 && p->m <= 128) pl->hslot = (long long)(kUmmaMatBytes / 4);     // 64 KiB images >= m * ldm * 4
-  if (p->dtype == LN_BF16 && p->m > 128) pl->hslot = kU2Slot;                                          // four 64 KiB block images
+  if (tcmid && p->m <= 64) pl->hslot = (long long)(kUmmaMatBytes64 / 4);                 // 16 KiB images >= m * ldm * 4
+  if (tcmid && p->m > 64 && p->m <= 128) pl->hslot = (long long)(kUmmaMatBytes / 4);     // 64 KiB images >= m * ldm * 4
+  if (tcmid && p->m > 128) pl->hslot = kU2Slot;                                          // four 64 KiB block images
   // token chunks per head for the reductions over tokens: about eight waves of CTAs (two per SM) so that
   // the last wave costs little, but at least 64 tokens per chunk
   const int mblk = (p->m + 63) / 64;
@@ -156,6 +160,7 @@ bool make_plan(const ln_problem* p, Plan* pl) {
     const int tpq = tiles_per_chunk(2 * kSMs - lost);
     pl->s2q_rpc = tpq * 8 * TG; pl->s2q_chunks = (p->n + pl->s2q_rpc - 1) / pl->s2q_rpc;
     pl->s2_smem = sign2_smem_bytes(p->m);
+    if (pl->two) pl->s2_chunks = pl->s2q_chunks = 0;      // two landmark sets: the tcgen05 sign pass or the two plain passes
   }
   // bf16 storage, 64 or 128 dims: one CTA per tile of 8 * TG tokens, upstream factor on the tensor cores in the kernel
   pl->H = p->H; pl->wmode = p->whiten_mode;
@@ -169,7 +174,7 @@ bool make_plan(const ln_problem* p, Plan* pl) {
 size_t image_floats(const Plan& pl) { return (size_t)((pl.m + GU_KB - 1) / GU_KB) * gu_block_floats(pl.d); }
 
 // Forward context (saved for the backward pass, or carved from ws for inference)
-struct Ctx { float *Lf, *C, *Rt, *mu, *W, *Xh, *Ph, *M, *Yt, *ybar, *Yimg, *Y, *cbar; NsHdr* hdr; size_t bytes; };
+struct Ctx { float *Lf, *C, *Rt, *mu, *W, *Xh, *Ph, *M, *Yt, *ybar, *Yimg, *Y, *cbar, *Lq; NsHdr* hdr; size_t bytes; };
 Ctx carve_ctx(const Plan& pl, void* base) {
   Carver c(base); Ctx x;
   const size_t BH = pl.BH, n = pl.n, d = pl.d, m = pl.m;
@@ -187,6 +192,7 @@ Ctx carve_ctx(const Plan& pl, void* base) {
   x.hdr = reinterpret_cast<NsHdr*>(c.take(BH * (sizeof(NsHdr) / sizeof(float))));
   x.Y = c.take(BH * m * d);                      // Y = X M before the map is folded in (batch-statistic whitening needs it)
   x.cbar = c.take((size_t)pl.H * m);             // column means of C over the batch (batch-statistic whitening)
+  x.Lq = c.take(pl.two ? BH * m * d : 0);        // second landmark set (pooled queries); Lf then holds the pooled keys
   x.bytes = c.off;
   return x;
 }
@@ -204,7 +210,7 @@ FwdWs carve_fwd_ws(const Plan& pl, void* base) {
 }
 
 struct BwdWs {
-  float *G, *G2, *dYtpart, *dybpart, *dLCpart, *dLRpart, *dY, *dM, *Wr, *P, *Hm, *Ga, *Gb, *dW, *dX, *GW, *dLW, *dLtot, *dKpart, *dMimg, *SB, *kap;
+  float *G, *G2, *dYtpart, *dybpart, *dLCpart, *dLRpart, *dY, *dM, *Wr, *P, *Hm, *Ga, *Gb, *dW, *dX, *GW, *dLW, *dLtot, *dKpart, *dMimg, *SB, *kap, *SBq, *dQpart, *dLqtot, *dLW2;
   size_t bytes;
 };
 BwdWs carve_bwd_ws(const Plan& pl, void* base) {
@@ -236,6 +242,12 @@ BwdWs carve_bwd_ws(const Plan& pl, void* base) {
   w.dMimg = c.take(BH * image_floats(pl));
   w.SB = c.take(pl.s3_tiles > 0 ? BH * m * 2 * d : 0);      // scale and offset of every landmark value (folded step)
   w.kap = c.take(pl.wmode == 1 ? (size_t)pl.H * m * 2 : 0); // batch-statistic whitening: (kappa_l, cbar_l) per head and landmark
+  // two landmark sets: folded step of the second set, fp32 query gradient before the pooling adjoint, gradient of the
+  // second set, column part of the landmark-block sign pass
+  w.SBq = c.take(pl.two && pl.s3_tiles > 0 ? BH * m * 2 * d : 0);
+  w.dQpart = c.take(pl.two ? BH * n * d : 0);
+  w.dLqtot = c.take(pl.two ? BH * m * d : 0);
+  w.dLW2 = c.take(pl.two ? BH * m * d : 0);
   w.bytes = c.off;
   return w;
 }
@@ -250,12 +262,13 @@ int validate(const ln_problem* p) {
   if (!isfinite(p->ns_alpha)) return LN_ERR_ARG;
   if (p->dtype != LN_F32 && p->dtype != LN_BF16) return LN_ERR_ARG;
   if (p->map_mode != 0 && p->map_mode != 1) return LN_ERR_ARG;
-  if (p->lm_mode < 0 || p->lm_mode > 2) return LN_ERR_ARG;
+  if (p->lm_mode < 0 || p->lm_mode > 3) return LN_ERR_ARG;
   if (p->whiten && !aligned16(p->whiten)) return LN_ERR_ARG;
   if (p->whiten_mode != 0 && p->whiten_mode != 1) return LN_ERR_ARG;
   if (p->whiten_mode == 1) {
     if (p->map_mode != 1 || p->whiten || !p->whiten_batch || !aligned16(p->whiten_batch)) return LN_ERR_ARG;
     if (!(p->whiten_eps >= 0.f) || !isfinite(p->whiten_eps)) return LN_ERR_ARG;
+    if (p->lm_mode == 3) return LN_ERR_UNSUPPORTED;
   }
   if (p->lm_mode >= 1) {
     if (p->prefix < 0 || p->gh <= 0 || p->gw <= 0 || p->mh <= 0 || p->mw <= 0) return LN_ERR_ARG;
@@ -428,7 +441,11 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const int BH = pl.BH, n = pl.n, m = pl.m, kSMs = sm_count();
   if (dev_status && clear_status) cudaMemsetAsync(dev_status, 0, sizeof(int32_t) * BH, st);   // the kernels OR their flags into it
   // landmarks (Sec. 4.2)
-  if (p->lm_mode >= 1) {      // pooled keys, or pooled queries (lm_mode 2)
+  const bool two = pl.two;    // two landmark sets: Lf = pooled keys (columns of C and W), Lq = pooled queries (rows of W, columns of R^T)
+  if (two) {
+    launch_pool<T>(p, K, x.Lf, st);
+    launch_pool<T>(p, Q, x.Lq, st);
+  } else if (p->lm_mode >= 1) {      // pooled keys, or pooled queries (lm_mode 2)
     launch_pool<T>(p, p->lm_mode == 1 ? K : Q, x.Lf, st);
   } else {
     const long long cnt = (long long)BH * m * D;
@@ -437,7 +454,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // the three kernel blocks: C = k(Q,L) with its row sums, R^T = k(K,L), W = k(L,L)
   // (not for many small heads, where the per-head kernel fills the GPU and the split launches cost more than the
   // overlap returns)
-  const Side side = side_acquire(std::is_same<T, bf16>::value && (2 * pl.mid_sms <= kSMs || (long long)n * m * D > (1ll << 22)), st);
+  const Side side = side_acquire(!two && std::is_same<T, bf16>::value && (2 * pl.mid_sms <= kSMs || (long long)n * m * D > (1ll << 22)), st);
   const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);   // tcgen05 products over the landmarks
   // Where the iteration is expected to outlast the two token-sized blocks (few heads of few tokens), only the iteration
   // goes to the side stream; estimates in microseconds: 5 / 12 / 100 per step for m <= 64 / <= 128 / larger, and the l1
@@ -459,7 +476,8 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
                                  whiten_eff, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, Mparts_src, Mparts, x.M, x.Y, x.Yt,
                                  x.ybar, dev_status, pl.hslot, umma_prod ? reinterpret_cast<bf16*>(x.Yimg) : nullptr, phase));
     };
-    if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * kUmmaMatBytes64);
+    if (two) launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));          // general (non-symmetric) matrix: mma.sync or FFMA engine
+    else if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * kUmmaMatBytes64);
     else if (TC && m <= 128) launch(k_mid_fwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
     else if (TC) launch(k_mid_fwd<D, TC, TC ? 256 : 0, TC ? kMidCluster : 1>, 3 * kUmmaMatBytes, kMidCluster);   // m > 128: a cluster per head
     else launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));
@@ -471,8 +489,15 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     const L1Prob pc = l1_prob(Q, is_f32<T>(), x.C, p->map_mode == 1 ? x.mu : nullptr, n, D, pl.ldm, 1.f / (float)m,  // row means (Prop. 3 step 2)
                               bw ? w.stat : nullptr);                                                                    // column statistics (Eq. 5)
     const L1Prob pr = l1_prob(K, is_f32<T>(), x.Rt, nullptr, n, D, pl.ldm, 1.f);
-    const L1Prob pw = l1_prob(x.Lf, 1, x.W, nullptr, m, D, m, 1.f);
-    if (side.on()) {
+    const L1Prob pw = l1_prob(two ? x.Lq : x.Lf, 1, x.W, nullptr, m, D, m, 1.f);
+    if (two) {
+      // C = k(Q, pool K) and W = k(pool Q, pool K) share their landmark operand; R^T = k(K, pool Q) has its own
+      a.p[0] = pc; a.p[1] = pw; a.p[2] = pw;
+      launch_l1_args("l1_CW", a, 2, BH, st);
+      a.Bm = x.Lq;
+      a.p[0] = pr; a.p[1] = pr; a.p[2] = pr;
+      launch_l1_args("l1_R", a, 1, BH, st);
+    } else if (side.on()) {
       // W first: the iteration on it runs beside the token-sized blocks.  Then R^T: M = R V (bound by memory) and the
       // rest of the per-head work run beside the query block C (bound by arithmetic), which only the last product needs.
       a.p[0] = pw; a.p[1] = pw; a.p[2] = pw;
@@ -561,6 +586,12 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   };
   const bool fused_sign = pl.s2_chunks > 0;
   const bool poolQ = p->lm_mode == 2;                 // the token-side gradient that still needs the pooling adjoint is dQ, not dK
+  const bool two = pl.two;                            // two landmark sets: both token-side gradients need a pooling adjoint
+  const float* const LfC = x.Lf;                      // landmarks of the query-side block C (pooled keys when two)
+  const float* const LfR = two ? x.Lq : x.Lf;         // landmarks of the key-side block R^T (pooled queries when two)
+  // fp32 row outputs of the sign passes that a pooling adjoint still follows (NULL: the pass writes the gradient itself)
+  float* const qrows_f = two ? w.dQpart : (poolQ ? w.dKpart : nullptr);
+  float* const krows_f = (two || !poolQ) ? w.dKpart : nullptr;
   const bool sign3 = pl.s3_tiles > 0;                 // the sign passes form their upstream factor themselves (tcgen05)
   const int chs = sign3 ? pl.s3_tiles : (fused_sign ? pl.s2_chunks : ch);
   const int chq = sign3 ? pl.s3_tiles : (fused_sign ? pl.s2q_chunks : ch);    // chunks of the query-side landmark-gradient partials
@@ -568,12 +599,12 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   const bool bw = p->whiten_mode == 1;                // batch-statistic whitening: the scale is the forward pass's own estimate
   const float* const whiten_eff = bw ? p->whiten_batch : p->whiten;
   auto launch_sign3 = [&](const char* name, const T* tokp, const T* Up, const float* Yimgp, const float* Ap, auto* rowsp, float* partp,
-                          const float* kap = nullptr) {
+                          const float* SBp, const float* kap = nullptr) {
     if constexpr (std::is_same<T, bf16>::value && (D == 64 || D == 128)) {
       auto go = [&](auto kern) {
         want_smem(kern, sign3_smem_bytes());
         LN_LAUNCH(name, st, kern<<<dim3(pl.s3_tiles, D / 64, BH), dim3(16, pl.s2_tg), sign3_smem_bytes(), st>>>(
-                      tokp, w.SB, Up, reinterpret_cast<const bf16*>(Yimgp), Ap, pl.ldm, rowsp, partp, n, m, inv_lambda, dev_status, kap, p->H));
+                      tokp, SBp, Up, reinterpret_cast<const bf16*>(Yimgp), Ap, pl.ldm, rowsp, partp, n, m, inv_lambda, dev_status, kap, p->H));
       };
       using TO = std::remove_pointer_t<decltype(rowsp)>;
       if (pl.s2_tg == S3_TGMAX) go(k_sign3<TO, D, 1, true>); else go(k_sign3<TO, D, 2, true>);
@@ -581,7 +612,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   };
   // The per-head kernel and the landmark-block sign pass need Z'^T dO only: with a side stream they run beside
   // the query-side kernels and are joined before the key side, which needs dM.
-  const Side side = side_acquire(std::is_same<T, bf16>::value, st);
+  const Side side = side_acquire(!two && std::is_same<T, bf16>::value, st);
   const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);
   auto launch_mid = [&](cudaStream_t s) {
     constexpr bool TC = std::is_same<T, bf16>::value;
@@ -590,9 +621,10 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
       LN_LAUNCH("k_mid_bwd", s, launch_clustered(kern, BH * cl, cl, smem, s, m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, whiten_eff,
                                                  x.W, x.Xh, x.Ph, x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P,
                                                  w.Hm, w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot,
-                                                 umma_prod ? reinterpret_cast<bf16*>(w.dMimg) : nullptr));
+                                                 umma_prod ? reinterpret_cast<bf16*>(w.dMimg) : nullptr, two ? 0 : 1));
     };
-    if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 4 * kUmmaMatBytes64);
+    if (two) launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
+    else if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 4 * kUmmaMatBytes64);
     else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
     else if (TC) launch(k_mid_bwd<D, TC, TC ? 256 : 0, TC ? kMidCluster : 1>, 3 * kUmmaMatBytes, kMidCluster);
     else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
@@ -624,7 +656,9 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     }
   };
   auto launch_sign_W = [&](cudaStream_t s) {
-    LN_LAUNCH("sign_rows_dLW", s, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, s>>>(x.Lf, x.Lf, w.GW, pl.ldm, w.dLW, m, m));
+    // one set: GW is symmetrised, so the row pass carries both roles of L.  Two sets: rows -> pooled queries, columns -> pooled keys
+    LN_LAUNCH("sign_rows_dLW", s, k_sign_rows<float, float, float, D><<<dim3(cdiv(m, 64), BH), 256, 0, s>>>(LfR, LfC, w.GW, pl.ldm, w.dLW, m, m));
+    if (two) LN_LAUNCH("sign_cols_dLW", s, k_sign_cols<float, float, D><<<dim3(1, cdiv(m, 64), BH), 256, 0, s>>>(LfR, LfC, w.GW, pl.ldm, w.dLW2, m, m, (m + 31) / 32 * 32));
   };
   // Side stream: the per-head kernel, the landmark-block sign pass and dV (bound by latency and by memory) run beside
   // the sign passes (bound by arithmetic).  The upstream of the key-side block, which the second sign pass waits for,
@@ -656,9 +690,10 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   }
   if (sign3) {
     const long long cnt = (long long)BH * m * D;
-    LN_LAUNCH("k_fold_landmarks", st, k_fold_landmarks<<<cdiv(cnt, 256), 256, 0, st>>>(x.Lf, w.SB, D, cnt));
-    if (poolQ) launch_sign3("sign3_dQ_dLC", Q, dO, x.Yimg, x.C, w.dKpart, w.dLCpart, kap);
-    else launch_sign3("sign3_dQ_dLC", Q, dO, x.Yimg, x.C, dQ, w.dLCpart, kap);
+    LN_LAUNCH("k_fold_landmarks", st, k_fold_landmarks<<<cdiv(cnt, 256), 256, 0, st>>>(LfC, w.SB, D, cnt));
+    if (two) LN_LAUNCH("k_fold_landmarks", st, k_fold_landmarks<<<cdiv(cnt, 256), 256, 0, st>>>(LfR, w.SBq, D, cnt));
+    if (qrows_f) launch_sign3("sign3_dQ_dLC", Q, dO, x.Yimg, x.C, qrows_f, w.dLCpart, w.SB, kap);
+    else launch_sign3("sign3_dQ_dLC", Q, dO, x.Yimg, x.C, dQ, w.dLCpart, w.SB, kap);
   } else {
     launch_ntg_C();
     if (bw) LN_LAUNCH("k_g_whiten_add", st, k_g_whiten_add<<<dim3(cdiv((long long)n * pl.ldm, 256), BH), 256, 0, st>>>(w.G, x.C, w.kap, p->H, n, m, pl.ldm, inv_lambda));
@@ -677,16 +712,16 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
       else launch2("sign2_dQ_dLC", k_sign2<T, T, 2>, Q, dQ, w.dLCpart);
     }
   } else {
-    if (poolQ) LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dKpart, n, m));
-    else LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, dQ, n, m));
-    LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, x.Lf, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
+    if (qrows_f) LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, LfC, w.G, pl.ldm, qrows_f, n, m));
+    else LN_LAUNCH("sign_rows_dQ", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(Q, LfC, w.G, pl.ldm, dQ, n, m));
+    LN_LAUNCH("sign_cols_dLC", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(Q, LfC, w.G, pl.ldm, w.dLCpart, n, m, pl.rpc));
   }
   if (side.on()) { side.join_mark(st); if (!ntg_on_side && !sign3) launch_ntg_R(st); }
   else { launch_mid(st); launch_sign_W(st); if (!sign3) launch_ntg_R(st); launch_nn_dV(st); }
   // key side: dK (kernel part); landmark part
   if (sign3) {
-    if (poolQ) launch_sign3("sign3_dK_dLR", K, V, w.dMimg, x.Rt, dK, w.dLRpart);
-    else launch_sign3("sign3_dK_dLR", K, V, w.dMimg, x.Rt, w.dKpart, w.dLRpart);
+    if (!krows_f) launch_sign3("sign3_dK_dLR", K, V, w.dMimg, x.Rt, dK, w.dLRpart, two ? w.SBq : w.SB);
+    else launch_sign3("sign3_dK_dLR", K, V, w.dMimg, x.Rt, krows_f, w.dLRpart, two ? w.SBq : w.SB);
   } else if (fused_sign) {
     auto launch2 = [&](const char* name, auto kern, const T* tokp, auto* rowsp, float* partp) {
       want_smem(kern, pl.s2_smem);
@@ -700,14 +735,19 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
       else launch2("sign2_dK_dLR", k_sign2<T, float, 2>, K, w.dKpart, w.dLRpart);
     }
   } else {
-    if (poolQ) LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G2, pl.ldm, dK, n, m));
-    else LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, x.Lf, w.G2, pl.ldm, w.dKpart, n, m));
-    LN_LAUNCH("sign_cols_dLR", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(K, x.Lf, w.G2, pl.ldm, w.dLRpart, n, m, pl.rpc));
+    if (!krows_f) LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, T, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, LfR, w.G2, pl.ldm, dK, n, m));
+    else LN_LAUNCH("sign_rows_dK", st, k_sign_rows<T, float, float, D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(K, LfR, w.G2, pl.ldm, krows_f, n, m));
+    LN_LAUNCH("sign_cols_dLR", st, k_sign_cols<T, float, D><<<dim3(ch, cdiv(m, 64), BH), 256, 0, st>>>(K, LfR, w.G2, pl.ldm, w.dLRpart, n, m, pl.rpc));
   }
   // landmark gradient and its way back to the keys
   if (side.on()) side.join(st);      // dV and the landmark-block part are complete
   const int md = m * D;
-  if (p->lm_mode >= 1) {      // the landmark gradient returns to the pooled tensor (keys, or queries for lm_mode 2)
+  if (two) {                  // pooled keys: columns of C and of W; pooled queries: columns of R^T and rows of W
+    LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLW2, 1, nullptr, 0, w.dLtot, md));
+    LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLRpart, chs, w.dLW, 1, nullptr, 0, w.dLqtot, md));
+    LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, w.dLtot, dK, geom_of(p), 1));
+    LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dQpart, w.dLqtot, dQ, geom_of(p), 1));
+  } else if (p->lm_mode >= 1) {      // the landmark gradient returns to the pooled tensor (keys, or queries for lm_mode 2)
     LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, w.dLtot, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, w.dLtot, poolQ ? dQ : dK, geom_of(p), 1));
   } else {
@@ -1158,16 +1198,18 @@ int laplace_nystrom_saved_array(const ln_problem* p, const char* name, int64_t i
   const Ctx x = carve_ctx(pl, reinterpret_cast<void*>(256));      // offsets relative to a fictitious base
   auto off = [](const void* q) { return (int64_t)((reinterpret_cast<uintptr_t>(q) - 256) / sizeof(float)); };
   const int64_t n = p->n, d = p->d, m = p->m, ldm = pl.ldm;
-  const bool img = p->dtype == LN_BF16;                            // tensor-core paths: history slots are operand images
+  const bool img = p->dtype == LN_BF16 && !pl.two;                 // tcgen05 paths: history slots are operand images
   const int64_t ldx = (img && m <= 128) ? ldm : m;
   const int64_t mx = img ? pl.hslot : m * ldx;
   struct { const char* nm; const void* ptr; int64_t rows, cols, ld, stride; } t[] = {
     {"L", x.Lf, m, d, d, m * d}, {"C", x.C, n, m, ldm, n * ldm}, {"Rt", x.Rt, n, m, ldm, n * ldm},
     {"mu", x.mu, 1, n, n, n}, {"W", x.W, m, m, m, m * m},
     {"X", x.Xh + (size_t)pl.T * mx, m, m, ldx, (int64_t)(pl.T + 1) * mx},
-    {"M", x.M, m, d, d, m * d}, {"Yt", x.Yt, m, d, d, m * d}, {"ybar", x.ybar, 1, d, d, d}};
+    {"M", x.M, m, d, d, m * d}, {"Yt", x.Yt, m, d, d, m * d}, {"ybar", x.ybar, 1, d, d, d},
+    {"Lq", x.Lq, m, d, d, m * d}};
   for (auto& e : t)
     if (strcmp(name, e.nm) == 0) {
+      if (e.ptr == x.Lq && !pl.two) return LN_ERR_ARG;
       info[0] = off(e.ptr); info[1] = e.rows; info[2] = e.cols; info[3] = e.ld; info[4] = e.stride;
       return LN_OK;
     }

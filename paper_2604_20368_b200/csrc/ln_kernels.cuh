@@ -1285,7 +1285,9 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
                                                  const float* dYtpart, const float* dybpart, int nchunks,
                                                  float eps, float* Wr, float* P, float* Hm, float* Ga, float* Gb,
                                                  float* dWm, float* dXm, float* dY, float* dM, float* GW, int* dev_status,
-                                                 long long hslot, bf16* dMimg) {
+                                                 long long hslot, bf16* dMimg, int sym) {
+  // sym: 1 = one landmark set (W = k(L, L): the gradient of both roles of L is carried by the symmetrised factor);
+  // 0 = two landmark sets, GW = dW o W / lambda as it is (MP == 0 only)
   extern __shared__ __align__(16) unsigned char dyn_smem[];
   NsSmem& sm = *reinterpret_cast<NsSmem*>(dyn_smem);
   __shared__ float red[2 * 256 + 8];
@@ -1354,7 +1356,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
       const int i = (int)(e / ldm), j = (int)(e % ldm);
       const bool in = j < m;
       a[u] = in ? dWm[(long long)i * ldx + j] : 0.f;  b[u] = in ? W[(long long)i * m + j] : 0.f;
-      c[u] = in ? dWm[(long long)j * ldx + i] : 0.f;  d4[u] = in ? W[(long long)j * m + i] : 0.f;
+      c[u] = (in && sym) ? dWm[(long long)j * ldx + i] : 0.f;  d4[u] = (in && sym) ? W[(long long)j * m + i] : 0.f;
     }
     *reinterpret_cast<float4*>(GW + e0) = make_float4((a[0] * b[0] + c[0] * d4[0]) * inv_lambda, (a[1] * b[1] + c[1] * d4[1]) * inv_lambda,
                                                       (a[2] * b[2] + c[2] * d4[2]) * inv_lambda, (a[3] * b[3] + c[3] * d4[3]) * inv_lambda);

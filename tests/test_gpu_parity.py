@@ -266,20 +266,31 @@ def test_given_landmarks_and_their_gradient(dtype):
         assert rel_err(f64(got), ref) < TOL[dtype], name
 
 
-@pytest.mark.parametrize("name,B,H", [("cfg2", 2, 2), ("cfg1", 1, 2), ("cfg5_m128_T8", 1, 1), ("cfg4a", 1, 1)])
-def test_landmarks_pooled_from_queries(name, B, H):
-    """lm_mode 2 (Sec. 4.2 pools the query tensor): L = pool(Q); the landmark gradient returns to dQ."""
+@pytest.mark.parametrize("lm_mode,name,B,H,fused", [
+    (2, "cfg2", 2, 2, True), (2, "cfg1", 1, 2, True), (2, "cfg5_m128_T8", 1, 1, True), (2, "cfg4a", 1, 1, True),
+    (3, "cfg2", 2, 2, True), (3, "cfg2", 1, 2, False), (3, "cfg1", 1, 2, True), (3, "cfg3", 1, 2, True),
+    (3, "cfg5_m128_T8", 1, 1, True), (3, "cfg4a", 1, 1, True), (3, "cfg5_m256_T4", 1, 1, True)])
+def test_landmarks_pooled_from_queries(lm_mode, name, B, H, fused):
+    """lm_mode 2 (Sec. 4.2 pools the query tensor): L = pool(Q); the landmark gradient returns to dQ.
+    lm_mode 3 (Alg. 1 as printed): two landmark sets, C = k(Q, pool K), W = k(pool Q, pool K), R = k(pool Q, K); W is
+    not symmetric, and both landmark gradients return to their tensors through the pooling adjoint."""
     from dataclasses import replace
     cfg = replace(synth.shrink(synth.CONFIGS[name], B=B, H=H), backward=True)
     inp = synth.make_inputs(cfg)
     Q, K, V, dO = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
     p = ln.problem_from_config(cfg, whiten=inp["whiten"].to(DEV))
-    p.lm_mode = 2
+    p.lm_mode = lm_mode
     saved = torch.empty(ln.laplace_nystrom_saved_bytes(p), dtype=torch.uint8, device=DEV)
-    O = ln.laplace_nystrom_fwd(p, Q, K, V, saved=saved)
-    dQ, dK, dV, dL = ln.laplace_nystrom_bwd(p, Q, K, V, dO, saved)
+    status = torch.full((cfg.B * cfg.H,), -1, dtype=torch.int32, device=DEV)
+    was = ln.set_fused_sign(fused)
+    try:
+        O = ln.laplace_nystrom_fwd(p, Q, K, V, saved=saved, dev_status=status)
+        dQ, dK, dV, dL = ln.laplace_nystrom_bwd(p, Q, K, V, dO, saved)
+    finally:
+        ln.set_fused_sign(was)
     assert dL is None
-    op = oracle_problem(cfg, lm_mode=2)
+    assert int(status.abs().max()) == 0
+    op = oracle_problem(cfg, lm_mode=lm_mode)
     wh = f64(inp["whiten"])
     Oo = oracle.forward(op, f64(inp["Q"]), f64(inp["K"]), f64(inp["V"]), whiten=wh)
     dQo, dKo, dVo, _ = oracle.backward(op, f64(inp["Q"]), f64(inp["K"]), f64(inp["V"]), f64(inp["dO"]), whiten=wh)
@@ -287,7 +298,7 @@ def test_landmarks_pooled_from_queries(name, B, H):
     BH = cfg.B * cfg.H
     errs = {k: metrics(f64(g).reshape(BH, cfg.n, cfg.d), r.reshape(BH, cfg.n, cfg.d), cfg.dtype == "bf16")
             for k, g, r in (("O", O, Oo), ("dQ", dQ, dQo), ("dK", dK, dKo), ("dV", dV, dVo))}
-    print(cfg.name, "pool(Q)", {k: {a: f"{b:.1e}" for a, b in e.items()} for k, e in errs.items()})
+    print(cfg.name, "lm_mode", lm_mode, {k: {a: f"{b:.1e}" for a, b in e.items()} for k, e in errs.items()})
     assert_parity(cfg, errs)
 
 
