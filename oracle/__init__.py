@@ -10,7 +10,8 @@ from __future__ import annotations
 import ctypes
 import os
 import subprocess
-from dataclasses import dataclass
+from dataclasses import dataclass, field
+from typing import Optional
 
 import numpy as np
 
@@ -44,6 +45,7 @@ class _Problem(ctypes.Structure):
         ("prefix", ctypes.c_int32), ("gh", ctypes.c_int32), ("gw", ctypes.c_int32),
         ("mh", ctypes.c_int32), ("mw", ctypes.c_int32),
         ("lm_f32", ctypes.c_int32),
+        ("lm_filter", ctypes.c_void_p),
     ]
 
 
@@ -67,11 +69,20 @@ class Problem:
     mh: int = 0
     mw: int = 0
     lm_f32: int = 0   # 1: pooled landmarks rounded to single precision (what the device stores)
+    # depth-wise-convolution landmark selection (Sec. 4.2): float64 [H, taps, d], taps = (gh/mh)*(gw/mw), or None
+    lm_filter: Optional[np.ndarray] = field(default=None, repr=False)
 
     def c(self) -> _Problem:
+        f = None
+        if self.lm_filter is not None:
+            assert self.lm_mode in (1, 2) and self.gh % self.mh == 0 and self.gw % self.mw == 0
+            f = self.lm_filter
+            assert f.dtype == np.float64 and f.flags["C_CONTIGUOUS"]
+            assert f.shape == (self.H, (self.gh // self.mh) * (self.gw // self.mw), self.d)
+            f = f.ctypes.data
         return _Problem(self.B, self.H, self.n, self.d, self.m, float(self.lam), self.ns_iters,
                         float(self.ridge_eps), float(self.ns_alpha), self.map_mode, self.lm_mode,
-                        self.prefix, self.gh, self.gw, self.mh, self.mw, self.lm_f32)
+                        self.prefix, self.gh, self.gw, self.mh, self.mw, self.lm_f32, f)
 
 
 def _load():
@@ -173,13 +184,17 @@ def forward(p: Problem, Q, K, V, L=None, whiten=None, want=()):
 
 
 def backward(p: Problem, Q, K, V, dO, L=None, whiten=None):
-    """Returns dQ, dK, dV, dL (dL is None when the landmarks are pooled from K)."""
+    """Returns dQ, dK, dV, dL (dL is None when the landmarks are pooled from K).  With a landmark-selection filter
+    (p.lm_filter) the fourth result is the filter's gradient [H, taps, d] instead (summed over the batch)."""
     Q, K, V, L, whiten, dO = _f64(Q), _f64(K), _f64(V), _f64(L), _f64(whiten), _f64(dO)
     dQ, dK, dV = np.empty_like(Q), np.empty_like(Q), np.empty_like(Q)
     dL = np.empty((p.B, p.H, p.m, p.d)) if p.lm_mode == 0 else None      # pooled landmarks (modes 1, 2): folded into dK / dQ
+    dF = np.empty((p.B, p.H) + p.lm_filter.shape[1:]) if p.lm_filter is not None else None
     cp = p.c()
     _load().oracle_bwd(ctypes.byref(cp), _p(Q), _p(K), _p(V), _p(L), _p(whiten), _p(dO),
-                       _p(dQ), _p(dK), _p(dV), _p(dL))
+                       _p(dQ), _p(dK), _p(dV), _p(dL), _p(dF))
+    if dF is not None:
+        return dQ, dK, dV, dF.sum(axis=0)
     return dQ, dK, dV, dL
 
 

@@ -38,7 +38,10 @@
  *   - pooling is adaptive (bin a covers rows floor(a*gh/mh) .. ceil((a+1)*gh/mh)-1),
  *     which equals r x r / stride r pooling whenever r divides the grid;
  *   - optionally (lm_f32) a pooled landmark is the single-precision value nearest to the
- *     exact mean, so that sign(token - landmark) is decided on the numbers the device holds.
+ *     exact mean, so that sign(token - landmark) is decided on the numbers the device holds;
+ *   - the depth-wise-convolution landmark selection Sec. 4.2 mentions as an alternative is one
+ *     r x r filter per head and channel applied with stride r to the regions average pooling
+ *     would average (no bias; the filter with all taps 1/r^2 is average pooling).
  *
  * Beside the path, the two steps that surround it inside the attention block (end of this file): the rotary
  * position embedding on Q and K (Sec. 5.1; positions over the flattened token grid, class tokens not rotated) and
@@ -70,6 +73,9 @@ typedef struct oracle_problem {
                        3: two landmark sets as Alg. 1 prints them, Lq = pool(Q) and Lk = pool(K): C = k(Q, Lk), W = k(Lq, Lk) (not symmetric), R = k(Lq, K) */
   int32_t prefix, gh, gw, mh, mw; /* lm_mode 1: n = prefix + gh*gw, m = mh*mw */
   int32_t lm_f32;   /* 1: pooled landmarks are rounded to single precision before use (see fwd_single) */
+  const double* lm_filter; /* NULL: average pooling.  Else [H][taps][d], taps = (gh/mh)*(gw/mw): the depth-wise convolution
+                              landmark selection of Sec. 4.2 (one r x r filter per head and channel, stride r; the grid must
+                              divide).  Tap (u,v) of a region is index u*(gw/mw)+v.  lm_mode 1 or 2 only. */
 } oracle_problem;
 
 int oracle_num_threads(void) {
@@ -312,8 +318,28 @@ void oracle_ns_pinv_bwd(int batch, int m, const double* W, int iters, double eps
 static int bin_lo(int a, int g, int mbin) { return (int)(((long long)a * g) / mbin); }
 static int bin_hi(int a, int g, int mbin) { return (int)((((long long)(a + 1)) * g + mbin - 1) / mbin); }
 
-static void pool_single(const oracle_problem* p, const double* K, double* L) {
+/* w: NULL, or this head's filter [taps][d] (depth-wise convolution selection, Sec. 4.2) */
+static const double* head_filter(const oracle_problem* p, int bh) {
+  if (!p->lm_filter) return NULL;
+  return p->lm_filter + (size_t)(bh % p->H) * (size_t)((p->gh / p->mh) * (p->gw / p->mw)) * p->d;
+}
+static void pool_single(const oracle_problem* p, const double* K, double* L, const double* w) {
   int d = p->d;
+  if (w) {                         /* L[(a,b)][c] = sum over the taps (u,v) of the region of w[(u,v)][c] K[token][c] */
+    int rh = p->gh / p->mh, rw = p->gw / p->mw;
+    for (int a = 0; a < p->mh; ++a)
+      for (int b = 0; b < p->mw; ++b) {
+        double* Ll = L + (size_t)(a * p->mw + b) * d;
+        for (int c = 0; c < d; ++c) Ll[c] = 0.0;
+        for (int u = 0; u < rh; ++u)
+          for (int v = 0; v < rw; ++v) {
+            const double* kt = K + (size_t)(p->prefix + (a * rh + u) * p->gw + (b * rw + v)) * d;
+            const double* wt = w + (size_t)(u * rw + v) * d;
+            for (int c = 0; c < d; ++c) Ll[c] += wt[c] * kt[c];
+          }
+      }
+    return;
+  }
   for (int a = 0; a < p->mh; ++a)
     for (int b = 0; b < p->mw; ++b) {
       int r0 = bin_lo(a, p->gh, p->mh), r1 = bin_hi(a, p->gh, p->mh);
@@ -330,9 +356,26 @@ static void pool_single(const oracle_problem* p, const double* K, double* L) {
     }
 }
 
-/* dK += pool^T(dL) */
-static void pool_single_bwd(const oracle_problem* p, const double* dL, double* dK) {
+/* dK += pool^T(dL); with a filter w also dw += the gradient of the filter (K: the tensor that was pooled) */
+static void pool_single_bwd(const oracle_problem* p, const double* dL, double* dK, const double* K, const double* w, double* dw) {
   int d = p->d;
+  if (w) {
+    int rh = p->gh / p->mh, rw = p->gw / p->mw;
+    for (int a = 0; a < p->mh; ++a)
+      for (int b = 0; b < p->mw; ++b) {
+        const double* dLl = dL + (size_t)(a * p->mw + b) * d;
+        for (int u = 0; u < rh; ++u)
+          for (int v = 0; v < rw; ++v) {
+            size_t tok = (size_t)(p->prefix + (a * rh + u) * p->gw + (b * rw + v)) * d;
+            const double* wt = w + (size_t)(u * rw + v) * d;
+            for (int c = 0; c < d; ++c) {
+              dK[tok + c] += wt[c] * dLl[c];
+              if (dw) dw[(size_t)(u * rw + v) * d + c] += dLl[c] * K[tok + c];
+            }
+          }
+      }
+    return;
+  }
   for (int a = 0; a < p->mh; ++a)
     for (int b = 0; b < p->mw; ++b) {
       int r0 = bin_lo(a, p->gh, p->mh), r1 = bin_hi(a, p->gh, p->mh);
@@ -351,7 +394,7 @@ void oracle_landmarks_pool(const oracle_problem* p, const double* K, double* L) 
   int BH = p->B * p->H;
 #pragma omp parallel for schedule(dynamic)
   for (int h = 0; h < BH; ++h)
-    pool_single(p, K + (size_t)h * p->n * p->d, L + (size_t)h * p->m * p->d);
+    pool_single(p, K + (size_t)h * p->n * p->d, L + (size_t)h * p->m * p->d, head_filter(p, h));
 }
 
 /* dK is overwritten with pool^T(dL) */
@@ -361,7 +404,7 @@ void oracle_landmarks_pool_bwd(const oracle_problem* p, const double* dL, double
   for (int h = 0; h < BH; ++h) {
     double* dKh = dK + (size_t)h * p->n * p->d;
     memset(dKh, 0, sizeof(double) * (size_t)p->n * p->d);
-    pool_single_bwd(p, dL + (size_t)h * p->m * p->d, dKh);
+    pool_single_bwd(p, dL + (size_t)h * p->m * p->d, dKh, NULL, head_filter(p, h), NULL);
   }
 }
 
@@ -392,10 +435,11 @@ static void ctx_free(head_ctx* x) {
 
 /* s: whitening scale of this head ([m]) or NULL for ones */
 static void fwd_single(const oracle_problem* p, const double* Q, const double* K, const double* V,
-                       const double* Lin, const double* s, head_ctx* x, double* O) {
+                       const double* Lin, const double* s, const double* wf, head_ctx* x, double* O) {
+  /* wf: this head's landmark-selection filter (see oracle_problem.lm_filter) or NULL for average pooling */
   int n = p->n, d = p->d, m = p->m;
   if (p->lm_mode == 1 || p->lm_mode == 2) {                         /* one landmark set: pooled keys (default) or pooled queries */
-    pool_single(p, p->lm_mode == 1 ? K : Q, x->L);
+    pool_single(p, p->lm_mode == 1 ? K : Q, x->L, wf);
     /* The gradient of the kernel holds sign(token - landmark), which is discontinuous: a pooled
        landmark that lies within rounding distance of a token decides that sign differently in
        different precisions.  With lm_f32 the landmark is DEFINED as the single-precision value
@@ -404,8 +448,8 @@ static void fwd_single(const oracle_problem* p, const double* Q, const double* K
     if (p->lm_f32)
       for (size_t e = 0; e < (size_t)m * d; ++e) x->L[e] = (double)(float)x->L[e];
   } else if (p->lm_mode == 3) {                                     /* Alg. 1 as printed: sample query and key landmarks */
-    pool_single(p, K, x->L);
-    pool_single(p, Q, x->Lq_own);
+    pool_single(p, K, x->L, NULL);
+    pool_single(p, Q, x->Lq_own, NULL);
     x->Lq = x->Lq_own;
     if (p->lm_f32)
       for (size_t e = 0; e < (size_t)m * d; ++e) { x->L[e] = (double)(float)x->L[e]; x->Lq[e] = (double)(float)x->Lq[e]; }
@@ -446,7 +490,7 @@ void oracle_fwd(const oracle_problem* p, const double* Q, const double* K, const
     head_ctx x; ctx_alloc(&x, n, d, m);
     size_t nd = (size_t)n * d, md = (size_t)m * d, nm = (size_t)n * m, mm = (size_t)m * m;
     fwd_single(p, Q + h * nd, K + h * nd, V + h * nd, Lin ? Lin + h * md : NULL,
-               whiten ? whiten + (size_t)(h % p->H) * m : NULL, &x, O + h * nd);
+               whiten ? whiten + (size_t)(h % p->H) * m : NULL, head_filter(p, h), &x, O + h * nd);
     if (oL) memcpy(oL + h * md, x.L, sizeof(double) * md);
     if (oC) memcpy(oC + h * nm, x.C, sizeof(double) * nm);
     if (oR) memcpy(oR + h * nm, x.R, sizeof(double) * nm);
@@ -465,13 +509,14 @@ void oracle_fwd(const oracle_problem* p, const double* Q, const double* K, const
  * it is folded into dK through the pooling adjoint).
  */
 static void bwd_single(const oracle_problem* p, const double* Q, const double* K, const double* V,
-                       const double* Lin, const double* s, const double* dO,
-                       double* dQ, double* dK, double* dV, double* dL) {
+                       const double* Lin, const double* s, const double* wf, const double* dO,
+                       double* dQ, double* dK, double* dV, double* dL, double* dwf) {
+  /* wf / dwf: this head's landmark-selection filter and its gradient ([taps][d], overwritten), or NULL */
   int n = p->n, d = p->d, m = p->m;
   size_t nd = (size_t)n * d, md = (size_t)m * d, nm = (size_t)n * m, mm = (size_t)m * m;
   head_ctx x; ctx_alloc(&x, n, d, m);
   double* O = (double*)malloc(sizeof(double) * nd);
-  fwd_single(p, Q, K, V, Lin, s, &x, O);
+  fwd_single(p, Q, K, V, Lin, s, wf, &x, O);
 
   double* dZ = (double*)malloc(sizeof(double) * nm);
   double* dC = (double*)malloc(sizeof(double) * nm);
@@ -508,9 +553,10 @@ static void bwd_single(const oracle_problem* p, const double* Q, const double* K
   l1_block_bwd(n, m, d, Q, x.L, p->lambda, x.C, dC, dQ, dLt);      /* C = k(Q, K~) */
   l1_block_bwd(m, n, d, x.Lq, K, p->lambda, x.R, dR, dLqt, dK);    /* R = k(Q~, K) */
   l1_block_bwd(m, m, d, x.Lq, x.L, p->lambda, x.W, dW, dLqt, dLt); /* W = k(Q~, K~) */
-  if (p->lm_mode == 1) pool_single_bwd(p, dLt, dK);
-  else if (p->lm_mode == 2) pool_single_bwd(p, dLt, dQ);
-  else if (p->lm_mode == 3) { pool_single_bwd(p, dLt, dK); pool_single_bwd(p, dLqt, dQ); }
+  if (dwf) memset(dwf, 0, sizeof(double) * (size_t)((p->gh / p->mh) * (p->gw / p->mw)) * d);
+  if (p->lm_mode == 1) pool_single_bwd(p, dLt, dK, K, wf, dwf);
+  else if (p->lm_mode == 2) pool_single_bwd(p, dLt, dQ, Q, wf, dwf);
+  else if (p->lm_mode == 3) { pool_single_bwd(p, dLt, dK, NULL, NULL, NULL); pool_single_bwd(p, dLqt, dQ, NULL, NULL, NULL); }
   else memcpy(dL, dLt, sizeof(double) * md);
   free(dLq_own);
 
@@ -519,14 +565,18 @@ static void bwd_single(const oracle_problem* p, const double* Q, const double* K
 }
 
 void oracle_bwd(const oracle_problem* p, const double* Q, const double* K, const double* V, const double* Lin,
-                const double* whiten, const double* dO, double* dQ, double* dK, double* dV, double* dL) {
+                const double* whiten, const double* dO, double* dQ, double* dK, double* dV, double* dL, double* dfilter) {
+  /* dfilter: NULL, or [B*H][taps][d]: the gradient of the landmark-selection filter from each batch element and head
+     (the caller adds up the batch elements of a head) */
   int BH = p->B * p->H, n = p->n, d = p->d, m = p->m;
+  size_t td = p->lm_filter ? (size_t)((p->gh / p->mh) * (p->gw / p->mw)) * d : 0;
 #pragma omp parallel for schedule(dynamic)
   for (int h = 0; h < BH; ++h) {
     size_t nd = (size_t)n * d, md = (size_t)m * d;
     bwd_single(p, Q + h * nd, K + h * nd, V + h * nd, Lin ? Lin + h * md : NULL,
-               whiten ? whiten + (size_t)(h % p->H) * m : NULL, dO + h * nd,
-               dQ + h * nd, dK + h * nd, dV + h * nd, dL ? dL + h * md : NULL);
+               whiten ? whiten + (size_t)(h % p->H) * m : NULL, head_filter(p, h), dO + h * nd,
+               dQ + h * nd, dK + h * nd, dV + h * nd, dL ? dL + h * md : NULL,
+               (dfilter && p->lm_filter) ? dfilter + h * td : NULL);
   }
 }
 
