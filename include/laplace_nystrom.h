@@ -76,6 +76,16 @@ typedef struct ln_problem {
                           /* coupled through the statistic.                                                         */
   float whiten_eps;       /* eps of Eq. 6 (whiten_mode 1), >= 0                                                     */
   float* whiten_batch;    /* whiten_mode 1: device [H,m] fp32 written by laplace_nystrom_fwd, read by _bwd         */
+  const float* lm_filter; /* NULL: landmarks are averages over their regions.  Else the depth-wise-convolution     */
+                          /* selection Sec. 4.2 describes as the alternative: device fp32 [H, taps, d], 16-byte     */
+                          /* aligned, taps = (gh/mh)*(gw/mw), one filter per head and channel applied with stride  */
+                          /* equal to the region (tap (u,v) of a region at index u*(gw/mw)+v; no bias; all taps    */
+                          /* 1/taps is average pooling).  lm_mode 1 or 2 with mh | gh and mw | gw (else            */
+                          /* LN_ERR_ARG); lm_mode 3 is LN_ERR_UNSUPPORTED.  A landmark is the fp32 value nearest   */
+                          /* to the exact weighted sum.                                                            */
+  float* lm_filter_grad;  /* with lm_filter: device fp32 [H, taps, d], 16-byte aligned, OVERWRITTEN by             */
+                          /* laplace_nystrom_bwd with the gradient of the filter, summed over the batch; required  */
+                          /* by the backward entry points (LN_ERR_ARG if NULL), ignored by the forward ones        */
 } ln_problem;
 
 const char* ln_status_string(int status);

@@ -184,19 +184,32 @@ static void matmul_nt(int p, int q, int r, const double* A, const double* Bm, do
 /* ------------------------------------------------------------------------- */
 /* Newton-Schulz, Alg. 2                                                      */
 /* ------------------------------------------------------------------------- */
-/* ||W||_1 = max absolute column sum, ||W||_inf = max absolute row sum; ties -> lowest index */
+/* ||W||_1 = max absolute column sum, ||W||_inf = max absolute row sum.  jstar / istar name the column / row the
+   gradient of the norm is taken through.  A maximum is not differentiable where two columns attain it, and two
+   identical landmarks (duplicated keys) make two column sums equal exactly, so that rounding alone would pick the
+   winner.  Reading: among the columns whose sum lies within NORM_TIE (relative) of the maximum the lowest index is
+   taken, which is one valid subgradient and does not depend on the order or precision of the summation.  The norm
+   itself is the true maximum. */
+#define NORM_TIE (1.0 / 16384.0)
 static void norms_1_inf(int m, const double* W, double* n1, int* jstar, double* ninf, int* istar) {
+  double* cs = (double*)malloc(sizeof(double) * 2 * (size_t)m);
+  double* rs = cs + m;
   *n1 = -1.0; *ninf = -1.0; *jstar = 0; *istar = 0;
   for (int j = 0; j < m; ++j) {
     double s = 0.0;
     for (int i = 0; i < m; ++i) s += fabs(W[(size_t)i * m + j]);
-    if (s > *n1) { *n1 = s; *jstar = j; }
+    cs[j] = s;
+    if (s > *n1) *n1 = s;
   }
   for (int i = 0; i < m; ++i) {
     double s = 0.0;
     for (int j = 0; j < m; ++j) s += fabs(W[(size_t)i * m + j]);
-    if (s > *ninf) { *ninf = s; *istar = i; }
+    rs[i] = s;
+    if (s > *ninf) *ninf = s;
   }
+  for (int j = 0; j < m; ++j) if (cs[j] >= *n1 * (1.0 - NORM_TIE)) { *jstar = j; break; }
+  for (int i = 0; i < m; ++i) if (rs[i] >= *ninf * (1.0 - NORM_TIE)) { *istar = i; break; }
+  free(cs);
 }
 
 /*

@@ -47,6 +47,7 @@ class _CProblem(ctypes.Structure):
         ("prefix", ctypes.c_int32), ("gh", ctypes.c_int32), ("gw", ctypes.c_int32),
         ("mh", ctypes.c_int32), ("mw", ctypes.c_int32),
         ("whiten_mode", ctypes.c_int32), ("whiten_eps", ctypes.c_float), ("whiten_batch", ctypes.c_void_p),
+        ("lm_filter", ctypes.c_void_p), ("lm_filter_grad", ctypes.c_void_p),
     ]
 
 
@@ -79,6 +80,10 @@ class Problem:
     whiten_mode: int = 0          # 1: s from this batch's kernel block (Eq. 5-6), gradient through the variance
     whiten_eps: float = 1e-5
     whiten_batch: Optional[torch.Tensor] = field(default=None, repr=False)   # device fp32 [H, m], written by the forward pass
+    # depth-wise-convolution landmark selection (Sec. 4.2): device fp32 [H, (gh/mh)*(gw/mw), d] each; the gradient is
+    # overwritten by the backward pass
+    lm_filter: Optional[torch.Tensor] = field(default=None, repr=False)
+    lm_filter_grad: Optional[torch.Tensor] = field(default=None, repr=False)
 
     def c(self) -> _CProblem:
         w = None
@@ -89,7 +94,15 @@ class Problem:
         return _CProblem(self.B, self.H, self.n, self.d, self.m, float(self.lam), self.ns_iters,
                          float(self.ridge_eps), float(self.ns_alpha), self.dtype, self.map_mode, w,
                          self.lm_mode, self.prefix, self.gh, self.gw, self.mh, self.mw, self.whiten_mode,
-                         float(self.whiten_eps), None if self.whiten_batch is None else self.whiten_batch.data_ptr())
+                         float(self.whiten_eps), None if self.whiten_batch is None else self.whiten_batch.data_ptr(),
+                         self._filter_ptr(self.lm_filter), self._filter_ptr(self.lm_filter_grad))
+
+    def _filter_ptr(self, t):
+        if t is None:
+            return None
+        assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+        assert tuple(t.shape) == (self.H, (self.gh // self.mh) * (self.gw // self.mw), self.d)
+        return t.data_ptr()
 
     @property
     def torch_dtype(self):
@@ -228,6 +241,8 @@ def laplace_nystrom_bwd(p: Problem, Q, K, V, dO, saved, L=None, dQ=None, dK=None
     dV = torch.empty_like(V) if dV is None else dV
     if p.lm_mode == 0 and dL is None:
         dL = torch.empty_like(L)
+    if p.lm_filter is not None and p.lm_filter_grad is None:       # the filter's gradient is left in p.lm_filter_grad
+        p.lm_filter_grad = torch.empty_like(p.lm_filter)
     if ws is None:
         ws = _bytes(laplace_nystrom_workspace_bytes(p, True), Q.device)
     cp = p.c()

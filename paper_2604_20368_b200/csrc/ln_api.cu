@@ -278,6 +278,11 @@ int validate(const ln_problem* p) {
     if ((long long)p->gh * (p->mh + 1) >= (1ll << 31) || (long long)p->gw * (p->mw + 1) >= (1ll << 31)) return LN_ERR_UNSUPPORTED;
     if ((long long)p->n * p->d / 4 >= (1ll << 32)) return LN_ERR_UNSUPPORTED;
   }
+  if (p->lm_filter) {          // depth-wise-convolution landmark selection: r x r regions with stride r, one pooled tensor
+    if (p->lm_mode == 0 || !aligned16(p->lm_filter)) return LN_ERR_ARG;
+    if (p->gh % p->mh != 0 || p->gw % p->mw != 0) return LN_ERR_ARG;
+    if (p->lm_mode == 3) return LN_ERR_UNSUPPORTED;
+  }
   if ((long long)p->B * p->H > 65535) return LN_ERR_UNSUPPORTED;
   if (p->d != 32 && p->d != 64 && p->d != 128) return LN_ERR_UNSUPPORTED;
   if (p->m > 256) return LN_ERR_UNSUPPORTED;
@@ -286,6 +291,7 @@ int validate(const ln_problem* p) {
 
 PoolGeom geom_of(const ln_problem* p) {
   PoolGeom g; g.n = p->n; g.d = p->d; g.m = p->m; g.prefix = p->prefix; g.gh = p->gh; g.gw = p->gw; g.mh = p->mh; g.mw = p->mw;
+  g.filt = p->lm_filter; g.H = p->H;
   return g;
 }
 
@@ -750,6 +756,9 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   } else if (p->lm_mode >= 1) {      // the landmark gradient returns to the pooled tensor (keys, or queries for lm_mode 2)
     LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, w.dLtot, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, w.dLtot, poolQ ? dQ : dK, geom_of(p), 1));
+    if (p->lm_filter)            // gradient of the selection filter, summed over the batch elements of a head
+      LN_LAUNCH("k_filter_grad", st, k_filter_grad<T><<<dim3((p->gh / p->mh) * (p->gw / p->mw), p->H), 256, 0, st>>>(poolQ ? Q : K, w.dLtot, p->lm_filter_grad,
+                                                                                                                 geom_of(p), p->B));
   } else {
     LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, dL, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, nullptr, dK, geom_of(p), 0));
@@ -915,6 +924,7 @@ int check_bwd_args(const ln_problem* p, const void* Q, const void* K, const void
   if (!Q || !K || !V || !dO || !saved || !dQ || !dK || !dV || !ws) return LN_ERR_ARG;
   if ((p->lm_mode == 0) != (L != nullptr)) return LN_ERR_ARG;
   if ((p->lm_mode == 0) != (dL != nullptr)) return LN_ERR_ARG;
+  if (p->lm_filter && (!p->lm_filter_grad || !aligned16(p->lm_filter_grad))) return LN_ERR_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dO) || !aligned16(saved) || !aligned16(dQ) ||
       !aligned16(dK) || !aligned16(dV) || !aligned16(dL) || !aligned16(ws))
     return LN_ERR_ARG;

@@ -70,6 +70,20 @@ __device__ __forceinline__ void fold_pair(float y, float& s, float& b) {
   b = fmaf(-y, s, 0.5f);
 }
 
+// Maximum of s[0..m) and the index the gradient of that maximum is taken through: the lowest index whose value lies
+// within kNormTie (relative) of the maximum.  Two identical landmarks make two column sums of the landmark kernel
+// matrix equal in exact arithmetic; without the window the rounding of the sums would pick the winner (Alg. 2's
+// scale depends on the 1- and infinity-norm; any of the tied columns gives a valid subgradient).
+constexpr float kNormTie = 1.f / 16384.f;
+__device__ __forceinline__ void norm_argmax(const float* s, int m, float& mx, int& idx) {
+  mx = -1.f;
+  for (int t = 0; t < m; ++t) mx = fmaxf(mx, s[t]);
+  const float thr = mx * (1.f - kNormTie);
+  idx = 0;
+  for (int t = 0; t < m; ++t)
+    if (s[t] >= thr) { idx = t; break; }
+}
+
 // Packed pair arithmetic (two fp32 lanes per instruction): the FP32 pipe does not get faster, but a
 // pair costs one issue slot instead of two, which leaves slots for the shared-memory loads.
 typedef unsigned long long f32x2;

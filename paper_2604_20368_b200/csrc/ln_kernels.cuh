@@ -359,7 +359,9 @@ template <typename T> __global__ void k_to_f32(const T* __restrict__ x, float* _
 // =====================================================================================
 // Landmark selection: adaptive average pooling of the keys over the token grid (Sec. 4.2)
 // =====================================================================================
-struct PoolGeom { int n, d, m, prefix, gh, gw, mh, mw; };
+// filt: NULL = average pooling; else the depth-wise-convolution selection of Sec. 4.2, one filter per head and channel,
+// [H][taps][d] with taps = (gh/mh) * (gw/mw) (the grid divides: the host checks), tap (u, v) of a region at u (gw/mw) + v
+struct PoolGeom { int n, d, m, prefix, gh, gw, mh, mw; const float* filt; int H; };
 // 32-bit on purpose (64-bit division costs two orders of magnitude more on the device); the host
 // checks that gh * mh and gw * mw stay below 2^31.
 __host__ __device__ inline int bin_lo(int a, int g, int mb) { return (int)(((unsigned)a * (unsigned)g) / (unsigned)mb); }
@@ -379,12 +381,16 @@ __global__ void __launch_bounds__(256) k_pool(const T* __restrict__ K, float* __
   // value nearest to the exact mean: sign(token - landmark) in the backward pass then does not
   // depend on the order of a single-precision summation.
   double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+  const float* wf = g.filt ? g.filt + (long long)(bh % g.H) * ((r1 - r0) * (c1 - c0)) * g.d + c : nullptr;
   for (int r = r0; r < r1; ++r)
     for (int q = c0; q < c1; ++q) {
       const float4 v = ld4(Kh + (long long)(g.prefix + r * g.gw + q) * g.d + c);
-      s0 += (double)v.x; s1 += (double)v.y; s2 += (double)v.z; s3 += (double)v.w;
+      if (wf) {                        // products of an fp32 weight and a token value are exact in double
+        const float4 w = ld4(wf + (long long)((r - r0) * (c1 - c0) + (q - c0)) * g.d);
+        s0 += (double)w.x * (double)v.x; s1 += (double)w.y * (double)v.y; s2 += (double)w.z * (double)v.z; s3 += (double)w.w * (double)v.w;
+      } else { s0 += (double)v.x; s1 += (double)v.y; s2 += (double)v.z; s3 += (double)v.w; }
     }
-  const double cnt = (double)((r1 - r0) * (c1 - c0));
+  const double cnt = wf ? 1.0 : (double)((r1 - r0) * (c1 - c0));
   st4(L + ((long long)bh * g.m + l) * g.d + c,
       make_float4((float)(s0 / cnt), (float)(s1 / cnt), (float)(s2 / cnt), (float)(s3 / cnt)));
 }
@@ -403,18 +409,22 @@ __global__ void __launch_bounds__(256) k_pool_wide(const T* __restrict__ K, floa
   const int bw = c1 - c0, cnt = (r1 - r0) * bw;
   const T* Kh = K + (long long)bh * g.n * g.d;
   double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+  const float* wf = g.filt ? g.filt + (long long)(bh % g.H) * cnt * g.d + c : nullptr;
   if (tl < lanes)
     for (int t = tl; t < cnt; t += lanes) {
       const int r = r0 + t / bw, q = c0 + t % bw;
       const float4 v = ld4(Kh + (long long)(g.prefix + r * g.gw + q) * g.d + c);
-      s0 += (double)v.x; s1 += (double)v.y; s2 += (double)v.z; s3 += (double)v.w;
+      if (wf) {
+        const float4 w = ld4(wf + (long long)t * g.d);
+        s0 += (double)w.x * (double)v.x; s1 += (double)w.y * (double)v.y; s2 += (double)w.z * (double)v.z; s3 += (double)w.w * (double)v.w;
+      } else { s0 += (double)v.x; s1 += (double)v.y; s2 += (double)v.z; s3 += (double)v.w; }
     }
   red[threadIdx.x][0] = s0; red[threadIdx.x][1] = s1; red[threadIdx.x][2] = s2; red[threadIdx.x][3] = s3;
   __syncthreads();
   if (tl == 0) {
     double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
     for (int u = 0; u < lanes; ++u) { const double* p = red[u * quads + qd]; t0 += p[0]; t1 += p[1]; t2 += p[2]; t3 += p[3]; }
-    const double n = (double)cnt;
+    const double n = wf ? 1.0 : (double)cnt;
     st4(L + ((long long)bh * g.m + l) * g.d + c, make_float4((float)(t0 / n), (float)(t1 / n), (float)(t2 / n), (float)(t3 / n)));
   }
 }
@@ -451,7 +461,10 @@ __global__ void __launch_bounds__(256) k_pool_bwd(const float* __restrict__ dKpa
       // bins of equal size that do not overlap: one bin per token
       const int r = (j - g.prefix) / g.gw, q = (j - g.prefix) % g.gw;
       const float4 t = ld4(dL + ((long long)bh * g.m + (r / bh_rows) * g.mw + q / bh_cols) * g.d + c);
-      v.x += t.x * even_inv; v.y += t.y * even_inv; v.z += t.z * even_inv; v.w += t.w * even_inv;
+      if (g.filt) {                      // selection filter: the token's tap of its region
+        const float4 w = ld4(g.filt + ((long long)(bh % g.H) * (bh_rows * bh_cols) + (r % bh_rows) * bh_cols + q % bh_cols) * g.d + c);
+        v.x += t.x * w.x; v.y += t.y * w.y; v.z += t.z * w.z; v.w += t.w * w.w;
+      } else { v.x += t.x * even_inv; v.y += t.y * even_inv; v.z += t.z * even_inv; v.w += t.w * even_inv; }
     } else if (pool && j >= g.prefix) {
       const int r = (j - g.prefix) / g.gw, q = (j - g.prefix) % g.gw;
       // a token row lies in bin floor(r mh / gh) and, where neighbouring bins overlap, in the next one too
@@ -467,6 +480,34 @@ __global__ void __launch_bounds__(256) k_pool_bwd(const float* __restrict__ dKpa
       }
     }
     st4(dK + ((long long)bh * g.n + j) * g.d + c, v);
+  }
+}
+
+// Gradient of the landmark-selection filter: dF[h][tap][c] = sum over the batch elements b and the landmarks l of
+// dL[b H + h][l][c] X[b H + h][token(l, tap)][c], X the tensor the landmarks were selected from.
+// grid (taps, H); 256 threads = d/4 channel quads x 1024/d lanes over the (b, l) pairs; double sums, lanes added in order.
+template <typename T>
+__global__ void __launch_bounds__(256) k_filter_grad(const T* __restrict__ X, const float* __restrict__ dL, float* __restrict__ dF,
+                                                     PoolGeom g, int B) {
+  __shared__ double red[256][4];
+  const int quads = g.d / 4, lanes = 256 / quads;
+  const int tap = blockIdx.x, h = blockIdx.y, qd = (int)threadIdx.x % quads, tl = (int)threadIdx.x / quads, c = qd * 4;
+  const int rh = g.gh / g.mh, rw = g.gw / g.mw, u = tap / rw, v = tap % rw;
+  double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+  if (tl < lanes)
+    for (int t = tl; t < B * g.m; t += lanes) {
+      const int b = t / g.m, l = t % g.m, a = l / g.mw, bb = l % g.mw;
+      const long long bh = (long long)b * g.H + h;
+      const float4 x = ld4(X + (bh * g.n + g.prefix + (a * rh + u) * g.gw + (bb * rw + v)) * g.d + c);
+      const float4 dl = ld4(dL + (bh * g.m + l) * g.d + c);
+      s0 += (double)dl.x * (double)x.x; s1 += (double)dl.y * (double)x.y; s2 += (double)dl.z * (double)x.z; s3 += (double)dl.w * (double)x.w;
+    }
+  red[threadIdx.x][0] = s0; red[threadIdx.x][1] = s1; red[threadIdx.x][2] = s2; red[threadIdx.x][3] = s3;
+  __syncthreads();
+  if (tl == 0) {
+    double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
+    for (int w = 0; w < lanes; ++w) { const double* p = red[w * quads + qd]; t0 += p[0]; t1 += p[1]; t2 += p[2]; t3 += p[3]; }
+    st4(dF + ((long long)h * (rh * rw) + tap) * g.d + c, make_float4((float)t0, (float)t1, (float)t2, (float)t3));
   }
 }
 
@@ -1011,11 +1052,9 @@ __device__ void ns_forward_dev(int m, int T, float eps, float alpha_in, const fl
   }
   __syncthreads();
   if (tid == 0) {               // every CTA of a cluster arrives at the same values
-    float n1 = -1.f, ninf = -1.f; int js = 0, is = 0;
-    for (int t = 0; t < m; ++t) {                 // strict > keeps the lowest index on ties
-      if (colsum[t] > n1) { n1 = colsum[t]; js = t; }
-      if (rowsum[t] > ninf) { ninf = rowsum[t]; is = t; }
-    }
+    float n1, ninf; int js, is;                   // near-ties (duplicated landmarks): the lowest index
+    norm_argmax(colsum, m, n1, js);
+    norm_argmax(rowsum, m, ninf, is);
     float* al = red + 512;
     al[0] = (alpha_in > 0.f) ? alpha_in : 1.f / (n1 * ninf);
     if (crank == 0) {

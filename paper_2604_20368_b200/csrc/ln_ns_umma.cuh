@@ -179,11 +179,9 @@ __device__ bool ns_forward_umma(int m, int T, float eps, float alpha_in, const f
     }
     __syncthreads();
     if (tid == 0) {
-      float n1 = -1.f, ninf = -1.f; int js = 0, is = 0;
-      for (int q = 0; q < m; ++q) {
-        if (colsum[q] > n1) { n1 = colsum[q]; js = q; }
-        if (rowsum[q] > ninf) { ninf = rowsum[q]; is = q; }
-      }
+      float n1, ninf; int js, is;
+      norm_argmax(colsum, m, n1, js);
+      norm_argmax(rowsum, m, ninf, is);
       hdr->n1 = n1; hdr->ninf = ninf; hdr->jstar = js; hdr->istar = is;
       hdr->auto_alpha = !(alpha_in > 0.f);
       hdr->alpha = (alpha_in > 0.f) ? alpha_in : 1.f / (n1 * ninf);

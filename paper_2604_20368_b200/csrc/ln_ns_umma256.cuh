@@ -132,9 +132,8 @@ __device__ bool ns_forward_umma256(int m, int T, float eps, float alpha_in, cons
     }
     __syncthreads();
     if (tid == 0) {               // every CTA of the cluster arrives at the same values
-      float n1 = -1.f; int js = 0;
-      for (int t = 0; t < m; ++t)
-        if (colsum[t] > n1) { n1 = colsum[t]; js = t; }          // strict >: the lowest index on ties
+      float n1; int js;
+      norm_argmax(colsum, m, n1, js);                            // near-ties (duplicated landmarks): the lowest index
       red[512] = (alpha_in > 0.f) ? alpha_in : 1.f / (n1 * n1);
       if (crank == 0) {
         hdr->n1 = n1; hdr->ninf = n1; hdr->jstar = js; hdr->istar = js;

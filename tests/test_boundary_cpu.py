@@ -132,6 +132,29 @@ def test_host_step_argument_errors_without_gpu():
     assert lib.laplace_nystrom_host_staging_bytes(ctypes.byref(_problem(n=0).c())) == 0
 
 
+def test_filter_selection_argument_errors_without_gpu():
+    """The landmark-selection filter (Sec. 4.2) needs regions that divide the grid, one pooled tensor, and in the
+    backward pass a buffer for its gradient: refused on the host before anything is enqueued."""
+    lib = binding.lib()
+    buf = ctypes.create_string_buffer(96)
+    a = ctypes.c_void_p((ctypes.addressof(buf) + 15) // 16 * 16)      # 16-byte aligned, never dereferenced
+
+    def with_filter(cfg_name, lm_mode, grad):
+        cp = ln.problem_from_config(synth.CONFIGS[cfg_name]).c()
+        cp.lm_mode, cp.lm_filter, cp.lm_filter_grad = lm_mode, a.value, (a.value if grad else None)
+        return cp
+    fwd = lambda cp: lib.laplace_nystrom_fwd(ctypes.byref(cp), a, a, a, None, a, a, a, 0, None, None)
+    bwd = lambda cp: lib.laplace_nystrom_bwd(ctypes.byref(cp), a, a, a, None, a, a, a, a, a, None, a, 0, None, None)
+    assert fwd(with_filter("cfg2", 1, False)) == -3                 # valid problem: only the (empty) workspace is refused
+    assert fwd(with_filter("cfg4a", 1, False)) == -1                # 56 columns do not divide into 16 regions
+    assert fwd(with_filter("cfg2", 3, False)) == -2                 # two landmark sets: not with a filter
+    assert fwd(with_filter("cfg2", 0, False)) == -1                 # given landmarks: nothing is selected
+    assert bwd(with_filter("cfg2", 1, False)) == -1                 # no buffer for the filter's gradient
+    assert bwd(with_filter("cfg2", 1, True)) == -3
+    odd = with_filter("cfg2", 1, False); odd.lm_filter = a.value + 4
+    assert fwd(odd) == -1                                           # not 16-byte aligned
+
+
 def test_overlap_switch_and_launch_counter_without_gpu():
     """ln_set_overlap returns the previous setting (default on); the launch counter is readable and has not moved
     without a launch."""

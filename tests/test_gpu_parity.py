@@ -302,6 +302,44 @@ def test_landmarks_pooled_from_queries(lm_mode, name, B, H, fused):
     assert_parity(cfg, errs)
 
 
+@pytest.mark.parametrize("lm_mode,name,B,H,dtype", [(1, "cfg2", 3, 2, "bf16"), (2, "cfg2", 2, 2, "bf16"), (1, "cfg2", 2, 2, "f32"),
+                                                    (1, "cfg3", 2, 1, "bf16"), (1, "cfg5_m128_T8", 2, 2, "bf16"),
+                                                    (2, "cfg5_m256_T4", 1, 2, "bf16"), (1, "cfg5_m64_T4", 2, 1, "f32")])
+def test_landmarks_selected_by_a_depthwise_filter(lm_mode, name, B, H, dtype):
+    """Sec. 4.2's alternative landmark selection: one r x r filter per head and channel, stride r, in place of the
+    average over a region; the backward pass also returns the filter's gradient, summed over the batch."""
+    from dataclasses import replace
+    from parity import metrics
+    cfg = replace(synth.shrink(synth.CONFIGS[name], B=B, H=H), backward=True, dtype=dtype)
+    inp = synth.make_inputs(cfg)
+    Q, K, V, dO = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
+    taps = (cfg.gh // cfg.mh) * (cfg.gw // cfg.mw)
+    rng = np.random.default_rng(cfg.seed + 77)
+    F = torch.from_numpy((rng.standard_normal((cfg.H, taps, cfg.d)) / taps + 1.0 / taps).astype(np.float32))
+    p = ln.problem_from_config(cfg, whiten=inp["whiten"].to(DEV))
+    p.lm_mode = lm_mode
+    p.lm_filter = F.to(DEV)
+    p.lm_filter_grad = torch.full_like(p.lm_filter, float("nan"))
+    saved = torch.empty(ln.laplace_nystrom_saved_bytes(p), dtype=torch.uint8, device=DEV)
+    O = ln.laplace_nystrom_fwd(p, Q, K, V, saved=saved)
+    dQ, dK, dV, _ = ln.laplace_nystrom_bwd(p, Q, K, V, dO, saved)
+    op = replace(oracle_problem(cfg, lm_mode=lm_mode), lm_filter=np.ascontiguousarray(F.numpy().astype(np.float64)))
+    wh = f64(inp["whiten"])
+    q, k, v, g = (f64(inp[x]) for x in ("Q", "K", "V", "dO"))
+    Oo = oracle.forward(op, q, k, v, whiten=wh)
+    dQo, dKo, dVo, dFo = oracle.backward(op, q, k, v, g, whiten=wh)
+    BH = cfg.B * cfg.H
+    errs = {kk: metrics(f64(a).reshape(BH, cfg.n, cfg.d), r.reshape(BH, cfg.n, cfg.d), cfg.dtype == "bf16")
+            for kk, a, r in (("O", O, Oo), ("dQ", dQ, dQo), ("dK", dK, dKo), ("dV", dV, dVo))}
+    print(cfg.name, "filter selection, lm_mode", lm_mode, {kk: {a: f"{b:.1e}" for a, b in e.items()} for kk, e in errs.items()})
+    assert_parity(cfg, errs)
+    # the filter's gradient is fp32 whatever the storage type: held to the fp32 bar of the gradients it is summed from
+    # (for bf16 storage the upstream dL carries the rounding of the bf16 inputs only, not of an output)
+    e = rel_err(f64(p.lm_filter_grad), dFo)
+    print("   filter gradient", f"{e:.1e}")
+    assert e < (1e-4 if dtype == "f32" else 1e-3)
+
+
 @pytest.mark.parametrize("name,B,H,dtype", [("cfg2", 3, 2, "bf16"), ("cfg2", 2, 1, "f32"), ("cfg4a", 2, 1, "bf16"),
                                             ("cfg5_m64_T4", 2, 1, "bf16"), ("cfg1", 2, 2, "f32")])
 def test_batch_statistic_whitening_training_mode(name, B, H, dtype):

@@ -229,6 +229,49 @@ def test_ns_bwd_finite_differences():
                 assert dW[0, i, j] == pytest.approx((f(p) - f(q)) / (2 * h), rel=2e-6, abs=1e-8)
 
 
+def test_norm_gradient_at_tied_columns_goes_through_the_lowest_index():
+    """alpha = 1/(||W||_1 ||W||_inf) (Alg. 2) is not differentiable where two columns attain the maximum, and two
+    identical landmarks make two column sums equal exactly.  The reading: the gradient of a norm is taken through the
+    lowest index whose sum lies within 2^-14 (relative) of the maximum, whatever the rounding of the sums says."""
+    rng = np.random.default_rng(88)
+    pts = rng.standard_normal((1, 7, 3)) * 2.0
+    pts[0, 5] = pts[0, 2]                                    # landmark 5 is a copy of landmark 2
+    W = oracle.l1_kernel(pts, pts, 3.0)
+    eps, T = 1e-6, 3
+    cs = np.abs(W[0] + eps * np.eye(7)).sum(0)
+    assert np.argsort(-cs)[:2].tolist() in ([2, 5], [5, 2]) and abs(cs[2] - cs[5]) < 1e-12      # the tied pair is the maximum
+    dX = rng.standard_normal((1, 7, 7))
+
+    def alpha_term(Wm):
+        # gradient with alpha derived from the norms minus the gradient with the same alpha given: what remains is
+        # d(loss)/d(alpha) * d(alpha)/dW, which lives in column jstar and row istar only
+        a = oracle.ns_pinv(Wm, T, eps=eps)[2][0]
+        D = oracle.ns_pinv_bwd(Wm, T, eps, 0.0, dX) - oracle.ns_pinv_bwd(Wm, T, eps, a, dX)
+        cols = sorted(set(np.nonzero(np.abs(D[0]).sum(0) > 1e-14 * np.abs(D).max())[0].tolist()))
+        rows = sorted(set(np.nonzero(np.abs(D[0]).sum(1) > 1e-14 * np.abs(D).max())[0].tolist()))
+        return D[0], cols, rows
+
+    D, cols, rows = alpha_term(W)
+    # column 2 and row 2 carry the two norm terms (every entry of W is positive: the whole column / row is touched);
+    # nothing else is
+    off = D.copy(); off[:, 2] = 0.0; off[2, :] = 0.0
+    assert np.abs(off).max() == 0.0 and np.abs(D[:, 2]).min() > 0.0 and np.abs(D[2, :]).min() > 0.0
+    # a perturbation far below the window that makes column 5 the strict maximum does not move the choice
+    Wp = W.copy(); Wp[0, 0, 5] += 1e-7; Wp[0, 5, 0] += 1e-7
+    Dp, _, _ = alpha_term(Wp)
+    off = Dp.copy(); off[:, 2] = 0.0; off[2, :] = 0.0
+    assert np.abs(off).max() == 0.0
+    # well outside the window the larger column wins
+    Wq = W.copy(); Wq[0, :, 5] *= 1.01; Wq[0, 5, :] *= 1.01
+    Dq, _, _ = alpha_term(Wq)
+    off = Dq.copy(); off[:, 5] = 0.0; off[5, :] = 0.0
+    assert np.abs(off).max() == 0.0 and np.abs(Dq[:, 5]).min() > 0.0
+    # and the norm itself is the true maximum in every case
+    for Wm in (W, Wp, Wq):
+        A = Wm[0] + eps * np.eye(7)
+        assert oracle.ns_pinv(Wm, T, eps=eps)[2][0] == pytest.approx(1.0 / (np.abs(A).sum(0).max() * np.abs(A).sum(1).max()), rel=1e-14)
+
+
 # --------------------------------------------------------------------------- pooling
 def test_pool_divisible_and_adjoint():
     p = Problem(B=1, H=2, n=1 + 6 * 4, d=3, m=6, lam=3.0, ns_iters=2, prefix=1, gh=6, gw=4, mh=3, mw=2)
