@@ -749,18 +749,20 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   if (side.on()) side.join(st);      // dV and the landmark-block part are complete
   const int md = m * D;
   if (two) {                  // pooled keys: columns of C and of W; pooled queries: columns of R^T and rows of W
-    LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLW2, 1, nullptr, 0, w.dLtot, md));
-    LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLRpart, chs, w.dLW, 1, nullptr, 0, w.dLqtot, md));
+    LN_LAUNCH("k_reduce3", st, k_reduce3_wide<float><<<dim3(cdiv(md, 128), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLW2, 1, nullptr, 0, w.dLtot, md));
+    LN_LAUNCH("k_reduce3", st, k_reduce3_wide<float><<<dim3(cdiv(md, 128), BH), 256, 0, st>>>(w.dLRpart, chs, w.dLW, 1, nullptr, 0, w.dLqtot, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, w.dLtot, dK, geom_of(p), 1));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dQpart, w.dLqtot, dQ, geom_of(p), 1));
   } else if (p->lm_mode >= 1) {      // the landmark gradient returns to the pooled tensor (keys, or queries for lm_mode 2)
-    LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, w.dLtot, md));
+    if (chq + chs >= 16) LN_LAUNCH("k_reduce3", st, k_reduce3_wide<float><<<dim3(cdiv(md, 128), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, w.dLtot, md));
+    else LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, w.dLtot, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, w.dLtot, poolQ ? dQ : dK, geom_of(p), 1));
     if (p->lm_filter)            // gradient of the selection filter, summed over the batch elements of a head
       LN_LAUNCH("k_filter_grad", st, k_filter_grad<T><<<dim3((p->gh / p->mh) * (p->gw / p->mw), p->H), 256, 0, st>>>(poolQ ? Q : K, w.dLtot, p->lm_filter_grad,
                                                                                                                  geom_of(p), p->B));
   } else {
-    LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, dL, md));
+    if (chq + chs >= 16) LN_LAUNCH("k_reduce3", st, k_reduce3_wide<T><<<dim3(cdiv(md, 128), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, dL, md));
+    else LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, dL, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, nullptr, dK, geom_of(p), 0));
   }
   return launch_ok();

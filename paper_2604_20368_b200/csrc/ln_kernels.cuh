@@ -483,6 +483,47 @@ __global__ void __launch_bounds__(256) k_pool_bwd(const float* __restrict__ dKpa
   }
 }
 
+// The same for many parts (one per token tile of the sign passes): warp w of a CTA adds the parts w, w + 8, ... of every
+// array for 128 consecutive elements (four loads in flight per thread), the eight warps are added in a fixed order.
+// Eight times the CTAs of k_reduce3, which on long sequences has too few of them to draw the memory bandwidth.
+__device__ __forceinline__ float4 sum_parts4_strided(const float* __restrict__ parts, int nparts, long long stride, long long off, int first, int step) {
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  int p = first;
+  for (; p + 3 * step < nparts; p += 4 * step) {
+    float4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const float4*>(parts + (long long)(p + u * step) * stride + off);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
+  }
+  for (; p < nparts; p += step) {
+    const float4 v = *reinterpret_cast<const float4*>(parts + (long long)p * stride + off);
+    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+  }
+  return s;
+}
+template <typename TO>
+__global__ void __launch_bounds__(256) k_reduce3_wide(const float* __restrict__ p0, int n0, const float* __restrict__ p1, int n1,
+                                                      const float* __restrict__ p2, int n2, TO* __restrict__ out, int count) {
+  __shared__ float4 red[8][32];
+  const int bh = blockIdx.y, w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  const int e = (blockIdx.x * 32 + l) * 4;
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (e < count) {
+    s = sum_parts4_strided(p0 + (long long)bh * n0 * count, n0, count, e, w, 8);
+    if (n1 > 0) { const float4 t = sum_parts4_strided(p1 + (long long)bh * n1 * count, n1, count, e, w, 8); s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w; }
+    if (n2 > 0) { const float4 t = sum_parts4_strided(p2 + (long long)bh * n2 * count, n2, count, e, w, 8); s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w; }
+  }
+  red[w][l] = s;
+  __syncthreads();
+  if (w == 0 && e < count) {
+    float4 t = red[0][l];
+#pragma unroll
+    for (int k = 1; k < 8; ++k) { t.x += red[k][l].x; t.y += red[k][l].y; t.z += red[k][l].z; t.w += red[k][l].w; }
+    st4(out + (long long)bh * count + e, t);
+  }
+}
+
 // Gradient of the landmark-selection filter: dF[h][tap][c] = sum over the batch elements b and the landmarks l of
 // dL[b H + h][l][c] X[b H + h][token(l, tap)][c], X the tensor the landmarks were selected from.
 // grid (taps, H); 256 threads = d/4 channel quads x 1024/d lanes over the (b, l) pairs; double sums, lanes added in order.
