@@ -511,3 +511,49 @@ def test_whiten_stats_match_the_oracle(name, B):
     O = ln.laplace_nystrom_fwd(p2, Q, K, V, saved=saved)
     o = run_oracle_heads(cfg, {**inp, "whiten": torch.from_numpy(ref).float()}, [0], backward=False)
     assert rel_err(f64(O).reshape(BH, cfg.n, cfg.d)[[0]], o["O"]) < TOL[cfg.dtype]
+
+
+def _random_cases(count, seed):
+    """Seeded draw of small problems over everything the entry points branch on: grid and landmark-grid shape (bins that
+    divide the grid or overlap), class tokens, head dim, iteration count, storage type, landmark mode, map mode,
+    duplicated bins."""
+    rng = np.random.default_rng(seed)
+    cases = []
+    while len(cases) < count:
+        gh, gw = int(rng.integers(3, 21)), int(rng.integers(3, 21))
+        mh, mw = int(rng.integers(1, min(gh, 16) + 1)), int(rng.integers(1, min(gw, 16) + 1))
+        if mh * mw > 256 or mh * mw < 2:
+            continue
+        even = gh % mh == 0 and gw % mw == 0          # bins of one size: only then can a bin's keys be copies of another's
+        cases.append(dict(gh=gh, gw=gw, mh=mh, mw=mw, prefix=int(rng.integers(0, 3)), d=int(rng.choice([32, 64, 128])),
+                          T=int(rng.integers(0, 9)), dtype=str(rng.choice(["bf16", "f32"])), lm_mode=int(rng.choice([1, 2, 3])),
+                          map_mode=int(rng.choice([0, 1])), dup=float(rng.choice([0.0, 0.2])) * even, B=int(rng.integers(1, 3)),
+                          H=int(rng.integers(1, 4)), seed=int(rng.integers(1, 1 << 20))))
+    return cases
+
+
+@pytest.mark.parametrize("case", _random_cases(32, 20260), ids=lambda c: "g{gh}x{gw}_m{mh}x{mw}_p{prefix}_d{d}_T{T}_{dtype}_lm{lm_mode}_map{map_mode}".format(**c))
+def test_random_shapes_and_modes(case):
+    from parity import metrics
+    cfg = synth.Config("random", B=case["B"], H=case["H"], d=case["d"], m=case["mh"] * case["mw"], T=case["T"], gh=case["gh"],
+                       gw=case["gw"], mh=case["mh"], mw=case["mw"], prefix=case["prefix"], dtype=case["dtype"],
+                       dup_frac=case["dup"], seed=case["seed"])
+    inp = synth.make_inputs(cfg)
+    Q, K, V, dO = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
+    p = ln.problem_from_config(cfg, whiten=inp["whiten"].to(DEV), map_mode=case["map_mode"])
+    p.lm_mode = case["lm_mode"]
+    saved = torch.empty(ln.laplace_nystrom_saved_bytes(p), dtype=torch.uint8, device=DEV)
+    status = torch.full((cfg.B * cfg.H,), -1, dtype=torch.int32, device=DEV)
+    O = ln.laplace_nystrom_fwd(p, Q, K, V, saved=saved, dev_status=status)
+    dQ, dK, dV, _ = ln.laplace_nystrom_bwd(p, Q, K, V, dO, saved)
+    assert int(status.abs().max()) == 0
+    op = oracle_problem(cfg, map_mode=case["map_mode"], lm_mode=case["lm_mode"])
+    wh = f64(inp["whiten"])
+    q, k, v, g = (f64(inp[x]) for x in ("Q", "K", "V", "dO"))
+    Oo = oracle.forward(op, q, k, v, whiten=wh)
+    dQo, dKo, dVo, _ = oracle.backward(op, q, k, v, g, whiten=wh)
+    BH = cfg.B * cfg.H
+    errs = {kk: metrics(f64(a).reshape(BH, cfg.n, cfg.d), r.reshape(BH, cfg.n, cfg.d), cfg.dtype == "bf16")
+            for kk, a, r in (("O", O, Oo), ("dQ", dQ, dQo), ("dK", dK, dKo), ("dV", dV, dVo))}
+    print(case, {kk: {a: f"{b:.1e}" for a, b in e.items()} for kk, e in errs.items()})
+    assert_parity(cfg, errs)
