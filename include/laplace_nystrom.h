@@ -156,7 +156,9 @@ int laplace_nystrom_fwd_bwd_host(const ln_problem* p, const void* hQ, const void
  *   off.  The rotated tensors are kept in the storage type (bf16 storage rounds them once more).
  * DWC: depth-wise ks x ks cross-correlation over the token grid, zero padded, one filter per head and channel,
  *   dwc_w device fp32 [H, d, ks, ks] (ks odd, <= 7), NULL = no convolution branch; prefix tokens receive nothing.
- * lm_mode must be 1 (the grid geometry of `p` is used), else LN_ERR_UNSUPPORTED.
+ *   For bf16 storage with d = 64 or 128 the branch is added inside the kernels that form O and dV, before their one
+ *   rounding; otherwise it is a pass of its own over O / dV.
+ * lm_mode must be 1, 2 or 3 (the grid geometry of `p` is used), else LN_ERR_UNSUPPORTED.
  *   saved: laplace_attention_block_saved_bytes bytes; ws: laplace_attention_block_workspace_bytes bytes (both
  *   passes); the other arguments as for laplace_nystrom_fwd / _bwd.  The backward returns dQ, dK, dV and, when the
  *   convolution branch is on, dWd device fp32 [H, d, ks, ks] (summed over the batch in a fixed order), else dWd = NULL.

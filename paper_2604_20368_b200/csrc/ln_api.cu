@@ -443,7 +443,8 @@ void launch_l1(const char* name, const TA* A, const TB* Bm, float* E, float* row
 // ------------------------------------------------------------------------------------------
 template <typename T, int D>
 int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const T* V, const T* L, T* O,
-             const Ctx& x, const FwdWs& w, int32_t* dev_status, cudaStream_t st, bool clear_status) {
+             const Ctx& x, const FwdWs& w, int32_t* dev_status, cudaStream_t st, bool clear_status, const DwcEpi* epi = nullptr) {
+  // epi: NULL, or the convolution branch DWC(V) of the attention block, added in the epilogue of the O product (bf16, d = 64 / 128)
   const int BH = pl.BH, n = pl.n, m = pl.m, kSMs = sm_count();
   if (dev_status && clear_status) cudaMemsetAsync(dev_status, 0, sizeof(int32_t) * BH, st);   // the kernels OR their flags into it
   // landmarks (Sec. 4.2)
@@ -550,10 +551,17 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   } else launch_mid(st, 3);
   // O = (C - mu) Ytilde + ybar
   if constexpr (std::is_same<T, bf16>::value && (D == 64 || D == 128)) {
-    const size_t smem = nn_umma_smem<D>();
-    want_smem(k_nn_umma<D>, smem);
-    LN_LAUNCH("nn_O", st, k_nn_umma<D><<<dim3(cdiv(n, 128), BH), 256, smem, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr,
-                                                                              reinterpret_cast<const bf16*>(x.Yimg), x.ybar, O, n, m, dev_status));
+    if (epi && epi->src) {
+      const size_t smem = nn_umma_smem_dwc<D>();
+      want_smem(k_nn_umma<D, true>, smem);
+      LN_LAUNCH("nn_O", st, k_nn_umma<D, true><<<dim3(cdiv(n, 128), BH), 256, smem, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr,
+                                                                                      reinterpret_cast<const bf16*>(x.Yimg), x.ybar, O, n, m, dev_status, *epi));
+    } else {
+      const size_t smem = nn_umma_smem<D>();
+      want_smem(k_nn_umma<D>, smem);
+      LN_LAUNCH("nn_O", st, k_nn_umma<D><<<dim3(cdiv(n, 128), BH), 256, smem, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr,
+                                                                                reinterpret_cast<const bf16*>(x.Yimg), x.ybar, O, n, m, dev_status, DwcEpi()));
+    }
   } else if constexpr (std::is_same<T, bf16>::value)
     LN_LAUNCH("nn_O", st, k_nn_mma<D><<<dim3(cdiv(n, 64), BH), 256, 0, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr, x.Yt, x.ybar, O, n, m));
   else
@@ -563,7 +571,9 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
 
 template <typename T, int D>
 int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const T* V, const T* dO,
-             const Ctx& x, const BwdWs& w, T* dQ, T* dK, T* dV, T* dL, int32_t* dev_status, cudaStream_t st, bool clear_status) {
+             const Ctx& x, const BwdWs& w, T* dQ, T* dK, T* dV, T* dL, int32_t* dev_status, cudaStream_t st, bool clear_status,
+             const DwcEpi* epi = nullptr) {
+  // epi: NULL, or the adjoint DWC^T(dO) of the block's convolution branch, added in the epilogue of the dV product
   const int BH = pl.BH, n = pl.n, m = pl.m, ch = pl.chunks, kSMs = sm_count();
   const float inv_lambda = 1.f / p->lambda;
   const float* mu = p->map_mode == 1 ? x.mu : nullptr;
@@ -651,10 +661,17 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   auto launch_nn_dV = [&](cudaStream_t s) {
     if constexpr (std::is_same<T, bf16>::value) {
       if constexpr (D == 64 || D == 128) {
-        const size_t smem = nn_umma_smem<D>();
-        want_smem(k_nn_umma<D>, smem);
-        LN_LAUNCH("nn_dV", s, k_nn_umma<D><<<dim3(cdiv(n, 128), BH), 256, smem, s>>>(x.Rt, pl.ldm, nullptr, reinterpret_cast<const bf16*>(w.dMimg),
-                                                                                 nullptr, dV, n, m, dev_status));
+        if (epi && epi->src) {
+          const size_t smem = nn_umma_smem_dwc<D>();
+          want_smem(k_nn_umma<D, true>, smem);
+          LN_LAUNCH("nn_dV", s, k_nn_umma<D, true><<<dim3(cdiv(n, 128), BH), 256, smem, s>>>(x.Rt, pl.ldm, nullptr, reinterpret_cast<const bf16*>(w.dMimg),
+                                                                                         nullptr, dV, n, m, dev_status, *epi));
+        } else {
+          const size_t smem = nn_umma_smem<D>();
+          want_smem(k_nn_umma<D>, smem);
+          LN_LAUNCH("nn_dV", s, k_nn_umma<D><<<dim3(cdiv(n, 128), BH), 256, smem, s>>>(x.Rt, pl.ldm, nullptr, reinterpret_cast<const bf16*>(w.dMimg),
+                                                                                   nullptr, dV, n, m, dev_status, DwcEpi()));
+        }
       } else
         LN_LAUNCH("nn_dV", s, k_nn_mma<D><<<dim3(cdiv(n, 64), BH), 256, 0, s>>>(x.Rt, pl.ldm, nullptr, w.dM, nullptr, dV, n, m));
     } else {
@@ -770,23 +787,24 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
 
 template <typename T>
 int fwd_dispatch_d(const ln_problem* p, const Plan& pl, const void* Q, const void* K, const void* V, const void* L,
-                   void* O, const Ctx& x, const FwdWs& w, int32_t* ds, cudaStream_t st, bool clear_status) {
+                   void* O, const Ctx& x, const FwdWs& w, int32_t* ds, cudaStream_t st, bool clear_status, const DwcEpi* epi) {
   const T *q = (const T*)Q, *k = (const T*)K, *v = (const T*)V, *l = (const T*)L; T* o = (T*)O;
   switch (p->d) {
-    case 32: return fwd_impl<T, 32>(p, pl, q, k, v, l, o, x, w, ds, st, clear_status);
-    case 64: return fwd_impl<T, 64>(p, pl, q, k, v, l, o, x, w, ds, st, clear_status);
-    case 128: return fwd_impl<T, 128>(p, pl, q, k, v, l, o, x, w, ds, st, clear_status);
+    case 32: return fwd_impl<T, 32>(p, pl, q, k, v, l, o, x, w, ds, st, clear_status, epi);
+    case 64: return fwd_impl<T, 64>(p, pl, q, k, v, l, o, x, w, ds, st, clear_status, epi);
+    case 128: return fwd_impl<T, 128>(p, pl, q, k, v, l, o, x, w, ds, st, clear_status, epi);
   }
   return LN_ERR_UNSUPPORTED;
 }
 template <typename T>
 int bwd_dispatch_d(const ln_problem* p, const Plan& pl, const void* Q, const void* K, const void* V, const void* dO,
-                   const Ctx& x, const BwdWs& w, void* dQ, void* dK, void* dV, void* dL, int32_t* ds, cudaStream_t st, bool clear_status) {
+                   const Ctx& x, const BwdWs& w, void* dQ, void* dK, void* dV, void* dL, int32_t* ds, cudaStream_t st, bool clear_status,
+                   const DwcEpi* epi) {
   const T *q = (const T*)Q, *k = (const T*)K, *v = (const T*)V, *g = (const T*)dO;
   switch (p->d) {
-    case 32: return bwd_impl<T, 32>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st, clear_status);
-    case 64: return bwd_impl<T, 64>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st, clear_status);
-    case 128: return bwd_impl<T, 128>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st, clear_status);
+    case 32: return bwd_impl<T, 32>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st, clear_status, epi);
+    case 64: return bwd_impl<T, 64>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st, clear_status, epi);
+    case 128: return bwd_impl<T, 128>(p, pl, q, k, v, g, x, w, (T*)dQ, (T*)dK, (T*)dV, (T*)dL, ds, st, clear_status, epi);
   }
   return LN_ERR_UNSUPPORTED;
 }
@@ -936,27 +954,27 @@ int check_bwd_args(const ln_problem* p, const void* Q, const void* K, const void
 // clear_status: zero dev_status first (the stand-alone entry points); the host-buffer step clears it once and lets
 // the backward pass OR its flags into what the forward pass left
 int fwd_entry(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L, void* O,
-              void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream, bool clear_status) {
+              void* saved, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream, bool clear_status, const DwcEpi* epi = nullptr) {
   const int s = check_fwd_args(p, Q, K, V, L, O, saved, ws, ws_bytes);
   if (s != LN_OK) return s;
   Plan pl; make_plan(p, &pl);
   const FwdWs w = carve_fwd_ws(pl, ws);
   const Ctx x = carve_ctx(pl, saved ? saved : static_cast<char*>(ws) + w.bytes);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (p->dtype == LN_F32) return fwd_dispatch_d<float>(p, pl, Q, K, V, L, O, x, w, dev_status, st, clear_status);
-  return fwd_dispatch_d<bf16>(p, pl, Q, K, V, L, O, x, w, dev_status, st, clear_status);
+  if (p->dtype == LN_F32) return fwd_dispatch_d<float>(p, pl, Q, K, V, L, O, x, w, dev_status, st, clear_status, epi);
+  return fwd_dispatch_d<bf16>(p, pl, Q, K, V, L, O, x, w, dev_status, st, clear_status, epi);
 }
 int bwd_entry(const ln_problem* p, const void* Q, const void* K, const void* V, const void* L,
               const void* dO, const void* saved, void* dQ, void* dK, void* dV, void* dL, void* ws,
-              size_t ws_bytes, int32_t* dev_status, void* stream, bool clear_status) {
+              size_t ws_bytes, int32_t* dev_status, void* stream, bool clear_status, const DwcEpi* epi = nullptr) {
   const int s = check_bwd_args(p, Q, K, V, L, dO, saved, dQ, dK, dV, dL, ws, ws_bytes);
   if (s != LN_OK) return s;
   Plan pl; make_plan(p, &pl);
   const BwdWs w = carve_bwd_ws(pl, ws);
   const Ctx x = carve_ctx(pl, const_cast<void*>(saved));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (p->dtype == LN_F32) return bwd_dispatch_d<float>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, dev_status, st, clear_status);
-  return bwd_dispatch_d<bf16>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, dev_status, st, clear_status);
+  if (p->dtype == LN_F32) return bwd_dispatch_d<float>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, dev_status, st, clear_status, epi);
+  return bwd_dispatch_d<bf16>(p, pl, Q, K, V, dO, x, w, dQ, dK, dV, dL, dev_status, st, clear_status, epi);
 }
 }  // namespace
 
@@ -1270,6 +1288,8 @@ void launch_rope(const char* name, const ln_problem* p, const ln_block* b, const
   LN_LAUNCH(name, st, k_rope<T><<<cdiv(rows * (p->d / 4), 256), 256, 0, st>>>((const T*)X, (T*)out, rows, p->n, p->d, p->prefix,
                                                                              log2((double)b->rope_base), sign));
 }
+// the tcgen05 product kernels (bf16 storage, 64 or 128 dims) take the convolution branch into their epilogue
+inline bool dwc_in_epilogue(const ln_problem* p) { return p->dtype == LN_BF16 && (p->d == 64 || p->d == 128); }
 template <typename T>
 void launch_dwc_add(const char* name, const ln_problem* p, const ln_block* b, const void* src, void* out, int flip, cudaStream_t st) {
   LN_LAUNCH(name, st, k_dwc_add<T><<<dim3(cdiv((long long)p->gh * p->gw * (p->d / 4), 256), p->B * p->H), 256, 0, st>>>(
@@ -1310,9 +1330,12 @@ int laplace_attention_block_fwd(const ln_problem* p, const ln_block* b, const vo
     else { launch_rope<bf16>("rope_Q", p, b, Q, sv, 1.f, st); launch_rope<bf16>("rope_K", p, b, K, sv + tb, 1.f, st); }
     q = sv; k = sv + tb; inner_saved = sv + 2 * tb;
   }
-  s = fwd_entry(p, q, k, V, nullptr, O, inner_saved, ws, ws_bytes, dev_status, stream, true);
+  // the convolution branch rides in the epilogue of the O product where that product is the tcgen05 kernel; else its own pass
+  const bool fused_dwc = b->dwc_w && dwc_in_epilogue(p);
+  const DwcEpi epi = {V, b->dwc_w, p->H, p->prefix, p->gh, p->gw, b->dwc_ks, 0};
+  s = fwd_entry(p, q, k, V, nullptr, O, inner_saved, ws, ws_bytes, dev_status, stream, true, fused_dwc ? &epi : nullptr);
   if (s != LN_OK) return s;
-  if (b->dwc_w) {
+  if (b->dwc_w && !fused_dwc) {
     if (p->dtype == LN_F32) launch_dwc_add<float>("dwc_O", p, b, V, O, 0, st); else launch_dwc_add<bf16>("dwc_O", p, b, V, O, 0, st);
   }
   return launch_ok();
@@ -1335,7 +1358,10 @@ int laplace_attention_block_bwd(const ln_problem* p, const ln_block* b, const vo
   const void *q = rope ? (const void*)sv : Q, *k = rope ? (const void*)(sv + tb) : K;
   void *dq = rope ? (void*)(w + base_ws) : dQ, *dk = rope ? (void*)(w + base_ws + tb) : dK;
   float* wpart = reinterpret_cast<float*>(w + base_ws + (rope ? 2 * tb : 0));
-  s = bwd_entry(p, q, k, V, nullptr, dO, rope ? sv + 2 * tb : sv, dq, dk, dV, nullptr, ws, base_ws, dev_status, stream, true);
+  const bool fused_dwc = b->dwc_w && dwc_in_epilogue(p);
+  const DwcEpi epi = {dO, b->dwc_w, p->H, p->prefix, p->gh, p->gw, b->dwc_ks, 1};
+  s = bwd_entry(p, q, k, V, nullptr, dO, rope ? sv + 2 * tb : sv, dq, dk, dV, nullptr, ws, base_ws, dev_status, stream, true,
+                fused_dwc ? &epi : nullptr);
   if (s != LN_OK) return s;
   if (rope) {
     if (p->dtype == LN_F32) { launch_rope<float>("rope_dQ", p, b, dq, dQ, -1.f, st); launch_rope<float>("rope_dK", p, b, dk, dK, -1.f, st); }
@@ -1348,7 +1374,7 @@ int laplace_attention_block_bwd(const ln_problem* p, const ln_block* b, const vo
       LN_LAUNCH("dwc_wgrad", st, k_dwc_wgrad<float><<<dim3(ch, BH), 128, 0, st>>>((const float*)V, (const float*)dO, wpart, p->n, p->d, p->prefix,
                                                                                  p->gh, p->gw, b->dwc_ks, kDwcTokensPerChunk));
     } else {
-      launch_dwc_add<bf16>("dwc_dV", p, b, dO, dV, 1, st);
+      if (!fused_dwc) launch_dwc_add<bf16>("dwc_dV", p, b, dO, dV, 1, st);
       LN_LAUNCH("dwc_wgrad", st, k_dwc_wgrad<bf16><<<dim3(ch, BH), 128, 0, st>>>((const bf16*)V, (const bf16*)dO, wpart, p->n, p->d, p->prefix,
                                                                                 p->gh, p->gw, b->dwc_ks, kDwcTokensPerChunk));
     }

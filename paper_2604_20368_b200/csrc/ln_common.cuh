@@ -173,6 +173,11 @@ template <int CL> __device__ __forceinline__ void phase_sync() {
   }
 }
 
+// Depth-wise convolution branch of the attention block (Eq. 7: Attention = Z V + DWC(V)) as an addition to the output of a
+// product kernel: out[bh][prefix + r gw + q][c] += sum_{a,b} w[h][c][a][b] src[bh][prefix + (r+a-ks/2) gw + (q+b-ks/2)][c]
+// (zero padding; flip = 1 mirrors the filter, which is the adjoint with respect to src).  src == NULL: nothing is added.
+struct DwcEpi { const void* src; const float* w; int H, prefix, gh, gw, ks, flip; };
+
 // Header kept per matrix beside the Newton-Schulz iterates.
 struct NsHdr { float alpha, n1, ninf; int jstar, istar, auto_alpha, pad0, pad1; };
 

@@ -38,12 +38,18 @@ __device__ __forceinline__ void gu_write_images(const float* __restrict__ src, b
 
 // shared memory of k_nn_umma: E block images and Y block images; the bf16 staging of the output tile reuses them
 template <int D> __host__ __device__ constexpr size_t nn_umma_smem() { return (size_t)(2 * 128 * GU_KB + 2 * GU_KB * D) * sizeof(bf16); }
+// with the convolution branch in the epilogue the output tile is staged in fp32 (one rounding, after the branch is added)
+template <int D> __host__ __device__ constexpr size_t nn_umma_smem_dwc() {
+  return nn_umma_smem<D>() > (size_t)128 * (D + 4) * sizeof(float) ? nn_umma_smem<D>() : (size_t)128 * (D + 4) * sizeof(float);
+}
 
 // One 128-token tile per CTA; three CTAs per SM hide each other's load latencies.
-template <int D>
+// DWC: the depth-wise convolution branch of the attention block (Eq. 7) is added in the epilogue, before the one rounding
+// to bf16 (O = Z V + DWC(V) in the forward pass; dV = R^T dM + DWC^T(dO) in the backward pass).
+template <int D, bool DWC = false>
 __global__ void __launch_bounds__(256, 3) k_nn_umma(const float* __restrict__ E, int lde, const float* __restrict__ mu,
                                                     const bf16* __restrict__ Yimg, const float* __restrict__ ybar,
-                                                    bf16* __restrict__ O, int n, int m, int* dev_status) {
+                                                    bf16* __restrict__ O, int n, int m, int* dev_status, DwcEpi epi = DwcEpi()) {
   extern __shared__ __align__(128) unsigned char gu_smem[];
   bf16* sZ = reinterpret_cast<bf16*>(gu_smem);                 // [2][128 * 64]: hi, lo of the E block (K-major image)
   bf16* sY = sZ + 2 * 128 * GU_KB;                             // [2][64 * D]: hi, lo of the Y block (image, rows = K)
@@ -123,6 +129,66 @@ __global__ void __launch_bounds__(256, 3) k_nn_umma(const float* __restrict__ E,
   // buffers, which no MMA reads any more)
   constexpr int HC = D / 2, LDS_ = D + 8;
   bf16* stage = reinterpret_cast<bf16*>(gu_smem);              // [128][D + 8]
+  if constexpr (DWC) {
+    constexpr int LDF = D + 4;
+    float* fstage = reinterpret_cast<float*>(gu_smem);         // [128][D + 4] fp32
+    {
+      const int row = (warp & 3) * 32 + (tid & 31), c0 = (warp >> 2) * HC;
+#pragma unroll
+      for (int cb = 0; cb < HC; cb += 32) {
+        float a[32];
+        umma::tmem_ld32(umma::tmem_addr(tacc, c0 + cb), a);
+#pragma unroll
+        for (int q = 0; q < 32; q += 4) {
+          const int c = c0 + cb + q;
+          float4 o = make_float4(a[q], a[q + 1], a[q + 2], a[q + 3]);
+          if (ybar) { o.x += ybar[c]; o.y += ybar[c + 1]; o.z += ybar[c + 2]; o.w += ybar[c + 3]; }
+          *reinterpret_cast<float4*>(fstage + row * LDF + c) = o;
+        }
+      }
+    }
+    umma::fence_before_sync();
+    __syncthreads();
+    const bf16* src = static_cast<const bf16*>(epi.src) + (long long)bh * n * D;
+    const int kk = epi.ks * epi.ks, half = epi.ks / 2;
+    const float* wh = epi.w + (long long)(bh % epi.H) * D * kk;
+    for (int p = tid; p < 128 * (D / 8); p += 256) {
+      const int r = p / (D / 8), c8 = (p % (D / 8)) * 8, i = i0 + r;
+      if (i >= n) continue;
+      float acc[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = fstage[r * LDF + c8 + e];
+      if (i >= epi.prefix) {
+        const int tok = i - epi.prefix, gr = tok / epi.gw, gq = tok % epi.gw;
+        for (int a = 0; a < epi.ks; ++a) {
+          const int rr = gr + a - half;
+          if (rr < 0 || rr >= epi.gh) continue;
+          for (int b = 0; b < epi.ks; ++b) {
+            const int qq = gq + b - half;
+            if (qq < 0 || qq >= epi.gw) continue;
+            const int tap = epi.flip ? (epi.ks - 1 - a) * epi.ks + (epi.ks - 1 - b) : a * epi.ks + b;
+            const uint4 v = *reinterpret_cast<const uint4*>(src + (long long)(epi.prefix + rr * epi.gw + qq) * D + c8);
+            const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              acc[2 * e] = fmaf(__ldg(wh + (c8 + 2 * e) * kk + tap), __uint_as_float(vw[e] << 16), acc[2 * e]);
+              acc[2 * e + 1] = fmaf(__ldg(wh + (c8 + 2 * e + 1) * kk + tap), __uint_as_float(vw[e] & 0xffff0000u), acc[2 * e + 1]);
+            }
+          }
+        }
+      }
+      uint32_t wo[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat162 pr = __floats2bfloat162_rn(acc[2 * e], acc[2 * e + 1]);
+        wo[e] = *reinterpret_cast<const uint32_t*>(&pr);
+      }
+      *reinterpret_cast<uint4*>(O + (long long)i * D + c8) = make_uint4(wo[0], wo[1], wo[2], wo[3]);
+    }
+    if (warp == 0) umma::tmem_dealloc(tmem_base, D);
+    if (!ok && dev_status && tid == 0) atomicOr(dev_status + bh, 2);
+    return;
+  }
   {
     const int row = (warp & 3) * 32 + (tid & 31), c0 = (warp >> 2) * HC;
 #pragma unroll

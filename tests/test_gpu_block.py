@@ -38,8 +38,10 @@ def _case(cfg, rope_base, ks, seed=0):
     for name, e in errs.items():
         assert e["fro"] < TOL[cfg.dtype] and e["maxabs"] < TOL[cfg.dtype], (name, e)
         assert e["row"] < 2 * TOL[cfg.dtype], (name, e)
-        if bf:      # O and dV are rounded twice on this path (once by the attention kernels, once after the convolution is added)
-            assert e["internal"] < 3e-3, (name, e)
+        if bf:
+            # O and dV are rounded once (the convolution branch is added in the epilogue of the tcgen05 products, before
+            # the rounding); dQ and dK are rounded by the attention kernels and again after the inverse rotation
+            assert e["internal"] < (1e-3 if name in ("O", "dV") else 3e-3), (name, e)
     if Wd is not None:
         ew = float(np.linalg.norm(f64(dWd) - dWo) / np.linalg.norm(dWo))
         print("dWd", ew)
@@ -59,6 +61,12 @@ def test_block_cfg2_shape(rope_base, ks, dtype):
 def test_block_large_grid_bf16():
     # 56 x 56 tokens: positions up to 3135, where the rotation angle has to be formed in double
     _case(synth.shrink(synth.CONFIGS["cfg4a"], B=1, H=2), 10000.0, 3)
+
+
+def test_block_128_dims_bf16():
+    # head dim 128: the convolution branch rides in the epilogue of the two tcgen05 products (O and dV), 7 x 7 and 3 x 3 filters
+    _case(synth.shrink(synth.CONFIGS["cfg5_m64_T4"], B=1, H=2), 10000.0, 3)
+    _case(synth.shrink(synth.CONFIGS["cfg5_m128_T4"], B=1, H=1), 0.0, 7, seed=3)
 
 
 def test_block_without_extras_is_the_path():
