@@ -141,7 +141,10 @@ int laplace_nystrom_bwd(const ln_problem* p, const void* Q, const void* K, const
  *   staging: DEVICE memory, laplace_nystrom_host_staging_bytes(p) bytes, 16-byte aligned, owned by the caller;
  *   saved, ws, dev_status: as for laplace_nystrom_fwd / _bwd (training sizes); dev_status is cleared once and
  *   collects the flags of both passes.  Every argument check of both passes is made before the first copy.
- * Two calls on two streams with two sets of device buffers overlap one step's copies with the other's kernels.
+ * The copies ride on two copy streams the library keeps per (device, stream), tied to `stream` by events (Q, K, V in,
+ * dO in beside the forward pass, O out beside the backward pass, the gradients out at the end); `stream` waits for the
+ * last copy, so to the caller the call is still ordered on `stream`.  With ln_set_overlap(0) everything goes on `stream`
+ * itself.  Several calls on several streams with their own device buffers overlap each other's copies and kernels.
  */
 size_t laplace_nystrom_host_staging_bytes(const ln_problem* p);
 int laplace_nystrom_fwd_bwd_host(const ln_problem* p, const void* hQ, const void* hK, const void* hV, const void* hdO,

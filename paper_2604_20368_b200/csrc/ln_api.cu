@@ -343,7 +343,9 @@ struct TraceScope {
 // time are not supported (the order of their work on that stream would be undefined anyway).
 constexpr int kSideSlots = 32, kSideEvents = 16;
 struct SideState { bool used = false, ok = false; int dev = -1; cudaStream_t caller = nullptr; cudaStream_t s = nullptr;
-                   cudaEvent_t ev[kSideEvents]; unsigned next = 0; };
+                   cudaEvent_t ev[kSideEvents]; unsigned next = 0; bool side_tried = false;
+                   // copy streams of the host-buffer entry point (created on its first call for this caller stream)
+                   bool copy_tried = false, copy_ok = false; cudaStream_t cin = nullptr, cout = nullptr; cudaEvent_t cev[6]; };
 SideState g_side[kSideSlots];
 std::mutex g_side_mu;
 std::atomic<bool> g_overlap{true};
@@ -372,6 +374,9 @@ Side side_acquire(bool want, cudaStream_t caller) {
     for (int i = 0; i < kSideSlots && !d; ++i) if (!g_side[i].used) d = &g_side[i];
     if (!d) return r;                  // table full: this caller stream runs without overlap
     d->used = true; d->dev = dev; d->caller = caller;
+  }
+  if (!d->side_tried) {
+    d->side_tried = true;
     // highest priority: its few large CTAs (up to a whole SM each) are placed before the pending small CTAs of
     // the kernels on the caller's stream, which would otherwise keep every SM partly occupied until their grids end
     int prio_lo = 0, prio_hi = 0;
@@ -384,6 +389,39 @@ Side side_acquire(bool want, cudaStream_t caller) {
   if (!d->ok) return r;
   r.s = d->s; r.fork_ev[0] = d->ev[d->next]; r.fork_ev[1] = d->ev[d->next + 1]; r.join_ev = d->ev[d->next + 2];
   d->next = (d->next + 4) % kSideEvents;
+  return r;
+}
+
+// Two copy streams per (device, caller stream) for the host-buffer entry point: host -> device copies on one, device ->
+// host copies on the other, tied to the caller's stream by events, so that a step's copies run beside its own kernels
+// (the copy of O back beside the backward pass, the copy of dO in beside the forward pass) and PCIe carries both
+// directions at once.  To the caller everything is still ordered on the stream it passed.  ok == false (creation
+// failed, or no room in the table): the entry point puts everything on the caller's stream.
+struct CopyStreams { bool ok = false; cudaStream_t cin = nullptr, cout = nullptr; cudaEvent_t ev[6] = {}; };
+CopyStreams copy_acquire(cudaStream_t caller) {
+  CopyStreams r;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return r;
+  std::lock_guard<std::mutex> lk(g_side_mu);
+  SideState* d = nullptr;
+  for (int i = 0; i < kSideSlots && !d; ++i)
+    if (g_side[i].used && g_side[i].dev == dev && g_side[i].caller == caller) d = &g_side[i];
+  if (!d) {
+    for (int i = 0; i < kSideSlots && !d; ++i) if (!g_side[i].used) d = &g_side[i];
+    if (!d) return r;
+    d->used = true; d->dev = dev; d->caller = caller;      // the compute side stream of this slot is created by side_acquire when first asked for
+  }
+  if (!d->copy_tried) {
+    d->copy_tried = true;
+    bool ok = cudaStreamCreateWithFlags(&d->cin, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&d->cout, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; ok && i < 6; ++i) ok = cudaEventCreateWithFlags(&d->cev[i], cudaEventDisableTiming) == cudaSuccess;
+    d->copy_ok = ok;
+    if (!ok) cudaGetLastError();
+  }
+  if (!d->copy_ok) return r;
+  r.ok = true; r.cin = d->cin; r.cout = d->cout;
+  for (int i = 0; i < 6; ++i) r.ev[i] = d->cev[i];
   return r;
 }
 
@@ -1057,19 +1095,48 @@ int laplace_nystrom_fwd_bwd_host(const ln_problem* p, const void* hQ, const void
   if (s != LN_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const void* hin[4] = {hQ, hK, hV, hdO};
-  for (int i = 0; i < 4; ++i)
-    if (cudaMemcpyAsync(d + i * one, hin[i], bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return LN_ERR_CUDA;
+  void* hout[3] = {hdQ, hdK, hdV};
+  const CopyStreams cs = g_overlap.load(std::memory_order_relaxed) ? copy_acquire(st) : CopyStreams();
+  if (!cs.ok) {                       // everything on the caller's stream, one after the other
+    for (int i = 0; i < 4; ++i)
+      if (cudaMemcpyAsync(d + i * one, hin[i], bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return LN_ERR_CUDA;
+    s = fwd_entry(p, d, d + one, d + 2 * one, nullptr, d + 4 * one, saved, ws, ws_bytes, dev_status, stream, true);
+    if (s != LN_OK) return s;
+    if (cudaMemcpyAsync(hO, d + 4 * one, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LN_ERR_CUDA;
+    // the backward pass ORs its flags into the status words the forward pass cleared and wrote
+    s = bwd_entry(p, d, d + one, d + 2 * one, nullptr, d + 3 * one, saved, d + 5 * one, d + 6 * one, d + 7 * one,
+                  nullptr, ws, ws_bytes, dev_status, stream, false);
+    if (s != LN_OK) return s;
+    for (int i = 0; i < 3; ++i)
+      if (cudaMemcpyAsync(hout[i], d + (5 + i) * one, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LN_ERR_CUDA;
+    return LN_OK;
+  }
+  // Copies on the two copy streams: Q, K, V in, then dO in beside the forward pass; O out beside the backward pass; the
+  // three gradients out at the end.  ev[0]: what the caller's stream held before this call (it may still use the
+  // staging buffers); ev[1]: Q, K, V have arrived; ev[2]: dO has arrived; ev[3]: forward pass done; ev[4]: backward
+  // pass done; ev[5]: every copy out done, which the caller's stream waits for before the call counts as complete.
+  bool okc = cudaEventRecord(cs.ev[0], st) == cudaSuccess;
+  okc = okc && cudaStreamWaitEvent(cs.cin, cs.ev[0], 0) == cudaSuccess && cudaStreamWaitEvent(cs.cout, cs.ev[0], 0) == cudaSuccess;
+  for (int i = 0; okc && i < 3; ++i) okc = cudaMemcpyAsync(d + i * one, hin[i], bytes, cudaMemcpyHostToDevice, cs.cin) == cudaSuccess;
+  okc = okc && cudaEventRecord(cs.ev[1], cs.cin) == cudaSuccess;
+  okc = okc && cudaMemcpyAsync(d + 3 * one, hin[3], bytes, cudaMemcpyHostToDevice, cs.cin) == cudaSuccess;
+  okc = okc && cudaEventRecord(cs.ev[2], cs.cin) == cudaSuccess;
+  okc = okc && cudaStreamWaitEvent(st, cs.ev[1], 0) == cudaSuccess;
+  if (!okc) return LN_ERR_CUDA;
   s = fwd_entry(p, d, d + one, d + 2 * one, nullptr, d + 4 * one, saved, ws, ws_bytes, dev_status, stream, true);
   if (s != LN_OK) return s;
-  if (cudaMemcpyAsync(hO, d + 4 * one, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LN_ERR_CUDA;
+  okc = cudaEventRecord(cs.ev[3], st) == cudaSuccess && cudaStreamWaitEvent(cs.cout, cs.ev[3], 0) == cudaSuccess;
+  okc = okc && cudaMemcpyAsync(hO, d + 4 * one, bytes, cudaMemcpyDeviceToHost, cs.cout) == cudaSuccess;
+  okc = okc && cudaStreamWaitEvent(st, cs.ev[2], 0) == cudaSuccess;
+  if (!okc) return LN_ERR_CUDA;
   // the backward pass ORs its flags into the status words the forward pass cleared and wrote
   s = bwd_entry(p, d, d + one, d + 2 * one, nullptr, d + 3 * one, saved, d + 5 * one, d + 6 * one, d + 7 * one,
                 nullptr, ws, ws_bytes, dev_status, stream, false);
   if (s != LN_OK) return s;
-  void* hout[3] = {hdQ, hdK, hdV};
-  for (int i = 0; i < 3; ++i)
-    if (cudaMemcpyAsync(hout[i], d + (5 + i) * one, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LN_ERR_CUDA;
-  return LN_OK;
+  okc = cudaEventRecord(cs.ev[4], st) == cudaSuccess && cudaStreamWaitEvent(cs.cout, cs.ev[4], 0) == cudaSuccess;
+  for (int i = 0; okc && i < 3; ++i) okc = cudaMemcpyAsync(hout[i], d + (5 + i) * one, bytes, cudaMemcpyDeviceToHost, cs.cout) == cudaSuccess;
+  okc = okc && cudaEventRecord(cs.ev[5], cs.cout) == cudaSuccess && cudaStreamWaitEvent(st, cs.ev[5], 0) == cudaSuccess;
+  return okc ? LN_OK : LN_ERR_CUDA;
 }
 
 size_t ns_pinv_workspace_bytes(int32_t batch, int32_t m, int32_t iters) {
