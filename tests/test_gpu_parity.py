@@ -486,6 +486,39 @@ def test_host_buffer_step_matches_device_path():
             assert torch.equal(hout[k], g[k].cpu()), k
 
 
+@pytest.mark.parametrize("overlap", [True, False])
+def test_host_buffer_steps_back_to_back_on_one_stream(overlap):
+    """Two host-buffer steps with DIFFERENT inputs enqueued on one stream, one behind the other, without a host
+    synchronisation in between and sharing their device buffers: the second step's copies in must not overtake the first
+    step's kernels and copies out (the copies ride on the library's copy streams, ordered by events), and each step must
+    return the bits of the device path on its own inputs.  With ln_set_overlap(0) everything is on the caller's stream."""
+    from dataclasses import replace
+    cfg = synth.shrink(synth.CONFIGS["cfg3"], B=2)
+    inps = [synth.make_inputs(cfg), synth.make_inputs(replace(cfg, seed=cfg.seed + 1))]
+    refs = [run_gpu(cfg, inp) for inp in inps]
+    p = ln.problem_from_config(cfg, whiten=inps[0]["whiten"].to(DEV))        # the whitening scale of the two seeds
+    # the second reference with the first problem's whitening scale (one problem struct serves both steps)
+    inp1 = dict(inps[1]); inp1["whiten"] = inps[0]["whiten"]
+    refs[1] = run_gpu(cfg, inp1)
+    bufs = ln.HostStep(p, DEV)
+    hin = [{k: inp[k].pin_memory() for k in ("Q", "K", "V", "dO")} for inp in inps]
+    hout = [{k: torch.empty_like(inps[0]["Q"]).pin_memory() for k in ("O", "dQ", "dK", "dV")} for _ in range(2)]
+    st = torch.cuda.Stream(device=DEV)
+    was = ln.set_overlap(overlap)
+    try:
+        for rep in range(3):
+            for i in (0, 1):
+                ln.laplace_nystrom_fwd_bwd_host(p, bufs, hin[i]["Q"], hin[i]["K"], hin[i]["V"], hin[i]["dO"], hout[i]["O"],
+                                                hout[i]["dQ"], hout[i]["dK"], hout[i]["dV"], stream=st)
+            st.synchronize()
+            for i in (0, 1):
+                for k in ("O", "dQ", "dK", "dV"):
+                    assert torch.equal(hout[i][k], refs[i][k].cpu()), (rep, i, k)
+                    hout[i][k].zero_()
+    finally:
+        ln.set_overlap(was)
+
+
 @pytest.mark.parametrize("name,B", [("cfg1", 1), ("cfg2", 5), ("cfg3", 2), ("cfg4a", 1), ("cfg5_m256_T4", 1)])
 def test_whiten_stats_match_the_oracle(name, B):
     """Eq. 5-6 on the device (from the kernel block the forward pass saved) against the float64 oracle applied to the
