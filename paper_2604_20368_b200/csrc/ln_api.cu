@@ -812,9 +812,23 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     if (chq + chs >= 16) LN_LAUNCH("k_reduce3", st, k_reduce3_wide<float><<<dim3(cdiv(md, 128), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, w.dLtot, md));
     else LN_LAUNCH("k_reduce3", st, k_reduce3<float><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, w.dLtot, md));
     LN_LAUNCH("k_pool_bwd", st, k_pool_bwd<T><<<dim3(cdiv((long long)n * (D / 4), 256 * POOL_EPT), BH), 256, 0, st>>>(w.dKpart, w.dLtot, poolQ ? dQ : dK, geom_of(p), 1));
-    if (p->lm_filter)            // gradient of the selection filter, summed over the batch elements of a head
-      LN_LAUNCH("k_filter_grad", st, k_filter_grad<T><<<dim3((p->gh / p->mh) * (p->gw / p->mw), p->H), 256, 0, st>>>(poolQ ? Q : K, w.dLtot, p->lm_filter_grad,
-                                                                                                                 geom_of(p), p->B));
+    if (p->lm_filter) {          // gradient of the selection filter, summed over the batch elements of a head
+      const int taps = (p->gh / p->mh) * (p->gw / p->mw);
+      // the (batch element, landmark) pairs are split over enough CTAs to fill the GPU; the partial sums go to the query-side
+      // landmark partials of the sign pass, which k_reduce3 has consumed by now
+      const long long room = (long long)BH * chq * m * D / ((long long)p->H * taps * D);
+      long long splits = cdiv(4ll * kSMs, (long long)taps * p->H);
+      if (splits > (long long)p->B * m / 64) splits = (long long)p->B * m / 64;
+      if (splits > room) splits = room;
+      if (splits > 65535) splits = 65535;
+      if (splits < 1) splits = 1;
+      float* fpart = splits > 1 ? w.dLCpart : p->lm_filter_grad;
+      LN_LAUNCH("k_filter_grad", st, k_filter_grad<T><<<dim3(taps, p->H, (unsigned)splits), 256, 0, st>>>(poolQ ? Q : K, w.dLtot, fpart, geom_of(p), p->B));
+      if (splits > 1) {
+        const int count = p->H * taps * D;
+        LN_LAUNCH("k_filter_reduce", st, k_filter_reduce<<<cdiv(count, 1024), 256, 0, st>>>(w.dLCpart, (int)splits, p->lm_filter_grad, count));
+      }
+    }
   } else {
     if (chq + chs >= 16) LN_LAUNCH("k_reduce3", st, k_reduce3_wide<T><<<dim3(cdiv(md, 128), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, dL, md));
     else LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(md, 1024), BH), 256, 0, st>>>(w.dLCpart, chq, w.dLRpart, chs, w.dLW, 1, dL, md));

@@ -526,7 +526,9 @@ __global__ void __launch_bounds__(256) k_reduce3_wide(const float* __restrict__ 
 
 // Gradient of the landmark-selection filter: dF[h][tap][c] = sum over the batch elements b and the landmarks l of
 // dL[b H + h][l][c] X[b H + h][token(l, tap)][c], X the tensor the landmarks were selected from.
-// grid (taps, H); 256 threads = d/4 channel quads x 1024/d lanes over the (b, l) pairs; double sums, lanes added in order.
+// grid (taps, H, splits); 256 threads = d/4 channel quads x 1024/d lanes over the (b, l) pairs of this split; double sums,
+// lanes added in order.  With splits > 1 the CTAs write partial sums [split][H][taps][d] that k_filter_reduce adds up in a
+// fixed order (taps x H alone are too few CTAs where the batch is large).
 template <typename T>
 __global__ void __launch_bounds__(256) k_filter_grad(const T* __restrict__ X, const float* __restrict__ dL, float* __restrict__ dF,
                                                      PoolGeom g, int B) {
@@ -535,21 +537,50 @@ __global__ void __launch_bounds__(256) k_filter_grad(const T* __restrict__ X, co
   const int tap = blockIdx.x, h = blockIdx.y, qd = (int)threadIdx.x % quads, tl = (int)threadIdx.x / quads, c = qd * 4;
   const int rh = g.gh / g.mh, rw = g.gw / g.mw, u = tap / rw, v = tap % rw;
   double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-  if (tl < lanes)
-    for (int t = tl; t < B * g.m; t += lanes) {
+  const int pairs = B * g.m, per = (pairs + (int)gridDim.z - 1) / (int)gridDim.z;
+  const int t_beg = (int)blockIdx.z * per, t_end = min(pairs, t_beg + per);
+  if (tl < lanes) {
+    auto addr = [&](int t, const T*& xp, const float*& lp) {
       const int b = t / g.m, l = t % g.m, a = l / g.mw, bb = l % g.mw;
       const long long bh = (long long)b * g.H + h;
-      const float4 x = ld4(X + (bh * g.n + g.prefix + (a * rh + u) * g.gw + (bb * rw + v)) * g.d + c);
-      const float4 dl = ld4(dL + (bh * g.m + l) * g.d + c);
+      xp = X + (bh * g.n + g.prefix + (a * rh + u) * g.gw + (bb * rw + v)) * g.d + c;
+      lp = dL + (bh * g.m + l) * g.d + c;
+    };
+    int t = t_beg + tl;
+    for (; t + 3 * lanes < t_end; t += 4 * lanes) {        // four pairs in flight per thread
+      float4 x[4], dl[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const T* xp; const float* lp;
+        addr(t + q * lanes, xp, lp);
+        x[q] = ld4(xp); dl[q] = ld4(lp);
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        s0 += (double)dl[q].x * (double)x[q].x; s1 += (double)dl[q].y * (double)x[q].y;
+        s2 += (double)dl[q].z * (double)x[q].z; s3 += (double)dl[q].w * (double)x[q].w;
+      }
+    }
+    for (; t < t_end; t += lanes) {
+      const T* xp; const float* lp;
+      addr(t, xp, lp);
+      const float4 x = ld4(xp), dl = ld4(lp);
       s0 += (double)dl.x * (double)x.x; s1 += (double)dl.y * (double)x.y; s2 += (double)dl.z * (double)x.z; s3 += (double)dl.w * (double)x.w;
     }
+  }
   red[threadIdx.x][0] = s0; red[threadIdx.x][1] = s1; red[threadIdx.x][2] = s2; red[threadIdx.x][3] = s3;
   __syncthreads();
   if (tl == 0) {
     double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
     for (int w = 0; w < lanes; ++w) { const double* p = red[w * quads + qd]; t0 += p[0]; t1 += p[1]; t2 += p[2]; t3 += p[3]; }
-    st4(dF + ((long long)h * (rh * rw) + tap) * g.d + c, make_float4((float)t0, (float)t1, (float)t2, (float)t3));
+    st4(dF + (((long long)blockIdx.z * g.H + h) * (rh * rw) + tap) * g.d + c, make_float4((float)t0, (float)t1, (float)t2, (float)t3));
   }
+}
+// dF[e] = sum over the splits of part[split][e], in order; count = H taps d (a multiple of 4)
+__global__ void __launch_bounds__(256) k_filter_reduce(const float* __restrict__ part, int splits, float* __restrict__ dF, int count) {
+  const int e = (blockIdx.x * 256 + threadIdx.x) * 4;
+  if (e >= count) return;
+  st4(dF + e, sum_parts4(part, splits, count, e));
 }
 
 // out[e] = sum_p parts[p][e] for up to three part arrays laid out [BH][np][count]; count % 4 == 0
