@@ -521,7 +521,9 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
                                  whiten_eff, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, Mparts_src, Mparts, x.M, x.Y, x.Yt,
                                  x.ybar, dev_status, pl.hslot, umma_prod ? reinterpret_cast<bf16*>(x.Yimg) : nullptr, phase));
     };
-    if (two) launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));          // general (non-symmetric) matrix: mma.sync or FFMA engine
+    // general (non-symmetric) matrix: the mma.sync or FFMA engine, shared by the CTAs of a cluster beyond 64 landmarks
+    if (two && m > 64) launch(k_mid_fwd<D, TC, 0, kMidCluster>, sizeof(NsSmem), kMidCluster);
+    else if (two) launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));
     else if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * kUmmaMatBytes64);
     else if (TC && m <= 128) launch(k_mid_fwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
     else if (TC) launch(k_mid_fwd<D, TC, TC ? 256 : 0, TC ? kMidCluster : 1>, 3 * kUmmaMatBytes, kMidCluster);   // m > 128: a cluster per head
@@ -666,7 +668,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   };
   // The per-head kernel and the landmark-block sign pass need Z'^T dO only: with a side stream they run beside
   // the query-side kernels and are joined before the key side, which needs dM.
-  const Side side = side_acquire(!two && std::is_same<T, bf16>::value, st);
+  const Side side = side_acquire(std::is_same<T, bf16>::value, st);
   const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);
   auto launch_mid = [&](cudaStream_t s) {
     constexpr bool TC = std::is_same<T, bf16>::value;
@@ -677,7 +679,8 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
                                                  w.Hm, w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot,
                                                  umma_prod ? reinterpret_cast<bf16*>(w.dMimg) : nullptr, two ? 0 : 1));
     };
-    if (two) launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
+    if (two && m > 64) launch(k_mid_bwd<D, TC, 0, kMidCluster>, sizeof(NsSmem), kMidCluster);
+    else if (two) launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
     else if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 4 * kUmmaMatBytes64);
     else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
     else if (TC) launch(k_mid_bwd<D, TC, TC ? 256 : 0, TC ? kMidCluster : 1>, 3 * kUmmaMatBytes, kMidCluster);
