@@ -592,7 +592,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // O = (C - mu) Ytilde + ybar
   if constexpr (std::is_same<T, bf16>::value && (D == 64 || D == 128)) {
     if (epi && epi->src) {
-      const size_t smem = nn_umma_smem_dwc<D>();
+      const size_t smem = nn_umma_stage_dwc<D>() + (size_t)epi->ks * epi->ks * D * sizeof(float);
       want_smem(k_nn_umma<D, true>, smem);
       LN_LAUNCH("nn_O", st, k_nn_umma<D, true><<<dim3(cdiv(n, 128), BH), 256, smem, st>>>(x.C, pl.ldm, p->map_mode == 1 ? x.mu : nullptr,
                                                                                       reinterpret_cast<const bf16*>(x.Yimg), x.ybar, O, n, m, dev_status, *epi));
@@ -703,7 +703,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     if constexpr (std::is_same<T, bf16>::value) {
       if constexpr (D == 64 || D == 128) {
         if (epi && epi->src) {
-          const size_t smem = nn_umma_smem_dwc<D>();
+          const size_t smem = nn_umma_stage_dwc<D>() + (size_t)epi->ks * epi->ks * D * sizeof(float);
           want_smem(k_nn_umma<D, true>, smem);
           LN_LAUNCH("nn_dV", s, k_nn_umma<D, true><<<dim3(cdiv(n, 128), BH), 256, smem, s>>>(x.Rt, pl.ldm, nullptr, reinterpret_cast<const bf16*>(w.dMimg),
                                                                                          nullptr, dV, n, m, dev_status, *epi));
@@ -1364,13 +1364,19 @@ int validate_block(const ln_problem* p, const ln_block* b) {
   return LN_OK;
 }
 size_t tensor_bytes(const ln_problem* p) { return align_up((size_t)p->B * p->H * p->n * p->d * (p->dtype == LN_F32 ? 4 : 2), 256); }
-constexpr int kDwcTokensPerChunk = 512;
-int dwc_chunks(const ln_problem* p) { return (p->gh * p->gw + kDwcTokensPerChunk - 1) / kDwcTokensPerChunk; }
+// tokens per chunk of the filter-gradient partial sums: at least 512, at most 32 chunks per head
+int dwc_tokens_per_chunk(const ln_problem* p) { const int g = p->gh * p->gw, t = (g + 31) / 32; return t < 512 ? 512 : t; }
+int dwc_chunks(const ln_problem* p) { const int t = dwc_tokens_per_chunk(p); return (p->gh * p->gw + t - 1) / t; }
+// rotation table of a call (at the end of the block workspace): one (cos, sin) pair of doubles per grid position and channel pair
+size_t rope_table_bytes(const ln_problem* p) { return align_up((size_t)p->gh * p->gw * (p->d / 2) * sizeof(double2), 256); }
+void launch_rope_table(const ln_problem* p, const ln_block* b, double2* tab, cudaStream_t st) {
+  const long long cnt = (long long)p->gh * p->gw * (p->d / 2);
+  LN_LAUNCH("rope_table", st, k_rope_table<<<cdiv(cnt, 256), 256, 0, st>>>(tab, cnt, p->d, log2((double)b->rope_base)));
+}
 template <typename T>
-void launch_rope(const char* name, const ln_problem* p, const ln_block* b, const void* X, void* out, double sign, cudaStream_t st) {
+void launch_rope(const char* name, const ln_problem* p, const double2* tab, const void* X, void* out, double sign, cudaStream_t st) {
   const long long rows = (long long)p->B * p->H * p->n;
-  LN_LAUNCH(name, st, k_rope<T><<<cdiv(rows * (p->d / 4), 256), 256, 0, st>>>((const T*)X, (T*)out, rows, p->n, p->d, p->prefix,
-                                                                             log2((double)b->rope_base), sign));
+  LN_LAUNCH(name, st, k_rope<T><<<cdiv(rows * (p->d / 4), 256), 256, 0, st>>>((const T*)X, (T*)out, rows, p->n, p->d, p->prefix, tab, sign));
 }
 // the tcgen05 product kernels (bf16 storage, 64 or 128 dims) take the convolution branch into their epilogue
 inline bool dwc_in_epilogue(const ln_problem* p) { return p->dtype == LN_BF16 && (p->d == 64 || p->d == 128); }
@@ -1392,6 +1398,8 @@ size_t laplace_attention_block_workspace_bytes(const ln_problem* p, const ln_blo
   size_t ws = laplace_nystrom_workspace_bytes(p, 1);
   if (b->rope_base > 0.f) ws += 2 * tensor_bytes(p);                           // gradients with respect to the rotated Q and K
   if (b->dwc_w) ws += align_up((size_t)p->B * p->H * dwc_chunks(p) * p->d * b->dwc_ks * b->dwc_ks * sizeof(float), 256);
+  ws = align_up(ws, 256);
+  if (b->rope_base > 0.f) ws += rope_table_bytes(p);                           // the rotation table, last
   return ws;
 }
 
@@ -1410,8 +1418,10 @@ int laplace_attention_block_fwd(const ln_problem* p, const ln_block* b, const vo
   if (b->rope_base > 0.f) {
     s = check_fwd_args(p, sv, sv + tb, V, nullptr, O, sv + 2 * tb, ws, ws_bytes);
     if (s != LN_OK) return s;
-    if (p->dtype == LN_F32) { launch_rope<float>("rope_Q", p, b, Q, sv, 1.f, st); launch_rope<float>("rope_K", p, b, K, sv + tb, 1.f, st); }
-    else { launch_rope<bf16>("rope_Q", p, b, Q, sv, 1.f, st); launch_rope<bf16>("rope_K", p, b, K, sv + tb, 1.f, st); }
+    double2* tab = reinterpret_cast<double2*>(static_cast<char*>(ws) + laplace_attention_block_workspace_bytes(p, b) - rope_table_bytes(p));
+    launch_rope_table(p, b, tab, st);
+    if (p->dtype == LN_F32) { launch_rope<float>("rope_Q", p, tab, Q, sv, 1.f, st); launch_rope<float>("rope_K", p, tab, K, sv + tb, 1.f, st); }
+    else { launch_rope<bf16>("rope_Q", p, tab, Q, sv, 1.f, st); launch_rope<bf16>("rope_K", p, tab, K, sv + tb, 1.f, st); }
     q = sv; k = sv + tb; inner_saved = sv + 2 * tb;
   }
   // the convolution branch rides in the epilogue of the O product where that product is the tcgen05 kernel; else its own pass
@@ -1448,21 +1458,23 @@ int laplace_attention_block_bwd(const ln_problem* p, const ln_block* b, const vo
                 fused_dwc ? &epi : nullptr);
   if (s != LN_OK) return s;
   if (rope) {
-    if (p->dtype == LN_F32) { launch_rope<float>("rope_dQ", p, b, dq, dQ, -1.f, st); launch_rope<float>("rope_dK", p, b, dk, dK, -1.f, st); }
-    else { launch_rope<bf16>("rope_dQ", p, b, dq, dQ, -1.f, st); launch_rope<bf16>("rope_dK", p, b, dk, dK, -1.f, st); }
+    double2* tab = reinterpret_cast<double2*>(w + laplace_attention_block_workspace_bytes(p, b) - rope_table_bytes(p));
+    launch_rope_table(p, b, tab, st);
+    if (p->dtype == LN_F32) { launch_rope<float>("rope_dQ", p, tab, dq, dQ, -1.f, st); launch_rope<float>("rope_dK", p, tab, dk, dK, -1.f, st); }
+    else { launch_rope<bf16>("rope_dQ", p, tab, dq, dQ, -1.f, st); launch_rope<bf16>("rope_dK", p, tab, dk, dK, -1.f, st); }
   }
   if (b->dwc_w) {
     const int ch = dwc_chunks(p), BH = p->B * p->H, cnt = p->d * b->dwc_ks * b->dwc_ks;
     if (p->dtype == LN_F32) {
       launch_dwc_add<float>("dwc_dV", p, b, dO, dV, 1, st);
-      LN_LAUNCH("dwc_wgrad", st, k_dwc_wgrad<float><<<dim3(ch, BH), 128, 0, st>>>((const float*)V, (const float*)dO, wpart, p->n, p->d, p->prefix,
-                                                                                 p->gh, p->gw, b->dwc_ks, kDwcTokensPerChunk));
+      LN_LAUNCH("dwc_wgrad", st, k_dwc_wgrad<float><<<dim3(ch, BH, b->dwc_ks), 256, 0, st>>>((const float*)V, (const float*)dO, wpart, p->n, p->d, p->prefix,
+                                                                                            p->gh, p->gw, b->dwc_ks, dwc_tokens_per_chunk(p)));
     } else {
       if (!fused_dwc) launch_dwc_add<bf16>("dwc_dV", p, b, dO, dV, 1, st);
-      LN_LAUNCH("dwc_wgrad", st, k_dwc_wgrad<bf16><<<dim3(ch, BH), 128, 0, st>>>((const bf16*)V, (const bf16*)dO, wpart, p->n, p->d, p->prefix,
-                                                                                p->gh, p->gw, b->dwc_ks, kDwcTokensPerChunk));
+      LN_LAUNCH("dwc_wgrad", st, k_dwc_wgrad<bf16><<<dim3(ch, BH, b->dwc_ks), 256, 0, st>>>((const bf16*)V, (const bf16*)dO, wpart, p->n, p->d, p->prefix,
+                                                                                           p->gh, p->gw, b->dwc_ks, dwc_tokens_per_chunk(p)));
     }
-    LN_LAUNCH("dwc_wreduce", st, k_dwc_wreduce<<<dim3(cdiv(cnt, 256), p->H), 256, 0, st>>>(wpart, dWd, p->B, p->H, ch, cnt));
+    LN_LAUNCH("dwc_wreduce", st, k_dwc_wreduce<<<dim3(cdiv(cnt, 128), p->H), 256, 0, st>>>(wpart, dWd, p->B, p->H, ch, cnt));
   }
   return launch_ok();
 }

@@ -16,9 +16,22 @@ template <typename T> __device__ __forceinline__ T from_d(double x);
 template <> __device__ __forceinline__ float from_d<float>(double x) { return (float)x; }
 template <> __device__ __forceinline__ bf16 from_d<bf16>(double x) { return __double2bfloat16(x); }
 
+// Table of the rotations: tab[pos][i] = (cos, sin) of pos * base^(-2i/d) in double, pos over the token grid, i over the
+// d / 2 channel pairs.  Every head and batch element of a call turns by the same angles, so the double-precision
+// sine and cosine are formed once per (position, pair) instead of once per element.
+__global__ void __launch_bounds__(256) k_rope_table(double2* __restrict__ tab, long long count, int d, double log2_base) {
+  const long long e = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (e >= count) return;
+  const int i = (int)(e % (d / 2));
+  const double pos = (double)(e / (d / 2));
+  double sn, cs;
+  sincos(pos * exp2(-(double)(2 * i) / (double)d * log2_base), &sn, &cs);
+  tab[e] = make_double2(cs, sn);
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) k_rope(const T* __restrict__ X, T* __restrict__ out, long long rows, int n, int d,
-                                             int prefix, double log2_base, double sign) {
+                                             int prefix, const double2* __restrict__ tab, double sign) {
   const long long e = (long long)blockIdx.x * 256 + threadIdx.x;
   const int quads = d / 4;
   if (e >= rows * quads) return;
@@ -27,11 +40,9 @@ __global__ void __launch_bounds__(256) k_rope(const T* __restrict__ X, T* __rest
   const float4 v = ld4(X + row * d + c);
   T* o = out + row * d + c;
   if (t < prefix) { st4(o, v); return; }
-  const double pos = (double)(t - prefix);
-  double s0, c0, s1, c1;
-  sincos(pos * exp2(-(double)c / (double)d * log2_base), &s0, &c0);             // pair index i = c / 2: exponent -2i/d = -c/d
-  sincos(pos * exp2(-(double)(c + 2) / (double)d * log2_base), &s1, &c1);
-  s0 *= sign; s1 *= sign;
+  const double2* tp = tab + (long long)(t - prefix) * (d / 2) + c / 2;         // pairs c / 2 and c / 2 + 1
+  const double2 r0 = tp[0], r1 = tp[1];
+  const double c0 = r0.x, s0 = r0.y * sign, c1 = r1.x, s1 = r1.y * sign;
   const double a0 = v.x, b0 = v.y, a1 = v.z, b1 = v.w;
   o[0] = from_d<T>(a0 * c0 - b0 * s0);
   o[1] = from_d<T>(a0 * s0 + b0 * c0);
@@ -70,48 +81,78 @@ __global__ void __launch_bounds__(256) k_dwc_add(const T* __restrict__ src, cons
   st4(op, acc);
 }
 
-// Filter gradient, partial over a chunk of grid tokens: part[bh][chunk][c][tap] = sum_{tokens of the chunk}
-// dO[token][c] V[neighbour(token, tap)][c].  grid (chunks, BH), block = d threads (thread = channel), ks <= 7.
+// Filter gradient, partial over a chunk of grid tokens and one row a of the filter:
+//   part[bh][chunk][c][a ks + b] = sum_{tokens of the chunk} dO[token][c] V[neighbour(token, (a, b))][c].
+// grid (chunks, BH, ks); 256 threads = d / 4 channel quads x 1024 / d token lanes: a thread walks the tokens lane,
+// lane + lanes, ... of the chunk with the ks taps of its filter row for four channels in registers; the lanes are added
+// in a fixed order through shared memory.
 template <typename T>
-__global__ void __launch_bounds__(128) k_dwc_wgrad(const T* __restrict__ V, const T* __restrict__ dO, float* __restrict__ part,
+__global__ void __launch_bounds__(256) k_dwc_wgrad(const T* __restrict__ V, const T* __restrict__ dO, float* __restrict__ part,
                                                   int n, int d, int prefix, int gh, int gw, int ks, int tpc) {
-  const int chunk = blockIdx.x, bh = blockIdx.y, c = threadIdx.x, half = ks / 2;
-  if (c >= d) return;
-  float acc[49];
+  __shared__ float red[256][7][4];
+  const int chunk = blockIdx.x, bh = blockIdx.y, a = blockIdx.z, half = ks / 2;
+  const int quads = d / 4, lanes = 256 / quads, q = (int)threadIdx.x % quads, tl = (int)threadIdx.x / quads, c = 4 * q;
+  float acc[7][4];
 #pragma unroll
-  for (int t = 0; t < 49; ++t) acc[t] = 0.f;
+  for (int b = 0; b < 7; ++b)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) acc[b][e] = 0.f;
   const T* Vh = V + (long long)bh * n * d + c;
   const T* Gh = dO + (long long)bh * n * d + c;
   const int t0 = chunk * tpc, t1 = min(gh * gw, t0 + tpc);
-  for (int tok = t0; tok < t1; ++tok) {
-    const int r = tok / gw, q = tok % gw;
-    const float g = to_f(Gh[(long long)(prefix + tok) * d]);
-#pragma unroll
-    for (int a = 0; a < 7; ++a)
+  if (tl < lanes)
+    for (int tok = t0 + tl; tok < t1; tok += lanes) {
+      const int r = tok / gw, q0 = tok % gw, rr = r + a - half;
+      if (rr < 0 || rr >= gh) continue;
+      const float4 g = ld4(Gh + (long long)(prefix + tok) * d);
 #pragma unroll
       for (int b = 0; b < 7; ++b) {
-        if (a < ks && b < ks) {
-          const int rr = r + a - half, qq = q + b - half;
-          if (rr >= 0 && rr < gh && qq >= 0 && qq < gw) acc[a * 7 + b] += g * to_f(Vh[(long long)(prefix + rr * gw + qq) * d]);
+        const int qq = q0 + b - half;
+        if (b < ks && qq >= 0 && qq < gw) {
+          const float4 v = ld4(Vh + (long long)(prefix + rr * gw + qq) * d);
+          acc[b][0] += g.x * v.x; acc[b][1] += g.y * v.y; acc[b][2] += g.z * v.z; acc[b][3] += g.w * v.w;
         }
       }
+    }
+#pragma unroll
+  for (int b = 0; b < 7; ++b)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) red[threadIdx.x][b][e] = acc[b][e];
+  __syncthreads();
+  if (tl == 0) {
+    float* o = part + (((long long)bh * gridDim.x + chunk) * d + c) * ks * ks + a * ks;
+    for (int b = 0; b < ks; ++b)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float s = 0.f;
+        for (int w = 0; w < lanes; ++w) s += red[w * quads + q][b][e];
+        o[(long long)e * ks * ks + b] = s;
+      }
   }
-  float* o = part + (((long long)bh * gridDim.x + chunk) * d + c) * ks * ks;
-#pragma unroll
-  for (int a = 0; a < 7; ++a)
-#pragma unroll
-    for (int b = 0; b < 7; ++b)
-      if (a < ks && b < ks) o[a * ks + b] = acc[a * 7 + b];
 }
 
-// dW[h][e] = sum over the batch elements b and the chunks of part[b H + h][chunk][e], in a fixed order; e < d ks ks
+// dW[h][e] = sum over the batch elements b and the chunks of part[b H + h][chunk][e]; e < count = d ks ks (a multiple of 4).
+// grid (ceil(count / 128), H): warp w of a CTA adds the parts w, w + 8, ... for 128 consecutive elements, the eight warps
+// are added in a fixed order.
 __global__ void __launch_bounds__(256) k_dwc_wreduce(const float* __restrict__ part, float* __restrict__ dW, int B, int H, int chunks, int count) {
-  const int h = blockIdx.y, e = blockIdx.x * 256 + threadIdx.x;
-  if (e >= count) return;
-  float s = 0.f;
-  for (int b = 0; b < B; ++b)
-    for (int k = 0; k < chunks; ++k) s += part[(((long long)(b * H + h)) * chunks + k) * count + e];
-  dW[(long long)h * count + e] = s;
+  __shared__ float4 red[8][32];
+  const int h = blockIdx.y, w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  const int e = (blockIdx.x * 32 + l) * 4, P = B * chunks;
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (e < count)
+    for (int p = w; p < P; p += 8) {
+      const int b = p / chunks, k = p % chunks;
+      const float4 v = *reinterpret_cast<const float4*>(part + (((long long)(b * H + h)) * chunks + k) * count + e);
+      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+  red[w][l] = s;
+  __syncthreads();
+  if (w == 0 && e < count) {
+    float4 t = red[0][l];
+#pragma unroll
+    for (int k = 1; k < 8; ++k) { t.x += red[k][l].x; t.y += red[k][l].y; t.z += red[k][l].z; t.w += red[k][l].w; }
+    *reinterpret_cast<float4*>(dW + (long long)h * count + e) = t;
+  }
 }
 
 }  // namespace ln

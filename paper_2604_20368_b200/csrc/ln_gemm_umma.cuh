@@ -39,9 +39,11 @@ __device__ __forceinline__ void gu_write_images(const float* __restrict__ src, b
 // shared memory of k_nn_umma: E block images and Y block images; the bf16 staging of the output tile reuses them
 template <int D> __host__ __device__ constexpr size_t nn_umma_smem() { return (size_t)(2 * 128 * GU_KB + 2 * GU_KB * D) * sizeof(bf16); }
 // with the convolution branch in the epilogue the output tile is staged in fp32 (one rounding, after the branch is added)
-template <int D> __host__ __device__ constexpr size_t nn_umma_smem_dwc() {
+// (behind the staged tile: the head's filters, transposed to [tap][channel], up to 7 x 7 taps)
+template <int D> __host__ __device__ constexpr size_t nn_umma_stage_dwc() {
   return nn_umma_smem<D>() > (size_t)128 * (D + 4) * sizeof(float) ? nn_umma_smem<D>() : (size_t)128 * (D + 4) * sizeof(float);
 }
+template <int D> __host__ __device__ constexpr size_t nn_umma_smem_dwc() { return nn_umma_stage_dwc<D>() + (size_t)49 * D * sizeof(float); }
 
 // One 128-token tile per CTA; three CTAs per SM hide each other's load latencies.
 // DWC: the depth-wise convolution branch of the attention block (Eq. 7) is added in the epilogue, before the one rounding
@@ -147,11 +149,15 @@ __global__ void __launch_bounds__(256, 3) k_nn_umma(const float* __restrict__ E,
         }
       }
     }
+    const int kk = epi.ks * epi.ks, half = epi.ks / 2;
+    float* wsm = reinterpret_cast<float*>(gu_smem + nn_umma_stage_dwc<D>());     // [tap][D]
+    {
+      const float* wh = epi.w + (long long)(bh % epi.H) * D * kk;
+      for (int e = tid; e < D * kk; e += 256) wsm[(e % kk) * D + e / kk] = wh[e];
+    }
     umma::fence_before_sync();
     __syncthreads();
     const bf16* src = static_cast<const bf16*>(epi.src) + (long long)bh * n * D;
-    const int kk = epi.ks * epi.ks, half = epi.ks / 2;
-    const float* wh = epi.w + (long long)(bh % epi.H) * D * kk;
     for (int p = tid; p < 128 * (D / 8); p += 256) {
       const int r = p / (D / 8), c8 = (p % (D / 8)) * 8, i = i0 + r;
       if (i >= n) continue;
@@ -169,10 +175,12 @@ __global__ void __launch_bounds__(256, 3) k_nn_umma(const float* __restrict__ E,
             const int tap = epi.flip ? (epi.ks - 1 - a) * epi.ks + (epi.ks - 1 - b) : a * epi.ks + b;
             const uint4 v = *reinterpret_cast<const uint4*>(src + (long long)(epi.prefix + rr * epi.gw + qq) * D + c8);
             const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
+            const float4 w0 = *reinterpret_cast<const float4*>(wsm + tap * D + c8), w1 = *reinterpret_cast<const float4*>(wsm + tap * D + c8 + 4);
+            const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              acc[2 * e] = fmaf(__ldg(wh + (c8 + 2 * e) * kk + tap), __uint_as_float(vw[e] << 16), acc[2 * e]);
-              acc[2 * e + 1] = fmaf(__ldg(wh + (c8 + 2 * e + 1) * kk + tap), __uint_as_float(vw[e] & 0xffff0000u), acc[2 * e + 1]);
+              acc[2 * e] = fmaf(wv[2 * e], __uint_as_float(vw[e] << 16), acc[2 * e]);
+              acc[2 * e + 1] = fmaf(wv[2 * e + 1], __uint_as_float(vw[e] & 0xffff0000u), acc[2 * e + 1]);
             }
           }
         }
