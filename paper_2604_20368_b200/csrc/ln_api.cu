@@ -457,7 +457,17 @@ L1Prob l1_prob(const void* A, int a_f32, float* E, float* rowsum, int na, int d,
 void launch_l1_args(const char* name, L1Args& a, int nprob, int batch, cudaStream_t st) {
   int na_max = 0;
   for (int i = 0; i < nprob; ++i) na_max = a.p[i].na > na_max ? a.p[i].na : na_max;
-  const L1Launch l = plan_l1(na_max, a.nb, a.d, batch, nprob);
+  L1Launch l = plan_l1(na_max, a.nb, a.d, batch, nprob);
+  // a single block without row sums (the stand-alone entry point on few, large matrices): the landmark range is split
+  // over blockIdx.z until the launch has about two CTAs per SM
+  a.jsplits = 1;
+  if (nprob == 1 && !a.p[0].rowsum && !a.p[0].stat) {
+    const long long ctas = (long long)l.grid.x * l.grid.y, tb = (long long)l.qn * l.block.x;
+    long long sp = (2ll * sm_count() + ctas - 1) / ctas;
+    const long long tiles = (a.nb + tb - 1) / tb;
+    if (sp > tiles) sp = tiles;
+    if (sp > 1) { a.jsplits = (int)sp; l.grid.z = (unsigned)sp; }
+  }
   if (l.qn == 4) {
     want_smem(k_l1<4>, l.smem);
     LN_LAUNCH(name, st, k_l1<4><<<l.grid, l.block, l.smem, st>>>(a));
@@ -890,15 +900,24 @@ void launch_ns_pinv(int batch, int m, int iters, float eps, float alpha, const f
 }  // namespace
 
 namespace {
-struct L1BwdWs { float *Kmat, *G, *part; int rpc, chunks; size_t bytes; };
+struct L1BwdWs { float *Kmat, *part, *rowpart; int rpc, chunks, lper, lsplits; size_t bytes; };
 L1BwdWs carve_l1bwd(int batch, int na, int nb, int d, void* base) {
   Carver c(base); L1BwdWs w;
-  int want = (2 * sm_count() + batch - 1) / batch; if (want < 1) want = 1;
+  // rows of A per CTA of the pass over the columns: whole 64-column tiles, about two CTAs per SM in all
+  const int coltiles = (nb + 63) / 64;
+  int want = (2 * sm_count() + batch * coltiles - 1) / (batch * coltiles); if (want < 1) want = 1;
   int rpc = (na + want - 1) / want; rpc = (rpc + 31) / 32 * 32;
   w.rpc = rpc; w.chunks = (na + rpc - 1) / rpc;
+  // columns per CTA of the pass over the rows: split while the 64-row tiles alone are fewer than two CTAs per SM
+  const int rowtiles = (na + 63) / 64;
+  int sp = (2 * sm_count() + batch * rowtiles - 1) / (batch * rowtiles);
+  if (sp > (nb + 31) / 32) sp = (nb + 31) / 32;
+  if (sp < 1) sp = 1;
+  w.lper = ((nb + sp - 1) / sp + 31) / 32 * 32;
+  w.lsplits = (nb + w.lper - 1) / w.lper;
   w.Kmat = c.take((size_t)batch * na * nb);
-  w.G = c.take((size_t)batch * na * nb);
   w.part = c.take((size_t)batch * w.chunks * nb * d);
+  w.rowpart = c.take(w.lsplits > 1 ? (size_t)batch * w.lsplits * na * d : 0);
   w.bytes = c.off;
   return w;
 }
@@ -906,10 +925,15 @@ template <typename T, int D>
 void l1_bwd_impl(int batch, int na, int nb, const T* A, const T* Bm, float lambda, const float* Kmat, const float* dK,
                  T* dA, T* dB, const L1BwdWs& w, cudaStream_t st) {
   if (!Kmat) { launch_l1<T, T>("l1_kernel", A, Bm, w.Kmat, nullptr, batch, na, nb, D, nb, lambda, st); Kmat = w.Kmat; }
-  const long long cnt = (long long)batch * na * nb;
-  LN_LAUNCH("k_g_elem", st, k_g_elem<<<cdiv(cnt, 256), 256, 0, st>>>(Kmat, dK, w.G, cnt, 1.f / lambda));
-  LN_LAUNCH("k_sign_rows", st, k_sign_rows<T, T, T, D><<<dim3(cdiv(na, 64), batch), 256, 0, st>>>(A, Bm, w.G, nb, dA, na, nb));
-  LN_LAUNCH("k_sign_cols", st, k_sign_cols<T, T, D><<<dim3(w.chunks, cdiv(nb, 64), batch), 256, 0, st>>>(A, Bm, w.G, nb, w.part, na, nb, w.rpc));
+  // the factor dK o K / lambda is formed where the two passes load their tiles of it
+  const float il = 1.f / lambda;
+  if (w.lsplits > 1) {
+    LN_LAUNCH("k_sign_rows", st, k_sign_rows<T, T, float, D><<<dim3(cdiv(na, 64), batch, w.lsplits), 256, 0, st>>>(A, Bm, dK, nb, w.rowpart, na, nb, w.lper, Kmat, il));
+    LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(na * D, 1024), batch), 256, 0, st>>>(w.rowpart, w.lsplits, nullptr, 0, nullptr, 0, dA, na * D));
+  } else {
+    LN_LAUNCH("k_sign_rows", st, k_sign_rows<T, T, T, D><<<dim3(cdiv(na, 64), batch), 256, 0, st>>>(A, Bm, dK, nb, dA, na, nb, 0, Kmat, il));
+  }
+  LN_LAUNCH("k_sign_cols", st, k_sign_cols<T, T, D><<<dim3(w.chunks, cdiv(nb, 64), batch), 256, 0, st>>>(A, Bm, dK, nb, w.part, na, nb, w.rpc, Kmat, il));
   LN_LAUNCH("k_reduce3", st, k_reduce3<T><<<dim3(cdiv(nb * D, 1024), batch), 256, 0, st>>>(w.part, w.chunks, nullptr, 0, nullptr, 0, dB, nb * D));
 }
 }  // namespace

@@ -37,6 +37,7 @@ struct L1Args {
   const void* Bm; long long sB;
   int nb, d, b_f32;
   float nscale;          // -log2(e) / lambda
+  int jsplits = 1;       // > 1 (one problem, no row sums or statistics): blockIdx.z splits the landmark range instead of naming a problem
 };
 
 // 8 consecutive elements of a row -> fp32 (zero outside [0, d)); vec: the row start is 16-byte aligned
@@ -69,7 +70,7 @@ __device__ __forceinline__ void l1_fetch8(const void* base, bool f32, long long 
 template <int QN>
 __global__ void __launch_bounds__(256, QN == 4 ? 2 : 3) k_l1(const L1Args args) {
   extern __shared__ __align__(16) float l1_smem[];
-  const L1Prob pr = args.p[blockIdx.z];
+  const L1Prob pr = args.p[args.jsplits > 1 ? 0 : blockIdx.z];
   const int LG = blockDim.x, TG = blockDim.y, tj = threadIdx.x, ti = threadIdx.y;
   const int tid = ti * LG + tj, nthr = LG * TG;
   const int TA = 8 * TG, TB = QN * LG;
@@ -85,7 +86,10 @@ __global__ void __launch_bounds__(256, QN == 4 ? 2 : 3) k_l1(const L1Args args) 
 #pragma unroll
   for (int k = 0; k < 8; ++k) rs[k] = 0.f;
 
-  for (int j0 = 0; j0 < nb; j0 += TB) {
+  // landmark tiles of this CTA: all of them, or its share of a split range (whole tiles)
+  const int jper = args.jsplits > 1 ? ((nb + args.jsplits - 1) / args.jsplits + TB - 1) / TB * TB : nb;
+  const int jbeg = args.jsplits > 1 ? (int)blockIdx.z * jper : 0, jend = min(nb, jbeg + jper);
+  for (int j0 = jbeg; j0 < jend; j0 += TB) {
     float acc[8][QN];
 #pragma unroll
     for (int k = 0; k < 8; ++k)
@@ -832,21 +836,17 @@ __global__ void __launch_bounds__(256) k_nt_g(const TU* __restrict__ U, const fl
   }
 }
 
-// G = dK o K / lambda, elementwise (stand-alone l1_kernel_bwd)
-__global__ void k_g_elem(const float* __restrict__ Kmat, const float* __restrict__ dK, float* __restrict__ G,
-                         long long count, float inv_lambda) {
-  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < count) G[i] = dK[i] * Kmat[i] * inv_lambda;
-}
-
 // =====================================================================================
 // Sign pass over the landmarks (App. A):  out[i][c] = -sum_l G[i][l] * sign(tok[i][c] - L[l][c])
-// grid (ceil(n/64), BH); thread: 4 tokens x D/16 dims, token values held in registers
-// =====================================================================================
+// grid (ceil(n/64), BH[, splits]); thread: 4 tokens x D/16 dims, token values held in registers.
+// lper > 0 (a multiple of 32): blockIdx.z takes the landmarks [z lper, (z + 1) lper) and writes the partial sum
+// out[bh][z][n][D] (few, long rows of landmarks: the stand-alone kernel gradient).  Gk != NULL: the factor is formed on
+// the fly as G[i][l] Gk[i][l] gscale (upstream gradient times kernel value over lambda).
 template <typename TT, typename TL, typename TO, int D>
 __global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, const TL* __restrict__ Lm,
                                                    const float* __restrict__ G, int ldg, TO* __restrict__ out,
-                                                   int n, int m) {
+                                                   int n, int m, int lper = 0, const float* __restrict__ Gk = nullptr,
+                                                   float gscale = 1.f) {
   constexpr int DC = D / 16;
   __shared__ __align__(16) float Ls[32][D + 4];
   __shared__ __align__(16) float Gs[64][32 + 4];
@@ -855,7 +855,9 @@ __global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, c
   tok += (long long)bh * n * D;
   Lm += (long long)bh * m * D;
   G += (long long)bh * n * ldg;
-  out += (long long)bh * n * D;
+  if (Gk) Gk += (long long)bh * n * ldg;
+  const int lbeg = lper > 0 ? (int)blockIdx.z * lper : 0, lend = lper > 0 ? min(m, lbeg + lper) : m;
+  out += lper > 0 ? ((long long)bh * gridDim.z + blockIdx.z) * n * D : (long long)bh * n * D;
   constexpr int DP = DC / 2;                 // packed pairs of adjacent dims
   f32x2 qp[4][DP], acc[4][DP];
   float gsum[4];
@@ -871,12 +873,12 @@ __global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, c
       qp[k][s] = pack2(q0, q1);
     }
   }
-  for (int l0 = 0; l0 < m; l0 += 32) {
+  for (int l0 = lbeg; l0 < lend; l0 += 32) {
     __syncthreads();
     for (int idx = tid; idx < 32 * (D / 4); idx += 256) {
       const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
       float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (l0 + r < m) v = ld4(Lm + (long long)(l0 + r) * D + c4);
+      if (l0 + r < lend) v = ld4(Lm + (long long)(l0 + r) * D + c4);
       *reinterpret_cast<float4*>(&Ls[r][c4]) = make_float4(-v.x, -v.y, -v.z, -v.w);   // negated: q - L is a packed add
     }
     {  // G tile: 64 tokens x 32 landmarks (zero outside)
@@ -884,11 +886,13 @@ __global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, c
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
         const int l = l0 + cb + k;
-        Gs[r][cb + k] = (i < n && l < m) ? G[(long long)i * ldg + l] : 0.f;
+        float gv = (i < n && l < lend) ? G[(long long)i * ldg + l] : 0.f;
+        if (Gk && i < n && l < lend) gv *= Gk[(long long)i * ldg + l] * gscale;
+        Gs[r][cb + k] = gv;
       }
     }
     __syncthreads();
-    const int lcount = min(32, (m - l0 + 3) & ~3);     // landmarks of this chunk, rounded up to 4 (the rest is zero)
+    const int lcount = min(32, (lend - l0 + 3) & ~3);  // landmarks of this chunk, rounded up to 4 (the rest is zero)
 #pragma unroll 2
     for (int ll = 0; ll < lcount; ll += 4) {
       float g[4][4];
@@ -930,7 +934,8 @@ __global__ void __launch_bounds__(256) k_sign_rows(const TT* __restrict__ tok, c
 template <typename TT, typename TL, int D>
 __global__ void __launch_bounds__(256) k_sign_cols(const TT* __restrict__ tok, const TL* __restrict__ Lm,
                                                    const float* __restrict__ G, int ldg, float* __restrict__ part,
-                                                   int n, int m, int rpc) {
+                                                   int n, int m, int rpc, const float* __restrict__ Gk = nullptr,
+                                                   float gscale = 1.f) {
   constexpr int DC = D / 16;
   __shared__ __align__(16) float Ts[32][D + 4];
   __shared__ __align__(16) float Gs[32][64 + 4];
@@ -939,6 +944,7 @@ __global__ void __launch_bounds__(256) k_sign_cols(const TT* __restrict__ tok, c
   tok += (long long)bh * n * D;
   Lm += (long long)bh * m * D;
   G += (long long)bh * n * ldg;
+  if (Gk) Gk += (long long)bh * n * ldg;
   const int ibeg = chunk * rpc, iend = min(n, ibeg + rpc);
   constexpr int DP = DC / 2;
   f32x2 nl[4][DP], acc[4][DP];                // negated landmark values, accumulators, as pairs of adjacent dims
@@ -968,7 +974,9 @@ __global__ void __launch_bounds__(256) k_sign_cols(const TT* __restrict__ tok, c
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
         const int l = l0 + cb + k;
-        Gs[r][cb + k] = (i < iend && l < m) ? G[(long long)i * ldg + l] : 0.f;
+        float gv = (i < iend && l < m) ? G[(long long)i * ldg + l] : 0.f;
+        if (Gk && i < iend && l < m) gv *= Gk[(long long)i * ldg + l] * gscale;
+        Gs[r][cb + k] = gv;
       }
     }
     __syncthreads();
