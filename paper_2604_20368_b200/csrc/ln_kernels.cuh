@@ -1243,6 +1243,91 @@ __device__ void ns_backward_tail_dev(int m, const float* Wr, const NsHdr* hdr, c
   }
 }
 
+// End of the adjoint and the landmark-block factor in one pass, for a landmark matrix that is symmetric bit for bit
+// (one landmark set) and was never written out with its ridge: Wr = W + eps I is formed where it is read.
+//   dW_total = dWacc + alpha G^T + dalpha d(alpha)/dW,   dalpha = <G, Wr^T> = <G, Wr>,
+//   GW = (dW_total o W + (dW_total o W)^T) / lambda = (F + F^T + E + E^T) o W / lambda,   F = dWacc + alpha G,
+// E the two rank-one corrections of the norm gradient (column jstar of ||.||_1, row istar of ||.||_inf).  Transposed
+// tiles go through shared memory (32 x 32, two per round); CL CTAs share the tiles.  G, dWacc: fp32 [m][m]; GW: [m][ldm],
+// columns >= m zero.  tile: >= 2 * 32 * 33 + 512 floats of shared memory.
+template <int CL>
+__device__ void ns_tail_gw_sym(int m, int ldm, const float* __restrict__ W, float eps, const NsHdr* hdr, const float* __restrict__ G,
+                               const float* __restrict__ dWacc, float inv_lambda, float* __restrict__ GW, float* red, float* tile, int crank) {
+  const int tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
+  const unsigned mm = (unsigned)m * (unsigned)m, dstep = (unsigned)m + 1u;
+  const float alpha = hdr->alpha;
+  const int js = hdr->jstar, is = hdr->istar;
+  float* sgc = tile + 2 * 32 * 33;          // sign of column jstar of Wr
+  float* sgr = sgc + 256;                   // sign of row istar of Wr
+  for (int i = tid; i < m; i += 256) {
+    const float wc = W[(long long)i * m + js] + (i == js ? eps : 0.f), wr = W[(long long)is * m + i] + (i == is ? eps : 0.f);
+    sgc[i] = wc > 0.f ? 1.f : (wc < 0.f ? -1.f : 0.f);
+    sgr[i] = wr > 0.f ? 1.f : (wr < 0.f ? -1.f : 0.f);
+  }
+  float p16[16];
+#pragma unroll
+  for (int u = 0; u < 16; ++u) p16[u] = 0.f;
+  unsigned e = (unsigned)tid;
+  for (; e + 15u * 256u < mm; e += 16u * 256u) {      // every CTA sums everything (same order, same value)
+    float g[16], w[16];
+#pragma unroll
+    for (int u = 0; u < 16; ++u) { g[u] = G[e + u * 256u]; w[u] = W[e + u * 256u]; }
+#pragma unroll
+    for (int u = 0; u < 16; ++u) p16[u] += g[u] * (w[u] + ((e + u * 256u) % dstep == 0u ? eps : 0.f));
+  }
+  for (; e < mm; e += 256u) p16[0] += G[e] * (W[e] + (e % dstep == 0u ? eps : 0.f));
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1)
+#pragma unroll
+    for (int u = 0; u < o; ++u) p16[u] += p16[u + o];
+  const float dalpha = block_sum(p16[0], red);          // ends with a barrier: sgc / sgr are complete as well
+  const float c1 = hdr->auto_alpha ? dalpha * (-alpha / hdr->n1) : 0.f, c2 = hdr->auto_alpha ? dalpha * (-alpha / hdr->ninf) : 0.f;
+  const int nti = (m + 31) / 32, ntj = (ldm + 31) / 32, ntiles = nti * ntj;
+  for (int t0 = crank; t0 < ntiles; t0 += 2 * CL) {
+    float f[2][4], w[2][4], ft[2][4];
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const int t = t0 + q * CL, I = t / ntj, J = t % ntj;
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int i = I * 32 + ty + 8 * r, j = J * 32 + tx;            // this thread's element of the tile
+        const int jj = J * 32 + ty + 8 * r, ii = I * 32 + tx;          // and of the mirrored tile
+        const bool in = t < ntiles && i < m && j < m, tin = t < ntiles && jj < m && ii < m;
+        f[q][r] = in ? dWacc[(long long)i * m + j] : 0.f;
+        ft[q][r] = in ? G[(long long)i * m + j] : 0.f;
+        w[q][r] = in ? W[(long long)i * m + j] : 0.f;
+        const float a = tin ? dWacc[(long long)jj * m + ii] : 0.f, b = tin ? G[(long long)jj * m + ii] : 0.f;
+        f[q][r] = fmaf(alpha, ft[q][r], f[q][r]);
+        ft[q][r] = fmaf(alpha, b, a);
+      }
+    }
+    __syncthreads();                                                   // the tiles of the previous round have been read
+#pragma unroll
+    for (int q = 0; q < 2; ++q)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) tile[q * (32 * 33) + (ty + 8 * r) * 33 + tx] = ft[q][r];
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const int t = t0 + q * CL, I = t / ntj, J = t % ntj;
+      if (t >= ntiles) continue;
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int i = I * 32 + ty + 8 * r, j = J * 32 + tx;
+        if (i >= m || j >= ldm) continue;
+        float sum = f[q][r] + tile[q * (32 * 33) + tx * 33 + ty + 8 * r];
+        if (j < m) {
+          if (j == js) sum += c1 * sgc[i];
+          if (i == is) sum += c2 * sgr[j];
+          if (i == js) sum += c1 * sgc[j];
+          if (j == is) sum += c2 * sgr[i];
+        }
+        GW[(long long)i * ldm + j] = (j < m) ? sum * w[q][r] * inv_lambda : 0.f;
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------ stand-alone ns_pinv / ns_pinv_bwd
 // CL CTAs of a thread-block cluster share a matrix (grid = batch * CL): every product is split by output tiles, the
 // hardware cluster barrier ends a phase.  fp32 FFMA throughout (held to 2e-5 against the oracle).
@@ -1360,25 +1445,34 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
   ns_gemm<TC, false, false>(m, D, m, XT, ldx, Mout, D, Y, D, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // Y = X M
   if (CL > 1) phase_sync<CL>();
   const float* s = whiten ? whiten + (long long)(bh % H) * m : nullptr;
-  // fold the injective map (Prop. 3): column means over the landmarks first (eight independent loads per
-  // batch), then every element in parallel
+  // fold the injective map (Prop. 3): column means over the landmarks first (256 / D thread groups share the
+  // landmarks of a column, eight independent loads per batch, the groups added in order), then every element in parallel
   float* colstat = red;            // [2][D]: mean_l s_l Y_lc and mean_l Y_lc
-  if (tid < D) {
+  {
+    constexpr int NG = 256 / D;
+    const int c = tid % D, g = tid / D;
     float sy = 0.f, y1 = 0.f;
-    for (int l0 = 0; l0 < m; l0 += 8) {
+    for (int l0 = g; l0 < m; l0 += 8 * NG) {
       float y[8], w[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
-        const int l = l0 + u;
-        y[u] = (l < m) ? Y[(long long)l * D + tid] : 0.f;
+        const int l = l0 + u * NG;
+        y[u] = (l < m) ? Y[(long long)l * D + c] : 0.f;
         w[u] = (l < m && s) ? s[l] : 1.f;
       }
 #pragma unroll
       for (int u = 0; u < 8; ++u) { sy += w[u] * y[u]; y1 += y[u]; }
     }
-    colstat[tid] = sy / (float)m;
-    colstat[D + tid] = y1 / (float)m;
-    if (crank == 0) ybar[tid] = (map_mode == 1) ? y1 / (float)m : 0.f;
+    red[tid] = sy; red[256 + tid] = y1;
+    __syncthreads();
+    if (tid < D) {                 // thread tid reads, then overwrites, slots that only it touches
+      sy = 0.f; y1 = 0.f;
+#pragma unroll
+      for (int q = 0; q < NG; ++q) { sy += red[q * D + tid]; y1 += red[256 + q * D + tid]; }
+      colstat[tid] = sy / (float)m;
+      colstat[D + tid] = y1 / (float)m;
+      if (crank == 0) ybar[tid] = (map_mode == 1) ? y1 / (float)m : 0.f;
+    }
   }
   __syncthreads();
   for (long long e = (long long)gt * 4; e < md; e += 4 * gn) {
@@ -1440,7 +1534,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     }
     *reinterpret_cast<float4*>(dY + e) = o;
   }
-  if constexpr (MP == 0 || MP == 256) {             // m <= 256: 32-bit index arithmetic (a 64-bit division costs far more)
+  if constexpr (MP == 0) {                          // m <= 256: 32-bit index arithmetic (a 64-bit division costs far more)
     for (unsigned e = (unsigned)gt; e < (unsigned)mm; e += (unsigned)gn) Wr[e] = W[e] + (e % (unsigned)(m + 1) == 0u ? eps : 0.f);
   }
   phase_sync<CL>();
@@ -1461,12 +1555,12 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     __shared__ __align__(8) unsigned long long mbar_free;
     const bool tc_ok = ns_backward_umma256(m, T, Xh, Ph, dXm, Ga, Gb, Hm, P, dWm, reinterpret_cast<bf16*>(dyn_smem), ctl, &mbar_free, crank);
     if (dev_status && !tc_ok && tid == 0 && crank == 0) atomicOr(dev_status + bh, 2);
-    ns_backward_tail_dev<CL, true>(m, Wr, hdr, P, dWm, red, crank);
-    phase_sync<CL>();
+    // end of the adjoint and GW in one pass (the operand buffers are free: the engine has ended with a cluster barrier)
+    ns_tail_gw_sym<CL>(m, ldm, W, eps, hdr, P, dWm, inv_lambda, GW, red, reinterpret_cast<float*>(dyn_smem), crank);
   } else { ns_backward_dev<TC, CL>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red, crank, Ph); if (CL > 1) phase_sync<CL>(); }
   // GW = (dW o K_LL + (dW o K_LL)^T) / lambda; four elements per batch so that the loads overlap
-  // (the single-CTA tcgen05 engines have written GW from shared memory already)
-  if constexpr (MP == 0 || MP == 256)
+  // (the tcgen05 engines have written GW already)
+  if constexpr (MP == 0)
   for (long long e0 = (long long)gt * 4; e0 < (long long)m * ldm; e0 += 4 * gn) {
     float a[4], b[4], c[4], d4[4];
 #pragma unroll

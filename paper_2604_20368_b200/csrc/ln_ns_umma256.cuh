@@ -103,8 +103,8 @@ __device__ __forceinline__ void u2_begin(U2Ctx& c, UmmaCtl& ctl, unsigned long l
   umma_begin(ctl, ncols);
 }
 
-// Forward iteration, called by the four CTAs of a cluster (crank = 0 .. 3).  W: fp32 [m][m]; Wr: fp32 scratch [m][m]
-// that receives W + eps I; Wimg: scratch slot for the images of Wr; Xh: slots 0 .. T-1 receive the images of X_k, slot T
+// Forward iteration, called by the four CTAs of a cluster (crank = 0 .. 3).  W: fp32 [m][m]; Wr: unused (W + eps I is
+// formed where it is read); Wimg: scratch slot for the images of Wr; Xh: slots 0 .. T-1 receive the images of X_k, slot T
 // X_T in fp32 [m][m]; Ph: slot k receives the images of Q_k.  Returns false if a wait ran out.
 __device__ bool ns_forward_umma256(int m, int T, float eps, float alpha_in, const float* W, float* Wr, float* Wimg,
                                    float* Xh, float* Ph, NsHdr* hdr, bf16* smem, float* red, UmmaCtl& ctl,
@@ -113,22 +113,30 @@ __device__ bool ns_forward_umma256(int m, int T, float eps, float alpha_in, cons
   const int ri = crank >> 1, ci = crank & 1;
   const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64;
   const int gi = ri * 128 + row, gj0 = ci * 128 + col0;          // this thread's row and first column in the matrix
-  const long long mm = (long long)m * m;
-  for (unsigned e = (unsigned)gt; e < (unsigned)mm; e += (unsigned)gn) Wr[e] = W[e] + (e % (unsigned)(m + 1) == 0u ? eps : 0.f);
-  phase_sync<4>();
+  // Wr = W + eps I is never written out on this path: the ridge is added where an element of the diagonal is read
+  (void)Wr;
   {
     // Norms: Wr is symmetric bit for bit (|a - b| = |b - a| term by term in the kernel block), so the absolute row sums
-    // are the absolute column sums; a column is read along the rows (threads side by side), four rows in flight.
+    // are the absolute column sums; a column is read along the rows (threads side by side), sixteen rows in flight.
     float* colsum = red;
     if (tid < m) {
-      float c4[4] = {0.f, 0.f, 0.f, 0.f};
-      int i = 0;
-      for (; i + 3 < m; i += 4) {
+      float c16[16];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) c4[u] += fabsf(Wr[(long long)(i + u) * m + tid]);
+      for (int u = 0; u < 16; ++u) c16[u] = 0.f;
+      int i = 0;
+      for (; i + 15 < m; i += 16) {
+        float w16[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) w16[u] = W[(long long)(i + u) * m + tid];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) c16[u] += fabsf(w16[u] + (i + u == tid ? eps : 0.f));
       }
-      for (; i < m; ++i) c4[0] += fabsf(Wr[(long long)i * m + tid]);
-      colsum[tid] = (c4[0] + c4[1]) + (c4[2] + c4[3]);
+      for (; i < m; ++i) c16[0] += fabsf(W[(long long)i * m + tid] + (i == tid ? eps : 0.f));
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1)
+#pragma unroll
+        for (int u = 0; u < o; ++u) c16[u] += c16[u + o];
+      colsum[tid] = c16[0];
     }
     __syncthreads();
     if (tid == 0) {               // every CTA of the cluster arrives at the same values
@@ -151,10 +159,10 @@ __device__ bool ns_forward_umma256(int m, int T, float eps, float alpha_in, cons
   {  // images of this CTA's block of Wr and of X_0 = alpha Wr^T
     float v[64];
 #pragma unroll
-    for (int q = 0; q < 64; ++q) v[q] = (gi < m && gj0 + q < m) ? Wr[(long long)gi * m + gj0 + q] : 0.f;
+    for (int q = 0; q < 64; ++q) v[q] = (gi < m && gj0 + q < m) ? W[(long long)gi * m + gj0 + q] + (gi == gj0 + q ? eps : 0.f) : 0.f;
     u2_store_block(c, v, row, col0, u2_block_w(Wimg, ri, ci));
 #pragma unroll
-    for (int q = 0; q < 64; ++q) v[q] = (gi < m && gj0 + q < m) ? alpha * Wr[(long long)(gj0 + q) * m + gi] : 0.f;
+    for (int q = 0; q < 64; ++q) v[q] = (gi < m && gj0 + q < m) ? alpha * (W[(long long)(gj0 + q) * m + gi] + (gi == gj0 + q ? eps : 0.f)) : 0.f;
     if (T == 0) {
       if (gi < m) {
 #pragma unroll
