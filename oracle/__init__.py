@@ -46,6 +46,7 @@ class _Problem(ctypes.Structure):
         ("mh", ctypes.c_int32), ("mw", ctypes.c_int32),
         ("lm_f32", ctypes.c_int32),
         ("lm_filter", ctypes.c_void_p),
+        ("solver", ctypes.c_int32),
     ]
 
 
@@ -71,6 +72,7 @@ class Problem:
     lm_f32: int = 0   # 1: pooled landmarks rounded to single precision (what the device stores)
     # depth-wise-convolution landmark selection (Sec. 4.2): float64 [H, taps, d], taps = (gh/mh)*(gw/mw), or None
     lm_filter: Optional[np.ndarray] = field(default=None, repr=False)
+    solver: int = 0   # 0: Newton-Schulz (Alg. 2); 1: conjugate gradients, ns_iters steps (Sec. 5.3, Table 4)
 
     def c(self) -> _Problem:
         f = None
@@ -80,9 +82,10 @@ class Problem:
             assert f.dtype == np.float64 and f.flags["C_CONTIGUOUS"]
             assert f.shape == (self.H, (self.gh // self.mh) * (self.gw // self.mw), self.d)
             f = f.ctypes.data
+        assert self.solver in (0, 1) and not (self.solver == 1 and self.lm_mode == 3), "conjugate gradients need the symmetric W of one landmark set"
         return _Problem(self.B, self.H, self.n, self.d, self.m, float(self.lam), self.ns_iters,
                         float(self.ridge_eps), float(self.ns_alpha), self.map_mode, self.lm_mode,
-                        self.prefix, self.gh, self.gw, self.mh, self.mw, self.lm_f32, f)
+                        self.prefix, self.gh, self.gw, self.mh, self.mw, self.lm_f32, f, self.solver)
 
 
 def _load():
@@ -126,6 +129,15 @@ def l1_kernel_bwd(A, Bm, lam, dK):
     dA, dB = np.empty_like(A), np.empty_like(Bm)
     _load().oracle_l1_kernel_bwd(batch, na, nb, d, _p(A), _p(Bm), ctypes.c_double(lam), _p(dK), _p(dA), _p(dB))
     return dA, dB
+
+
+def cg_solve(W, Bm, iters, eps=0.0):
+    """T-step conjugate-gradient iterates of (W + eps I) X = B (Sec. 5.3).  W [batch,m,m], B [batch,m,d]."""
+    W, Bm = _f64(W), _f64(Bm)
+    batch, m, d = Bm.shape
+    X = np.empty_like(Bm)
+    _load().oracle_cg_solve(batch, m, d, _p(W), ctypes.c_double(eps), iters, _p(Bm), _p(X))
+    return X
 
 
 def ns_pinv(W, iters, eps=0.0, alpha=0.0, want_hist=False):

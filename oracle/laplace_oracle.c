@@ -42,6 +42,9 @@
  *   - the depth-wise-convolution landmark selection Sec. 4.2 mentions as an alternative is one
  *     r x r filter per head and channel applied with stride r to the regions average pooling
  *     would average (no bias; the filter with all taps 1/r^2 is average pooling).
+ *   - the conjugate-gradient solver of the ablation (Sec. 5.3, Table 4; solver = 1) is the textbook method from
+ *     x_0 = 0 for exactly T steps on (W + eps I) Y = M, column by column, and its backward pass differentiates the
+ *     linear system it approximates, each adjoint system by the same T-step method (the paper names the solver only).
  *
  * Beside the path, the two steps that surround it inside the attention block (end of this file): the rotary
  * position embedding on Q and K (Sec. 5.1; positions over the flattened token grid, class tokens not rotated) and
@@ -51,7 +54,9 @@
  * Kac-Murdock-Szego closed-form inverse, the spectral closed form of the
  * unconverged Newton-Schulz iterate, m = n reproducing exact Laplacian
  * attention, rows of Z summing to one, adjoint identities and central finite
- * differences.  Parity unpinned: how close the m < n approximation is to
+ * differences; for conjugate gradients the one-step closed form, every iterate
+ * against the Krylov-subspace minimiser from a dense projected solve,
+ * termination in m steps against the library's solve.  Parity unpinned: how close the m < n approximation is to
  * exact attention (the paper prints no error figure).
  */
 #include <math.h>
@@ -76,6 +81,8 @@ typedef struct oracle_problem {
   const double* lm_filter; /* NULL: average pooling.  Else [H][taps][d], taps = (gh/mh)*(gw/mw): the depth-wise convolution
                               landmark selection of Sec. 4.2 (one r x r filter per head and channel, stride r; the grid must
                               divide).  Tap (u,v) of a region is index u*(gw/mw)+v.  lm_mode 1 or 2 only. */
+  int32_t solver;   /* 0: Newton-Schulz (Alg. 2), Y = X_T M.  1: conjugate gradients (the solver of the ablation, Sec. 5.3,
+                       Table 4): Y = the ns_iters-step CG iterate of (W + eps I) Y = M, see cg_solve.  One landmark set only. */
 } oracle_problem;
 
 int oracle_num_threads(void) {
@@ -290,6 +297,54 @@ static void ns_single_bwd(int m, const double* Win, int T, double eps, double al
   free(W); free(X); free(Xh); free(G); free(P); free(H); free(T1); free(T2);
 }
 
+/* ------------------------------------------------------------------------- */
+/* Conjugate gradients (the other solver of Sec. 5.3 / Table 4)              */
+/* ------------------------------------------------------------------------- */
+/*
+ * The paper names the solver and prints nothing else about it, so this is the textbook method (Hestenes-Stiefel) for
+ * the symmetric positive definite system (W + eps I) x = b, started from x_0 = 0, run for exactly T steps, one
+ * independent solve per column of B [m][d]:
+ *     r_0 = b, p_0 = r_0;   a_k = r_k.r_k / p_k.(Wr p_k);   x_{k+1} = x_k + a_k p_k;   r_{k+1} = r_k - a_k Wr p_k;
+ *     b_k = r_{k+1}.r_{k+1} / r_k.r_k;   p_{k+1} = r_{k+1} + b_k p_k.
+ * A column whose residual is exactly zero, or whose curvature p.(Wr p) is not positive, stops moving.
+ */
+static void cg_solve(int m, int d, const double* Win, double eps, int T, const double* Bm, double* X) {
+  size_t mm = (size_t)m * m;
+  double* Wr = (double*)malloc(sizeof(double) * mm);
+  double* r = (double*)malloc(sizeof(double) * m);
+  double* pv = (double*)malloc(sizeof(double) * m);
+  double* q = (double*)malloc(sizeof(double) * m);
+  memcpy(Wr, Win, sizeof(double) * mm);
+  for (int i = 0; i < m; ++i) Wr[(size_t)i * m + i] += eps;
+  for (int c = 0; c < d; ++c) {
+    double rr = 0.0;
+    for (int i = 0; i < m; ++i) { X[(size_t)i * d + c] = 0.0; r[i] = Bm[(size_t)i * d + c]; pv[i] = r[i]; rr += r[i] * r[i]; }
+    for (int k = 0; k < T; ++k) {
+      if (rr == 0.0) break;
+      double pq = 0.0;
+      for (int i = 0; i < m; ++i) {
+        double t = 0.0;
+        for (int j = 0; j < m; ++j) t += Wr[(size_t)i * m + j] * pv[j];
+        q[i] = t; pq += pv[i] * t;
+      }
+      if (!(pq > 0.0)) break;
+      double a = rr / pq, rn = 0.0;
+      for (int i = 0; i < m; ++i) { X[(size_t)i * d + c] += a * pv[i]; r[i] -= a * q[i]; rn += r[i] * r[i]; }
+      double be = rn / rr;
+      for (int i = 0; i < m; ++i) pv[i] = r[i] + be * pv[i];
+      rr = rn;
+    }
+  }
+  free(Wr); free(r); free(pv); free(q);
+}
+
+/* X [batch][m][d] = T-step CG iterates of (W + eps I) X = B, W [batch][m][m], B [batch][m][d] */
+void oracle_cg_solve(int batch, int m, int d, const double* W, double eps, int iters, const double* Bm, double* X) {
+#pragma omp parallel for schedule(dynamic)
+  for (int b = 0; b < batch; ++b)
+    cg_solve(m, d, W + (size_t)b * m * m, eps, iters, Bm + (size_t)b * m * d, X + (size_t)b * m * d);
+}
+
 void oracle_ns_pinv(int batch, int m, const double* W, int iters, double eps, double alpha,
                     double* X, double* Xhist, double* resid, double* alpha_out) {
 #pragma omp parallel for schedule(dynamic)
@@ -471,9 +526,14 @@ static void fwd_single(const oracle_problem* p, const double* Q, const double* K
   l1_block(n, m, d, Q, x->L, p->lambda, x->C);                      /* Eq. 8: C = k(Q, K~) */
   l1_block(m, m, d, x->Lq, x->L, p->lambda, x->W);                  /* Eq. 9: W = k(Q~, K~) (ridge added inside Newton-Schulz) */
   l1_block(m, n, d, x->Lq, K, p->lambda, x->R);                     /* k(Q~, K) */
-  ns_single(m, x->W, p->ns_iters, p->ridge_eps, p->ns_alpha, x->X, NULL);   /* Alg. 2 */
   matmul(m, n, d, x->R, V, x->M);                                   /* M = R V */
-  matmul(m, m, d, x->X, x->M, x->Y);                                /* Y = X M */
+  if (p->solver == 1) {                                             /* Sec. 5.3: Y from conjugate gradients on Wr Y = M */
+    memset(x->X, 0, sizeof(double) * (size_t)m * m);                /* no inverse is formed */
+    cg_solve(m, d, x->W, p->ridge_eps, p->ns_iters, x->M, x->Y);
+  } else {
+    ns_single(m, x->W, p->ns_iters, p->ridge_eps, p->ns_alpha, x->X, NULL);   /* Alg. 2 */
+    matmul(m, m, d, x->X, x->M, x->Y);                              /* Y = X M */
+  }
   for (int i = 0; i < n; ++i) {
     if (p->map_mode == 1) {                                         /* Prop. 3 steps 2-4 */
       double mu = 0.0;
@@ -552,11 +612,21 @@ static void bwd_single(const oracle_problem* p, const double* Q, const double* K
       for (int l = 0; l < m; ++l) dC[(size_t)i * m + l] = dZ[(size_t)i * m + l];
     }
   }
-  matmul_nt(m, d, m, dY, x.M, dX);          /* Y = X M:  dX = dY M^T */
-  matmul_tn(m, m, d, x.X, dY, dM);          /*           dM = X^T dY */
+  if (p->solver == 1) {
+    /* Y solves Wr Y = M (to the accuracy T steps give).  The solve is differentiated as the linear system it
+       approximates, each adjoint system by the same T-step method (the paper does not say how its CG kernel is
+       differentiated; this is the usual rule for a linear solve):
+           dM = Wr^-T dY  ->  CG on Wr dM = dY (Wr is symmetric),      dWr = -dM Y^T. */
+    cg_solve(m, d, x.W, p->ridge_eps, p->ns_iters, dY, dM);
+    matmul_nt(m, d, m, dM, x.Y, dW);
+    for (size_t e = 0; e < mm; ++e) dW[e] = -dW[e];
+  } else {
+    matmul_nt(m, d, m, dY, x.M, dX);        /* Y = X M:  dX = dY M^T */
+    matmul_tn(m, m, d, x.X, dY, dM);        /*           dM = X^T dY */
+    ns_single_bwd(m, x.W, p->ns_iters, p->ridge_eps, p->ns_alpha, dX, dW);
+  }
   matmul_nt(m, d, n, dM, V, dR);            /* M = R V:  dR = dM V^T */
   matmul_tn(m, n, d, x.R, dM, dV);          /*           dV = R^T dM */
-  ns_single_bwd(m, x.W, p->ns_iters, p->ridge_eps, p->ns_alpha, dX, dW);
 
   memset(dQ, 0, sizeof(double) * nd);
   memset(dK, 0, sizeof(double) * nd);
