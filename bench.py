@@ -49,6 +49,8 @@ def parse():
     ap.add_argument("--fig5", action="store_true", help="the kernel micro-benchmark of the paper's Fig. 5 setting instead of a step")
     ap.add_argument("--fig5-T", type=int, default=8, help="Newton-Schulz steps of the micro-benchmark")
     ap.add_argument("--B", type=int, default=0, help="override the batch size (profiling of a smaller case)")
+    ap.add_argument("--solver", default="ns", choices=["ns", "cg"],
+                    help="per-head solver: Newton-Schulz (the path) or the conjugate gradients of the paper's ablation")
     return ap.parse_args()
 
 
@@ -291,7 +293,7 @@ def alu_probe(ln, dev):
 class Workload:
     """Device buffers and the step function of one configuration."""
 
-    def __init__(self, ln, cfg, dev, inp=None):
+    def __init__(self, ln, cfg, dev, inp=None, solver="ns"):
         self.ln, self.cfg, self.dev = ln, cfg, dev
         self.inp = synth.make_inputs(cfg) if inp is None else inp
         names = ("Q", "K", "V", "dO")
@@ -302,6 +304,7 @@ class Workload:
         self.nsets = min(max(2, int(np.ceil(3 * 126e6 / self.in_bytes))), 16)
         self.sets = [{k: self.inp[k].to(dev).clone() for k in names} for _ in range(self.nsets)]
         self.p = ln.problem_from_config(cfg, whiten=self.inp["whiten"].to(dev))
+        self.p.solver = 1 if solver == "cg" else 0
         self.saved = torch.empty(ln.laplace_nystrom_saved_bytes(self.p), dtype=torch.uint8, device=dev)
         self.ws = torch.empty(ln.laplace_nystrom_workspace_bytes(self.p, True), dtype=torch.uint8, device=dev)
         self.O = torch.empty_like(self.sets[0]["Q"])
@@ -386,7 +389,9 @@ def run_ours(args):
     cfg = synth.CONFIGS[args.config]
     if args.B > 0:
         cfg = synth.shrink(cfg, B=args.B)
-    w = Workload(ln, cfg, dev)
+    if args.solver == "cg":         # the ablation's solver: timed, but the oracle legs and the sweep describe the path itself
+        args.no_cpu_baseline = args.no_sweep = True
+    w = Workload(ln, cfg, dev, solver=args.solver)
     inp, p, es, names = w.inp, w.p, w.es, ("Q", "K", "V", "dO")
     step = w.step
 
@@ -554,7 +559,8 @@ def run_ours(args):
         "data": "synthetic",
         "config": workload_dict(cfg, {"l2": f"rotating {w.nsets} input sets ({w.nsets * w.in_bytes / 1e6:.0f} MB > 126 MB L2)",
                                       "parallelism": f"replicas x{world} (heads independent, no collective)",
-                                      "timed_regions": repeats, "region_ms": regions}),
+                                      "timed_regions": repeats, "region_ms": regions,
+                                      **({"solver": "conjugate gradients (Sec. 5.3) in place of Newton-Schulz"} if args.solver == "cg" else {})}),
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_timed,
         "roofline": roofline, "kernels": kernels,
     }

@@ -86,6 +86,15 @@ typedef struct ln_problem {
   float* lm_filter_grad;  /* with lm_filter: device fp32 [H, taps, d], 16-byte aligned, OVERWRITTEN by             */
                           /* laplace_nystrom_bwd with the gradient of the filter, summed over the batch; required  */
                           /* by the backward entry points (LN_ERR_ARG if NULL), ignored by the forward ones        */
+  int32_t solver;         /* 0: Newton-Schulz (Alg. 2), Y = X_T M.  1: conjugate gradients, the other solver of the        */
+                          /* ablation (Sec. 5.3, Table 4): Y = the ns_iters-step iterate of (k(L,L) + eps I) Y = M from    */
+                          /* Y_0 = 0, every column of M on its own (Hestenes-Stiefel; a column whose residual is zero or   */
+                          /* whose curvature is not positive stops); ns_alpha is ignored.  The backward pass               */
+                          /* differentiates the linear system the solver approximates: dM = the same ns_iters-step         */
+                          /* iterate of the system with right-hand side dY, dW = -dM Y^T (the paper names the solver       */
+                          /* only).  The recurrence runs in double precision, one CTA per head, for either storage dtype.  Needs the symmetric     */
+                          /* matrix of one landmark set: lm_mode 3 is LN_ERR_UNSUPPORTED.  dev_status bit 0 then means a   */
+                          /* non-finite entry of Y.                                                                        */
 } ln_problem;
 
 const char* ln_status_string(int status);

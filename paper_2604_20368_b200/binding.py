@@ -48,6 +48,7 @@ class _CProblem(ctypes.Structure):
         ("mh", ctypes.c_int32), ("mw", ctypes.c_int32),
         ("whiten_mode", ctypes.c_int32), ("whiten_eps", ctypes.c_float), ("whiten_batch", ctypes.c_void_p),
         ("lm_filter", ctypes.c_void_p), ("lm_filter_grad", ctypes.c_void_p),
+        ("solver", ctypes.c_int32),
     ]
 
 
@@ -84,6 +85,7 @@ class Problem:
     # overwritten by the backward pass
     lm_filter: Optional[torch.Tensor] = field(default=None, repr=False)
     lm_filter_grad: Optional[torch.Tensor] = field(default=None, repr=False)
+    solver: int = 0   # 0: Newton-Schulz (Alg. 2); 1: conjugate gradients, ns_iters steps (Sec. 5.3, Table 4)
 
     def c(self) -> _CProblem:
         w = None
@@ -95,7 +97,7 @@ class Problem:
                          float(self.ridge_eps), float(self.ns_alpha), self.dtype, self.map_mode, w,
                          self.lm_mode, self.prefix, self.gh, self.gw, self.mh, self.mw, self.whiten_mode,
                          float(self.whiten_eps), None if self.whiten_batch is None else self.whiten_batch.data_ptr(),
-                         self._filter_ptr(self.lm_filter), self._filter_ptr(self.lm_filter_grad))
+                         self._filter_ptr(self.lm_filter), self._filter_ptr(self.lm_filter_grad), self.solver)
 
     def _filter_ptr(self, t):
         if t is None:

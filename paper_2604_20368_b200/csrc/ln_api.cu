@@ -97,6 +97,7 @@ struct Plan {
   int s3_tiles;                      // sign pass with the upstream factor formed in the kernel: token tiles per head (0 = not used)
   int H, wmode, l1_tiles;            // heads; whitening mode; token tiles of the l1 launch that forms C (statistics partials)
   bool two;                          // two landmark sets (Alg. 1 as printed): W = k(pool(Q), pool(K)) is not symmetric
+  bool cg;                           // conjugate gradients in place of Newton-Schulz (fp32 per-head kernels)
 };
 
 bool make_plan(const ln_problem* p, Plan* pl) {
@@ -106,6 +107,7 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   pl->ldm = (p->m + 3) & ~3;
   pl->scr = (size_t)p->m * pl->ldm;
   pl->two = p->lm_mode == 3;
+  pl->cg = p->solver == 1;
   // the tcgen05 per-head kernels use the symmetry of the landmark kernel matrix; two landmark sets take the general engine
   const bool tcmid = p->dtype == LN_BF16 && !pl->two;
   if (tcmid && p->m > 128) pl->scr = (size_t)kU2Slot;
@@ -197,7 +199,7 @@ Ctx carve_ctx(const Plan& pl, void* base) {
   return x;
 }
 
-struct FwdWs { float *Mpart, *Wr, *P; double* stat; size_t bytes; };
+struct FwdWs { float *Mpart, *Wr, *P, *cg; double* stat; size_t bytes; };
 FwdWs carve_fwd_ws(const Plan& pl, void* base) {
   Carver c(base); FwdWs w;
   const size_t BH = pl.BH, d = pl.d, m = pl.m;
@@ -205,12 +207,13 @@ FwdWs carve_fwd_ws(const Plan& pl, void* base) {
   w.Wr = c.take(BH * pl.scr);
   w.P = c.take(BH * pl.scr);
   w.stat = reinterpret_cast<double*>(c.take(pl.wmode == 1 ? BH * (size_t)pl.l1_tiles * m * 4 : 0));   // [BH][tiles][m][2] doubles
+  w.cg = c.take(pl.cg ? BH * 8 * m * d : 0);                    // conjugate gradients: iterate, residual, direction, W times direction (doubles)
   w.bytes = c.off;
   return w;
 }
 
 struct BwdWs {
-  float *G, *G2, *dYtpart, *dybpart, *dLCpart, *dLRpart, *dY, *dM, *Wr, *P, *Hm, *Ga, *Gb, *dW, *dX, *GW, *dLW, *dLtot, *dKpart, *dMimg, *SB, *kap, *SBq, *dQpart, *dLqtot, *dLW2;
+  float *G, *G2, *dYtpart, *dybpart, *dLCpart, *dLRpart, *dY, *dM, *Wr, *P, *Hm, *Ga, *Gb, *dW, *dX, *GW, *dLW, *dLtot, *dKpart, *dMimg, *SB, *kap, *SBq, *dQpart, *dLqtot, *dLW2, *cg;
   size_t bytes;
 };
 BwdWs carve_bwd_ws(const Plan& pl, void* base) {
@@ -248,6 +251,7 @@ BwdWs carve_bwd_ws(const Plan& pl, void* base) {
   w.dQpart = c.take(pl.two ? BH * n * d : 0);
   w.dLqtot = c.take(pl.two ? BH * m * d : 0);
   w.dLW2 = c.take(pl.two ? BH * m * d : 0);
+  w.cg = c.take(pl.cg ? BH * 8 * m * d : 0);
   w.bytes = c.off;
   return w;
 }
@@ -263,6 +267,8 @@ int validate(const ln_problem* p) {
   if (p->dtype != LN_F32 && p->dtype != LN_BF16) return LN_ERR_ARG;
   if (p->map_mode != 0 && p->map_mode != 1) return LN_ERR_ARG;
   if (p->lm_mode < 0 || p->lm_mode > 3) return LN_ERR_ARG;
+  if (p->solver != 0 && p->solver != 1) return LN_ERR_ARG;
+  if (p->solver == 1 && p->lm_mode == 3) return LN_ERR_UNSUPPORTED;
   if (p->whiten && !aligned16(p->whiten)) return LN_ERR_ARG;
   if (p->whiten_mode != 0 && p->whiten_mode != 1) return LN_ERR_ARG;
   if (p->whiten_mode == 1) {
@@ -509,7 +515,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // the three kernel blocks: C = k(Q,L) with its row sums, R^T = k(K,L), W = k(L,L)
   // (not for many small heads, where the per-head kernel fills the GPU and the split launches cost more than the
   // overlap returns)
-  const Side side = side_acquire(!two && std::is_same<T, bf16>::value && (2 * pl.mid_sms <= kSMs || (long long)n * m * D > (1ll << 22)), st);
+  const Side side = side_acquire(!two && !pl.cg && std::is_same<T, bf16>::value && (2 * pl.mid_sms <= kSMs || (long long)n * m * D > (1ll << 22)), st);
   const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);   // tcgen05 products over the landmarks
   // Where the iteration is expected to outlast the two token-sized blocks (few heads of few tokens), only the iteration
   // goes to the side stream; estimates in microseconds: 5 / 12 / 100 per step for m <= 64 / <= 128 / larger, and the l1
@@ -529,8 +535,11 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
       LN_LAUNCH(phase == 3 ? "k_mid_fwd" : (phase == 1 ? "k_mid_fwd_ns" : "k_mid_fwd_y"), s,
                 launch_clustered(kern, BH * cl, cl, smem, s, m, pl.ldm, pl.T, p->ridge_eps, p->ns_alpha, p->H, p->map_mode,
                                  whiten_eff, x.W, w.Wr, w.P, x.Xh, x.Ph, x.hdr, Mparts_src, Mparts, x.M, x.Y, x.Yt,
-                                 x.ybar, dev_status, pl.hslot, umma_prod ? reinterpret_cast<bf16*>(x.Yimg) : nullptr, phase));
+                                 x.ybar, dev_status, pl.hslot, umma_prod ? reinterpret_cast<bf16*>(x.Yimg) : nullptr, phase,
+                                 pl.cg ? 1 : 0, w.cg));
     };
+    // conjugate gradients (Sec. 5.3): fp32, one CTA per head, whatever the storage type
+    if (pl.cg) { launch(k_mid_fwd<D, false, 0>, sizeof(NsSmem)); return; }
     // general (non-symmetric) matrix: the mma.sync or FFMA engine, shared by the CTAs of a cluster beyond 64 landmarks
     if (two && m > 64) launch(k_mid_fwd<D, TC, 0, kMidCluster>, sizeof(NsSmem), kMidCluster);
     else if (two) launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));
@@ -687,8 +696,10 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
       LN_LAUNCH("k_mid_bwd", s, launch_clustered(kern, BH * cl, cl, smem, s, m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, whiten_eff,
                                                  x.W, x.Xh, x.Ph, x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P,
                                                  w.Hm, w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot,
-                                                 umma_prod ? reinterpret_cast<bf16*>(w.dMimg) : nullptr, two ? 0 : 1));
+                                                 umma_prod ? reinterpret_cast<bf16*>(w.dMimg) : nullptr, two ? 0 : 1,
+                                                 pl.cg ? 1 : 0, x.Y, w.cg));
     };
+    if (pl.cg) { launch(k_mid_bwd<D, false, 0>, sizeof(NsSmem)); return; }
     if (two && m > 64) launch(k_mid_bwd<D, TC, 0, kMidCluster>, sizeof(NsSmem), kMidCluster);
     else if (two) launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
     else if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 4 * kUmmaMatBytes64);

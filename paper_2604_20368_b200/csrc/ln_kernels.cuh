@@ -1328,6 +1328,143 @@ __device__ void ns_tail_gw_sym(int m, int ldm, const float* __restrict__ W, floa
   }
 }
 
+// =====================================================================================
+// Conjugate gradients (the other solver of Sec. 5.3 / Table 4) for one head, whole CTA (256 threads):
+//   X = the T-step iterate of (W + eps I) X = B from X_0 = 0, one independent solve per column of B [m][D]
+//   (Hestenes-Stiefel: a = r.r / p.(Wr p), x += a p, r -= a Wr p, b = r'.r' / r.r, p = r' + b p).
+// A column whose residual is exactly zero, or whose curvature p.(Wr p) is not positive, stops moving.
+// The recurrence runs in DOUBLE precision: in single precision the iterates drift from the exact-arithmetic ones by
+// 1e-4 after three steps and 3e-2 after four on the landmark matrices of this path (the directions lose their
+// conjugacy), although the iterate itself depends on W and B only mildly; the inputs stay fp32.
+// W: fp32 [m][m] without the ridge; Bsrc: fp32 [m][D]; Xout: fp32 [m][D]; scratch: 4 m D doubles (x, r, p, Wr p).
+// Thread t always works on column t % D (256 % D == 0); the dot products of a column are added over the 256 / D
+// threads that share it in a fixed order.  red: >= 2 * 256 + 8 floats; gsm: >= 16 KiB of shared memory.
+// =====================================================================================
+// Q = (W + eps I) P in double: 64 x 64 output tiles, K in chunks of 16, a 4 x 4 block per thread
+template <int D>
+__device__ void cg_matvec(int m, float eps, const float* __restrict__ W, const double* __restrict__ P, double* __restrict__ Q, double* gsm) {
+  double (*As)[64] = reinterpret_cast<double (*)[64]>(gsm);            // [16][64]: As[kk][i] = Wr[i0 + i][k0 + kk]
+  double (*Bs)[64] = reinterpret_cast<double (*)[64]>(gsm + 16 * 64);  // [16][64]: Bs[kk][j] = P[k0 + kk][j0 + j]
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  for (int i0 = 0; i0 < m; i0 += 64)
+    for (int j0 = 0; j0 < D; j0 += 64) {
+      double acc[4][4];
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+      for (int k0 = 0; k0 < m; k0 += 16) {
+        __syncthreads();
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int e = tid + 256 * u;
+          { const int i = e >> 4, kk = e & 15, gi = i0 + i, gk = k0 + kk;                 // consecutive threads along k
+            As[kk][i] = (gi < m && gk < m) ? (double)W[(long long)gi * m + gk] + (gi == gk ? (double)eps : 0.0) : 0.0; }
+          { const int kk = e >> 6, j = e & 63, gk = k0 + kk, gj = j0 + j;
+            Bs[kk][j] = (gk < m && gj < D) ? P[(long long)gk * D + gj] : 0.0; }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) {
+          double a4[4], b4[4];
+          {
+            const double2 a01 = *reinterpret_cast<const double2*>(&As[kk][ty * 4]), a23 = *reinterpret_cast<const double2*>(&As[kk][ty * 4 + 2]);
+            const double2 b01 = *reinterpret_cast<const double2*>(&Bs[kk][tx * 4]), b23 = *reinterpret_cast<const double2*>(&Bs[kk][tx * 4 + 2]);
+            a4[0] = a01.x; a4[1] = a01.y; a4[2] = a23.x; a4[3] = a23.y;
+            b4[0] = b01.x; b4[1] = b01.y; b4[2] = b23.x; b4[3] = b23.y;
+          }
+#pragma unroll
+          for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) acc[a][b] = fma(a4[a], b4[b], acc[a][b]);
+        }
+      }
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const int gi = i0 + ty * 4 + a;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const int gj = j0 + tx * 4 + b;
+          if (gi < m && gj < D) Q[(long long)gi * D + gj] = acc[a][b];
+        }
+      }
+    }
+  __syncthreads();
+}
+
+template <int D>
+__device__ void cg_dev(int m, int T, float eps, const float* W, const float* Bsrc, float* Xout, double* scratch, double* gsm, float* red) {
+  constexpr int NG = 256 / D;
+  const int tid = threadIdx.x, c = tid % D, md = m * D;
+  // four disjoint arrays: the element-wise passes may keep several loads in flight
+  double* __restrict__ X = scratch; double* __restrict__ R = scratch + md; double* __restrict__ P = scratch + 2 * md;
+  double* __restrict__ Qv = scratch + 3 * md;
+  double* dred = reinterpret_cast<double*>(red);     // [256] partial dot products (2 * 256 floats)
+  __shared__ double rr_s[D], coef_s[D];
+  __shared__ int frozen_s[D];
+  auto column_sum = [&](double part) {               // sum over the threads of a column; valid in threads tid < D
+    dred[tid] = part;
+    __syncthreads();
+    double t = 0.0;
+    if (tid < D)
+#pragma unroll
+      for (int q = 0; q < NG; ++q) t += dred[q * D + tid];
+    __syncthreads();
+    return t;
+  };
+  double part = 0.0;
+  for (int e = tid; e < md; e += 256) {
+    const double b = (double)Bsrc[e];
+    X[e] = 0.0; R[e] = b; P[e] = b;
+    part += b * b;
+  }
+  {
+    const double t = column_sum(part);
+    if (tid < D) { rr_s[tid] = t; frozen_s[tid] = (t == 0.0) ? 1 : 0; }
+  }
+  __syncthreads();
+  for (int k = 0; k < T; ++k) {
+    cg_matvec<D>(m, eps, W, P, Qv, gsm);                                                 // Q = (W + eps I) P (ends with a barrier)
+    part = 0.0;
+#pragma unroll 4
+    for (int e = tid; e < md; e += 256) part += P[e] * Qv[e];
+    {
+      const double pq = column_sum(part);
+      if (tid < D) {
+        if (!frozen_s[tid] && !(pq > 0.0)) frozen_s[tid] = 1;
+        coef_s[tid] = frozen_s[tid] ? 0.0 : rr_s[tid] / pq;
+      }
+    }
+    __syncthreads();
+    const double a = coef_s[c];
+    part = 0.0;
+#pragma unroll 4
+    for (int e = tid; e < md; e += 256) {
+      X[e] = fma(a, P[e], X[e]);
+      const double r = fma(-a, Qv[e], R[e]);
+      R[e] = r;
+      part += r * r;
+    }
+    {
+      const double rn = column_sum(part);
+      if (tid < D && !frozen_s[tid]) {
+        coef_s[tid] = rn / rr_s[tid];
+        rr_s[tid] = rn;
+        if (rn == 0.0) frozen_s[tid] = 1;
+      }
+    }
+    __syncthreads();
+    if (!frozen_s[c]) {                              // a column that has stopped keeps its direction
+      const double be = coef_s[c];
+#pragma unroll 4
+      for (int e = tid; e < md; e += 256) P[e] = fma(be, P[e], R[e]);
+    }
+    __syncthreads();
+  }
+  for (int e = tid; e < md; e += 256) Xout[e] = (float)X[e];
+  __syncthreads();
+}
+
 // ------------------------------------------------------------------ stand-alone ns_pinv / ns_pinv_bwd
 // CL CTAs of a thread-block cluster share a matrix (grid = batch * CL): every product is split by output tiles, the
 // hardware cluster barrier ends a phase.  fp32 FFMA throughout (held to 2e-5 against the oracle).
@@ -1393,7 +1530,9 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
                                                  const float* __restrict__ whiten, const float* W, float* Wr,
                                                  float* P, float* Xh, float* Ph, NsHdr* hdr, const float* Mpart, int nchunks,
                                                  float* Mout, float* Y, float* Yt, float* ybar, int* dev_status,
-                                                 long long hslot, bf16* Yimg, int phase) {
+                                                 long long hslot, bf16* Yimg, int phase, int solver = 0, float* cgws = nullptr) {
+  // solver: 0 = Newton-Schulz (Alg. 2) and Y = X_T M; 1 = conjugate gradients on (W + eps I) Y = M (Sec. 5.3, Table 4;
+  // the single-CTA instantiation without tensor cores only), cgws = 4 m D doubles of scratch per head
   // phase: bit 0 = Newton-Schulz (needs W only), bit 1 = everything that needs M (sum of the partials, Y, map fold).
   // The two halves may run as two launches, the first beside the kernels that produce M; X_T passes through
   // global memory either way.
@@ -1418,7 +1557,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     for (long long e = (long long)gt * 4; e < md; e += 4 * gn)
       *reinterpret_cast<float4*>(Mout + e) = sum_parts4(Mpart, nchunks, md, e);
   const float* XT = Xh + (long long)T * mx;
-  if (phase & 1) {
+  if ((phase & 1) && solver == 0) {
   bool tc_ok = true;
   float bad = 0.f;                               // non-finite entries of X_T seen by this thread
   if constexpr (MP == 128 || MP == 64) {        // tcgen05 + TMEM, the matrix padded to MP x MP
@@ -1442,8 +1581,21 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
   }
   if (!(phase & 2)) return;
   if (!(phase & 1)) phase_sync<CL>();             // the M sums of all threads that share the head
-  ns_gemm<TC, false, false>(m, D, m, XT, ldx, Mout, D, Y, D, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // Y = X M
-  if (CL > 1) phase_sync<CL>();
+  if (solver == 1) {
+    if constexpr (!TC && MP == 0 && CL == 1) {
+      __syncthreads();
+      cg_dev<D>(m, T, eps, W, Mout, Y, reinterpret_cast<double*>(cgws) + (long long)bh * 4 * md, reinterpret_cast<double*>(dyn_smem), red);
+      if (dev_status) {
+        float bad = 0.f;
+        for (int e = tid; e < m * D; e += 256) bad += isfinite(Y[e]) ? 0.f : 1.f;
+        bad = block_sum(bad, red);
+        if (tid == 0 && bad > 0.f) atomicOr(dev_status + bh, 1);
+      }
+    }
+  } else {
+    ns_gemm<TC, false, false>(m, D, m, XT, ldx, Mout, D, Y, D, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // Y = X M
+    if (CL > 1) phase_sync<CL>();
+  }
   const float* s = whiten ? whiten + (long long)(bh % H) * m : nullptr;
   // fold the injective map (Prop. 3): column means over the landmarks first (256 / D thread groups share the
   // landmarks of a column, eight independent loads per batch, the groups added in order), then every element in parallel
@@ -1498,7 +1650,10 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
                                                  const float* dYtpart, const float* dybpart, int nchunks,
                                                  float eps, float* Wr, float* P, float* Hm, float* Ga, float* Gb,
                                                  float* dWm, float* dXm, float* dY, float* dM, float* GW, int* dev_status,
-                                                 long long hslot, bf16* dMimg, int sym) {
+                                                 long long hslot, bf16* dMimg, int sym, int solver = 0, const float* Ysaved = nullptr,
+                                                 float* cgws = nullptr) {
+  // solver 1 (conjugate gradients, the fp32 single-CTA instantiation only): the solve is differentiated as the linear
+  // system it approximates, dM = the T-step iterate of (W + eps I) dM = dY, dW = -dM Y^T (Ysaved: Y of the forward pass)
   // sym: 1 = one landmark set (W = k(L, L): the gradient of both roles of L is carried by the symmetrised factor);
   // 0 = two landmark sets, GW = dW o W / lambda as it is (MP == 0 only)
   extern __shared__ __align__(16) unsigned char dyn_smem[];
@@ -1539,8 +1694,15 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
   }
   phase_sync<CL>();
   const float* XT = Xh + (long long)T * mx;
-  ns_gemm<TC, false, true>(m, m, D, dY, D, Msaved, D, dXm, ldx, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // dX = dY M^T
-  ns_gemm<TC, true, false>(m, D, m, XT, ldx, dY, D, dM, D, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);        // dM = X^T dY
+  if (solver == 1) {
+    if constexpr (!TC && MP == 0 && CL == 1) {
+      cg_dev<D>(m, T, eps, W, dY, dM, reinterpret_cast<double*>(cgws) + (long long)bh * 4 * md, reinterpret_cast<double*>(dyn_smem), red);
+      ns_gemm<TC, false, true>(m, m, D, dM, D, Ysaved + bh * md, D, dWm, ldx, -1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // dW = -dM Y^T
+    }
+  } else {
+    ns_gemm<TC, false, true>(m, m, D, dY, D, Msaved, D, dXm, ldx, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // dX = dY M^T
+    ns_gemm<TC, true, false>(m, D, m, XT, ldx, dY, D, dM, D, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);        // dM = X^T dY
+  }
   if (CL > 1) phase_sync<CL>();
   if (dMimg != nullptr) {                         // dM also as split operand images (for the tcgen05 product dV = R^T dM)
     const int nkb = (m + GU_KB - 1) / GU_KB;
@@ -1557,7 +1719,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     if (dev_status && !tc_ok && tid == 0 && crank == 0) atomicOr(dev_status + bh, 2);
     // end of the adjoint and GW in one pass (the operand buffers are free: the engine has ended with a cluster barrier)
     ns_tail_gw_sym<CL>(m, ldm, W, eps, hdr, P, dWm, inv_lambda, GW, red, reinterpret_cast<float*>(dyn_smem), crank);
-  } else { ns_backward_dev<TC, CL>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red, crank, Ph); if (CL > 1) phase_sync<CL>(); }
+  } else if (solver == 0) { ns_backward_dev<TC, CL>(m, T, Wr, Xh, hdr, dXm, dWm, P, Hm, Ga, Gb, sm, red, crank, Ph); if (CL > 1) phase_sync<CL>(); }
   // GW = (dW o K_LL + (dW o K_LL)^T) / lambda; four elements per batch so that the loads overlap
   // (the tcgen05 engines have written GW already)
   if constexpr (MP == 0)

@@ -109,7 +109,7 @@ __device__ __forceinline__ void u2_begin(U2Ctx& c, UmmaCtl& ctl, unsigned long l
 __device__ bool ns_forward_umma256(int m, int T, float eps, float alpha_in, const float* W, float* Wr, float* Wimg,
                                    float* Xh, float* Ph, NsHdr* hdr, bf16* smem, float* red, UmmaCtl& ctl,
                                    unsigned long long* mbar_free, int crank, float& bad) {
-  const int tid = threadIdx.x, warp = tid >> 5, gt = crank * 256 + tid, gn = 1024;
+  const int tid = threadIdx.x, warp = tid >> 5;
   const int ri = crank >> 1, ci = crank & 1;
   const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64;
   const int gi = ri * 128 + row, gj0 = ci * 128 + col0;          // this thread's row and first column in the matrix

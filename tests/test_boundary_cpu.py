@@ -155,6 +155,29 @@ def test_filter_selection_argument_errors_without_gpu():
     assert fwd(odd) == -1                                           # not 16-byte aligned
 
 
+def test_solver_argument_errors_without_gpu():
+    """ln_problem.solver: 0 (Newton-Schulz) or 1 (conjugate gradients, Sec. 5.3); conjugate gradients need the symmetric
+    matrix of one landmark set."""
+    lib = binding.lib()
+    buf = ctypes.create_string_buffer(96)
+    a = ctypes.c_void_p((ctypes.addressof(buf) + 15) // 16 * 16)      # 16-byte aligned, never dereferenced
+
+    def with_solver(solver, lm_mode):
+        cp = ln.problem_from_config(synth.CONFIGS["cfg2"]).c()
+        cp.solver, cp.lm_mode = solver, lm_mode
+        return cp
+    fwd = lambda cp: lib.laplace_nystrom_fwd(ctypes.byref(cp), a, a, a, None, a, a, a, 0, None, None)
+    assert fwd(with_solver(1, 1)) == -3                             # valid: only the (empty) workspace is refused
+    assert fwd(with_solver(1, 2)) == -3
+    assert fwd(with_solver(2, 1)) == -1
+    assert fwd(with_solver(-1, 1)) == -1
+    assert fwd(with_solver(1, 3)) == -2                             # W = k(pool Q, pool K) is not symmetric
+    # the solver's scratch is part of the workspace the caller is told to bring
+    p0, p1 = with_solver(0, 1), with_solver(1, 1)
+    for with_saved in (0, 1):
+        assert lib.laplace_nystrom_workspace_bytes(ctypes.byref(p1), with_saved) > lib.laplace_nystrom_workspace_bytes(ctypes.byref(p0), with_saved)
+
+
 def test_overlap_switch_and_launch_counter_without_gpu():
     """ln_set_overlap returns the previous setting (default on); the launch counter is readable and has not moved
     without a launch."""

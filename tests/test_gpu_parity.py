@@ -340,6 +340,52 @@ def test_landmarks_selected_by_a_depthwise_filter(lm_mode, name, B, H, dtype):
     assert e < (1e-4 if dtype == "f32" else 1e-3)
 
 
+@pytest.mark.parametrize("name,B,H,dtype,T,lm_mode,ridge", [
+    ("cfg1", 2, 2, "f32", 6, 1, 1e-6), ("cfg2", 2, 2, "bf16", 6, 1, 1e-6), ("cfg2", 1, 2, "f32", 0, 1, 1e-6),
+    ("cfg2", 1, 2, "bf16", 1, 2, 1e-6), ("cfg3", 1, 2, "bf16", 4, 1, 1e-6), ("cfg4a", 1, 1, "bf16", 4, 1, 1e-6),
+    ("cfg5_m128_T8", 1, 2, "bf16", 4, 1, 1e-6), ("cfg5_m256_T4", 1, 1, "bf16", 4, 1, 1e-6),
+    ("cfg5_m64_T4", 1, 2, "f32", 12, 1, 1e-2)])
+def test_conjugate_gradient_solver(name, B, H, dtype, T, lm_mode, ridge):
+    """solver = 1 (Sec. 5.3, Table 4): Y from T steps of conjugate gradients on (W + eps I) Y = M; the backward pass
+    solves the adjoint system by the same T steps.  Forward and backward against the oracle's plain CG.
+
+    The step counts are the ones at which the T-step iterate is a stable function of its inputs.  Measured with the
+    oracle alone (a relative perturbation of 1e-7 of the right-hand side, change of the iterate): 1e-5 at T = 4 on
+    every shape here (the columns of M = R V lie almost along one eigenvector, and the other components decide the
+    iterate), but 2.5e-4 on cfg3 at T = 6, 2.5e-2 on cfg4a at T = 6, 1e-2 on cfg5 m = 256 at T = 6 and 4e-2 on the
+    adjoint solve of cfg5 m = 128 at T = 8, the same for a perturbation of 1e-5: the iterate jumps where a step reaches
+    the small end of the spectrum (cfg5 duplicates landmarks: W is singular up to the ridge).  No two precisions agree
+    there, whatever the implementation; the device runs the recurrence in double precision and differs from the
+    oracle through the rounding of M, dY and W only."""
+    from dataclasses import replace
+    from parity import metrics
+    cfg = replace(synth.shrink(synth.CONFIGS[name], B=B, H=H), backward=True, dtype=dtype, T=T, ridge_eps=ridge)
+    inp = synth.make_inputs(cfg)
+    Q, K, V, dO = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
+    p = ln.problem_from_config(cfg, whiten=inp["whiten"].to(DEV))
+    p.lm_mode = lm_mode
+    p.solver = 1
+    saved = torch.empty(ln.laplace_nystrom_saved_bytes(p), dtype=torch.uint8, device=DEV)
+    status = torch.full((cfg.B * cfg.H,), -1, dtype=torch.int32, device=DEV)
+    O = ln.laplace_nystrom_fwd(p, Q, K, V, saved=saved, dev_status=status)
+    dQ, dK, dV, _ = ln.laplace_nystrom_bwd(p, Q, K, V, dO, saved)
+    assert int(status.abs().max()) == 0
+    op = replace(oracle_problem(cfg, lm_mode=lm_mode), solver=1)
+    wh = f64(inp["whiten"])
+    q, k, v, g = (f64(inp[x]) for x in ("Q", "K", "V", "dO"))
+    Oo = oracle.forward(op, q, k, v, whiten=wh)
+    dQo, dKo, dVo, _ = oracle.backward(op, q, k, v, g, whiten=wh)
+    # the two solvers do differ on this input (otherwise the comparison would not show which one ran)
+    if T > 0:
+        O_ns = oracle.forward(replace(op, solver=0), q, k, v, whiten=wh)
+        assert rel_err(O_ns, Oo) > 1e-3
+    BH = cfg.B * cfg.H
+    errs = {kk: metrics(f64(a).reshape(BH, cfg.n, cfg.d), r.reshape(BH, cfg.n, cfg.d), cfg.dtype == "bf16")
+            for kk, a, r in (("O", O, Oo), ("dQ", dQ, dQo), ("dK", dK, dKo), ("dV", dV, dVo))}
+    print(cfg.name, "conjugate gradients, T", T, {kk: {a: f"{b:.1e}" for a, b in e.items()} for kk, e in errs.items()})
+    assert_parity(cfg, errs)
+
+
 @pytest.mark.parametrize("name,B,H,dtype", [("cfg2", 3, 2, "bf16"), ("cfg2", 2, 1, "f32"), ("cfg4a", 2, 1, "bf16"),
                                             ("cfg5_m64_T4", 2, 1, "bf16"), ("cfg1", 2, 2, "f32")])
 def test_batch_statistic_whitening_training_mode(name, B, H, dtype):
