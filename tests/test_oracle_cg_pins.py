@@ -147,3 +147,26 @@ def test_backward_rule_at_few_steps_is_the_stated_one():
     dY = x["Z"][0].T @ dO[0, 0]
     dM = oracle.cg_solve(x["W"], dY[None], T, eps=1e-3)[0]
     np.testing.assert_allclose(dV[0, 0], x["R"][0].T @ dM, rtol=1e-12, atol=1e-14)
+
+
+@pytest.mark.parametrize("kappa", [2.0, 10.0, 50.0])
+def test_energy_norm_error_bound_over_condition_numbers(kappa):
+    # the textbook bound ||x_k - x*||_W <= 2 ((sqrt(kappa) - 1) / (sqrt(kappa) + 1))^k ||x*||_W, the behaviour the paper's
+    # convergence figure (Sec. 5.3) describes: fast at kappa = 2, slower as the condition number grows
+    rng = np.random.default_rng(100 + int(kappa))
+    m, d = 24, 3
+    W = spd(rng, m, kappa)
+    Bm = rng.standard_normal((1, m, d))
+    exact = np.linalg.solve(W, Bm[0])
+    e0 = np.sqrt(np.einsum("ic,ij,jc->c", exact, W, exact))
+    rho = (np.sqrt(kappa) - 1) / (np.sqrt(kappa) + 1)
+    errs = []
+    for k in (1, 2, 4, 8):
+        E = oracle.cg_solve(W[None], Bm, k)[0] - exact
+        en = np.sqrt(np.einsum("ic,ij,jc->c", E, W, E))
+        assert (en <= 2 * rho ** k * e0 * (1 + 1e-10)).all(), (kappa, k)
+        errs.append(en.max() / e0.max())
+    if kappa == 2.0:
+        assert errs[-1] < 1e-5          # eight steps at kappa = 2: converged
+    if kappa == 50.0:
+        assert errs[-1] > 1e-5          # and not yet at kappa = 50
