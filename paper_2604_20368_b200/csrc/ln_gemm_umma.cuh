@@ -45,6 +45,19 @@ template <int D> __host__ __device__ constexpr size_t nn_umma_stage_dwc() {
 }
 template <int D> __host__ __device__ constexpr size_t nn_umma_smem_dwc() { return nn_umma_stage_dwc<D>() + (size_t)49 * D * sizeof(float); }
 
+// one tap of the depth-wise convolution on eight channels: acc += w * v (v: eight bf16 values, w: eight fp32 weights in
+// shared memory; a tap outside the grid arrives as zeros)
+__device__ __forceinline__ void dwc_tap8(float (&acc)[8], const uint4& v, const float* w) {
+  const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
+  const float4 w0 = *reinterpret_cast<const float4*>(w), w1 = *reinterpret_cast<const float4*>(w + 4);
+  const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    acc[2 * e] = fmaf(wv[2 * e], __uint_as_float(vw[e] << 16), acc[2 * e]);
+    acc[2 * e + 1] = fmaf(wv[2 * e + 1], __uint_as_float(vw[e] & 0xffff0000u), acc[2 * e + 1]);
+  }
+}
+
 // One 128-token tile per CTA; three CTAs per SM hide each other's load latencies.
 // DWC: the depth-wise convolution branch of the attention block (Eq. 7) is added in the epilogue, before the one rounding
 // to bf16 (O = Z V + DWC(V) in the forward pass; dV = R^T dM + DWC^T(dO) in the backward pass).
@@ -166,22 +179,31 @@ __global__ void __launch_bounds__(256, 3) k_nn_umma(const float* __restrict__ E,
       for (int e = 0; e < 8; ++e) acc[e] = fstage[r * LDF + c8 + e];
       if (i >= epi.prefix) {
         const int tok = i - epi.prefix, gr = tok / epi.gw, gq = tok % epi.gw;
-        for (int a = 0; a < epi.ks; ++a) {
-          const int rr = gr + a - half;
-          if (rr < 0 || rr >= epi.gh) continue;
-          for (int b = 0; b < epi.ks; ++b) {
-            const int qq = gq + b - half;
-            if (qq < 0 || qq >= epi.gw) continue;
-            const int tap = epi.flip ? (epi.ks - 1 - a) * epi.ks + (epi.ks - 1 - b) : a * epi.ks + b;
-            const uint4 v = *reinterpret_cast<const uint4*>(src + (long long)(epi.prefix + rr * epi.gw + qq) * D + c8);
-            const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
-            const float4 w0 = *reinterpret_cast<const float4*>(wsm + tap * D + c8), w1 = *reinterpret_cast<const float4*>(wsm + tap * D + c8 + 4);
-            const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+        const bf16* srow = src + (long long)epi.prefix * D + c8;
+        if (epi.ks == 3) {                        // the common 3 x 3 filter: all nine loads in flight before the first use
+          uint4 v[9];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              acc[2 * e] = fmaf(wv[2 * e], __uint_as_float(vw[e] << 16), acc[2 * e]);
-              acc[2 * e + 1] = fmaf(wv[2 * e + 1], __uint_as_float(vw[e] & 0xffff0000u), acc[2 * e + 1]);
+          for (int t = 0; t < 9; ++t) {
+            const int rr = gr + t / 3 - 1, qq = gq + t % 3 - 1;
+            v[t] = (rr >= 0 && rr < epi.gh && qq >= 0 && qq < epi.gw) ? *reinterpret_cast<const uint4*>(srow + (long long)(rr * epi.gw + qq) * D)
+                                                                      : make_uint4(0u, 0u, 0u, 0u);
+          }
+#pragma unroll
+          for (int t = 0; t < 9; ++t) dwc_tap8(acc, v[t], wsm + (epi.flip ? 8 - t : t) * D + c8);
+        } else {
+          for (int a = 0; a < epi.ks; ++a) {      // a filter row at a time (up to seven loads in flight)
+            const int rr = gr + a - half;
+            if (rr < 0 || rr >= epi.gh) continue;
+            uint4 v[7];
+#pragma unroll
+            for (int b = 0; b < 7; ++b) {
+              const int qq = gq + b - half;
+              v[b] = (b < epi.ks && qq >= 0 && qq < epi.gw) ? *reinterpret_cast<const uint4*>(srow + (long long)(rr * epi.gw + qq) * D)
+                                                            : make_uint4(0u, 0u, 0u, 0u);
             }
+#pragma unroll
+            for (int b = 0; b < 7; ++b)
+              if (b < epi.ks) dwc_tap8(acc, v[b], wsm + (epi.flip ? (epi.ks - 1 - a) * epi.ks + (epi.ks - 1 - b) : a * epi.ks + b) * D + c8);
           }
         }
       }
