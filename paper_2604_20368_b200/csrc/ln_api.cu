@@ -1410,8 +1410,11 @@ void launch_rope_table(const ln_problem* p, const ln_block* b, double2* tab, cud
 }
 template <typename T>
 void launch_rope(const char* name, const ln_problem* p, const double2* tab, const void* X, void* out, double sign, cudaStream_t st) {
-  const long long rows = (long long)p->B * p->H * p->n;
-  LN_LAUNCH(name, st, k_rope<T><<<cdiv(rows * (p->d / 4), 256), 256, 0, st>>>((const T*)X, (T*)out, rows, p->n, p->d, p->prefix, tab, sign));
+  // a thread per (token, channel quad) walks a share of the heads; shares so that about four CTAs per SM are launched
+  const int BH = p->B * p->H, gx = (int)cdiv((long long)p->n * (p->d / 4), 256);
+  int gy = (int)cdiv(4ll * sm_count(), gx); if (gy > BH) gy = BH; if (gy < 1) gy = 1;
+  const int hpc = (BH + gy - 1) / gy; gy = (BH + hpc - 1) / hpc;
+  LN_LAUNCH(name, st, k_rope<T><<<dim3(gx, gy), 256, 0, st>>>((const T*)X, (T*)out, BH, hpc, p->n, p->d, p->prefix, tab, sign));
 }
 // the tcgen05 product kernels (bf16 storage, 64 or 128 dims) take the convolution branch into their epilogue
 inline bool dwc_in_epilogue(const ln_problem* p) { return p->dtype == LN_BF16 && (p->d == 64 || p->d == 128); }

@@ -29,25 +29,39 @@ __global__ void __launch_bounds__(256) k_rope_table(double2* __restrict__ tab, l
   tab[e] = make_double2(cs, sn);
 }
 
+// A thread owns one (token, channel quad) and walks the heads and batch elements of its share (blockIdx.y): the two table
+// entries are read once and stay in registers, so the table costs 1 / (heads per share) of what the tensor does.
 template <typename T>
-__global__ void __launch_bounds__(256) k_rope(const T* __restrict__ X, T* __restrict__ out, long long rows, int n, int d,
+__global__ void __launch_bounds__(256) k_rope(const T* __restrict__ X, T* __restrict__ out, int BH, int hpc, int n, int d,
                                              int prefix, const double2* __restrict__ tab, double sign) {
-  const long long e = (long long)blockIdx.x * 256 + threadIdx.x;
-  const int quads = d / 4;
-  if (e >= rows * quads) return;
-  const long long row = e / quads;
-  const int c = (int)(e % quads) * 4, t = (int)(row % n);
-  const float4 v = ld4(X + row * d + c);
-  T* o = out + row * d + c;
-  if (t < prefix) { st4(o, v); return; }
+  const int e = blockIdx.x * 256 + threadIdx.x, quads = d / 4;
+  if (e >= n * quads) return;
+  const int t = e / quads, c = (e % quads) * 4;
+  const int h0 = blockIdx.y * hpc, h1 = min(BH, h0 + hpc);
+  const long long off = (long long)t * d + c, hstride = (long long)n * d;
+  if (t < prefix) {
+    for (int h = h0; h < h1; ++h) st4(out + h * hstride + off, ld4(X + h * hstride + off));
+    return;
+  }
   const double2* tp = tab + (long long)(t - prefix) * (d / 2) + c / 2;         // pairs c / 2 and c / 2 + 1
   const double2 r0 = tp[0], r1 = tp[1];
   const double c0 = r0.x, s0 = r0.y * sign, c1 = r1.x, s1 = r1.y * sign;
-  const double a0 = v.x, b0 = v.y, a1 = v.z, b1 = v.w;
-  o[0] = from_d<T>(a0 * c0 - b0 * s0);
-  o[1] = from_d<T>(a0 * s0 + b0 * c0);
-  o[2] = from_d<T>(a1 * c1 - b1 * s1);
-  o[3] = from_d<T>(a1 * s1 + b1 * c1);
+  auto turn = [&](const float4& v, T* o) {
+    const double a0 = v.x, b0 = v.y, a1 = v.z, b1 = v.w;
+    float4 w;
+    w.x = to_f(from_d<T>(a0 * c0 - b0 * s0)); w.y = to_f(from_d<T>(a0 * s0 + b0 * c0));
+    w.z = to_f(from_d<T>(a1 * c1 - b1 * s1)); w.w = to_f(from_d<T>(a1 * s1 + b1 * c1));
+    st4(o, w);                                                                // already rounded to T: the store converts exactly
+  };
+  int h = h0;
+  for (; h + 3 < h1; h += 4) {                                                // four loads in flight
+    float4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v[u] = ld4(X + (h + u) * hstride + off);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) turn(v[u], out + (h + u) * hstride + off);
+  }
+  for (; h < h1; ++h) turn(ld4(X + h * hstride + off), out + h * hstride + off);
 }
 
 // out[bh][prefix + r gw + q][c] += sum_{a,b} w[h][c][a][b] src[bh][prefix + (r + a - ks/2) gw + (q + b - ks/2)][c]   (flip = 0)
