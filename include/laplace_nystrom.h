@@ -93,7 +93,7 @@ typedef struct ln_problem {
                           /* differentiates the linear system the solver approximates: dM = the same ns_iters-step         */
                           /* iterate of the system with right-hand side dY, dW = -dM Y^T (the paper names the solver       */
                           /* only).  The recurrence runs in double precision, one CTA per head, for either storage dtype.  Needs the symmetric     */
-                          /* matrix of one landmark set: lm_mode 3 is LN_ERR_UNSUPPORTED.  dev_status bit 0 then means a   */
+                          /* matrix of one landmark set: lm_mode 3 is LN_ERR_UNSUPPORTED, and so is whiten_mode 1 (not built).  dev_status bit 0 then means a   */
                           /* non-finite entry of Y.                                                                        */
 } ln_problem;
 

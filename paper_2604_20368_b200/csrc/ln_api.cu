@@ -268,7 +268,7 @@ int validate(const ln_problem* p) {
   if (p->map_mode != 0 && p->map_mode != 1) return LN_ERR_ARG;
   if (p->lm_mode < 0 || p->lm_mode > 3) return LN_ERR_ARG;
   if (p->solver != 0 && p->solver != 1) return LN_ERR_ARG;
-  if (p->solver == 1 && p->lm_mode == 3) return LN_ERR_UNSUPPORTED;
+  if (p->solver == 1 && (p->lm_mode == 3 || p->whiten_mode == 1)) return LN_ERR_UNSUPPORTED;
   if (p->whiten && !aligned16(p->whiten)) return LN_ERR_ARG;
   if (p->whiten_mode != 0 && p->whiten_mode != 1) return LN_ERR_ARG;
   if (p->whiten_mode == 1) {

@@ -172,6 +172,8 @@ def test_solver_argument_errors_without_gpu():
     assert fwd(with_solver(2, 1)) == -1
     assert fwd(with_solver(-1, 1)) == -1
     assert fwd(with_solver(1, 3)) == -2                             # W = k(pool Q, pool K) is not symmetric
+    bw = with_solver(1, 1); bw.whiten_mode, bw.whiten, bw.whiten_batch = 1, None, a.value
+    assert fwd(bw) == -2                                            # batch-statistic whitening with this solver: not built
     # the solver's scratch is part of the workspace the caller is told to bring
     p0, p1 = with_solver(0, 1), with_solver(1, 1)
     for with_saved in (0, 1):
