@@ -34,6 +34,40 @@ def test_l1_kernel(batch, na, nb, d, dtype):
     assert rel_err(f64(rs), rso) < 2e-6
 
 
+@pytest.mark.parametrize("batch,na,nb,d", [(1, 300, 1000, 64), (2, 64, 2049, 32), (1, 1025, 513, 128), (1, 8, 4100, 40)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_l1_kernel_few_large_blocks_split_their_columns(batch, na, nb, d, dtype):
+    """Few, large blocks without row sums (the setting of the paper's kernel micro-benchmark, Sec. 4.3): the launch
+    splits the column range over the grid's third dimension; ragged last tiles in both directions."""
+    A, Bm = _rand((batch, na, d), 11, dtype), _rand((batch, nb, d), 12, dtype)
+    lam = float(max(d, 2))
+    K = ln.l1_kernel(A.to(DEV), Bm.to(DEV), lam)
+    Ko = oracle.l1_kernel(f64(A), f64(Bm), lam)
+    assert rel_err(f64(K), Ko) < 2e-6
+    assert np.abs(f64(K) - Ko).max() < 4e-6
+    # and the same values as the unsplit launch that also returns row sums
+    K2, _ = ln.l1_kernel(A.to(DEV), Bm.to(DEV), lam, want_rowsum=True)
+    assert torch.equal(K, K2)
+
+
+@pytest.mark.parametrize("batch,na,nb,d", [(1, 300, 777, 64), (2, 130, 1000, 32), (1, 70, 2049, 128)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_l1_kernel_bwd_few_large_blocks(batch, na, nb, d, dtype):
+    """Gradient of few, large kernel blocks: the pass over the rows splits the columns into partial sums; the upstream
+    factor dK o K / lambda is formed inside the two sign kernels."""
+    A, Bm = _rand((batch, na, d), 14, dtype), _rand((batch, nb, d), 15, dtype)
+    A[0, 3] = Bm[0, 700]                                   # exact ties in the last column range: sign(0) = 0
+    A[0, 4, : d // 2] = Bm[0, 2, : d // 2]
+    dK = _rand((batch, na, nb), 16, torch.float32)
+    lam = float(d)
+    for Kmat in (None, ln.l1_kernel(A.to(DEV), Bm.to(DEV), lam)):
+        dA, dB = ln.l1_kernel_bwd(A.to(DEV), Bm.to(DEV), lam, dK.to(DEV), Kmat=Kmat)
+        dAo, dBo = oracle.l1_kernel_bwd(f64(A), f64(Bm), lam, f64(dK))
+        tol = 1e-5 if dtype == torch.float32 else 5e-3    # bf16: only the output rounding
+        assert rel_err(f64(dA), dAo) < tol
+        assert rel_err(f64(dB), dBo) < tol
+
+
 def test_l1_kernel_exact_properties():
     A = _rand((2, 90, 64), 3, torch.float32).to(DEV)
     K = ln.l1_kernel(A, A, 64.0)
