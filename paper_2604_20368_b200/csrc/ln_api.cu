@@ -1505,10 +1505,18 @@ int laplace_attention_block_bwd(const ln_problem* p, const ln_block* b, const vo
     const int ch = dwc_chunks(p), BH = p->B * p->H, cnt = p->d * b->dwc_ks * b->dwc_ks;
     if (p->dtype == LN_F32) {
       launch_dwc_add<float>("dwc_dV", p, b, dO, dV, 1, st);
+      if (b->dwc_ks == 3)
+        LN_LAUNCH("dwc_wgrad", st, k_dwc_wgrad3<float><<<dim3(ch, BH), 256, 0, st>>>((const float*)V, (const float*)dO, wpart, p->n, p->d, p->prefix,
+                                                                                     p->gh, p->gw, dwc_tokens_per_chunk(p)));
+      else
       LN_LAUNCH("dwc_wgrad", st, k_dwc_wgrad<float><<<dim3(ch, BH, b->dwc_ks), 256, 0, st>>>((const float*)V, (const float*)dO, wpart, p->n, p->d, p->prefix,
                                                                                             p->gh, p->gw, b->dwc_ks, dwc_tokens_per_chunk(p)));
     } else {
       if (!fused_dwc) launch_dwc_add<bf16>("dwc_dV", p, b, dO, dV, 1, st);
+      if (b->dwc_ks == 3)
+        LN_LAUNCH("dwc_wgrad", st, k_dwc_wgrad3<bf16><<<dim3(ch, BH), 256, 0, st>>>((const bf16*)V, (const bf16*)dO, wpart, p->n, p->d, p->prefix,
+                                                                                    p->gh, p->gw, dwc_tokens_per_chunk(p)));
+      else
       LN_LAUNCH("dwc_wgrad", st, k_dwc_wgrad<bf16><<<dim3(ch, BH, b->dwc_ks), 256, 0, st>>>((const bf16*)V, (const bf16*)dO, wpart, p->n, p->d, p->prefix,
                                                                                            p->gh, p->gw, b->dwc_ks, dwc_tokens_per_chunk(p)));
     }

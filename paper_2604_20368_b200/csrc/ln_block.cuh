@@ -145,6 +145,55 @@ __global__ void __launch_bounds__(256) k_dwc_wgrad(const T* __restrict__ V, cons
   }
 }
 
+// The same for the common 3 x 3 filter with all nine taps in one CTA (grid (chunks, BH)): the upstream row of a token is
+// read once, not once per filter row, and the nine neighbour loads of a token are in flight together; a tap outside the
+// grid contributes a zero.
+template <typename T>
+__global__ void __launch_bounds__(256) k_dwc_wgrad3(const T* __restrict__ V, const T* __restrict__ dO, float* __restrict__ part,
+                                                   int n, int d, int prefix, int gh, int gw, int tpc) {
+  __shared__ float red[256][9][4];
+  const int chunk = blockIdx.x, bh = blockIdx.y;
+  const int quads = d / 4, lanes = 256 / quads, q = (int)threadIdx.x % quads, tl = (int)threadIdx.x / quads, c = 4 * q;
+  float acc[9][4];
+#pragma unroll
+  for (int t = 0; t < 9; ++t)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) acc[t][e] = 0.f;
+  const T* Vh = V + (long long)bh * n * d + c;
+  const T* Gh = dO + (long long)bh * n * d + c;
+  const int t0 = chunk * tpc, t1 = min(gh * gw, t0 + tpc);
+  if (tl < lanes)
+    for (int tok = t0 + tl; tok < t1; tok += lanes) {
+      const int r = tok / gw, q0 = tok % gw;
+      const float4 g = ld4(Gh + (long long)(prefix + tok) * d);
+      float4 v[9];
+#pragma unroll
+      for (int t = 0; t < 9; ++t) {
+        const int rr = r + t / 3 - 1, qq = q0 + t % 3 - 1;
+        v[t] = (rr >= 0 && rr < gh && qq >= 0 && qq < gw) ? ld4(Vh + (long long)(prefix + rr * gw + qq) * d) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int t = 0; t < 9; ++t) {
+        acc[t][0] = fmaf(g.x, v[t].x, acc[t][0]); acc[t][1] = fmaf(g.y, v[t].y, acc[t][1]);
+        acc[t][2] = fmaf(g.z, v[t].z, acc[t][2]); acc[t][3] = fmaf(g.w, v[t].w, acc[t][3]);
+      }
+    }
+#pragma unroll
+  for (int t = 0; t < 9; ++t)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) red[threadIdx.x][t][e] = acc[t][e];
+  __syncthreads();
+  // 36 outputs per channel quad: thread (quad q, lane tl) adds the lanes for outputs tl, tl + lanes, ... in a fixed order
+  float* o = part + (((long long)bh * gridDim.x + chunk) * d + c) * 9;
+  if (tl < lanes)
+    for (int k = tl; k < 36; k += lanes) {
+      const int e = k / 9, t = k % 9;
+      float sacc = 0.f;
+      for (int w = 0; w < lanes; ++w) sacc += red[w * quads + q][t][e];
+      o[e * 9 + t] = sacc;
+    }
+}
+
 // dW[h][e] = sum over the batch elements b and the chunks of part[b H + h][chunk][e]; e < count = d ks ks (a multiple of 4).
 // grid (ceil(count / 128), H): warp w of a CTA adds the parts w, w + 8, ... for 128 consecutive elements, the eight warps
 // are added in a fixed order.
