@@ -1338,54 +1338,62 @@ __device__ void ns_tail_gw_sym(int m, int ldm, const float* __restrict__ W, floa
 // conjugacy), although the iterate itself depends on W and B only mildly; the inputs stay fp32.
 // W: fp32 [m][m] without the ridge; Bsrc: fp32 [m][D]; Xout: fp32 [m][D]; scratch: 4 m D doubles (x, r, p, Wr p).
 // Thread t always works on column t % D (256 % D == 0); the dot products of a column are added over the 256 / D
-// threads that share it in a fixed order.  red: >= 2 * 256 + 8 floats; gsm: >= 16 KiB of shared memory.
+// threads that share it in a fixed order.  red: >= 2 * 256 + 8 floats; gsm: >= 18 KiB of shared memory.
 // =====================================================================================
-// Q = (W + eps I) P in double: 64 x 64 output tiles, K in chunks of 16, a 4 x 4 block per thread
+// Q = (W + eps I) P in double on the FP64 tensor-core instruction (mma.sync m8n8k4; plain DFMA runs at 8 per clock
+// and SM on this part, a sixteenth of the FP32 rate, and bound the solver): 64 x 64 output tiles, K in chunks of 16
+// staged in shared memory; warp w owns rows 32 (w / 4) .. + 31 and columns 16 (w % 4) .. + 15 of the tile, i.e. 4 x 2
+// fragments of 8 x 8.  Fragment layout of the instruction: lane T holds A[T / 4][T % 4], B[T % 4][T / 4] and
+// C[T / 4][2 (T % 4)], C[T / 4][2 (T % 4) + 1].
+__device__ __forceinline__ void dmma884(double (&c)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};" : "+d"(c[0]), "+d"(c[1]) : "d"(a), "d"(b));
+}
 template <int D>
 __device__ void cg_matvec(int m, float eps, const float* __restrict__ W, const double* __restrict__ P, double* __restrict__ Q, double* gsm) {
-  double (*As)[64] = reinterpret_cast<double (*)[64]>(gsm);            // [16][64]: As[kk][i] = Wr[i0 + i][k0 + kk]
-  double (*Bs)[64] = reinterpret_cast<double (*)[64]>(gsm + 16 * 64);  // [16][64]: Bs[kk][j] = P[k0 + kk][j0 + j]
-  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  constexpr int PA = 17, PB = 72;                                      // pitches (doubles): conflict-free fragment reads
+  double* As = gsm;                                                    // [64][PA]: As[i][kk] = Wr[i0 + i][k0 + kk]
+  double* Bs = gsm + 64 * PA;                                          // [16][PB]: Bs[kk][j] = P[k0 + kk][j0 + j]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, lr = lane >> 2, lc = lane & 3;
+  const int wr = (warp >> 2) * 32, wc = (warp & 3) * 16;
   for (int i0 = 0; i0 < m; i0 += 64)
     for (int j0 = 0; j0 < D; j0 += 64) {
-      double acc[4][4];
+      double acc[4][2][2];
 #pragma unroll
       for (int a = 0; a < 4; ++a)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+        for (int b = 0; b < 2; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
       for (int k0 = 0; k0 < m; k0 += 16) {
         __syncthreads();
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const int e = tid + 256 * u;
           { const int i = e >> 4, kk = e & 15, gi = i0 + i, gk = k0 + kk;                 // consecutive threads along k
-            As[kk][i] = (gi < m && gk < m) ? (double)W[(long long)gi * m + gk] + (gi == gk ? (double)eps : 0.0) : 0.0; }
+            As[i * PA + kk] = (gi < m && gk < m) ? (double)W[(long long)gi * m + gk] + (gi == gk ? (double)eps : 0.0) : 0.0; }
           { const int kk = e >> 6, j = e & 63, gk = k0 + kk, gj = j0 + j;
-            Bs[kk][j] = (gk < m && gj < D) ? P[(long long)gk * D + gj] : 0.0; }
+            Bs[kk * PB + j] = (gk < m && gj < D) ? P[(long long)gk * D + gj] : 0.0; }
         }
         __syncthreads();
 #pragma unroll
-        for (int kk = 0; kk < 16; ++kk) {
-          double a4[4], b4[4];
-          {
-            const double2 a01 = *reinterpret_cast<const double2*>(&As[kk][ty * 4]), a23 = *reinterpret_cast<const double2*>(&As[kk][ty * 4 + 2]);
-            const double2 b01 = *reinterpret_cast<const double2*>(&Bs[kk][tx * 4]), b23 = *reinterpret_cast<const double2*>(&Bs[kk][tx * 4 + 2]);
-            a4[0] = a01.x; a4[1] = a01.y; a4[2] = a23.x; a4[3] = a23.y;
-            b4[0] = b01.x; b4[1] = b01.y; b4[2] = b23.x; b4[3] = b23.y;
-          }
+        for (int k4 = 0; k4 < 16; k4 += 4) {
+          double af[4], bf[2];
+#pragma unroll
+          for (int a = 0; a < 4; ++a) af[a] = As[(wr + 8 * a + lr) * PA + k4 + lc];
+#pragma unroll
+          for (int b = 0; b < 2; ++b) bf[b] = Bs[(k4 + lc) * PB + wc + 8 * b + lr];
 #pragma unroll
           for (int a = 0; a < 4; ++a)
 #pragma unroll
-            for (int b = 0; b < 4; ++b) acc[a][b] = fma(a4[a], b4[b], acc[a][b]);
+            for (int b = 0; b < 2; ++b) dmma884(acc[a][b], af[a], bf[b]);
         }
       }
 #pragma unroll
       for (int a = 0; a < 4; ++a) {
-        const int gi = i0 + ty * 4 + a;
+        const int gi = i0 + wr + 8 * a + lr;
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-          const int gj = j0 + tx * 4 + b;
-          if (gi < m && gj < D) Q[(long long)gi * D + gj] = acc[a][b];
+        for (int b = 0; b < 2; ++b) {
+          const int gj = j0 + wc + 8 * b + 2 * lc;
+          if (gi < m && gj < D) Q[(long long)gi * D + gj] = acc[a][b][0];
+          if (gi < m && gj + 1 < D) Q[(long long)gi * D + gj + 1] = acc[a][b][1];
         }
       }
     }
