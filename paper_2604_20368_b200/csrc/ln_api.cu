@@ -130,7 +130,7 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   // fused sign pass (64-dim slabs): token tiles of 8 * TG tokens that hug n, chunks for about three waves
   pl->s2_tg = pl->s2_rpc = pl->s2_chunks = pl->s2q_rpc = pl->s2q_chunks = 0; pl->s2_smem = 0;
   // per-head kernels (bf16 storage): three CTAs per SM for m <= 64, one for m <= 128, else clusters of four CTAs, two per SM
-  pl->mid_sms = p->m <= 64 ? (pl->BH + 2) / 3 : (p->m <= 128 ? pl->BH : 4 * pl->BH);
+  pl->mid_sms = p->m <= 64 ? (pl->BH + 2) / 3 : (p->m <= 128 ? pl->BH : kU2Cluster * pl->BH);
   if (p->d % 64 == 0) {
     const int groups = (p->n + 7) / 8;
     int tiles = (groups + S2_TGMAX - 1) / S2_TGMAX;
@@ -545,7 +545,7 @@ int fwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     else if (two) launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));
     else if (TC && m <= 64) launch(k_mid_fwd<D, TC, TC ? 64 : 0>, 3 * kUmmaMatBytes64);
     else if (TC && m <= 128) launch(k_mid_fwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
-    else if (TC) launch(k_mid_fwd<D, TC, TC ? 256 : 0, TC ? kMidCluster : 1>, 3 * kUmmaMatBytes, kMidCluster);   // m > 128: a cluster per head
+    else if (TC) launch(k_mid_fwd<D, TC, TC ? 256 : 0, TC ? kU2Cluster : 1>, 3 * kUmmaMatBytes, kU2Cluster);   // m > 128: a cluster per head
     else launch(k_mid_fwd<D, TC, 0>, sizeof(NsSmem));
   };
   {
@@ -704,7 +704,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
     else if (two) launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
     else if (TC && m <= 64) launch(k_mid_bwd<D, TC, TC ? 64 : 0>, 4 * kUmmaMatBytes64);
     else if (TC && m <= 128) launch(k_mid_bwd<D, TC, TC ? 128 : 0>, 3 * kUmmaMatBytes);
-    else if (TC) launch(k_mid_bwd<D, TC, TC ? 256 : 0, TC ? kMidCluster : 1>, 3 * kUmmaMatBytes, kMidCluster);
+    else if (TC) launch(k_mid_bwd<D, TC, TC ? 256 : 0, TC ? kU2Cluster : 1>, 3 * kUmmaMatBytes, kU2Cluster);
     else launch(k_mid_bwd<D, TC, 0>, sizeof(NsSmem));
   };
   // key-side products: g^R = (V dM^T) o R^T / lambda and dV = R^T dM (they need dM from the per-head kernel)
@@ -753,7 +753,7 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // Z'^T dO is needed by the per-head kernel only: it goes to the side stream too unless that stream is expected to be
   // the longer one anyway (estimates in microseconds: 7 / 16 / 30 per step and wave of heads for m <= 64 / <= 128 /
   // larger; the sign pass at 0.43 of the FP32 peak, 0.25 for small launches)
-  const int mid_waves = (int)(m <= 64 ? cdiv(BH, 3 * kSMs) : (m <= 128 ? cdiv(BH, kSMs) : cdiv(4ll * BH, kSMs)));
+  const int mid_waves = (int)(m <= 64 ? cdiv(BH, 3 * kSMs) : (m <= 128 ? cdiv(BH, kSMs) : cdiv((long long)kU2Cluster * BH, kSMs)));
   const double side_us = pl.T * (m <= 64 ? 7.0 : (m <= 128 ? 16.0 : 30.0)) * mid_waves;
   const double sign_ops = 3.0 * n * m * D * BH;
   const double main_us = sign_ops / (37.2e6 * (sign_ops > 4e9 ? 0.43 : 0.25));

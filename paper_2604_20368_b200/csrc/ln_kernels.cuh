@@ -1574,8 +1574,9 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     __syncthreads();
   } else if constexpr (MP == 256) {             // tcgen05 + TMEM, 2 x 2 blocks of 128 shared by the four CTAs of a cluster
     __shared__ UmmaCtl ctl;
-    __shared__ __align__(8) unsigned long long mbar_free;
-    tc_ok = ns_forward_umma256(m, T, eps, alpha_in, W, Wr, P, Xh, Ph, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl, &mbar_free, crank, bad);
+    __shared__ __align__(8) unsigned long long mbars[3];
+    static_assert(MP != 256 || CL == kU2Cluster, "the 256-wide engine is written for its own cluster size");
+    tc_ok = ns_forward_umma256(m, T, eps, alpha_in, W, P, Xh, Ph, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl, mbars, crank, bad);
     __syncthreads();
   } else {
     ns_forward_dev<TC, CL>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red, crank, Ph);
@@ -1722,8 +1723,8 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     if (dev_status && !tc_ok && tid == 0) atomicOr(dev_status + bh, 2);
   } else if constexpr (MP == 256) {
     __shared__ UmmaCtl ctl;
-    __shared__ __align__(8) unsigned long long mbar_free;
-    const bool tc_ok = ns_backward_umma256(m, T, Xh, Ph, dXm, Ga, Gb, Hm, P, dWm, reinterpret_cast<bf16*>(dyn_smem), ctl, &mbar_free, crank);
+    __shared__ __align__(8) unsigned long long mbars[3];
+    const bool tc_ok = ns_backward_umma256(m, T, Xh, Ph, dXm, Ga, Gb, Hm, Wr, P, dWm, reinterpret_cast<bf16*>(dyn_smem), ctl, mbars, crank);
     if (dev_status && !tc_ok && tid == 0 && crank == 0) atomicOr(dev_status + bh, 2);
     // end of the adjoint and GW in one pass (the operand buffers are free: the engine has ended with a cluster barrier)
     ns_tail_gw_sym<CL>(m, ldm, W, eps, hdr, P, dWm, inv_lambda, GW, red, reinterpret_cast<float*>(dyn_smem), crank);
