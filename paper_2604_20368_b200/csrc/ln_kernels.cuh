@@ -1248,8 +1248,8 @@ __device__ void ns_backward_tail_dev(int m, const float* Wr, const NsHdr* hdr, c
 //   dW_total = dWacc + alpha G^T + dalpha d(alpha)/dW,   dalpha = <G, Wr^T> = <G, Wr>,
 //   GW = (dW_total o W + (dW_total o W)^T) / lambda = (F + F^T + E + E^T) o W / lambda,   F = dWacc + alpha G,
 // E the two rank-one corrections of the norm gradient (column jstar of ||.||_1, row istar of ||.||_inf).  Transposed
-// tiles go through shared memory (32 x 32, two per round); CL CTAs share the tiles.  G, dWacc: fp32 [m][m]; GW: [m][ldm],
-// columns >= m zero.  tile: >= 2 * 32 * 33 + 512 floats of shared memory.
+// tiles go through shared memory (32 x 32, four per round); CL CTAs share the tiles.  G, dWacc: fp32 [m][m]; GW: [m][ldm],
+// columns >= m zero.  tile: >= 4 * 32 * 33 + 512 floats of shared memory.
 template <int CL>
 __device__ void ns_tail_gw_sym(int m, int ldm, const float* __restrict__ W, float eps, const NsHdr* hdr, const float* __restrict__ G,
                                const float* __restrict__ dWacc, float inv_lambda, float* __restrict__ GW, float* red, float* tile, int crank) {
@@ -1257,7 +1257,7 @@ __device__ void ns_tail_gw_sym(int m, int ldm, const float* __restrict__ W, floa
   const unsigned mm = (unsigned)m * (unsigned)m, dstep = (unsigned)m + 1u;
   const float alpha = hdr->alpha;
   const int js = hdr->jstar, is = hdr->istar;
-  float* sgc = tile + 2 * 32 * 33;          // sign of column jstar of Wr
+  float* sgc = tile + 4 * 32 * 33;          // sign of column jstar of Wr
   float* sgr = sgc + 256;                   // sign of row istar of Wr
   for (int i = tid; i < m; i += 256) {
     const float wc = W[(long long)i * m + js] + (i == js ? eps : 0.f), wr = W[(long long)is * m + i] + (i == is ? eps : 0.f);
@@ -1283,10 +1283,11 @@ __device__ void ns_tail_gw_sym(int m, int ldm, const float* __restrict__ W, floa
   const float dalpha = block_sum(p16[0], red);          // ends with a barrier: sgc / sgr are complete as well
   const float c1 = hdr->auto_alpha ? dalpha * (-alpha / hdr->n1) : 0.f, c2 = hdr->auto_alpha ? dalpha * (-alpha / hdr->ninf) : 0.f;
   const int nti = (m + 31) / 32, ntj = (ldm + 31) / 32, ntiles = nti * ntj;
-  for (int t0 = crank; t0 < ntiles; t0 += 2 * CL) {
-    float f[2][4], w[2][4], ft[2][4];
+  constexpr int NT = 4;                      // tiles per round: their loads are in flight together
+  for (int t0 = crank; t0 < ntiles; t0 += NT * CL) {
+    float f[NT][4], w[NT][4], ft[NT][4];
 #pragma unroll
-    for (int q = 0; q < 2; ++q) {
+    for (int q = 0; q < NT; ++q) {
       const int t = t0 + q * CL, I = t / ntj, J = t % ntj;
 #pragma unroll
       for (int r = 0; r < 4; ++r) {
@@ -1303,12 +1304,12 @@ __device__ void ns_tail_gw_sym(int m, int ldm, const float* __restrict__ W, floa
     }
     __syncthreads();                                                   // the tiles of the previous round have been read
 #pragma unroll
-    for (int q = 0; q < 2; ++q)
+    for (int q = 0; q < NT; ++q)
 #pragma unroll
       for (int r = 0; r < 4; ++r) tile[q * (32 * 33) + (ty + 8 * r) * 33 + tx] = ft[q][r];
     __syncthreads();
 #pragma unroll
-    for (int q = 0; q < 2; ++q) {
+    for (int q = 0; q < NT; ++q) {
       const int t = t0 + q * CL, I = t / ntj, J = t % ntj;
       if (t >= ntiles) continue;
 #pragma unroll

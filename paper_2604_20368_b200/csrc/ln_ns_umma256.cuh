@@ -178,9 +178,21 @@ __device__ bool ns_forward_umma256(int m, int T, float eps, float alpha_in, cons
 #pragma unroll 1
     for (int pass = (T == 0 ? 2 : 0); pass < 4; ++pass) {      // passes 0, 1: Wr blocks (ri, 0), (ri, 1); 2, 3: X_0 blocks
       const int ci = pass & 1, gj0 = ci * 128 + col0;
-      if (pass < 2) {
+      if (pass < 2) {                                          // a row of W: 128-bit loads where the row allows
 #pragma unroll
-        for (int q = 0; q < 64; ++q) v[q] = (gi < m && gj0 + q < m) ? W[(long long)gi * m + gj0 + q] + (gi == gj0 + q ? eps : 0.f) : 0.f;
+        for (int q = 0; q < 64; q += 4) {
+          if (gi < m && gj0 + q + 3 < m && (m & 3) == 0) {
+            const float4 t = *reinterpret_cast<const float4*>(W + (long long)gi * m + gj0 + q);
+            v[q] = t.x; v[q + 1] = t.y; v[q + 2] = t.z; v[q + 3] = t.w;
+          } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[q + u] = (gi < m && gj0 + q + u < m) ? W[(long long)gi * m + gj0 + q + u] : 0.f;
+          }
+        }
+        if (gi < m && gi >= gj0 && gi < gj0 + 64) {
+#pragma unroll
+          for (int q = 0; q < 64; ++q) if (gi == gj0 + q) v[q] += eps;
+        }
       } else {
 #pragma unroll
         for (int q = 0; q < 64; ++q) v[q] = (gi < m && gj0 + q < m) ? alpha * (W[(long long)(gj0 + q) * m + gi] + (gi == gj0 + q ? eps : 0.f)) : 0.f;
