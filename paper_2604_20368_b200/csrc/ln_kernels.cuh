@@ -1566,6 +1566,10 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     for (long long e = (long long)gt * 4; e < md; e += 4 * gn)
       *reinterpret_cast<float4*>(Mout + e) = sum_parts4(Mpart, nchunks, md, e);
   const float* XT = Xh + (long long)T * mx;
+  // the 256-wide engine keeps one tensor-memory allocation for the iteration and the product Y = X_T M
+  __shared__ UmmaCtl ctl256;
+  __shared__ __align__(8) unsigned long long mbars256[3];
+  U2Ctx u2c;
   if ((phase & 1) && solver == 0) {
   bool tc_ok = true;
   float bad = 0.f;                               // non-finite entries of X_T seen by this thread
@@ -1574,10 +1578,10 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     tc_ok = ns_forward_umma<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl, bad);
     __syncthreads();
   } else if constexpr (MP == 256) {             // tcgen05 + TMEM, 2 x 2 blocks of 128 shared by the four CTAs of a cluster
-    __shared__ UmmaCtl ctl;
-    __shared__ __align__(8) unsigned long long mbars[3];
     static_assert(MP != 256 || CL == kU2Cluster, "the 256-wide engine is written for its own cluster size");
-    tc_ok = ns_forward_umma256(m, T, eps, alpha_in, W, P, Xh, Ph, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl, mbars, crank, bad);
+    u2_begin(u2c, ctl256, mbars256, reinterpret_cast<bf16*>(dyn_smem), 256);
+    tc_ok = ns_forward_umma256(u2c, m, T, eps, alpha_in, W, P, Wr, Xh, Ph, hdr, red, crank, bad);
+    if (!(phase & 2)) umma_end(ctl256, 256);
     __syncthreads();
   } else {
     ns_forward_dev<TC, CL>(m, T, eps, alpha_in, W, Wr, P, Xh, hdr, sm, red, crank, Ph);
@@ -1602,6 +1606,12 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
         if (tid == 0 && bad > 0.f) atomicOr(dev_status + bh, 1);
       }
     }
+  } else if constexpr (MP == 256) {               // Y = X M on the engine of the iteration (images of X_T in Wr, of M in P)
+    if (!(phase & 1)) u2_begin(u2c, ctl256, mbars256, reinterpret_cast<bf16*>(dyn_smem), 256);
+    const bool y_ok = u2_product_y(u2c, m, D, Wr, Mout, P, Y, crank);
+    umma_end(ctl256, 256);
+    if (dev_status && !y_ok && tid == 0 && crank == 0) atomicOr(dev_status + bh, 2);
+    phase_sync<CL>();
   } else {
     ns_gemm<TC, false, false>(m, D, m, XT, ldx, Mout, D, Y, D, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // Y = X M
     if (CL > 1) phase_sync<CL>();

@@ -37,7 +37,7 @@ __device__ __forceinline__ const bf16* u2_block(const float* slot, int bi, int b
 __device__ __forceinline__ float* u2_block_w(float* slot, int bi, int bj) { return slot + (long long)(bi * 2 + bj) * kU2BlockFloats; }
 
 // one group of a product: the A-side block S (how it is read), the two B-side blocks it multiplies (how they are
-// read), the two accumulators, and whether they are added to
+// read; Y may be NULL: one block product only), the two accumulators, and whether they are added to
 struct U2Group { const bf16* S; bool s_k; const bf16* X; const bf16* Y; bool b_k; uint32_t d0, d1; bool accumulate; };
 
 struct U2Ctx {
@@ -62,8 +62,10 @@ __device__ __forceinline__ void u2_run(U2Ctx& c, const U2Group (&g)[NG]) {
     umma::mbar_expect_tx(&c.ctl->mbar_ld, 2 * MATB);
     umma::bulk_load(c.buf[is], g[0].S, MATB, &c.ctl->mbar_ld);
     umma::bulk_load(c.buf[ix], g[0].X, MATB, &c.ctl->mbar_ld);
-    umma::mbar_expect_tx(c.mbar_ldy, MATB);
-    umma::bulk_load(c.buf[iy], g[0].Y, MATB, c.mbar_ldy);
+    if (g[0].Y) {
+      umma::mbar_expect_tx(c.mbar_ldy, MATB);
+      umma::bulk_load(c.buf[iy], g[0].Y, MATB, c.mbar_ldy);
+    }
 #pragma unroll 1
     for (int i = 0; i < NG; ++i) {
       c.ok &= umma::mbar_wait(&c.ctl->mbar_ld, c.ph_ld & 1);         // S and x are here: S x starts while y is still arriving
@@ -71,10 +73,12 @@ __device__ __forceinline__ void u2_run(U2Ctx& c, const U2Group (&g)[NG]) {
       umma::fence_after_sync();
       umma_gemm<128>(g[i].d0, c.buf[is], g[i].s_k, c.buf[ix], g[i].b_k, g[i].accumulate);
       if (i + 1 < NG) umma::commit(c.mbar_x);
-      c.ok &= umma::mbar_wait(c.mbar_ldy, c.ph_ldy & 1);
-      c.ph_ldy ^= 1u;
-      umma::fence_after_sync();
-      umma_gemm<128>(g[i].d1, c.buf[is], g[i].s_k, c.buf[iy], g[i].b_k, g[i].accumulate);
+      if (g[i].Y) {                                                    // a group may have one B-side block only
+        c.ok &= umma::mbar_wait(c.mbar_ldy, c.ph_ldy & 1);
+        c.ph_ldy ^= 1u;
+        umma::fence_after_sync();
+        umma_gemm<128>(g[i].d1, c.buf[is], g[i].s_k, c.buf[iy], g[i].b_k, g[i].accumulate);
+      }
       if (i + 1 < NG) {
         umma::commit(c.mbar_y);
         c.ok &= umma::mbar_wait(c.mbar_x, c.ph_x & 1);               // x's buffer has been read
@@ -84,8 +88,10 @@ __device__ __forceinline__ void u2_run(U2Ctx& c, const U2Group (&g)[NG]) {
         c.ok &= umma::mbar_wait(c.mbar_y, c.ph_y & 1);               // S's and y's buffers have been read
         c.ph_y ^= 1u;
         umma::bulk_load(c.buf[is], g[i + 1].X, MATB, &c.ctl->mbar_ld);
-        umma::mbar_expect_tx(c.mbar_ldy, MATB);
-        umma::bulk_load(c.buf[iy], g[i + 1].Y, MATB, c.mbar_ldy);
+        if (g[i + 1].Y) {
+          umma::mbar_expect_tx(c.mbar_ldy, MATB);
+          umma::bulk_load(c.buf[iy], g[i + 1].Y, MATB, c.mbar_ldy);
+        }
         const int t = is; is = ix; ix = t;                             // the next S sits where x was, the next x where S was
       }
     }
@@ -123,12 +129,13 @@ __device__ __forceinline__ void u2_begin(U2Ctx& c, UmmaCtl& ctl, unsigned long l
   umma_begin(ctl, ncols);
 }
 
-// Forward iteration, called by the two CTAs of a cluster (ri = 0, 1).  W: fp32 [m][m] (W + eps I is formed where it
-// is read); Wimg: scratch slot for the images of W + eps I; Xh: slots 0 .. T-1 receive the images of X_k, slot T X_T in
-// fp32 [m][m]; Ph: slot k receives the images of Q_k.  Returns false if a wait ran out.
-__device__ bool ns_forward_umma256(int m, int T, float eps, float alpha_in, const float* W, float* Wimg,
-                                   float* Xh, float* Ph, NsHdr* hdr, bf16* smem, float* red, UmmaCtl& ctl,
-                                   unsigned long long* mbars, int ri, float& bad) {
+// Forward iteration, called by the two CTAs of a cluster (ri = 0, 1) between u2_begin (256 columns of tensor memory)
+// and umma_end.  W: fp32 [m][m] (W + eps I is formed where it is read); Wimg: scratch slot for the images of W + eps I;
+// Xh: slots 0 .. T-1 receive the images of X_k, slot T X_T in fp32 [m][m]; XTimg: slot that receives the images of X_T
+// (for the product Y = X_T M); Ph: slot k receives the images of Q_k.  Returns false if a wait ran out.
+__device__ bool ns_forward_umma256(U2Ctx& c, int m, int T, float eps, float alpha_in, const float* W, float* Wimg, float* XTimg,
+                                   float* Xh, float* Ph, NsHdr* hdr, float* red, int ri, float& bad) {
+  UmmaCtl& ctl = *c.ctl;
   const int tid = threadIdx.x, warp = tid >> 5;
   const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64;
   const int gi = ri * 128 + row;                                 // this thread's row in the matrix
@@ -170,10 +177,8 @@ __device__ bool ns_forward_umma256(int m, int T, float eps, float alpha_in, cons
     __syncthreads();
   }
   const float alpha = red[512];
-  U2Ctx c;
-  u2_begin(c, ctl, mbars, smem, 256);
   const uint32_t t_acc[2] = {ctl.tmem_base, ctl.tmem_base + 128};
-  {  // X_0 = alpha Wr^T in fp32 (no steps), else the images of this CTA's blocks of Wr and of X_0
+  {  // the images of this CTA's blocks of Wr (not without steps) and of X_0 = alpha Wr^T (without steps also in fp32)
     float v[64];
 #pragma unroll 1
     for (int pass = (T == 0 ? 2 : 0); pass < 4; ++pass) {      // passes 0, 1: Wr blocks (ri, 0), (ri, 1); 2, 3: X_0 blocks
@@ -197,13 +202,14 @@ __device__ bool ns_forward_umma256(int m, int T, float eps, float alpha_in, cons
 #pragma unroll
         for (int q = 0; q < 64; ++q) v[q] = (gi < m && gj0 + q < m) ? alpha * (W[(long long)(gj0 + q) * m + gi] + (gi == gj0 + q ? eps : 0.f)) : 0.f;
       }
-      if (T == 0) {
+      if (T == 0) {                                            // X_T = X_0: fp32 to its slot, images to XTimg
         if (gi < m) {
 #pragma unroll
           for (int q = 0; q < 64; ++q) if (gj0 + q < m) Xh[(long long)gi * m + gj0 + q] = v[q];
         }
 #pragma unroll
         for (int q = 0; q < 64; ++q) bad += isfinite(v[q]) ? 0.f : 1.f;
+        u2_store_block(c, v, row, col0, u2_block_w(XTimg, ri, ci), ci, ci == 1);
       } else if (pass < 3) {
         u2_store_block(c, v, row, col0, pass < 2 ? u2_block_w(Wimg, ri, ci) : u2_block_w(Xh, ri, ci), pass, false);
       } else {
@@ -254,7 +260,7 @@ __device__ bool ns_forward_umma256(int m, int T, float eps, float alpha_in, cons
           }
 #pragma unroll
           for (int q = 0; q < 64; ++q) bad += isfinite(v[q]) ? 0.f : 1.f;
-          if (ci == 1) { umma::fence_before_sync(); __syncthreads(); }
+          u2_store_block(c, v, row, col0, u2_block_w(XTimg, ri, ci), ci, ci == 1);    // and as images, for Y = X_T M
         } else {
           u2_store_block(c, v, row, col0, u2_block_w(Xn, ri, ci), ci, ci == 1);
         }
@@ -262,9 +268,37 @@ __device__ bool ns_forward_umma256(int m, int T, float eps, float alpha_in, cons
     }
     phase_sync<kU2Cluster>();
   }
-  const bool ok = c.ok && ctl.timeout == 0;
-  umma_end(ctl, 256);
-  return ok;
+  return c.ok && ctl.timeout == 0;
+}
+
+// Y = X_T M on the same engine, between u2_begin and umma_end: M [m][D] (D <= 128, padded with zero columns) becomes two
+// block images (one per CTA, slot Mimg), Y[ri] = X_T[ri][0] M[0] + X_T[ri][1] M[1] goes into one accumulator and
+// leaves as fp32 rows.  Both CTAs must have passed a cluster barrier since M and the images of X_T were written.
+__device__ bool u2_product_y(U2Ctx& c, int m, int D, const float* XTimg, const float* M, float* Mimg, float* Y, int ri) {
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64, gi = ri * 128 + row;
+  const uint32_t t_acc = c.ctl->tmem_base;
+  float v[64];
+#pragma unroll
+  for (int q = 0; q < 64; q += 4) {
+    float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (gi < m && col0 + q < D) t = *reinterpret_cast<const float4*>(M + (long long)gi * D + col0 + q);   // D is a multiple of 4
+    v[q] = t.x; v[q + 1] = t.y; v[q + 2] = t.z; v[q + 3] = t.w;
+  }
+  u2_store_block(c, v, row, col0, u2_block_w(Mimg, 0, ri), 0, true);
+  phase_sync<kU2Cluster>();
+  const U2Group g[2] = {{u2_block(XTimg, ri, 0), true, u2_block(Mimg, 0, 0), nullptr, false, t_acc, t_acc, false},
+                        {u2_block(XTimg, ri, 1), true, u2_block(Mimg, 0, 1), nullptr, false, t_acc, t_acc, true}};
+  u2_run<2>(c, g);
+  umma_row<64>(t_acc, col0, v);
+  if (gi < m) {
+#pragma unroll
+    for (int q = 0; q < 64; q += 4)
+      if (col0 + q < D) *reinterpret_cast<float4*>(Y + (long long)gi * D + col0 + q) = make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+  }
+  umma::fence_before_sync();
+  __syncthreads();
+  return c.ok && c.ctl->timeout == 0;
 }
 
 // Adjoint for a symmetric W (same algebra as the 128 x 128 path): per step k, with A = X_k and Q = Q_k as the forward
