@@ -45,22 +45,31 @@ struct U2Ctx {
   unsigned long long* mbar_ldy;                 // arrival of the y block (S and x are counted on ctl->mbar_ld)
   bf16* buf[3];
   uint32_t phase, ph_ld, ph_ldy, ph_x, ph_y;    // ph_ld / ph_ldy / ph_x / ph_y are used by thread 0 only
+  bool pre;                                     // thread 0: the first S block of the next product is on its way into buffer 2
   bool ok;
 };
 
 // Writes of other CTAs to global memory (bulk copies, then the cluster barrier) are read here by bulk copies.
 __device__ __forceinline__ void u2_fence_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// All groups, one after the other; one thread fetches and issues, everybody waits for the last MMA.  All three
-// buffers are free on entry (the output images of the previous product have left).
+// All groups, one after the other; one thread fetches and issues, everybody waits for the last MMA.  Buffers 0 and 1
+// are free on entry (the output images of the previous product have left); buffer 2 is free, or already receives the
+// first S block (see next_S).
+// next_S: NULL, or the first S block of the NEXT call, which must not depend on what this product or the other CTA is
+// still writing: its fetch into buffer 2 starts as soon as the last MMA of this call has completed and runs beside the
+// epilogue (which stages the output images in buffers 0 and 1) and the cluster barrier.
 template <int NG>
-__device__ __forceinline__ void u2_run(U2Ctx& c, const U2Group (&g)[NG]) {
+__device__ __forceinline__ void u2_run(U2Ctx& c, const U2Group (&g)[NG], const bf16* next_S = nullptr) {
   constexpr uint32_t MATB = (uint32_t)kUmmaMatBytes;
   if (threadIdx.x == 0) {
     int is = 0, ix = 1, iy = 2;                                       // buffers of S, x, y of the current group
     u2_fence_async();
-    umma::mbar_expect_tx(&c.ctl->mbar_ld, 2 * MATB);
-    umma::bulk_load(c.buf[is], g[0].S, MATB, &c.ctl->mbar_ld);
+    if (c.pre) {                                                       // S is on its way (its bytes and x's were announced then)
+      is = 2; ix = 0; iy = 1;
+    } else {
+      umma::mbar_expect_tx(&c.ctl->mbar_ld, 2 * MATB);
+      umma::bulk_load(c.buf[is], g[0].S, MATB, &c.ctl->mbar_ld);
+    }
     umma::bulk_load(c.buf[ix], g[0].X, MATB, &c.ctl->mbar_ld);
     if (g[0].Y) {
       umma::mbar_expect_tx(c.mbar_ldy, MATB);
@@ -101,6 +110,13 @@ __device__ __forceinline__ void u2_run(U2Ctx& c, const U2Group (&g)[NG]) {
   c.ok &= umma::mbar_wait(&c.ctl->mbar, c.phase & 1);
   c.phase ^= 1u;
   umma::fence_after_sync();
+  if (threadIdx.x == 0) {
+    c.pre = next_S != nullptr;
+    if (next_S) {                                                      // every buffer has been read; the epilogue uses 0 and 1
+      umma::mbar_expect_tx(&c.ctl->mbar_ld, 2 * MATB);
+      umma::bulk_load(c.buf[2], next_S, MATB, &c.ctl->mbar_ld);
+    }
+  }
 }
 
 // This thread's 64 values of a block -> image in buffer `b`; then one thread sends the image to `dst` (a block in
@@ -124,7 +140,7 @@ __device__ __forceinline__ void u2_store_block(U2Ctx& c, const float (&v)[64], i
 __device__ __forceinline__ void u2_begin(U2Ctx& c, UmmaCtl& ctl, unsigned long long* mbars, bf16* smem, int ncols) {
   c.ctl = &ctl; c.mbar_x = mbars; c.mbar_y = mbars + 1; c.mbar_ldy = mbars + 2;
   c.buf[0] = smem; c.buf[1] = smem + 2 * UmmaGeo<128>::UIMG; c.buf[2] = smem + 4 * UmmaGeo<128>::UIMG;
-  c.phase = c.ph_ld = c.ph_ldy = c.ph_x = c.ph_y = 0; c.ok = true;
+  c.phase = c.ph_ld = c.ph_ldy = c.ph_x = c.ph_y = 0; c.ok = true; c.pre = false;
   if (threadIdx.x == 0) { umma::mbar_init(mbars, 1); umma::mbar_init(mbars + 1, 1); umma::mbar_init(mbars + 2, 1); }
   umma_begin(ctl, ncols);
 }
@@ -227,7 +243,7 @@ __device__ bool ns_forward_umma256(U2Ctx& c, int m, int T, float eps, float alph
     {  // Q_k = 2I - Wr X_k
       const U2Group g[2] = {{u2_block(Wimg, ri, 0), true, u2_block(X, 0, 0), u2_block(X, 0, 1), false, t_acc[0], t_acc[1], false},
                             {u2_block(Wimg, ri, 1), true, u2_block(X, 1, 0), u2_block(X, 1, 1), false, t_acc[0], t_acc[1], true}};
-      u2_run<2>(c, g);
+      u2_run<2>(c, g, u2_block(X, ri, 0));                      // X_k is complete: its block is fetched beside the epilogue
 #pragma unroll 1
       for (int ci = 0; ci < 2; ++ci) {
         const int gj0 = ci * 128 + col0;
@@ -242,7 +258,7 @@ __device__ bool ns_forward_umma256(U2Ctx& c, int m, int T, float eps, float alph
     {  // X_{k+1} = X_k Q_k
       const U2Group g[2] = {{u2_block(X, ri, 0), true, u2_block(Q, 0, 0), u2_block(Q, 0, 1), false, t_acc[0], t_acc[1], false},
                             {u2_block(X, ri, 1), true, u2_block(Q, 1, 0), u2_block(Q, 1, 1), false, t_acc[0], t_acc[1], true}};
-      u2_run<2>(c, g);
+      u2_run<2>(c, g, k + 1 < T ? u2_block(Wimg, ri, 0) : nullptr);
       float* Xn = Xh + (long long)(k + 1) * kU2Slot;
 #pragma unroll 1
       for (int ci = 0; ci < 2; ++ci) {
@@ -362,7 +378,7 @@ __device__ bool ns_backward_umma256(int m, int T, const float* Xh, const float* 
     {  // H = A^T G:  H[ri][ci] = sum_kb (A[kb][ri])^T G[kb][ci]
       const U2Group g[2] = {{u2_block(A, 0, ri), false, u2_block(Gcur, 0, 0), u2_block(Gcur, 0, 1), false, t_acc[0], t_acc[1], false},
                             {u2_block(A, 1, ri), false, u2_block(Gcur, 1, 0), u2_block(Gcur, 1, 1), false, t_acc[0], t_acc[1], true}};
-      u2_run<2>(c, g);
+      u2_run<2>(c, g, u2_block(Q, 0, ri));                      // the history is complete: first S of the next phase
 #pragma unroll 1
       for (int ci = 0; ci < 2; ++ci) {
         float v[64];
@@ -373,13 +389,14 @@ __device__ bool ns_backward_umma256(int m, int T, const float* Xh, const float* 
     phase_sync<kU2Cluster>();
     {  // dW accumulators += H A^T;  G Q^T + Q^T G
       const bool acc = k != T - 1;
-      const U2Group g[6] = {{u2_block(Himg, ri, 0), true, u2_block(A, 0, 0), u2_block(A, 1, 0), true, t_dw[0], t_dw[1], acc},
-                            {u2_block(Himg, ri, 1), true, u2_block(A, 0, 1), u2_block(A, 1, 1), true, t_dw[0], t_dw[1], true},
-                            {u2_block(Gcur, ri, 0), true, u2_block(Q, 0, 0), u2_block(Q, 1, 0), true, t_acc[0], t_acc[1], false},
+      // (the groups that read the history come first: their S block can be fetched before H has arrived)
+      const U2Group g[6] = {{u2_block(Q, 0, ri), false, u2_block(Gcur, 0, 0), u2_block(Gcur, 0, 1), false, t_acc[0], t_acc[1], false},
+                            {u2_block(Q, 1, ri), false, u2_block(Gcur, 1, 0), u2_block(Gcur, 1, 1), false, t_acc[0], t_acc[1], true},
+                            {u2_block(Gcur, ri, 0), true, u2_block(Q, 0, 0), u2_block(Q, 1, 0), true, t_acc[0], t_acc[1], true},
                             {u2_block(Gcur, ri, 1), true, u2_block(Q, 0, 1), u2_block(Q, 1, 1), true, t_acc[0], t_acc[1], true},
-                            {u2_block(Q, 0, ri), false, u2_block(Gcur, 0, 0), u2_block(Gcur, 0, 1), false, t_acc[0], t_acc[1], true},
-                            {u2_block(Q, 1, ri), false, u2_block(Gcur, 1, 0), u2_block(Gcur, 1, 1), false, t_acc[0], t_acc[1], true}};
-      u2_run<6>(c, g);
+                            {u2_block(Himg, ri, 0), true, u2_block(A, 0, 0), u2_block(A, 1, 0), true, t_dw[0], t_dw[1], acc},
+                            {u2_block(Himg, ri, 1), true, u2_block(A, 0, 1), u2_block(A, 1, 1), true, t_dw[0], t_dw[1], true}};
+      u2_run<6>(c, g, k > 0 ? u2_block(Xh + (long long)(k - 1) * kU2Slot, 0, ri) : nullptr);   // A of the next step
 #pragma unroll 1
       for (int ci = 0; ci < 2; ++ci) {
         const int gj0 = ci * 128 + col0;
