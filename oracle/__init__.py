@@ -280,29 +280,36 @@ def round_bf16(x):
     return np.ldexp(np.rint(mant * 256.0) / 256.0, expo)      # rint rounds halves to even
 
 
-def block_forward(p: Problem, Q, K, V, Wd=None, rope_base=0.0, whiten=None, store_bf16=False):
+def _round_storage(x, store_bf16, store_f32):
+    if store_bf16:
+        return round_bf16(x)
+    if store_f32:
+        return x.astype(np.float32).astype(np.float64)       # numpy rounds to nearest, ties to even
+    return x
+
+
+def block_forward(p: Problem, Q, K, V, Wd=None, rope_base=0.0, whiten=None, store_bf16=False, store_f32=False):
     """The attention block around the path: rotary embedding on Q and K (rope_base > 0), the Nystrom Laplacian
-    attention, plus DWC(V) (Wd given).  store_bf16: the rotated Q and K are rounded to bf16, as a device that keeps
-    them in bf16 storage does (the kernel gradient's sign(token - landmark) must be decided on the same numbers)."""
+    attention, plus DWC(V) (Wd given).  store_bf16 / store_f32: the rotated Q and K are rounded once to the type a
+    device keeps them in (the kernel gradient's sign(token - landmark) must be decided on the same numbers: a landmark
+    pooled from a single token equals that token only if both went through the same rounding)."""
     Qr, Kr = _f64(Q), _f64(K)
     if rope_base > 0:
         Qr, Kr = rope(Qr, p.prefix, rope_base), rope(Kr, p.prefix, rope_base)
-        if store_bf16:
-            Qr, Kr = round_bf16(Qr), round_bf16(Kr)
+        Qr, Kr = _round_storage(Qr, store_bf16, store_f32), _round_storage(Kr, store_bf16, store_f32)
     O = forward(p, Qr, Kr, V, whiten=whiten)
     if Wd is not None:
         O = O + dwc(V, Wd, p.prefix, p.gh, p.gw)
     return O
 
 
-def block_backward(p: Problem, Q, K, V, dO, Wd=None, rope_base=0.0, whiten=None, store_bf16=False):
+def block_backward(p: Problem, Q, K, V, dO, Wd=None, rope_base=0.0, whiten=None, store_bf16=False, store_f32=False):
     """Adjoint of block_forward: dQ, dK, dV, dWd (None without the convolution).  The rounding of the rotated
     tensors, where asked for, is treated as the identity (straight-through), as storage rounding is everywhere."""
     Qr, Kr = _f64(Q), _f64(K)
     if rope_base > 0:
         Qr, Kr = rope(Qr, p.prefix, rope_base), rope(Kr, p.prefix, rope_base)
-        if store_bf16:
-            Qr, Kr = round_bf16(Qr), round_bf16(Kr)
+        Qr, Kr = _round_storage(Qr, store_bf16, store_f32), _round_storage(Kr, store_bf16, store_f32)
     dQr, dKr, dV, _ = backward(p, Qr, Kr, V, dO, whiten=whiten)
     dWd = None
     if Wd is not None:

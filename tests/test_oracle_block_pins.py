@@ -130,3 +130,32 @@ def test_block_backward_finite_differences(rope_base, use_dwc):
         assert dWd is None
     # without rotation and convolution the block is the path itself
     np.testing.assert_array_equal(oracle.block_forward(p, Q, K, V, whiten=s), oracle.forward(p, Q, K, V, whiten=s))
+
+
+def test_rotated_tokens_enter_the_path_in_storage_precision():
+    # The rotated Q and K are rounded once to the storage type before the path sees them (what a device that stores them
+    # does): sign(token - landmark) in the kernel gradient is then decided on the stored numbers.  With fp32 storage a
+    # token coordinate lies within one rounding of a landmark coordinate about once per few hundred thousand (token,
+    # landmark, dim) triples; decided on the unrounded double it falls on the other side in half of those cases and one
+    # gradient entry changes by 2 g / lambda.
+    from dataclasses import replace
+    rng = np.random.default_rng(9)
+    d = 4
+    p = Problem(B=1, H=1, n=6, d=d, m=6, lam=float(d), ns_iters=3, ridge_eps=1e-3, map_mode=1, lm_mode=1, gh=2, gw=3, mh=2, mw=3, lm_f32=1)
+    Q, K, V, dO = (rng.standard_normal((1, 1, p.n, d)) for _ in range(4))
+    for flags in (dict(store_f32=True), dict(store_bf16=True)):
+        rnd = (lambda x: oracle.round_bf16(x)) if "store_bf16" in flags else (lambda x: x.astype(np.float32).astype(np.float64))
+        Qr, Kr = rnd(oracle.rope(Q, 0, 100.0)), rnd(oracle.rope(K, 0, 100.0))
+        # bins of one token: a landmark is its key, bit for bit, also after the landmarks' own cast to single precision
+        np.testing.assert_array_equal(oracle.landmarks_pool(replace(p, lm_f32=0), Kr), Kr)
+        assert (Kr.astype(np.float32).astype(np.float64) == Kr).all()
+        # the block entry points do exactly this: rotate, round, run the path; the gradient returns through the inverse rotation
+        np.testing.assert_array_equal(oracle.block_forward(p, Q, K, V, rope_base=100.0, **flags), oracle.forward(p, Qr, Kr, V))
+        dQr, dKr, dV, _ = oracle.backward(p, Qr, Kr, V, dO)
+        dQ, dK, dV2, _ = oracle.block_backward(p, Q, K, V, dO, rope_base=100.0, **flags)
+        np.testing.assert_array_equal(dQ, oracle.rope(dQr, 0, 100.0, inverse=True))
+        np.testing.assert_array_equal(dK, oracle.rope(dKr, 0, 100.0, inverse=True))
+        np.testing.assert_array_equal(dV, dV2)
+    # without a flag nothing is rounded
+    np.testing.assert_array_equal(oracle.block_forward(p, Q, K, V, rope_base=100.0),
+                                  oracle.forward(p, oracle.rope(Q, 0, 100.0), oracle.rope(K, 0, 100.0), V))
