@@ -129,7 +129,7 @@ bool make_plan(const ln_problem* p, Plan* pl) {
   pl->chunks = (p->n + rpc - 1) / rpc;
   // fused sign pass (64-dim slabs): token tiles of 8 * TG tokens that hug n, chunks for about three waves
   pl->s2_tg = pl->s2_rpc = pl->s2_chunks = pl->s2q_rpc = pl->s2q_chunks = 0; pl->s2_smem = 0;
-  // per-head kernels (bf16 storage): three CTAs per SM for m <= 64, one for m <= 128, else clusters of four CTAs, two per SM
+  // per-head kernels (bf16 storage): three CTAs per SM for m <= 64, one for m <= 128, else a cluster of two CTAs per head, one per SM
   pl->mid_sms = p->m <= 64 ? (pl->BH + 2) / 3 : (p->m <= 128 ? pl->BH : kU2Cluster * pl->BH);
   if (p->d % 64 == 0) {
     const int groups = (p->n + 7) / 8;
@@ -432,7 +432,7 @@ CopyStreams copy_acquire(cudaStream_t caller) {
 }
 
 // Launch with `cl` CTAs per thread-block cluster (cl = 1: an ordinary launch).
-constexpr int kMidCluster = 4;     // CTAs that share one head on the m > 128 Newton-Schulz path
+constexpr int kMidCluster = 4;     // CTAs that share one head on the general (two landmark sets) engine beyond 64 landmarks
 template <typename... KArgs, typename... Args>
 void launch_clustered(void (*kern)(KArgs...), int grid, int cl, size_t smem, cudaStream_t st, Args... args) {
   cudaLaunchConfig_t cfg = {};

@@ -1532,7 +1532,7 @@ __global__ void __launch_bounds__(256) k_ns_pinv_bwd(int m, int T, float eps, fl
 // so that O = (C - mu) Ytilde + ybar.  One CTA per head.
 // =====================================================================================
 // MP: 0 = matrices in global memory (fp32 FFMA or the cluster-shared mma.sync engine); 64 / 128 = one CTA per head on
-// tcgen05 with the matrix padded to MP; 256 = tcgen05 on 2 x 2 blocks of 128, CL = 4 CTAs of a thread-block cluster
+// tcgen05 with the matrix padded to MP; 256 = tcgen05 on 2 x 2 blocks of 128, CL = 2 CTAs of a thread-block cluster
 // per head (grid = heads * CL).
 template <int D, bool TC, int MP, int CL = 1>
 __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 : 1)) k_mid_fwd(int m, int ldm, int T, float eps, float alpha_in, int H, int map_mode,
@@ -1577,7 +1577,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     __shared__ UmmaCtl ctl;
     tc_ok = ns_forward_umma<MP>(m, T, eps, alpha_in, W, Xh, Ph, ldx, mx, hdr, reinterpret_cast<bf16*>(dyn_smem), red, ctl, bad);
     __syncthreads();
-  } else if constexpr (MP == 256) {             // tcgen05 + TMEM, 2 x 2 blocks of 128 shared by the four CTAs of a cluster
+  } else if constexpr (MP == 256) {             // tcgen05 + TMEM, 2 x 2 blocks of 128 shared by the two CTAs of a cluster
     static_assert(MP != 256 || CL == kU2Cluster, "the 256-wide engine is written for its own cluster size");
     u2_begin(u2c, ctl256, mbars256, reinterpret_cast<bf16*>(dyn_smem), 256);
     tc_ok = ns_forward_umma256(u2c, m, T, eps, alpha_in, W, P, Wr, Xh, Ph, hdr, red, crank, bad);
