@@ -1563,8 +1563,27 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
   Mout += bh * md; Y += bh * md; Yt += bh * md; ybar += (long long)bh * D;
   Mpart += (long long)bh * nchunks * md;
   if ((phase & 2) && nchunks > 0)                // nchunks == 0: the single partial result was written to Mout directly
-    for (long long e = (long long)gt * 4; e < md; e += 4 * gn)
-      *reinterpret_cast<float4*>(Mout + e) = sum_parts4(Mpart, nchunks, md, e);
+    // eight elements of this thread at a time: their loads of a part are in flight together, the parts in order
+    for (long long e0 = (long long)gt * 4; e0 < md; e0 += 32ll * gn) {
+      float4 acc[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int p = 0; p < nchunks; ++p) {
+        float4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const long long e = e0 + 4ll * u * gn;
+          v[u] = e < md ? *reinterpret_cast<const float4*>(Mpart + (long long)p * md + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { acc[u].x += v[u].x; acc[u].y += v[u].y; acc[u].z += v[u].z; acc[u].w += v[u].w; }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const long long e = e0 + 4ll * u * gn;
+        if (e < md) *reinterpret_cast<float4*>(Mout + e) = acc[u];
+      }
+    }
   const float* XT = Xh + (long long)T * mx;
   // the 256-wide engine keeps one tensor-memory allocation for the iteration and the product Y = X_T M
   __shared__ UmmaCtl ctl256;
@@ -1697,17 +1716,36 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     dyb[tid] = t;
   }
   __syncthreads();
-  for (long long e = (long long)gt * 4; e < md; e += 4 * gn) {
-    const float4 t = sum_parts4(dYtpart, nchunks, md, e);
-    const int l = (int)(e / D), c = (int)(e % D);
-    // Ytilde = P_c diag(s) Y, ybar = Y^T 1/m  ->  dY = diag(s) (centred Z'^T dO) + (1/m) 1 dyb^T
-    float4 o = t;
-    if (map_mode == 1) {
-      const float sl = s ? s[l] : 1.f, im = 1.f / (float)m;
-      o.x = sl * t.x + dyb[c] * im; o.y = sl * t.y + dyb[c + 1] * im;
-      o.z = sl * t.z + dyb[c + 2] * im; o.w = sl * t.w + dyb[c + 3] * im;
+  // eight elements of this thread at a time: their loads of a part are in flight together, the parts in order
+  for (long long e0 = (long long)gt * 4; e0 < md; e0 += 32ll * gn) {
+    float4 acc[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int p = 0; p < nchunks; ++p) {
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const long long e = e0 + 4ll * u * gn;
+        v[u] = e < md ? *reinterpret_cast<const float4*>(dYtpart + (long long)p * md + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { acc[u].x += v[u].x; acc[u].y += v[u].y; acc[u].z += v[u].z; acc[u].w += v[u].w; }
     }
-    *reinterpret_cast<float4*>(dY + e) = o;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const long long e = e0 + 4ll * u * gn;
+      if (e >= md) continue;
+      const float4 t = acc[u];
+      const int l = (int)(e / D), c = (int)(e % D);
+      // Ytilde = P_c diag(s) Y, ybar = Y^T 1/m  ->  dY = diag(s) (centred Z'^T dO) + (1/m) 1 dyb^T
+      float4 o = t;
+      if (map_mode == 1) {
+        const float sl = s ? s[l] : 1.f, im = 1.f / (float)m;
+        o.x = sl * t.x + dyb[c] * im; o.y = sl * t.y + dyb[c + 1] * im;
+        o.z = sl * t.z + dyb[c + 2] * im; o.w = sl * t.w + dyb[c + 3] * im;
+      }
+      *reinterpret_cast<float4*>(dY + e) = o;
+    }
   }
   if constexpr (MP == 0) {                          // m <= 256: 32-bit index arithmetic (a 64-bit division costs far more)
     for (unsigned e = (unsigned)gt; e < (unsigned)mm; e += (unsigned)gn) Wr[e] = W[e] + (e % (unsigned)(m + 1) == 0u ? eps : 0.f);
