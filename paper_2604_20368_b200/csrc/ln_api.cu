@@ -689,15 +689,16 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   // the query-side kernels and are joined before the key side, which needs dM.
   const Side side = side_acquire(std::is_same<T, bf16>::value, st);
   const bool umma_prod = std::is_same<T, bf16>::value && (D == 64 || D == 128);
-  auto launch_mid = [&](cudaStream_t s) {
+  auto launch_mid = [&](cudaStream_t s, int phase = 3) {
     constexpr bool TC = std::is_same<T, bf16>::value;
     auto launch = [&](auto kern, size_t smem, int cl = 1) {
       want_smem(kern, smem);
-      LN_LAUNCH("k_mid_bwd", s, launch_clustered(kern, BH * cl, cl, smem, s, m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, whiten_eff,
+      LN_LAUNCH(phase == 3 ? "k_mid_bwd" : (phase == 1 ? "k_mid_bwd_dM" : "k_mid_bwd_adj"), s,
+                launch_clustered(kern, BH * cl, cl, smem, s, m, pl.T, p->H, p->map_mode, inv_lambda, pl.ldm, whiten_eff,
                                                  x.W, x.Xh, x.Ph, x.hdr, x.M, w.dYtpart, w.dybpart, ch, p->ridge_eps, w.Wr, w.P,
                                                  w.Hm, w.Ga, w.Gb, w.dW, w.dX, w.dY, w.dM, w.GW, dev_status, pl.hslot,
                                                  umma_prod ? reinterpret_cast<bf16*>(w.dMimg) : nullptr, two ? 0 : 1,
-                                                 pl.cg ? 1 : 0, x.Y, w.cg));
+                                                 pl.cg ? 1 : 0, x.Y, w.cg, phase));
     };
     if (pl.cg) { launch(k_mid_bwd<D, false, 0>, sizeof(NsSmem)); return; }
     if (two && m > 64) launch(k_mid_bwd<D, TC, 0, kMidCluster>, sizeof(NsSmem), kMidCluster);
@@ -767,9 +768,13 @@ int bwd_impl(const ln_problem* p, const Plan& pl, const T* Q, const T* K, const 
   if (side.on()) {
     side.fork(st);
     if (tn_on_side) launch_tn_dY(side.s);
-    launch_mid(side.s);
+    // with the sign passes forming their factor themselves, the second one waits for dM only: the per-head kernel runs
+    // as two launches and the adjoint of the iteration, which nothing token-sized needs, follows the mark
+    const bool split_mid = sign3 && !pl.cg;
+    launch_mid(side.s, split_mid ? 1 : 3);
     if (ntg_on_side && !sign3) launch_ntg_R(side.s);
     side.mark();                     // what the second sign pass needs from this stream ends here
+    if (split_mid) launch_mid(side.s, 2);
     launch_nn_dV(side.s);
     launch_sign_W(side.s);
   }

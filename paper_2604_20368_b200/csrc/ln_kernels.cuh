@@ -1690,7 +1690,9 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
                                                  float eps, float* Wr, float* P, float* Hm, float* Ga, float* Gb,
                                                  float* dWm, float* dXm, float* dY, float* dM, float* GW, int* dev_status,
                                                  long long hslot, bf16* dMimg, int sym, int solver = 0, const float* Ysaved = nullptr,
-                                                 float* cgws = nullptr) {
+                                                 float* cgws = nullptr, int phase = 3) {
+  // phase: bit 0 = dY, dX and dM (what the key-side kernels wait for), bit 1 = the adjoint of the iteration and GW.
+  // The two halves may run as two launches on one stream: the key-side sign pass then starts after the first.
   // solver 1 (conjugate gradients, the fp32 single-CTA instantiation only): the solve is differentiated as the linear
   // system it approximates, dM = the T-step iterate of (W + eps I) dM = dY, dW = -dM Y^T (Ysaved: Y of the forward pass)
   // sym: 1 = one landmark set (W = k(L, L): the gradient of both roles of L is carried by the symmetrised factor);
@@ -1709,6 +1711,7 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
   dY += bh * md; dM += bh * md; GW += (long long)bh * m * ldm;
   dYtpart += (long long)bh * nchunks * md; dybpart += (long long)bh * nchunks * D;
   const float* s = whiten ? whiten + (long long)(bh % H) * m : nullptr;
+  if (phase & 1) {
   float* dyb = red;   // [D] column sums of dO
   if (tid < D) {
     float t = 0.f;
@@ -1766,6 +1769,8 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     const int nkb = (m + GU_KB - 1) / GU_KB;
     gu_write_images(dM, dMimg + (long long)bh * nkb * (2 * GU_KB * D), m, D, gt, gn);
   }
+  }
+  if (!(phase & 2)) return;
   if constexpr (MP == 128 || MP == 64) {
     __shared__ UmmaCtl ctl;
     const bool tc_ok = ns_backward_umma<MP>(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, GW, ldm, inv_lambda, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
