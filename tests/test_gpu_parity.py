@@ -645,7 +645,26 @@ def _random_cases(count, seed):
     return cases
 
 
-@pytest.mark.parametrize("case", _random_cases(32, 20260), ids=lambda c: "g{gh}x{gw}_m{mh}x{mw}_p{prefix}_d{d}_T{T}_{dtype}_lm{lm_mode}_map{map_mode}".format(**c))
+def _random_cases_many_landmarks(count, seed):
+    """The same draw restricted to 100 ... 256 landmarks and bf16 storage: the per-head engines above 64 and above 128
+    landmarks at their ragged sizes (odd m, m not a multiple of 4, blocks of the 2 x 2 cut that are almost empty)."""
+    rng = np.random.default_rng(seed)
+    cases = []
+    while len(cases) < count:
+        gh, gw = int(rng.integers(10, 25)), int(rng.integers(10, 25))
+        mh, mw = int(rng.integers(4, min(gh, 16) + 1)), int(rng.integers(4, min(gw, 16) + 1))
+        if not 100 <= mh * mw <= 256:
+            continue
+        even = gh % mh == 0 and gw % mw == 0
+        cases.append(dict(gh=gh, gw=gw, mh=mh, mw=mw, prefix=int(rng.integers(0, 3)), d=int(rng.choice([32, 64, 128])),
+                          T=int(rng.integers(0, 9)), dtype="bf16", lm_mode=int(rng.choice([1, 1, 2, 3])),
+                          map_mode=int(rng.choice([0, 1])), dup=float(rng.choice([0.0, 0.2])) * even, B=int(rng.integers(1, 3)),
+                          H=int(rng.integers(1, 4)), seed=int(rng.integers(1, 1 << 20))))
+    return cases
+
+
+@pytest.mark.parametrize("case", _random_cases(32, 20260) + _random_cases_many_landmarks(16, 31),
+                         ids=lambda c: "g{gh}x{gw}_m{mh}x{mw}_p{prefix}_d{d}_T{T}_{dtype}_lm{lm_mode}_map{map_mode}".format(**c))
 def test_random_shapes_and_modes(case):
     from parity import metrics
     cfg = synth.Config("random", B=case["B"], H=case["H"], d=case["d"], m=case["mh"] * case["mw"], T=case["T"], gh=case["gh"],
