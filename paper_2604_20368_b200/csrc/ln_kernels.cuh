@@ -1711,6 +1711,10 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
   dY += bh * md; dM += bh * md; GW += (long long)bh * m * ldm;
   dYtpart += (long long)bh * nchunks * md; dybpart += (long long)bh * nchunks * D;
   const float* s = whiten ? whiten + (long long)(bh % H) * m : nullptr;
+  // the 256-wide engine keeps one tensor-memory allocation for the products in front of the adjoint and the adjoint
+  __shared__ UmmaCtl ctl256;
+  __shared__ __align__(8) unsigned long long mbars256[3];
+  U2Ctx u2c;
   if (phase & 1) {
   float* dyb = red;   // [D] column sums of dO
   if (tid < D) {
@@ -1760,11 +1764,16 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
       cg_dev<D>(m, T, eps, W, dY, dM, reinterpret_cast<double*>(cgws) + (long long)bh * 4 * md, reinterpret_cast<double*>(dyn_smem), red);
       ns_gemm<TC, false, true>(m, m, D, dM, D, Ysaved + bh * md, D, dWm, ldx, -1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // dW = -dM Y^T
     }
+  } else if constexpr (MP == 256) {                  // dX = dY M^T and dM = X^T dY on the engine of the adjoint
+    u2_begin(u2c, ctl256, mbars256, reinterpret_cast<bf16*>(dyn_smem), 512);
+    const bool p_ok = u2_products_dx_dm(u2c, m, D, dY, Msaved, XT, Hm, Gb, dXm, dM, crank);
+    if (!(phase & 2)) umma_end(ctl256, 512);
+    if (dev_status && !p_ok && tid == 0 && crank == 0) atomicOr(dev_status + bh, 2);
   } else {
     ns_gemm<TC, false, true>(m, m, D, dY, D, Msaved, D, dXm, ldx, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);   // dX = dY M^T
     ns_gemm<TC, true, false>(m, D, m, XT, ldx, dY, D, dM, D, 1.f, 0.f, nullptr, 0.f, sm, crank, CL);        // dM = X^T dY
   }
-  if (CL > 1) phase_sync<CL>();
+  if (CL > 1 && MP != 256) phase_sync<CL>();
   if (dMimg != nullptr) {                         // dM also as split operand images (for the tcgen05 product dV = R^T dM)
     const int nkb = (m + GU_KB - 1) / GU_KB;
     gu_write_images(dM, dMimg + (long long)bh * nkb * (2 * GU_KB * D), m, D, gt, gn);
@@ -1776,9 +1785,9 @@ __global__ void __launch_bounds__(256, MP == 64 ? 3 : ((CL > 1 && MP == 0) ? 2 :
     const bool tc_ok = ns_backward_umma<MP>(m, T, eps, W, Xh, Ph, ldx, mx, hdr, dXm, GW, ldm, inv_lambda, reinterpret_cast<bf16*>(dyn_smem), red, ctl);
     if (dev_status && !tc_ok && tid == 0) atomicOr(dev_status + bh, 2);
   } else if constexpr (MP == 256) {
-    __shared__ UmmaCtl ctl;
-    __shared__ __align__(8) unsigned long long mbars[3];
-    const bool tc_ok = ns_backward_umma256(m, T, Xh, Ph, dXm, Ga, Gb, Hm, Wr, P, dWm, reinterpret_cast<bf16*>(dyn_smem), ctl, mbars, crank);
+    if (!(phase & 1)) u2_begin(u2c, ctl256, mbars256, reinterpret_cast<bf16*>(dyn_smem), 512);
+    const bool tc_ok = ns_backward_umma256(u2c, m, T, Xh, Ph, dXm, Ga, Gb, Hm, Wr, P, dWm, crank);
+    umma_end(ctl256, 512);
     if (dev_status && !tc_ok && tid == 0 && crank == 0) atomicOr(dev_status + bh, 2);
     // end of the adjoint and GW in one pass (the operand buffers are free: the engine has ended with a cluster barrier)
     ns_tail_gw_sym<CL>(m, ldm, W, eps, hdr, P, dWm, inv_lambda, GW, red, reinterpret_cast<float*>(dyn_smem), crank);

@@ -323,16 +323,14 @@ __device__ bool u2_product_y(U2Ctx& c, int m, int D, const float* XTimg, const f
 // the steps in Gpriv, which only the thread that owns an element reads and writes: laid out [ri][ci][16][256 threads][4]
 // so that a warp's accesses are contiguous (a thread's 64 values of a row, read from an [m][m] matrix, would touch 32
 // rows per instruction).  Outputs, fp32 [m][m]: Gout = dLoss/dX_0 and dW = -(sum over the steps of H A^T).  Returns
-// false if a wait ran out.
-__device__ bool ns_backward_umma256(int m, int T, const float* Xh, const float* Ph, const float* G0, float* Gimg0,
-                                    float* Gimg1, float* Himg, float* Gpriv, float* Gout, float* dW, bf16* smem, UmmaCtl& ctl,
-                                    unsigned long long* mbars, int ri) {
+// false if a wait ran out.  Called between u2_begin (512 columns of tensor memory) and umma_end.
+__device__ bool ns_backward_umma256(U2Ctx& c, int m, int T, const float* Xh, const float* Ph, const float* G0, float* Gimg0,
+                                    float* Gimg1, float* Himg, float* Gpriv, float* Gout, float* dW, int ri) {
+  UmmaCtl& ctl = *c.ctl;
   const int tid = threadIdx.x, warp = tid >> 5;
   const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64;
   const int gi = ri * 128 + row;
   const bool vec = (m & 3) == 0;
-  U2Ctx c;
-  u2_begin(c, ctl, mbars, smem, 512);
   const uint32_t t_acc[2] = {ctl.tmem_base, ctl.tmem_base + 128}, t_dw[2] = {ctl.tmem_base + 256, ctl.tmem_base + 384};
   // this thread's 64 elements of a block row of an fp32 [m][m] matrix (zero outside)
   auto load_row = [&](const float* src, int gj0, float (&v)[64]) {
@@ -432,7 +430,84 @@ __device__ bool ns_backward_umma256(int m, int T, const float* Xh, const float* 
     store_row(dW, gj0, v);
   }
   const bool ok = c.ok && ctl.timeout == 0;
-  umma_end(ctl, 512);
+  phase_sync<kU2Cluster>();
+  return ok;
+}
+
+// dX = dY M^T and dM = X_T^T dY in front of the adjoint, on the same engine (between u2_begin with 512 columns and
+// umma_end).  dY, M: fp32 [m][D] (D <= 128, padded with zero columns); XT: fp32 [m][m].  Each CTA turns its block rows
+// of dY and M and its two blocks of X_T into images (scratch slots S1: dY blocks 0, 1 and M blocks 2, 3; S2: X_T);
+// after a cluster barrier  dX[ri][ci] = dY[ri] M[ci]^T  is one group into two accumulators and
+// dM[ri] = sum_kb X_T[kb][ri]^T dY[kb]  two one-sided groups into a third.  Results leave as fp32 rows.  Both CTAs must
+// have passed a cluster barrier since dY was written; ends with one.
+__device__ bool u2_products_dx_dm(U2Ctx& c, int m, int D, const float* dY, const float* M, const float* XT, float* S1, float* S2,
+                                  float* dX, float* dM, int ri) {
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int row = (warp & 3) * 32 + (tid & 31), col0 = (warp >> 2) * 64, gi = ri * 128 + row;
+  const uint32_t tb = c.ctl->tmem_base;
+  const bool vec = (m & 3) == 0;
+  float v[64];
+#pragma unroll 1
+  for (int pass = 0; pass < 4; ++pass) {
+    if (pass < 2) {                                              // a block row of dY or of M, D columns of it
+      const float* src = pass == 0 ? dY : M;
+#pragma unroll
+      for (int q = 0; q < 64; q += 4) {
+        float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (gi < m && col0 + q < D) t = *reinterpret_cast<const float4*>(src + (long long)gi * D + col0 + q);   // D is a multiple of 4
+        v[q] = t.x; v[q + 1] = t.y; v[q + 2] = t.z; v[q + 3] = t.w;
+      }
+    } else {                                                     // block (ri, pass - 2) of X_T
+      const int gj0 = (pass - 2) * 128 + col0;
+#pragma unroll
+      for (int q = 0; q < 64; q += 4) {
+        if (gi < m && gj0 + q + 3 < m && vec) {
+          const float4 t = *reinterpret_cast<const float4*>(XT + (long long)gi * m + gj0 + q);
+          v[q] = t.x; v[q + 1] = t.y; v[q + 2] = t.z; v[q + 3] = t.w;
+        } else {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) v[q + u] = (gi < m && gj0 + q + u < m) ? XT[(long long)gi * m + gj0 + q + u] : 0.f;
+        }
+      }
+    }
+    float* dst = pass == 0 ? u2_block_w(S1, 0, ri) : (pass == 1 ? u2_block_w(S1, 1, ri) : u2_block_w(S2, ri, pass - 2));
+    if (pass < 3) {
+      u2_store_block(c, v, row, col0, dst, pass, false);
+    } else {
+      if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // buffer 0 is on its way out
+      __syncthreads();
+      u2_store_block(c, v, row, col0, dst, 0, true);
+    }
+  }
+  phase_sync<kU2Cluster>();
+  const U2Group g[3] = {{u2_block(S1, 0, ri), true, u2_block(S1, 1, 0), u2_block(S1, 1, 1), true, tb, tb + 128, false},
+                        {u2_block(S2, 0, ri), false, u2_block(S1, 0, 0), nullptr, false, tb + 256, tb + 256, false},
+                        {u2_block(S2, 1, ri), false, u2_block(S1, 0, 1), nullptr, false, tb + 256, tb + 256, true}};
+  u2_run<3>(c, g);
+#pragma unroll 1
+  for (int ci = 0; ci < 2; ++ci) {
+    const int gj0 = ci * 128 + col0;
+    umma_row<64>(tb + 128 * ci, col0, v);
+    if (gi < m) {
+#pragma unroll
+      for (int q = 0; q < 64; q += 4) {
+        if (gj0 + q + 3 < m && vec) *reinterpret_cast<float4*>(dX + (long long)gi * m + gj0 + q) = make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+        else {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) if (gj0 + q + u < m) dX[(long long)gi * m + gj0 + q + u] = v[q + u];
+        }
+      }
+    }
+  }
+  umma_row<64>(tb + 256, col0, v);
+  if (gi < m) {
+#pragma unroll
+    for (int q = 0; q < 64; q += 4)
+      if (col0 + q < D) *reinterpret_cast<float4*>(dM + (long long)gi * D + col0 + q) = make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+  }
+  umma::fence_before_sync();
+  __syncthreads();
+  const bool ok = c.ok && c.ctl->timeout == 0;
   phase_sync<kU2Cluster>();
   return ok;
 }
