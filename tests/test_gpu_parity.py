@@ -663,7 +663,21 @@ def _random_cases_many_landmarks(count, seed):
     return cases
 
 
-@pytest.mark.parametrize("case", _random_cases(32, 20260) + _random_cases_many_landmarks(16, 31),
+def _cases_two_block_rows():
+    """129 ... 256 landmarks at every head width: the 2 x 2 block cut of the per-head kernels with a second block row of
+    one, a few, and all 128 landmarks; odd counts and counts that are no multiple of 4 (the backward products
+    dX = dY M^T and dM = X_T^T dY read M, dY and X_T in 128-bit pieces where the row length allows)."""
+    cases = []
+    for (mh, mw, gh, gw), d, T, lm_mode, map_mode in (((3, 43, 6, 43), 64, 3, 1, 1), ((10, 13, 20, 13), 64, 5, 2, 0),
+                                                       ((11, 13, 11, 26), 128, 4, 1, 1), ((11, 17, 22, 17), 64, 6, 1, 0),
+                                                       ((15, 17, 15, 17), 128, 3, 2, 1), ((16, 16, 16, 32), 64, 8, 1, 1),
+                                                       ((13, 17, 13, 34), 32, 7, 3, 0), ((7, 19, 14, 19), 128, 0, 1, 1)):
+        cases.append(dict(gh=gh, gw=gw, mh=mh, mw=mw, prefix=len(cases) % 3, d=d, T=T, dtype="bf16", lm_mode=lm_mode,
+                          map_mode=map_mode, dup=0.0, B=1 + len(cases) % 2, H=1 + len(cases) % 3, seed=4100 + len(cases)))
+    return cases
+
+
+@pytest.mark.parametrize("case", _random_cases(32, 20260) + _random_cases_many_landmarks(16, 31) + _cases_two_block_rows(),
                          ids=lambda c: "g{gh}x{gw}_m{mh}x{mw}_p{prefix}_d{d}_T{T}_{dtype}_lm{lm_mode}_map{map_mode}".format(**c))
 def test_random_shapes_and_modes(case):
     from parity import metrics
