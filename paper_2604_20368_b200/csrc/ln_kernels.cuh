@@ -435,25 +435,83 @@ __global__ void __launch_bounds__(256) k_pool_wide(const T* __restrict__ K, floa
 
 // dK[j] = dKpart[j] (may be NULL) + sum over the bins containing token j of dL[bin] / |bin|
 // (pooling adjoint); with pool == 0 it only converts dKpart to the storage type.
-constexpr int POOL_EPT = 4;      // elements (of four dims) per thread of k_pool_bwd
+constexpr int POOL_EPT = 8;      // elements (of four dims) per thread of k_pool_bwd
 template <typename T>
-__global__ void __launch_bounds__(256) k_pool_bwd(const float* __restrict__ dKpart, const float* __restrict__ dL, T* __restrict__ dK,
+__global__ void __launch_bounds__(256, 4) k_pool_bwd(const float* __restrict__ dKpart, const float* __restrict__ dL, T* __restrict__ dK,
                                                   PoolGeom g, int pool) {
   // bin boundaries once per CTA (a division each) instead of several per thread
   __shared__ int rlo[256], rhi[256], clo[256], chi[256];
-  if (pool) {
-    for (int a = threadIdx.x; a < g.mh; a += 256) { rlo[a] = bin_lo(a, g.gh, g.mh); rhi[a] = bin_hi(a, g.gh, g.mh); }
-    for (int b = threadIdx.x; b < g.mw; b += 256) { clo[b] = bin_lo(b, g.gw, g.mw); chi[b] = bin_hi(b, g.gw, g.mw); }
-    __syncthreads();
-  }
+  __shared__ int s_lm[POOL_EPT * 256 / 8], s_tap[POOL_EPT * 256 / 8];   // per token of this CTA: its landmark and its tap (even bins)
   const int bh = blockIdx.y;
   const unsigned per_row = g.d / 4;
   const unsigned total = (unsigned)g.n * per_row;                  // n * d / 4 < 2^32
   const bool even = (g.gh % g.mh) == 0 && (g.gw % g.mw) == 0;      // the pooling of Sec. 4.2 proper: r x r windows, stride r
   const int bh_rows = g.gh / g.mh, bh_cols = g.gw / g.mw;
   const float even_inv = 1.f / (float)(bh_rows * bh_cols);
-  // POOL_EPT elements of four dims per thread, a CTA's share contiguous, so that the bin tables are built once
-  // per 1024 elements
+  // POOL_EPT elements of four dims per thread, a CTA's share contiguous, so that the tables are built once per 2048
+  // elements.  With a head width of 32, 64 or 128 the share is 256, 128 or 64 whole tokens: their landmark (and tap) is
+  // worked out once per token and CTA, and an element finds its token by a shift, not by five integer divisions.
+  const bool table = pool && even && (per_row == 8u || per_row == 16u || per_row == 32u);
+  const int sh = 31 - __clz((int)per_row);
+  const unsigned base = blockIdx.x * (unsigned)(POOL_EPT * 256);
+  const int j0 = (int)(base >> sh);
+  // this CTA's share of the partial gradient is contiguous: one bulk copy (cp.async.bulk, up to 32 KB) stages it in
+  // shared memory, so that the bytes in flight from HBM do not depend on the registers of the threads
+  __shared__ __align__(128) float4 stage[POOL_EPT * 256];
+  __shared__ __align__(8) unsigned long long bar;
+  if (table && dKpart && threadIdx.x == 0) {
+    const unsigned cnt = min(total - base, (unsigned)(POOL_EPT * 256));
+    umma::mbar_init(&bar, 1);
+    umma::mbar_expect_tx(&bar, cnt * 16u);
+    umma::bulk_load(stage, dKpart + (long long)bh * g.n * g.d + (long long)base * 4, cnt * 16u, &bar);
+  }
+  if (pool) {
+    if (!table) {
+      for (int a = threadIdx.x; a < g.mh; a += 256) { rlo[a] = bin_lo(a, g.gh, g.mh); rhi[a] = bin_hi(a, g.gh, g.mh); }
+      for (int b = threadIdx.x; b < g.mw; b += 256) { clo[b] = bin_lo(b, g.gw, g.mw); chi[b] = bin_hi(b, g.gw, g.mw); }
+    } else {
+      for (int t = threadIdx.x; t < ((POOL_EPT * 256) >> sh); t += 256) {
+        const int j = j0 + t;
+        int lm = -1, tap = 0;
+        if (j < g.n && j >= g.prefix) {
+          const int r = (j - g.prefix) / g.gw, q = (j - g.prefix) % g.gw;
+          lm = (r / bh_rows) * g.mw + q / bh_cols;
+          tap = (r % bh_rows) * bh_cols + q % bh_cols;
+        }
+        s_lm[t] = lm; s_tap[t] = tap;
+      }
+    }
+    __syncthreads();
+  }
+  if (table) {
+    // the landmark rows (L2) are loaded while the bulk copy of the partial gradient (HBM) is on its way
+    float4 t[POOL_EPT];
+    int lm[POOL_EPT];
+#pragma unroll
+    for (int u = 0; u < POOL_EPT; ++u) {
+      const unsigned idx = base + (unsigned)u * 256u + threadIdx.x;
+      lm[u] = idx < total ? s_lm[(int)(idx >> sh) - j0] : -2;    // -2: past the end; -1: a prefix token
+      t[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (lm[u] >= 0) t[u] = ld4(dL + ((long long)bh * g.m + lm[u]) * g.d + (int)(idx & (per_row - 1u)) * 4);
+    }
+    // a wait that ran out (it cannot, short of a fault elsewhere) falls back to plain loads of the same values
+    const bool staged = dKpart != nullptr && umma::mbar_wait(&bar, 0);
+#pragma unroll
+    for (int u = 0; u < POOL_EPT; ++u) {
+      if (lm[u] == -2) continue;
+      const unsigned idx = base + (unsigned)u * 256u + threadIdx.x;
+      float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (staged) o = stage[u * 256 + threadIdx.x];
+      else if (dKpart) o = ld4(dKpart + (long long)bh * g.n * g.d + (long long)idx * 4);
+      if (lm[u] >= 0) {
+        float4 w = make_float4(even_inv, even_inv, even_inv, even_inv);
+        if (g.filt) w = ld4(g.filt + ((long long)(bh % g.H) * (bh_rows * bh_cols) + s_tap[(int)(idx >> sh) - j0]) * g.d + (int)(idx & (per_row - 1u)) * 4);
+        o.x += t[u].x * w.x; o.y += t[u].y * w.y; o.z += t[u].z * w.z; o.w += t[u].w * w.w;
+      }
+      st4(dK + (long long)bh * g.n * g.d + (long long)idx * 4, o);
+    }
+    return;
+  }
 #pragma unroll
   for (int u = 0; u < POOL_EPT; ++u) {
     const unsigned idx = (blockIdx.x * POOL_EPT + u) * blockDim.x + threadIdx.x;
